@@ -1,0 +1,119 @@
+/*
+ * hyenand.h -- C ABI of the B200 (sm_100a) gated N-D long convolution.
+ *
+ * The library computes, for every batch entry b, channel c and grid position i
+ * of a 1-D, 2-D or 3-D grid L_1 x ... x L_N,
+ *
+ *     y[b,c,i] = q[b,c,i] * sum_j h[b,c, i - j] * k[b,c,j] * v[b,c,j]
+ *
+ * i.e. the gated Hyena mixer (Definition A.3; Eq. 1-2 without the pointwise
+ * activations and norms, which the caller applies to q, k, v beforehand): k*v is
+ * the inner gate, h the depthwise long-convolution kernel whose weight depends
+ * on the displacement i - j only (Definition A.2, Theorem A.5), q the outer
+ * gate.  The sum is evaluated through FFTs on the zero-padded grid (Section
+ * 3.2.1 "non-circular convolutions", Appendix B.1 Eq. 11-13): pad each axis to
+ * P_n >= 2 L_n - 1 (a power of two), transform k*v and h, multiply the
+ * spectra, transform back, crop, apply q.  All arithmetic is fp32; bf16 is an
+ * I/O format only (one round-to-nearest-even at the final store).
+ *
+ * Layout (all buffers dense, row-major, last axis contiguous):
+ *     q, k, v, y : [B][C][L_1]...[L_N]
+ *     h          : [B][C][K_1]...[K_N]
+ *       non-causal: K_n = 2 L_n - 1, tap index m_n = (i_n - j_n) + (L_n - 1)
+ *       causal (N = 1 only, Appendix A.3 masking strategy): K_1 = L_1, tap
+ *       index m = i - j >= 0, negative displacements have weight zero.
+ *     One dtype for all five buffers.
+ *
+ * Ownership: the caller owns q, k, v, h, y.  A plan owns its device workspace
+ * and twiddle tables.  hyenand_forward* never allocates device memory, never
+ * synchronises and only enqueues work on the given stream (hyenand_forward_host
+ * is the exception, see below).  One forward may be in flight per plan; use one
+ * plan per concurrent stream.  Plans belong to the device that was current
+ * when they were created.
+ *
+ * Errors: functions returning int return HYENAND_OK or an error code and
+ * record a message for hyenand_last_error() (thread-local).  On error nothing
+ * is launched.  NaN/Inf in an input spreads to its whole (b,c) slice; that is
+ * not an error.
+ */
+#ifndef HYENAND_H
+#define HYENAND_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hyenand_plan hyenand_plan;   /* opaque, library-owned */
+
+enum { HYENAND_F32 = 0, HYENAND_BF16 = 1 };
+
+enum {
+    HYENAND_OK = 0,
+    HYENAND_ERR_INVALID_ARG = 1,   /* bad count, null or misaligned pointer, aliasing */
+    HYENAND_ERR_UNSUPPORTED = 2,   /* causal with ndim > 1, axis too long */
+    HYENAND_ERR_ALLOC = 3,         /* workspace could not be allocated */
+    HYENAND_ERR_CUDA = 4           /* a CUDA call or launch failed */
+};
+
+/*
+ * Create a plan for grids dims[0..ndim-1] (host array), batch B, C channels.
+ * ndim in {1,2,3}; every L_n >= 1; causal in {0,1} (1 requires ndim == 1);
+ * dtype HYENAND_F32 or HYENAND_BF16.  Allocates the workspace and twiddle
+ * tables on the current device (this call may synchronise).  Returns NULL on
+ * failure, reason in hyenand_last_error().
+ * Limits: for ndim >= 2 each padded axis P_n <= 8192; for ndim == 1,
+ * P_1 <= 2^26.
+ */
+hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype);
+
+/*
+ * One forward pass, one kernel per (b,c) as in Section 3.2.2 ("B different
+ * convolutional kernels, one for each of the inputs in a batch").
+ * q, k, v, h, y: DEVICE pointers, 16-byte aligned, y must not alias an input.
+ * cuda_stream: a cudaStream_t (NULL = the legacy default stream).
+ */
+int hyenand_forward(hyenand_plan *plan, const void *q, const void *k, const void *v,
+                    const void *h, void *y, void *cuda_stream);
+
+/*
+ * Same with an explicit batch stride for h, in elements: 0 means h is
+ * [C][K_1]..[K_N], one kernel per channel shared by the whole batch (the
+ * static kernel of Section 3.2.1); C*K_1*..*K_N is the dense per-sample layout.
+ * Other values are rejected.
+ */
+int hyenand_forward_ex(hyenand_plan *plan, const void *q, const void *k, const void *v,
+                       const void *h, long long h_batch_stride_elems, void *y, void *cuda_stream);
+
+/*
+ * End-to-end variant: q, k, v, h, y are HOST pointers (pinned memory gives the
+ * fastest copies but any host memory works).  Copies the inputs to device
+ * staging buffers owned by the plan (allocated on the first call, which
+ * therefore may synchronise), runs the same kernels as hyenand_forward_ex and
+ * copies y back, all on cuda_stream; returns after y has arrived on the host
+ * (the call synchronises the stream).
+ */
+int hyenand_forward_host(hyenand_plan *plan, const void *q, const void *k, const void *v,
+                         const void *h, long long h_batch_stride_elems, void *y, void *cuda_stream);
+
+/* Frees the workspace (synchronises the device).  NULL is accepted. */
+void hyenand_destroy_plan(hyenand_plan *plan);
+
+/* Message of the last error on this thread ("" if none).  Never NULL. */
+const char *hyenand_last_error(void);
+
+/* Code of the last error on this thread (HYENAND_OK if the last call succeeded);
+ * tells why hyenand_create_plan returned NULL. */
+int hyenand_last_error_code(void);
+
+/* Reporting helpers (host-only, no device work). */
+size_t hyenand_plan_workspace_bytes(const hyenand_plan *plan);        /* device bytes owned by the plan */
+int hyenand_plan_fft_dims(const hyenand_plan *plan, int *out_P);      /* writes ndim padded sizes P_n */
+int hyenand_plan_launches(const hyenand_plan *plan, int h_shared);    /* kernels enqueued by one forward */
+const char *hyenand_plan_path(const hyenand_plan *plan);              /* name of the kernel path chosen */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYENAND_H */

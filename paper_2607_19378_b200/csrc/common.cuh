@@ -1,0 +1,90 @@
+// Shared declarations of the library's translation units (internal).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace hn {
+
+typedef __nv_bfloat16 bf16;
+
+template <typename T> struct IO;
+template <> struct IO<float> {
+    static __device__ __forceinline__ float ld(const float *p, long long i) { return __ldg(p + i); }
+    static __device__ __forceinline__ void st(float *p, long long i, float v) { p[i] = v; }
+};
+template <> struct IO<bf16> {
+    static __device__ __forceinline__ float ld(const bf16 *p, long long i)
+    {
+        return __bfloat162float(__ldg(p + i));
+    }
+    static __device__ __forceinline__ void st(bf16 *p, long long i, float v) { p[i] = __float2bfloat16_rn(v); }
+};
+
+constexpr int kMaxLineLog2 = 13;          // longest line transformed in shared memory: 8192 points
+constexpr int kThreads = 256;             // threads per CTA of the generic kernels
+
+// ---- generic N-D path (nd_kernels.cu) ---------------------------------------------
+//
+// Workspace arrays hold half spectra along the contiguous axis: XH = P3/2 + 1
+// complex bins per row.  "Rows" are lines along the contiguous axis; all other
+// axes are transformed by the axis kernels on tiles of adjacent bins.
+
+struct RowsArgs {
+    const void *a;        // k (or h)
+    const void *b;        // v (or nullptr: plain copy of a)
+    float2 *out;          // [rows][XH]
+    long long rows;       // number of rows
+    int len;              // valid elements per row (L3, or K3 for the filter)
+    int shift;            // element m of a row goes to padded position (m - shift) mod P
+    int log2p;            // log2 of the padded row length P
+    int prune_in;         // 1: all valid positions are < P/2 (u, causal h)
+    const float2 *gtw;    // global twiddle table, gtw_n points
+    int gtw_n;
+};
+
+struct RowsInvArgs {
+    const float2 *in;     // [rows][XH]
+    const void *q;        // [rows][len]
+    void *y;              // [rows][len]
+    long long rows;
+    int len;              // L3
+    int log2p;
+    const float2 *gtw;
+    int gtw_n;
+};
+
+// A family of strided lines: line (o, c), element a at base[o*outer + a*nc + c].
+struct AxisArgs {
+    // u lines (in) -> out lines; for the core, in place (out == in, n_out == n_in)
+    const float2 *in;
+    float2 *out;
+    long long n_outer;        // number of outer indices
+    long long in_outer;       // element stride between outer indices (input)
+    long long out_outer;      // element stride between outer indices (output)
+    int nc;                   // contiguous lines per outer index (= element stride along the axis)
+    int n_in;                 // valid input entries along the axis
+    int n_out;                // entries written along the axis
+    int shift;                // input entry m goes to position (m - shift) mod P
+    int log2p;
+    int prune_in;
+    // core only: filter lines, outer index oh = h_shared ? o % h_mod : o
+    const float2 *h;
+    long long h_outer;
+    int h_n_in;
+    int h_shift;
+    int h_prune_in;
+    long long h_mod;          // 0: oh = o, else oh = (o + h_off) % h_mod
+    long long h_off;
+    float scale;              // applied to the product (1/P_total)
+    const float2 *gtw;
+    int gtw_n;
+};
+
+enum AxisMode { AXIS_FWD = 0, AXIS_INV = 1, AXIS_CORE = 2 };
+
+int launch_rows_fwd(const RowsArgs &a, int dtype, cudaStream_t st);
+int launch_rows_inv(const RowsInvArgs &a, int dtype, cudaStream_t st);
+int launch_axis(const AxisArgs &a, int mode, cudaStream_t st);
+
+}  // namespace hn

@@ -1,0 +1,27 @@
+// Long 1-D path (padded length above the shared-memory line limit): the
+// transform is split Cooley-Tukey style into two passes over a 2-D view of the
+// sequence (Appendix B.3 of the paper describes the same decomposition).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+namespace hn {
+
+struct Ct1dPlan {
+    int L, K, log2p, B, C, causal, dtype;
+    int log2p1, log2p2;       // P = P1 * P2, n = n1*P2 + n2, k = k1 + P1*k2
+    float2 *wu;               // [slices_per_chunk][P1/2+1][P2]
+    float2 *wh;               // [C or slices_per_chunk][P1/2+1][P2]
+    float2 *tw1, *tw2;        // twiddle tables for P1 and P2
+    float2 *twp_coarse, *twp_fine;   // W_P^j = coarse[j >> lo] * fine[j & (2^lo - 1)]
+    int lo;
+    long long slices_per_chunk, wh_slices;
+};
+
+int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, int dtype, size_t *bytes);
+void ct1d_free(Ct1dPlan *c);
+int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const void *h, bool shared,
+                 void *y, cudaStream_t st, int *launches);
+int ct1d_launches(const Ct1dPlan *c, bool shared);
+
+}  // namespace hn

@@ -1,0 +1,248 @@
+// Shared-memory complex FFT engine (fp32) for power-of-two line lengths.
+//
+// A "line" is N complex points in shared memory.  Transforms are Stockham
+// autosort passes of radix 4/8/16 (radix 2 only for N = 2): every pass reads
+// R points at stride N/R, applies the pass twiddles, runs an R-point DFT in
+// registers and writes R points back, so data leaves registers once per pass.
+// Lines are stored with one pad element every 16 (phys()) so that both the
+// contiguous reads and the strided writes of a pass are bank-conflict free.
+//
+// Pruning: the padded convolution (Section 3.2.1; Appendix B.1, Eq. 11-13 of
+// the paper) transforms inputs whose upper half is zero and keeps only the
+// lower half of every inverse.  PRUNE_IN drops the arithmetic on the zero half
+// in the first pass, PRUNE_OUT skips the unused outputs of the last pass.
+#pragma once
+#include <cuda_runtime.h>
+
+namespace hn {
+
+enum { PRUNE_NONE = 0, PRUNE_IN = 1, PRUNE_OUT = 2 };
+
+__host__ __device__ __forceinline__ constexpr int phys(int i) { return i + (i >> 4); }
+// shared-memory floats2 needed for one line of n points (odd, so lines do not alias banks)
+__host__ __device__ __forceinline__ constexpr int line_stride(int n) { return (phys(n) + 1) | 1; }
+
+__device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
+__device__ __forceinline__ float2 cmul(float2 a, float2 w)
+{
+    return make_float2(fmaf(a.x, w.x, -a.y * w.y), fmaf(a.x, w.y, a.y * w.x));
+}
+__device__ __forceinline__ float2 cmulc(float2 a, float2 w)   // a * conj(w)
+{
+    return make_float2(fmaf(a.x, w.x, a.y * w.y), fmaf(a.y, w.x, -a.x * w.y));
+}
+// multiply by -i (forward transforms) or +i (inverse)
+template <bool INV> __device__ __forceinline__ float2 rot90(float2 a)
+{
+    return INV ? make_float2(-a.y, a.x) : make_float2(a.y, -a.x);
+}
+
+#define HN_SQ2 0.70710678118654752440f
+#define HN_C8  0.92387953251128675613f   // cos(pi/8)
+#define HN_S8  0.38268343236508977173f   // sin(pi/8)
+
+// a * W_16^T (forward sign; conjugate for INV), T compile-time
+template <int T, bool INV> __device__ __forceinline__ float2 mul_w16(float2 a)
+{
+    constexpr int t = T & 15;
+    if constexpr (t == 0) return a;
+    else if constexpr (t == 4) return rot90<INV>(a);
+    else if constexpr (t == 8) return make_float2(-a.x, -a.y);
+    else if constexpr (t == 12) return rot90<!INV>(a);
+    else if constexpr (t == 2) {
+        return INV ? make_float2((a.x - a.y) * HN_SQ2, (a.x + a.y) * HN_SQ2)
+                   : make_float2((a.x + a.y) * HN_SQ2, (a.y - a.x) * HN_SQ2);
+    } else if constexpr (t == 6) {
+        return INV ? make_float2(-(a.x + a.y) * HN_SQ2, (a.x - a.y) * HN_SQ2)
+                   : make_float2((a.y - a.x) * HN_SQ2, -(a.x + a.y) * HN_SQ2);
+    } else if constexpr (t == 10) {
+        float2 m = mul_w16<2, INV>(a); return make_float2(-m.x, -m.y);
+    } else if constexpr (t == 14) {
+        float2 m = mul_w16<6, INV>(a); return make_float2(-m.x, -m.y);
+    } else {
+        // odd powers: cos/sin of t*pi/8
+        constexpr float c = (t == 1 || t == 15) ? HN_C8 : (t == 3 || t == 13) ? HN_S8
+                          : (t == 5 || t == 11) ? -HN_S8 : -HN_C8;
+        constexpr float s0 = (t == 1 || t == 7) ? HN_S8 : (t == 3 || t == 5) ? HN_C8
+                           : (t == 9 || t == 15) ? -HN_S8 : -HN_C8;     // sin(t*pi/8)
+        constexpr float s = INV ? s0 : -s0;                              // forward: e^{-i..}
+        return make_float2(fmaf(a.x, c, -a.y * s), fmaf(a.x, s, a.y * c));
+    }
+}
+
+// ---- register DFTs, natural order in and out ------------------------------------
+
+template <bool INV, int PR> __device__ __forceinline__ void dft2(float2 &a, float2 &b)
+{
+    if constexpr (PR == PRUNE_IN) { b = a; }
+    else if constexpr (PR == PRUNE_OUT) { a = cadd(a, b); }
+    else { float2 t = a; a = cadd(t, b); b = csub(t, b); }
+}
+
+template <bool INV, int PR>
+__device__ __forceinline__ void dft4(float2 &a0, float2 &a1, float2 &a2, float2 &a3)
+{
+    if constexpr (PR == PRUNE_IN) {            // a2 = a3 = 0
+        float2 r = rot90<INV>(a1);
+        float2 x0 = cadd(a0, a1), x2 = csub(a0, a1);
+        float2 x1 = cadd(a0, r), x3 = csub(a0, r);
+        a0 = x0; a1 = x1; a2 = x2; a3 = x3;
+    } else {
+        float2 t0 = cadd(a0, a2), t1 = csub(a0, a2);
+        float2 t2 = cadd(a1, a3), t3 = rot90<INV>(csub(a1, a3));
+        a0 = cadd(t0, t2);
+        a1 = cadd(t1, t3);
+        if constexpr (PR != PRUNE_OUT) { a2 = csub(t0, t2); a3 = csub(t1, t3); }
+    }
+}
+
+template <bool INV, int PR> __device__ __forceinline__ void dft8(float2 (&x)[8])
+{
+    // evens / odds as two 4-point transforms (inputs 4..7 are zero under PRUNE_IN)
+    constexpr int P4 = (PR == PRUNE_IN) ? PRUNE_IN : PRUNE_NONE;
+    float2 e0 = x[0], e1 = x[2], e2 = x[4], e3 = x[6];
+    float2 o0 = x[1], o1 = x[3], o2 = x[5], o3 = x[7];
+    dft4<INV, P4>(e0, e1, e2, e3);
+    dft4<INV, P4>(o0, o1, o2, o3);
+    o1 = mul_w16<2, INV>(o1);
+    o2 = mul_w16<4, INV>(o2);
+    o3 = mul_w16<6, INV>(o3);
+    x[0] = cadd(e0, o0); x[1] = cadd(e1, o1); x[2] = cadd(e2, o2); x[3] = cadd(e3, o3);
+    if constexpr (PR != PRUNE_OUT) {
+        x[4] = csub(e0, o0); x[5] = csub(e1, o1); x[6] = csub(e2, o2); x[7] = csub(e3, o3);
+    }
+}
+
+template <bool INV, int PR> __device__ __forceinline__ void dft16(float2 (&x)[16])
+{
+    // n = 4*n1 + n2, k = k1 + 4*k2: 4-point transforms over n1, twiddle W16^(n2*k1),
+    // 4-point transforms over n2.
+    constexpr int PIN = (PR == PRUNE_IN) ? PRUNE_IN : PRUNE_NONE;
+    constexpr int POUT = (PR == PRUNE_OUT) ? PRUNE_OUT : PRUNE_NONE;
+    float2 a[4][4];                                  // a[n2][k1]
+#pragma unroll
+    for (int n2 = 0; n2 < 4; ++n2) {
+        a[n2][0] = x[n2]; a[n2][1] = x[n2 + 4]; a[n2][2] = x[n2 + 8]; a[n2][3] = x[n2 + 12];
+        dft4<INV, PIN>(a[n2][0], a[n2][1], a[n2][2], a[n2][3]);
+    }
+    a[1][1] = mul_w16<1, INV>(a[1][1]); a[1][2] = mul_w16<2, INV>(a[1][2]); a[1][3] = mul_w16<3, INV>(a[1][3]);
+    a[2][1] = mul_w16<2, INV>(a[2][1]); a[2][2] = mul_w16<4, INV>(a[2][2]); a[2][3] = mul_w16<6, INV>(a[2][3]);
+    a[3][1] = mul_w16<3, INV>(a[3][1]); a[3][2] = mul_w16<6, INV>(a[3][2]); a[3][3] = mul_w16<9, INV>(a[3][3]);
+#pragma unroll
+    for (int k1 = 0; k1 < 4; ++k1) {
+        dft4<INV, POUT>(a[0][k1], a[1][k1], a[2][k1], a[3][k1]);
+        x[k1] = a[0][k1]; x[k1 + 4] = a[1][k1];
+        if constexpr (PR != PRUNE_OUT) { x[k1 + 8] = a[2][k1]; x[k1 + 12] = a[3][k1]; }
+    }
+}
+
+template <int R, bool INV, int PR> __device__ __forceinline__ void dft(float2 (&x)[R])
+{
+    if constexpr (R == 2) dft2<INV, PR>(x[0], x[1]);
+    else if constexpr (R == 4) dft4<INV, PR>(x[0], x[1], x[2], x[3]);
+    else if constexpr (R == 8) dft8<INV, PR>(x);
+    else dft16<INV, PR>(x);
+}
+
+// ---- pass plan: log2(N) split as evenly as possible into passes of <= 4 bits ------
+
+__host__ __device__ constexpr int n_passes(int log2n) { return (log2n + 3) / 4; }
+__host__ __device__ constexpr int pass_bits(int log2n, int s)
+{
+    const int np = n_passes(log2n);
+    return np == 0 ? 0 : log2n / np + (s < log2n % np ? 1 : 0);
+}
+__host__ __device__ constexpr int bits_before(int log2n, int s)
+{
+    int b = 0;
+    for (int i = 0; i < s; ++i) b += pass_bits(log2n, i);
+    return b;
+}
+
+// Twiddle table in shared memory: tw[t] = exp(-2 pi i t / N), t in [0, N/2).
+template <int N, bool INV> __device__ __forceinline__ float2 twiddle(const float2 *tw, int t)
+{
+    // t in [0, N)
+    float2 w = tw[t & (N / 2 - 1)];
+    if (t & (N / 2)) { w.x = -w.x; w.y = -w.y; }
+    if (INV) w.y = -w.y;
+    return w;
+}
+
+// One Stockham pass for item j (0 <= j < N/R) of one line: load + twiddle + DFT.
+template <int N, int R, int NS, bool INV, int PR>
+__device__ __forceinline__ void pass_load(const float2 *line, int j, const float2 *tw, float2 (&x)[R])
+{
+    constexpr int NIN = (PR == PRUNE_IN) ? R / 2 : R;
+#pragma unroll
+    for (int r = 0; r < NIN; ++r) x[r] = line[phys(j + r * (N / R))];
+#pragma unroll
+    for (int r = NIN; r < R; ++r) x[r] = make_float2(0.f, 0.f);
+    if constexpr (NS > 1) {
+        const int k = j & (NS - 1);
+#pragma unroll
+        for (int r = 1; r < NIN; ++r)
+            x[r] = cmul(x[r], twiddle<N, INV>(tw, r * k * (N / (NS * R))));
+    }
+    dft<R, INV, PR>(x);
+}
+
+template <int N, int R, int NS, int PR>
+__device__ __forceinline__ void pass_store(float2 *line, int j, const float2 (&x)[R])
+{
+    constexpr int NOUT = (PR == PRUNE_OUT) ? R / 2 : R;
+    const int k = j & (NS - 1);
+    const int base = (j - k) * R + k;
+#pragma unroll
+    for (int r = 0; r < NOUT; ++r) line[phys(base + r * NS)] = x[r];
+}
+
+// All T threads of the CTA transform G lines (line g at buf + g*LS) in place.
+// Ends with a __syncthreads(); callers must have synchronised after filling buf.
+template <int LOG2N, bool INV, int PRUNE, int T, int S = 0>
+__device__ __forceinline__ void fft_lines(float2 *buf, int G, int LS, const float2 *tw, int tid)
+{
+    constexpr int N = 1 << LOG2N;
+    constexpr int NP = n_passes(LOG2N);
+    if constexpr (S < NP) {
+        constexpr int R = 1 << pass_bits(LOG2N, S);
+        constexpr int NS = 1 << bits_before(LOG2N, S);
+        constexpr int PR = (PRUNE == PRUNE_IN && S == 0) ? PRUNE_IN
+                         : (PRUNE == PRUNE_OUT && S == NP - 1) ? PRUNE_OUT : PRUNE_NONE;
+        constexpr int IPL = N / R;                         // items per line
+        if constexpr (IPL <= T) {
+            constexpr int LPR = T / IPL;                   // lines per round
+            const int gl = tid / IPL, j = tid % IPL;
+            for (int g0 = 0; g0 < G; g0 += LPR) {
+                const int g = g0 + gl;
+                float2 x[R];
+                if (g < G) pass_load<N, R, NS, INV, PR>(buf + g * LS, j, tw, x);
+                __syncthreads();
+                if (g < G) pass_store<N, R, NS, PR>(buf + g * LS, j, x);
+            }
+        } else {
+            constexpr int IT = IPL / T;                    // items per thread per line
+            for (int g = 0; g < G; ++g) {
+                float2 x[IT][R];
+#pragma unroll
+                for (int i = 0; i < IT; ++i) pass_load<N, R, NS, INV, PR>(buf + g * LS, tid + i * T, tw, x[i]);
+                __syncthreads();
+#pragma unroll
+                for (int i = 0; i < IT; ++i) pass_store<N, R, NS, PR>(buf + g * LS, tid + i * T, x[i]);
+            }
+        }
+        __syncthreads();
+        fft_lines<LOG2N, INV, PRUNE, T, S + 1>(buf, G, LS, tw, tid);
+    }
+}
+
+// Fill the half twiddle table for N points from a global table of NT >= N points
+// (gt[t] = exp(-2 pi i t / NT)); caller synchronises afterwards.
+__device__ __forceinline__ void load_twiddles(float2 *tw, const float2 *gt, int N, int NT, int tid, int T)
+{
+    const int step = NT / N;
+    for (int t = tid; t < N / 2; t += T) tw[t] = gt[t * step];
+}
+
+}  // namespace hn

@@ -1,0 +1,398 @@
+// C ABI of the library: plan construction, argument checking, pass scheduling.
+// See include/hyenand.h for the contract of every entry point.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <vector>
+
+#include "../../include/hyenand.h"
+#include "common.cuh"
+#include "ct1d.cuh"
+
+using namespace hn;
+
+static thread_local char g_err[512] = "";
+static thread_local int g_code = 0;
+
+static int fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    g_code = code;
+    return code;
+}
+
+enum Path { PATH_ND_GENERIC = 0, PATH_CT1D = 1 };
+
+struct hyenand_plan {
+    int ndim, B, C, causal, dtype;
+    int dims[3];
+    int L[3], K[3], P[3], log2p[3];   // internal 3-axis form (leading axes of extent 1)
+    int XH;                           // half-spectrum bins along the contiguous axis
+    long long vol, kvol;              // elements per slice of q/k/v/y and of h
+    int path;
+    int device;
+    // generic path
+    long long slices_per_chunk;
+    long long ws_a_slice, ws_b_slice, wh_a_slice, wh_b_slice;   // float2 elements per slice
+    float2 *ws_a, *ws_b, *wh_a, *wh_b;
+    long long wh_slices;              // slices the filter workspace holds
+    float2 *gtw;
+    int gtw_n;
+    // long 1-D path
+    Ct1dPlan ct;
+    // host-staging for hyenand_forward_host
+    void *stage[5];
+    size_t stage_bytes[5];
+    size_t ws_bytes;
+};
+
+static int next_pow2_log(int x)
+{
+    int l = 0;
+    while ((1 << l) < x) ++l;
+    return l;
+}
+
+static size_t elsize(int dtype) { return dtype == HYENAND_F32 ? 4 : 2; }
+
+static int dev_alloc(hyenand_plan *p, void **ptr, size_t bytes)
+{
+    if (bytes == 0) bytes = 16;
+    cudaError_t e = cudaMalloc(ptr, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        *ptr = nullptr;
+        return fail(HYENAND_ERR_ALLOC, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+    }
+    p->ws_bytes += bytes;
+    return HYENAND_OK;
+}
+
+extern "C" const char *hyenand_last_error(void) { return g_err; }
+extern "C" int hyenand_last_error_code(void) { return g_err[0] ? g_code : HYENAND_OK; }
+
+extern "C" void hyenand_destroy_plan(hyenand_plan *p)
+{
+    if (!p) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != p->device) cudaSetDevice(p->device);
+    cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw);
+    ct1d_free(&p->ct);
+    for (int i = 0; i < 5; ++i) cudaFree(p->stage[i]);
+    if (cur != p->device) cudaSetDevice(cur);
+    delete p;
+}
+
+extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype)
+{
+    g_err[0] = 0;
+    if (ndim < 1 || ndim > 3) { fail(HYENAND_ERR_INVALID_ARG, "ndim must be 1, 2 or 3 (got %d)", ndim); return nullptr; }
+    if (!dims) { fail(HYENAND_ERR_INVALID_ARG, "dims is NULL"); return nullptr; }
+    if (B < 1 || C < 1) { fail(HYENAND_ERR_INVALID_ARG, "B and C must be >= 1 (got %d, %d)", B, C); return nullptr; }
+    if (dtype != HYENAND_F32 && dtype != HYENAND_BF16) { fail(HYENAND_ERR_INVALID_ARG, "unknown dtype %d", dtype); return nullptr; }
+    if (causal != 0 && causal != 1) { fail(HYENAND_ERR_INVALID_ARG, "causal must be 0 or 1"); return nullptr; }
+    for (int a = 0; a < ndim; ++a)
+        if (dims[a] < 1) { fail(HYENAND_ERR_INVALID_ARG, "dims[%d] = %d must be >= 1", a, dims[a]); return nullptr; }
+    if (causal && ndim != 1) { fail(HYENAND_ERR_UNSUPPORTED, "causal kernels are defined for 1-D grids only"); return nullptr; }
+
+    hyenand_plan *p = new hyenand_plan();
+    memset(p, 0, sizeof(*p));
+    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype;
+    cudaGetDevice(&p->device);
+    p->vol = 1; p->kvol = 1;
+    for (int a = 0; a < 3; ++a) { p->L[a] = 1; p->K[a] = 1; p->P[a] = 1; p->log2p[a] = 0; }
+    for (int a = 0; a < ndim; ++a) {
+        const int ia = 3 - ndim + a;
+        p->dims[a] = dims[a];
+        if ((long long)dims[a] > (1ll << 25)) { fail(HYENAND_ERR_UNSUPPORTED, "dims[%d] too long", a); delete p; return nullptr; }
+        p->L[ia] = dims[a];
+        p->K[ia] = causal ? dims[a] : 2 * dims[a] - 1;
+        p->log2p[ia] = next_pow2_log(2 * dims[a] - 1);
+        p->P[ia] = 1 << p->log2p[ia];
+        p->vol *= dims[a];
+        p->kvol *= p->K[ia];
+    }
+    p->XH = p->P[2] / 2 + 1;
+    const long long S = (long long)B * C;
+
+    if (ndim == 1 && p->log2p[2] > kMaxLineLog2) {
+        p->path = PATH_CT1D;
+        if (p->log2p[2] > 26) { fail(HYENAND_ERR_UNSUPPORTED, "1-D grid too long (padded size 2^%d > 2^26)", p->log2p[2]); delete p; return nullptr; }
+        size_t bytes = 0;
+        int e = ct1d_init(&p->ct, p->L[2], p->K[2], p->log2p[2], B, C, causal, dtype, &bytes);
+        if (e != HYENAND_OK) {
+            fail(e, "long 1-D path: workspace allocation of %zu bytes failed", bytes);
+            ct1d_free(&p->ct); delete p; return nullptr;
+        }
+        p->ws_bytes += bytes;
+        return p;
+    }
+    for (int a = 0; a < 3; ++a)
+        if (p->log2p[a] > kMaxLineLog2) {
+            fail(HYENAND_ERR_UNSUPPORTED, "padded axis of %d points exceeds the limit of %d for ndim >= 2",
+                 p->P[a], 1 << kMaxLineLog2);
+            delete p; return nullptr;
+        }
+
+    p->path = PATH_ND_GENERIC;
+    const bool three = p->P[0] > 1;
+    p->ws_a_slice = (long long)p->L[0] * p->L[1] * p->XH;
+    p->wh_a_slice = (long long)p->K[0] * p->K[1] * p->XH;
+    p->ws_b_slice = three ? (long long)p->L[0] * p->P[1] * p->XH : 0;
+    p->wh_b_slice = three ? (long long)p->K[0] * p->P[1] * p->XH : 0;
+    const long long per_slice = p->ws_a_slice + p->ws_b_slice + p->wh_a_slice + p->wh_b_slice;
+    const long long budget = (3ll << 30) / (long long)sizeof(float2);      // 3 GiB of workspace
+    long long spc = budget / per_slice;
+    if (spc < 1) spc = 1;
+    if (spc > S) spc = S;
+    p->slices_per_chunk = spc;
+    p->wh_slices = spc > C ? spc : C;      // room for all channels when the filter is shared
+
+    int gl = 1;
+    for (int a = 0; a < 3; ++a) if (p->log2p[a] > gl) gl = p->log2p[a];
+    p->gtw_n = 1 << gl;
+    std::vector<float2> tw(p->gtw_n);
+    for (int t = 0; t < p->gtw_n; ++t) {
+        const double ang = -2.0 * M_PI * (double)t / (double)p->gtw_n;
+        tw[t] = make_float2((float)cos(ang), (float)sin(ang));
+    }
+    int e = dev_alloc(p, (void **)&p->gtw, sizeof(float2) * p->gtw_n);
+    if (!e) e = dev_alloc(p, (void **)&p->ws_a, sizeof(float2) * p->ws_a_slice * spc);
+    if (!e && three) e = dev_alloc(p, (void **)&p->ws_b, sizeof(float2) * p->ws_b_slice * spc);
+    if (!e) e = dev_alloc(p, (void **)&p->wh_a, sizeof(float2) * p->wh_a_slice * p->wh_slices);
+    if (!e && three) e = dev_alloc(p, (void **)&p->wh_b, sizeof(float2) * p->wh_b_slice * p->wh_slices);
+    if (!e && cudaMemcpy(p->gtw, tw.data(), sizeof(float2) * p->gtw_n, cudaMemcpyHostToDevice) != cudaSuccess)
+        e = fail(HYENAND_ERR_CUDA, "twiddle upload failed: %s", cudaGetErrorString(cudaGetLastError()));
+    if (e) { hyenand_destroy_plan(p); return nullptr; }
+    return p;
+}
+
+// ---- generic path scheduling -----------------------------------------------------------
+
+static int filter_spectrum_generic(hyenand_plan *p, const char *h, long long n_slices, cudaStream_t st, int *launches)
+{
+    // rows of h, then (3-D) the middle axis
+    RowsArgs r{};
+    r.a = h; r.b = nullptr; r.out = p->wh_a;
+    r.rows = n_slices * p->K[0] * p->K[1];
+    r.len = p->K[2];
+    r.shift = p->causal ? 0 : p->L[2] - 1;
+    r.log2p = p->log2p[2];
+    r.prune_in = p->causal && p->P[2] >= 2;
+    r.gtw = p->gtw; r.gtw_n = p->gtw_n;
+    int n = launch_rows_fwd(r, p->dtype, st);
+    if (n < 0) return -1;
+    *launches += n;
+    if (p->P[0] > 1) {
+        AxisArgs a{};
+        a.in = p->wh_a; a.out = p->wh_b;
+        a.n_outer = n_slices * p->K[0];
+        a.in_outer = (long long)p->K[1] * p->XH;
+        a.out_outer = (long long)p->P[1] * p->XH;
+        a.nc = p->XH; a.n_in = p->K[1]; a.n_out = p->P[1];
+        a.shift = p->L[1] - 1; a.log2p = p->log2p[1]; a.prune_in = 0;
+        a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        n = launch_axis(a, AXIS_FWD, st);
+        if (n < 0) return -1;
+        *launches += n;
+    }
+    return 0;
+}
+
+static int forward_generic(hyenand_plan *p, const char *q, const char *k, const char *v, const char *h,
+                           bool shared, char *y, cudaStream_t st, int *launches)
+{
+    const long long S = (long long)p->B * p->C;
+    const size_t es = elsize(p->dtype);
+    const bool three = p->P[0] > 1;
+    if (shared && filter_spectrum_generic(p, h, p->C, st, launches)) return -1;
+    for (long long s0 = 0; s0 < S; s0 += p->slices_per_chunk) {
+        const long long n = S - s0 < p->slices_per_chunk ? S - s0 : p->slices_per_chunk;
+        if (!shared && filter_spectrum_generic(p, h + (size_t)s0 * p->kvol * es, n, st, launches)) return -1;
+        RowsArgs r{};
+        r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = p->ws_a;
+        r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
+        r.prune_in = 1; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
+        int c = launch_rows_fwd(r, p->dtype, st);
+        if (c < 0) return -1;
+        *launches += c;
+        if (three) {
+            AxisArgs a{};
+            a.in = p->ws_a; a.out = p->ws_b;
+            a.n_outer = n * p->L[0];
+            a.in_outer = (long long)p->L[1] * p->XH; a.out_outer = (long long)p->P[1] * p->XH;
+            a.nc = p->XH; a.n_in = p->L[1]; a.n_out = p->P[1]; a.shift = 0;
+            a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2;
+            a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+            c = launch_axis(a, AXIS_FWD, st);
+            if (c < 0) return -1;
+            *launches += c;
+        }
+        {
+            AxisArgs a{};
+            const int ax = three ? 0 : 1;                       // core axis
+            const long long inner = three ? (long long)p->P[1] * p->XH : p->XH;
+            a.in = three ? p->ws_b : p->ws_a; a.out = (float2 *)a.in;
+            a.n_outer = n;
+            a.in_outer = a.out_outer = (long long)p->L[ax] * inner;
+            a.nc = (int)inner; a.n_in = p->L[ax]; a.n_out = p->L[ax]; a.shift = 0;
+            a.log2p = p->log2p[ax]; a.prune_in = 1;
+            a.h = three ? p->wh_b : p->wh_a;
+            a.h_outer = (long long)p->K[ax] * inner;
+            a.h_n_in = p->K[ax];
+            a.h_shift = p->causal ? 0 : p->L[ax] - 1;
+            a.h_mod = shared ? p->C : 0;
+            a.h_off = shared ? s0 % p->C : 0;
+            a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
+            a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+            c = launch_axis(a, AXIS_CORE, st);
+            if (c < 0) return -1;
+            *launches += c;
+        }
+        if (three) {
+            AxisArgs a{};
+            a.in = p->ws_b; a.out = p->ws_a;
+            a.n_outer = n * p->L[0];
+            a.in_outer = (long long)p->P[1] * p->XH; a.out_outer = (long long)p->L[1] * p->XH;
+            a.nc = p->XH; a.n_in = p->P[1]; a.n_out = p->L[1]; a.shift = 0;
+            a.log2p = p->log2p[1]; a.prune_in = 0;
+            a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+            c = launch_axis(a, AXIS_INV, st);
+            if (c < 0) return -1;
+            *launches += c;
+        }
+        RowsInvArgs ri{};
+        ri.in = p->ws_a; ri.q = q + (size_t)s0 * p->vol * es; ri.y = y + (size_t)s0 * p->vol * es;
+        ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
+        ri.gtw = p->gtw; ri.gtw_n = p->gtw_n;
+        c = launch_rows_inv(ri, p->dtype, st);
+        if (c < 0) return -1;
+        *launches += c;
+    }
+    return 0;
+}
+
+static int run_forward(hyenand_plan *p, const void *q, const void *k, const void *v, const void *h,
+                       bool shared, void *y, cudaStream_t st, int *launches)
+{
+    int rc;
+    if (p->path == PATH_CT1D)
+        rc = ct1d_forward(&p->ct, q, k, v, h, shared, y, st, launches);
+    else
+        rc = forward_generic(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
+                             (char *)y, st, launches);
+    if (rc) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(HYENAND_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    return HYENAND_OK;
+}
+
+static int check_stride(hyenand_plan *p, long long hs, bool *shared)
+{
+    if (hs == 0) { *shared = true; return HYENAND_OK; }
+    if (hs == (long long)p->C * p->kvol) { *shared = false; return HYENAND_OK; }
+    return fail(HYENAND_ERR_INVALID_ARG, "h_batch_stride_elems must be 0 or C*K_1*..*K_N = %lld (got %lld)",
+                (long long)p->C * p->kvol, hs);
+}
+
+extern "C" int hyenand_forward_ex(hyenand_plan *p, const void *q, const void *k, const void *v, const void *h,
+                                  long long h_batch_stride_elems, void *y, void *cuda_stream)
+{
+    g_err[0] = 0;
+    if (!p) return fail(HYENAND_ERR_INVALID_ARG, "plan is NULL");
+    if (!q || !k || !v || !h || !y) return fail(HYENAND_ERR_INVALID_ARG, "q, k, v, h, y must be non-NULL");
+    const void *ptrs[5] = {q, k, v, h, y};
+    for (int i = 0; i < 5; ++i)
+        if (((uintptr_t)ptrs[i]) & 15) return fail(HYENAND_ERR_INVALID_ARG, "pointer %d is not 16-byte aligned", i);
+    bool shared = false;
+    int e = check_stride(p, h_batch_stride_elems, &shared);
+    if (e) return e;
+    const size_t es = elsize(p->dtype);
+    const size_t nbytes = (size_t)p->B * p->C * p->vol * es;
+    const size_t hbytes = (size_t)(shared ? 1 : p->B) * p->C * p->kvol * es;
+    const char *yb = (const char *)y;
+    const void *ins[4] = {q, k, v, h};
+    for (int i = 0; i < 4; ++i) {
+        const char *ib = (const char *)ins[i];
+        const size_t ilen = i == 3 ? hbytes : nbytes;
+        if (yb < ib + ilen && ib < yb + nbytes) return fail(HYENAND_ERR_INVALID_ARG, "y overlaps input %d", i);
+    }
+    int launches = 0;
+    return run_forward(p, q, k, v, h, shared, y, (cudaStream_t)cuda_stream, &launches);
+}
+
+extern "C" int hyenand_forward(hyenand_plan *p, const void *q, const void *k, const void *v, const void *h,
+                               void *y, void *cuda_stream)
+{
+    if (!p) { g_err[0] = 0; return fail(HYENAND_ERR_INVALID_ARG, "plan is NULL"); }
+    return hyenand_forward_ex(p, q, k, v, h, (long long)p->C * p->kvol, y, cuda_stream);
+}
+
+extern "C" int hyenand_forward_host(hyenand_plan *p, const void *q, const void *k, const void *v, const void *h,
+                                    long long h_batch_stride_elems, void *y, void *cuda_stream)
+{
+    g_err[0] = 0;
+    if (!p) return fail(HYENAND_ERR_INVALID_ARG, "plan is NULL");
+    if (!q || !k || !v || !h || !y) return fail(HYENAND_ERR_INVALID_ARG, "q, k, v, h, y must be non-NULL");
+    bool shared = false;
+    int e = check_stride(p, h_batch_stride_elems, &shared);
+    if (e) return e;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t es = elsize(p->dtype);
+    const size_t nbytes = (size_t)p->B * p->C * p->vol * es;
+    const size_t hbytes = (size_t)(shared ? 1 : p->B) * p->C * p->kvol * es;
+    const size_t want[5] = {nbytes, nbytes, nbytes, hbytes, nbytes};
+    for (int i = 0; i < 5; ++i) {
+        if (p->stage_bytes[i] < want[i]) {
+            if (p->stage[i]) { cudaFree(p->stage[i]); p->ws_bytes -= p->stage_bytes[i]; p->stage[i] = nullptr; p->stage_bytes[i] = 0; }
+            e = dev_alloc(p, &p->stage[i], want[i]);
+            if (e) return e;
+            p->stage_bytes[i] = want[i];
+        }
+    }
+    const void *src[4] = {q, k, v, h};
+    for (int i = 0; i < 4; ++i)
+        if (cudaMemcpyAsync(p->stage[i], src[i], want[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return fail(HYENAND_ERR_CUDA, "host-to-device copy %d failed: %s", i, cudaGetErrorString(cudaGetLastError()));
+    int launches = 0;
+    e = run_forward(p, p->stage[0], p->stage[1], p->stage[2], p->stage[3], shared, p->stage[4], st, &launches);
+    if (e) return e;
+    if (cudaMemcpyAsync(y, p->stage[4], nbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return fail(HYENAND_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+    cudaError_t ce = cudaStreamSynchronize(st);
+    if (ce != cudaSuccess) return fail(HYENAND_ERR_CUDA, "stream synchronise failed: %s", cudaGetErrorString(ce));
+    return HYENAND_OK;
+}
+
+extern "C" size_t hyenand_plan_workspace_bytes(const hyenand_plan *p) { return p ? p->ws_bytes : 0; }
+
+extern "C" int hyenand_plan_fft_dims(const hyenand_plan *p, int *out_P)
+{
+    g_err[0] = 0;
+    if (!p || !out_P) return fail(HYENAND_ERR_INVALID_ARG, "NULL argument");
+    for (int a = 0; a < p->ndim; ++a) out_P[a] = p->P[3 - p->ndim + a];
+    return HYENAND_OK;
+}
+
+extern "C" int hyenand_plan_launches(const hyenand_plan *p, int h_shared)
+{
+    if (!p) return 0;
+    if (p->path == PATH_CT1D) return ct1d_launches(&p->ct, h_shared != 0);
+    const long long S = (long long)p->B * p->C;
+    const long long chunks = (S + p->slices_per_chunk - 1) / p->slices_per_chunk;
+    const int three = p->P[0] > 1;
+    const int filt = 1 + three, body = 3 + 2 * three;
+    return (int)(h_shared ? filt + chunks * body : chunks * (filt + body));
+}
+
+extern "C" const char *hyenand_plan_path(const hyenand_plan *p)
+{
+    if (!p) return "";
+    return p->path == PATH_CT1D ? "ct1d" : "nd_generic";
+}

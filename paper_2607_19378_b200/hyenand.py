@@ -1,0 +1,172 @@
+"""ctypes binding of libhyenand.so: argument marshalling only.
+
+Every function has the name and meaning of the C entry point declared in
+include/hyenand.h; tensors are passed as raw device (or host) pointers and all
+arithmetic happens in the library's CUDA kernels.  There is no fallback: if the
+library has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhyenand.so")
+
+HYENAND_F32 = 0
+HYENAND_BF16 = 1
+HYENAND_OK = 0
+HYENAND_ERR_INVALID_ARG = 1
+HYENAND_ERR_UNSUPPORTED = 2
+HYENAND_ERR_ALLOC = 3
+HYENAND_ERR_CUDA = 4
+
+_DTYPES = {torch.float32: HYENAND_F32, torch.bfloat16: HYENAND_BF16}
+_lib = None
+
+
+class HyenaNDError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"hyenand error {code}: {msg}")
+        self.code = code
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C library (raises if it was never built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise OSError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_19378_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ip, ll = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.c_longlong
+        L.hyenand_create_plan.restype = vp
+        L.hyenand_create_plan.argtypes = [ctypes.c_int, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        L.hyenand_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.hyenand_forward_ex.argtypes = [vp, vp, vp, vp, vp, ll, vp, vp]
+        L.hyenand_forward_host.argtypes = [vp, vp, vp, vp, vp, ll, vp, vp]
+        L.hyenand_destroy_plan.argtypes = [vp]
+        L.hyenand_destroy_plan.restype = None
+        L.hyenand_last_error.restype = ctypes.c_char_p
+        L.hyenand_plan_workspace_bytes.argtypes = [vp]
+        L.hyenand_plan_workspace_bytes.restype = ctypes.c_size_t
+        L.hyenand_plan_fft_dims.argtypes = [vp, ip]
+        L.hyenand_plan_launches.argtypes = [vp, ctypes.c_int]
+        L.hyenand_plan_path.argtypes = [vp]
+        L.hyenand_plan_path.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def hyenand_last_error() -> str:
+    return lib().hyenand_last_error().decode()
+
+
+def hyenand_last_error_code() -> int:
+    return int(lib().hyenand_last_error_code())
+
+
+def _check(code: int):
+    if code != HYENAND_OK:
+        raise HyenaNDError(code, hyenand_last_error())
+
+
+def hyenand_create_plan(ndim: int, dims, B: int, C: int, causal: int, dtype: int) -> int:
+    arr = (ctypes.c_int * max(1, len(dims)))(*[int(d) for d in dims])
+    h = lib().hyenand_create_plan(int(ndim), arr, int(B), int(C), int(causal), int(dtype))
+    if not h:
+        msg = hyenand_last_error()
+        code = hyenand_last_error_code() or HYENAND_ERR_INVALID_ARG
+        raise HyenaNDError(code, msg)
+    return h
+
+
+def hyenand_destroy_plan(plan: int) -> None:
+    lib().hyenand_destroy_plan(plan)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def hyenand_forward(plan: int, q, k, v, h, y, stream=None) -> None:
+    _check(lib().hyenand_forward(plan, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
+                                 y.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_forward_ex(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stream=None) -> None:
+    _check(lib().hyenand_forward_ex(plan, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
+                                    int(h_batch_stride_elems), y.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_forward_host(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stream=None) -> None:
+    _check(lib().hyenand_forward_host(plan, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
+                                      int(h_batch_stride_elems), y.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_plan_workspace_bytes(plan: int) -> int:
+    return int(lib().hyenand_plan_workspace_bytes(plan))
+
+
+def hyenand_plan_fft_dims(plan: int, ndim: int):
+    out = (ctypes.c_int * ndim)()
+    _check(lib().hyenand_plan_fft_dims(plan, out))
+    return tuple(out)
+
+
+def hyenand_plan_launches(plan: int, h_shared: bool) -> int:
+    return int(lib().hyenand_plan_launches(plan, 1 if h_shared else 0))
+
+
+def hyenand_plan_path(plan: int) -> str:
+    return lib().hyenand_plan_path(plan).decode()
+
+
+class Plan:
+    """Convenience owner of a plan handle (create on construction, destroy on close)."""
+
+    def __init__(self, dims, B: int, C: int, causal: bool = False, dtype=torch.float32):
+        self.dims = tuple(int(d) for d in dims)
+        self.B, self.C, self.causal, self.dtype = B, C, bool(causal), dtype
+        self.handle = hyenand_create_plan(len(self.dims), self.dims, B, C, int(self.causal), _DTYPES[dtype])
+
+    def _stride(self, h) -> int:
+        taps = tuple(L if self.causal else 2 * L - 1 for L in self.dims)
+        if tuple(h.shape) == (self.C,) + taps:
+            return 0
+        if tuple(h.shape) == (self.B, self.C) + taps:
+            return self.C * h[0, 0].numel()
+        raise ValueError(f"h has shape {tuple(h.shape)}")
+
+    def forward(self, q, k, v, h, y=None, stream=None):
+        """Device tensors in, device tensor out (enqueued on the current stream)."""
+        for t in (q, k, v, h):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == self.dtype):
+                raise ValueError("inputs must be contiguous CUDA tensors of the plan's dtype")
+        if y is None:
+            y = torch.empty_like(q)
+        hyenand_forward_ex(self.handle, q, k, v, h, self._stride(h), y, stream)
+        return y
+
+    def forward_host(self, q, k, v, h, y, stream=None):
+        """Host tensors in, host tensor out; copies run inside the call."""
+        hyenand_forward_host(self.handle, q, k, v, h, self._stride(h), y, stream)
+        return y
+
+    @property
+    def launches_per_forward(self):
+        return lambda shared: hyenand_plan_launches(self.handle, shared)
+
+    def close(self):
+        if self.handle:
+            hyenand_destroy_plan(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
