@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the gated N-D long convolution (HyenaND FFT hot path) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one forward of the whole path (gate+pad, forward transforms of k*v
+and h, spectral product, inverse, crop, output gate) over one synthetic batch of
+the chosen workload.  Rank 0 prints ONE JSON line.  `value` is B*C*L elements
+per second over all ranks with inputs resident in HBM; `e2e` is the same metric
+through hyenand_forward_host (host buffers, copies inside the timed region).
+With more than one GPU every rank runs its own batch of the same shape (weak
+scaling, no collective on the data path).
+
+--impl reference times the CPU oracle (fp64, radix-2 FFT path) on a bounded
+sample of the same workload on the host cores; it is a deliberately plain
+program, reported as a baseline only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2607_19378_b200 import workloads as W  # noqa: E402
+
+METRIC = "hyenand_forward_throughput"
+UNIT = "Gelem/s"
+DEFAULT_WORKLOAD = "volume3d"
+FP32_LANES_PER_SM = 128
+
+
+# ---- roofline bookkeeping ----------------------------------------------------------------
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured", float(d.get("sm_max_mhz", 1965.0))
+    return 6650.0, "fallback", 1965.0
+
+
+def fp32_peak_tflops(sm_count: int, sm_max_mhz: float) -> float:
+    # 2 flops (FMA) x 128 FP32 lanes x SMs x max SM clock
+    return 2.0 * FP32_LANES_PER_SM * sm_count * sm_max_mhz * 1e6 / 1e12
+
+
+def op_algorithmic(w: W.Workload):
+    """Minimal bytes (q,k,v,h,y once) and nominal flops (2.5 P log2 P per real transform:
+    k*v forward and the inverse per slice, h forward per filter) of one forward."""
+    s = 4 if w.dtype == "f32" else 2
+    E = w.elements
+    hcount = w.C if w.h_shared else w.B * w.C
+    hbytes = hcount * math.prod(w.taps) * s
+    P = 1
+    for L in w.dims:
+        P *= 1 << max(0, (2 * L - 2).bit_length())
+    transforms = 2 * w.B * w.C + hcount
+    flops = transforms * 2.5 * P * math.log2(P) if P > 1 else 0.0
+    return 4 * E * s + hbytes, flops, P
+
+
+# ---- clocks ---------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.lines = []
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t0: float, t1: float):
+        """Median SM clock and the throttle reasons seen between wall-clock t0 and t1."""
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return out
+        import datetime
+        sm, reasons, smax = [], set(), None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in text.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if not (t0 - 0.05 <= ts <= t1 + 0.05):
+                    continue
+                sm.append(float(parts[1]))
+                smax = float(parts[2])
+                for n, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ---- our arm ----------------------------------------------------------------------------------
+
+def time_workload(w: W.Workload, steps: int, warmup: int, dist, device, want_kernels: bool,
+                  sampler_device=None):
+    """Device-resident timing of `steps` forwards.  Returns a dict of raw measurements."""
+    from paper_2607_19378_b200 import hyenand as hn
+    q, k, v, h = W.make_inputs(w, device=device)
+    y = torch.empty_like(q)
+    plan = hn.Plan(w.dims, w.B, w.C, causal=w.causal, dtype=w.torch_dtype)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(warmup, 3)):
+        plan.forward(q, k, v, h, y)
+    torch.cuda.synchronize()
+    if want_kernels:
+        hn.hyenand_plan_set_timing(plan.handle, True)
+    sampler = ClockSampler(sampler_device) if sampler_device is not None else None
+    if sampler is not None:
+        time.sleep(0.6)                       # let nvidia-smi start sampling
+        for _ in range(3):                    # re-warm after the pause
+            plan.forward(q, k, v, h, y)
+        torch.cuda.synchronize()
+        if want_kernels:
+            hn.hyenand_plan_set_timing(plan.handle, True)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record(stream)
+    for _ in range(steps):
+        plan.forward(q, k, v, h, y)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    if dist is not None:
+        dist.barrier()
+    ms = e0.elapsed_time(e1) / steps
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
+    kernels = []
+    if want_kernels:
+        for kid in range(hn.hyenand_plan_kernel_count(plan.handle)):
+            name, launches, nbytes, flops = hn.hyenand_plan_kernel_info(plan.handle, kid, w.h_shared)
+            tot_ms, n = hn.hyenand_plan_kernel_time(plan.handle, kid)
+            if n > 0:
+                kernels.append({"name": name, "launches_per_step": n / steps, "ms_per_step": tot_ms / steps,
+                                "ms_per_launch": tot_ms / n, "bytes_per_launch": nbytes / launches,
+                                "flops_per_launch": flops / launches})
+        hn.hyenand_plan_set_timing(plan.handle, False)
+    res = {"ms": ms, "clocks": clocks, "kernels": kernels,
+           "launches": hn.hyenand_plan_launches(plan.handle, w.h_shared),
+           "path": hn.hyenand_plan_path(plan.handle),
+           "workspace_bytes": hn.hyenand_plan_workspace_bytes(plan.handle)}
+    return res, plan, (q, k, v, h, y)
+
+
+def time_e2e(w: W.Workload, plan, tensors, steps: int, dist):
+    q, k, v, h, y = tensors
+    host = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (q, k, v, h, y)]
+    for dst, src in zip(host[:4], (q, k, v, h)):
+        dst.copy_(src)
+    torch.cuda.synchronize()
+    plan.forward_host(*host)                          # allocates the staging buffers, warms up
+    plan.forward_host(*host)
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        plan.forward_host(*host)                      # returns after y is back on the host
+    dt = (time.perf_counter() - t0) / steps
+    if dist is not None:
+        dist.barrier()
+    h2d = sum(t.numel() * t.element_size() for t in host[:4])
+    d2h = host[4].numel() * host[4].element_size()
+    return dt * 1e3, h2d, d2h
+
+
+def cpu_oracle_sample(w: W.Workload, budget_s: float = 15.0):
+    """Times the oracle (as it stands) on a bounded sample of slices of the workload."""
+    import oracle
+    threads = oracle.threads()
+    mode = "causal" if w.causal else "linear"
+
+    def run(n_slices):
+        ws = w.scaled(B=1, C=n_slices)
+        q, k, v, h = W.make_inputs(ws, device="cpu")
+        t0 = time.perf_counter()
+        oracle.conv_fft(q, k, v, h, mode)
+        return time.perf_counter() - t0, ws.elements
+
+    S = w.B * w.C
+    n = min(S, threads)
+    dt, elems = run(n)
+    if dt < budget_s / 3 and n < S:
+        n2 = min(S, max(n, int(n * (budget_s / max(dt, 1e-3)) // threads * threads)))
+        if n2 > n:
+            n = n2
+            dt, elems = run(n)
+    return {"value": elems / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{n} of {S} (b,c) slices of {w.name}, oracle FFT path (fp64, radix-2), {dt:.1f} s"}
+
+
+def roofline_of(kern, hbm_gbs, peak_src, fp32_tf, traffic):
+    t_h = kern["bytes_per_launch"] / (hbm_gbs * 1e9)
+    t_a = kern["flops_per_launch"] / (fp32_tf * 1e12)
+    dur = kern["ms_per_launch"] * 1e-3
+    if t_h >= t_a:
+        ach = kern["bytes_per_launch"] / dur / 1e9
+        return {"kernel": kern["name"], "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                "frac": ach / hbm_gbs, "traffic": traffic, "peak_source": f"of {peak_src}"}
+    ach = kern["flops_per_launch"] / dur / 1e12
+    return {"kernel": kern["name"], "bound": "alu", "achieved": ach, "peak": fp32_tf, "unit": "TFLOP/s",
+            "frac": ach / fp32_tf, "traffic": traffic,
+            "peak_source": "derived: 2 x 128 FP32 lanes x SMs x max SM clock"}
+
+
+def load_traffic(workload: str, kernel: str):
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    try:
+        with open(path) as f:
+            return json.load(f).get(workload, {}).get(kernel)
+    except Exception:
+        return None
+
+
+def main_ours(args):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    w = W.WORKLOADS[args.workload]
+    if world > 1:
+        from dataclasses import replace
+        w = replace(w, seed=w.seed + 100 * rank)
+    hbm_gbs, peak_src, sm_max = measured_peaks()
+    props = torch.cuda.get_device_properties(local)
+    fp32_tf = fp32_peak_tflops(props.multi_processor_count, sm_max)
+
+    res, plan, tensors = time_workload(w, args.steps, args.warmup, dist, device, True, sampler_device=local)
+    ms = res["ms"]
+    e2e_ms, h2d, d2h = time_e2e(w, plan, tensors, max(2, min(args.steps, 5)), dist)
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+    plan.close()
+    del tensors
+    torch.cuda.empty_cache()
+
+    total_elems = w.elements * world
+    nbytes, flops, P = op_algorithmic(w)
+    t_hbm = nbytes / (hbm_gbs * 1e9) * 1e3
+    t_alu = flops / (fp32_tf * 1e12) * 1e3
+    kernels = sorted(res["kernels"], key=lambda kk: -kk["ms_per_step"])
+    dom = kernels[0] if kernels else None
+    out = {
+        "metric": METRIC, "value": total_elems / (ms * 1e-3) / 1e9, "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "dims": list(w.dims), "B": w.B, "C": w.C, "causal": w.causal,
+                   "h_shared_over_batch": w.h_shared, "padded_points_per_slice": P,
+                   "l2": "inputs larger than L2 (no flush needed)" if nbytes > 126e6 else "fits L2; latency-bound",
+                   "path": res["path"], "per_gpu_batch": "fixed (each rank runs the full workload)"},
+        "clocks": res["clocks"],
+        "e2e": {"value": total_elems / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": res["launches"] * args.steps,
+        "roofline": roofline_of(dom, hbm_gbs, peak_src, fp32_tf, load_traffic(w.name, dom["name"])) if dom else None,
+        "op_roofline": {"t_hbm_ms": t_hbm, "t_fp32_ms": t_alu, "roofline_ms": max(t_hbm, t_alu),
+                        "frac": max(t_hbm, t_alu) / ms, "hbm_peak_gbs": hbm_gbs, "hbm_peak_source": peak_src,
+                        "fp32_peak_tflops": fp32_tf, "min_bytes": nbytes, "nominal_flops": flops},
+        "kernels": [{"name": kk["name"], "launches_per_step": kk["launches_per_step"],
+                     "ms_per_step": round(kk["ms_per_step"], 5),
+                     "share": kk["ms_per_step"] / max(sum(x["ms_per_step"] for x in kernels), 1e-12),
+                     "GBps_algorithmic": kk["bytes_per_launch"] / (kk["ms_per_launch"] * 1e-3) / 1e9,
+                     "TFLOPs_nominal": kk["flops_per_launch"] / (kk["ms_per_launch"] * 1e-3) / 1e12}
+                    for kk in kernels],
+        "workspace_bytes": res["workspace_bytes"],
+    }
+    if world == 1 and rank == 0:
+        if not args.no_all:
+            table = []
+            for name, ww in W.WORKLOADS.items():
+                if name == w.name:
+                    r_ms, path = ms, res["path"]
+                else:
+                    r, p2, tens = time_workload(ww, max(3, min(args.steps, 10)), 3, None, device, False)
+                    r_ms, path = r["ms"], r["path"]
+                    p2.close()
+                    del tens, p2
+                    torch.cuda.empty_cache()
+                nb, fl, _ = op_algorithmic(ww)
+                th, ta = nb / (hbm_gbs * 1e9) * 1e3, fl / (fp32_tf * 1e12) * 1e3
+                table.append({"workload": name, "ms": r_ms, "gelem_s": ww.elements / (r_ms * 1e-3) / 1e9,
+                              "t_hbm_ms": th, "t_fp32_ms": ta, "roofline_frac": max(th, ta) / r_ms, "path": path})
+            out["all_workloads"] = table
+        if not args.no_cpu:
+            out["cpu_baseline"] = cpu_oracle_sample(w)
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ---- reference arm: the CPU oracle ----------------------------------------------------------------
+
+def main_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = W.WORKLOADS[args.workload]
+    threads = oracle.threads()
+    mode = "causal" if w.causal else "linear"
+    S = w.B * w.C
+    # size one step at roughly 2 s of oracle time: probe with one slice per thread first
+    n = min(S, threads)
+    ws = w.scaled(B=1, C=n)
+    q, k, v, h = W.make_inputs(ws, device="cpu")
+    t0 = time.perf_counter()
+    oracle.conv_fft(q, k, v, h, mode)
+    probe = time.perf_counter() - t0
+    if probe < 1.0 and n < S:
+        n = min(S, max(n, int(n * (2.0 / max(probe, 1e-3)) // threads * threads)))
+        ws = w.scaled(B=1, C=n)
+        q, k, v, h = W.make_inputs(ws, device="cpu")
+    warm = max(0, min(args.warmup, 1 if probe > 5 else args.warmup))
+    steps = args.steps if probe * args.steps < 240 else max(1, int(240 / probe))
+    for _ in range(warm):
+        oracle.conv_fft(q, k, v, h, mode)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.conv_fft(q, k, v, h, mode)
+    dt = (time.perf_counter() - t0) / steps
+    val = ws.elements / dt / 1e9
+    sample = f"{n} of {S} (b,c) slices of {w.name} per step, oracle FFT path (fp64, radix-2)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "dims": list(w.dims), "B": w.B, "C": w.C, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+if __name__ == "__main__":
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.WORKLOADS))
+    ap.add_argument("--no-all", action="store_true", help="skip the table over the other workloads")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    a = ap.parse_args()
+    if a.impl == "reference":
+        main_reference(a)
+    else:
+        main_ours(a)

@@ -113,6 +113,29 @@ int hyenand_plan_fft_dims(const hyenand_plan *plan, int *out_P);      /* writes 
 int hyenand_plan_launches(const hyenand_plan *plan, int h_shared);    /* kernels enqueued by one forward */
 const char *hyenand_plan_path(const hyenand_plan *plan);              /* name of the kernel path chosen */
 
+
+/*
+ * Per-kernel accounting, for benchmarks.  Kernel ids run from 0 to
+ * hyenand_plan_kernel_count()-1.  hyenand_plan_kernel_info gives, for one
+ * forward of this plan (h_shared: filter shared over the batch or not), the
+ * kernel's name, how often it is launched, and the ALGORITHMIC bytes and flops
+ * of all its launches together: bytes = its inputs read once plus its outputs
+ * written once; flops = 5 N log2 N per complex N-point line transform it
+ * performs (un-pruned count) plus 12 per padded bin where it multiplies
+ * spectra.  A kernel this plan never launches reports zeros.
+ * hyenand_plan_set_timing(plan, 1) makes every later forward bracket each
+ * kernel launch with CUDA events on the launching stream (and clears the
+ * totals); hyenand_plan_kernel_time returns the accumulated device time and
+ * launch count of one kernel and must only be called after the stream has
+ * been synchronised.  At most 4096 launches are recorded between two calls of
+ * hyenand_plan_kernel_time.
+ */
+int hyenand_plan_kernel_count(const hyenand_plan *plan);
+int hyenand_plan_kernel_info(const hyenand_plan *plan, int kernel_id, int h_shared, const char **name,
+                             double *launches, double *bytes, double *flops);
+int hyenand_plan_set_timing(hyenand_plan *plan, int enable);
+int hyenand_plan_kernel_time(hyenand_plan *plan, int kernel_id, double *total_ms, double *launches);
+
 #ifdef __cplusplus
 }
 #endif

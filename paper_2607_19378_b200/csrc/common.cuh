@@ -21,6 +21,61 @@ template <> struct IO<bf16> {
     static __device__ __forceinline__ void st(bf16 *p, long long i, float v) { p[i] = __float2bfloat16_rn(v); }
 };
 
+// Optional per-kernel timing: when enabled, every kernel launch of a forward is
+// bracketed by CUDA events on the launching stream; collect() (after the caller
+// synchronised) adds the elapsed times to per-kernel totals.
+enum KernelId {
+    KID_ROWS_H = 0, KID_AXIS_H, KID_ROWS_U, KID_AXIS_U, KID_CORE, KID_AXIS_INV, KID_ROWS_INV,
+    KID_CT_COLS_H, KID_CT_COLS_U, KID_CT_CORE, KID_CT_COLS_INV, KID_COUNT
+};
+
+struct Prof {
+    bool on = false;
+    struct Rec { cudaEvent_t a, b; int kid; };
+    Rec recs[4096];
+    int created = 0, used = 0;
+    double ms[KID_COUNT] = {0};
+    long long launches[KID_COUNT] = {0};
+    void begin(int kid, cudaStream_t st)
+    {
+        if (!on || used >= 4096) return;
+        if (used == created) {
+            cudaEventCreate(&recs[created].a);
+            cudaEventCreate(&recs[created].b);
+            ++created;
+        }
+        recs[used].kid = kid;
+        cudaEventRecord(recs[used].a, st);
+    }
+    void end(cudaStream_t st)
+    {
+        if (!on || used >= 4096) return;
+        cudaEventRecord(recs[used].b, st);
+        ++used;
+    }
+    void collect()
+    {
+        for (int i = 0; i < used; ++i) {
+            float t = 0.f;
+            if (cudaEventElapsedTime(&t, recs[i].a, recs[i].b) == cudaSuccess) {
+                ms[recs[i].kid] += t;
+                launches[recs[i].kid] += 1;
+            }
+        }
+        used = 0;
+    }
+    void reset()
+    {
+        used = 0;
+        for (int i = 0; i < KID_COUNT; ++i) { ms[i] = 0; launches[i] = 0; }
+    }
+    void destroy()
+    {
+        for (int i = 0; i < created; ++i) { cudaEventDestroy(recs[i].a); cudaEventDestroy(recs[i].b); }
+        created = used = 0;
+    }
+};
+
 constexpr int kMaxLineLog2 = 13;          // longest line transformed in shared memory: 8192 points
 constexpr int kThreads = 256;             // threads per CTA of the generic kernels
 

@@ -400,34 +400,38 @@ void ct1d_free(Ct1dPlan *c)
     c->wu = c->wh = c->tw1 = c->tw2 = c->twp_fine = c->twp_coarse = nullptr;
 }
 
-static int filter_pass(Ct1dPlan *c, const char *h, long long n, cudaStream_t st, int *launches)
+static int filter_pass(Ct1dPlan *c, const char *h, long long n, cudaStream_t st, int *launches, Prof *prof)
 {
     ColsFwdArgs a{};
     a.a = h; a.b = nullptr; a.out = c->wh; a.slices = n; a.in_slice = c->K; a.len = c->K;
     a.shift = c->causal ? 0 : c->L - 1;
     a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.tw1_n = 1 << c->log2p1;
     a.twp = TwoLevel{c->twp_coarse, c->twp_fine, c->lo};
+    prof->begin(KID_CT_COLS_H, st);
     int r = launch_cols_fwd(a, c->log2p1, c->causal != 0, c->dtype, st);
+    prof->end(st);
     if (r < 0) return -1;
     *launches += r;
     return 0;
 }
 
 int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const void *h, bool shared,
-                 void *y, cudaStream_t st, int *launches)
+                 void *y, cudaStream_t st, int *launches, Prof *prof)
 {
     const long long S = (long long)c->B * c->C;
     const size_t es = c->dtype == 0 ? 4 : 2;
     const TwoLevel twp{c->twp_coarse, c->twp_fine, c->lo};
-    if (shared && filter_pass(c, (const char *)h, c->C, st, launches)) return -1;
+    if (shared && filter_pass(c, (const char *)h, c->C, st, launches, prof)) return -1;
     for (long long s0 = 0; s0 < S; s0 += c->slices_per_chunk) {
         const long long n = S - s0 < c->slices_per_chunk ? S - s0 : c->slices_per_chunk;
-        if (!shared && filter_pass(c, (const char *)h + (size_t)s0 * c->K * es, n, st, launches)) return -1;
+        if (!shared && filter_pass(c, (const char *)h + (size_t)s0 * c->K * es, n, st, launches, prof)) return -1;
         ColsFwdArgs a{};
         a.a = (const char *)k + (size_t)s0 * c->L * es; a.b = (const char *)v + (size_t)s0 * c->L * es;
         a.out = c->wu; a.slices = n; a.in_slice = c->L; a.len = c->L; a.shift = 0;
         a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.tw1_n = 1 << c->log2p1; a.twp = twp;
+        prof->begin(KID_CT_COLS_U, st);
         int r = launch_cols_fwd(a, c->log2p1, true, c->dtype, st);
+        prof->end(st);
         if (r < 0) return -1;
         *launches += r;
         CoreArgs cr{};
@@ -435,13 +439,17 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
         cr.h_mod = shared ? c->C : 0; cr.h_off = shared ? s0 % c->C : 0;
         cr.scale = (float)ldexp(1.0, -c->log2p);
         cr.tw2 = c->tw2; cr.tw2_n = 1 << c->log2p2; cr.twp = twp;
+        prof->begin(KID_CT_CORE, st);
         r = launch_core(cr, c->log2p2, st);
+        prof->end(st);
         if (r < 0) return -1;
         *launches += r;
         ColsInvArgs ci{};
         ci.in = c->wu; ci.q = (const char *)q + (size_t)s0 * c->L * es; ci.y = (char *)y + (size_t)s0 * c->L * es;
         ci.slices = n; ci.len = c->L; ci.log2p2 = c->log2p2; ci.tw1 = c->tw1; ci.tw1_n = 1 << c->log2p1;
+        prof->begin(KID_CT_COLS_INV, st);
         r = launch_cols_inv(ci, c->log2p1, c->dtype, st);
+        prof->end(st);
         if (r < 0) return -1;
         *launches += r;
     }

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stddef.h>
 
+#include "common.cuh"
+
 namespace hn {
 
 struct Ct1dPlan {
@@ -21,7 +23,7 @@ struct Ct1dPlan {
 int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, int dtype, size_t *bytes);
 void ct1d_free(Ct1dPlan *c);
 int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const void *h, bool shared,
-                 void *y, cudaStream_t st, int *launches);
+                 void *y, cudaStream_t st, int *launches, Prof *prof);
 int ct1d_launches(const Ct1dPlan *c, bool shared);
 
 }  // namespace hn

@@ -49,6 +49,7 @@ struct hyenand_plan {
     void *stage[5];
     size_t stage_bytes[5];
     size_t ws_bytes;
+    Prof prof;
 };
 
 static int next_pow2_log(int x)
@@ -85,6 +86,7 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
     cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw);
     ct1d_free(&p->ct);
     for (int i = 0; i < 5; ++i) cudaFree(p->stage[i]);
+    p->prof.destroy();
     if (cur != p->device) cudaSetDevice(cur);
     delete p;
 }
@@ -186,7 +188,9 @@ static int filter_spectrum_generic(hyenand_plan *p, const char *h, long long n_s
     r.log2p = p->log2p[2];
     r.prune_in = p->causal && p->P[2] >= 2;
     r.gtw = p->gtw; r.gtw_n = p->gtw_n;
+    p->prof.begin(KID_ROWS_H, st);
     int n = launch_rows_fwd(r, p->dtype, st);
+    p->prof.end(st);
     if (n < 0) return -1;
     *launches += n;
     if (p->P[0] > 1) {
@@ -198,7 +202,9 @@ static int filter_spectrum_generic(hyenand_plan *p, const char *h, long long n_s
         a.nc = p->XH; a.n_in = p->K[1]; a.n_out = p->P[1];
         a.shift = p->L[1] - 1; a.log2p = p->log2p[1]; a.prune_in = 0;
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        p->prof.begin(KID_AXIS_H, st);
         n = launch_axis(a, AXIS_FWD, st);
+        p->prof.end(st);
         if (n < 0) return -1;
         *launches += n;
     }
@@ -219,7 +225,9 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = p->ws_a;
         r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
         r.prune_in = 1; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
+        p->prof.begin(KID_ROWS_U, st);
         int c = launch_rows_fwd(r, p->dtype, st);
+        p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;
         if (three) {
@@ -230,7 +238,9 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.nc = p->XH; a.n_in = p->L[1]; a.n_out = p->P[1]; a.shift = 0;
             a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+            p->prof.begin(KID_AXIS_U, st);
             c = launch_axis(a, AXIS_FWD, st);
+            p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
         }
@@ -251,7 +261,9 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.h_off = shared ? s0 % p->C : 0;
             a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+            p->prof.begin(KID_CORE, st);
             c = launch_axis(a, AXIS_CORE, st);
+            p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
         }
@@ -263,7 +275,9 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.nc = p->XH; a.n_in = p->P[1]; a.n_out = p->L[1]; a.shift = 0;
             a.log2p = p->log2p[1]; a.prune_in = 0;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+            p->prof.begin(KID_AXIS_INV, st);
             c = launch_axis(a, AXIS_INV, st);
+            p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
         }
@@ -271,7 +285,9 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         ri.in = p->ws_a; ri.q = q + (size_t)s0 * p->vol * es; ri.y = y + (size_t)s0 * p->vol * es;
         ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
         ri.gtw = p->gtw; ri.gtw_n = p->gtw_n;
+        p->prof.begin(KID_ROWS_INV, st);
         c = launch_rows_inv(ri, p->dtype, st);
+        p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;
     }
@@ -283,7 +299,7 @@ static int run_forward(hyenand_plan *p, const void *q, const void *k, const void
 {
     int rc;
     if (p->path == PATH_CT1D)
-        rc = ct1d_forward(&p->ct, q, k, v, h, shared, y, st, launches);
+        rc = ct1d_forward(&p->ct, q, k, v, h, shared, y, st, launches, &p->prof);
     else
         rc = forward_generic(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
                              (char *)y, st, launches);
@@ -395,4 +411,100 @@ extern "C" const char *hyenand_plan_path(const hyenand_plan *p)
 {
     if (!p) return "";
     return p->path == PATH_CT1D ? "ct1d" : "nd_generic";
+}
+
+// ---- per-kernel accounting (reporting only) ---------------------------------------------
+
+static const char *kKernelNames[KID_COUNT] = {
+    "rows_fwd(h)", "axis_fwd(h)", "rows_fwd(k*v)", "axis_fwd(k*v)", "axis_core", "axis_inv", "rows_inv",
+    "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv"};
+
+static double fft_flops(double lines, int log2n) { return lines * 5.0 * ldexp(1.0, log2n) * log2n; }
+
+extern "C" int hyenand_plan_kernel_count(const hyenand_plan *p) { return p ? KID_COUNT : 0; }
+
+extern "C" int hyenand_plan_kernel_info(const hyenand_plan *p, int kid, int h_shared, const char **name,
+                                        double *launches, double *bytes, double *flops)
+{
+    g_err[0] = 0;
+    if (!p || kid < 0 || kid >= KID_COUNT || !name || !launches || !bytes || !flops)
+        return fail(HYENAND_ERR_INVALID_ARG, "bad argument");
+    *name = kKernelNames[kid];
+    *launches = *bytes = *flops = 0.0;
+    const double S = (double)p->B * p->C, Sh = h_shared ? p->C : S;
+    const double es = (double)elsize(p->dtype), c8 = 8.0;
+    if (p->path == PATH_CT1D) {
+        const Ct1dPlan &c = p->ct;
+        const double P1 = ldexp(1.0, c.log2p1), P2 = ldexp(1.0, c.log2p2), F1 = P1 / 2 + 1;
+        const double chunks = ceil(S / (double)c.slices_per_chunk);
+        switch (kid) {
+        case KID_CT_COLS_H:
+            *launches = h_shared ? 1 : chunks; *bytes = Sh * (c.K * es + F1 * P2 * c8);
+            *flops = fft_flops(Sh * P2 / 2, c.log2p1); break;
+        case KID_CT_COLS_U:
+            *launches = chunks; *bytes = S * (2 * c.L * es + F1 * P2 * c8);
+            *flops = fft_flops(S * P2 / 2, c.log2p1); break;
+        case KID_CT_CORE:
+            *launches = chunks; *bytes = S * 3 * F1 * P2 * c8;
+            *flops = 3 * fft_flops(S * F1, c.log2p2) + 12.0 * S * F1 * P2; break;
+        case KID_CT_COLS_INV:
+            *launches = chunks; *bytes = S * (F1 * P2 * c8 + 2 * c.L * es);
+            *flops = fft_flops(S * P2 / 2, c.log2p1); break;
+        default: break;
+        }
+        return HYENAND_OK;
+    }
+    const bool three = p->P[0] > 1;
+    const double chunks = ceil(S / (double)p->slices_per_chunk);
+    const double XH = p->XH, L0 = p->L[0], L1 = p->L[1], L2 = p->L[2], K0 = p->K[0], K1 = p->K[1], P1 = p->P[1];
+    const int ax = three ? 0 : 1;
+    const double inner = three ? P1 * XH : XH;
+    switch (kid) {
+    case KID_ROWS_H:
+        *launches = h_shared ? 1 : chunks; *bytes = Sh * ((double)p->kvol * es + K0 * K1 * XH * c8);
+        *flops = fft_flops(Sh * K0 * K1 / 2, p->log2p[2]); break;
+    case KID_AXIS_H:
+        if (three) { *launches = h_shared ? 1 : chunks; *bytes = Sh * K0 * XH * c8 * (K1 + P1);
+                     *flops = fft_flops(Sh * K0 * XH, p->log2p[1]); }
+        break;
+    case KID_ROWS_U:
+        *launches = chunks; *bytes = S * (2.0 * p->vol * es + L0 * L1 * XH * c8);
+        *flops = fft_flops(S * L0 * L1 / 2, p->log2p[2]); break;
+    case KID_AXIS_U:
+        if (three) { *launches = chunks; *bytes = S * L0 * XH * c8 * (L1 + P1);
+                     *flops = fft_flops(S * L0 * XH, p->log2p[1]); }
+        break;
+    case KID_CORE:
+        *launches = chunks; *bytes = S * inner * c8 * (2.0 * p->L[ax] + p->K[ax]);
+        *flops = 3 * fft_flops(S * inner, p->log2p[ax]) + 12.0 * S * inner * p->P[ax]; break;
+    case KID_AXIS_INV:
+        if (three) { *launches = chunks; *bytes = S * L0 * XH * c8 * (L1 + P1);
+                     *flops = fft_flops(S * L0 * XH, p->log2p[1]); }
+        break;
+    case KID_ROWS_INV:
+        *launches = chunks; *bytes = S * (L0 * L1 * XH * c8 + 2.0 * p->vol * es);
+        *flops = fft_flops(S * L0 * L1 / 2, p->log2p[2]); break;
+    default: break;
+    }
+    (void)L2;
+    return HYENAND_OK;
+}
+
+extern "C" int hyenand_plan_set_timing(hyenand_plan *p, int enable)
+{
+    g_err[0] = 0;
+    if (!p) return fail(HYENAND_ERR_INVALID_ARG, "plan is NULL");
+    p->prof.on = enable != 0;
+    p->prof.reset();
+    return HYENAND_OK;
+}
+
+extern "C" int hyenand_plan_kernel_time(hyenand_plan *p, int kid, double *total_ms, double *launches)
+{
+    g_err[0] = 0;
+    if (!p || kid < 0 || kid >= KID_COUNT || !total_ms || !launches) return fail(HYENAND_ERR_INVALID_ARG, "bad argument");
+    p->prof.collect();
+    *total_ms = p->prof.ms[kid];
+    *launches = (double)p->prof.launches[kid];
+    return HYENAND_OK;
 }

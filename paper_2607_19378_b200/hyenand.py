@@ -55,6 +55,12 @@ def lib() -> ctypes.CDLL:
         L.hyenand_plan_launches.argtypes = [vp, ctypes.c_int]
         L.hyenand_plan_path.argtypes = [vp]
         L.hyenand_plan_path.restype = ctypes.c_char_p
+        dpp = ctypes.POINTER(ctypes.c_double)
+        L.hyenand_plan_kernel_count.argtypes = [vp]
+        L.hyenand_plan_kernel_info.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_char_p),
+                                               dpp, dpp, dpp]
+        L.hyenand_plan_set_timing.argtypes = [vp, ctypes.c_int]
+        L.hyenand_plan_kernel_time.argtypes = [vp, ctypes.c_int, dpp, dpp]
         _lib = L
     return _lib
 
@@ -123,6 +129,30 @@ def hyenand_plan_launches(plan: int, h_shared: bool) -> int:
 
 def hyenand_plan_path(plan: int) -> str:
     return lib().hyenand_plan_path(plan).decode()
+
+
+def hyenand_plan_kernel_count(plan: int) -> int:
+    return int(lib().hyenand_plan_kernel_count(plan))
+
+
+def hyenand_plan_kernel_info(plan: int, kernel_id: int, h_shared: bool):
+    """(name, launches, algorithmic bytes, algorithmic flops) of one kernel, per forward."""
+    name = ctypes.c_char_p()
+    n, b, f = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    _check(lib().hyenand_plan_kernel_info(plan, kernel_id, 1 if h_shared else 0, ctypes.byref(name),
+                                          ctypes.byref(n), ctypes.byref(b), ctypes.byref(f)))
+    return name.value.decode(), n.value, b.value, f.value
+
+
+def hyenand_plan_set_timing(plan: int, enable: bool) -> None:
+    _check(lib().hyenand_plan_set_timing(plan, 1 if enable else 0))
+
+
+def hyenand_plan_kernel_time(plan: int, kernel_id: int):
+    """(accumulated device ms, recorded launches) since timing was switched on."""
+    ms, n = ctypes.c_double(), ctypes.c_double()
+    _check(lib().hyenand_plan_kernel_time(plan, kernel_id, ctypes.byref(ms), ctypes.byref(n)))
+    return ms.value, n.value
 
 
 class Plan:
