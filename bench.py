@@ -264,7 +264,7 @@ def main_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
-    w = W.WORKLOADS[args.workload]
+    w = W.WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
     if world > 1:
         from dataclasses import replace
         w = replace(w, seed=w.seed + 100 * rank)
@@ -346,7 +346,7 @@ def main_reference(args):
     if rank != 0:
         return
     import oracle
-    w = W.WORKLOADS[args.workload]
+    w = W.WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
     threads = oracle.threads()
     mode = "causal" if w.causal else "linear"
     S = w.B * w.C
@@ -389,6 +389,8 @@ if __name__ == "__main__":
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.WORKLOADS))
+    ap.add_argument("--batch", type=int, default=None, help="override B (profiling on a smaller case)")
+    ap.add_argument("--channels", type=int, default=None, help="override C (profiling on a smaller case)")
     ap.add_argument("--no-all", action="store_true", help="skip the table over the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     a = ap.parse_args()

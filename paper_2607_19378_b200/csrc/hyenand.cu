@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <vector>
@@ -10,6 +11,7 @@
 #include "../../include/hyenand.h"
 #include "common.cuh"
 #include "ct1d.cuh"
+#include "planes.cuh"
 
 using namespace hn;
 
@@ -26,7 +28,7 @@ static int fail(int code, const char *fmt, ...)
     return code;
 }
 
-enum Path { PATH_ND_GENERIC = 0, PATH_CT1D = 1 };
+enum Path { PATH_ND_GENERIC = 0, PATH_CT1D = 1, PATH_PLANES3D = 2 };
 
 struct hyenand_plan {
     int ndim, B, C, causal, dtype;
@@ -43,6 +45,7 @@ struct hyenand_plan {
     long long wh_slices;              // slices the filter workspace holds
     float2 *gtw;
     int gtw_n;
+    float2 *plane_scratch;
     // long 1-D path
     Ct1dPlan ct;
     // host-staging for hyenand_forward_host
@@ -83,7 +86,7 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
     int cur = 0;
     cudaGetDevice(&cur);
     if (cur != p->device) cudaSetDevice(p->device);
-    cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw);
+    cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw); cudaFree(p->plane_scratch);
     ct1d_free(&p->ct);
     for (int i = 0; i < 5; ++i) cudaFree(p->stage[i]);
     p->prof.destroy();
@@ -144,12 +147,21 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
 
     p->path = PATH_ND_GENERIC;
     const bool three = p->P[0] > 1;
-    p->ws_a_slice = (long long)p->L[0] * p->L[1] * p->XH;
-    p->wh_a_slice = (long long)p->K[0] * p->K[1] * p->XH;
-    p->ws_b_slice = three ? (long long)p->L[0] * p->P[1] * p->XH : 0;
-    p->wh_b_slice = three ? (long long)p->K[0] * p->P[1] * p->XH : 0;
+    if (three && p->log2p[1] == p->log2p[2] && plane_supported(p->log2p[2]) && !getenv("HYENAND_FORCE_GENERIC"))
+        p->path = PATH_PLANES3D;
+    if (p->path == PATH_PLANES3D) {
+        // spectra [plane][XH][P_y]; the z pass works in place on the k*v spectra
+        p->ws_a_slice = (long long)p->L[0] * p->XH * p->P[1];
+        p->wh_a_slice = (long long)p->K[0] * p->XH * p->P[1];
+        p->ws_b_slice = p->wh_b_slice = 0;
+    } else {
+        p->ws_a_slice = (long long)p->L[0] * p->L[1] * p->XH;
+        p->wh_a_slice = (long long)p->K[0] * p->K[1] * p->XH;
+        p->ws_b_slice = three ? (long long)p->L[0] * p->P[1] * p->XH : 0;
+        p->wh_b_slice = three ? (long long)p->K[0] * p->P[1] * p->XH : 0;
+    }
     const long long per_slice = p->ws_a_slice + p->ws_b_slice + p->wh_a_slice + p->wh_b_slice;
-    const long long budget = (3ll << 30) / (long long)sizeof(float2);      // 3 GiB of workspace
+    const long long budget = (8ll << 30) / (long long)sizeof(float2);      // 8 GiB of workspace
     long long spc = budget / per_slice;
     if (spc < 1) spc = 1;
     if (spc > S) spc = S;
@@ -166,9 +178,11 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     }
     int e = dev_alloc(p, (void **)&p->gtw, sizeof(float2) * p->gtw_n);
     if (!e) e = dev_alloc(p, (void **)&p->ws_a, sizeof(float2) * p->ws_a_slice * spc);
-    if (!e && three) e = dev_alloc(p, (void **)&p->ws_b, sizeof(float2) * p->ws_b_slice * spc);
+    if (!e && p->ws_b_slice) e = dev_alloc(p, (void **)&p->ws_b, sizeof(float2) * p->ws_b_slice * spc);
     if (!e) e = dev_alloc(p, (void **)&p->wh_a, sizeof(float2) * p->wh_a_slice * p->wh_slices);
-    if (!e && three) e = dev_alloc(p, (void **)&p->wh_b, sizeof(float2) * p->wh_b_slice * p->wh_slices);
+    if (!e && p->path == PATH_PLANES3D)
+        e = dev_alloc(p, (void **)&p->plane_scratch, sizeof(float2) * plane_scratch_elems(p->log2p[2]));
+    if (!e && p->wh_b_slice) e = dev_alloc(p, (void **)&p->wh_b, sizeof(float2) * p->wh_b_slice * p->wh_slices);
     if (!e && cudaMemcpy(p->gtw, tw.data(), sizeof(float2) * p->gtw_n, cudaMemcpyHostToDevice) != cudaSuccess)
         e = fail(HYENAND_ERR_CUDA, "twiddle upload failed: %s", cudaGetErrorString(cudaGetLastError()));
     if (e) { hyenand_destroy_plan(p); return nullptr; }
@@ -294,11 +308,69 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
     return 0;
 }
 
+static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const char *v, const char *h,
+                            bool shared, char *y, cudaStream_t st, int *launches)
+{
+    const long long S = (long long)p->B * p->C;
+    const size_t es = elsize(p->dtype);
+    const long long nc = (long long)p->XH * p->P[1];
+    auto filter = [&](const char *hp, long long n) -> int {
+        PlaneArgs a{};
+        a.a = hp; a.out = p->wh_a; a.scratch = p->plane_scratch; a.planes = n * p->K[0];
+        a.lx = p->L[2]; a.ly = p->L[1]; a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        p->prof.begin(KID_PLANE_H, st);
+        int c = launch_plane(a, PLANE_H, p->log2p[2], p->dtype, st);
+        p->prof.end(st);
+        if (c < 0) return -1;
+        *launches += c;
+        return 0;
+    };
+    if (shared && filter(h, p->C)) return -1;
+    for (long long s0 = 0; s0 < S; s0 += p->slices_per_chunk) {
+        const long long n = S - s0 < p->slices_per_chunk ? S - s0 : p->slices_per_chunk;
+        if (!shared && filter(h + (size_t)s0 * p->kvol * es, n)) return -1;
+        PlaneArgs u{};
+        u.a = k + (size_t)s0 * p->vol * es; u.b = v + (size_t)s0 * p->vol * es; u.out = p->ws_a;
+        u.planes = n * p->L[0]; u.lx = p->L[2]; u.ly = p->L[1]; u.gtw = p->gtw; u.gtw_n = p->gtw_n;
+        p->prof.begin(KID_PLANE_U, st);
+        int c = launch_plane(u, PLANE_U, p->log2p[2], p->dtype, st);
+        p->prof.end(st);
+        if (c < 0) return -1;
+        *launches += c;
+        AxisArgs a{};
+        a.in = p->ws_a; a.out = p->ws_a;
+        a.n_outer = n; a.in_outer = a.out_outer = (long long)p->L[0] * nc;
+        a.nc = (int)nc; a.n_in = p->L[0]; a.n_out = p->L[0]; a.shift = 0;
+        a.log2p = p->log2p[0]; a.prune_in = 1;
+        a.h = p->wh_a; a.h_outer = (long long)p->K[0] * nc; a.h_n_in = p->K[0]; a.h_shift = p->L[0] - 1;
+        a.h_mod = shared ? p->C : 0; a.h_off = shared ? s0 % p->C : 0;
+        a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
+        a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        p->prof.begin(KID_CORE, st);
+        c = launch_axis(a, AXIS_CORE, st);
+        p->prof.end(st);
+        if (c < 0) return -1;
+        *launches += c;
+        PlaneArgs iv{};
+        iv.a = q + (size_t)s0 * p->vol * es; iv.y = y + (size_t)s0 * p->vol * es; iv.in = p->ws_a;
+        iv.planes = n * p->L[0]; iv.lx = p->L[2]; iv.ly = p->L[1]; iv.gtw = p->gtw; iv.gtw_n = p->gtw_n;
+        p->prof.begin(KID_PLANE_INV, st);
+        c = launch_plane(iv, PLANE_INV, p->log2p[2], p->dtype, st);
+        p->prof.end(st);
+        if (c < 0) return -1;
+        *launches += c;
+    }
+    return 0;
+}
+
 static int run_forward(hyenand_plan *p, const void *q, const void *k, const void *v, const void *h,
                        bool shared, void *y, cudaStream_t st, int *launches)
 {
     int rc;
-    if (p->path == PATH_CT1D)
+    if (p->path == PATH_PLANES3D)
+        rc = forward_planes3d(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
+                              (char *)y, st, launches);
+    else if (p->path == PATH_CT1D)
         rc = ct1d_forward(&p->ct, q, k, v, h, shared, y, st, launches, &p->prof);
     else
         rc = forward_generic(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
@@ -403,6 +475,7 @@ extern "C" int hyenand_plan_launches(const hyenand_plan *p, int h_shared)
     const long long S = (long long)p->B * p->C;
     const long long chunks = (S + p->slices_per_chunk - 1) / p->slices_per_chunk;
     const int three = p->P[0] > 1;
+    if (p->path == PATH_PLANES3D) return (int)(h_shared ? 1 + chunks * 3 : chunks * 4);
     const int filt = 1 + three, body = 3 + 2 * three;
     return (int)(h_shared ? filt + chunks * body : chunks * (filt + body));
 }
@@ -410,14 +483,14 @@ extern "C" int hyenand_plan_launches(const hyenand_plan *p, int h_shared)
 extern "C" const char *hyenand_plan_path(const hyenand_plan *p)
 {
     if (!p) return "";
-    return p->path == PATH_CT1D ? "ct1d" : "nd_generic";
+    return p->path == PATH_CT1D ? "ct1d" : p->path == PATH_PLANES3D ? "planes3d" : "nd_generic";
 }
 
 // ---- per-kernel accounting (reporting only) ---------------------------------------------
 
 static const char *kKernelNames[KID_COUNT] = {
     "rows_fwd(h)", "axis_fwd(h)", "rows_fwd(k*v)", "axis_fwd(k*v)", "axis_core", "axis_inv", "rows_inv",
-    "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv"};
+    "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv", "plane_fwd(h)", "plane_fwd(k*v)", "plane_inv"};
 
 static double fft_flops(double lines, int log2n) { return lines * 5.0 * ldexp(1.0, log2n) * log2n; }
 
@@ -456,6 +529,26 @@ extern "C" int hyenand_plan_kernel_info(const hyenand_plan *p, int kid, int h_sh
     }
     const bool three = p->P[0] > 1;
     const double chunks = ceil(S / (double)p->slices_per_chunk);
+    if (p->path == PATH_PLANES3D) {
+        const double PY = p->P[1], nc = (double)p->XH * PY, Lz = p->L[0], Kz = p->K[0];
+        const double rowsU = p->L[1] / 2.0, colsU = PY / 2.0;
+        switch (kid) {
+        case KID_PLANE_H:
+            *launches = h_shared ? 1 : chunks; *bytes = Sh * ((double)p->kvol * es + Kz * nc * c8);
+            *flops = fft_flops(Sh * Kz * PY / 2.0, p->log2p[2]) + fft_flops(Sh * Kz * p->P[2] / 2.0, p->log2p[1]); break;
+        case KID_PLANE_U:
+            *launches = chunks; *bytes = S * (2.0 * p->vol * es + Lz * nc * c8);
+            *flops = fft_flops(S * Lz * rowsU, p->log2p[2]) + fft_flops(S * Lz * colsU, p->log2p[1]); break;
+        case KID_CORE:
+            *launches = chunks; *bytes = S * nc * c8 * (2.0 * Lz + Kz);
+            *flops = 3 * fft_flops(S * nc, p->log2p[0]) + 12.0 * S * nc * p->P[0]; break;
+        case KID_PLANE_INV:
+            *launches = chunks; *bytes = S * (Lz * nc * c8 + 2.0 * p->vol * es);
+            *flops = fft_flops(S * Lz * rowsU, p->log2p[2]) + fft_flops(S * Lz * colsU, p->log2p[1]); break;
+        default: break;
+        }
+        return HYENAND_OK;
+    }
     const double XH = p->XH, L0 = p->L[0], L1 = p->L[1], L2 = p->L[2], K0 = p->K[0], K1 = p->K[1], P1 = p->P[1];
     const int ax = three ? 0 : 1;
     const double inner = three ? P1 * XH : XH;

@@ -1,0 +1,363 @@
+// Plane-fused kernels for 3-D grids (and the building blocks of the fused 2-D path).
+//
+// One CTA transforms a whole x-y plane on chip, so the two in-plane axes cost
+// one trip through HBM instead of two (the paper's nSubQ keeps intermediates in
+// shared memory the same way for 1-D and 2-D; it describes no 3-D kernel):
+//
+//   uplane     k*v plane: gate, zero-pad, real-to-complex along x (two real rows
+//              per complex transform), transpose through a shared-memory column
+//              store, complex transform along y.  Output lines are [kx][ky].
+//   hplane     filter plane, which has twice the rows: handled as the rows at even
+//              and at odd padded positions (two half planes of the size of a k*v
+//              plane) joined by one radix-2 step; the first half's spectrum waits
+//              in a per-CTA global scratch that stays in L2.
+//   plane_inv  inverse along y (keeping the cropped rows), inverse complex-to-real
+//              along x, crop, output gate q, store.
+//
+// Column 0 of the column store carries the two purely real bins of every row (kx = 0 and
+// kx = P/2) as one complex number, so a plane has exactly P/2 columns.
+#include "common.cuh"
+#include "planes.cuh"
+#include "wfft.cuh"
+
+namespace hn {
+
+constexpr int kPlaneThreads = 512;
+
+template <int LOG2P> struct PlaneCfg {
+    static constexpr int P = 1 << LOG2P, HP = P / 2, XH = HP + 1;
+    static constexpr int CSS = HP + 1;                       // column-store stride (odd)
+    using F = WF<LOG2P, false>;
+    using FI = WF<LOG2P, true>;
+    using FH = WF<LOG2P - 1, false>;                         // half-length columns of hplane
+    static constexpr int NG = kPlaneThreads / F::TPL;        // groups working on P-point lines
+    static constexpr int NGH = kPlaneThreads / FH::TPL;      // groups working on P/2-point lines
+    static constexpr int LS = line_stride(P);
+    static constexpr int LSH = line_stride(HP);
+    static constexpr int WBUF = (NG * LS > NGH * LSH) ? NG * LS : NGH * LSH;
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * CSS + WBUF + HP + HP / 2);
+};
+
+// Separate the spectra of the two real rows packed in one complex transform (results in
+// `line`, natural order) and scatter them into column store rows y0, y1.
+template <int LOG2P>
+__device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, int y0, int y1, int l)
+{
+    using C = PlaneCfg<LOG2P>;
+    constexpr int P = C::P, HP = C::HP, TPL = C::F::TPL;
+    float a0 = 0.f, b0 = 0.f;
+    for (int kx = l; kx <= HP; kx += TPL) {
+        const float2 z1 = line[phys(kx)];
+        const float2 z2 = line[phys((P - kx) & (P - 1))];
+        const float2 A = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
+        const float2 B = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
+        if (kx == 0) { a0 = A.x; b0 = B.x; }
+        else if (kx == HP) {                                 // same lane as kx == 0
+            cs[y0] = make_float2(a0, A.x);
+            cs[y1] = make_float2(b0, B.x);
+        } else {
+            cs[kx * C::CSS + y0] = A;
+            cs[kx * C::CSS + y1] = B;
+        }
+    }
+}
+
+template <int LOG2P> __device__ __forceinline__ void load_plane_twiddles(float2 *tw, float2 *twh, const float2 *gtw, int gtw_n, int tid)
+{
+    constexpr int HP = 1 << (LOG2P - 1);
+    const int step = gtw_n >> LOG2P;
+    for (int t = tid; t < HP; t += kPlaneThreads) tw[t] = gtw[t * step];
+    for (int t = tid; t < HP / 2; t += kPlaneThreads) twh[t] = gtw[2 * t * step];
+}
+
+// ---- k*v planes ---------------------------------------------------------------------------------
+
+template <typename T, int LOG2P>
+__global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
+{
+    using C = PlaneCfg<LOG2P>;
+    using F = typename C::F;
+    constexpr int P = C::P, HP = C::HP, TPL = F::TPL;
+    extern __shared__ float2 smem[];
+    float2 *cs = smem;
+    float2 *wbuf = cs + HP * C::CSS;
+    float2 *tw = wbuf + C::WBUF;
+    float2 *twh = tw + HP;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = F::group_mask(tid);
+    float2 *line = wbuf + gid * C::LS;
+    load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
+    __syncthreads();
+    const T *pk = (const T *)p.a;
+    const T *pv = (const T *)p.b;
+    const int Lx = p.lx, Ly = p.ly;
+    for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
+        const long long ib = pl * (long long)Ly * Lx;
+        for (int rp = gid; 2 * rp < HP; rp += C::NG) {
+            const int y0 = 2 * rp, y1 = y0 + 1;
+            if (y0 < Ly) {
+                const bool has1 = y1 < Ly;
+                const long long o0 = ib + (long long)y0 * Lx, o1 = o0 + Lx;
+                F::template run_to_line<PRUNE_IN>(l, m, tw, line, [&](int, int, int idx) {
+                    float a = 0.f, b = 0.f;
+                    if (idx < Lx) {
+                        a = IO<T>::ld(pk, o0 + idx) * IO<T>::ld(pv, o0 + idx);
+                        if (has1) b = IO<T>::ld(pk, o1 + idx) * IO<T>::ld(pv, o1 + idx);
+                    }
+                    return make_float2(a, b);
+                });
+                separate_rows<LOG2P>(line, cs, y0, y1, l);
+                __syncwarp(m);
+            }
+        }
+        __syncthreads();
+        float2 *dst = p.out + pl * (long long)C::XH * P;
+        for (int kx = gid; kx < HP; kx += C::NG) {
+            const float2 *col = cs + kx * C::CSS;
+            if (kx != 0) {
+                float2 *d = dst + (long long)kx * P;
+                F::template run<PRUNE_IN>(l, m, tw, line,
+                    [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); },
+                    [&](int, int, int idx, float2 v) { d[idx] = v; });
+            } else {
+                F::template run_to_line<PRUNE_IN>(l, m, tw, line,
+                    [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); });
+                for (int ky = l; ky < P; ky += TPL) {
+                    const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
+                    dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
+                    dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
+                }
+            }
+            __syncwarp(m);
+        }
+        __syncthreads();
+    }
+}
+
+// ---- filter planes ----------------------------------------------------------------------------------
+
+template <typename T, int LOG2P>
+__global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
+{
+    using C = PlaneCfg<LOG2P>;
+    using F = typename C::F;
+    using FH = typename C::FH;
+    constexpr int P = C::P, HP = C::HP, TPL = F::TPL, TPLH = FH::TPL;
+    extern __shared__ float2 smem[];
+    float2 *cs = smem;
+    float2 *wbuf = cs + HP * C::CSS;
+    float2 *tw = wbuf + C::WBUF;
+    float2 *twh = tw + HP;
+    const int tid = threadIdx.x;
+    const int l = tid % TPL, gid = tid / TPL;
+    const int lh = tid % TPLH, gidh = tid / TPLH;
+    const unsigned m = F::group_mask(tid), mh = FH::group_mask(tid);
+    float2 *line = wbuf + gid * C::LS;
+    float2 *lineh = wbuf + gidh * C::LSH;
+    load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
+    __syncthreads();
+    const T *ph = (const T *)p.a;
+    const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
+    float2 *scratch = p.scratch + (long long)blockIdx.x * C::XH * HP;     // E[kx][ky'], XH lines
+    for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
+        const long long ib = pl * (long long)Ky * Kx;
+        float2 *dst = p.out + pl * (long long)C::XH * P;
+        for (int e = 0; e < 2; ++e) {
+            // rows at padded positions yp = 2*yy + e, i.e. taps my = (yp + Ly - 1) mod P
+            for (int rp = gid; 2 * rp < HP; rp += C::NG) {
+                const int yy0 = 2 * rp, yy1 = yy0 + 1;
+                const int my0 = (2 * yy0 + e + Ly - 1) & (P - 1), my1 = (2 * yy1 + e + Ly - 1) & (P - 1);
+                const bool v0 = my0 < Ky, v1 = my1 < Ky;
+                const long long o0 = ib + (long long)my0 * Kx, o1 = ib + (long long)my1 * Kx;
+                if (v0 || v1) {
+                    F::template run_to_line<PRUNE_NONE>(l, m, tw, line, [&](int, int, int idx) {
+                        const int mx = (idx + Lx - 1) & (P - 1);
+                        float a = 0.f, b = 0.f;
+                        if (mx < Kx) {
+                            if (v0) a = IO<T>::ld(ph, o0 + mx);
+                            if (v1) b = IO<T>::ld(ph, o1 + mx);
+                        }
+                        return make_float2(a, b);
+                    });
+                    separate_rows<LOG2P>(line, cs, yy0, yy1, l);
+                    __syncwarp(m);
+                } else {
+                    for (int kx = l; kx < HP; kx += TPL) {
+                        cs[kx * C::CSS + yy0] = make_float2(0.f, 0.f);
+                        cs[kx * C::CSS + yy1] = make_float2(0.f, 0.f);
+                    }
+                }
+            }
+            __syncthreads();
+            // columns: HP-point transforms over yy
+            for (int kx = gidh; kx < HP; kx += C::NGH) {
+                const float2 *col = cs + kx * C::CSS;
+                if (kx != 0) {
+                    if (e == 0) {
+                        float2 *d = scratch + (long long)kx * HP;
+                        FH::template run<PRUNE_NONE>(lh, mh, twh, lineh,
+                            [&](int, int, int idx) { return col[idx]; },
+                            [&](int, int, int idx, float2 v) { d[idx] = v; });
+                    } else {
+                        const float2 *es = scratch + (long long)kx * HP;
+                        float2 *d = dst + (long long)kx * P;
+                        FH::template run<PRUNE_NONE>(lh, mh, twh, lineh,
+                            [&](int, int, int idx) { return col[idx]; },
+                            [&](int, int, int idx, float2 v) {
+                                const float2 E = es[idx];
+                                const float2 t = cmul(v, tw[idx]);            // W_P^ky' * O
+                                d[idx] = cadd(E, t);
+                                d[idx + HP] = csub(E, t);
+                            });
+                    }
+                } else {
+                    FH::template run_to_line<PRUNE_NONE>(lh, mh, twh, lineh,
+                        [&](int, int, int idx) { return col[idx]; });
+                    for (int ky = lh; ky < HP; ky += TPLH) {
+                        const float2 c1 = lineh[phys(ky)], c2 = lineh[phys((HP - ky) & (HP - 1))];
+                        const float2 s0 = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));   // bin kx = 0
+                        const float2 sn = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));   // bin kx = P/2
+                        if (e == 0) {
+                            scratch[ky] = s0;
+                            scratch[(long long)HP * HP + ky] = sn;
+                        } else {
+                            const float2 w = tw[ky];
+                            const float2 E0 = scratch[ky], EN = scratch[(long long)HP * HP + ky];
+                            const float2 t0 = cmul(s0, w), tn = cmul(sn, w);
+                            dst[ky] = cadd(E0, t0);
+                            dst[ky + HP] = csub(E0, t0);
+                            dst[(long long)HP * P + ky] = cadd(EN, tn);
+                            dst[(long long)HP * P + ky + HP] = csub(EN, tn);
+                        }
+                    }
+                }
+                __syncwarp(mh);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// ---- inverse planes ------------------------------------------------------------------------------------
+
+template <typename T, int LOG2P>
+__global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p)
+{
+    using C = PlaneCfg<LOG2P>;
+    using FI = typename C::FI;
+    constexpr int P = C::P, HP = C::HP, TPL = FI::TPL;
+    extern __shared__ float2 smem[];
+    float2 *cs = smem;
+    float2 *wbuf = cs + HP * C::CSS;
+    float2 *tw = wbuf + C::WBUF;
+    float2 *twh = tw + HP;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = FI::group_mask(tid);
+    float2 *line = wbuf + gid * C::LS;
+    load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
+    __syncthreads();
+    const T *pq = (const T *)p.a;
+    T *py = (T *)p.y;
+    const int Lx = p.lx, Ly = p.ly;
+    for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
+        const float2 *src = p.in + pl * (long long)C::XH * P;
+        for (int kx = gid; kx < HP; kx += C::NG) {
+            float2 *col = cs + kx * C::CSS;
+            if (kx != 0) {
+                const float2 *s = src + (long long)kx * P;
+                FI::template run<PRUNE_OUT>(l, m, tw, line,
+                    [&](int, int, int idx) { return s[idx]; },
+                    [&](int, int, int idx, float2 v) { col[idx] = v; });
+            } else {
+                const float2 *sn = src + (long long)HP * P;
+                FI::template run<PRUNE_OUT>(l, m, tw, line,
+                    [&](int, int, int idx) {
+                        const float2 g0 = src[idx], gn = sn[idx];
+                        return make_float2(g0.x - gn.y, g0.y + gn.x);
+                    },
+                    [&](int, int, int idx, float2 v) { col[idx] = v; });
+            }
+            __syncwarp(m);
+        }
+        __syncthreads();
+        const long long ob = pl * (long long)Ly * Lx;
+        for (int rp = gid; 2 * rp < Ly; rp += C::NG) {
+            const int y0 = 2 * rp, y1 = y0 + 1;
+            const bool has1 = y1 < Ly;
+            const long long o0 = ob + (long long)y0 * Lx, o1 = o0 + Lx;
+            FI::template run<PRUNE_OUT>(l, m, tw, line,
+                [&](int, int, int idx) {
+                    const int kx = idx <= HP ? idx : P - idx;
+                    if (kx == 0 || kx == HP) {
+                        const float2 A = cs[y0];
+                        const float2 B = has1 ? cs[y1] : make_float2(0.f, 0.f);
+                        return kx == 0 ? make_float2(A.x, B.x) : make_float2(A.y, B.y);
+                    }
+                    const float2 A = cs[kx * C::CSS + y0];
+                    const float2 B = has1 ? cs[kx * C::CSS + y1] : make_float2(0.f, 0.f);
+                    return idx <= HP ? make_float2(A.x - B.y, A.y + B.x) : make_float2(A.x + B.y, B.x - A.y);
+                },
+                [&](int, int, int idx, float2 v) {
+                    if (idx < Lx) {
+                        IO<T>::st(py, o0 + idx, v.x * IO<T>::ld(pq, o0 + idx));
+                        if (has1) IO<T>::st(py, o1 + idx, v.y * IO<T>::ld(pq, o1 + idx));
+                    }
+                });
+            __syncwarp(m);
+        }
+        __syncthreads();
+    }
+}
+
+// ---- launchers --------------------------------------------------------------------------------------------
+
+static int plane_sms()
+{
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+int plane_grid(long long planes)
+{
+    const int s = plane_sms();
+    return (int)(planes < s ? planes : s);
+}
+
+size_t plane_scratch_elems(int log2p)
+{
+    const size_t hp = (size_t)1 << (log2p - 1);
+    return (size_t)plane_sms() * (hp + 1) * hp;
+}
+
+template <typename T, int LOG2P> static int launch_plane_t(const PlaneArgs &a, int which, cudaStream_t st)
+{
+    using C = PlaneCfg<LOG2P>;
+    const int grid = plane_grid(a.planes);
+    if (grid <= 0) return 0;
+    static bool attr[3] = {false, false, false};
+    void (*fn)(PlaneArgs) = which == PLANE_U ? uplane_kernel<T, LOG2P>
+                          : which == PLANE_H ? hplane_kernel<T, LOG2P> : plane_inv_kernel<T, LOG2P>;
+    if (!attr[which]) {
+        cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+        attr[which] = true;
+    }
+    fn<<<grid, kPlaneThreads, C::SMEM, st>>>(a);
+    return 1;
+}
+
+int launch_plane(const PlaneArgs &a, int which, int log2p, int dtype, cudaStream_t st)
+{
+    if (log2p == 8) return dtype == 0 ? launch_plane_t<float, 8>(a, which, st) : launch_plane_t<bf16, 8>(a, which, st);
+    if (log2p == 7) return dtype == 0 ? launch_plane_t<float, 7>(a, which, st) : launch_plane_t<bf16, 7>(a, which, st);
+    return -1;
+}
+
+bool plane_supported(int log2p) { return log2p == 7 || log2p == 8; }
+
+}  // namespace hn

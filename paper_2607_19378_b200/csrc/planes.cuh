@@ -1,0 +1,27 @@
+// Plane-fused kernels (planes.cu): interface used by the scheduler.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+namespace hn {
+
+enum PlaneKind { PLANE_U = 0, PLANE_H = 1, PLANE_INV = 2 };
+
+struct PlaneArgs {
+    const void *a;        // k (PLANE_U), h (PLANE_H), q (PLANE_INV)
+    const void *b;        // v (PLANE_U)
+    float2 *out;          // spectra [plane][P/2+1][P] written by PLANE_U / PLANE_H
+    const float2 *in;     // spectra read by PLANE_INV
+    void *y;              // output of PLANE_INV
+    float2 *scratch;      // PLANE_H: plane_scratch_elems() float2
+    long long planes;     // number of x-y planes
+    int lx, ly;           // grid extent along x (contiguous) and y
+    const float2 *gtw;    // global twiddle table with gtw_n >= P points
+    int gtw_n;
+};
+
+bool plane_supported(int log2p);
+size_t plane_scratch_elems(int log2p);
+int launch_plane(const PlaneArgs &a, int which, int log2p, int dtype, cudaStream_t st);
+
+}  // namespace hn

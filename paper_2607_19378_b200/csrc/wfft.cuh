@@ -1,0 +1,150 @@
+// Warp-local FFT engine: a group of TPL lanes (TPL <= 32) of one warp owns one
+// line of N = 2^LOG2N complex points.  Each Stockham pass keeps R points per
+// item in registers; passes are joined through a private shared-memory line
+// and separated by __syncwarp() over the group's lanes only, so warps never wait for the rest of the
+// CTA while transforming.  Inputs of the first pass and outputs of the last
+// pass go through caller-supplied functors, which lets the callers read
+// straight from global memory, zero-pad, gate, transpose, multiply spectra or
+// chain a forward transform into an inverse one without extra round trips.
+//
+// The inverse uses the reversed radix sequence of the forward transform: the
+// last forward pass then leaves, in each lane, exactly the points that lane
+// needs for the first inverse pass (positions j + r*N/R), so the spectral
+// product (Eq. 12 of the paper) happens in registers.
+#pragma once
+#include "fft_engine.cuh"
+
+namespace hn {
+
+template <int LOG2N> struct WPlan;
+template <> struct WPlan<5>  { static constexpr int NP = 2, TPL = 4;  static constexpr int R[3] = {8, 4, 1}; };
+template <> struct WPlan<6>  { static constexpr int NP = 2, TPL = 8;  static constexpr int R[3] = {8, 8, 1}; };
+template <> struct WPlan<7>  { static constexpr int NP = 2, TPL = 8;  static constexpr int R[3] = {8, 16, 1}; };
+template <> struct WPlan<8>  { static constexpr int NP = 2, TPL = 16; static constexpr int R[3] = {16, 16, 1}; };
+template <> struct WPlan<9>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 8}; };
+template <> struct WPlan<10> { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 16}; };
+
+template <int LOG2N, bool INV> struct WF {
+    using P = WPlan<LOG2N>;
+    static constexpr int N = 1 << LOG2N;
+    static constexpr int NP = P::NP;
+    static constexpr int TPL = P::TPL;
+    static constexpr int LPW = 32 / TPL;                  // lines per warp
+    // mask of the lanes that share a line with this thread (argument `m` of the functions below)
+    static __device__ __forceinline__ unsigned group_mask(int tid)
+    {
+        return TPL == 32 ? 0xffffffffu : (((1u << TPL) - 1u) << ((tid & 31) / TPL * TPL));
+    }
+    __host__ __device__ static constexpr int radix(int s) { return INV ? P::R[NP - 1 - s] : P::R[s]; }
+    __host__ __device__ static constexpr int ns(int s)
+    {
+        int n = 1;
+        for (int i = 0; i < s; ++i) n *= radix(i);
+        return n;
+    }
+    template <int S> struct Pass {
+        static constexpr int R = radix(S);
+        static constexpr int NS = ns(S);
+        static constexpr int ITEMS = N / R;
+        static constexpr int IPL = ITEMS >= TPL ? ITEMS / TPL : 1;   // items per lane
+        static constexpr bool PARTIAL = ITEMS < TPL;                 // only lanes < ITEMS work
+    };
+
+    // One pass.  in(i, r, idx) -> float2 gives the point at position idx (item i of this
+    // lane, leg r); out(i, r, idx, v) receives the result for position idx.
+    // PR: PRUNE_IN (first pass only: positions >= N/2 are zero and never requested),
+    //     PRUNE_OUT (last pass only: positions >= N/2 are not produced).
+    // tw: shared-memory table tw[t] = exp(-2 pi i t / N), t < N/2.
+    template <int S, int PR, class In, class Out>
+    static __device__ __forceinline__ void pass(int l, const float2 *tw, In in, Out out)
+    {
+        using PS = Pass<S>;
+        constexpr int R = PS::R, NS = PS::NS;
+        constexpr int NIN = (PR == PRUNE_IN) ? R / 2 : R;
+        constexpr int NOUT = (PR == PRUNE_OUT) ? R / 2 : R;
+        if (PS::PARTIAL && l >= PS::ITEMS) return;
+#pragma unroll
+        for (int i = 0; i < PS::IPL; ++i) {
+            const int j = l + i * TPL;
+            float2 x[R];
+#pragma unroll
+            for (int r = 0; r < NIN; ++r) x[r] = in(i, r, j + r * (N / R));
+#pragma unroll
+            for (int r = NIN; r < R; ++r) x[r] = make_float2(0.f, 0.f);
+            if constexpr (NS > 1) {
+                const int k = j & (NS - 1);
+#pragma unroll
+                for (int r = 1; r < NIN; ++r) x[r] = cmul(x[r], twiddle<N, INV>(tw, r * k * (N / (NS * R))));
+            }
+            dft<R, INV, PR>(x);
+            const int k = j & (NS - 1);
+            const int base = (j - k) * R + k;
+#pragma unroll
+            for (int r = 0; r < NOUT; ++r) out(i, r, base + r * NS, x[r]);
+        }
+    }
+
+    // Middle of a transform: passes [S0, S1) line -> line, each followed by __syncwarp().
+    template <int S0, int S1>
+    static __device__ __forceinline__ void mid(int l, unsigned m, const float2 *tw, float2 *line)
+    {
+        if constexpr (S0 < S1) {
+            // loads of all items must precede the stores of any item of the same line
+            using PS = Pass<S0>;
+            constexpr int R = PS::R;
+            float2 keep[PS::IPL][R];
+            pass<S0, PRUNE_NONE>(l, tw,
+                [&](int, int, int idx) { return line[phys(idx)]; },
+                [&](int i, int r, int, float2 v) { keep[i][r] = v; });
+            __syncwarp(m);
+            if (!(PS::PARTIAL && l >= PS::ITEMS)) {
+#pragma unroll
+                for (int i = 0; i < PS::IPL; ++i) {
+                    const int j = l + i * TPL;
+                    const int k = j & (PS::NS - 1);
+                    const int base = (j - k) * R + k;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) line[phys(base + r * PS::NS)] = keep[i][r];
+                }
+            }
+            __syncwarp(m);
+            mid<S0 + 1, S1>(l, m, tw, line);
+        }
+    }
+
+    // Full transform: first-pass inputs from `in`, last-pass outputs to `out`; the line is
+    // scratch.  Callers must __syncwarp() before reusing the line for something else.
+    template <int PR, class In, class Out>
+    static __device__ __forceinline__ void run(int l, unsigned m, const float2 *tw, float2 *line, In in, Out out)
+    {
+        constexpr int PF = (PR == PRUNE_IN) ? PRUNE_IN : PRUNE_NONE;
+        constexpr int PL = (PR == PRUNE_OUT) ? PRUNE_OUT : PRUNE_NONE;
+        pass<0, PF>(l, tw, in, [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+        __syncwarp(m);
+        mid<1, NP - 1>(l, m, tw, line);
+        pass<NP - 1, PL>(l, tw, [&](int, int, int idx) { return line[phys(idx)]; }, out);
+    }
+
+    // Full transform whose results end up in the line itself (natural order); ends with a
+    // __syncwarp(), so every lane of the group may read any position afterwards.
+    template <int PR, class In>
+    static __device__ __forceinline__ void run_to_line(int l, unsigned m, const float2 *tw, float2 *line, In in)
+    {
+        using PS = Pass<NP - 1>;
+        float2 keep[PS::IPL][PS::R];
+        run<PR>(l, m, tw, line, in, [&](int i, int r, int, float2 v) { keep[i][r] = v; });
+        __syncwarp(m);
+        if (!(PS::PARTIAL && l >= PS::ITEMS)) {
+            constexpr int NOUT = (PR == PRUNE_OUT) ? PS::R / 2 : PS::R;
+#pragma unroll
+            for (int i = 0; i < PS::IPL; ++i) {
+                const int j = l + i * TPL;
+#pragma unroll
+                for (int r = 0; r < NOUT; ++r) line[phys(j + r * (N / PS::R))] = keep[i][r];
+            }
+        }
+        __syncwarp(m);
+    }
+};
+
+}  // namespace hn

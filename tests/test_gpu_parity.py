@@ -78,6 +78,30 @@ def test_causal_1d(L, dtype, shared):
     check(w, q, k, v, h, full_direct=L <= 1000)
 
 
+PLANE_SHAPES = [(3, 40, 50), (2, 64, 64), (3, 33, 64), (2, 65, 128), (4, 128, 100), (1, 128, 128), (5, 1, 70)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dims", PLANE_SHAPES, ids=str)
+def test_plane_fused_3d_path(dims, dtype):
+    """3-D grids whose two inner padded axes are 128 or 256 take the plane-fused kernels."""
+    w, (q, k, v, h) = W.random_problem(dims, B=1, C=2, dtype=dtype, seed=21)
+    from paper_2607_19378_b200 import hyenand as hn
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    path = hn.hyenand_plan_path(plan.handle)
+    plan.close()
+    if dims[1] == 1:
+        assert path == "nd_generic"
+    elif dims[0] > 1:
+        assert path == "planes3d"
+    check(w, q, k, v, h)
+
+
+def test_plane_fused_3d_shared_filter():
+    w, (q, k, v, h) = W.random_problem((3, 40, 50), B=3, C=2, dtype="f32", h_shared=True, seed=22)
+    check(w, q, k, v, h)
+
+
 def test_tiny2d_workload_full():
     w = W.WORKLOADS["tiny2d"]
     q, k, v, h = W.make_inputs(w)
