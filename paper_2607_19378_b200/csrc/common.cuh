@@ -142,4 +142,8 @@ int launch_rows_fwd(const RowsArgs &a, int dtype, cudaStream_t st);
 int launch_rows_inv(const RowsInvArgs &a, int dtype, cudaStream_t st);
 int launch_axis(const AxisArgs &a, int mode, cudaStream_t st);
 
+// warp-engine version of AXIS_CORE (core_w.cu); needs n_in <= P/2, h_n_in <= P, n_out <= P/2
+bool core_w_supported(int log2p);
+int launch_core_w(const AxisArgs &a, cudaStream_t st);
+
 }  // namespace hn

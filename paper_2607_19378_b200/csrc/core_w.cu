@@ -1,0 +1,187 @@
+// Fused spectral core along a strided axis, warp-engine version.
+//
+// For a tile of adjacent bins the CTA loads the k*v lines and the filter lines
+// (coalesced rows, transposed into shared-memory lines), and each group of lanes
+// then owns one line: forward transform of the filter line into registers,
+// forward transform of the k*v line into registers, spectral product (Eq. 12 of
+// the paper), and the inverse transform started from those registers.  Only the
+// cropped half of the inverse is produced and written back in place.
+#include "common.cuh"
+#include "wfft.cuh"
+
+namespace hn {
+
+constexpr int kCoreThreads = 256;
+
+__device__ __forceinline__ void cp_async8(void *smem_dst, const void *gmem_src)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+template <int LOG2P>
+__global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core_w_kernel(AxisArgs p)
+{
+    using F = WF<LOG2P, false>;
+    using FI = WF<LOG2P, true>;
+    constexpr int N = 1 << LOG2P, TPL = F::TPL, NP = F::NP;
+    constexpr int TX = kCoreThreads / TPL;                 // lines per tile
+    constexpr int LS = line_stride(N);
+    using PL = typename F::template Pass<NP - 1>;          // last forward pass == first inverse pass
+    extern __shared__ float2 smem[];
+    float2 *bu = smem;
+    float2 *bh = smem + TX * LS;
+    float2 *tw = smem + 2 * TX * LS;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = F::group_mask(tid);
+    float2 *uline = bu + gid * LS;
+    float2 *hline = bh + gid * LS;
+    load_twiddles(tw, p.gtw, N, p.gtw_n, tid, kCoreThreads);
+    const long long tpo = (p.nc + TX - 1) / TX;
+    const long long tiles = p.n_outer * tpo;
+    // Tile loads are asynchronous copies (one complex bin per thread and row) straight into the
+    // lines; the filter lines of the next tile are fetched while this tile's k*v lines are
+    // transformed, and the next k*v lines while the next filter lines are transformed.
+    constexpr int RPS = kCoreThreads / TX;                 // rows per step
+    const int x = tid % TX, r0 = tid / TX;
+    auto issue_h = [&](long long t) {
+        const long long o = t / tpo;
+        const int c0 = (int)(t % tpo) * TX;
+        const long long oh = p.h_mod ? (o + p.h_off) % p.h_mod : o;
+        const float2 *hs = p.h + oh * p.h_outer + c0 + x;
+        const bool inside = c0 + x < p.nc;
+#pragma unroll 4
+        for (int pos = r0; pos < N; pos += RPS) {
+            const int mm = (pos + p.h_shift) & (N - 1);
+            float2 *d = bh + x * LS + phys(pos);
+            if (inside && mm < p.h_n_in) cp_async8(d, hs + (long long)mm * p.nc);
+            else *d = make_float2(0.f, 0.f);
+        }
+    };
+    auto issue_u = [&](long long t) {
+        const long long o = t / tpo;
+        const int c0 = (int)(t % tpo) * TX;
+        const float2 *us = p.in + o * p.in_outer + c0 + x;
+        const bool inside = c0 + x < p.nc;
+#pragma unroll 4
+        for (int pos = r0; pos < N / 2; pos += RPS) {
+            float2 *d = bu + x * LS + phys(pos);
+            if (inside && pos < p.n_in) cp_async8(d, us + (long long)pos * p.nc);
+            else *d = make_float2(0.f, 0.f);
+        }
+    };
+    long long t = blockIdx.x;
+    if (t < tiles) { issue_h(t); }
+    cp_async_commit();
+    if (t < tiles) { issue_u(t); }
+    cp_async_commit();
+    while (t < tiles) {
+        const long long tn = t + gridDim.x;
+        using PL2 = PL;
+        constexpr bool HREG = PL2::IPL * PL2::R <= 16;
+        float2 H[HREG ? PL2::IPL : 1][HREG ? PL2::R : 1];
+        cp_async_wait<1>();                                // filter lines of this tile have landed
+        __syncthreads();
+        if constexpr (HREG) {
+            F::template mid<0, NP - 1, PRUNE_NONE>(l, m, tw, hline);
+            F::template pass<NP - 1, PRUNE_NONE>(l, tw,
+                [&](int, int, int idx) { return hline[phys(idx)]; },
+                [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * p.scale); });
+            __syncthreads();                               // filter lines are free again
+            if (tn < tiles) issue_h(tn);
+            cp_async_commit();
+            cp_async_wait<1>();                            // k*v lines of this tile have landed
+        } else {
+            F::template mid<0, NP, PRUNE_NONE>(l, m, tw, hline);   // spectrum stays in the line
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        {
+            F::template mid<0, NP - 1, PRUNE_IN>(l, m, tw, uline);
+            float2 Y[PL::IPL][PL::R];
+            F::template pass<NP - 1, PRUNE_NONE>(l, tw,
+                [&](int, int, int idx) { return uline[phys(idx)]; },
+                [&](int i, int r, int idx, float2 v) {
+                    if constexpr (HREG) Y[i][r] = cmul(v, H[i][r]);
+                    else {
+                        const float2 hh = hline[phys(idx)];
+                        Y[i][r] = cmul(v, make_float2(hh.x * p.scale, hh.y * p.scale));
+                    }
+                });
+            __syncwarp(m);
+            FI::template pass<0, PRUNE_NONE>(l, tw,
+                [&](int i, int r, int) { return Y[i][r]; },
+                [&](int, int, int idx, float2 v) { uline[phys(idx)] = v; });
+            __syncwarp(m);
+            FI::template mid<1, NP - 1>(l, m, tw, uline);
+            using PE = typename FI::template Pass<NP - 1>;
+            float2 keep[PE::IPL][PE::R];
+            FI::template pass<NP - 1, PRUNE_OUT>(l, tw,
+                [&](int, int, int idx) { return uline[phys(idx)]; },
+                [&](int i, int r, int, float2 v) { keep[i][r] = v; });
+            __syncwarp(m);
+            if (!(PE::PARTIAL && l >= PE::ITEMS)) {
+#pragma unroll
+                for (int i = 0; i < PE::IPL; ++i)
+#pragma unroll
+                    for (int r = 0; r < PE::R / 2; ++r)
+                        uline[phys(l + i * TPL + r * (N / PE::R))] = keep[i][r];
+            }
+        }
+        __syncthreads();
+        if constexpr (!HREG) {
+            if (tn < tiles) issue_h(tn);
+            cp_async_commit();
+        }
+        {
+            const long long o = t / tpo;
+            const int c0 = (int)(t % tpo) * TX;
+            float2 *dst = p.out + o * p.out_outer + c0 + x;
+            if (c0 + x < p.nc)
+                for (int pos = r0; pos < p.n_out; pos += RPS) dst[(long long)pos * p.nc] = bu[x * LS + phys(pos)];
+        }
+        __syncthreads();
+        if (tn < tiles) issue_u(tn);
+        cp_async_commit();
+        t = tn;
+    }
+    cp_async_wait<0>();
+}
+
+template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t st)
+{
+    using F = WF<LOG2P, false>;
+    constexpr int N = 1 << LOG2P, TX = kCoreThreads / F::TPL;
+    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + N / 2);
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms <= 0) sms = 148;
+        cudaFuncSetAttribute(axis_core_w_kernel<LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    }
+    const long long tiles = a.n_outer * ((a.nc + TX - 1) / TX);
+    const int grid = (int)(tiles < (long long)sms * 2 ? tiles : (long long)sms * 2);
+    if (grid <= 0) return 0;
+    axis_core_w_kernel<LOG2P><<<grid, kCoreThreads, sm, st>>>(a);
+    return 1;
+}
+
+bool core_w_supported(int log2p) { return log2p >= 6 && log2p <= 10; }
+
+int launch_core_w(const AxisArgs &a, cudaStream_t st)
+{
+    switch (a.log2p) {
+    case 6: return launch_core_w_t<6>(a, st);
+    case 7: return launch_core_w_t<7>(a, st);
+    case 8: return launch_core_w_t<8>(a, st);
+    case 9: return launch_core_w_t<9>(a, st);
+    case 10: return launch_core_w_t<10>(a, st);
+    default: return -1;
+    }
+}
+
+}  // namespace hn

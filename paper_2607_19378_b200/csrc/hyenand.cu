@@ -276,7 +276,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
             p->prof.begin(KID_CORE, st);
-            c = launch_axis(a, AXIS_CORE, st);
+            c = (core_w_supported(a.log2p) && !getenv("HYENAND_GENERIC_CORE")) ? launch_core_w(a, st) : launch_axis(a, AXIS_CORE, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
@@ -347,7 +347,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         p->prof.begin(KID_CORE, st);
-        c = launch_axis(a, AXIS_CORE, st);
+        c = (core_w_supported(a.log2p) && !getenv("HYENAND_GENERIC_CORE")) ? launch_core_w(a, st) : launch_axis(a, AXIS_CORE, st);
         p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;

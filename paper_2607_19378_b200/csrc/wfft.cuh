@@ -84,8 +84,9 @@ template <int LOG2N, bool INV> struct WF {
         }
     }
 
-    // Middle of a transform: passes [S0, S1) line -> line, each followed by __syncwarp().
-    template <int S0, int S1>
+    // Passes [S0, S1) line -> line, each followed by __syncwarp().  PR0 applies to pass S0
+    // (PRUNE_IN is only meaningful when S0 == 0).
+    template <int S0, int S1, int PR0 = PRUNE_NONE>
     static __device__ __forceinline__ void mid(int l, unsigned m, const float2 *tw, float2 *line)
     {
         if constexpr (S0 < S1) {
@@ -93,7 +94,7 @@ template <int LOG2N, bool INV> struct WF {
             using PS = Pass<S0>;
             constexpr int R = PS::R;
             float2 keep[PS::IPL][R];
-            pass<S0, PRUNE_NONE>(l, tw,
+            pass<S0, PR0>(l, tw,
                 [&](int, int, int idx) { return line[phys(idx)]; },
                 [&](int i, int r, int, float2 v) { keep[i][r] = v; });
             __syncwarp(m);
