@@ -33,12 +33,20 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
     extern __shared__ float2 smem[];
     float2 *bu = smem;
     float2 *bh = smem + TX * LS;
-    float2 *tw = smem + 2 * TX * LS;
+    float2 *twt = smem + 2 * TX * LS;
+    const TableTw<N> tw{twt};
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *uline = bu + gid * LS;
     float2 *hline = bh + gid * LS;
-    load_twiddles(tw, p.gtw, N, p.gtw_n, tid, kCoreThreads);
+    for (int t = tid; t < N; t += kCoreThreads) twt[t] = p.gtw[t * (p.gtw_n / N)];
+    __syncthreads();
+    // two equal passes: the last forward pass and the last inverse pass use the same twiddles,
+    // which depend on the lane only -> keep them in registers
+    constexpr bool HOIST = NP == 2 && WPlan<LOG2P>::R[0] == WPlan<LOG2P>::R[1];
+    typename F::template Hoist<NP - 1> hw;
+    if constexpr (HOIST) hw.load(l, twt);
+    auto twl = [&](int i, int r, int t) { if constexpr (HOIST) return hw(i, r, t); else return tw(i, r, t); };
     const long long tpo = (p.nc + TX - 1) / TX;
     const long long tiles = p.n_outer * tpo;
     // Tile loads are asynchronous copies (one complex bin per thread and row) straight into the
@@ -86,7 +94,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         __syncthreads();
         if constexpr (HREG) {
             F::template mid<0, NP - 1, PRUNE_NONE>(l, m, tw, hline);
-            F::template pass<NP - 1, PRUNE_NONE>(l, tw,
+            F::template pass<NP - 1, PRUNE_NONE>(l, twl,
                 [&](int, int, int idx) { return hline[phys(idx)]; },
                 [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * p.scale); });
             __syncthreads();                               // filter lines are free again
@@ -101,7 +109,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         {
             F::template mid<0, NP - 1, PRUNE_IN>(l, m, tw, uline);
             float2 Y[PL::IPL][PL::R];
-            F::template pass<NP - 1, PRUNE_NONE>(l, tw,
+            F::template pass<NP - 1, PRUNE_NONE>(l, twl,
                 [&](int, int, int idx) { return uline[phys(idx)]; },
                 [&](int i, int r, int idx, float2 v) {
                     if constexpr (HREG) Y[i][r] = cmul(v, H[i][r]);
@@ -118,7 +126,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
             FI::template mid<1, NP - 1>(l, m, tw, uline);
             using PE = typename FI::template Pass<NP - 1>;
             float2 keep[PE::IPL][PE::R];
-            FI::template pass<NP - 1, PRUNE_OUT>(l, tw,
+            FI::template pass<NP - 1, PRUNE_OUT>(l, twl,
                 [&](int, int, int idx) { return uline[phys(idx)]; },
                 [&](int i, int r, int, float2 v) { keep[i][r] = v; });
             __syncwarp(m);
@@ -154,7 +162,7 @@ template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t 
 {
     using F = WF<LOG2P, false>;
     constexpr int N = 1 << LOG2P, TX = kCoreThreads / F::TPL;
-    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + N / 2);
+    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + N);
     static int sms = 0;
     if (!sms) {
         int dev = 0;

@@ -35,7 +35,7 @@ template <int LOG2P> struct PlaneCfg {
     static constexpr int LS = line_stride(P);
     static constexpr int LSH = line_stride(HP);
     static constexpr int WBUF = (NG * LS > NGH * LSH) ? NG * LS : NGH * LSH;
-    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * CSS + WBUF + HP + HP / 2);
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * CSS + WBUF + P + HP);
 };
 
 // Separate the spectra of the two real rows packed in one complex transform (results in
@@ -62,12 +62,31 @@ __device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, in
     }
 }
 
+// Twiddle source of the P-point transforms of a plane kernel: registers when the plan has two
+// equal passes (the twiddles of the second pass then depend on the lane only), else the table.
+template <int LOG2P, bool INV> struct PlaneTw {
+    using F = WF<LOG2P, INV>;
+    static constexpr bool HOIST = F::NP == 2 && WPlan<LOG2P>::R[0] == WPlan<LOG2P>::R[1];
+    typename F::template Hoist<F::NP - 1> hw;
+    const float2 *table;
+    __device__ __forceinline__ void init(int l, const float2 *tw)
+    {
+        table = tw;
+        if constexpr (HOIST) hw.load(l, tw);
+    }
+    __device__ __forceinline__ float2 operator()(int i, int r, int t) const
+    {
+        if constexpr (HOIST) return hw(i, r, t);
+        else return table[t];
+    }
+};
+
 template <int LOG2P> __device__ __forceinline__ void load_plane_twiddles(float2 *tw, float2 *twh, const float2 *gtw, int gtw_n, int tid)
 {
-    constexpr int HP = 1 << (LOG2P - 1);
+    constexpr int P = 1 << LOG2P;
     const int step = gtw_n >> LOG2P;
-    for (int t = tid; t < HP; t += kPlaneThreads) tw[t] = gtw[t * step];
-    for (int t = tid; t < HP / 2; t += kPlaneThreads) twh[t] = gtw[2 * t * step];
+    for (int t = tid; t < P; t += kPlaneThreads) tw[t] = gtw[t * step];
+    for (int t = tid; t < P / 2; t += kPlaneThreads) twh[t] = gtw[2 * t * step];
 }
 
 // ---- k*v planes ---------------------------------------------------------------------------------
@@ -82,12 +101,14 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
     float2 *cs = smem;
     float2 *wbuf = cs + HP * C::CSS;
     float2 *tw = wbuf + C::WBUF;
-    float2 *twh = tw + HP;
+    float2 *twh = tw + P;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
+    PlaneTw<LOG2P, false> twp;
+    twp.init(l, tw);
     const T *pk = (const T *)p.a;
     const T *pv = (const T *)p.b;
     const int Lx = p.lx, Ly = p.ly;
@@ -98,7 +119,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
             if (y0 < Ly) {
                 const bool has1 = y1 < Ly;
                 const long long o0 = ib + (long long)y0 * Lx, o1 = o0 + Lx;
-                F::template run_to_line<PRUNE_IN>(l, m, tw, line, [&](int, int, int idx) {
+                F::template run_to_line<PRUNE_IN>(l, m, twp, line, [&](int, int, int idx) {
                     float a = 0.f, b = 0.f;
                     if (idx < Lx) {
                         a = IO<T>::ld(pk, o0 + idx) * IO<T>::ld(pv, o0 + idx);
@@ -116,11 +137,11 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
             const float2 *col = cs + kx * C::CSS;
             if (kx != 0) {
                 float2 *d = dst + (long long)kx * P;
-                F::template run<PRUNE_IN>(l, m, tw, line,
+                F::template run<PRUNE_IN>(l, m, twp, line,
                     [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); },
                     [&](int, int, int idx, float2 v) { d[idx] = v; });
             } else {
-                F::template run_to_line<PRUNE_IN>(l, m, tw, line,
+                F::template run_to_line<PRUNE_IN>(l, m, twp, line,
                     [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); });
                 for (int ky = l; ky < P; ky += TPL) {
                     const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
@@ -147,7 +168,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     float2 *cs = smem;
     float2 *wbuf = cs + HP * C::CSS;
     float2 *tw = wbuf + C::WBUF;
-    float2 *twh = tw + HP;
+    float2 *twh = tw + P;
     const int tid = threadIdx.x;
     const int l = tid % TPL, gid = tid / TPL;
     const int lh = tid % TPLH, gidh = tid / TPLH;
@@ -156,6 +177,8 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     float2 *lineh = wbuf + gidh * C::LSH;
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
+    PlaneTw<LOG2P, false> twp;
+    twp.init(l, tw);
     const T *ph = (const T *)p.a;
     const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
     float2 *scratch = p.scratch + (long long)blockIdx.x * C::XH * HP;     // E[kx][ky'], XH lines
@@ -170,7 +193,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                 const bool v0 = my0 < Ky, v1 = my1 < Ky;
                 const long long o0 = ib + (long long)my0 * Kx, o1 = ib + (long long)my1 * Kx;
                 if (v0 || v1) {
-                    F::template run_to_line<PRUNE_NONE>(l, m, tw, line, [&](int, int, int idx) {
+                    F::template run_to_line<PRUNE_NONE>(l, m, twp, line, [&](int, int, int idx) {
                         const int mx = (idx + Lx - 1) & (P - 1);
                         float a = 0.f, b = 0.f;
                         if (mx < Kx) {
@@ -195,39 +218,69 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                 if (kx != 0) {
                     if (e == 0) {
                         float2 *d = scratch + (long long)kx * HP;
-                        FH::template run<PRUNE_NONE>(lh, mh, twh, lineh,
+                        FH::template run<PRUNE_NONE>(lh, mh, TableTw<HP>{twh}, lineh,
                             [&](int, int, int idx) { return col[idx]; },
                             [&](int, int, int idx, float2 v) { d[idx] = v; });
                     } else {
                         const float2 *es = scratch + (long long)kx * HP;
                         float2 *d = dst + (long long)kx * P;
-                        FH::template run<PRUNE_NONE>(lh, mh, twh, lineh,
+                        using LP = typename FH::LastPass;
+                        float2 O[LP::IPL][LP::R], E[LP::IPL][LP::R];
+                        FH::template run<PRUNE_NONE>(lh, mh, TableTw<HP>{twh}, lineh,
                             [&](int, int, int idx) { return col[idx]; },
-                            [&](int, int, int idx, float2 v) {
-                                const float2 E = es[idx];
-                                const float2 t = cmul(v, tw[idx]);            // W_P^ky' * O
-                                d[idx] = cadd(E, t);
-                                d[idx + HP] = csub(E, t);
-                            });
+                            [&](int i, int r, int, float2 v) { O[i][r] = v; });
+                        if (!(LP::PARTIAL && lh >= LP::ITEMS)) {
+                            // fetch the whole first half before the stores so the loads overlap
+#pragma unroll
+                            for (int i = 0; i < LP::IPL; ++i)
+#pragma unroll
+                                for (int r = 0; r < LP::R; ++r) E[i][r] = __ldcg(es + FH::last_pos(lh, i, r));
+#pragma unroll
+                            for (int i = 0; i < LP::IPL; ++i)
+#pragma unroll
+                                for (int r = 0; r < LP::R; ++r) {
+                                    const int idx = FH::last_pos(lh, i, r);
+                                    const float2 t = cmul(O[i][r], tw[idx]);          // W_P^ky' * O
+                                    d[idx] = cadd(E[i][r], t);
+                                    d[idx + HP] = csub(E[i][r], t);
+                                }
+                        }
                     }
                 } else {
-                    FH::template run_to_line<PRUNE_NONE>(lh, mh, twh, lineh,
+                    FH::template run_to_line<PRUNE_NONE>(lh, mh, TableTw<HP>{twh}, lineh,
                         [&](int, int, int idx) { return col[idx]; });
-                    for (int ky = lh; ky < HP; ky += TPLH) {
-                        const float2 c1 = lineh[phys(ky)], c2 = lineh[phys((HP - ky) & (HP - 1))];
-                        const float2 s0 = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));   // bin kx = 0
-                        const float2 sn = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));   // bin kx = P/2
-                        if (e == 0) {
-                            scratch[ky] = s0;
-                            scratch[(long long)HP * HP + ky] = sn;
-                        } else {
-                            const float2 w = tw[ky];
-                            const float2 E0 = scratch[ky], EN = scratch[(long long)HP * HP + ky];
-                            const float2 t0 = cmul(s0, w), tn = cmul(sn, w);
-                            dst[ky] = cadd(E0, t0);
-                            dst[ky + HP] = csub(E0, t0);
-                            dst[(long long)HP * P + ky] = cadd(EN, tn);
-                            dst[(long long)HP * P + ky + HP] = csub(EN, tn);
+                    constexpr int NK = HP / TPLH;
+                    if (e == 0) {
+#pragma unroll 4
+                        for (int t = 0; t < NK; ++t) {
+                            const int ky = lh + t * TPLH;
+                            const float2 c1 = lineh[phys(ky)], c2 = lineh[phys((HP - ky) & (HP - 1))];
+                            scratch[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));                   // bin kx = 0
+                            scratch[(long long)HP * HP + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));  // bin kx = P/2
+                        }
+                    } else {
+                        // all first-half values are fetched before any store, in batches of 8 rows
+                        for (int t0 = 0; t0 < NK; t0 += 8) {
+                            float2 E0[8], EN[8];
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) {
+                                const int ky = lh + (t0 + t) * TPLH;
+                                E0[t] = __ldcg(scratch + ky);
+                                EN[t] = __ldcg(scratch + (long long)HP * HP + ky);
+                            }
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) {
+                                const int ky = lh + (t0 + t) * TPLH;
+                                const float2 c1 = lineh[phys(ky)], c2 = lineh[phys((HP - ky) & (HP - 1))];
+                                const float2 s0 = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
+                                const float2 sn = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
+                                const float2 w = tw[ky];
+                                const float2 t0v = cmul(s0, w), tnv = cmul(sn, w);
+                                dst[ky] = cadd(E0[t], t0v);
+                                dst[ky + HP] = csub(E0[t], t0v);
+                                dst[(long long)HP * P + ky] = cadd(EN[t], tnv);
+                                dst[(long long)HP * P + ky + HP] = csub(EN[t], tnv);
+                            }
                         }
                     }
                 }
@@ -250,12 +303,14 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
     float2 *cs = smem;
     float2 *wbuf = cs + HP * C::CSS;
     float2 *tw = wbuf + C::WBUF;
-    float2 *twh = tw + HP;
+    float2 *twh = tw + P;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = FI::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
+    PlaneTw<LOG2P, true> twp;
+    twp.init(l, tw);
     const T *pq = (const T *)p.a;
     T *py = (T *)p.y;
     const int Lx = p.lx, Ly = p.ly;
@@ -265,12 +320,12 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
             float2 *col = cs + kx * C::CSS;
             if (kx != 0) {
                 const float2 *s = src + (long long)kx * P;
-                FI::template run<PRUNE_OUT>(l, m, tw, line,
+                FI::template run<PRUNE_OUT>(l, m, twp, line,
                     [&](int, int, int idx) { return s[idx]; },
                     [&](int, int, int idx, float2 v) { col[idx] = v; });
             } else {
                 const float2 *sn = src + (long long)HP * P;
-                FI::template run<PRUNE_OUT>(l, m, tw, line,
+                FI::template run<PRUNE_OUT>(l, m, twp, line,
                     [&](int, int, int idx) {
                         const float2 g0 = src[idx], gn = sn[idx];
                         return make_float2(g0.x - gn.y, g0.y + gn.x);
@@ -285,7 +340,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
             const int y0 = 2 * rp, y1 = y0 + 1;
             const bool has1 = y1 < Ly;
             const long long o0 = ob + (long long)y0 * Lx, o1 = o0 + Lx;
-            FI::template run<PRUNE_OUT>(l, m, tw, line,
+            FI::template run<PRUNE_OUT>(l, m, twp, line,
                 [&](int, int, int idx) {
                     const int kx = idx <= HP ? idx : P - idx;
                     if (kx == 0 || kx == HP) {

@@ -24,6 +24,13 @@ template <> struct WPlan<8>  { static constexpr int NP = 2, TPL = 16; static con
 template <> struct WPlan<9>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 8}; };
 template <> struct WPlan<10> { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 16}; };
 
+// Twiddle sources.  A source is called as src(i, r, t): item i of the lane, leg r, table index t
+// (the twiddle wanted is exp(-2 pi i t / N); the engine conjugates it for inverse transforms).
+template <int N> struct TableTw {               // full table of N entries in shared memory
+    const float2 *tw;
+    __device__ __forceinline__ float2 operator()(int, int, int t) const { return tw[t]; }
+};
+
 template <int LOG2N, bool INV> struct WF {
     using P = WPlan<LOG2N>;
     static constexpr int N = 1 << LOG2N;
@@ -54,9 +61,9 @@ template <int LOG2N, bool INV> struct WF {
     // lane, leg r); out(i, r, idx, v) receives the result for position idx.
     // PR: PRUNE_IN (first pass only: positions >= N/2 are zero and never requested),
     //     PRUNE_OUT (last pass only: positions >= N/2 are not produced).
-    // tw: shared-memory table tw[t] = exp(-2 pi i t / N), t < N/2.
-    template <int S, int PR, class In, class Out>
-    static __device__ __forceinline__ void pass(int l, const float2 *tw, In in, Out out)
+    // tw: twiddle source (see TableTw).
+    template <int S, int PR, class Tw, class In, class Out>
+    static __device__ __forceinline__ void pass(int l, Tw tw, In in, Out out)
     {
         using PS = Pass<S>;
         constexpr int R = PS::R, NS = PS::NS;
@@ -74,7 +81,10 @@ template <int LOG2N, bool INV> struct WF {
             if constexpr (NS > 1) {
                 const int k = j & (NS - 1);
 #pragma unroll
-                for (int r = 1; r < NIN; ++r) x[r] = cmul(x[r], twiddle<N, INV>(tw, r * k * (N / (NS * R))));
+                for (int r = 1; r < NIN; ++r) {
+                    const float2 w = tw(i, r, r * k * (N / (NS * R)));
+                    x[r] = INV ? cmulc(x[r], w) : cmul(x[r], w);
+                }
             }
             dft<R, INV, PR>(x);
             const int k = j & (NS - 1);
@@ -86,8 +96,8 @@ template <int LOG2N, bool INV> struct WF {
 
     // Passes [S0, S1) line -> line, each followed by __syncwarp().  PR0 applies to pass S0
     // (PRUNE_IN is only meaningful when S0 == 0).
-    template <int S0, int S1, int PR0 = PRUNE_NONE>
-    static __device__ __forceinline__ void mid(int l, unsigned m, const float2 *tw, float2 *line)
+    template <int S0, int S1, int PR0 = PRUNE_NONE, class Tw>
+    static __device__ __forceinline__ void mid(int l, unsigned m, Tw tw, float2 *line)
     {
         if constexpr (S0 < S1) {
             // loads of all items must precede the stores of any item of the same line
@@ -109,27 +119,47 @@ template <int LOG2N, bool INV> struct WF {
                 }
             }
             __syncwarp(m);
-            mid<S0 + 1, S1>(l, m, tw, line);
+            mid<S0 + 1, S1, PRUNE_NONE>(l, m, tw, line);
         }
     }
 
     // Full transform: first-pass inputs from `in`, last-pass outputs to `out`; the line is
     // scratch.  Callers must __syncwarp() before reusing the line for something else.
-    template <int PR, class In, class Out>
-    static __device__ __forceinline__ void run(int l, unsigned m, const float2 *tw, float2 *line, In in, Out out)
+    template <int PR, class Tw, class In, class Out>
+    static __device__ __forceinline__ void run(int l, unsigned m, Tw tw, float2 *line, In in, Out out)
     {
         constexpr int PF = (PR == PRUNE_IN) ? PRUNE_IN : PRUNE_NONE;
         constexpr int PL = (PR == PRUNE_OUT) ? PRUNE_OUT : PRUNE_NONE;
         pass<0, PF>(l, tw, in, [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
         __syncwarp(m);
-        mid<1, NP - 1>(l, m, tw, line);
+        mid<1, NP - 1, PRUNE_NONE>(l, m, tw, line);
         pass<NP - 1, PL>(l, tw, [&](int, int, int idx) { return line[phys(idx)]; }, out);
     }
 
+    // Position (natural order) of output leg r of item i of lane l after the last pass.
+    using LastPass = Pass<NP - 1>;
+    static __device__ __forceinline__ int last_pos(int l, int i, int r) { return l + i * TPL + r * (N / LastPass::R); }
+
+    // Register copy of the twiddles of pass S (they depend on the lane only).
+    template <int S> struct Hoist {
+        using PS = Pass<S>;
+        float2 w[PS::IPL][PS::R];
+        __device__ __forceinline__ void load(int l, const float2 *table)
+        {
+#pragma unroll
+            for (int i = 0; i < PS::IPL; ++i) {
+                const int k = (l + i * TPL) & (PS::NS - 1);
+#pragma unroll
+                for (int r = 1; r < PS::R; ++r) w[i][r] = table[r * k * (N / (PS::NS * PS::R))];
+            }
+        }
+        __device__ __forceinline__ float2 operator()(int i, int r, int) const { return w[i][r]; }
+    };
+
     // Full transform whose results end up in the line itself (natural order); ends with a
     // __syncwarp(), so every lane of the group may read any position afterwards.
-    template <int PR, class In>
-    static __device__ __forceinline__ void run_to_line(int l, unsigned m, const float2 *tw, float2 *line, In in)
+    template <int PR, class Tw, class In>
+    static __device__ __forceinline__ void run_to_line(int l, unsigned m, Tw tw, float2 *line, In in)
     {
         using PS = Pass<NP - 1>;
         float2 keep[PS::IPL][PS::R];
