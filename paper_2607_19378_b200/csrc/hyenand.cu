@@ -317,6 +317,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
     auto filter = [&](const char *hp, long long n) -> int {
         PlaneArgs a{};
         a.a = hp; a.out = p->wh_a; a.scratch = p->plane_scratch; a.planes = n * p->K[0];
+        a.a_elems = n * p->kvol;
         a.lx = p->L[2]; a.ly = p->L[1]; a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         p->prof.begin(KID_PLANE_H, st);
         int c = launch_plane(a, PLANE_H, p->log2p[2], p->dtype, st);
@@ -331,6 +332,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         if (!shared && filter(h + (size_t)s0 * p->kvol * es, n)) return -1;
         PlaneArgs u{};
         u.a = k + (size_t)s0 * p->vol * es; u.b = v + (size_t)s0 * p->vol * es; u.out = p->ws_a;
+        u.a_elems = n * p->vol;
         u.planes = n * p->L[0]; u.lx = p->L[2]; u.ly = p->L[1]; u.gtw = p->gtw; u.gtw_n = p->gtw_n;
         p->prof.begin(KID_PLANE_U, st);
         int c = launch_plane(u, PLANE_U, p->log2p[2], p->dtype, st);

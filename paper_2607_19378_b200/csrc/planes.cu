@@ -32,11 +32,60 @@ template <int LOG2P> struct PlaneCfg {
     using FH = WF<LOG2P - 1, false>;                         // half-length columns of hplane
     static constexpr int NG = kPlaneThreads / F::TPL;        // groups working on P-point lines
     static constexpr int NGH = kPlaneThreads / FH::TPL;      // groups working on P/2-point lines
-    static constexpr int LS = line_stride(P);
-    static constexpr int LSH = line_stride(HP);
+    // lines start on 16-byte boundaries (asynchronous 16-byte copies land in them) and two
+    // neighbouring lines do not share banks: stride = 8 mod 16 complex numbers
+    static constexpr int plane_ls(int n) { return ((phys(n) + 1 + 7) / 16) * 16 + 8; }
+    static constexpr int LS = plane_ls(P);
+    static constexpr int LSH = plane_ls(HP);
     static constexpr int WBUF = (NG * LS > NGH * LSH) ? NG * LS : NGH * LSH;
     static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * CSS + WBUF + P + HP);
 };
+
+// Ask the memory system to bring [ptr, ptr + bytes) into L2 (bulk prefetch, 16-byte granules);
+// the CTA issues it for the plane it will work on next, so that plane's loads hit L2.
+__device__ __forceinline__ void prefetch_l2(const void *ptr, long long bytes, int tid)
+{
+    const unsigned long long a0 = (unsigned long long)ptr & ~15ull;
+    const unsigned long long a1 = ((unsigned long long)ptr + (unsigned long long)bytes + 15ull) & ~15ull;
+    constexpr unsigned long long CH = 4096;
+    for (unsigned long long a = a0 + (unsigned long long)tid * CH; a < a1; a += (unsigned long long)kPlaneThreads * CH) {
+        const unsigned sz = (unsigned)(a1 - a < CH ? a1 - a : CH);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(a), "r"(sz) : "memory");
+    }
+}
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
+// Copy n bytes starting at src (aligned to 2 or 4 bytes only: rows of odd length) into shared
+// memory with 16-byte copies of the surrounding aligned chunks: byte k of the row lands at
+// dst + (src & 15) + k.  [lo, hi) bounds the tensor; a chunk that would cross it (only at the
+// two ends of the tensor) is filled 2 bytes at a time.  TPL lanes cooperate.
+template <int TPL>
+__device__ __forceinline__ void stage_row(unsigned char *dst, const unsigned char *src, int n,
+                                          const unsigned char *lo, const unsigned char *hi, int l)
+{
+    const unsigned char *a = src - ((unsigned long long)src & 15ull);
+    const int nch = (int)((src + n - a + 15) >> 4);
+    for (int c = l; c < nch; c += TPL) {
+        const unsigned char *g = a + 16 * c;
+        if (g >= lo && g + 16 <= hi) cp_async16(dst + 16 * c, g);
+        else {
+            for (int b = 0; b < 16; b += 2)
+                if (g + b >= src && g + b < src + n)
+                    *reinterpret_cast<unsigned short *>(dst + 16 * c + b) = *reinterpret_cast<const unsigned short *>(g + b);
+        }
+    }
+}
+template <typename T> __device__ __forceinline__ float staged(const unsigned char *row, int off, int i)
+{
+    if constexpr (sizeof(T) == 4) return *reinterpret_cast<const float *>(row + off + 4 * i);
+    else return __bfloat162float(*reinterpret_cast<const bf16 *>(row + off + 2 * i));
+}
 
 // Separate the spectra of the two real rows packed in one complex transform (results in
 // `line`, natural order) and scatter them into column store rows y0, y1.
@@ -111,19 +160,36 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
     twp.init(l, tw);
     const T *pk = (const T *)p.a;
     const T *pv = (const T *)p.b;
+    const unsigned char *kb = (const unsigned char *)p.a, *vb = (const unsigned char *)p.b;
     const int Lx = p.lx, Ly = p.ly;
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const long long ib = pl * (long long)Ly * Lx;
+        if (pl + gridDim.x < p.planes) {
+            const long long nb = (pl + gridDim.x) * (long long)Ly * Lx;
+            prefetch_l2(pk + nb, (long long)Ly * Lx * sizeof(T), tid);
+            prefetch_l2(pv + nb, (long long)Ly * Lx * sizeof(T), tid);
+        }
         for (int rp = gid; 2 * rp < HP; rp += C::NG) {
             const int y0 = 2 * rp, y1 = y0 + 1;
             if (y0 < Ly) {
                 const bool has1 = y1 < Ly;
-                const long long o0 = ib + (long long)y0 * Lx, o1 = o0 + Lx;
-                F::template run_to_line<PRUNE_IN>(l, m, twp, line, [&](int, int, int idx) {
+                // the two rows of k and of v (consecutive in memory) are fetched with 16-byte copies
+                // into the line itself, which the first pass reads before anything is written to it
+                const int nrow = (has1 ? 2 : 1) * Lx * (int)sizeof(T);
+                const unsigned char *gk = kb + (ib + (long long)y0 * Lx) * sizeof(T);
+                const unsigned char *gv = vb + (ib + (long long)y0 * Lx) * sizeof(T);
+                unsigned char *sk = reinterpret_cast<unsigned char *>(line);
+                unsigned char *sv = sk + C::LS * 4;                       // second half of the line
+                stage_row<TPL>(sk, gk, nrow, kb, kb + p.a_elems * sizeof(T), l);
+                stage_row<TPL>(sv, gv, nrow, vb, vb + p.a_elems * sizeof(T), l);
+                cp_async_wait_all();
+                __syncwarp(m);
+                const int ok = (int)((unsigned long long)gk & 15ull), ov = (int)((unsigned long long)gv & 15ull);
+                F::template run_to_line<PRUNE_IN, true>(l, m, twp, line, [&](int, int, int idx) {
                     float a = 0.f, b = 0.f;
                     if (idx < Lx) {
-                        a = IO<T>::ld(pk, o0 + idx) * IO<T>::ld(pv, o0 + idx);
-                        if (has1) b = IO<T>::ld(pk, o1 + idx) * IO<T>::ld(pv, o1 + idx);
+                        a = staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx);
+                        if (has1) b = staged<T>(sk, ok, Lx + idx) * staged<T>(sv, ov, Lx + idx);
                     }
                     return make_float2(a, b);
                 });
@@ -179,12 +245,14 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     __syncthreads();
     PlaneTw<LOG2P, false> twp;
     twp.init(l, tw);
-    const T *ph = (const T *)p.a;
+    const unsigned char *hb = (const unsigned char *)p.a;
     const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
     float2 *scratch = p.scratch + (long long)blockIdx.x * C::XH * HP;     // E[kx][ky'], XH lines
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const long long ib = pl * (long long)Ky * Kx;
         float2 *dst = p.out + pl * (long long)C::XH * P;
+        if (pl + gridDim.x < p.planes)
+            prefetch_l2(hb + (pl + gridDim.x) * (long long)Ky * Kx * sizeof(T), (long long)Ky * Kx * sizeof(T), tid);
         for (int e = 0; e < 2; ++e) {
             // rows at padded positions yp = 2*yy + e, i.e. taps my = (yp + Ly - 1) mod P
             for (int rp = gid; 2 * rp < HP; rp += C::NG) {
@@ -193,12 +261,21 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                 const bool v0 = my0 < Ky, v1 = my1 < Ky;
                 const long long o0 = ib + (long long)my0 * Kx, o1 = ib + (long long)my1 * Kx;
                 if (v0 || v1) {
-                    F::template run_to_line<PRUNE_NONE>(l, m, twp, line, [&](int, int, int idx) {
+                    constexpr int SLOT = ((C::P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;   // bytes kept per staged row
+                    static_assert(2 * SLOT <= C::LS * 8, "staged rows must fit the line");
+                    unsigned char *s0 = reinterpret_cast<unsigned char *>(line), *s1 = s0 + SLOT;
+                    const unsigned char *g0 = hb + o0 * sizeof(T), *g1 = hb + o1 * sizeof(T);
+                    if (v0) stage_row<TPL>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), l);
+                    if (v1) stage_row<TPL>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), l);
+                    cp_async_wait_all();
+                    __syncwarp(m);
+                    const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
+                    F::template run_to_line<PRUNE_NONE, true>(l, m, twp, line, [&](int, int, int idx) {
                         const int mx = (idx + Lx - 1) & (P - 1);
                         float a = 0.f, b = 0.f;
                         if (mx < Kx) {
-                            if (v0) a = IO<T>::ld(ph, o0 + mx);
-                            if (v1) b = IO<T>::ld(ph, o1 + mx);
+                            if (v0) a = staged<T>(s0, f0, mx);
+                            if (v1) b = staged<T>(s1, f1, mx);
                         }
                         return make_float2(a, b);
                     });

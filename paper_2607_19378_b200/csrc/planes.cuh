@@ -18,6 +18,7 @@ struct PlaneArgs {
     int lx, ly;           // grid extent along x (contiguous) and y
     const float2 *gtw;    // global twiddle table with gtw_n >= P points
     int gtw_n;
+    long long a_elems;    // total elements of a (and b): bounds for the aligned row fetches
 };
 
 bool plane_supported(int log2p);

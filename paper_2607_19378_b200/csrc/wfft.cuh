@@ -125,12 +125,27 @@ template <int LOG2N, bool INV> struct WF {
 
     // Full transform: first-pass inputs from `in`, last-pass outputs to `out`; the line is
     // scratch.  Callers must __syncwarp() before reusing the line for something else.
-    template <int PR, class Tw, class In, class Out>
+    // ALIAS: the first-pass inputs live in the line itself (in another format), so all of them
+    // are read before the first pass writes its results.
+    template <int PR, bool ALIAS = false, class Tw, class In, class Out>
     static __device__ __forceinline__ void run(int l, unsigned m, Tw tw, float2 *line, In in, Out out)
     {
         constexpr int PF = (PR == PRUNE_IN) ? PRUNE_IN : PRUNE_NONE;
         constexpr int PL = (PR == PRUNE_OUT) ? PRUNE_OUT : PRUNE_NONE;
-        pass<0, PF>(l, tw, in, [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+        if constexpr (ALIAS) {
+            using P0 = Pass<0>;
+            float2 keep[P0::IPL][P0::R];
+            pass<0, PF>(l, tw, in, [&](int i, int r, int, float2 v) { keep[i][r] = v; });
+            __syncwarp(m);
+            if (!(P0::PARTIAL && l >= P0::ITEMS)) {
+#pragma unroll
+                for (int i = 0; i < P0::IPL; ++i)
+#pragma unroll
+                    for (int r = 0; r < P0::R; ++r) line[phys((l + i * TPL) * P0::R + r)] = keep[i][r];
+            }
+        } else {
+            pass<0, PF>(l, tw, in, [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+        }
         __syncwarp(m);
         mid<1, NP - 1, PRUNE_NONE>(l, m, tw, line);
         pass<NP - 1, PL>(l, tw, [&](int, int, int idx) { return line[phys(idx)]; }, out);
@@ -158,12 +173,12 @@ template <int LOG2N, bool INV> struct WF {
 
     // Full transform whose results end up in the line itself (natural order); ends with a
     // __syncwarp(), so every lane of the group may read any position afterwards.
-    template <int PR, class Tw, class In>
+    template <int PR, bool ALIAS = false, class Tw, class In>
     static __device__ __forceinline__ void run_to_line(int l, unsigned m, Tw tw, float2 *line, In in)
     {
         using PS = Pass<NP - 1>;
         float2 keep[PS::IPL][PS::R];
-        run<PR>(l, m, tw, line, in, [&](int i, int r, int, float2 v) { keep[i][r] = v; });
+        run<PR, ALIAS>(l, m, tw, line, in, [&](int i, int r, int, float2 v) { keep[i][r] = v; });
         __syncwarp(m);
         if (!(PS::PARTIAL && l >= PS::ITEMS)) {
             constexpr int NOUT = (PR == PRUNE_OUT) ? PS::R / 2 : PS::R;
