@@ -1,0 +1,233 @@
+// Fused 2-D path: the whole operator for one (b,c) slice in one CTA, nothing but
+// q, k, v, h, y touches HBM (the single-stage kernel the paper's Appendix B.4 names
+// as its goal for 2-D; its published pipeline still uses three kernels).
+//
+// Per slice: rows of the filter and of k*v are transformed two real rows per complex
+// transform and scattered into shared-memory column stores (half spectra, with the two
+// purely real bins of a row packed into column 0); every column then runs
+//   forward(filter column) -> registers, forward(k*v column), product (Eq. 12),
+//   inverse, keep the cropped half
+// in one group of lanes; finally the rows are transformed back, cropped, gated by q
+// and stored.  Used when both padded axes are equal and at most 128 points.
+#include "common.cuh"
+#include "fused2d.cuh"
+#include "plane_util.cuh"
+
+namespace hn {
+
+template <int LOG2P> struct F2Cfg {
+    static constexpr int P = 1 << LOG2P, HP = P / 2;
+    static constexpr int HCSS = P + 1;                       // filter column store stride (odd)
+    static constexpr int UCSS = HP + 1;                      // k*v column store stride (odd)
+    using F = WF<LOG2P, false>;
+    using FI = WF<LOG2P, true>;
+    static constexpr int NG = kPlaneThreads / F::TPL;
+    static constexpr int LS = plane_ls(P);
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * HCSS + (size_t)HP * UCSS + (size_t)NG * LS + 3 * P);
+};
+
+template <typename T, int LOG2P>
+__global__ void __launch_bounds__(kPlaneThreads, 1) fused2d_kernel(Fused2dArgs p)
+{
+    using C = F2Cfg<LOG2P>;
+    using F = typename C::F;
+    using FI = typename C::FI;
+    constexpr int P = C::P, HP = C::HP, TPL = F::TPL, NP = F::NP;
+    extern __shared__ float2 smem[];
+    float2 *hcs = smem;
+    float2 *ucs = hcs + HP * C::HCSS;
+    float2 *wbuf = ucs + HP * C::UCSS;
+    float2 *x0 = wbuf + C::NG * C::LS;                       // packed column: filter bins kx = 0 ...
+    float2 *xn = x0 + P;                                     // ... and kx = P/2
+    float2 *tw = xn + P;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = F::group_mask(tid);
+    float2 *line = wbuf + gid * C::LS;
+    for (int t = tid; t < P; t += kPlaneThreads) tw[t] = p.gtw[t * (p.gtw_n >> LOG2P)];
+    __syncthreads();
+    PlaneTw<LOG2P, false> twf;
+    twf.init(l, tw);
+    PlaneTw<LOG2P, true> twi;
+    twi.init(l, tw);
+    const unsigned char *kb = (const unsigned char *)p.k, *vb = (const unsigned char *)p.v;
+    const unsigned char *hb = (const unsigned char *)p.h;
+    const T *pq = (const T *)p.q;
+    T *py = (T *)p.y;
+    const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
+    const long long vol = (long long)Lx * Ly, kvol = (long long)Kx * Ky;
+    using PL = typename F::LastPass;
+
+    for (long long s = blockIdx.x; s < p.slices; s += gridDim.x) {
+        const long long hs = p.h_mod ? (s + p.h_off) % p.h_mod : s;
+        const long long sn = s + gridDim.x;
+        if (sn < p.slices) {
+            const long long hn2 = p.h_mod ? (sn + p.h_off) % p.h_mod : sn;
+            prefetch_l2(hb + hn2 * kvol * sizeof(T), kvol * sizeof(T), tid);
+            prefetch_l2(kb + sn * vol * sizeof(T), vol * sizeof(T), tid);
+            prefetch_l2(vb + sn * vol * sizeof(T), vol * sizeof(T), tid);
+            prefetch_l2(pq + sn * vol, vol * sizeof(T), tid);
+        }
+        // ---- filter rows: padded position yp holds tap my = (yp + Ly - 1) mod P --------------
+        for (int rp = gid; 2 * rp < P; rp += C::NG) {
+            const int yp0 = 2 * rp, yp1 = yp0 + 1;
+            const int my0 = (yp0 + Ly - 1) & (P - 1), my1 = (yp1 + Ly - 1) & (P - 1);
+            const bool v0 = my0 < Ky, v1 = my1 < Ky;
+            if (v0 || v1) {
+                constexpr int SLOT = ((P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;
+                static_assert(2 * SLOT <= C::LS * 8, "staged rows must fit the line");
+                unsigned char *s0 = reinterpret_cast<unsigned char *>(line), *s1 = s0 + SLOT;
+                const unsigned char *g0 = hb + (hs * kvol + (long long)my0 * Kx) * sizeof(T);
+                const unsigned char *g1 = hb + (hs * kvol + (long long)my1 * Kx) * sizeof(T);
+                if (v0) stage_row<TPL>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.h_elems * sizeof(T), l);
+                if (v1) stage_row<TPL>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.h_elems * sizeof(T), l);
+                cp_async_wait_all();
+                __syncwarp(m);
+                const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
+                F::template run_to_line<PRUNE_NONE, true>(l, m, twf, line, [&](int, int, int idx) {
+                    const int mx = (idx + Lx - 1) & (P - 1);
+                    float a = 0.f, b = 0.f;
+                    if (mx < Kx) {
+                        if (v0) a = staged<T>(s0, f0, mx);
+                        if (v1) b = staged<T>(s1, f1, mx);
+                    }
+                    return make_float2(a, b);
+                });
+                separate_rows<LOG2P, C::HCSS>(line, hcs, yp0, yp1, l);
+                __syncwarp(m);
+            } else {
+                for (int kx = l; kx < HP; kx += TPL) {
+                    hcs[kx * C::HCSS + yp0] = make_float2(0.f, 0.f);
+                    hcs[kx * C::HCSS + yp1] = make_float2(0.f, 0.f);
+                }
+            }
+        }
+        // ---- k*v rows -----------------------------------------------------------------------------
+        for (int rp = gid; 2 * rp < Ly; rp += C::NG) {
+            const int y0 = 2 * rp, y1 = y0 + 1;
+            const bool has1 = y1 < Ly;
+            const int nrow = (has1 ? 2 : 1) * Lx * (int)sizeof(T);
+            const unsigned char *gk = kb + (s * vol + (long long)y0 * Lx) * sizeof(T);
+            const unsigned char *gv = vb + (s * vol + (long long)y0 * Lx) * sizeof(T);
+            unsigned char *sk = reinterpret_cast<unsigned char *>(line);
+            unsigned char *sv = sk + C::LS * 4;
+            stage_row<TPL>(sk, gk, nrow, kb, kb + p.kv_elems * sizeof(T), l);
+            stage_row<TPL>(sv, gv, nrow, vb, vb + p.kv_elems * sizeof(T), l);
+            cp_async_wait_all();
+            __syncwarp(m);
+            const int ok = (int)((unsigned long long)gk & 15ull), ov = (int)((unsigned long long)gv & 15ull);
+            F::template run_to_line<PRUNE_IN, true>(l, m, twf, line, [&](int, int, int idx) {
+                float a = 0.f, b = 0.f;
+                if (idx < Lx) {
+                    a = staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx);
+                    if (has1) b = staged<T>(sk, ok, Lx + idx) * staged<T>(sv, ov, Lx + idx);
+                }
+                return make_float2(a, b);
+            });
+            separate_rows<LOG2P, C::UCSS>(line, ucs, y0, y1, l);
+            __syncwarp(m);
+        }
+        __syncthreads();
+        // ---- columns: filter spectrum, k*v spectrum, product, inverse --------------------------
+        for (int kx = gid; kx < HP; kx += C::NG) {
+            const float2 *hc = hcs + kx * C::HCSS;
+            float2 *uc = ucs + kx * C::UCSS;
+            if (kx != 0) {
+                float2 H[PL::IPL][PL::R];
+                F::template run<PRUNE_NONE>(l, m, twf, line,
+                    [&](int, int, int idx) { return hc[idx]; },
+                    [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * p.scale); });
+                __syncwarp(m);
+                float2 Y[PL::IPL][PL::R];
+                F::template run<PRUNE_IN>(l, m, twf, line,
+                    [&](int, int, int idx) { return idx < Ly ? uc[idx] : make_float2(0.f, 0.f); },
+                    [&](int i, int r, int, float2 v) { Y[i][r] = cmul(v, H[i][r]); });
+                __syncwarp(m);
+                FI::template pass<0, PRUNE_NONE>(l, twi,
+                    [&](int i, int r, int) { return Y[i][r]; },
+                    [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+                __syncwarp(m);
+                FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, line);
+                FI::template pass<NP - 1, PRUNE_OUT>(l, twi,
+                    [&](int, int, int idx) { return line[phys(idx)]; },
+                    [&](int, int, int idx, float2 v) { uc[idx] = v; });
+            } else {
+                // column 0 carries the real bins kx = 0 and kx = P/2 as one complex column: split the
+                // spectra with the Hermitian symmetry, multiply bin by bin, pack again
+                F::template run_to_line<PRUNE_NONE>(l, m, twf, line, [&](int, int, int idx) { return hc[idx]; });
+                for (int ky = l; ky < P; ky += TPL) {
+                    const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
+                    x0[ky] = make_float2(0.5f * p.scale * (c1.x + c2.x), 0.5f * p.scale * (c1.y - c2.y));
+                    xn[ky] = make_float2(0.5f * p.scale * (c1.y + c2.y), 0.5f * p.scale * (c2.x - c1.x));
+                }
+                __syncwarp(m);
+                F::template run_to_line<PRUNE_IN>(l, m, twf, line,
+                    [&](int, int, int idx) { return idx < Ly ? uc[idx] : make_float2(0.f, 0.f); });
+                FI::template run<PRUNE_OUT, true>(l, m, twi, line,
+                    [&](int, int, int idx) {
+                        const float2 c1 = line[phys(idx)], c2 = line[phys((P - idx) & (P - 1))];
+                        const float2 u0 = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
+                        const float2 un = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
+                        const float2 y0 = cmul(u0, x0[idx]), yn = cmul(un, xn[idx]);
+                        return make_float2(y0.x - yn.y, y0.y + yn.x);
+                    },
+                    [&](int, int, int idx, float2 v) { uc[idx] = v; });
+            }
+            __syncwarp(m);
+        }
+        __syncthreads();
+        // ---- rows back: complex-to-real, crop, gate, store ------------------------------------------
+        for (int rp = gid; 2 * rp < Ly; rp += C::NG) {
+            const int y0 = 2 * rp, y1 = y0 + 1;
+            const bool has1 = y1 < Ly;
+            const long long o0 = s * vol + (long long)y0 * Lx, o1 = o0 + Lx;
+            FI::template run<PRUNE_OUT>(l, m, twi, line,
+                [&](int, int, int idx) {
+                    const int kx = idx <= HP ? idx : P - idx;
+                    if (kx == 0 || kx == HP) {
+                        const float2 A = ucs[y0];
+                        const float2 B = has1 ? ucs[y1] : make_float2(0.f, 0.f);
+                        return kx == 0 ? make_float2(A.x, B.x) : make_float2(A.y, B.y);
+                    }
+                    const float2 A = ucs[kx * C::UCSS + y0];
+                    const float2 B = has1 ? ucs[kx * C::UCSS + y1] : make_float2(0.f, 0.f);
+                    return idx <= HP ? make_float2(A.x - B.y, A.y + B.x) : make_float2(A.x + B.y, B.x - A.y);
+                },
+                [&](int, int, int idx, float2 v) {
+                    if (idx < Lx) {
+                        IO<T>::st(py, o0 + idx, v.x * IO<T>::ld(pq, o0 + idx));
+                        if (has1) IO<T>::st(py, o1 + idx, v.y * IO<T>::ld(pq, o1 + idx));
+                    }
+                });
+            __syncwarp(m);
+        }
+        __syncthreads();
+    }
+}
+
+template <typename T, int LOG2P> static int launch_fused2d_t(const Fused2dArgs &a, cudaStream_t st)
+{
+    using C = F2Cfg<LOG2P>;
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms <= 0) sms = 148;
+        cudaFuncSetAttribute(fused2d_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+    }
+    const int grid = (int)(a.slices < sms ? a.slices : sms);
+    if (grid <= 0) return 0;
+    fused2d_kernel<T, LOG2P><<<grid, kPlaneThreads, C::SMEM, st>>>(a);
+    return 1;
+}
+
+bool fused2d_supported(int log2p) { return log2p == 6 || log2p == 7; }
+
+int launch_fused2d(const Fused2dArgs &a, int log2p, int dtype, cudaStream_t st)
+{
+    if (log2p == 7) return dtype == 0 ? launch_fused2d_t<float, 7>(a, st) : launch_fused2d_t<bf16, 7>(a, st);
+    if (log2p == 6) return dtype == 0 ? launch_fused2d_t<float, 6>(a, st) : launch_fused2d_t<bf16, 6>(a, st);
+    return -1;
+}
+
+}  // namespace hn

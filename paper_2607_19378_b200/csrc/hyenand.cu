@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "ct1d.cuh"
 #include "planes.cuh"
+#include "fused2d.cuh"
 
 using namespace hn;
 
@@ -28,7 +29,7 @@ static int fail(int code, const char *fmt, ...)
     return code;
 }
 
-enum Path { PATH_ND_GENERIC = 0, PATH_CT1D = 1, PATH_PLANES3D = 2 };
+enum Path { PATH_ND_GENERIC = 0, PATH_CT1D = 1, PATH_PLANES3D = 2, PATH_FUSED2D = 3 };
 
 struct hyenand_plan {
     int ndim, B, C, causal, dtype;
@@ -149,7 +150,11 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     const bool three = p->P[0] > 1;
     if (three && p->log2p[1] == p->log2p[2] && plane_supported(p->log2p[2]) && !getenv("HYENAND_FORCE_GENERIC"))
         p->path = PATH_PLANES3D;
-    if (p->path == PATH_PLANES3D) {
+    if (ndim == 2 && p->log2p[1] == p->log2p[2] && fused2d_supported(p->log2p[2]) && !getenv("HYENAND_FORCE_GENERIC"))
+        p->path = PATH_FUSED2D;
+    if (p->path == PATH_FUSED2D) {
+        p->ws_a_slice = p->wh_a_slice = p->ws_b_slice = p->wh_b_slice = 0;   // nothing leaves the chip
+    } else if (p->path == PATH_PLANES3D) {
         // spectra [plane][XH][P_y]; the z pass works in place on the k*v spectra
         p->ws_a_slice = (long long)p->L[0] * p->XH * p->P[1];
         p->wh_a_slice = (long long)p->K[0] * p->XH * p->P[1];
@@ -162,7 +167,7 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     }
     const long long per_slice = p->ws_a_slice + p->ws_b_slice + p->wh_a_slice + p->wh_b_slice;
     const long long budget = (8ll << 30) / (long long)sizeof(float2);      // 8 GiB of workspace
-    long long spc = budget / per_slice;
+    long long spc = per_slice ? budget / per_slice : S;
     if (spc < 1) spc = 1;
     if (spc > S) spc = S;
     p->slices_per_chunk = spc;
@@ -365,11 +370,32 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
     return 0;
 }
 
+static int forward_fused2d(hyenand_plan *p, const void *q, const void *k, const void *v, const void *h,
+                           bool shared, void *y, cudaStream_t st, int *launches)
+{
+    Fused2dArgs a{};
+    a.q = q; a.k = k; a.v = v; a.h = h; a.y = y;
+    a.slices = (long long)p->B * p->C; a.lx = p->L[2]; a.ly = p->L[1];
+    a.h_mod = shared ? p->C : 0; a.h_off = 0;
+    a.scale = (float)(1.0 / ((double)p->P[1] * p->P[2]));
+    a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+    a.kv_elems = a.slices * p->vol;
+    a.h_elems = (shared ? p->C : a.slices) * p->kvol;
+    p->prof.begin(KID_FUSED2D, st);
+    int c = launch_fused2d(a, p->log2p[2], p->dtype, st);
+    p->prof.end(st);
+    if (c < 0) return -1;
+    *launches += c;
+    return 0;
+}
+
 static int run_forward(hyenand_plan *p, const void *q, const void *k, const void *v, const void *h,
                        bool shared, void *y, cudaStream_t st, int *launches)
 {
     int rc;
-    if (p->path == PATH_PLANES3D)
+    if (p->path == PATH_FUSED2D)
+        rc = forward_fused2d(p, q, k, v, h, shared, y, st, launches);
+    else if (p->path == PATH_PLANES3D)
         rc = forward_planes3d(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
                               (char *)y, st, launches);
     else if (p->path == PATH_CT1D)
@@ -477,6 +503,7 @@ extern "C" int hyenand_plan_launches(const hyenand_plan *p, int h_shared)
     const long long S = (long long)p->B * p->C;
     const long long chunks = (S + p->slices_per_chunk - 1) / p->slices_per_chunk;
     const int three = p->P[0] > 1;
+    if (p->path == PATH_FUSED2D) return 1;
     if (p->path == PATH_PLANES3D) return (int)(h_shared ? 1 + chunks * 3 : chunks * 4);
     const int filt = 1 + three, body = 3 + 2 * three;
     return (int)(h_shared ? filt + chunks * body : chunks * (filt + body));
@@ -485,14 +512,15 @@ extern "C" int hyenand_plan_launches(const hyenand_plan *p, int h_shared)
 extern "C" const char *hyenand_plan_path(const hyenand_plan *p)
 {
     if (!p) return "";
-    return p->path == PATH_CT1D ? "ct1d" : p->path == PATH_PLANES3D ? "planes3d" : "nd_generic";
+    return p->path == PATH_CT1D ? "ct1d" : p->path == PATH_PLANES3D ? "planes3d"
+         : p->path == PATH_FUSED2D ? "fused2d" : "nd_generic";
 }
 
 // ---- per-kernel accounting (reporting only) ---------------------------------------------
 
 static const char *kKernelNames[KID_COUNT] = {
     "rows_fwd(h)", "axis_fwd(h)", "rows_fwd(k*v)", "axis_fwd(k*v)", "axis_core", "axis_inv", "rows_inv",
-    "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv", "plane_fwd(h)", "plane_fwd(k*v)", "plane_inv"};
+    "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv", "plane_fwd(h)", "plane_fwd(k*v)", "plane_inv", "fused2d"};
 
 static double fft_flops(double lines, int log2n) { return lines * 5.0 * ldexp(1.0, log2n) * log2n; }
 
@@ -531,6 +559,16 @@ extern "C" int hyenand_plan_kernel_info(const hyenand_plan *p, int kid, int h_sh
     }
     const bool three = p->P[0] > 1;
     const double chunks = ceil(S / (double)p->slices_per_chunk);
+    if (p->path == PATH_FUSED2D) {
+        if (kid == KID_FUSED2D) {
+            const double PP = p->P[2], XHd = p->XH;
+            *launches = 1;
+            *bytes = 4.0 * S * p->vol * es + Sh * (double)p->kvol * es;
+            *flops = fft_flops(S * PP / 2.0, p->log2p[2]) + 2.0 * fft_flops(S * p->L[1] / 2.0, p->log2p[2])
+                   + 3.0 * fft_flops(S * XHd, p->log2p[1]) + 12.0 * S * XHd * PP;
+        }
+        return HYENAND_OK;
+    }
     if (p->path == PATH_PLANES3D) {
         const double PY = p->P[1], nc = (double)p->XH * PY, Lz = p->L[0], Kz = p->K[0];
         const double rowsU = p->L[1] / 2.0, colsU = PY / 2.0;

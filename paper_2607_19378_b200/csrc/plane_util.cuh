@@ -1,0 +1,102 @@
+// Device helpers shared by the plane-fused 3-D kernels and the fused 2-D kernel.
+#pragma once
+#include "common.cuh"
+#include "wfft.cuh"
+
+namespace hn {
+
+constexpr int kPlaneThreads = 512;
+
+// lines start on 16-byte boundaries (asynchronous 16-byte copies land in them) and two
+// neighbouring lines do not share banks: stride = 8 mod 16 complex numbers
+__host__ __device__ constexpr int plane_ls(int n) { return ((phys(n) + 1 + 7) / 16) * 16 + 8; }
+
+// Ask the memory system to bring [ptr, ptr + bytes) into L2 (bulk prefetch, 16-byte granules);
+// the CTA issues it for the plane it will work on next, so that plane's loads hit L2.
+__device__ __forceinline__ void prefetch_l2(const void *ptr, long long bytes, int tid)
+{
+    const unsigned long long a0 = (unsigned long long)ptr & ~15ull;
+    const unsigned long long a1 = ((unsigned long long)ptr + (unsigned long long)bytes + 15ull) & ~15ull;
+    constexpr unsigned long long CH = 4096;
+    for (unsigned long long a = a0 + (unsigned long long)tid * CH; a < a1; a += (unsigned long long)kPlaneThreads * CH) {
+        const unsigned sz = (unsigned)(a1 - a < CH ? a1 - a : CH);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(a), "r"(sz) : "memory");
+    }
+}
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
+// Copy n bytes starting at src (aligned to 2 or 4 bytes only: rows of odd length) into shared
+// memory with 16-byte copies of the surrounding aligned chunks: byte k of the row lands at
+// dst + (src & 15) + k.  [lo, hi) bounds the tensor; a chunk that would cross it (only at the
+// two ends of the tensor) is filled 2 bytes at a time.  TPL lanes cooperate.
+template <int TPL>
+__device__ __forceinline__ void stage_row(unsigned char *dst, const unsigned char *src, int n,
+                                          const unsigned char *lo, const unsigned char *hi, int l)
+{
+    const unsigned char *a = src - ((unsigned long long)src & 15ull);
+    const int nch = (int)((src + n - a + 15) >> 4);
+    for (int c = l; c < nch; c += TPL) {
+        const unsigned char *g = a + 16 * c;
+        if (g >= lo && g + 16 <= hi) cp_async16(dst + 16 * c, g);
+        else {
+            for (int b = 0; b < 16; b += 2)
+                if (g + b >= src && g + b < src + n)
+                    *reinterpret_cast<unsigned short *>(dst + 16 * c + b) = *reinterpret_cast<const unsigned short *>(g + b);
+        }
+    }
+}
+template <typename T> __device__ __forceinline__ float staged(const unsigned char *row, int off, int i)
+{
+    if constexpr (sizeof(T) == 4) return *reinterpret_cast<const float *>(row + off + 4 * i);
+    else return __bfloat162float(*reinterpret_cast<const bf16 *>(row + off + 2 * i));
+}
+
+// Separate the spectra of the two real rows packed in one complex transform (results in
+// `line`, natural order) and scatter them into column store rows y0, y1.
+template <int LOG2P, int CSS>
+__device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, int y0, int y1, int l)
+{
+    constexpr int P = 1 << LOG2P, HP = P / 2, TPL = WF<LOG2P, false>::TPL;
+    float a0 = 0.f, b0 = 0.f;
+    for (int kx = l; kx <= HP; kx += TPL) {
+        const float2 z1 = line[phys(kx)];
+        const float2 z2 = line[phys((P - kx) & (P - 1))];
+        const float2 A = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
+        const float2 B = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
+        if (kx == 0) { a0 = A.x; b0 = B.x; }
+        else if (kx == HP) {                                 // same lane as kx == 0
+            cs[y0] = make_float2(a0, A.x);
+            cs[y1] = make_float2(b0, B.x);
+        } else {
+            cs[kx * CSS + y0] = A;
+            cs[kx * CSS + y1] = B;
+        }
+    }
+}
+
+// Twiddle source of the P-point transforms of a plane kernel: registers when the plan has two
+// equal passes (the twiddles of the second pass then depend on the lane only), else the table.
+template <int LOG2P, bool INV> struct PlaneTw {
+    using F = WF<LOG2P, INV>;
+    static constexpr bool HOIST = F::NP == 2 && WPlan<LOG2P>::R[0] == WPlan<LOG2P>::R[1];
+    typename F::template Hoist<F::NP - 1> hw;
+    const float2 *table;
+    __device__ __forceinline__ void init(int l, const float2 *tw)
+    {
+        table = tw;
+        if constexpr (HOIST) hw.load(l, tw);
+    }
+    __device__ __forceinline__ float2 operator()(int i, int r, int t) const
+    {
+        if constexpr (HOIST) return hw(i, r, t);
+        else return table[t];
+    }
+};
+
+}  // namespace hn

@@ -97,6 +97,23 @@ def test_plane_fused_3d_path(dims, dtype):
     check(w, q, k, v, h)
 
 
+FUSED2D_SHAPES = [(20, 30), (17, 32), (33, 64), (40, 50), (63, 33), (64, 64)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shared", [False, True])
+@pytest.mark.parametrize("dims", FUSED2D_SHAPES, ids=str)
+def test_fused_2d_path(dims, dtype, shared):
+    """2-D grids whose padded axes are both 64 or both 128 run as one fused kernel."""
+    w, (q, k, v, h) = W.random_problem(dims, B=3, C=2, dtype=dtype, h_shared=shared, seed=23)
+    from paper_2607_19378_b200 import hyenand as hn
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    assert hn.hyenand_plan_path(plan.handle) == "fused2d"
+    assert hn.hyenand_plan_launches(plan.handle, shared) == 1
+    plan.close()
+    check(w, q, k, v, h)
+
+
 def test_plane_fused_3d_shared_filter():
     w, (q, k, v, h) = W.random_problem((3, 40, 50), B=3, C=2, dtype="f32", h_shared=True, seed=22)
     check(w, q, k, v, h)
