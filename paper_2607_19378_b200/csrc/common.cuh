@@ -26,7 +26,7 @@ template <> struct IO<bf16> {
 // synchronised) adds the elapsed times to per-kernel totals.
 enum KernelId {
     KID_ROWS_H = 0, KID_AXIS_H, KID_ROWS_U, KID_AXIS_U, KID_CORE, KID_AXIS_INV, KID_ROWS_INV,
-    KID_CT_COLS_H, KID_CT_COLS_U, KID_CT_CORE, KID_CT_COLS_INV, KID_PLANE_H, KID_PLANE_U, KID_PLANE_INV, KID_FUSED2D, KID_COUNT
+    KID_CT_COLS_H, KID_CT_COLS_U, KID_CT_CORE, KID_CT_COLS_INV, KID_PLANE_H, KID_PLANE_U, KID_PLANE_INV, KID_FUSED2D, KID_CT_HSPEC, KID_COUNT
 };
 
 struct Prof {

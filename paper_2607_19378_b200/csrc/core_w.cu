@@ -7,7 +7,7 @@
 // the paper), and the inverse transform started from those registers.  Only the
 // cropped half of the inverse is produced and written back in place.
 #include "common.cuh"
-#include "wfft.cuh"
+#include "plane_util.cuh"
 
 namespace hn {
 
@@ -34,19 +34,19 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
     float2 *bu = smem;
     float2 *bh = smem + TX * LS;
     float2 *twt = smem + 2 * TX * LS;
-    const TableTw<N> tw{twt};
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *uline = bu + gid * LS;
     float2 *hline = bh + gid * LS;
     for (int t = tid; t < N; t += kCoreThreads) twt[t] = p.gtw[t * (p.gtw_n / N)];
     __syncthreads();
-    // two equal passes: the last forward pass and the last inverse pass use the same twiddles,
-    // which depend on the lane only -> keep them in registers
-    constexpr bool HOIST = NP == 2 && WPlan<LOG2P>::R[0] == WPlan<LOG2P>::R[1];
-    typename F::template Hoist<NP - 1> hw;
-    if constexpr (HOIST) hw.load(l, twt);
-    auto twl = [&](int i, int r, int t) { if constexpr (HOIST) return hw(i, r, t); else return tw(i, r, t); };
+    // twiddles: registers when both passes are equal (they depend on the lane only), else
+    // per-pass tables
+    PlaneTw<LOG2P, false> tw;
+    tw.init(l, twt, twt + N, tid, kCoreThreads);
+    PlaneTw<LOG2P, true> twi;
+    twi.init(l, twt, twt + 2 * N, tid, kCoreThreads);
+    __syncthreads();
     const long long tpo = (p.nc + TX - 1) / TX;
     const long long tiles = p.n_outer * tpo;
     // Tile loads are asynchronous copies (one complex bin per thread and row) straight into the
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         __syncthreads();
         if constexpr (HREG) {
             F::template mid<0, NP - 1, PRUNE_NONE>(l, m, tw, hline);
-            F::template pass<NP - 1, PRUNE_NONE>(l, twl,
+            F::template pass<NP - 1, PRUNE_NONE>(l, tw,
                 [&](int, int, int idx) { return hline[phys(idx)]; },
                 [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * p.scale); });
             __syncthreads();                               // filter lines are free again
@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         {
             F::template mid<0, NP - 1, PRUNE_IN>(l, m, tw, uline);
             float2 Y[PL::IPL][PL::R];
-            F::template pass<NP - 1, PRUNE_NONE>(l, twl,
+            F::template pass<NP - 1, PRUNE_NONE>(l, tw,
                 [&](int, int, int idx) { return uline[phys(idx)]; },
                 [&](int i, int r, int idx, float2 v) {
                     if constexpr (HREG) Y[i][r] = cmul(v, H[i][r]);
@@ -119,14 +119,14 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
                     }
                 });
             __syncwarp(m);
-            FI::template pass<0, PRUNE_NONE>(l, tw,
+            FI::template pass<0, PRUNE_NONE>(l, twi,
                 [&](int i, int r, int) { return Y[i][r]; },
                 [&](int, int, int idx, float2 v) { uline[phys(idx)] = v; });
             __syncwarp(m);
-            FI::template mid<1, NP - 1>(l, m, tw, uline);
+            FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, uline);
             using PE = typename FI::template Pass<NP - 1>;
             float2 keep[PE::IPL][PE::R];
-            FI::template pass<NP - 1, PRUNE_OUT>(l, twl,
+            FI::template pass<NP - 1, PRUNE_OUT>(l, twi,
                 [&](int, int, int idx) { return uline[phys(idx)]; },
                 [&](int i, int r, int, float2 v) { keep[i][r] = v; });
             __syncwarp(m);
@@ -162,7 +162,7 @@ template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t 
 {
     using F = WF<LOG2P, false>;
     constexpr int N = 1 << LOG2P, TX = kCoreThreads / F::TPL;
-    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + N);
+    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + 3 * N);
     static int sms = 0;
     if (!sms) {
         int dev = 0;

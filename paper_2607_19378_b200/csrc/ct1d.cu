@@ -12,6 +12,7 @@
 //   cols_inv  rebuild the mirrored half, inverse transform along f1, keep
 //             t < L (crop), apply the output gate q, store.
 #include <math.h>
+#include <stdlib.h>
 
 #include <vector>
 
@@ -421,6 +422,20 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
     const long long S = (long long)c->B * c->C;
     const size_t es = c->dtype == 0 ? 4 : 2;
     const TwoLevel twp{c->twp_coarse, c->twp_fine, c->lo};
+    if (ct1d_uses_w(c)) {
+        const bool staged_ok = c->causal != 0;
+        if (shared && ct1d_w_filter(c, h, c->C, staged_ok, st, launches, prof, filter_pass)) return -1;
+        for (long long s0 = 0; s0 < S; s0 += c->slices_per_chunk) {
+            const long long n = S - s0 < c->slices_per_chunk ? S - s0 : c->slices_per_chunk;
+            if (!shared && ct1d_w_filter(c, (const char *)h + (size_t)s0 * c->K * es, n, staged_ok, st, launches, prof, filter_pass))
+                return -1;
+            if (ct1d_w_body(c, (const char *)q + (size_t)s0 * c->L * es, (const char *)k + (size_t)s0 * c->L * es,
+                            (const char *)v + (size_t)s0 * c->L * es, n, shared, s0, (char *)y + (size_t)s0 * c->L * es,
+                            st, launches, prof))
+                return -1;
+        }
+        return 0;
+    }
     if (shared && filter_pass(c, (const char *)h, c->C, st, launches, prof)) return -1;
     for (long long s0 = 0; s0 < S; s0 += c->slices_per_chunk) {
         const long long n = S - s0 < c->slices_per_chunk ? S - s0 : c->slices_per_chunk;
@@ -456,10 +471,16 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
     return 0;
 }
 
+bool ct1d_uses_w(const Ct1dPlan *c)
+{
+    return ct1d_w_supported(c->log2p1, c->log2p2, c->L, c->K, c->causal, c->dtype) && !getenv("HYENAND_FORCE_GENERIC");
+}
+
 int ct1d_launches(const Ct1dPlan *c, bool shared)
 {
     const long long S = (long long)c->B * c->C;
     const long long chunks = (S + c->slices_per_chunk - 1) / c->slices_per_chunk;
+    if (ct1d_uses_w(c)) return (int)(shared ? 2 + 3 * chunks : 5 * chunks);
     return (int)(shared ? 1 + 3 * chunks : 4 * chunks);
 }
 

@@ -25,5 +25,13 @@ void ct1d_free(Ct1dPlan *c);
 int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const void *h, bool shared,
                  void *y, cudaStream_t st, int *launches, Prof *prof);
 int ct1d_launches(const Ct1dPlan *c, bool shared);
+bool ct1d_uses_w(const Ct1dPlan *c);
+
+// warp-engine kernels (ct1d_w.cu)
+bool ct1d_w_supported(int log2p1, int log2p2, int L, int K, int causal, int dtype);
+int ct1d_w_filter(Ct1dPlan *c, const void *h, long long n, bool staged_ok, cudaStream_t st, int *launches, Prof *prof,
+                  int (*fallback)(Ct1dPlan *, const char *, long long, cudaStream_t, int *, Prof *));
+int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long long n, bool shared, long long s0,
+                void *y, cudaStream_t st, int *launches, Prof *prof);
 
 }  // namespace hn

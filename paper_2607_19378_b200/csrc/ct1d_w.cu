@@ -1,0 +1,508 @@
+// Long 1-D path, warp-engine kernels (same decomposition as ct1d.cu: P = P1*P2,
+// t = t1*P2 + t2, f = f1 + P1*f2; Appendix B.3 of the paper).
+//
+//   cols_fwd_w   tile of adjacent column pairs fetched with 16-byte asynchronous copies,
+//                one warp-group per column pair: transform along t1 (upper half of the
+//                padded input is zero), separate the two real columns, multiply by the
+//                inter-pass twiddle, coalesced store of [f1][t2].
+//   hspec_w      filter only: transform each kept row along t2 in place and fold in 1/P,
+//                so the filter spectrum is computed once per filter, not once per use.
+//   core_w       one warp-group per row: transform along t2, multiply by the filter
+//                spectrum (Eq. 12), inverse transform chained in registers, undo twiddle.
+//   cols_inv_w   rebuild the mirrored half, inverse along f1 keeping t < P/2, crop, gate
+//                with q, coalesced store.
+#include "common.cuh"
+#include "ct1d.cuh"
+#include "plane_util.cuh"
+
+namespace hn {
+
+constexpr int kCtThreads = 256;
+// column pairs per tile: at least 16 (64-byte rows of bf16), one or two lines per group of lanes
+// line stride of the column kernels: 16-byte aligned and = 2 (mod 16) complex numbers, so that the
+// 16-byte accesses of neighbouring lines (tile loads and stores run across lines) hit different banks
+__host__ __device__ constexpr int ct_ls(int n) { return (n + 15) / 16 * 16 + 2; }
+__host__ __device__ constexpr int ct_tx(int tpl) { return kCtThreads / tpl > 8 ? kCtThreads / tpl : 8; }
+
+template <int BYTES> __device__ __forceinline__ void cp_async_n(void *smem_dst, const void *gmem_src)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2;\n" ::"r"(d), "l"(gmem_src), "n"(BYTES) : "memory");
+}
+
+struct TwoLevelW {
+    const float2 *coarse, *fine;
+    int lo;
+};
+__device__ __forceinline__ float2 twp_w(const TwoLevelW &t, unsigned j)
+{
+    const float2 c = __ldg(t.coarse + (j >> t.lo));
+    const float2 f = __ldg(t.fine + (j & ((1u << t.lo) - 1)));
+    return cmul(c, f);
+}
+
+// ---- columns, forward ---------------------------------------------------------------------------
+
+struct ColsFwdWArgs {
+    const void *a, *b;        // k, v (b == nullptr: plain copy of a, used for a causal filter)
+    float2 *out;              // [slices][P1/2+1][P2]
+    long long slices;
+    long long in_slice;       // elements per slice of the input (multiple of 16 bytes)
+    int len;                  // valid elements (<= P/2)
+    int log2p2;
+    const float2 *tw1;        // P1-point table
+    TwoLevelW twp;
+};
+
+template <typename T, int LOG2P1, bool HAS_B>
+__global__ void __launch_bounds__(kCtThreads, 4) ct_cols_fwd_w_kernel(ColsFwdWArgs p)
+{
+    using F = WF<LOG2P1, false>;
+    constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = F::TPL;
+    constexpr int TX = ct_tx(TPL);                         // column pairs per tile
+    constexpr int NGRP = kCtThreads / TPL;                 // groups of lanes per CTA
+    constexpr int LS = ct_ls(phys(P1) + 2);                // room for the skewed line and for 2*(P1/2+1) bins
+    constexpr int PAIRB = 2 * (int)sizeof(T);              // bytes of one column pair of one row
+    extern __shared__ float2 smem[];
+    float2 *lines = smem;
+    float2 *twt = lines + TX * LS;
+    // staged inputs, pair-major: [tensor][pair x][row t1], so that the lanes of a group (which
+    // differ in t1) read consecutive words
+    unsigned char *raw = reinterpret_cast<unsigned char *>(twt + P1);
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = F::group_mask(tid);
+    PassTw<LOG2P1, false>::build(twt, p.tw1, P1, tid, kCtThreads);
+    const PassTw<LOG2P1, false> tw{twt};
+    const int P2 = 1 << p.log2p2;
+    const int tpc = (P2 / 2) / TX;                         // tiles per slice (P2/2 is a multiple of TX)
+    const long long tiles = p.slices * tpc;
+    const unsigned char *ab = (const unsigned char *)p.a, *bb = (const unsigned char *)p.b;
+    for (long long t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const long long s = t / tpc;
+        const int c0 = (int)(t % tpc) * TX;
+        const long long base = s * p.in_slice;
+        __syncthreads();                                   // previous tile done with raw and lines
+        for (int idx = tid; idx < HP1 * TX; idx += kCtThreads) {
+            const int t1 = idx / TX, x = idx % TX;
+            const long long e0 = (long long)t1 * P2 + 2 * (c0 + x);
+            unsigned char *d = raw + ((size_t)x * HP1 + t1) * PAIRB;
+            if (e0 + 2 <= p.len) {
+                cp_async_n<PAIRB>(d, ab + (base + e0) * sizeof(T));
+                if (HAS_B) cp_async_n<PAIRB>(d + (size_t)TX * HP1 * PAIRB, bb + (base + e0) * sizeof(T));
+            } else {
+                for (int e = 0; e < 2; ++e) {
+                    const bool ok = e0 + e < p.len;
+                    reinterpret_cast<T *>(d)[e] = ok ? reinterpret_cast<const T *>(ab)[base + e0 + e] : T(0.f);
+                    if (HAS_B)
+                        reinterpret_cast<T *>(d + (size_t)TX * HP1 * PAIRB)[e] = ok ? reinterpret_cast<const T *>(bb)[base + e0 + e] : T(0.f);
+                }
+            }
+        }
+        cp_async_wait_all();
+        __syncthreads();
+        for (int x = gid; x < TX; x += NGRP) {
+        float2 *line = lines + x * LS;
+        const unsigned char *ra = raw + (size_t)x * HP1 * PAIRB;
+        const unsigned char *rb = ra + (size_t)TX * HP1 * PAIRB;
+        F::template run_to_line<PRUNE_IN>(l, m, tw, line, [&](int, int, int idx) {
+            float a0 = staged<T>(ra + (size_t)idx * PAIRB, 0, 0), a1 = staged<T>(ra + (size_t)idx * PAIRB, 0, 1);
+            if (HAS_B) {
+                a0 *= staged<T>(rb + (size_t)idx * PAIRB, 0, 0);
+                a1 *= staged<T>(rb + (size_t)idx * PAIRB, 0, 1);
+            }
+            return make_float2(a0, a1);
+        });
+        // separate the two real columns, apply W_P^(t2*f1), park both bins in the line
+        const unsigned t2 = 2u * (unsigned)(c0 + x);
+        {
+            // W_P^(t2*f1) with f1 = l + i*TPL is the product of a per-lane factor W_P^(t2*l) (one
+            // gathered lookup) and a per-line factor W_P^(t2*TPL*i) (the same address in all lanes)
+            const float2 cl0 = twp_w(p.twp, t2 * (unsigned)l), cl1 = twp_w(p.twp, (t2 + 1u) * (unsigned)l);
+            float2 A0[(F1 + TPL - 1) / TPL], A1[(F1 + TPL - 1) / TPL];
+#pragma unroll
+            for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
+                const int f1 = l + i * TPL;
+                if (f1 < F1) {
+                    const float2 z1 = line[phys(f1)], z2 = line[phys((P1 - f1) & (P1 - 1))];
+                    const float2 w0 = cmul(cl0, twp_w(p.twp, t2 * (unsigned)(i * TPL)));
+                    const float2 w1 = cmul(cl1, twp_w(p.twp, (t2 + 1u) * (unsigned)(i * TPL)));
+                    A0[i] = cmul(make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y)), w0);
+                    A1[i] = cmul(make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x)), w1);
+                }
+            }
+            __syncwarp(m);
+#pragma unroll
+            for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
+                const int f1 = l + i * TPL;
+                if (f1 < F1) *reinterpret_cast<float4 *>(line + 2 * f1) = make_float4(A0[i].x, A0[i].y, A1[i].x, A1[i].y);
+            }
+        }
+        }
+        __syncthreads();
+        float2 *dst = p.out + s * (long long)F1 * P2 + 2 * c0;
+        for (int idx = tid; idx < F1 * TX; idx += kCtThreads) {
+            const int f1 = idx / TX, x = idx % TX;
+            *reinterpret_cast<float4 *>(dst + (long long)f1 * P2 + 2 * x) =
+                *reinterpret_cast<const float4 *>(lines + x * LS + 2 * f1);
+        }
+    }
+}
+
+// ---- filter rows: spectrum in place -----------------------------------------------------------------
+
+struct HspecArgs {
+    float2 *h;                // [rows][P2]
+    long long rows;
+    float scale;
+    const float2 *tw2;
+};
+
+template <int LOG2P2>
+__global__ void __launch_bounds__(256, 2) ct_hspec_w_kernel(HspecArgs p)
+{
+    using F = WF<LOG2P2, false>;
+    constexpr int P2 = 1 << LOG2P2, TPL = F::TPL, G = 256 / TPL, LS = plane_ls(P2);
+    extern __shared__ float2 smem[];
+    float2 *twt = smem + G * LS;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = F::group_mask(tid);
+    float2 *line = smem + gid * LS;
+    PassTw<LOG2P2, false>::build(twt, p.tw2, P2, tid, 256);
+    __syncthreads();
+    const PassTw<LOG2P2, false> tw{twt};
+    for (long long r = (long long)blockIdx.x * G + gid; r < p.rows; r += (long long)gridDim.x * G) {
+        float2 *row = p.h + r * P2;
+        F::template run<PRUNE_NONE>(l, m, tw, line,
+            [&](int, int, int idx) { return row[idx]; },
+            [&](int, int, int idx, float2 v) { row[idx] = make_float2(v.x * p.scale, v.y * p.scale); });
+        __syncwarp(m);
+    }
+}
+
+// ---- core --------------------------------------------------------------------------------------------
+
+struct CoreWArgs {
+    float2 *u;                // [slices][F1][P2], in place
+    const float2 *hspec;      // [filters][F1][P2] spectra along t2 (scaled)
+    long long slices;
+    int f1n;
+    long long h_mod, h_off;
+    const float2 *tw2;
+    TwoLevelW twp;
+};
+
+template <int LOG2P2>
+__global__ void __launch_bounds__(256, 2) ct_core_w_kernel(CoreWArgs p)
+{
+    using F = WF<LOG2P2, false>;
+    using FI = WF<LOG2P2, true>;
+    constexpr int P2 = 1 << LOG2P2, TPL = F::TPL, NP = F::NP, G = 256 / TPL, LS = plane_ls(P2);
+    using PL = typename F::LastPass;
+    extern __shared__ float2 smem[];
+    float2 *twt = smem + G * LS;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = F::group_mask(tid);
+    float2 *line = smem + gid * LS;
+    PassTw<LOG2P2, false>::build(twt, p.tw2, P2, tid, 256);
+    PassTw<LOG2P2, true>::build(twt + P2, p.tw2, P2, tid, 256);
+    __syncthreads();
+    const PassTw<LOG2P2, false> tw{twt};
+    const PassTw<LOG2P2, true> twi{twt + P2};
+    const long long rows = p.slices * p.f1n;
+    for (long long r = (long long)blockIdx.x * G + gid; r < rows; r += (long long)gridDim.x * G) {
+        const long long s = r / p.f1n;
+        const int f1 = (int)(r % p.f1n);
+        const long long hs = p.h_mod ? (s + p.h_off) % p.h_mod : s;
+        float2 *row = p.u + r * P2;
+        const float2 *hrow = p.hspec + (hs * p.f1n + f1) * P2;
+        // the row is fetched with 16-byte asynchronous copies into the line (two bins per copy)
+        for (int c = l; c < P2 / 2; c += TPL) cp_async16(line + 2 * c, row + 2 * c);
+        cp_async_wait_all();
+        __syncwarp(m);
+        float2 Y[PL::IPL][PL::R];
+        {
+            // first pass reads the unskewed copy, then the usual skewed layout is used
+            using P0 = typename F::template Pass<0>;
+            float2 keep[P0::IPL][P0::R];
+            F::template pass<0, PRUNE_NONE>(l, tw,
+                [&](int, int, int idx) { return line[idx]; },
+                [&](int i, int rr, int, float2 v) { keep[i][rr] = v; });
+            __syncwarp(m);
+#pragma unroll
+            for (int i = 0; i < P0::IPL; ++i)
+#pragma unroll
+                for (int rr = 0; rr < P0::R; ++rr) line[phys((l + i * TPL) * P0::R + rr)] = keep[i][rr];
+            __syncwarp(m);
+        }
+        F::template mid<1, NP - 1, PRUNE_NONE>(l, m, tw, line);
+        F::template pass<NP - 1, PRUNE_NONE>(l, tw,
+            [&](int, int, int idx) { return line[phys(idx)]; },
+            [&](int i, int rr, int, float2 v) { Y[i][rr] = v; });
+        // spectral product with the precomputed filter spectrum (coalesced loads, no stores between)
+#pragma unroll
+        for (int i = 0; i < PL::IPL; ++i)
+#pragma unroll
+            for (int rr = 0; rr < PL::R; ++rr) Y[i][rr] = cmul(Y[i][rr], __ldg(hrow + F::last_pos(l, i, rr)));
+        __syncwarp(m);
+        FI::template pass<0, PRUNE_NONE>(l, twi,
+            [&](int i, int rr, int) { return Y[i][rr]; },
+            [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+        __syncwarp(m);
+        FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, line);
+        // undo the inter-pass twiddle W_P^(t2*f1), t2 = l + TPL*q: per-lane factor W_P^(f1*l) times a
+        // per-row factor W_P^(f1*TPL*q) whose address is the same in all lanes
+        const float2 cl = twp_w(p.twp, (unsigned)f1 * (unsigned)l);
+        FI::template pass<NP - 1, PRUNE_NONE>(l, twi,
+            [&](int, int, int idx) { return line[phys(idx)]; },
+            [&](int, int, int idx, float2 v) {
+                const float2 w = cmul(cl, twp_w(p.twp, (unsigned)f1 * (unsigned)(idx - l)));
+                row[idx] = cmulc(v, w);
+            });
+        __syncwarp(m);
+    }
+}
+
+// ---- columns, inverse ------------------------------------------------------------------------------------
+
+struct ColsInvWArgs {
+    const float2 *in;         // [slices][F1][P2]
+    const void *q;
+    void *y;
+    long long slices;
+    int len;                  // L (multiple of 16 bytes worth of elements)
+    int log2p2;
+    const float2 *tw1;
+};
+
+template <typename T, int LOG2P1>
+__global__ void __launch_bounds__(kCtThreads, 4) ct_cols_inv_w_kernel(ColsInvWArgs p)
+{
+    using FI = WF<LOG2P1, true>;
+    constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = FI::TPL;
+    constexpr int TX = ct_tx(TPL);
+    constexpr int NGRP = kCtThreads / TPL;
+    constexpr int LS = ct_ls(phys(P1) + 2);
+    extern __shared__ float2 smem[];
+    float2 *lines = smem;
+    float2 *twt = lines + TX * LS;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = FI::group_mask(tid);
+    PassTw<LOG2P1, true>::build(twt, p.tw1, P1, tid, kCtThreads);
+    const PassTw<LOG2P1, true> tw{twt};
+    const int P2 = 1 << p.log2p2;
+    const int tpc = (P2 / 2) / TX;
+    const long long tiles = p.slices * tpc;
+    const T *pq = (const T *)p.q;
+    T *py = (T *)p.y;
+    for (long long t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const long long s = t / tpc;
+        const int c0 = (int)(t % tpc) * TX;
+        const float2 *src = p.in + s * (long long)F1 * P2 + 2 * c0;
+        __syncthreads();
+        // both bins of a column pair land side by side in slot f1 of that pair's line
+        for (int idx = tid; idx < F1 * TX; idx += kCtThreads) {
+            const int f1 = idx / TX, x = idx % TX;
+            cp_async16(lines + x * LS + 2 * f1, src + (long long)f1 * P2 + 2 * x);
+        }
+        cp_async_wait_all();
+        __syncthreads();
+        for (int x = gid; x < TX; x += NGRP) {
+            float2 *line = lines + x * LS;
+            FI::template run_to_line<PRUNE_OUT, true>(l, m, tw, line, [&](int, int, int idx) {
+                const bool mirror = idx > HP1;
+                const int f1 = mirror ? P1 - idx : idx;
+                float4 ab = *reinterpret_cast<const float4 *>(line + 2 * f1);
+                if (mirror) { ab.y = -ab.y; ab.w = -ab.w; }
+                return make_float2(ab.x - ab.w, ab.y + ab.z);
+            });
+        }
+        __syncthreads();
+        // line x now holds, at position t1 < P1/2, the two real outputs of columns 2x, 2x+1
+        const long long base = s * (long long)p.len + 2 * c0;
+        for (int idx = tid; idx < HP1 * TX; idx += kCtThreads) {
+            const int t1 = idx / TX, x = idx % TX;
+            const long long tt = (long long)t1 * P2 + 2 * (c0 + x);
+            if (tt < p.len) {
+                const float2 z = lines[x * LS + phys(t1)];
+                const long long o = base + (long long)t1 * P2 + 2 * x;
+                if constexpr (sizeof(T) == 4) {
+                    const float2 qq = __ldg(reinterpret_cast<const float2 *>(pq + o));
+                    *reinterpret_cast<float2 *>(py + o) = make_float2(z.x * qq.x, z.y * qq.y);
+                } else {
+                    const __nv_bfloat162 qq = *reinterpret_cast<const __nv_bfloat162 *>(pq + o);
+                    *reinterpret_cast<__nv_bfloat162 *>(py + o) =
+                        __floats2bfloat162_rn(z.x * __low2float(qq), z.y * __high2float(qq));
+                }
+            }
+        }
+    }
+}
+
+// ---- launchers ----------------------------------------------------------------------------------------------
+
+static int ctw_sms()
+{
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+bool ct1d_w_supported(int log2p1, int log2p2, int L, int K, int causal, int dtype)
+{
+    const int es = dtype == 0 ? 4 : 2;
+    if (log2p1 < 7 || log2p1 > 10 || log2p2 < 7 || log2p2 > 10) return false;
+    if (((long long)L * es) % 16 != 0) return false;               // 16-byte copies of whole chunks
+    if (causal && ((long long)K * es) % 16 != 0) return false;
+    const int tx = ct_tx(log2p1 >= 9 ? 32 : (log2p1 == 8 ? 16 : 8));
+    if (((1 << log2p2) / 2) % tx != 0) return false;
+    return true;
+}
+
+template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWArgs &a, cudaStream_t st)
+{
+    using F = WF<LOG2P1, false>;
+    constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys(P1) + 2);
+    const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1) + (size_t)2 * (P1 / 2) * 2 * TX * sizeof(T);
+    const int P2 = 1 << a.log2p2;
+    const long long tiles = a.slices * ((P2 / 2) / TX);
+    const int grid = (int)(tiles < 4ll * ctw_sms() ? tiles : 4ll * ctw_sms());
+    if (grid <= 0) return 0;
+    if (a.b) {
+        static bool attr = false;
+        if (!attr) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); attr = true; }
+        ct_cols_fwd_w_kernel<T, LOG2P1, true><<<grid, kCtThreads, sm, st>>>(a);
+    } else {
+        static bool attr = false;
+        if (!attr) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); attr = true; }
+        ct_cols_fwd_w_kernel<T, LOG2P1, false><<<grid, kCtThreads, sm, st>>>(a);
+    }
+    return 1;
+}
+
+template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWArgs &a, cudaStream_t st)
+{
+    using F = WF<LOG2P1, true>;
+    constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys(P1) + 2);
+    const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1);
+    const int P2 = 1 << a.log2p2;
+    const long long tiles = a.slices * ((P2 / 2) / TX);
+    const int grid = (int)(tiles < 4ll * ctw_sms() ? tiles : 4ll * ctw_sms());
+    if (grid <= 0) return 0;
+    static bool attr = false;
+    if (!attr) { cudaFuncSetAttribute(ct_cols_inv_w_kernel<T, LOG2P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); attr = true; }
+    ct_cols_inv_w_kernel<T, LOG2P1><<<grid, kCtThreads, sm, st>>>(a);
+    return 1;
+}
+
+template <int LOG2P2> static int launch_rows_w_t(const HspecArgs *hs, const CoreWArgs *co, cudaStream_t st)
+{
+    using F = WF<LOG2P2, false>;
+    constexpr int P2 = 1 << LOG2P2, G = 256 / F::TPL, LS = plane_ls(P2);
+    const size_t sm = sizeof(float2) * ((size_t)G * LS + 2 * P2);
+    static bool attr = false;
+    if (!attr) {
+        cudaFuncSetAttribute(ct_hspec_w_kernel<LOG2P2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        cudaFuncSetAttribute(ct_core_w_kernel<LOG2P2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        attr = true;
+    }
+    const long long rows = hs ? hs->rows : co->slices * co->f1n;
+    const long long want = (rows + G - 1) / G;
+    const int grid = (int)(want < (long long)ctw_sms() * 2 ? want : (long long)ctw_sms() * 2);
+    if (grid <= 0) return 0;
+    if (hs) ct_hspec_w_kernel<LOG2P2><<<grid, 256, sm, st>>>(*hs);
+    else ct_core_w_kernel<LOG2P2><<<grid, 256, sm, st>>>(*co);
+    return 1;
+}
+
+#define HN_SWITCH_CTW(x, CALL)                                                                  \
+    switch (x) {                                                                                \
+    case 7: CALL(7); break; case 8: CALL(8); break; case 9: CALL(9); break; case 10: CALL(10); break; \
+    default: return -1;                                                                         \
+    }
+
+static int launch_rows_w(int log2p2, const HspecArgs *hs, const CoreWArgs *co, cudaStream_t st)
+{
+    int n = 0;
+#define CALLR(L) n = launch_rows_w_t<L>(hs, co, st)
+    HN_SWITCH_CTW(log2p2, CALLR)
+#undef CALLR
+    return n;
+}
+
+int ct1d_w_filter(Ct1dPlan *c, const void *h, long long n, bool staged_ok, cudaStream_t st, int *launches, Prof *prof,
+                  int (*fallback)(Ct1dPlan *, const char *, long long, cudaStream_t, int *, Prof *))
+{
+    const TwoLevelW twp{c->twp_coarse, c->twp_fine, c->lo};
+    if (staged_ok) {
+        ColsFwdWArgs a{};
+        a.a = h; a.b = nullptr; a.out = c->wh; a.slices = n; a.in_slice = c->K; a.len = c->K;
+        a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.twp = twp;
+        prof->begin(KID_CT_COLS_H, st);
+        int r = 0;
+#define CALLF(L) r = launch_cols_fwd_w_t<float, L>(a, st)
+#define CALLB(L) r = launch_cols_fwd_w_t<bf16, L>(a, st)
+        if (c->dtype == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
+#undef CALLF
+#undef CALLB
+        prof->end(st);
+        if (r < 0) return -1;
+        *launches += r;
+    } else if (fallback(c, (const char *)h, n, st, launches, prof)) {
+        return -1;
+    }
+    HspecArgs hs{};
+    hs.h = c->wh; hs.rows = n * ((1 << c->log2p1) / 2 + 1); hs.scale = (float)ldexp(1.0, -c->log2p); hs.tw2 = c->tw2;
+    prof->begin(KID_CT_HSPEC, st);
+    int r = launch_rows_w(c->log2p2, &hs, nullptr, st);
+    prof->end(st);
+    if (r < 0) return -1;
+    *launches += r;
+    return 0;
+}
+
+int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long long n, bool shared, long long s0,
+                void *y, cudaStream_t st, int *launches, Prof *prof)
+{
+    const TwoLevelW twp{c->twp_coarse, c->twp_fine, c->lo};
+    ColsFwdWArgs a{};
+    a.a = k; a.b = v; a.out = c->wu; a.slices = n; a.in_slice = c->L; a.len = c->L;
+    a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.twp = twp;
+    prof->begin(KID_CT_COLS_U, st);
+    int r = 0;
+#define CALLF(L) r = launch_cols_fwd_w_t<float, L>(a, st)
+#define CALLB(L) r = launch_cols_fwd_w_t<bf16, L>(a, st)
+    if (c->dtype == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
+#undef CALLF
+#undef CALLB
+    prof->end(st);
+    if (r < 0) return -1;
+    *launches += r;
+    CoreWArgs co{};
+    co.u = c->wu; co.hspec = c->wh; co.slices = n; co.f1n = (1 << c->log2p1) / 2 + 1;
+    co.h_mod = shared ? c->C : 0; co.h_off = shared ? s0 % c->C : 0;
+    co.tw2 = c->tw2; co.twp = twp;
+    prof->begin(KID_CT_CORE, st);
+    r = launch_rows_w(c->log2p2, nullptr, &co, st);
+    prof->end(st);
+    if (r < 0) return -1;
+    *launches += r;
+    ColsInvWArgs ci{};
+    ci.in = c->wu; ci.q = q; ci.y = y; ci.slices = n; ci.len = c->L; ci.log2p2 = c->log2p2; ci.tw1 = c->tw1;
+    prof->begin(KID_CT_COLS_INV, st);
+#define CALLF(L) r = launch_cols_inv_w_t<float, L>(ci, st)
+#define CALLB(L) r = launch_cols_inv_w_t<bf16, L>(ci, st)
+    if (c->dtype == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
+#undef CALLF
+#undef CALLB
+    prof->end(st);
+    if (r < 0) return -1;
+    *launches += r;
+    return 0;
+}
+
+}  // namespace hn

@@ -23,7 +23,7 @@ template <int LOG2P> struct F2Cfg {
     using FI = WF<LOG2P, true>;
     static constexpr int NG = kPlaneThreads / F::TPL;
     static constexpr int LS = plane_ls(P);
-    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * HCSS + (size_t)HP * UCSS + (size_t)NG * LS + 3 * P);
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * HCSS + (size_t)HP * UCSS + (size_t)NG * LS + 5 * P);
 };
 
 template <typename T, int LOG2P>
@@ -46,9 +46,10 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) fused2d_kernel(Fused2dArgs p
     for (int t = tid; t < P; t += kPlaneThreads) tw[t] = p.gtw[t * (p.gtw_n >> LOG2P)];
     __syncthreads();
     PlaneTw<LOG2P, false> twf;
-    twf.init(l, tw);
+    twf.init(l, tw, tw + P, tid, kPlaneThreads);
     PlaneTw<LOG2P, true> twi;
-    twi.init(l, tw);
+    twi.init(l, tw, tw + 2 * P, tid, kPlaneThreads);
+    __syncthreads();
     const unsigned char *kb = (const unsigned char *)p.k, *vb = (const unsigned char *)p.v;
     const unsigned char *hb = (const unsigned char *)p.h;
     const T *pq = (const T *)p.q;

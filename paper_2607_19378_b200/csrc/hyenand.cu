@@ -520,7 +520,7 @@ extern "C" const char *hyenand_plan_path(const hyenand_plan *p)
 
 static const char *kKernelNames[KID_COUNT] = {
     "rows_fwd(h)", "axis_fwd(h)", "rows_fwd(k*v)", "axis_fwd(k*v)", "axis_core", "axis_inv", "rows_inv",
-    "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv", "plane_fwd(h)", "plane_fwd(k*v)", "plane_inv", "fused2d"};
+    "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv", "plane_fwd(h)", "plane_fwd(k*v)", "plane_inv", "fused2d", "ct_hspec"};
 
 static double fft_flops(double lines, int log2n) { return lines * 5.0 * ldexp(1.0, log2n) * log2n; }
 
@@ -548,8 +548,20 @@ extern "C" int hyenand_plan_kernel_info(const hyenand_plan *p, int kid, int h_sh
             *launches = chunks; *bytes = S * (2 * c.L * es + F1 * P2 * c8);
             *flops = fft_flops(S * P2 / 2, c.log2p1); break;
         case KID_CT_CORE:
-            *launches = chunks; *bytes = S * 3 * F1 * P2 * c8;
-            *flops = 3 * fft_flops(S * F1, c.log2p2) + 12.0 * S * F1 * P2; break;
+            if (ct1d_uses_w(&c)) {
+                *launches = chunks; *bytes = S * 3 * F1 * P2 * c8;
+                *flops = 2 * fft_flops(S * F1, c.log2p2) + 12.0 * S * F1 * P2;
+            } else {
+                *launches = chunks; *bytes = S * 3 * F1 * P2 * c8;
+                *flops = 3 * fft_flops(S * F1, c.log2p2) + 12.0 * S * F1 * P2;
+            }
+            break;
+        case KID_CT_HSPEC:
+            if (ct1d_uses_w(&c)) {
+                *launches = h_shared ? 1 : chunks; *bytes = Sh * 2 * F1 * P2 * c8;
+                *flops = fft_flops(Sh * F1, c.log2p2);
+            }
+            break;
         case KID_CT_COLS_INV:
             *launches = chunks; *bytes = S * (F1 * P2 * c8 + 2 * c.L * es);
             *flops = fft_flops(S * P2 / 2, c.log2p1); break;

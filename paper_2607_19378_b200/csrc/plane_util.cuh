@@ -81,21 +81,33 @@ __device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, in
 }
 
 // Twiddle source of the P-point transforms of a plane kernel: registers when the plan has two
-// equal passes (the twiddles of the second pass then depend on the lane only), else the table.
+// equal passes (the twiddles of the second pass then depend on the lane only), else per-pass
+// tables in shared memory.
 template <int LOG2P, bool INV> struct PlaneTw {
     using F = WF<LOG2P, INV>;
     static constexpr bool HOIST = F::NP == 2 && WPlan<LOG2P>::R[0] == WPlan<LOG2P>::R[1];
+    static constexpr int TABLE = HOIST ? 0 : PassTw<LOG2P, INV>::TOTAL;   // shared-memory entries needed
     typename F::template Hoist<F::NP - 1> hw;
-    const float2 *table;
-    __device__ __forceinline__ void init(int l, const float2 *tw)
+    PassTw<LOG2P, INV> pt;
+    // full: N-point table in shared memory (already filled); tab: room for TABLE entries
+    __device__ __forceinline__ void init(int l, const float2 *full, float2 *tab, int tid, int nthr)
     {
-        table = tw;
-        if constexpr (HOIST) hw.load(l, tw);
+        pt.base = tab;
+        if constexpr (HOIST) hw.load(l, full);
+        else {
+            for (int s = 1; s < F::NP; ++s) {
+                const int ns = F::ns(s), rad = F::radix(s), off = PassTw<LOG2P, INV>::offset(s);
+                for (int e = tid; e < (rad - 1) * ns; e += nthr) {
+                    const int r = e / ns + 1, k = e % ns;
+                    tab[off + e] = full[r * k * ((1 << LOG2P) / (ns * rad))];
+                }
+            }
+        }
     }
-    __device__ __forceinline__ float2 operator()(int i, int r, int t) const
+    template <int S> __device__ __forceinline__ float2 get(int i, int r, int k, int t) const
     {
-        if constexpr (HOIST) return hw(i, r, t);
-        else return table[t];
+        if constexpr (HOIST) return hw.template get<S>(i, r, k, t);
+        else return pt.template get<S>(i, r, k, t);
     }
 };
 

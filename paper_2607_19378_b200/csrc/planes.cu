@@ -34,7 +34,7 @@ template <int LOG2P> struct PlaneCfg {
     static constexpr int LS = plane_ls(P);
     static constexpr int LSH = plane_ls(HP);
     static constexpr int WBUF = (NG * LS > NGH * LSH) ? NG * LS : NGH * LSH;
-    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * CSS + WBUF + P + HP);
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * CSS + WBUF + P + HP + 2 * P);
 };
 
 template <int LOG2P> __device__ __forceinline__ void load_plane_twiddles(float2 *tw, float2 *twh, const float2 *gtw, int gtw_n, int tid)
@@ -64,7 +64,8 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
     PlaneTw<LOG2P, false> twp;
-    twp.init(l, tw);
+    twp.init(l, tw, twh + HP, tid, kPlaneThreads);
+    __syncthreads();
     const T *pk = (const T *)p.a;
     const T *pv = (const T *)p.b;
     const unsigned char *kb = (const unsigned char *)p.a, *vb = (const unsigned char *)p.b;
@@ -151,7 +152,11 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
     PlaneTw<LOG2P, false> twp;
-    twp.init(l, tw);
+    twp.init(l, tw, twh + HP, tid, kPlaneThreads);
+    PassTw<LOG2P - 1, false> twc;                            // columns of the half planes
+    twc.base = twh + HP + P;
+    PassTw<LOG2P - 1, false>::build(twh + HP + P, p.gtw, p.gtw_n, tid, kPlaneThreads);
+    __syncthreads();
     const unsigned char *hb = (const unsigned char *)p.a;
     const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
     float2 *scratch = p.scratch + (long long)blockIdx.x * C::XH * HP;     // E[kx][ky'], XH lines
@@ -202,7 +207,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                 if (kx != 0) {
                     if (e == 0) {
                         float2 *d = scratch + (long long)kx * HP;
-                        FH::template run<PRUNE_NONE>(lh, mh, TableTw<HP>{twh}, lineh,
+                        FH::template run<PRUNE_NONE>(lh, mh, twc, lineh,
                             [&](int, int, int idx) { return col[idx]; },
                             [&](int, int, int idx, float2 v) { d[idx] = v; });
                     } else {
@@ -210,7 +215,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                         float2 *d = dst + (long long)kx * P;
                         using LP = typename FH::LastPass;
                         float2 O[LP::IPL][LP::R], E[LP::IPL][LP::R];
-                        FH::template run<PRUNE_NONE>(lh, mh, TableTw<HP>{twh}, lineh,
+                        FH::template run<PRUNE_NONE>(lh, mh, twc, lineh,
                             [&](int, int, int idx) { return col[idx]; },
                             [&](int i, int r, int, float2 v) { O[i][r] = v; });
                         if (!(LP::PARTIAL && lh >= LP::ITEMS)) {
@@ -231,7 +236,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                         }
                     }
                 } else {
-                    FH::template run_to_line<PRUNE_NONE>(lh, mh, TableTw<HP>{twh}, lineh,
+                    FH::template run_to_line<PRUNE_NONE>(lh, mh, twc, lineh,
                         [&](int, int, int idx) { return col[idx]; });
                     constexpr int NK = HP / TPLH;
                     if (e == 0) {
@@ -294,7 +299,8 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
     PlaneTw<LOG2P, true> twp;
-    twp.init(l, tw);
+    twp.init(l, tw, twh + HP, tid, kPlaneThreads);
+    __syncthreads();
     const T *pq = (const T *)p.a;
     T *py = (T *)p.y;
     const int Lx = p.lx, Ly = p.ly;

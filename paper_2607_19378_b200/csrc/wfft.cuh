@@ -17,18 +17,25 @@
 namespace hn {
 
 template <int LOG2N> struct WPlan;
-template <> struct WPlan<5>  { static constexpr int NP = 2, TPL = 4;  static constexpr int R[3] = {8, 4, 1}; };
-template <> struct WPlan<6>  { static constexpr int NP = 2, TPL = 8;  static constexpr int R[3] = {8, 8, 1}; };
-template <> struct WPlan<7>  { static constexpr int NP = 2, TPL = 8;  static constexpr int R[3] = {8, 16, 1}; };
-template <> struct WPlan<8>  { static constexpr int NP = 2, TPL = 16; static constexpr int R[3] = {16, 16, 1}; };
-template <> struct WPlan<9>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 8}; };
-template <> struct WPlan<10> { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 16}; };
+template <> struct WPlan<5>  { static constexpr int NP = 2, TPL = 4; static constexpr int R[3] = {8, 4, 1};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 4 : 1; } };
+template <> struct WPlan<6>  { static constexpr int NP = 2, TPL = 8; static constexpr int R[3] = {8, 8, 1};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 8 : 1; } };
+template <> struct WPlan<7>  { static constexpr int NP = 2, TPL = 8; static constexpr int R[3] = {8, 16, 1};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 16 : 1; } };
+template <> struct WPlan<8>  { static constexpr int NP = 2, TPL = 16; static constexpr int R[3] = {16, 16, 1};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 16 : s == 1 ? 16 : 1; } };
+template <> struct WPlan<9>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 8};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 8 : 8; } };
+template <> struct WPlan<10>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 16};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 8 : 16; } };
 
-// Twiddle sources.  A source is called as src(i, r, t): item i of the lane, leg r, table index t
-// (the twiddle wanted is exp(-2 pi i t / N); the engine conjugates it for inverse transforms).
+// Twiddle sources.  A source answers get<S>(i, r, k, t) for pass S: item i of the lane, leg r,
+// k = position of the item inside its sub-transform, t = index into a full N-point table (the
+// twiddle wanted is exp(-2 pi i t / N); the engine conjugates it for inverse transforms).
 template <int N> struct TableTw {               // full table of N entries in shared memory
     const float2 *tw;
-    __device__ __forceinline__ float2 operator()(int, int, int t) const { return tw[t]; }
+    template <int S> __device__ __forceinline__ float2 get(int, int, int, int t) const { return tw[t]; }
 };
 
 template <int LOG2N, bool INV> struct WF {
@@ -42,7 +49,7 @@ template <int LOG2N, bool INV> struct WF {
     {
         return TPL == 32 ? 0xffffffffu : (((1u << TPL) - 1u) << ((tid & 31) / TPL * TPL));
     }
-    __host__ __device__ static constexpr int radix(int s) { return INV ? P::R[NP - 1 - s] : P::R[s]; }
+    __host__ __device__ static constexpr int radix(int s) { return INV ? P::r(NP - 1 - s) : P::r(s); }
     __host__ __device__ static constexpr int ns(int s)
     {
         int n = 1;
@@ -82,7 +89,7 @@ template <int LOG2N, bool INV> struct WF {
                 const int k = j & (NS - 1);
 #pragma unroll
                 for (int r = 1; r < NIN; ++r) {
-                    const float2 w = tw(i, r, r * k * (N / (NS * R)));
+                    const float2 w = tw.template get<S>(i, r, k, r * k * (N / (NS * R)));
                     x[r] = INV ? cmulc(x[r], w) : cmul(x[r], w);
                 }
             }
@@ -168,7 +175,7 @@ template <int LOG2N, bool INV> struct WF {
                 for (int r = 1; r < PS::R; ++r) w[i][r] = table[r * k * (N / (PS::NS * PS::R))];
             }
         }
-        __device__ __forceinline__ float2 operator()(int i, int r, int) const { return w[i][r]; }
+        template <int S2> __device__ __forceinline__ float2 get(int i, int r, int, int) const { return w[i][r]; }
     };
 
     // Full transform whose results end up in the line itself (natural order); ends with a
@@ -190,6 +197,38 @@ template <int LOG2N, bool INV> struct WF {
             }
         }
         __syncwarp(m);
+    }
+};
+
+// Per-pass twiddle tables in shared memory, laid out [leg][k] so that the lanes of a warp (which
+// differ in k) read consecutive entries: no bank conflicts, unlike a shared N-point table.
+template <int LOG2N, bool INV> struct PassTw {
+    using F = WF<LOG2N, INV>;
+    const float2 *base;
+    __host__ __device__ static constexpr int size(int s) { return s == 0 ? 0 : (F::radix(s) - 1) * F::ns(s); }
+    __host__ __device__ static constexpr int offset(int s)
+    {
+        int o = 0;
+        for (int i = 0; i < s; ++i) o += size(i);
+        return o;
+    }
+    static constexpr int TOTAL = offset(F::NP);
+    // gtw: global table of gtw_n >= N points; all nthr threads take part; caller synchronises
+    static __device__ __forceinline__ void build(float2 *dst, const float2 *gtw, int gtw_n, int tid, int nthr)
+    {
+        constexpr int N = 1 << LOG2N;
+        const int step = gtw_n >> LOG2N;
+        for (int s = 1; s < F::NP; ++s) {
+            const int ns = F::ns(s), rad = F::radix(s), off = offset(s);
+            for (int e = tid; e < (rad - 1) * ns; e += nthr) {
+                const int r = e / ns + 1, k = e % ns;
+                dst[off + e] = gtw[r * k * (N / (ns * rad)) * step];
+            }
+        }
+    }
+    template <int S> __device__ __forceinline__ float2 get(int, int r, int k, int) const
+    {
+        return base[offset(S) + (r - 1) * F::ns(S) + k];
     }
 };
 

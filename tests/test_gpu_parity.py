@@ -119,6 +119,19 @@ def test_plane_fused_3d_shared_filter():
     check(w, q, k, v, h)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("causal,shared", [(True, True), (True, False), (False, False)])
+@pytest.mark.parametrize("L", [8192, 10000, 9001, 40000])
+def test_long_1d_path(L, causal, shared, dtype):
+    """Sequences beyond one shared-memory line take the two-pass (Cooley-Tukey) 1-D path."""
+    w, (q, k, v, h) = W.random_problem((L,), B=2, C=2, dtype=dtype, causal=causal, h_shared=shared, seed=31)
+    from paper_2607_19378_b200 import hyenand as hn
+    plan = hn.Plan(w.dims, w.B, w.C, causal=causal, dtype=w.torch_dtype)
+    assert hn.hyenand_plan_path(plan.handle) == "ct1d"
+    plan.close()
+    check(w, q, k, v, h)
+
+
 def test_tiny2d_workload_full():
     w = W.WORKLOADS["tiny2d"]
     q, k, v, h = W.make_inputs(w)
