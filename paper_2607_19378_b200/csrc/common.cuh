@@ -88,7 +88,8 @@ constexpr int kThreads = 256;             // threads per CTA of the generic kern
 struct RowsArgs {
     const void *a;        // k (or h)
     const void *b;        // v (or nullptr: plain copy of a)
-    float2 *out;          // [rows][XH]
+    float2 *out;          // [rows][pitch], P/2+1 bins written per row
+    int pitch;            // elements between rows of out (even, so rows are 16-byte aligned)
     long long rows;       // number of rows
     int len;              // valid elements per row (L3, or K3 for the filter)
     int shift;            // element m of a row goes to padded position (m - shift) mod P
@@ -99,7 +100,8 @@ struct RowsArgs {
 };
 
 struct RowsInvArgs {
-    const float2 *in;     // [rows][XH]
+    const float2 *in;     // [rows][pitch]
+    int pitch;
     const void *q;        // [rows][len]
     void *y;              // [rows][len]
     long long rows;
@@ -140,6 +142,11 @@ enum AxisMode { AXIS_FWD = 0, AXIS_INV = 1, AXIS_CORE = 2 };
 
 int launch_rows_fwd(const RowsArgs &a, int dtype, cudaStream_t st);
 int launch_rows_inv(const RowsInvArgs &a, int dtype, cudaStream_t st);
+
+// warp-engine versions (rows_w.cu) for padded row lengths 64..1024
+bool rows_w_supported(int log2p);
+int launch_rows_fwd_w(const RowsArgs &a, int dtype, cudaStream_t st);
+int launch_rows_inv_w(const RowsInvArgs &a, int dtype, cudaStream_t st);
 int launch_axis(const AxisArgs &a, int mode, cudaStream_t st);
 
 // warp-engine version of AXIS_CORE (core_w.cu); needs n_in <= P/2, h_n_in <= P, n_out <= P/2

@@ -36,6 +36,7 @@ struct hyenand_plan {
     int dims[3];
     int L[3], K[3], P[3], log2p[3];   // internal 3-axis form (leading axes of extent 1)
     int XH;                           // half-spectrum bins along the contiguous axis
+    int XP;                           // pitch of a half-spectrum row in the generic path (even)
     long long vol, kvol;              // elements per slice of q/k/v/y and of h
     int path;
     int device;
@@ -125,6 +126,7 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
         p->kvol *= p->K[ia];
     }
     p->XH = p->P[2] / 2 + 1;
+    p->XP = (p->XH + 1) & ~1;
     const long long S = (long long)B * C;
 
     if (ndim == 1 && p->log2p[2] > kMaxLineLog2) {
@@ -160,10 +162,10 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
         p->wh_a_slice = (long long)p->K[0] * p->XH * p->P[1];
         p->ws_b_slice = p->wh_b_slice = 0;
     } else {
-        p->ws_a_slice = (long long)p->L[0] * p->L[1] * p->XH;
-        p->wh_a_slice = (long long)p->K[0] * p->K[1] * p->XH;
-        p->ws_b_slice = three ? (long long)p->L[0] * p->P[1] * p->XH : 0;
-        p->wh_b_slice = three ? (long long)p->K[0] * p->P[1] * p->XH : 0;
+        p->ws_a_slice = (long long)p->L[0] * p->L[1] * p->XP;
+        p->wh_a_slice = (long long)p->K[0] * p->K[1] * p->XP;
+        p->ws_b_slice = three ? (long long)p->L[0] * p->P[1] * p->XP : 0;
+        p->wh_b_slice = three ? (long long)p->K[0] * p->P[1] * p->XP : 0;
     }
     const long long per_slice = p->ws_a_slice + p->ws_b_slice + p->wh_a_slice + p->wh_b_slice;
     const long long budget = (8ll << 30) / (long long)sizeof(float2);      // 8 GiB of workspace
@@ -200,7 +202,7 @@ static int filter_spectrum_generic(hyenand_plan *p, const char *h, long long n_s
 {
     // rows of h, then (3-D) the middle axis
     RowsArgs r{};
-    r.a = h; r.b = nullptr; r.out = p->wh_a;
+    r.a = h; r.b = nullptr; r.out = p->wh_a; r.pitch = p->XP;
     r.rows = n_slices * p->K[0] * p->K[1];
     r.len = p->K[2];
     r.shift = p->causal ? 0 : p->L[2] - 1;
@@ -208,7 +210,8 @@ static int filter_spectrum_generic(hyenand_plan *p, const char *h, long long n_s
     r.prune_in = p->causal && p->P[2] >= 2;
     r.gtw = p->gtw; r.gtw_n = p->gtw_n;
     p->prof.begin(KID_ROWS_H, st);
-    int n = launch_rows_fwd(r, p->dtype, st);
+    const bool roww = rows_w_supported(r.log2p) && !getenv("HYENAND_GENERIC_ROWS");
+    int n = roww ? launch_rows_fwd_w(r, p->dtype, st) : launch_rows_fwd(r, p->dtype, st);
     p->prof.end(st);
     if (n < 0) return -1;
     *launches += n;
@@ -216,9 +219,9 @@ static int filter_spectrum_generic(hyenand_plan *p, const char *h, long long n_s
         AxisArgs a{};
         a.in = p->wh_a; a.out = p->wh_b;
         a.n_outer = n_slices * p->K[0];
-        a.in_outer = (long long)p->K[1] * p->XH;
-        a.out_outer = (long long)p->P[1] * p->XH;
-        a.nc = p->XH; a.n_in = p->K[1]; a.n_out = p->P[1];
+        a.in_outer = (long long)p->K[1] * p->XP;
+        a.out_outer = (long long)p->P[1] * p->XP;
+        a.nc = p->XP; a.n_in = p->K[1]; a.n_out = p->P[1];
         a.shift = p->L[1] - 1; a.log2p = p->log2p[1]; a.prune_in = 0;
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         p->prof.begin(KID_AXIS_H, st);
@@ -241,11 +244,12 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         const long long n = S - s0 < p->slices_per_chunk ? S - s0 : p->slices_per_chunk;
         if (!shared && filter_spectrum_generic(p, h + (size_t)s0 * p->kvol * es, n, st, launches)) return -1;
         RowsArgs r{};
-        r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = p->ws_a;
+        r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = p->ws_a; r.pitch = p->XP;
         r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
         r.prune_in = 1; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
         p->prof.begin(KID_ROWS_U, st);
-        int c = launch_rows_fwd(r, p->dtype, st);
+        const bool roww = rows_w_supported(r.log2p) && !getenv("HYENAND_GENERIC_ROWS");
+        int c = roww ? launch_rows_fwd_w(r, p->dtype, st) : launch_rows_fwd(r, p->dtype, st);
         p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;
@@ -253,8 +257,8 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             AxisArgs a{};
             a.in = p->ws_a; a.out = p->ws_b;
             a.n_outer = n * p->L[0];
-            a.in_outer = (long long)p->L[1] * p->XH; a.out_outer = (long long)p->P[1] * p->XH;
-            a.nc = p->XH; a.n_in = p->L[1]; a.n_out = p->P[1]; a.shift = 0;
+            a.in_outer = (long long)p->L[1] * p->XP; a.out_outer = (long long)p->P[1] * p->XP;
+            a.nc = p->XP; a.n_in = p->L[1]; a.n_out = p->P[1]; a.shift = 0;
             a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
             p->prof.begin(KID_AXIS_U, st);
@@ -266,7 +270,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         {
             AxisArgs a{};
             const int ax = three ? 0 : 1;                       // core axis
-            const long long inner = three ? (long long)p->P[1] * p->XH : p->XH;
+            const long long inner = three ? (long long)p->P[1] * p->XP : p->XP;
             a.in = three ? p->ws_b : p->ws_a; a.out = (float2 *)a.in;
             a.n_outer = n;
             a.in_outer = a.out_outer = (long long)p->L[ax] * inner;
@@ -290,8 +294,8 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             AxisArgs a{};
             a.in = p->ws_b; a.out = p->ws_a;
             a.n_outer = n * p->L[0];
-            a.in_outer = (long long)p->P[1] * p->XH; a.out_outer = (long long)p->L[1] * p->XH;
-            a.nc = p->XH; a.n_in = p->P[1]; a.n_out = p->L[1]; a.shift = 0;
+            a.in_outer = (long long)p->P[1] * p->XP; a.out_outer = (long long)p->L[1] * p->XP;
+            a.nc = p->XP; a.n_in = p->P[1]; a.n_out = p->L[1]; a.shift = 0;
             a.log2p = p->log2p[1]; a.prune_in = 0;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
             p->prof.begin(KID_AXIS_INV, st);
@@ -301,11 +305,11 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             *launches += c;
         }
         RowsInvArgs ri{};
-        ri.in = p->ws_a; ri.q = q + (size_t)s0 * p->vol * es; ri.y = y + (size_t)s0 * p->vol * es;
+        ri.in = p->ws_a; ri.pitch = p->XP; ri.q = q + (size_t)s0 * p->vol * es; ri.y = y + (size_t)s0 * p->vol * es;
         ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
         ri.gtw = p->gtw; ri.gtw_n = p->gtw_n;
         p->prof.begin(KID_ROWS_INV, st);
-        c = launch_rows_inv(ri, p->dtype, st);
+        c = roww ? launch_rows_inv_w(ri, p->dtype, st) : launch_rows_inv(ri, p->dtype, st);
         p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;
@@ -601,7 +605,7 @@ extern "C" int hyenand_plan_kernel_info(const hyenand_plan *p, int kid, int h_sh
         }
         return HYENAND_OK;
     }
-    const double XH = p->XH, L0 = p->L[0], L1 = p->L[1], L2 = p->L[2], K0 = p->K[0], K1 = p->K[1], P1 = p->P[1];
+    const double XH = p->XP, L0 = p->L[0], L1 = p->L[1], L2 = p->L[2], K0 = p->K[0], K1 = p->K[1], P1 = p->P[1];
     const int ax = three ? 0 : 1;
     const double inner = three ? P1 * XH : XH;
     switch (kid) {

@@ -84,8 +84,8 @@ __global__ void __launch_bounds__(kThreads) rows_fwd_kernel(RowsArgs p)
             const long long r0 = 2 * (ch * G + g), r1 = r0 + 1;
             const float2 z1 = buf[g * LS + phys(kx)];
             const float2 z2 = buf[g * LS + phys((N - kx) & (N - 1))];
-            if (r0 < p.rows) p.out[r0 * XH + kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
-            if (r1 < p.rows) p.out[r1 * XH + kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
+            if (r0 < p.rows) p.out[r0 * p.pitch + kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
+            if (r1 < p.rows) p.out[r1 * p.pitch + kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
         }
         __syncthreads();
     }
@@ -163,8 +163,8 @@ __global__ void __launch_bounds__(kThreads) rows_inv_kernel(RowsInvArgs p)
             const bool mirror = pos > N / 2;
             const int kx = mirror ? N - pos : pos;
             float2 A = make_float2(0.f, 0.f), B = A;
-            if (r0 < p.rows) A = p.in[r0 * XH + kx];
-            if (r1 < p.rows) B = p.in[r1 * XH + kx];
+            if (r0 < p.rows) A = p.in[r0 * p.pitch + kx];
+            if (r1 < p.rows) B = p.in[r1 * p.pitch + kx];
             if (mirror) { A.y = -A.y; B.y = -B.y; }
             buf[g * LS + phys(pos)] = make_float2(A.x - B.y, A.y + B.x);
         }
