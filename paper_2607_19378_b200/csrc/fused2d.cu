@@ -15,40 +15,51 @@
 
 namespace hn {
 
+constexpr int kF2Threads = kPlaneThreads + 32;               // one extra warp for the packed column
+
 template <int LOG2P> struct F2Cfg {
     static constexpr int P = 1 << LOG2P, HP = P / 2;
     static constexpr int HCSS = P + 1;                       // filter column store stride (odd)
     static constexpr int UCSS = HP + 1;                      // k*v column store stride (odd)
     using F = WF<LOG2P, false>;
     using FI = WF<LOG2P, true>;
-    static constexpr int NG = kPlaneThreads / F::TPL;
+    static constexpr int NGM = kPlaneThreads / F::TPL;       // groups of the 16 main warps
+    static constexpr int NG = kF2Threads / F::TPL;           // all groups
     static constexpr int LS = plane_ls(P);
-    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * HCSS + (size_t)HP * UCSS + (size_t)NG * LS + 5 * P);
+    static constexpr size_t SMEM =
+        sizeof(float2) * ((size_t)HP * HCSS + 2 * (size_t)HP * UCSS + (size_t)NG * LS + 5 * P);
 };
 
+// Schedule per CTA (slices s0, s1, ... of this CTA):
+//   phase 1  all main groups: filter rows of s_i; then half of them k*v rows of s_i while the other
+//            half turns the finished columns of s_(i-1) back into rows, crops, gates and stores
+//   phase 2  main groups: one column each (filter spectrum -> registers, k*v spectrum, product,
+//            inverse); the extra warp: the packed column (bins kx = 0 and kx = P/2), its filter part
+//            and its k*v part on two groups side by side
+// so every phase keeps all groups busy; the k*v column store is double buffered.
 template <typename T, int LOG2P>
-__global__ void __launch_bounds__(kPlaneThreads, 1) fused2d_kernel(Fused2dArgs p)
+__global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
 {
     using C = F2Cfg<LOG2P>;
     using F = typename C::F;
     using FI = typename C::FI;
-    constexpr int P = C::P, HP = C::HP, TPL = F::TPL, NP = F::NP;
+    constexpr int P = C::P, HP = C::HP, TPL = F::TPL, NP = F::NP, NGM = C::NGM;
     extern __shared__ float2 smem[];
     float2 *hcs = smem;
-    float2 *ucs = hcs + HP * C::HCSS;
-    float2 *wbuf = ucs + HP * C::UCSS;
+    float2 *ucs0 = hcs + HP * C::HCSS;
+    float2 *wbuf = ucs0 + 2 * HP * C::UCSS;
     float2 *x0 = wbuf + C::NG * C::LS;                       // packed column: filter bins kx = 0 ...
     float2 *xn = x0 + P;                                     // ... and kx = P/2
     float2 *tw = xn + P;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
-    for (int t = tid; t < P; t += kPlaneThreads) tw[t] = p.gtw[t * (p.gtw_n >> LOG2P)];
+    for (int t = tid; t < P; t += kF2Threads) tw[t] = p.gtw[t * (p.gtw_n >> LOG2P)];
     __syncthreads();
     PlaneTw<LOG2P, false> twf;
-    twf.init(l, tw, tw + P, tid, kPlaneThreads);
+    twf.init(l, tw, tw + P, tid, kF2Threads);
     PlaneTw<LOG2P, true> twi;
-    twi.init(l, tw, tw + 2 * P, tid, kPlaneThreads);
+    twi.init(l, tw, tw + 2 * P, tid, kF2Threads);
     __syncthreads();
     const unsigned char *kb = (const unsigned char *)p.k, *vb = (const unsigned char *)p.v;
     const unsigned char *hb = (const unsigned char *)p.h;
@@ -58,81 +69,120 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) fused2d_kernel(Fused2dArgs p
     const long long vol = (long long)Lx * Ly, kvol = (long long)Kx * Ky;
     using PL = typename F::LastPass;
 
+    // rows back for slice sp, reading column store ub; groups g0, g0 + gstep, ... take part
+    auto rows_back = [&](long long sp, const float2 *ub, int g0, int gstep) {
+        for (int rp = g0; 2 * rp < Ly; rp += gstep) {
+            const int y0 = 2 * rp, y1 = y0 + 1;
+            const bool has1 = y1 < Ly;
+            const long long o0 = sp * vol + (long long)y0 * Lx, o1 = o0 + Lx;
+            FI::template run<PRUNE_OUT>(l, m, twi, line,
+                [&](int, int, int idx) {
+                    const int kx = idx <= HP ? idx : P - idx;
+                    if (kx == 0 || kx == HP) {
+                        const float2 A = ub[y0];
+                        const float2 B = has1 ? ub[y1] : make_float2(0.f, 0.f);
+                        return kx == 0 ? make_float2(A.x, B.x) : make_float2(A.y, B.y);
+                    }
+                    const float2 A = ub[kx * C::UCSS + y0];
+                    const float2 B = has1 ? ub[kx * C::UCSS + y1] : make_float2(0.f, 0.f);
+                    return idx <= HP ? make_float2(A.x - B.y, A.y + B.x) : make_float2(A.x + B.y, B.x - A.y);
+                },
+                [&](int, int, int idx, float2 v) {
+                    if (idx < Lx) {
+                        IO<T>::st(py, o0 + idx, v.x * IO<T>::ld(pq, o0 + idx));
+                        if (has1) IO<T>::st(py, o1 + idx, v.y * IO<T>::ld(pq, o1 + idx));
+                    }
+                });
+            __syncwarp(m);
+        }
+    };
+
+    int cur = 0;
+    long long sprev = -1;
     for (long long s = blockIdx.x; s < p.slices; s += gridDim.x) {
+        float2 *ucs = ucs0 + cur * HP * C::UCSS;
         const long long hs = p.h_mod ? (s + p.h_off) % p.h_mod : s;
         const long long sn = s + gridDim.x;
-        if (sn < p.slices) {
+        if (sn < p.slices && tid < kPlaneThreads) {
             const long long hn2 = p.h_mod ? (sn + p.h_off) % p.h_mod : sn;
             prefetch_l2(hb + hn2 * kvol * sizeof(T), kvol * sizeof(T), tid);
             prefetch_l2(kb + sn * vol * sizeof(T), vol * sizeof(T), tid);
             prefetch_l2(vb + sn * vol * sizeof(T), vol * sizeof(T), tid);
             prefetch_l2(pq + sn * vol, vol * sizeof(T), tid);
         }
-        // ---- filter rows: padded position yp holds tap my = (yp + Ly - 1) mod P --------------
-        for (int rp = gid; 2 * rp < P; rp += C::NG) {
-            const int yp0 = 2 * rp, yp1 = yp0 + 1;
-            const int my0 = (yp0 + Ly - 1) & (P - 1), my1 = (yp1 + Ly - 1) & (P - 1);
-            const bool v0 = my0 < Ky, v1 = my1 < Ky;
-            if (v0 || v1) {
-                constexpr int SLOT = ((P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;
-                static_assert(2 * SLOT <= C::LS * 8, "staged rows must fit the line");
-                unsigned char *s0 = reinterpret_cast<unsigned char *>(line), *s1 = s0 + SLOT;
-                const unsigned char *g0 = hb + (hs * kvol + (long long)my0 * Kx) * sizeof(T);
-                const unsigned char *g1 = hb + (hs * kvol + (long long)my1 * Kx) * sizeof(T);
-                if (v0) stage_row<TPL>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.h_elems * sizeof(T), l);
-                if (v1) stage_row<TPL>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.h_elems * sizeof(T), l);
-                cp_async_wait_all();
-                __syncwarp(m);
-                const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
-                F::template run_to_line<PRUNE_NONE, true>(l, m, twf, line, [&](int, int, int idx) {
-                    const int mx = (idx + Lx - 1) & (P - 1);
-                    float a = 0.f, b = 0.f;
-                    if (mx < Kx) {
-                        if (v0) a = staged<T>(s0, f0, mx);
-                        if (v1) b = staged<T>(s1, f1, mx);
+        if (gid < NGM) {
+            // ---- filter rows: padded position yp holds tap my = (yp + Ly - 1) mod P ----------
+            for (int rp = gid; 2 * rp < P; rp += NGM) {
+                const int yp0 = 2 * rp, yp1 = yp0 + 1;
+                const int my0 = (yp0 + Ly - 1) & (P - 1), my1 = (yp1 + Ly - 1) & (P - 1);
+                const bool v0 = my0 < Ky, v1 = my1 < Ky;
+                if (v0 || v1) {
+                    constexpr int SLOT = ((P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;
+                    static_assert(2 * SLOT <= C::LS * 8, "staged rows must fit the line");
+                    unsigned char *s0 = reinterpret_cast<unsigned char *>(line), *s1 = s0 + SLOT;
+                    const unsigned char *g0 = hb + (hs * kvol + (long long)my0 * Kx) * sizeof(T);
+                    const unsigned char *g1 = hb + (hs * kvol + (long long)my1 * Kx) * sizeof(T);
+                    if (v0) stage_row<TPL>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.h_elems * sizeof(T), l);
+                    if (v1) stage_row<TPL>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.h_elems * sizeof(T), l);
+                    cp_async_wait_all();
+                    __syncwarp(m);
+                    const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
+                    F::template run_to_line<PRUNE_NONE, true>(l, m, twf, line, [&](int, int, int idx) {
+                        const int mx = (idx + Lx - 1) & (P - 1);
+                        float a = 0.f, b = 0.f;
+                        if (mx < Kx) {
+                            if (v0) a = staged<T>(s0, f0, mx);
+                            if (v1) b = staged<T>(s1, f1, mx);
+                        }
+                        return make_float2(a, b);
+                    });
+                    separate_rows<LOG2P, C::HCSS>(line, hcs, yp0, yp1, l);
+                    __syncwarp(m);
+                } else {
+                    for (int kx = l; kx < HP; kx += TPL) {
+                        hcs[kx * C::HCSS + yp0] = make_float2(0.f, 0.f);
+                        hcs[kx * C::HCSS + yp1] = make_float2(0.f, 0.f);
                     }
-                    return make_float2(a, b);
-                });
-                separate_rows<LOG2P, C::HCSS>(line, hcs, yp0, yp1, l);
-                __syncwarp(m);
-            } else {
-                for (int kx = l; kx < HP; kx += TPL) {
-                    hcs[kx * C::HCSS + yp0] = make_float2(0.f, 0.f);
-                    hcs[kx * C::HCSS + yp1] = make_float2(0.f, 0.f);
                 }
             }
-        }
-        // ---- k*v rows -----------------------------------------------------------------------------
-        for (int rp = gid; 2 * rp < Ly; rp += C::NG) {
-            const int y0 = 2 * rp, y1 = y0 + 1;
-            const bool has1 = y1 < Ly;
-            const int nrow = (has1 ? 2 : 1) * Lx * (int)sizeof(T);
-            const unsigned char *gk = kb + (s * vol + (long long)y0 * Lx) * sizeof(T);
-            const unsigned char *gv = vb + (s * vol + (long long)y0 * Lx) * sizeof(T);
-            unsigned char *sk = reinterpret_cast<unsigned char *>(line);
-            unsigned char *sv = sk + C::LS * 4;
-            stage_row<TPL>(sk, gk, nrow, kb, kb + p.kv_elems * sizeof(T), l);
-            stage_row<TPL>(sv, gv, nrow, vb, vb + p.kv_elems * sizeof(T), l);
-            cp_async_wait_all();
-            __syncwarp(m);
-            const int ok = (int)((unsigned long long)gk & 15ull), ov = (int)((unsigned long long)gv & 15ull);
-            F::template run_to_line<PRUNE_IN, true>(l, m, twf, line, [&](int, int, int idx) {
-                float a = 0.f, b = 0.f;
-                if (idx < Lx) {
-                    a = staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx);
-                    if (has1) b = staged<T>(sk, ok, Lx + idx) * staged<T>(sv, ov, Lx + idx);
+            if (gid < NGM / 2) {
+                // ---- k*v rows of this slice ---------------------------------------------------------
+                for (int rp = gid; 2 * rp < Ly; rp += NGM / 2) {
+                    const int y0 = 2 * rp, y1 = y0 + 1;
+                    const bool has1 = y1 < Ly;
+                    const int nrow = (has1 ? 2 : 1) * Lx * (int)sizeof(T);
+                    const unsigned char *gk = kb + (s * vol + (long long)y0 * Lx) * sizeof(T);
+                    const unsigned char *gv = vb + (s * vol + (long long)y0 * Lx) * sizeof(T);
+                    unsigned char *sk = reinterpret_cast<unsigned char *>(line);
+                    unsigned char *sv = sk + C::LS * 4;
+                    stage_row<TPL>(sk, gk, nrow, kb, kb + p.kv_elems * sizeof(T), l);
+                    stage_row<TPL>(sv, gv, nrow, vb, vb + p.kv_elems * sizeof(T), l);
+                    cp_async_wait_all();
+                    __syncwarp(m);
+                    const int ok = (int)((unsigned long long)gk & 15ull), ov = (int)((unsigned long long)gv & 15ull);
+                    F::template run_to_line<PRUNE_IN, true>(l, m, twf, line, [&](int, int, int idx) {
+                        float a = 0.f, b = 0.f;
+                        if (idx < Lx) {
+                            a = staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx);
+                            if (has1) b = staged<T>(sk, ok, Lx + idx) * staged<T>(sv, ov, Lx + idx);
+                        }
+                        return make_float2(a, b);
+                    });
+                    separate_rows<LOG2P, C::UCSS>(line, ucs, y0, y1, l);
+                    __syncwarp(m);
                 }
-                return make_float2(a, b);
-            });
-            separate_rows<LOG2P, C::UCSS>(line, ucs, y0, y1, l);
-            __syncwarp(m);
+            } else if (sprev >= 0) {
+                // ---- rows back of the previous slice (its columns were finished last iteration) ----
+                rows_back(sprev, ucs0 + (cur ^ 1) * HP * C::UCSS, gid - NGM / 2, NGM / 2);
+            }
         }
         __syncthreads();
         // ---- columns: filter spectrum, k*v spectrum, product, inverse --------------------------
-        for (int kx = gid; kx < HP; kx += C::NG) {
-            const float2 *hc = hcs + kx * C::HCSS;
-            float2 *uc = ucs + kx * C::UCSS;
-            if (kx != 0) {
+        if (gid < NGM) {
+            for (int kx = gid; kx < HP; kx += NGM) {
+                if (kx == 0) continue;                       // the packed column belongs to the extra warp
+                const float2 *hc = hcs + kx * C::HCSS;
+                float2 *uc = ucs + kx * C::UCSS;
                 float2 H[PL::IPL][PL::R];
                 F::template run<PRUNE_NONE>(l, m, twf, line,
                     [&](int, int, int idx) { return hc[idx]; },
@@ -151,18 +201,26 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) fused2d_kernel(Fused2dArgs p
                 FI::template pass<NP - 1, PRUNE_OUT>(l, twi,
                     [&](int, int, int idx) { return line[phys(idx)]; },
                     [&](int, int, int idx, float2 v) { uc[idx] = v; });
-            } else {
-                // column 0 carries the real bins kx = 0 and kx = P/2 as one complex column: split the
-                // spectra with the Hermitian symmetry, multiply bin by bin, pack again
-                F::template run_to_line<PRUNE_NONE>(l, m, twf, line, [&](int, int, int idx) { return hc[idx]; });
+                __syncwarp(m);
+            }
+        } else if (gid < NGM + 2) {
+            // Column 0 carries the real bins kx = 0 and kx = P/2 of every row as one complex column:
+            // the spectra are split with the Hermitian symmetry, multiplied bin by bin and packed
+            // again.  Group NGM transforms and splits the filter part while group NGM+1 transforms
+            // the k*v part; they meet once, then group NGM+1 runs the inverse.
+            const unsigned m2 = (1u << (2 * TPL)) - 1u;      // lanes of the two groups (same warp)
+            if (gid == NGM) {
+                F::template run_to_line<PRUNE_NONE>(l, m, twf, line, [&](int, int, int idx) { return hcs[idx]; });
                 for (int ky = l; ky < P; ky += TPL) {
                     const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
                     x0[ky] = make_float2(0.5f * p.scale * (c1.x + c2.x), 0.5f * p.scale * (c1.y - c2.y));
                     xn[ky] = make_float2(0.5f * p.scale * (c1.y + c2.y), 0.5f * p.scale * (c2.x - c1.x));
                 }
-                __syncwarp(m);
+                __syncwarp(m2);
+            } else {
                 F::template run_to_line<PRUNE_IN>(l, m, twf, line,
-                    [&](int, int, int idx) { return idx < Ly ? uc[idx] : make_float2(0.f, 0.f); });
+                    [&](int, int, int idx) { return idx < Ly ? ucs[idx] : make_float2(0.f, 0.f); });
+                __syncwarp(m2);
                 FI::template run<PRUNE_OUT, true>(l, m, twi, line,
                     [&](int, int, int idx) {
                         const float2 c1 = line[phys(idx)], c2 = line[phys((P - idx) & (P - 1))];
@@ -171,38 +229,14 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) fused2d_kernel(Fused2dArgs p
                         const float2 y0 = cmul(u0, x0[idx]), yn = cmul(un, xn[idx]);
                         return make_float2(y0.x - yn.y, y0.y + yn.x);
                     },
-                    [&](int, int, int idx, float2 v) { uc[idx] = v; });
+                    [&](int, int, int idx, float2 v) { ucs[idx] = v; });
             }
-            __syncwarp(m);
         }
         __syncthreads();
-        // ---- rows back: complex-to-real, crop, gate, store ------------------------------------------
-        for (int rp = gid; 2 * rp < Ly; rp += C::NG) {
-            const int y0 = 2 * rp, y1 = y0 + 1;
-            const bool has1 = y1 < Ly;
-            const long long o0 = s * vol + (long long)y0 * Lx, o1 = o0 + Lx;
-            FI::template run<PRUNE_OUT>(l, m, twi, line,
-                [&](int, int, int idx) {
-                    const int kx = idx <= HP ? idx : P - idx;
-                    if (kx == 0 || kx == HP) {
-                        const float2 A = ucs[y0];
-                        const float2 B = has1 ? ucs[y1] : make_float2(0.f, 0.f);
-                        return kx == 0 ? make_float2(A.x, B.x) : make_float2(A.y, B.y);
-                    }
-                    const float2 A = ucs[kx * C::UCSS + y0];
-                    const float2 B = has1 ? ucs[kx * C::UCSS + y1] : make_float2(0.f, 0.f);
-                    return idx <= HP ? make_float2(A.x - B.y, A.y + B.x) : make_float2(A.x + B.y, B.x - A.y);
-                },
-                [&](int, int, int idx, float2 v) {
-                    if (idx < Lx) {
-                        IO<T>::st(py, o0 + idx, v.x * IO<T>::ld(pq, o0 + idx));
-                        if (has1) IO<T>::st(py, o1 + idx, v.y * IO<T>::ld(pq, o1 + idx));
-                    }
-                });
-            __syncwarp(m);
-        }
-        __syncthreads();
+        sprev = s;
+        cur ^= 1;
     }
+    if (sprev >= 0 && gid < NGM) rows_back(sprev, ucs0 + (cur ^ 1) * HP * C::UCSS, gid, NGM);
 }
 
 template <typename T, int LOG2P> static int launch_fused2d_t(const Fused2dArgs &a, cudaStream_t st)
@@ -218,7 +252,7 @@ template <typename T, int LOG2P> static int launch_fused2d_t(const Fused2dArgs &
     }
     const int grid = (int)(a.slices < sms ? a.slices : sms);
     if (grid <= 0) return 0;
-    fused2d_kernel<T, LOG2P><<<grid, kPlaneThreads, C::SMEM, st>>>(a);
+    fused2d_kernel<T, LOG2P><<<grid, kF2Threads, C::SMEM, st>>>(a);
     return 1;
 }
 
