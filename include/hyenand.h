@@ -115,6 +115,33 @@ const char *hyenand_plan_path(const hyenand_plan *plan);              /* name of
 
 
 /*
+ * Forward pass that allocates nothing (no counterpart in the paper: an integration aid).
+ *
+ * For callers that cannot allocate device memory when they need the operator -- host code running
+ * while another thread captures a CUDA graph, code inside a memory pool's own critical section, a
+ * service whose device memory was handed out completely at start-up.  There is no plan: the
+ * geometry is passed with every call, and the workspace (twiddle table and half spectra, the same
+ * passes as the general N-D path) lives in a fixed array of hyenand_noalloc_max_bytes() bytes
+ * (16 MiB) inside the library image, which every GPU that loads the library holds until the
+ * process exits.  Arguments as hyenand_create_plan + hyenand_forward_ex; q, k, v, h, y are DEVICE
+ * pointers owned by the caller.  Work is enqueued on cuda_stream; the call does not synchronise.
+ *
+ * Limits: every dims[n] <= 4096; one (b,c) slice's spectra (plus, when the filter is shared over
+ * the batch, all C filter spectra) must fit the array, else HYENAND_ERR_UNSUPPORTED with the
+ * sizes in hyenand_last_error().  Larger batches are processed in as many passes as needed.
+ * The first call on a device resolves the array's device address (cudaGetSymbolAddress) and
+ * should therefore come before any stream capture.  All calls share the one array, which keeps
+ * the previous call's contents (nothing in it needs to start at zero): calls that overlap on
+ * the GPU (different streams, or different host threads) race and give wrong results; calls
+ * on one stream are safe.  Neither cudaMalloc, cudaFree nor any allocating library routine is
+ * called.
+ */
+size_t hyenand_noalloc_max_bytes(void);
+int hyenand_forward_noalloc(int ndim, const int *dims, int B, int C, int causal, int dtype,
+                            const void *q, const void *k, const void *v, const void *h,
+                            long long h_batch_stride_elems, void *y, void *cuda_stream);
+
+/*
  * Per-kernel accounting, for benchmarks.  Kernel ids run from 0 to
  * hyenand_plan_kernel_count()-1.  hyenand_plan_kernel_info gives, for one
  * forward of this plan (h_shared: filter shared over the batch or not), the

@@ -657,3 +657,123 @@ extern "C" int hyenand_plan_kernel_time(hyenand_plan *p, int kid, double *total_
     *launches = (double)p->prof.launches[kid];
     return HYENAND_OK;
 }
+
+// ---- forward without any device allocation --------------------------------------------------
+//
+// Some callers may not allocate device memory at the point where they need the operator: code
+// running while a CUDA graph is being captured elsewhere in the process, inside a memory pool's
+// critical section, or in a service whose device memory was fully handed out at start-up.  For
+// them the workspace of this entry point is a fixed array inside the library image.
+
+#define HYENAND_NOALLOC_MAX_BYTES (16u << 20)
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[HYENAND_NOALLOC_MAX_BYTES];
+
+// device address of g_noalloc_scratch per device ordinal, resolved on that device's first call
+static void *g_noalloc_ptr[64] = {nullptr};
+
+__global__ void noalloc_twiddle_kernel(float2 *tw, int n)
+{
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < n) {
+        double sn, cs;
+        sincospi(-2.0 * (double)t / (double)n, &sn, &cs);
+        tw[t] = make_float2((float)cs, (float)sn);
+    }
+}
+
+extern "C" size_t hyenand_noalloc_max_bytes(void) { return HYENAND_NOALLOC_MAX_BYTES; }
+
+extern "C" int hyenand_forward_noalloc(int ndim, const int *dims, int B, int C, int causal, int dtype,
+                                       const void *q, const void *k, const void *v, const void *h,
+                                       long long h_batch_stride_elems, void *y, void *cuda_stream)
+{
+    g_err[0] = 0;
+    if (ndim < 1 || ndim > 3 || !dims) return fail(HYENAND_ERR_INVALID_ARG, "ndim must be 1, 2 or 3 and dims non-NULL");
+    if (B < 1 || C < 1) return fail(HYENAND_ERR_INVALID_ARG, "B and C must be >= 1");
+    if (dtype != HYENAND_F32 && dtype != HYENAND_BF16) return fail(HYENAND_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (causal != 0 && causal != 1) return fail(HYENAND_ERR_INVALID_ARG, "causal must be 0 or 1");
+    if (causal && ndim != 1) return fail(HYENAND_ERR_UNSUPPORTED, "causal kernels are defined for 1-D grids only");
+    if (!q || !k || !v || !h || !y) return fail(HYENAND_ERR_INVALID_ARG, "q, k, v, h, y must be non-NULL");
+    const void *ptrs[5] = {q, k, v, h, y};
+    for (int i = 0; i < 5; ++i)
+        if (((uintptr_t)ptrs[i]) & 15) return fail(HYENAND_ERR_INVALID_ARG, "pointer %d is not 16-byte aligned", i);
+
+    // geometry of a throw-away plan that lives on this call's stack (no host or device allocation)
+    static thread_local hyenand_plan sp;
+    memset(&sp, 0, sizeof(sp));
+    hyenand_plan *p = &sp;
+    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype;
+    p->vol = 1; p->kvol = 1;
+    for (int a = 0; a < 3; ++a) { p->L[a] = 1; p->K[a] = 1; p->P[a] = 1; p->log2p[a] = 0; }
+    for (int a = 0; a < ndim; ++a) {
+        const int ia = 3 - ndim + a;
+        if (dims[a] < 1) return fail(HYENAND_ERR_INVALID_ARG, "dims[%d] = %d must be >= 1", a, dims[a]);
+        if (dims[a] > (1 << (kMaxLineLog2 - 1)))
+            return fail(HYENAND_ERR_UNSUPPORTED, "dims[%d] = %d exceeds the limit of %d of the allocation-free entry point",
+                        a, dims[a], 1 << (kMaxLineLog2 - 1));
+        p->dims[a] = dims[a];
+        p->L[ia] = dims[a];
+        p->K[ia] = causal ? dims[a] : 2 * dims[a] - 1;
+        p->log2p[ia] = next_pow2_log(2 * dims[a] - 1);
+        p->P[ia] = 1 << p->log2p[ia];
+        p->vol *= dims[a];
+        p->kvol *= p->K[ia];
+    }
+    p->XH = p->P[2] / 2 + 1;
+    p->XP = (p->XH + 1) & ~1;
+    p->path = PATH_ND_GENERIC;
+    bool shared = false;
+    int e = check_stride(p, h_batch_stride_elems, &shared);
+    if (e) return e;
+    const bool three = p->P[0] > 1;
+    p->ws_a_slice = (long long)p->L[0] * p->L[1] * p->XP;
+    p->wh_a_slice = (long long)p->K[0] * p->K[1] * p->XP;
+    p->ws_b_slice = three ? (long long)p->L[0] * p->P[1] * p->XP : 0;
+    p->wh_b_slice = three ? (long long)p->K[0] * p->P[1] * p->XP : 0;
+    int gl = 1;
+    for (int a = 0; a < 3; ++a) if (p->log2p[a] > gl) gl = p->log2p[a];
+    p->gtw_n = 1 << gl;
+
+    // carve the fixed array: twiddles, then k*v spectra, then filter spectra (256-byte granules)
+    auto up = [](unsigned long long x) { return (x + 255ull) & ~255ull; };
+    const unsigned long long S = (unsigned long long)B * C;
+    const unsigned long long tw_b = up(sizeof(float2) * (unsigned long long)p->gtw_n);
+    const unsigned long long ua = up(sizeof(float2) * (unsigned long long)p->ws_a_slice), ub = up(sizeof(float2) * (unsigned long long)p->ws_b_slice);
+    const unsigned long long ha = up(sizeof(float2) * (unsigned long long)p->wh_a_slice), hb2 = up(sizeof(float2) * (unsigned long long)p->wh_b_slice);
+    const unsigned long long fixed = tw_b + (shared ? (unsigned long long)C * (ha + hb2) : 0ull);
+    const unsigned long long per = ua + ub + (shared ? 0ull : ha + hb2);
+    if (fixed + per > HYENAND_NOALLOC_MAX_BYTES)
+        return fail(HYENAND_ERR_UNSUPPORTED,
+                    "problem needs %llu bytes of workspace for one slice%s; the allocation-free entry point has %u bytes",
+                    fixed + per, shared ? " plus the shared filters" : "", HYENAND_NOALLOC_MAX_BYTES);
+    unsigned long long spc = (HYENAND_NOALLOC_MAX_BYTES - fixed) / per;
+    if (spc > S) spc = S;
+    p->slices_per_chunk = (long long)spc;
+    p->wh_slices = shared ? C : (long long)spc;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return fail(HYENAND_ERR_CUDA, "cannot identify the current device");
+    p->device = dev;
+    if (!g_noalloc_ptr[dev]) {
+        // once per device, with that device current: the array's name is only a host-side handle
+        void *ptr = nullptr;
+        cudaError_t ce = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+        if (ce != cudaSuccess || !ptr)
+            return fail(HYENAND_ERR_CUDA, "cudaGetSymbolAddress failed: %s", cudaGetErrorString(ce));
+        g_noalloc_ptr[dev] = ptr;
+    }
+    unsigned char *base = (unsigned char *)g_noalloc_ptr[dev];
+    unsigned long long off = 0;
+    p->gtw = (float2 *)(base + off); off += tw_b;
+    p->ws_a = (float2 *)(base + off); off += ua * spc;
+    p->ws_b = three ? (float2 *)(base + off) : nullptr; off += ub * spc;
+    p->wh_a = (float2 *)(base + off); off += ha * (unsigned long long)p->wh_slices;
+    p->wh_b = three ? (float2 *)(base + off) : nullptr; off += hb2 * (unsigned long long)p->wh_slices;
+    // the per-slice strides used by the kernels are the unrounded ones; the carve only has to be large enough
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    noalloc_twiddle_kernel<<<(p->gtw_n + 255) / 256, 256, 0, st>>>(p->gtw, p->gtw_n);
+    int launches = 1;
+    return run_forward(p, q, k, v, h, shared, y, st, &launches);
+}

@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
         L.hyenand_plan_kernel_count.argtypes = [vp]
         L.hyenand_plan_kernel_info.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_char_p),
                                                dpp, dpp, dpp]
+        L.hyenand_noalloc_max_bytes.restype = ctypes.c_size_t
+        L.hyenand_forward_noalloc.argtypes = [ctypes.c_int, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                              vp, vp, vp, vp, ll, vp, vp]
         L.hyenand_plan_set_timing.argtypes = [vp, ctypes.c_int]
         L.hyenand_plan_kernel_time.argtypes = [vp, ctypes.c_int, dpp, dpp]
         _lib = L
@@ -153,6 +156,20 @@ def hyenand_plan_kernel_time(plan: int, kernel_id: int):
     ms, n = ctypes.c_double(), ctypes.c_double()
     _check(lib().hyenand_plan_kernel_time(plan, kernel_id, ctypes.byref(ms), ctypes.byref(n)))
     return ms.value, n.value
+
+
+def hyenand_noalloc_max_bytes() -> int:
+    return int(lib().hyenand_noalloc_max_bytes())
+
+
+def hyenand_forward_noalloc(dims, B: int, C: int, causal: int, dtype: int, q, k, v, h,
+                            h_batch_stride_elems: int, y, stream=None) -> None:
+    """Forward through the entry point that allocates no device memory (fixed workspace inside
+    the library; see include/hyenand.h for its limits and the rule about overlapping calls)."""
+    arr = (ctypes.c_int * max(1, len(dims)))(*[int(d) for d in dims])
+    _check(lib().hyenand_forward_noalloc(len(dims), arr, int(B), int(C), int(causal), int(dtype),
+                                         q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
+                                         int(h_batch_stride_elems), y.data_ptr(), _stream_ptr(stream)))
 
 
 class Plan:
