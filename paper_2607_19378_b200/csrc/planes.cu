@@ -326,6 +326,11 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
         }
         __syncthreads();
         const long long ob = pl * (long long)Ly * Lx;
+        if (pl + gridDim.x < p.planes) {
+            // while the rows are transformed, bring the next plane's spectra and gate into L2
+            prefetch_l2(p.in + (pl + gridDim.x) * (long long)C::XH * P, (long long)C::XH * P * sizeof(float2), tid);
+            prefetch_l2(pq + (pl + gridDim.x) * (long long)Ly * Lx, (long long)Ly * Lx * sizeof(T), tid);
+        }
         for (int rp = gid; 2 * rp < Ly; rp += C::NG) {
             const int y0 = 2 * rp, y1 = y0 + 1;
             const bool has1 = y1 < Ly;
