@@ -60,10 +60,15 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if jobs:
         with ThreadPoolExecutor(max_workers=min(8, len(jobs))) as ex:
             list(ex.map(compile_one, jobs))
-    if jobs or not os.path.exists(LIB):
+    stale = not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs)
+    manifest = os.path.join(OBJ, "objects.txt")
+    listed = open(manifest).read() if os.path.exists(manifest) else ""
+    if jobs or stale or listed != "\n".join(objs):
         tmp = LIB + ".tmp.%d" % os.getpid()
         subprocess.check_call([NVCC, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs + ["-lcudart"])
         os.replace(tmp, LIB)
+        with open(manifest, "w") as f:
+            f.write("\n".join(objs))
     return LIB
 
 
