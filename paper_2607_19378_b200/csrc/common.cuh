@@ -76,6 +76,20 @@ struct Prof {
     }
 };
 
+// One-time-per-device guard (kernel attributes such as the dynamic shared-memory limit are per device).
+struct DevOnce {
+    unsigned long long mask = 0;
+    bool first()
+    {
+        int d = 0;
+        cudaGetDevice(&d);
+        const unsigned long long b = 1ull << (d & 63);
+        if (mask & b) return false;
+        mask |= b;
+        return true;
+    }
+};
+
 constexpr int kMaxLineLog2 = 13;          // longest line transformed in shared memory: 8192 points
 constexpr int kThreads = 256;             // threads per CTA of the generic kernels
 

@@ -18,6 +18,10 @@ __device__ __forceinline__ void cp_async8(void *smem_dst, const void *gmem_src)
     const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(d), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void cp_async8_s(unsigned smem_addr, const void *gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(smem_addr), "l"(gmem_src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
@@ -54,18 +58,34 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
     // transformed, and the next k*v lines while the next filter lines are transformed.
     constexpr int RPS = kCoreThreads / TX;                 // rows per step
     const int x = tid % TX, r0 = tid / TX;
+    // Row pos of the padded line holds filter row (pos + h_shift) mod N: rows [h_shift, h_n_in) sit at
+    // positions [0, h_n_in - h_shift), rows [0, h_shift) at [N - h_shift, N), the gap is zero.  Each
+    // thread walks its positions with running pointers (no wrap arithmetic per copy).
+    const unsigned bh_x = (unsigned)__cvta_generic_to_shared(bh + x * LS);
+    const unsigned bu_x = (unsigned)__cvta_generic_to_shared(bu + x * LS);
     auto issue_h = [&](long long t) {
         const long long o = t / tpo;
         const int c0 = (int)(t % tpo) * TX;
         const long long oh = p.h_mod ? (o + p.h_off) % p.h_mod : o;
         const float2 *hs = p.h + oh * p.h_outer + c0 + x;
         const bool inside = c0 + x < p.nc;
+        const int head = p.h_n_in - p.h_shift;             // positions [0, head) <- rows [h_shift, h_n_in)
+        const int tail0 = N - p.h_shift;                   // positions [tail0, N) <- rows [0, h_shift)
+        const long long step = (long long)RPS * p.nc;
+        if (inside) {
+            const float2 *src = hs + (long long)(p.h_shift + r0) * p.nc;
 #pragma unroll 4
-        for (int pos = r0; pos < N; pos += RPS) {
-            const int mm = (pos + p.h_shift) & (N - 1);
-            float2 *d = bh + x * LS + phys(pos);
-            if (inside && mm < p.h_n_in) cp_async8(d, hs + (long long)mm * p.nc);
-            else *d = make_float2(0.f, 0.f);
+            for (int pos = r0; pos < head; pos += RPS, src += step)
+                cp_async8_s(bh_x + 8u * (unsigned)phys(pos), src);
+            int pos = tail0 + ((r0 - tail0) & (RPS - 1));   // first position >= tail0 owned by this thread
+            src = hs + (long long)(pos - tail0) * p.nc;
+#pragma unroll 4
+            for (; pos < N; pos += RPS, src += step)
+                cp_async8_s(bh_x + 8u * (unsigned)phys(pos), src);
+            for (int z = head + ((r0 - head) & (RPS - 1)); z < tail0; z += RPS)
+                bh[x * LS + phys(z)] = make_float2(0.f, 0.f);
+        } else {
+            for (int pos = r0; pos < N; pos += RPS) bh[x * LS + phys(pos)] = make_float2(0.f, 0.f);
         }
     };
     auto issue_u = [&](long long t) {
@@ -73,12 +93,13 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         const int c0 = (int)(t % tpo) * TX;
         const float2 *us = p.in + o * p.in_outer + c0 + x;
         const bool inside = c0 + x < p.nc;
+        const int nin = inside ? p.n_in : 0;
+        const long long step = (long long)RPS * p.nc;
+        const float2 *src = us + (long long)r0 * p.nc;
+        int pos = r0;
 #pragma unroll 4
-        for (int pos = r0; pos < N / 2; pos += RPS) {
-            float2 *d = bu + x * LS + phys(pos);
-            if (inside && pos < p.n_in) cp_async8(d, us + (long long)pos * p.nc);
-            else *d = make_float2(0.f, 0.f);
-        }
+        for (; pos < nin; pos += RPS, src += step) cp_async8_s(bu_x + 8u * (unsigned)phys(pos), src);
+        for (; pos < N / 2; pos += RPS) bu[x * LS + phys(pos)] = make_float2(0.f, 0.f);
     };
     long long t = blockIdx.x;
     if (t < tiles) { issue_h(t); }
@@ -146,9 +167,10 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         {
             const long long o = t / tpo;
             const int c0 = (int)(t % tpo) * TX;
-            float2 *dst = p.out + o * p.out_outer + c0 + x;
+            float2 *dst = p.out + o * p.out_outer + c0 + x + (long long)r0 * p.nc;
+            const long long step = (long long)RPS * p.nc;
             if (c0 + x < p.nc)
-                for (int pos = r0; pos < p.n_out; pos += RPS) dst[(long long)pos * p.nc] = bu[x * LS + phys(pos)];
+                for (int pos = r0; pos < p.n_out; pos += RPS, dst += step) *dst = bu[x * LS + phys(pos)];
         }
         __syncthreads();
         if (tn < tiles) issue_u(tn);
@@ -169,8 +191,9 @@ template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t 
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms <= 0) sms = 148;
-        cudaFuncSetAttribute(axis_core_w_kernel<LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     }
+    static DevOnce attr;
+    if (attr.first()) cudaFuncSetAttribute(axis_core_w_kernel<LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     const long long tiles = a.n_outer * ((a.nc + TX - 1) / TX);
     const int grid = (int)(tiles < (long long)sms * 2 ? tiles : (long long)sms * 2);
     if (grid <= 0) return 0;

@@ -272,11 +272,10 @@ static int launch_cols_fwd_t(const ColsFwdArgs &a, bool prune, cudaStream_t st)
     const int grid = (int)(tiles < (long long)sms() * 8 ? tiles : (long long)sms() * 8);
 #define HN_LAUNCH(HASB, PR)                                                                     \
     do {                                                                                        \
-        static bool attr = false;                                                               \
-        if (!attr) {                                                                            \
+        static DevOnce attr;                                                               \
+        if (attr.first()) {                                                                            \
             cudaFuncSetAttribute(ct_cols_fwd_kernel<T, LOG2P1, HASB, PR>,                       \
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);         \
-            attr = true;                                                                        \
         }                                                                                       \
         ct_cols_fwd_kernel<T, LOG2P1, HASB, PR><<<grid, kThreads, sm, st>>>(a);                 \
     } while (0)
@@ -304,10 +303,9 @@ template <int LOG2P2> static int launch_core_t(const CoreArgs &a, cudaStream_t s
     const size_t sm = smem_for(LOG2P2, G, 2);
     const long long chunks = (a.slices * a.f1n + G - 1) / G;
     const int grid = (int)(chunks < (long long)sms() * 8 ? chunks : (long long)sms() * 8);
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (attr.first()) {
         cudaFuncSetAttribute(ct_core_kernel<LOG2P2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        attr = true;
     }
     ct_core_kernel<LOG2P2><<<grid, kThreads, sm, st>>>(a);
     return 1;
@@ -329,10 +327,9 @@ template <typename T, int LOG2P1> static int launch_cols_inv_t(const ColsInvArgs
     const int P2 = 1 << a.log2p2;
     const long long tiles = a.slices * ((P2 / 2 + TX - 1) / TX);
     const int grid = (int)(tiles < (long long)sms() * 8 ? tiles : (long long)sms() * 8);
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (attr.first()) {
         cudaFuncSetAttribute(ct_cols_inv_kernel<T, LOG2P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        attr = true;
     }
     ct_cols_inv_kernel<T, LOG2P1><<<grid, kThreads, sm, st>>>(a);
     return 1;

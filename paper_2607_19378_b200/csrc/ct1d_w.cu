@@ -373,12 +373,12 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
     const int grid = (int)(tiles < 4ll * ctw_sms() ? tiles : 4ll * ctw_sms());
     if (grid <= 0) return 0;
     if (a.b) {
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); attr = true; }
+        static DevOnce attr;
+        if (attr.first()) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }
         ct_cols_fwd_w_kernel<T, LOG2P1, true><<<grid, kCtThreads, sm, st>>>(a);
     } else {
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); attr = true; }
+        static DevOnce attr;
+        if (attr.first()) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }
         ct_cols_fwd_w_kernel<T, LOG2P1, false><<<grid, kCtThreads, sm, st>>>(a);
     }
     return 1;
@@ -393,8 +393,8 @@ template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWA
     const long long tiles = a.slices * ((P2 / 2) / TX);
     const int grid = (int)(tiles < 4ll * ctw_sms() ? tiles : 4ll * ctw_sms());
     if (grid <= 0) return 0;
-    static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(ct_cols_inv_w_kernel<T, LOG2P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); attr = true; }
+    static DevOnce attr;
+    if (attr.first()) { cudaFuncSetAttribute(ct_cols_inv_w_kernel<T, LOG2P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }
     ct_cols_inv_w_kernel<T, LOG2P1><<<grid, kCtThreads, sm, st>>>(a);
     return 1;
 }
@@ -404,11 +404,10 @@ template <int LOG2P2> static int launch_rows_w_t(const HspecArgs *hs, const Core
     using F = WF<LOG2P2, false>;
     constexpr int P2 = 1 << LOG2P2, G = 256 / F::TPL, LS = plane_ls(P2);
     const size_t sm = sizeof(float2) * ((size_t)G * LS + 2 * P2);
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (attr.first()) {
         cudaFuncSetAttribute(ct_hspec_w_kernel<LOG2P2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
         cudaFuncSetAttribute(ct_core_w_kernel<LOG2P2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        attr = true;
     }
     const long long rows = hs ? hs->rows : co->slices * co->f1n;
     const long long want = (rows + G - 1) / G;

@@ -248,8 +248,9 @@ template <typename T, int LOG2P> static int launch_fused2d_t(const Fused2dArgs &
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms <= 0) sms = 148;
-        cudaFuncSetAttribute(fused2d_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
     }
+    static DevOnce attr;
+    if (attr.first()) cudaFuncSetAttribute(fused2d_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
     const int grid = (int)(a.slices < sms ? a.slices : sms);
     if (grid <= 0) return 0;
     fused2d_kernel<T, LOG2P><<<grid, kF2Threads, C::SMEM, st>>>(a);

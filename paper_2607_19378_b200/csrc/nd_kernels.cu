@@ -102,11 +102,10 @@ static int launch_rows_fwd_t(const RowsArgs &a, cudaStream_t st)
     if (grid <= 0) return 0;
 #define HN_LAUNCH(HASB, PR)                                                                     \
     do {                                                                                        \
-        static bool attr = false;                                                               \
-        if (!attr) {                                                                            \
+        static DevOnce attr;                                                               \
+        if (attr.first()) {                                                                            \
             cudaFuncSetAttribute(rows_fwd_kernel<T, LOG2P, HASB, PR>,                           \
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);         \
-            attr = true;                                                                        \
         }                                                                                       \
         rows_fwd_kernel<T, LOG2P, HASB, PR><<<grid, kThreads, sm, st>>>(a);                     \
     } while (0)
@@ -190,10 +189,9 @@ static int launch_rows_inv_t(const RowsInvArgs &a, cudaStream_t st)
     const long long chunks = (pairs + G - 1) / G;
     const int grid = (int)(chunks < (long long)sm_count() * 8 ? chunks : (long long)sm_count() * 8);
     if (grid <= 0) return 0;
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (attr.first()) {
         cudaFuncSetAttribute(rows_inv_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        attr = true;
     }
     rows_inv_kernel<T, LOG2P><<<grid, kThreads, sm, st>>>(a);
     return 1;
@@ -285,10 +283,9 @@ static int launch_axis_t(const AxisArgs &a, cudaStream_t st)
     const long long tiles = a.n_outer * ((a.nc + TX - 1) / TX);
     const int grid = (int)(tiles < (long long)sm_count() * 8 ? tiles : (long long)sm_count() * 8);
     if (grid <= 0) return 0;
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (attr.first()) {
         cudaFuncSetAttribute(axis_kernel<MODE, LOG2P, PRUNE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        attr = true;
     }
     axis_kernel<MODE, LOG2P, PRUNE><<<grid, kThreads, sm, st>>>(a);
     return 1;

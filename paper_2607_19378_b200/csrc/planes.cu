@@ -390,12 +390,11 @@ template <typename T, int LOG2P> static int launch_plane_t(const PlaneArgs &a, i
     using C = PlaneCfg<LOG2P>;
     const int grid = plane_grid(a.planes);
     if (grid <= 0) return 0;
-    static bool attr[3] = {false, false, false};
+    static DevOnce attr[3];
     void (*fn)(PlaneArgs) = which == PLANE_U ? uplane_kernel<T, LOG2P>
                           : which == PLANE_H ? hplane_kernel<T, LOG2P> : plane_inv_kernel<T, LOG2P>;
-    if (!attr[which]) {
+    if (attr[which].first()) {
         cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
-        attr[which] = true;
     }
     fn<<<grid, kPlaneThreads, C::SMEM, st>>>(a);
     return 1;

@@ -152,10 +152,9 @@ template <typename T, int LOG2P> static int launch_rows_fwd_w_t(const RowsArgs &
     if (grid <= 0) return 0;
 #define HN_LAUNCH(MODE)                                                                                  \
     do {                                                                                                 \
-        static bool attr = false;                                                                        \
-        if (!attr) {                                                                                     \
+        static DevOnce attr;                                                                        \
+        if (attr.first()) {                                                                                     \
             cudaFuncSetAttribute(rows_fwd_w_kernel<T, LOG2P, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); \
-            attr = true;                                                                                 \
         }                                                                                                \
         rows_fwd_w_kernel<T, LOG2P, MODE><<<grid, kRowThreads, sm, st>>>(a);                             \
     } while (0)
@@ -174,10 +173,9 @@ template <typename T, int LOG2P> static int launch_rows_inv_w_t(const RowsInvArg
     const long long want = ((a.rows + 1) / 2 + G - 1) / G;
     const int grid = (int)(want < 2ll * rows_sms() ? want : 2ll * rows_sms());
     if (grid <= 0) return 0;
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (attr.first()) {
         cudaFuncSetAttribute(rows_inv_w_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        attr = true;
     }
     rows_inv_w_kernel<T, LOG2P><<<grid, kRowThreads, sm, st>>>(a);
     return 1;
