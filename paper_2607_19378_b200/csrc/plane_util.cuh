@@ -57,6 +57,14 @@ template <typename T> __device__ __forceinline__ float staged(const unsigned cha
     else return __bfloat162float(*reinterpret_cast<const bf16 *>(row + off + 2 * i));
 }
 
+// Zero elements [from, to) of a staged row (element i sits at row + off + i*sizeof(T)); used to blank
+// the padding positions once so that the transform's input functor needs no bounds test.
+template <typename T, int TPL>
+__device__ __forceinline__ void zero_staged(unsigned char *row, int off, int from, int to, int l)
+{
+    for (int i = from + l; i < to; i += TPL) *reinterpret_cast<T *>(row + off + (int)sizeof(T) * i) = T(0.f);
+}
+
 // Separate the spectra of the two real rows packed in one complex transform (results in
 // `line`, natural order) and scatter them into column store rows y0, y1.
 template <int LOG2P, int CSS>
