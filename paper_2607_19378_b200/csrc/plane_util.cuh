@@ -71,20 +71,21 @@ template <int LOG2P, int CSS>
 __device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, int y0, int y1, int l)
 {
     constexpr int P = 1 << LOG2P, HP = P / 2, TPL = WF<LOG2P, false>::TPL;
-    float a0 = 0.f, b0 = 0.f;
-    for (int kx = l; kx <= HP; kx += TPL) {
+    // bins 1 .. HP-1 (lane 0's first entry, bin 0, is overwritten below)
+#pragma unroll
+    for (int t = 0; t < HP / TPL; ++t) {
+        const int kx = l + t * TPL;
         const float2 z1 = line[phys(kx)];
         const float2 z2 = line[phys((P - kx) & (P - 1))];
-        const float2 A = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
-        const float2 B = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
-        if (kx == 0) { a0 = A.x; b0 = B.x; }
-        else if (kx == HP) {                                 // same lane as kx == 0
-            cs[y0] = make_float2(a0, A.x);
-            cs[y1] = make_float2(b0, B.x);
-        } else {
-            cs[kx * CSS + y0] = A;
-            cs[kx * CSS + y1] = B;
-        }
+        cs[kx * CSS + y0] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
+        cs[kx * CSS + y1] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
+    }
+    __syncwarp(WF<LOG2P, false>::group_mask(threadIdx.x));
+    if (l == 0) {
+        // the two purely real bins (kx = 0 and kx = P/2) of each row share column 0
+        const float2 z0 = line[phys(0)], zh = line[phys(HP)];
+        cs[y0] = make_float2(z0.x, zh.x);
+        cs[y1] = make_float2(z0.y, zh.y);
     }
 }
 

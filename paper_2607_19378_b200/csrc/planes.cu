@@ -93,14 +93,22 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
                 cp_async_wait_all();
                 __syncwarp(m);
                 const int ok = (int)((unsigned long long)gk & 15ull), ov = (int)((unsigned long long)gv & 15ull);
-                F::template run_to_line<PRUNE_IN, true>(l, m, twp, line, [&](int, int, int idx) {
-                    float a = 0.f, b = 0.f;
-                    if (idx < Lx) {
-                        a = staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx);
-                        if (has1) b = staged<T>(sk, ok, Lx + idx) * staged<T>(sv, ov, Lx + idx);
-                    }
-                    return make_float2(a, b);
-                });
+                if (Lx == HP && has1) {
+                    // full rows: no bounds tests in the input functor
+                    F::template run_to_line<PRUNE_IN, true>(l, m, twp, line, [&](int, int, int idx) {
+                        return make_float2(staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx),
+                                           staged<T>(sk, ok, HP + idx) * staged<T>(sv, ov, HP + idx));
+                    });
+                } else {
+                    F::template run_to_line<PRUNE_IN, true>(l, m, twp, line, [&](int, int, int idx) {
+                        float a = 0.f, b = 0.f;
+                        if (idx < Lx) {
+                            a = staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx);
+                            if (has1) b = staged<T>(sk, ok, Lx + idx) * staged<T>(sv, ov, Lx + idx);
+                        }
+                        return make_float2(a, b);
+                    });
+                }
                 separate_rows<LOG2P, C::CSS>(line, cs, y0, y1, l);
                 __syncwarp(m);
             }
@@ -337,15 +345,18 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
             const long long o0 = ob + (long long)y0 * Lx, o1 = o0 + Lx;
             FI::template run<PRUNE_OUT>(l, m, twp, line,
                 [&](int, int, int idx) {
-                    const int kx = idx <= HP ? idx : P - idx;
-                    if (kx == 0 || kx == HP) {
-                        const float2 A = cs[y0];
-                        const float2 B = has1 ? cs[y1] : make_float2(0.f, 0.f);
-                        return kx == 0 ? make_float2(A.x, B.x) : make_float2(A.y, B.y);
-                    }
-                    const float2 A = cs[kx * C::CSS + y0];
-                    const float2 B = has1 ? cs[kx * C::CSS + y1] : make_float2(0.f, 0.f);
-                    return idx <= HP ? make_float2(A.x - B.y, A.y + B.x) : make_float2(A.x + B.y, B.x - A.y);
+                    // branch-free merge of two half spectra into one complex row (column 0 is packed)
+                    const bool mirror = idx > HP;
+                    const int kx = mirror ? P - idx : idx;
+                    const int col = kx == HP ? 0 : kx;
+                    const float2 A = cs[col * C::CSS + y0];
+                    float2 B = cs[col * C::CSS + y1];
+                    if (!has1) B = make_float2(0.f, 0.f);
+                    const float sg = mirror ? -1.f : 1.f;
+                    float2 g = make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
+                    g = kx == 0 ? make_float2(A.x, B.x) : g;
+                    g = kx == HP ? make_float2(A.y, B.y) : g;
+                    return g;
                 },
                 [&](int, int, int idx, float2 v) {
                     if (idx < Lx) {
