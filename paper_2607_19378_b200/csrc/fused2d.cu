@@ -130,14 +130,14 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
                     cp_async_wait_all();
                     __syncwarp(m);
                     const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
-                    F::template run_to_line<PRUNE_NONE, true>(l, m, twf, line, [&](int, int, int idx) {
-                        const int mx = (idx + Lx - 1) & (P - 1);
-                        float a = 0.f, b = 0.f;
-                        if (mx < Kx) {
-                            if (v0) a = staged<T>(s0, f0, mx);
-                            if (v1) b = staged<T>(s1, f1, mx);
-                        }
-                        return make_float2(a, b);
+                    // blank the padding taps (and a missing row) once: the input functor is branch-free
+                    zero_staged<T, TPL>(s0, f0, v0 ? Kx : 0, P, l);
+                    zero_staged<T, TPL>(s1, f1, v1 ? Kx : 0, P, l);
+                    __syncwarp(m);
+                    const int cw = (l + Lx - 1) & (P - 1);
+                    F::template run_to_line<PRUNE_NONE, true>(l, m, twf, line, [&](int i, int r, int) {
+                        const int mx = (cw + i * TPL + r * (P / F::template Pass<0>::R)) & (P - 1);
+                        return make_float2(staged<T>(s0, f0, mx), staged<T>(s1, f1, mx));
                     });
                     separate_rows<LOG2P, C::HCSS>(line, hcs, yp0, yp1, l);
                     __syncwarp(m);

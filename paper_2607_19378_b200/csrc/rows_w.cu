@@ -57,19 +57,30 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
         cp_async_wait_all();
         __syncwarp(m);
         const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
-        F::template run_to_line<PR, true>(l, m, tw, line, [&](int, int, int idx) {
-            const int mm = MODE == 1 ? ((idx + p.shift) & (P - 1)) : idx;
-            float a = 0.f, b = 0.f;
-            if (mm < p.len) {
-                a = staged<T>(s, f0, mm);
-                if (has1) b = staged<T>(s + SLOT, f1, mm);
-                if (MODE == 0) {
-                    a *= staged<T>(s + 2 * SLOT, fb0, mm);
-                    if (has1) b *= staged<T>(s + 3 * SLOT, fb1, mm);
+        if (MODE == 1) {
+            // filter rows: blank the padding taps (and a missing second row) once, then no bounds tests
+            zero_staged<T, TPL>(s, f0, p.len, P, l);
+            zero_staged<T, TPL>(s + SLOT, f1, has1 ? p.len : 0, P, l);
+            __syncwarp(m);
+            const int cw = (l + p.shift) & (P - 1);
+            F::template run_to_line<PR, true>(l, m, tw, line, [&](int i, int r, int) {
+                const int mm = (cw + i * TPL + r * (P / F::template Pass<0>::R)) & (P - 1);
+                return make_float2(staged<T>(s, f0, mm), staged<T>(s + SLOT, f1, mm));
+            });
+        } else {
+            F::template run_to_line<PR, true>(l, m, tw, line, [&](int, int, int idx) {
+                float a = 0.f, b = 0.f;
+                if (idx < p.len) {
+                    a = staged<T>(s, f0, idx);
+                    if (has1) b = staged<T>(s + SLOT, f1, idx);
+                    if (MODE == 0) {
+                        a *= staged<T>(s + 2 * SLOT, fb0, idx);
+                        if (has1) b *= staged<T>(s + 3 * SLOT, fb1, idx);
+                    }
                 }
-            }
-            return make_float2(a, b);
-        });
+                return make_float2(a, b);
+            });
+        }
         float2 *o0 = p.out + r0 * p.pitch, *o1 = p.out + r1 * p.pitch;
         for (int kx = l; kx <= HP; kx += TPL) {
             const float2 z1 = line[phys(kx)], z2 = line[phys((P - kx) & (P - 1))];
