@@ -47,7 +47,6 @@ struct hyenand_plan {
     long long wh_slices;              // slices the filter workspace holds
     float2 *gtw;
     int gtw_n;
-    float2 *plane_scratch;
     // long 1-D path
     Ct1dPlan ct;
     // host-staging for hyenand_forward_host
@@ -88,7 +87,7 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
     int cur = 0;
     cudaGetDevice(&cur);
     if (cur != p->device) cudaSetDevice(p->device);
-    cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw); cudaFree(p->plane_scratch);
+    cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw);
     ct1d_free(&p->ct);
     for (int i = 0; i < 5; ++i) cudaFree(p->stage[i]);
     p->prof.destroy();
@@ -187,8 +186,6 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     if (!e) e = dev_alloc(p, (void **)&p->ws_a, sizeof(float2) * p->ws_a_slice * spc);
     if (!e && p->ws_b_slice) e = dev_alloc(p, (void **)&p->ws_b, sizeof(float2) * p->ws_b_slice * spc);
     if (!e) e = dev_alloc(p, (void **)&p->wh_a, sizeof(float2) * p->wh_a_slice * p->wh_slices);
-    if (!e && p->path == PATH_PLANES3D)
-        e = dev_alloc(p, (void **)&p->plane_scratch, sizeof(float2) * plane_scratch_elems(p->log2p[2]));
     if (!e && p->wh_b_slice) e = dev_alloc(p, (void **)&p->wh_b, sizeof(float2) * p->wh_b_slice * p->wh_slices);
     if (!e && cudaMemcpy(p->gtw, tw.data(), sizeof(float2) * p->gtw_n, cudaMemcpyHostToDevice) != cudaSuccess)
         e = fail(HYENAND_ERR_CUDA, "twiddle upload failed: %s", cudaGetErrorString(cudaGetLastError()));
@@ -325,7 +322,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
     const long long nc = (long long)p->XH * p->P[1];
     auto filter = [&](const char *hp, long long n) -> int {
         PlaneArgs a{};
-        a.a = hp; a.out = p->wh_a; a.scratch = p->plane_scratch; a.planes = n * p->K[0];
+        a.a = hp; a.out = p->wh_a; a.planes = n * p->K[0];
         a.a_elems = n * p->kvol;
         a.lx = p->L[2]; a.ly = p->L[1]; a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         p->prof.begin(KID_PLANE_H, st);

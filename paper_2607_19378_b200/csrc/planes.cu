@@ -7,10 +7,10 @@
 //   uplane     k*v plane: gate, zero-pad, real-to-complex along x (two real rows
 //              per complex transform), transpose through a shared-memory column
 //              store, complex transform along y.  Output lines are [kx][ky].
-//   hplane     filter plane, which has twice the rows: handled as the rows at even
-//              and at odd padded positions (two half planes of the size of a k*v
-//              plane) joined by one radix-2 step; the first half's spectrum waits
-//              in a per-CTA global scratch that stays in L2.
+//   hplane     filter plane, which has twice the rows and columns: the even and the odd
+//              bins along x are produced one after the other (one radix-2
+//              decimation-in-frequency step applied to the taps as they are read), each
+//              half filling a column store of the size of a k*v plane's.
 //   plane_inv  inverse along y (keeping the cropped rows), inverse complex-to-real
 //              along x, crop, output gate q, store.
 //
@@ -139,13 +139,36 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
 
 // ---- filter planes ----------------------------------------------------------------------------------
 
+// Spectra of two real rows packed in one half-length transform of the ODD bins (kx = 2k+1): the
+// partner of bin k is bin HP-1-k.  Results go to column k of the column store, rows y0 and y1.
+template <int LOG2H, int CSS>
+__device__ __forceinline__ void separate_rows_odd(const float2 *line, float2 *cs, int y0, int y1, int l)
+{
+    constexpr int H = 1 << LOG2H, TPL = WF<LOG2H, false>::TPL;
+#pragma unroll
+    for (int t = 0; t < H / 2 / TPL; ++t) {
+        const int k = l + t * TPL;
+        const float2 z1 = line[phys(k)];
+        const float2 z2 = line[phys(H - 1 - k)];
+        cs[k * CSS + y0] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
+        cs[k * CSS + y1] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
+    }
+}
+
+// A filter plane has P rows of P taps: twice the rows and columns of a k*v plane, too much for one
+// column store.  The transform along x is split by one decimation-in-frequency step: the even bins
+// of a row are the half-length transform of f[x] + f[x + P/2], the odd bins that of
+// (f[x] - f[x + P/2]) W_P^x.  Each half (e = 0: even kx, e = 1: odd kx) fills a column store of
+// P/4 columns by P rows, whose columns are then transformed along y and written out as whole lines.
 template <typename T, int LOG2P>
 __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
 {
     using C = PlaneCfg<LOG2P>;
     using F = typename C::F;
     using FH = typename C::FH;
-    constexpr int P = C::P, HP = C::HP, TPL = F::TPL, TPLH = FH::TPL;
+    constexpr int P = C::P, HP = C::HP, QP = P / 4, TPL = F::TPL, TPLH = FH::TPL;
+    constexpr int CSH = P + 1;                               // column-store stride (odd): QP columns of P rows
+    static_assert(QP * CSH <= HP * C::CSS, "column store of a half fits the plane buffer");
     extern __shared__ float2 smem[];
     float2 *cs = smem;
     float2 *wbuf = cs + HP * C::CSS;
@@ -161,132 +184,102 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     __syncthreads();
     PlaneTw<LOG2P, false> twp;
     twp.init(l, tw, twh + HP, tid, kPlaneThreads);
-    PassTw<LOG2P - 1, false> twc;                            // columns of the half planes
-    twc.base = twh + HP + P;
+    PassTw<LOG2P - 1, false> twr;                            // half-length rows
+    twr.base = twh + HP + P;
     PassTw<LOG2P - 1, false>::build(twh + HP + P, p.gtw, p.gtw_n, tid, kPlaneThreads);
     __syncthreads();
     const unsigned char *hb = (const unsigned char *)p.a;
     const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
-    float2 *scratch = p.scratch + (long long)blockIdx.x * C::XH * HP;     // E[kx][ky'], XH lines
+    constexpr int R0 = FH::template Pass<0>::R;
+    const int c0 = (lh + Lx - 1) & (P - 1);                  // tap of padded position x: (x + Lx - 1) mod P
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const long long ib = pl * (long long)Ky * Kx;
         float2 *dst = p.out + pl * (long long)C::XH * P;
         if (pl + gridDim.x < p.planes)
             prefetch_l2(hb + (pl + gridDim.x) * (long long)Ky * Kx * sizeof(T), (long long)Ky * Kx * sizeof(T), tid);
         for (int e = 0; e < 2; ++e) {
-            // rows at padded positions yp = 2*yy + e, i.e. taps my = (yp + Ly - 1) mod P
-            for (int rp = gid; 2 * rp < HP; rp += C::NG) {
-                const int yy0 = 2 * rp, yy1 = yy0 + 1;
-                const int my0 = (2 * yy0 + e + Ly - 1) & (P - 1), my1 = (2 * yy1 + e + Ly - 1) & (P - 1);
+            // rows: padded row y holds tap row (y + Ly - 1) mod P; two rows per transform
+            for (int rp = gidh; rp < HP; rp += C::NGH) {
+                const int y0 = 2 * rp, y1 = y0 + 1;
+                const int my0 = (y0 + Ly - 1) & (P - 1), my1 = (y1 + Ly - 1) & (P - 1);
                 const bool v0 = my0 < Ky, v1 = my1 < Ky;
-                const long long o0 = ib + (long long)my0 * Kx, o1 = ib + (long long)my1 * Kx;
                 if (v0 || v1) {
+                    // STAGED: both tap rows are fetched with 16-byte copies into the line itself, which
+                    // the first pass reads before anything is written to it; 4-byte taps do not fit the
+                    // half-length line and are read from global memory (L2) directly
+                    constexpr bool STAGED = sizeof(T) == 2;
                     constexpr int SLOT = ((C::P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;   // bytes kept per staged row
-                    static_assert(2 * SLOT <= C::LS * 8, "staged rows must fit the line");
-                    unsigned char *s0 = reinterpret_cast<unsigned char *>(line), *s1 = s0 + SLOT;
-                    const unsigned char *g0 = hb + o0 * sizeof(T), *g1 = hb + o1 * sizeof(T);
-                    if (v0) stage_row<TPL>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), l);
-                    if (v1) stage_row<TPL>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), l);
-                    cp_async_wait_all();
-                    __syncwarp(m);
+                    static_assert(!STAGED || 2 * SLOT <= C::LSH * 8, "staged rows must fit the line");
+                    unsigned char *s0 = reinterpret_cast<unsigned char *>(lineh), *s1 = s0 + SLOT;
+                    const unsigned char *g0 = hb + (ib + (long long)my0 * Kx) * sizeof(T);
+                    const unsigned char *g1 = hb + (ib + (long long)my1 * Kx) * sizeof(T);
                     const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
-                    // blank the padding taps (and a missing row) once: the input functor is branch-free
-                    zero_staged<T, TPL>(s0, f0, v0 ? Kx : 0, P, l);
-                    zero_staged<T, TPL>(s1, f1, v1 ? Kx : 0, P, l);
-                    __syncwarp(m);
-                    const int c0 = (l + Lx - 1) & (P - 1);
-                    F::template run_to_line<PRUNE_NONE, true>(l, m, twp, line, [&](int i, int r, int) {
-                        const int mx = (c0 + i * TPL + r * (P / F::template Pass<0>::R)) & (P - 1);
-                        return make_float2(staged<T>(s0, f0, mx), staged<T>(s1, f1, mx));
-                    });
-                    separate_rows<LOG2P, C::CSS>(line, cs, yy0, yy1, l);
-                    __syncwarp(m);
+                    if constexpr (STAGED) {
+                        if (v0) stage_row<TPLH>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
+                        if (v1) stage_row<TPLH>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
+                        cp_async_wait_all();
+                        __syncwarp(mh);
+                        // blank the padding taps (and a missing row) once: the input functors are branch-free
+                        zero_staged<T, TPLH>(s0, f0, v0 ? Kx : 0, P, lh);
+                        zero_staged<T, TPLH>(s1, f1, v1 ? Kx : 0, P, lh);
+                        __syncwarp(mh);
+                    }
+                    const int n0 = v0 ? Kx : 0, n1 = v1 ? Kx : 0;
+                    auto tap0 = [&](int mx) -> float {
+                        if constexpr (STAGED) return staged<T>(s0, f0, mx);
+                        else return mx < n0 ? IO<T>::ld(reinterpret_cast<const T *>(g0), mx) : 0.f;
+                    };
+                    auto tap1 = [&](int mx) -> float {
+                        if constexpr (STAGED) return staged<T>(s1, f1, mx);
+                        else return mx < n1 ? IO<T>::ld(reinterpret_cast<const T *>(g1), mx) : 0.f;
+                    };
+                    if (e == 0) {
+                        FH::template run_to_line<PRUNE_NONE, STAGED>(lh, mh, twr, lineh, [&](int i, int r, int) {
+                            const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
+                            return make_float2(tap0(ma) + tap0(mb), tap1(ma) + tap1(mb));
+                        });
+                        separate_rows<LOG2P - 1, CSH>(lineh, cs, y0, y1, lh);
+                    } else {
+                        FH::template run_to_line<PRUNE_NONE, STAGED>(lh, mh, twr, lineh, [&](int i, int r, int idx) {
+                            const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
+                            return cmul(make_float2(tap0(ma) - tap0(mb), tap1(ma) - tap1(mb)), tw[idx]);
+                        });
+                        separate_rows_odd<LOG2P - 1, CSH>(lineh, cs, y0, y1, lh);
+                    }
+                    __syncwarp(mh);
                 } else {
-                    for (int kx = l; kx < HP; kx += TPL) {
-                        cs[kx * C::CSS + yy0] = make_float2(0.f, 0.f);
-                        cs[kx * C::CSS + yy1] = make_float2(0.f, 0.f);
+                    for (int k = lh; k < QP; k += TPLH) {
+                        cs[k * CSH + y0] = make_float2(0.f, 0.f);
+                        cs[k * CSH + y1] = make_float2(0.f, 0.f);
                     }
                 }
             }
             __syncthreads();
-            // columns: HP-point transforms over yy
-            for (int kx = gidh; kx < HP; kx += C::NGH) {
-                const float2 *col = cs + kx * C::CSS;
-                if (kx != 0) {
-                    if (e == 0) {
-                        float2 *d = scratch + (long long)kx * HP;
-                        FH::template run<PRUNE_NONE>(lh, mh, twc, lineh,
-                            [&](int, int, int idx) { return col[idx]; },
-                            [&](int, int, int idx, float2 v) { d[idx] = v; });
-                    } else {
-                        const float2 *es = scratch + (long long)kx * HP;
-                        float2 *d = dst + (long long)kx * P;
-                        using LP = typename FH::LastPass;
-                        float2 O[LP::IPL][LP::R], E[LP::IPL][LP::R];
-                        FH::template run<PRUNE_NONE>(lh, mh, twc, lineh,
-                            [&](int, int, int idx) { return col[idx]; },
-                            [&](int i, int r, int, float2 v) { O[i][r] = v; });
-                        if (!(LP::PARTIAL && lh >= LP::ITEMS)) {
-                            // fetch the whole first half before the stores so the loads overlap
-#pragma unroll
-                            for (int i = 0; i < LP::IPL; ++i)
-#pragma unroll
-                                for (int r = 0; r < LP::R; ++r) E[i][r] = __ldcg(es + FH::last_pos(lh, i, r));
-#pragma unroll
-                            for (int i = 0; i < LP::IPL; ++i)
-#pragma unroll
-                                for (int r = 0; r < LP::R; ++r) {
-                                    const int idx = FH::last_pos(lh, i, r);
-                                    const float2 t = cmul(O[i][r], tw[idx]);          // W_P^ky' * O
-                                    d[idx] = cadd(E[i][r], t);
-                                    d[idx + HP] = csub(E[i][r], t);
-                                }
-                        }
-                    }
+            // columns: P-point transforms over y of the bins kx = 2k + e
+            for (int k = gid; k < QP; k += C::NG) {
+                const float2 *col = cs + k * CSH;
+                if (e == 1 || k != 0) {
+                    float2 *d = dst + (long long)(2 * k + e) * P;
+                    F::template run<PRUNE_NONE>(l, m, twp, line,
+                        [&](int, int, int idx) { return col[idx]; },
+                        [&](int, int, int idx, float2 v) { d[idx] = v; });
                 } else {
-                    FH::template run_to_line<PRUNE_NONE>(lh, mh, twc, lineh,
+                    // column 0 of the even half carries bins kx = 0 and kx = P/2 of every row
+                    F::template run_to_line<PRUNE_NONE>(l, m, twp, line,
                         [&](int, int, int idx) { return col[idx]; });
-                    constexpr int NK = HP / TPLH;
-                    if (e == 0) {
-#pragma unroll 4
-                        for (int t = 0; t < NK; ++t) {
-                            const int ky = lh + t * TPLH;
-                            const float2 c1 = lineh[phys(ky)], c2 = lineh[phys((HP - ky) & (HP - 1))];
-                            scratch[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));                   // bin kx = 0
-                            scratch[(long long)HP * HP + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));  // bin kx = P/2
-                        }
-                    } else {
-                        // all first-half values are fetched before any store, in batches of 8 rows
-                        for (int t0 = 0; t0 < NK; t0 += 8) {
-                            float2 E0[8], EN[8];
-#pragma unroll
-                            for (int t = 0; t < 8; ++t) {
-                                const int ky = lh + (t0 + t) * TPLH;
-                                E0[t] = __ldcg(scratch + ky);
-                                EN[t] = __ldcg(scratch + (long long)HP * HP + ky);
-                            }
-#pragma unroll
-                            for (int t = 0; t < 8; ++t) {
-                                const int ky = lh + (t0 + t) * TPLH;
-                                const float2 c1 = lineh[phys(ky)], c2 = lineh[phys((HP - ky) & (HP - 1))];
-                                const float2 s0 = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
-                                const float2 sn = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
-                                const float2 w = tw[ky];
-                                const float2 t0v = cmul(s0, w), tnv = cmul(sn, w);
-                                dst[ky] = cadd(E0[t], t0v);
-                                dst[ky + HP] = csub(E0[t], t0v);
-                                dst[(long long)HP * P + ky] = cadd(EN[t], tnv);
-                                dst[(long long)HP * P + ky + HP] = csub(EN[t], tnv);
-                            }
-                        }
+                    for (int ky = l; ky < P; ky += TPL) {
+                        const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
+                        dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
+                        dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                     }
                 }
-                __syncwarp(mh);
+                __syncwarp(m);
             }
             __syncthreads();
         }
     }
 }
+
 
 // ---- inverse planes ------------------------------------------------------------------------------------
 
@@ -388,12 +381,6 @@ int plane_grid(long long planes)
 {
     const int s = plane_sms();
     return (int)(planes < s ? planes : s);
-}
-
-size_t plane_scratch_elems(int log2p)
-{
-    const size_t hp = (size_t)1 << (log2p - 1);
-    return (size_t)plane_sms() * (hp + 1) * hp;
 }
 
 template <typename T, int LOG2P> static int launch_plane_t(const PlaneArgs &a, int which, cudaStream_t st)

@@ -13,7 +13,6 @@ struct PlaneArgs {
     float2 *out;          // spectra [plane][P/2+1][P] written by PLANE_U / PLANE_H
     const float2 *in;     // spectra read by PLANE_INV
     void *y;              // output of PLANE_INV
-    float2 *scratch;      // PLANE_H: plane_scratch_elems() float2
     long long planes;     // number of x-y planes
     int lx, ly;           // grid extent along x (contiguous) and y
     const float2 *gtw;    // global twiddle table with gtw_n >= P points
@@ -22,7 +21,6 @@ struct PlaneArgs {
 };
 
 bool plane_supported(int log2p);
-size_t plane_scratch_elems(int log2p);
 int launch_plane(const PlaneArgs &a, int which, int log2p, int dtype, cudaStream_t st);
 
 }  // namespace hn
