@@ -76,16 +76,16 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
             const float2 *src = hs + (long long)(p.h_shift + r0) * p.nc;
 #pragma unroll 4
             for (int pos = r0; pos < head; pos += RPS, src += step)
-                cp_async8_s(bh_x + 8u * (unsigned)phys(pos), src);
+                cp_async8_s(bh_x + 8u * (unsigned)F::ph(pos), src);
             int pos = tail0 + ((r0 - tail0) & (RPS - 1));   // first position >= tail0 owned by this thread
             src = hs + (long long)(pos - tail0) * p.nc;
 #pragma unroll 4
             for (; pos < N; pos += RPS, src += step)
-                cp_async8_s(bh_x + 8u * (unsigned)phys(pos), src);
+                cp_async8_s(bh_x + 8u * (unsigned)F::ph(pos), src);
             for (int z = head + ((r0 - head) & (RPS - 1)); z < tail0; z += RPS)
-                bh[x * LS + phys(z)] = make_float2(0.f, 0.f);
+                bh[x * LS + F::ph(z)] = make_float2(0.f, 0.f);
         } else {
-            for (int pos = r0; pos < N; pos += RPS) bh[x * LS + phys(pos)] = make_float2(0.f, 0.f);
+            for (int pos = r0; pos < N; pos += RPS) bh[x * LS + F::ph(pos)] = make_float2(0.f, 0.f);
         }
     };
     auto issue_u = [&](long long t) {
@@ -98,8 +98,8 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         const float2 *src = us + (long long)r0 * p.nc;
         int pos = r0;
 #pragma unroll 4
-        for (; pos < nin; pos += RPS, src += step) cp_async8_s(bu_x + 8u * (unsigned)phys(pos), src);
-        for (; pos < N / 2; pos += RPS) bu[x * LS + phys(pos)] = make_float2(0.f, 0.f);
+        for (; pos < nin; pos += RPS, src += step) cp_async8_s(bu_x + 8u * (unsigned)F::ph(pos), src);
+        for (; pos < N / 2; pos += RPS) bu[x * LS + F::ph(pos)] = make_float2(0.f, 0.f);
     };
     long long t = blockIdx.x;
     if (t < tiles) { issue_h(t); }
@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
         if constexpr (HREG) {
             F::template mid<0, NP - 1, PRUNE_NONE>(l, m, tw, hline);
             F::template pass<NP - 1, PRUNE_NONE>(l, tw,
-                [&](int, int, int idx) { return hline[phys(idx)]; },
+                [&](int, int, int idx) { return hline[F::ph(idx)]; },
                 [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * p.scale); });
             __syncthreads();                               // filter lines are free again
             if (tn < tiles) issue_h(tn);
@@ -131,24 +131,24 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
             F::template mid<0, NP - 1, PRUNE_IN>(l, m, tw, uline);
             float2 Y[PL::IPL][PL::R];
             F::template pass<NP - 1, PRUNE_NONE>(l, tw,
-                [&](int, int, int idx) { return uline[phys(idx)]; },
+                [&](int, int, int idx) { return uline[F::ph(idx)]; },
                 [&](int i, int r, int idx, float2 v) {
                     if constexpr (HREG) Y[i][r] = cmul(v, H[i][r]);
                     else {
-                        const float2 hh = hline[phys(idx)];
+                        const float2 hh = hline[F::ph(idx)];
                         Y[i][r] = cmul(v, make_float2(hh.x * p.scale, hh.y * p.scale));
                     }
                 });
             __syncwarp(m);
             FI::template pass<0, PRUNE_NONE>(l, twi,
                 [&](int i, int r, int) { return Y[i][r]; },
-                [&](int, int, int idx, float2 v) { uline[phys(idx)] = v; });
+                [&](int, int, int idx, float2 v) { uline[FI::ph(idx)] = v; });
             __syncwarp(m);
             FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, uline);
             using PE = typename FI::template Pass<NP - 1>;
             float2 keep[PE::IPL][PE::R];
             FI::template pass<NP - 1, PRUNE_OUT>(l, twi,
-                [&](int, int, int idx) { return uline[phys(idx)]; },
+                [&](int, int, int idx) { return uline[FI::ph(idx)]; },
                 [&](int i, int r, int, float2 v) { keep[i][r] = v; });
             __syncwarp(m);
             if (!(PE::PARTIAL && l >= PE::ITEMS)) {
@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
                 for (int i = 0; i < PE::IPL; ++i)
 #pragma unroll
                     for (int r = 0; r < PE::R / 2; ++r)
-                        uline[phys(l + i * TPL + r * (N / PE::R))] = keep[i][r];
+                        uline[FI::ph(l + i * TPL + r * (N / PE::R))] = keep[i][r];
             }
         }
         __syncthreads();
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
             float2 *dst = p.out + o * p.out_outer + c0 + x + (long long)r0 * p.nc;
             const long long step = (long long)RPS * p.nc;
             if (c0 + x < p.nc)
-                for (int pos = r0; pos < p.n_out; pos += RPS, dst += step) *dst = bu[x * LS + phys(pos)];
+                for (int pos = r0; pos < p.n_out; pos += RPS, dst += step) *dst = bu[x * LS + FI::ph(pos)];
         }
         __syncthreads();
         if (tn < tiles) issue_u(tn);

@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_fwd_w_kernel(ColsFwdWAr
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = F::TPL;
     constexpr int TX = ct_tx(TPL);                         // column pairs per tile
     constexpr int NGRP = kCtThreads / TPL;                 // groups of lanes per CTA
-    constexpr int LS = ct_ls(phys(P1) + 2);                // room for the skewed line and for 2*(P1/2+1) bins
+    constexpr int LS = ct_ls(phys_max(P1) + 2);                // room for the skewed line and for 2*(P1/2+1) bins
     constexpr int PAIRB = 2 * (int)sizeof(T);              // bytes of one column pair of one row
     extern __shared__ float2 smem[];
     float2 *lines = smem;
@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_fwd_w_kernel(ColsFwdWAr
             for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
                 const int f1 = l + i * TPL;
                 if (f1 < F1) {
-                    const float2 z1 = line[phys(f1)], z2 = line[phys((P1 - f1) & (P1 - 1))];
+                    const float2 z1 = line[F::ph(f1)], z2 = line[F::ph((P1 - f1) & (P1 - 1))];
                     const float2 w0 = cmul(cl0, twp_w(p.twp, t2 * (unsigned)(i * TPL)));
                     const float2 w1 = cmul(cl1, twp_w(p.twp, (t2 + 1u) * (unsigned)(i * TPL)));
                     A0[i] = cmul(make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y)), w0);
@@ -231,12 +231,12 @@ __global__ void __launch_bounds__(256, 2) ct_core_w_kernel(CoreWArgs p)
 #pragma unroll
             for (int i = 0; i < P0::IPL; ++i)
 #pragma unroll
-                for (int rr = 0; rr < P0::R; ++rr) line[phys((l + i * TPL) * P0::R + rr)] = keep[i][rr];
+                for (int rr = 0; rr < P0::R; ++rr) line[F::ph((l + i * TPL) * P0::R + rr)] = keep[i][rr];
             __syncwarp(m);
         }
         F::template mid<1, NP - 1, PRUNE_NONE>(l, m, tw, line);
         F::template pass<NP - 1, PRUNE_NONE>(l, tw,
-            [&](int, int, int idx) { return line[phys(idx)]; },
+            [&](int, int, int idx) { return line[F::ph(idx)]; },
             [&](int i, int rr, int, float2 v) { Y[i][rr] = v; });
         // spectral product with the precomputed filter spectrum (coalesced loads, no stores between)
 #pragma unroll
@@ -246,14 +246,14 @@ __global__ void __launch_bounds__(256, 2) ct_core_w_kernel(CoreWArgs p)
         __syncwarp(m);
         FI::template pass<0, PRUNE_NONE>(l, twi,
             [&](int i, int rr, int) { return Y[i][rr]; },
-            [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+            [&](int, int, int idx, float2 v) { line[FI::ph(idx)] = v; });
         __syncwarp(m);
         FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, line);
         // undo the inter-pass twiddle W_P^(t2*f1), t2 = l + TPL*q: per-lane factor W_P^(f1*l) times a
         // per-row factor W_P^(f1*TPL*q) whose address is the same in all lanes
         const float2 cl = twp_w(p.twp, (unsigned)f1 * (unsigned)l);
         FI::template pass<NP - 1, PRUNE_NONE>(l, twi,
-            [&](int, int, int idx) { return line[phys(idx)]; },
+            [&](int, int, int idx) { return line[FI::ph(idx)]; },
             [&](int, int, int idx, float2 v) {
                 const float2 w = cmul(cl, twp_w(p.twp, (unsigned)f1 * (unsigned)(idx - l)));
                 row[idx] = cmulc(v, w);
@@ -281,7 +281,7 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_inv_w_kernel(ColsInvWAr
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = FI::TPL;
     constexpr int TX = ct_tx(TPL);
     constexpr int NGRP = kCtThreads / TPL;
-    constexpr int LS = ct_ls(phys(P1) + 2);
+    constexpr int LS = ct_ls(phys_max(P1) + 2);
     extern __shared__ float2 smem[];
     float2 *lines = smem;
     float2 *twt = lines + TX * LS;
@@ -323,7 +323,7 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_inv_w_kernel(ColsInvWAr
             const int t1 = idx / TX, x = idx % TX;
             const long long tt = (long long)t1 * P2 + 2 * (c0 + x);
             if (tt < p.len) {
-                const float2 z = lines[x * LS + phys(t1)];
+                const float2 z = lines[x * LS + FI::ph(t1)];
                 const long long o = base + (long long)t1 * P2 + 2 * x;
                 if constexpr (sizeof(T) == 4) {
                     const float2 qq = __ldg(reinterpret_cast<const float2 *>(pq + o));
@@ -366,7 +366,7 @@ bool ct1d_w_supported(int log2p1, int log2p2, int L, int K, int causal, int dtyp
 template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWArgs &a, cudaStream_t st)
 {
     using F = WF<LOG2P1, false>;
-    constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys(P1) + 2);
+    constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys_max(P1) + 2);
     const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1) + (size_t)2 * (P1 / 2) * 2 * TX * sizeof(T);
     const int P2 = 1 << a.log2p2;
     const long long tiles = a.slices * ((P2 / 2) / TX);
@@ -387,7 +387,7 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
 template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWArgs &a, cudaStream_t st)
 {
     using F = WF<LOG2P1, true>;
-    constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys(P1) + 2);
+    constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys_max(P1) + 2);
     const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1);
     const int P2 = 1 << a.log2p2;
     const long long tiles = a.slices * ((P2 / 2) / TX);

@@ -20,7 +20,10 @@ enum { PRUNE_NONE = 0, PRUNE_IN = 1, PRUNE_OUT = 2 };
 
 __host__ __device__ __forceinline__ constexpr int phys(int i) { return i + (i >> 4); }
 // shared-memory floats2 needed for one line of n points (odd, so lines do not alias banks)
-__host__ __device__ __forceinline__ constexpr int line_stride(int n) { return (phys(n) + 1) | 1; }
+// largest skewed position + 1 of an n-point line under any engine (the warp engine skews short
+// lines by i >> 3)
+__host__ __device__ __forceinline__ constexpr int phys_max(int n) { return n <= 128 ? n + (n >> 3) : n + (n >> 4); }
+__host__ __device__ __forceinline__ constexpr int line_stride(int n) { return (phys_max(n) + 1) | 1; }
 
 __device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
 __device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }

@@ -206,11 +206,11 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
                 __syncwarp(m);
                 FI::template pass<0, PRUNE_NONE>(l, twi,
                     [&](int i, int r, int) { return Y[i][r]; },
-                    [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+                    [&](int, int, int idx, float2 v) { line[FI::ph(idx)] = v; });
                 __syncwarp(m);
                 FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, line);
                 FI::template pass<NP - 1, PRUNE_OUT>(l, twi,
-                    [&](int, int, int idx) { return line[phys(idx)]; },
+                    [&](int, int, int idx) { return line[FI::ph(idx)]; },
                     [&](int, int, int idx, float2 v) { uc[idx] = v; });
                 __syncwarp(m);
             }
@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
             if (gid == NGM) {
                 F::template run_to_line<PRUNE_NONE>(l, m, twf, line, [&](int, int, int idx) { return hcs[idx]; });
                 for (int ky = l; ky < P; ky += TPL) {
-                    const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
+                    const float2 c1 = line[F::ph(ky)], c2 = line[F::ph((P - ky) & (P - 1))];
                     x0[ky] = make_float2(0.5f * p.scale * (c1.x + c2.x), 0.5f * p.scale * (c1.y - c2.y));
                     xn[ky] = make_float2(0.5f * p.scale * (c1.y + c2.y), 0.5f * p.scale * (c2.x - c1.x));
                 }
@@ -234,7 +234,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
                 __syncwarp(m2);
                 FI::template run<PRUNE_OUT, true>(l, m, twi, line,
                     [&](int, int, int idx) {
-                        const float2 c1 = line[phys(idx)], c2 = line[phys((P - idx) & (P - 1))];
+                        const float2 c1 = line[F::ph(idx)], c2 = line[F::ph((P - idx) & (P - 1))];
                         const float2 u0 = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
                         const float2 un = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                         const float2 y0 = cmul(u0, x0[idx]), yn = cmul(un, xn[idx]);

@@ -9,7 +9,7 @@ constexpr int kPlaneThreads = 512;
 
 // lines start on 16-byte boundaries (asynchronous 16-byte copies land in them) and two
 // neighbouring lines do not share banks: stride = 8 mod 16 complex numbers
-__host__ __device__ constexpr int plane_ls(int n) { return ((phys(n) + 1 + 7) / 16) * 16 + 8; }
+__host__ __device__ constexpr int plane_ls(int n) { return ((phys_max(n) + 1 + 7) / 16) * 16 + 8; }
 
 // Ask the memory system to bring [ptr, ptr + bytes) into L2 (bulk prefetch, 16-byte granules);
 // the CTA issues it for the plane it will work on next, so that plane's loads hit L2.
@@ -70,20 +70,21 @@ __device__ __forceinline__ void zero_staged(unsigned char *row, int off, int fro
 template <int LOG2P, int CSS>
 __device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, int y0, int y1, int l)
 {
-    constexpr int P = 1 << LOG2P, HP = P / 2, TPL = WF<LOG2P, false>::TPL;
+    using FW = WF<LOG2P, false>;
+    constexpr int P = 1 << LOG2P, HP = P / 2, TPL = FW::TPL;
     // bins 1 .. HP-1 (lane 0's first entry, bin 0, is overwritten below)
 #pragma unroll
     for (int t = 0; t < HP / TPL; ++t) {
         const int kx = l + t * TPL;
-        const float2 z1 = line[phys(kx)];
-        const float2 z2 = line[phys((P - kx) & (P - 1))];
+        const float2 z1 = line[FW::ph(kx)];
+        const float2 z2 = line[FW::ph((P - kx) & (P - 1))];
         cs[kx * CSS + y0] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
         cs[kx * CSS + y1] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
     }
     __syncwarp(WF<LOG2P, false>::group_mask(threadIdx.x));
     if (l == 0) {
         // the two purely real bins (kx = 0 and kx = P/2) of each row share column 0
-        const float2 z0 = line[phys(0)], zh = line[phys(HP)];
+        const float2 z0 = line[FW::ph(0)], zh = line[FW::ph(HP)];
         cs[y0] = make_float2(z0.x, zh.x);
         cs[y1] = make_float2(z0.y, zh.y);
     }

@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
                 F::template run_to_line<PRUNE_IN>(l, m, twp, line,
                     [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); });
                 for (int ky = l; ky < P; ky += TPL) {
-                    const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
+                    const float2 c1 = line[F::ph(ky)], c2 = line[F::ph((P - ky) & (P - 1))];
                     dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
                     dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                 }
@@ -148,8 +148,8 @@ __device__ __forceinline__ void separate_rows_odd(const float2 *line, float2 *cs
 #pragma unroll
     for (int t = 0; t < H / 2 / TPL; ++t) {
         const int k = l + t * TPL;
-        const float2 z1 = line[phys(k)];
-        const float2 z2 = line[phys(H - 1 - k)];
+        const float2 z1 = line[WF<LOG2H, false>::ph(k)];
+        const float2 z2 = line[WF<LOG2H, false>::ph(H - 1 - k)];
         cs[k * CSS + y0] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
         cs[k * CSS + y1] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
     }
@@ -199,7 +199,9 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
             prefetch_l2(hb + (pl + gridDim.x) * (long long)Ky * Kx * sizeof(T), (long long)Ky * Kx * sizeof(T), tid);
         for (int e = 0; e < 2; ++e) {
             // rows: padded row y holds tap row (y + Ly - 1) mod P; two rows per transform
-            for (int rp = gidh; rp < HP; rp += C::NGH) {
+            // the two groups of a half warp take rows 8 apart, so their column-store writes (one
+            // row per group, consecutive columns per lane) fall into different banks
+            for (int rp = ((gidh >> 1) & 3) | ((gidh & 1) << 2) | (gidh & ~7); rp < HP; rp += C::NGH) {
                 const int y0 = 2 * rp, y1 = y0 + 1;
                 const int my0 = (y0 + Ly - 1) & (P - 1), my1 = (y1 + Ly - 1) & (P - 1);
                 const bool v0 = my0 < Ky, v1 = my1 < Ky;
@@ -209,8 +211,10 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                     // half-length line and are read from global memory (L2) directly
                     constexpr bool STAGED = sizeof(T) == 2;
                     constexpr int SLOT = ((C::P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;   // bytes kept per staged row
-                    static_assert(!STAGED || 2 * SLOT <= C::LSH * 8, "staged rows must fit the line");
-                    unsigned char *s0 = reinterpret_cast<unsigned char *>(lineh), *s1 = s0 + SLOT;
+                    static_assert(!STAGED || 2 * SLOT + 32 <= C::LSH * 8, "staged rows must fit the line");
+                    // the four lines of a warp start 0, 64, 0, 64 bytes into the 128-byte bank row:
+                    // lines 2 and 3 stage 32 bytes further in, so the narrow tap loads do not collide
+                    unsigned char *s0 = reinterpret_cast<unsigned char *>(lineh) + 16 * (gidh & 2), *s1 = s0 + SLOT;
                     const unsigned char *g0 = hb + (ib + (long long)my0 * Kx) * sizeof(T);
                     const unsigned char *g1 = hb + (ib + (long long)my1 * Kx) * sizeof(T);
                     const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
@@ -268,7 +272,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                     F::template run_to_line<PRUNE_NONE>(l, m, twp, line,
                         [&](int, int, int idx) { return col[idx]; });
                     for (int ky = l; ky < P; ky += TPL) {
-                        const float2 c1 = line[phys(ky)], c2 = line[phys((P - ky) & (P - 1))];
+                        const float2 c1 = line[F::ph(ky)], c2 = line[F::ph((P - ky) & (P - 1))];
                         dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
                         dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                     }

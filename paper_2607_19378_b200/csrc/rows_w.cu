@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
         }
         float2 *o0 = p.out + r0 * p.pitch, *o1 = p.out + r1 * p.pitch;
         for (int kx = l; kx <= HP; kx += TPL) {
-            const float2 z1 = line[phys(kx)], z2 = line[phys((P - kx) & (P - 1))];
+            const float2 z1 = line[F::ph(kx)], z2 = line[F::ph((P - kx) & (P - 1))];
             o0[kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
             if (has1) o1[kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
         }
@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
             return make_float2(A.x - B.y, A.y + B.x);
         });
         for (int n = l; n < p.len; n += TPL) {
-            const float2 z = line[phys(n)];
+            const float2 z = line[FI::ph(n)];
             IO<T>::st(py, r0 * p.len + n, z.x * IO<T>::ld(pq, r0 * p.len + n));
             if (has1) IO<T>::st(py, r1 * p.len + n, z.y * IO<T>::ld(pq, r1 * p.len + n));
         }

@@ -56,6 +56,11 @@ template <int LOG2N, bool INV> struct WF {
         for (int i = 0; i < s; ++i) n *= radix(i);
         return n;
     }
+    // Lines are stored skewed: position i sits at ph(i).  The shift follows the radix of the first
+    // pass, whose results land R points apart per lane: with it the groups of a warp that work on
+    // neighbouring lines never meet in a bank.
+    static constexpr int SKEW = (LOG2N <= 7 && radix(0) == 8) ? 3 : 4;
+    __host__ __device__ static constexpr int ph(int i) { return i + (i >> SKEW); }
     template <int S> struct Pass {
         static constexpr int R = radix(S);
         static constexpr int NS = ns(S);
@@ -112,7 +117,7 @@ template <int LOG2N, bool INV> struct WF {
             constexpr int R = PS::R;
             float2 keep[PS::IPL][R];
             pass<S0, PR0>(l, tw,
-                [&](int, int, int idx) { return line[phys(idx)]; },
+                [&](int, int, int idx) { return line[ph(idx)]; },
                 [&](int i, int r, int, float2 v) { keep[i][r] = v; });
             __syncwarp(m);
             if (!(PS::PARTIAL && l >= PS::ITEMS)) {
@@ -122,7 +127,7 @@ template <int LOG2N, bool INV> struct WF {
                     const int k = j & (PS::NS - 1);
                     const int base = (j - k) * R + k;
 #pragma unroll
-                    for (int r = 0; r < R; ++r) line[phys(base + r * PS::NS)] = keep[i][r];
+                    for (int r = 0; r < R; ++r) line[ph(base + r * PS::NS)] = keep[i][r];
                 }
             }
             __syncwarp(m);
@@ -148,14 +153,14 @@ template <int LOG2N, bool INV> struct WF {
 #pragma unroll
                 for (int i = 0; i < P0::IPL; ++i)
 #pragma unroll
-                    for (int r = 0; r < P0::R; ++r) line[phys((l + i * TPL) * P0::R + r)] = keep[i][r];
+                    for (int r = 0; r < P0::R; ++r) line[ph((l + i * TPL) * P0::R + r)] = keep[i][r];
             }
         } else {
-            pass<0, PF>(l, tw, in, [&](int, int, int idx, float2 v) { line[phys(idx)] = v; });
+            pass<0, PF>(l, tw, in, [&](int, int, int idx, float2 v) { line[ph(idx)] = v; });
         }
         __syncwarp(m);
         mid<1, NP - 1, PRUNE_NONE>(l, m, tw, line);
-        pass<NP - 1, PL>(l, tw, [&](int, int, int idx) { return line[phys(idx)]; }, out);
+        pass<NP - 1, PL>(l, tw, [&](int, int, int idx) { return line[ph(idx)]; }, out);
     }
 
     // Position (natural order) of output leg r of item i of lane l after the last pass.
@@ -193,7 +198,7 @@ template <int LOG2N, bool INV> struct WF {
             for (int i = 0; i < PS::IPL; ++i) {
                 const int j = l + i * TPL;
 #pragma unroll
-                for (int r = 0; r < NOUT; ++r) line[phys(j + r * (N / PS::R))] = keep[i][r];
+                for (int r = 0; r < NOUT; ++r) line[ph(j + r * (N / PS::R))] = keep[i][r];
             }
         }
         __syncwarp(m);
