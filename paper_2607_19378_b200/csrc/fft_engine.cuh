@@ -140,12 +140,70 @@ template <bool INV, int PR> __device__ __forceinline__ void dft16(float2 (&x)[16
     }
 }
 
+// cos and sin of 2 pi t / 32
+__host__ __device__ constexpr float w32_cos(int t)
+{
+    t &= 31;
+    if (t > 16) t = 32 - t;
+    const bool neg = t > 8;
+    if (neg) t = 16 - t;
+    const float v = t == 0 ? 1.f : t == 1 ? 0.98078528040323044913f : t == 2 ? 0.92387953251128675613f
+                  : t == 3 ? 0.83146961230254523708f : t == 4 ? 0.70710678118654752440f
+                  : t == 5 ? 0.55557023301960222474f : t == 6 ? 0.38268343236508977173f
+                  : t == 7 ? 0.19509032201612826785f : 0.f;
+    return neg ? -v : v;
+}
+__host__ __device__ constexpr float w32_sin(int t) { return w32_cos(t - 8); }
+
+// a * W_32^T (forward sign; conjugate for INV), T compile-time
+template <int T, bool INV> __device__ __forceinline__ float2 mul_w32(float2 a)
+{
+    constexpr int t = T & 31;
+    if constexpr (t % 2 == 0) return mul_w16<t / 2, INV>(a);
+    else {
+        constexpr float c = w32_cos(t);
+        constexpr float s = INV ? w32_sin(t) : -w32_sin(t);
+        return make_float2(fmaf(a.x, c, -a.y * s), fmaf(a.x, s, a.y * c));
+    }
+}
+
+template <int N2, bool INV> __device__ __forceinline__ void tw32_row(float2 (&a)[4])
+{
+    a[1] = mul_w32<N2, INV>(a[1]); a[2] = mul_w32<2 * N2, INV>(a[2]); a[3] = mul_w32<3 * N2, INV>(a[3]);
+}
+
+template <bool INV, int PR> __device__ __forceinline__ void dft32(float2 (&x)[32])
+{
+    // n = 8*n1 + n2, k = k1 + 4*k2: 4-point transforms over n1, twiddle W32^(n2*k1),
+    // 8-point transforms over n2.
+    constexpr int PIN = (PR == PRUNE_IN) ? PRUNE_IN : PRUNE_NONE;
+    constexpr int POUT = (PR == PRUNE_OUT) ? PRUNE_OUT : PRUNE_NONE;
+    float2 a[8][4];                                  // a[n2][k1]
+#pragma unroll
+    for (int n2 = 0; n2 < 8; ++n2) {
+        a[n2][0] = x[n2]; a[n2][1] = x[n2 + 8]; a[n2][2] = x[n2 + 16]; a[n2][3] = x[n2 + 24];
+        dft4<INV, PIN>(a[n2][0], a[n2][1], a[n2][2], a[n2][3]);
+    }
+    tw32_row<1, INV>(a[1]); tw32_row<2, INV>(a[2]); tw32_row<3, INV>(a[3]); tw32_row<4, INV>(a[4]);
+    tw32_row<5, INV>(a[5]); tw32_row<6, INV>(a[6]); tw32_row<7, INV>(a[7]);
+#pragma unroll
+    for (int k1 = 0; k1 < 4; ++k1) {
+        float2 c[8];
+#pragma unroll
+        for (int n2 = 0; n2 < 8; ++n2) c[n2] = a[n2][k1];
+        dft8<INV, POUT>(c);
+#pragma unroll
+        for (int k2 = 0; k2 < (PR == PRUNE_OUT ? 4 : 8); ++k2) x[k1 + 4 * k2] = c[k2];
+    }
+}
+
 template <int R, bool INV, int PR> __device__ __forceinline__ void dft(float2 (&x)[R])
 {
     if constexpr (R == 2) dft2<INV, PR>(x[0], x[1]);
     else if constexpr (R == 4) dft4<INV, PR>(x[0], x[1], x[2], x[3]);
     else if constexpr (R == 8) dft8<INV, PR>(x);
-    else dft16<INV, PR>(x);
+    else if constexpr (R == 16) dft16<INV, PR>(x);
+    else dft32<INV, PR>(x);
 }
 
 // ---- pass plan: log2(N) split as evenly as possible into passes of <= 4 bits ------

@@ -27,8 +27,8 @@ template <> struct WPlan<8>  { static constexpr int NP = 2, TPL = 16; static con
     __host__ __device__ static constexpr int r(int s) { return s == 0 ? 16 : s == 1 ? 16 : 1; } };
 template <> struct WPlan<9>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 8};
     __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 8 : 8; } };
-template <> struct WPlan<10>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 16};
-    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 8 : 16; } };
+template <> struct WPlan<10>  { static constexpr int NP = 2, TPL = 32; static constexpr int R[3] = {32, 32, 1};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 32 : s == 1 ? 32 : 1; } };
 
 // Twiddle sources.  A source answers get<S>(i, r, k, t) for pass S: item i of the lane, leg r,
 // k = position of the item inside its sub-transform, t = index into a full N-point table (the
@@ -59,7 +59,7 @@ template <int LOG2N, bool INV> struct WF {
     // Lines are stored skewed: position i sits at ph(i).  The shift follows the radix of the first
     // pass, whose results land R points apart per lane: with it the groups of a warp that work on
     // neighbouring lines never meet in a bank.
-    static constexpr int SKEW = (LOG2N <= 7 && radix(0) == 8) ? 3 : 4;
+    static constexpr int SKEW = (LOG2N <= 7 && radix(0) == 8) ? 3 : radix(0) == 32 ? 5 : 4;
     __host__ __device__ static constexpr int ph(int i) { return i + (i >> SKEW); }
     template <int S> struct Pass {
         static constexpr int R = radix(S);
