@@ -11,6 +11,7 @@
 //                spectrum (Eq. 12), inverse transform chained in registers, undo twiddle.
 //   cols_inv_w   rebuild the mirrored half, inverse along f1 keeping t < P/2, crop, gate
 //                with q, coalesced store.
+#include <type_traits>
 #include "common.cuh"
 #include "ct1d.cuh"
 #include "plane_util.cuh"
@@ -55,7 +56,7 @@ struct ColsFwdWArgs {
 };
 
 template <typename T, int LOG2P1, bool HAS_B>
-__global__ void __launch_bounds__(kCtThreads, 4) ct_cols_fwd_w_kernel(ColsFwdWArgs p)
+__global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_fwd_w_kernel(ColsFwdWArgs p)
 {
     using F = WF<LOG2P1, false>;
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = F::TPL;
@@ -66,8 +67,10 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_fwd_w_kernel(ColsFwdWAr
     extern __shared__ float2 smem[];
     float2 *lines = smem;
     float2 *twt = lines + TX * LS;
-    // staged inputs, pair-major: [tensor][pair x][row t1], so that the lanes of a group (which
-    // differ in t1) read consecutive words
+    // staged inputs [tensor][row t1][pair x], fetched 8 bytes at a time; a row is padded by 8 bytes,
+    // which sends the lanes of a group (they differ in t1) to different banks
+    constexpr int PG = 8 / PAIRB;                          // column pairs per 8-byte copy
+    constexpr int RS = TX * PAIRB + 8;                     // bytes per staged row
     unsigned char *raw = reinterpret_cast<unsigned char *>(twt + P1);
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
@@ -82,19 +85,19 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_fwd_w_kernel(ColsFwdWAr
         const int c0 = (int)(t % tpc) * TX;
         const long long base = s * p.in_slice;
         __syncthreads();                                   // previous tile done with raw and lines
-        for (int idx = tid; idx < HP1 * TX; idx += kCtThreads) {
-            const int t1 = idx / TX, x = idx % TX;
-            const long long e0 = (long long)t1 * P2 + 2 * (c0 + x);
-            unsigned char *d = raw + ((size_t)x * HP1 + t1) * PAIRB;
-            if (e0 + 2 <= p.len) {
-                cp_async_n<PAIRB>(d, ab + (base + e0) * sizeof(T));
-                if (HAS_B) cp_async_n<PAIRB>(d + (size_t)TX * HP1 * PAIRB, bb + (base + e0) * sizeof(T));
+        for (int idx = tid; idx < HP1 * (TX / PG); idx += kCtThreads) {
+            const int t1 = idx / (TX / PG), xg = idx % (TX / PG);
+            const long long e0 = (long long)t1 * P2 + 2 * (c0 + PG * xg);
+            unsigned char *d = raw + (size_t)t1 * RS + 8 * xg;
+            if (e0 + 2 * PG <= p.len) {
+                cp_async_n<8>(d, ab + (base + e0) * sizeof(T));
+                if (HAS_B) cp_async_n<8>(d + (size_t)HP1 * RS, bb + (base + e0) * sizeof(T));
             } else {
-                for (int e = 0; e < 2; ++e) {
+                for (int e = 0; e < 2 * PG; ++e) {
                     const bool ok = e0 + e < p.len;
                     reinterpret_cast<T *>(d)[e] = ok ? reinterpret_cast<const T *>(ab)[base + e0 + e] : T(0.f);
                     if (HAS_B)
-                        reinterpret_cast<T *>(d + (size_t)TX * HP1 * PAIRB)[e] = ok ? reinterpret_cast<const T *>(bb)[base + e0 + e] : T(0.f);
+                        reinterpret_cast<T *>(d + (size_t)HP1 * RS)[e] = ok ? reinterpret_cast<const T *>(bb)[base + e0 + e] : T(0.f);
                 }
             }
         }
@@ -102,13 +105,13 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_fwd_w_kernel(ColsFwdWAr
         __syncthreads();
         for (int x = gid; x < TX; x += NGRP) {
         float2 *line = lines + x * LS;
-        const unsigned char *ra = raw + (size_t)x * HP1 * PAIRB;
-        const unsigned char *rb = ra + (size_t)TX * HP1 * PAIRB;
+        const unsigned char *ra = raw + (size_t)x * PAIRB;
+        const unsigned char *rb = ra + (size_t)HP1 * RS;
         F::template run_to_line<PRUNE_IN>(l, m, tw, line, [&](int, int, int idx) {
-            float a0 = staged<T>(ra + (size_t)idx * PAIRB, 0, 0), a1 = staged<T>(ra + (size_t)idx * PAIRB, 0, 1);
+            float a0 = staged<T>(ra + (size_t)idx * RS, 0, 0), a1 = staged<T>(ra + (size_t)idx * RS, 0, 1);
             if (HAS_B) {
-                a0 *= staged<T>(rb + (size_t)idx * PAIRB, 0, 0);
-                a1 *= staged<T>(rb + (size_t)idx * PAIRB, 0, 1);
+                a0 *= staged<T>(rb + (size_t)idx * RS, 0, 0);
+                a1 *= staged<T>(rb + (size_t)idx * RS, 0, 1);
             }
             return make_float2(a0, a1);
         });
@@ -275,7 +278,7 @@ struct ColsInvWArgs {
 };
 
 template <typename T, int LOG2P1>
-__global__ void __launch_bounds__(kCtThreads, 4) ct_cols_inv_w_kernel(ColsInvWArgs p)
+__global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_inv_w_kernel(ColsInvWArgs p)
 {
     using FI = WF<LOG2P1, true>;
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = FI::TPL;
@@ -319,19 +322,35 @@ __global__ void __launch_bounds__(kCtThreads, 4) ct_cols_inv_w_kernel(ColsInvWAr
         __syncthreads();
         // line x now holds, at position t1 < P1/2, the two real outputs of columns 2x, 2x+1
         const long long base = s * (long long)p.len + 2 * c0;
-        for (int idx = tid; idx < HP1 * TX; idx += kCtThreads) {
-            const int t1 = idx / TX, x = idx % TX;
+        // gate values first (all requests in flight together), then products and stores
+        constexpr int NE = HP1 * TX / kCtThreads;
+        static_assert(HP1 * TX % kCtThreads == 0, "whole epilogue rounds");
+        // a half warp takes 8 pairs of two neighbouring rows: line stride and skew then spread its
+        // 16 reads over all banks, and each row still receives whole 32-byte sectors
+        const int x = (tid & 7) + 8 * ((tid >> 4) % (TX / 8));
+        const int tb = ((tid >> 3) & 1) + 2 * ((tid >> 4) / (TX / 8));
+        constexpr int TSTEP = kCtThreads / TX;
+        const long long ox = base + 2 * x;
+        using Q2 = typename std::conditional<sizeof(T) == 4, float2, __nv_bfloat162>::type;
+        Q2 qv[NE];
+#pragma unroll
+        for (int e = 0; e < NE; ++e) {
+            const int t1 = tb + e * TSTEP;
+            const long long tt = (long long)t1 * P2 + 2 * (c0 + x);
+            if (tt < p.len) qv[e] = __ldg(reinterpret_cast<const Q2 *>(pq + ox + (long long)t1 * P2));
+        }
+#pragma unroll
+        for (int e = 0; e < NE; ++e) {
+            const int t1 = tb + e * TSTEP;
             const long long tt = (long long)t1 * P2 + 2 * (c0 + x);
             if (tt < p.len) {
                 const float2 z = lines[x * LS + FI::ph(t1)];
-                const long long o = base + (long long)t1 * P2 + 2 * x;
+                const long long o = ox + (long long)t1 * P2;
                 if constexpr (sizeof(T) == 4) {
-                    const float2 qq = __ldg(reinterpret_cast<const float2 *>(pq + o));
-                    *reinterpret_cast<float2 *>(py + o) = make_float2(z.x * qq.x, z.y * qq.y);
+                    *reinterpret_cast<float2 *>(py + o) = make_float2(z.x * qv[e].x, z.y * qv[e].y);
                 } else {
-                    const __nv_bfloat162 qq = *reinterpret_cast<const __nv_bfloat162 *>(pq + o);
                     *reinterpret_cast<__nv_bfloat162 *>(py + o) =
-                        __floats2bfloat162_rn(z.x * __low2float(qq), z.y * __high2float(qq));
+                        __floats2bfloat162_rn(z.x * __low2float(qv[e]), z.y * __high2float(qv[e]));
                 }
             }
         }
@@ -358,7 +377,7 @@ bool ct1d_w_supported(int log2p1, int log2p2, int L, int K, int causal, int dtyp
     if (log2p1 < 7 || log2p1 > 10 || log2p2 < 7 || log2p2 > 10) return false;
     if (((long long)L * es) % 16 != 0) return false;               // 16-byte copies of whole chunks
     if (causal && ((long long)K * es) % 16 != 0) return false;
-    const int tx = ct_tx(log2p1 >= 9 ? 32 : (log2p1 == 8 ? 16 : 8));
+    const int tx = ct_tx(log2p1 >= 10 ? 32 : (log2p1 >= 8 ? 16 : 8));
     if (((1 << log2p2) / 2) % tx != 0) return false;
     return true;
 }
@@ -367,10 +386,11 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
 {
     using F = WF<LOG2P1, false>;
     constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys_max(P1) + 2);
-    const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1) + (size_t)2 * (P1 / 2) * 2 * TX * sizeof(T);
+    const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1) + (size_t)2 * (P1 / 2) * (2 * TX * sizeof(T) + 8);
     const int P2 = 1 << a.log2p2;
     const long long tiles = a.slices * ((P2 / 2) / TX);
-    const int grid = (int)(tiles < 4ll * ctw_sms() ? tiles : 4ll * ctw_sms());
+    const long long res = (LOG2P1 >= 9 ? 2ll : 4ll) * ctw_sms();   // resident CTAs
+    const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
     if (a.b) {
         static DevOnce attr;
@@ -391,7 +411,8 @@ template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWA
     const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1);
     const int P2 = 1 << a.log2p2;
     const long long tiles = a.slices * ((P2 / 2) / TX);
-    const int grid = (int)(tiles < 4ll * ctw_sms() ? tiles : 4ll * ctw_sms());
+    const long long res = (LOG2P1 >= 9 ? 2ll : 4ll) * ctw_sms();   // resident CTAs
+    const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
     static DevOnce attr;
     if (attr.first()) { cudaFuncSetAttribute(ct_cols_inv_w_kernel<T, LOG2P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }

@@ -25,8 +25,8 @@ template <> struct WPlan<7>  { static constexpr int NP = 2, TPL = 8; static cons
     __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 16 : 1; } };
 template <> struct WPlan<8>  { static constexpr int NP = 2, TPL = 16; static constexpr int R[3] = {16, 16, 1};
     __host__ __device__ static constexpr int r(int s) { return s == 0 ? 16 : s == 1 ? 16 : 1; } };
-template <> struct WPlan<9>  { static constexpr int NP = 3, TPL = 32; static constexpr int R[3] = {8, 8, 8};
-    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 8 : s == 1 ? 8 : 8; } };
+template <> struct WPlan<9>  { static constexpr int NP = 2, TPL = 16; static constexpr int R[3] = {32, 16, 1};
+    __host__ __device__ static constexpr int r(int s) { return s == 0 ? 32 : s == 1 ? 16 : 1; } };
 template <> struct WPlan<10>  { static constexpr int NP = 2, TPL = 32; static constexpr int R[3] = {32, 32, 1};
     __host__ __device__ static constexpr int r(int s) { return s == 0 ? 32 : s == 1 ? 32 : 1; } };
 
