@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
 
     // rows back for slice sp, reading column store ub; groups g0, g0 + gstep, ... take part
     auto rows_back = [&](long long sp, const float2 *ub, int g0, int gstep) {
-        for (int rp = g0; 2 * rp < Ly; rp += gstep) {
+        for (int rp = spread_pair<4>(g0); 2 * rp < Ly; rp += gstep) {
             const int y0 = 2 * rp, y1 = y0 + 1;
             const bool has1 = y1 < Ly;
             const long long o0 = sp * vol + (long long)y0 * Lx, o1 = o0 + Lx;
@@ -115,14 +115,16 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
         }
         if (gid < NGM) {
             // ---- filter rows: padded position yp holds tap my = (yp + Ly - 1) mod P ----------
-            for (int rp = gid; 2 * rp < P; rp += NGM) {
+            for (int rp = spread_pair<4>(gid); 2 * rp < P; rp += NGM) {
                 const int yp0 = 2 * rp, yp1 = yp0 + 1;
                 const int my0 = (yp0 + Ly - 1) & (P - 1), my1 = (yp1 + Ly - 1) & (P - 1);
                 const bool v0 = my0 < Ky, v1 = my1 < Ky;
                 if (v0 || v1) {
                     constexpr int SLOT = ((P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;
-                    static_assert(2 * SLOT <= C::LS * 8, "staged rows must fit the line");
-                    unsigned char *s0 = reinterpret_cast<unsigned char *>(line), *s1 = s0 + SLOT;
+                    static_assert(2 * SLOT + 32 <= C::LS * 8, "staged rows must fit the line");
+                    // lines 2 and 3 of a warp stage 32 bytes further in: the narrow tap loads of the four lines
+                    // then use different banks
+                    unsigned char *s0 = reinterpret_cast<unsigned char *>(line) + 16 * (gid & 2), *s1 = s0 + SLOT;
                     const unsigned char *g0 = hb + (hs * kvol + (long long)my0 * Kx) * sizeof(T);
                     const unsigned char *g1 = hb + (hs * kvol + (long long)my1 * Kx) * sizeof(T);
                     if (v0) stage_row<TPL>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.h_elems * sizeof(T), l);
@@ -150,7 +152,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
             }
             if (gid < NGM / 2) {
                 // ---- k*v rows of this slice ---------------------------------------------------------
-                for (int rp = gid; 2 * rp < Ly; rp += NGM / 2) {
+                for (int rp = spread_pair<4>(gid); 2 * rp < Ly; rp += NGM / 2) {
                     const int y0 = 2 * rp, y1 = y0 + 1;
                     const bool has1 = y1 < Ly;
                     const int nrow = (has1 ? 2 : 1) * Lx * (int)sizeof(T);
@@ -190,7 +192,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
         __syncthreads();
         // ---- columns: filter spectrum, k*v spectrum, product, inverse --------------------------
         if (gid < NGM) {
-            for (int kx = gid; kx < HP; kx += NGM) {
+            for (int kx = spread_pair<8>(gid); kx < HP; kx += NGM) {
                 if (kx == 0) continue;                       // the packed column belongs to the extra warp
                 const float2 *hc = hcs + kx * C::HCSS;
                 float2 *uc = ucs + kx * C::UCSS;

@@ -65,6 +65,15 @@ __device__ __forceinline__ void zero_staged(unsigned char *row, int off, int fro
     for (int i = from + l; i < to; i += TPL) *reinterpret_cast<T *>(row + off + (int)sizeof(T) * i) = T(0.f);
 }
 
+// Engines with 8 lanes per line put two lines into each half warp.  When both lines walk a column
+// store (consecutive columns per lane, one row or column offset per line), the two must sit D
+// entries apart to use different banks: spread_pair<D>(g) renumbers the groups so that g and g ^ 1
+// get numbers D apart (a bijection on every aligned block of 2*D groups).
+template <int D> __host__ __device__ __forceinline__ constexpr int spread_pair(int g)
+{
+    return ((g >> 1) & (D - 1)) | ((g & 1) * D) | (g & ~(2 * D - 1));
+}
+
 // Separate the spectra of the two real rows packed in one complex transform (results in
 // `line`, natural order) and scatter them into column store rows y0, y1.
 template <int LOG2P, int CSS>

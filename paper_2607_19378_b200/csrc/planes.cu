@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
             // rows: padded row y holds tap row (y + Ly - 1) mod P; two rows per transform
             // the two groups of a half warp take rows 8 apart, so their column-store writes (one
             // row per group, consecutive columns per lane) fall into different banks
-            for (int rp = ((gidh >> 1) & 3) | ((gidh & 1) << 2) | (gidh & ~7); rp < HP; rp += C::NGH) {
+            for (int rp = spread_pair<4>(gidh); rp < HP; rp += C::NGH) {
                 const int y0 = 2 * rp, y1 = y0 + 1;
                 const int my0 = (y0 + Ly - 1) & (P - 1), my1 = (y1 + Ly - 1) & (P - 1);
                 const bool v0 = my0 < Ky, v1 = my1 < Ky;
