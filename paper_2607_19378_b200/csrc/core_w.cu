@@ -11,7 +11,9 @@
 
 namespace hn {
 
-constexpr int kCoreThreads = 256;
+// threads per CTA.  For 1024-point lines (one CTA of 8 groups per SM) both 12 groups per CTA and three CTAs of
+// 4 groups were measured slower: tiles that are not 64 bytes wide per row cost more than the extra warps give.
+__host__ __device__ constexpr int core_threads(int) { return 256; }
 
 __device__ __forceinline__ void cp_async8(void *smem_dst, const void *gmem_src)
 {
@@ -26,8 +28,9 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
 template <int LOG2P>
-__global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core_w_kernel(AxisArgs p)
+__global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) axis_core_w_kernel(AxisArgs p)
 {
+    constexpr int kCoreThreads = core_threads(LOG2P);
     using F = WF<LOG2P, false>;
     using FI = WF<LOG2P, true>;
     constexpr int N = 1 << LOG2P, TPL = F::TPL, NP = F::NP;
@@ -49,7 +52,7 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
     PlaneTw<LOG2P, false> tw;
     tw.init(l, twt, twt + N, tid, kCoreThreads);
     PlaneTw<LOG2P, true> twi;
-    twi.init(l, twt, twt + 2 * N, tid, kCoreThreads);
+    twi.init(l, twt, twt + N + PlaneTw<LOG2P, false>::TABLE, tid, kCoreThreads);
     __syncthreads();
     const long long tpo = (p.nc + TX - 1) / TX;
     const long long tiles = p.n_outer * tpo;
@@ -183,8 +186,9 @@ __global__ void __launch_bounds__(kCoreThreads, (LOG2P >= 10 ? 1 : 2)) axis_core
 template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t st)
 {
     using F = WF<LOG2P, false>;
+    constexpr int kCoreThreads = core_threads(LOG2P);
     constexpr int N = 1 << LOG2P, TX = kCoreThreads / F::TPL;
-    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + 3 * N);
+    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + N + PlaneTw<LOG2P, false>::TABLE + PlaneTw<LOG2P, true>::TABLE);
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -195,7 +199,8 @@ template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t 
     static DevOnce attr;
     if (attr.first()) cudaFuncSetAttribute(axis_core_w_kernel<LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     const long long tiles = a.n_outer * ((a.nc + TX - 1) / TX);
-    const int grid = (int)(tiles < (long long)sms * 2 ? tiles : (long long)sms * 2);
+    const long long res = (long long)sms * 2;
+    const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
     axis_core_w_kernel<LOG2P><<<grid, kCoreThreads, sm, st>>>(a);
     return 1;
