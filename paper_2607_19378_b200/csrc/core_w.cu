@@ -27,6 +27,20 @@ __device__ __forceinline__ void cp_async8_s(unsigned smem_addr, const void *gmem
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
+// Line stride.  Tile copies and the final stores walk the lines with one lane per line (x) and
+// row (pos): with 16 or more lines per tile a half warp touches 16 lines at one row and any odd stride
+// separates them; with 8 lines it touches 8 lines at two neighbouring rows, which a stride of
+// 2 mod 16 separates.
+template <int LOG2P> __host__ __device__ constexpr int core_ls()
+{
+    using F = WF<LOG2P, false>;
+    constexpr int N = 1 << LOG2P, TX = core_threads(LOG2P) / F::TPL;
+    if (TX >= 16) return line_stride(N);
+    int n = (F::ph(N - 1) > WF<LOG2P, true>::ph(N - 1) ? F::ph(N - 1) : WF<LOG2P, true>::ph(N - 1)) + 1;
+    while (n % 16 != 2) ++n;
+    return n;
+}
+
 template <int LOG2P>
 __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) axis_core_w_kernel(AxisArgs p)
 {
@@ -35,7 +49,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
     using FI = WF<LOG2P, true>;
     constexpr int N = 1 << LOG2P, TPL = F::TPL, NP = F::NP;
     constexpr int TX = kCoreThreads / TPL;                 // lines per tile
-    constexpr int LS = line_stride(N);
+    constexpr int LS = core_ls<LOG2P>();
     using PL = typename F::template Pass<NP - 1>;          // last forward pass == first inverse pass
     extern __shared__ float2 smem[];
     float2 *bu = smem;
@@ -188,7 +202,7 @@ template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t 
     using F = WF<LOG2P, false>;
     constexpr int kCoreThreads = core_threads(LOG2P);
     constexpr int N = 1 << LOG2P, TX = kCoreThreads / F::TPL;
-    const size_t sm = sizeof(float2) * ((size_t)2 * TX * line_stride(N) + N + PlaneTw<LOG2P, false>::TABLE + PlaneTw<LOG2P, true>::TABLE);
+    const size_t sm = sizeof(float2) * ((size_t)2 * TX * core_ls<LOG2P>() + N + PlaneTw<LOG2P, false>::TABLE + PlaneTw<LOG2P, true>::TABLE);
     static int sms = 0;
     if (!sms) {
         int dev = 0;
