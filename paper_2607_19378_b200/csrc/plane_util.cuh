@@ -41,6 +41,10 @@ __device__ __forceinline__ void stage_row(unsigned char *dst, const unsigned cha
 {
     const unsigned char *a = src - ((unsigned long long)src & 15ull);
     const int nch = (int)((src + n - a + 15) >> 4);
+    if (a >= lo && a + 16 * nch <= hi) {                   // all but the first and last rows of a tensor
+        for (int c = l; c < nch; c += TPL) cp_async16(dst + 16 * c, a + 16 * c);
+        return;
+    }
     for (int c = l; c < nch; c += TPL) {
         const unsigned char *g = a + 16 * c;
         if (g >= lo && g + 16 <= hi) cp_async16(dst + 16 * c, g);
