@@ -202,6 +202,58 @@ def time_e2e(w: W.Workload, plan, tensors, steps: int, dist):
     return dt * 1e3, h2d, d2h
 
 
+def cufft_composition(w: W.Workload, tensors, reps: int = 3):
+    """Reference point only (never on the product path): the same operator written as a composition of
+    library calls -- torch.fft (cuFFT) real transforms in fp32 on the padded grid, spectral product,
+    inverse, crop, gate -- on the same device-resident inputs, in chunks of slices that bound its memory.
+    Returns its time per forward and its error against our result."""
+    q, k, v, h, y = tensors
+    nd = len(w.dims)
+    P = [1 << max(0, (2 * L - 2)).bit_length() if L > 1 else 1 for L in w.dims]
+    S = w.B * w.C
+    axes = tuple(range(1, nd + 1))
+    qf, kf, vf = (t.reshape(S, *w.dims) for t in (q, k, v))
+    hf = h.reshape(-1, *h.shape[-nd:])                        # [S or C, K...]
+    per_slice = 4 * 6 * int(torch.tensor(P).prod())           # bytes of fp32 work arrays per slice, roughly
+    chunk = max(1, min(S, int(4e9) // max(per_slice, 1)))
+    out = torch.empty_like(qf)
+    crop0 = [0 if w.causal else L - 1 for L in w.dims]
+
+    def run():
+        for s0 in range(0, S, chunk):
+            s1 = min(S, s0 + chunk)
+            u = kf[s0:s1].float() * vf[s0:s1].float()
+            if w.h_shared:
+                idx = torch.arange(s0, s1, device=q.device) % w.C
+                hh = hf[idx].float()
+            else:
+                hh = hf[s0:s1].float()
+            Y = torch.fft.irfftn(torch.fft.rfftn(u, s=P, dim=axes) * torch.fft.rfftn(hh, s=P, dim=axes), s=P, dim=axes)
+            sl = (slice(None),) + tuple(slice(c, c + L) for c, L in zip(crop0, w.dims))
+            out[s0:s1] = (qf[s0:s1].float() * Y[sl]).to(out.dtype)
+
+    run()
+    if q.is_cuda:
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+    else:                                                     # host tensors: only the unit test comes here
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            run()
+        ms = (time.perf_counter() - t0) / reps * 1e3
+    a, b = out.reshape(-1)[:1 << 24].double(), y.reshape(-1)[:1 << 24].double()
+    diff = float((a - b).norm() / b.norm().clamp_min(1e-300))
+    return {"kind": "torch.fft (cuFFT) composition, fp32, same inputs", "ms_per_step": ms,
+            "value": w.elements / (ms * 1e-3) / 1e9, "unit": UNIT, "slices_per_chunk": chunk,
+            "rel_l2_vs_ours_first_16M": diff}
+
+
 def cpu_oracle_sample(w: W.Workload, budget_s: float = 15.0):
     """Times the oracle (as it stands) on a bounded sample of slices of the workload."""
     import oracle
@@ -295,6 +347,12 @@ def main_ours(args):
     e2e_ms, h2d, d2h = time_e2e(w, plan, tensors, max(2, min(args.steps, 5)), dist)
     ms, e2e_ms = max_over_ranks([ms, e2e_ms], dist, device)
     plan.close()
+    cufft_ref = None
+    if world == 1 and not args.no_cufft:
+        try:
+            cufft_ref = cufft_composition(w, tensors)
+        except Exception as exc:                              # reference point only: never fails the bench
+            cufft_ref = {"unavailable": repr(exc)[:200]}
     del tensors
     torch.cuda.empty_cache()
 
@@ -329,6 +387,8 @@ def main_ours(args):
                     for kk in kernels],
         "workspace_bytes": res["workspace_bytes"],
     }
+    if cufft_ref is not None:
+        out["cufft_reference"] = cufft_ref
     if world == 1 and rank == 0:
         if not args.no_all:
             table = []
@@ -408,6 +468,7 @@ if __name__ == "__main__":
     ap.add_argument("--channels", type=int, default=None, help="override C (profiling on a smaller case)")
     ap.add_argument("--no-all", action="store_true", help="skip the table over the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--no-cufft", action="store_true", help="skip the torch.fft (cuFFT) composition reference point")
     a = ap.parse_args()
     if a.impl == "reference":
         main_reference(a)

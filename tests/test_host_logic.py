@@ -5,6 +5,7 @@ import os
 import re
 
 import pytest
+import torch
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 HEADER = os.path.join(ROOT, "include", "hyenand.h")
@@ -63,3 +64,22 @@ def test_null_plan_is_rejected_everywhere(lib):
     assert L.hyenand_plan_workspace_bytes(None) == 0
     assert L.hyenand_plan_launches(None, 0) == 0
     L.hyenand_destroy_plan(None)
+
+
+def test_cufft_composition_reference_matches_oracle():
+    """The library-composition reference point of bench.py computes the same operator as the oracle
+    (checked on host tensors; on the GPU machine it is only timed beside the product path)."""
+    import dataclasses
+    import bench
+    import oracle
+    from paper_2607_19378_b200 import workloads as W
+    cases = [W.WORKLOADS["tiny2d"],
+             dataclasses.replace(W.WORKLOADS["genomics1d"], dims=(200,), B=2, C=3),
+             dataclasses.replace(W.WORKLOADS["volume3d"], dims=(6, 5, 7), B=1, C=2, dtype="f32")]
+    for w in cases:
+        q, k, v, h = W.make_inputs(w, device="cpu")
+        yref = oracle.conv_fft(oracle.to_f64(q), oracle.to_f64(k), oracle.to_f64(v), oracle.to_f64(h),
+                               mode="causal" if w.causal else "linear")
+        y = torch.from_numpy(yref).to(q.dtype)
+        r = bench.cufft_composition(w, (q, k, v, h, y), reps=1)
+        assert r["rel_l2_vs_ours_first_16M"] < (1e-5 if w.dtype == "f32" else 4e-3), (w.name, r)
