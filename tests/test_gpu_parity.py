@@ -50,8 +50,8 @@ def check(w, q, k, v, h, full_direct=False):
     return err
 
 
-SHAPES_1D = [(1,), (2,), (3,), (5,), (17,), (64,), (1000,), (4096,)]
-SHAPES_ND = [(3, 5), (15, 14), (32, 32), (33, 70), (64, 64), (1, 9), (9, 1),
+SHAPES_1D = [(1,), (2,), (3,), (5,), (17,), (64,), (200,), (400,), (1000,), (4096,)]
+SHAPES_ND = [(3, 5), (15, 14), (32, 32), (33, 70), (64, 64), (1, 9), (9, 1), (150, 200), (300, 129),
              (5, 3, 2), (7, 1, 4), (16, 16, 16), (20, 9, 12), (1, 1, 6)]
 
 
