@@ -311,12 +311,29 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
     const int Lx = p.lx, Ly = p.ly;
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const float2 *src = p.in + pl * (long long)C::XH * P;
+        // Column kx + NG is requested (into registers) between the two passes of column kx: the loads
+        // are in flight during the second pass and the stores, and the registers are free by then.
+        static_assert(FI::NP == 2, "two-pass plans");
+        using P0 = typename FI::template Pass<0>;
+        float2 pre[P0::IPL][P0::R];
+        auto fetch = [&](int kx) {
+            const float2 *s = src + (long long)kx * P + l;
+#pragma unroll
+            for (int i = 0; i < P0::IPL; ++i)
+#pragma unroll
+                for (int r = 0; r < P0::R; ++r) pre[i][r] = __ldcg(s + i * TPL + r * (P / P0::R));
+        };
+        if (gid != 0 && gid < HP) fetch(gid);
         for (int kx = gid; kx < HP; kx += C::NG) {
             float2 *col = cs + kx * C::CSS;
             if (kx != 0) {
-                const float2 *s = src + (long long)kx * P;
-                FI::template run<PRUNE_OUT>(l, m, twp, line,
-                    [&](int, int, int idx) { return s[idx]; },
+                FI::template pass<0, PRUNE_NONE>(l, twp,
+                    [&](int i, int r, int) { return pre[i][r]; },
+                    [&](int, int, int idx, float2 v) { line[FI::ph(idx)] = v; });
+                __syncwarp(m);
+                if (kx + C::NG < HP) fetch(kx + C::NG);
+                FI::template pass<1, PRUNE_OUT>(l, twp,
+                    [&](int, int, int idx) { return line[FI::ph(idx)]; },
                     [&](int, int, int idx, float2 v) { col[idx] = v; });
             } else {
                 const float2 *sn = src + (long long)HP * P;
@@ -326,6 +343,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
                         return make_float2(g0.x - gn.y, g0.y + gn.x);
                     },
                     [&](int, int, int idx, float2 v) { col[idx] = v; });
+                if (kx + C::NG < HP) fetch(kx + C::NG);
             }
             __syncwarp(m);
         }
@@ -340,6 +358,18 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
             const int y0 = 2 * rp, y1 = y0 + 1;
             const bool has1 = y1 < Ly;
             const long long o0 = ob + (long long)y0 * Lx, o1 = o0 + Lx;
+            // the gate values of this lane's outputs are requested before the transform starts
+            using PE = typename FI::LastPass;
+            constexpr int NQ = PE::IPL * (PE::R / 2);
+            T q0[NQ], q1[NQ];
+#pragma unroll
+            for (int i = 0; i < PE::IPL; ++i)
+#pragma unroll
+                for (int r = 0; r < PE::R / 2; ++r) {
+                    const int idx = FI::last_pos(l, i, r);
+                    q0[i * (PE::R / 2) + r] = idx < Lx ? __ldg(pq + o0 + idx) : T(0.f);
+                    q1[i * (PE::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
+                }
             FI::template run<PRUNE_OUT>(l, m, twp, line,
                 [&](int, int, int idx) {
                     // branch-free merge of two half spectra into one complex row (column 0 is packed)
@@ -355,10 +385,10 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
                     g = kx == HP ? make_float2(A.y, B.y) : g;
                     return g;
                 },
-                [&](int, int, int idx, float2 v) {
+                [&](int i, int r, int idx, float2 v) {
                     if (idx < Lx) {
-                        IO<T>::st(py, o0 + idx, v.x * IO<T>::ld(pq, o0 + idx));
-                        if (has1) IO<T>::st(py, o1 + idx, v.y * IO<T>::ld(pq, o1 + idx));
+                        IO<T>::st(py, o0 + idx, v.x * (float)q0[i * (PE::R / 2) + r]);
+                        if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[i * (PE::R / 2) + r]);
                     }
                 });
             __syncwarp(m);
