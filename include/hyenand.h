@@ -107,6 +107,13 @@ const char *hyenand_last_error(void);
  * tells why hyenand_create_plan returned NULL. */
 int hyenand_last_error_code(void);
 
+/* Device-side status of the plan's kernels.  Every wait a kernel makes on an asynchronous copy is
+ * bounded; a kernel whose wait gave up writes a non-zero code here and returns instead of hanging.
+ * Reads that word back (a blocking device-to-host copy of 4 bytes: call it after synchronising the
+ * stream).  Returns 0 if no kernel reported anything, the code otherwise, -1 on error.  The paper has
+ * no counterpart; it exists so that a failed copy is observable from the host. */
+int hyenand_plan_device_status(hyenand_plan *plan);
+
 /* Reporting helpers (host-only, no device work). */
 size_t hyenand_plan_workspace_bytes(const hyenand_plan *plan);        /* device bytes owned by the plan */
 int hyenand_plan_fft_dims(const hyenand_plan *plan, int *out_P);      /* writes ndim padded sizes P_n */

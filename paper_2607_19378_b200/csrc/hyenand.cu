@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "ct1d.cuh"
 #include "planes.cuh"
+#include "core_tma.cuh"
 #include "fused2d.cuh"
 
 using namespace hn;
@@ -47,6 +48,9 @@ struct hyenand_plan {
     long long wh_slices;              // slices the filter workspace holds
     float2 *gtw;
     int gtw_n;
+    // 3-D path: tensor maps of the z core's workspace buffers (valid only if the TMA core applies)
+    CoreTmaMaps tma;
+    int *dev_status;                  // device word set by a kernel whose bounded wait gave up
     // long 1-D path
     Ct1dPlan ct;
     // host-staging for hyenand_forward_host
@@ -87,13 +91,15 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
     int cur = 0;
     cudaGetDevice(&cur);
     if (cur != p->device) cudaSetDevice(p->device);
-    cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw);
+    cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw); cudaFree(p->dev_status);
     ct1d_free(&p->ct);
     for (int i = 0; i < 5; ++i) cudaFree(p->stage[i]);
     p->prof.destroy();
     if (cur != p->device) cudaSetDevice(cur);
     delete p;
 }
+
+static AxisArgs planes3d_core_args(const hyenand_plan *p, long long n, bool shared, long long s0);
 
 extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype)
 {
@@ -189,8 +195,25 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     if (!e && p->wh_b_slice) e = dev_alloc(p, (void **)&p->wh_b, sizeof(float2) * p->wh_b_slice * p->wh_slices);
     if (!e && cudaMemcpy(p->gtw, tw.data(), sizeof(float2) * p->gtw_n, cudaMemcpyHostToDevice) != cudaSuccess)
         e = fail(HYENAND_ERR_CUDA, "twiddle upload failed: %s", cudaGetErrorString(cudaGetLastError()));
+    if (!e) e = dev_alloc(p, (void **)&p->dev_status, sizeof(int));
+    if (!e && cudaMemset(p->dev_status, 0, sizeof(int)) != cudaSuccess)
+        e = fail(HYENAND_ERR_CUDA, "status word: %s", cudaGetErrorString(cudaGetLastError()));
     if (e) { hyenand_destroy_plan(p); return nullptr; }
+    if (p->path == PATH_PLANES3D)      // tensor maps of the z core's buffers; left invalid where the TMA core does not apply
+        core_tma_make(&p->tma, planes3d_core_args(p, spc, false, 0), spc, p->wh_slices);
     return p;
+}
+
+extern "C" int hyenand_plan_device_status(hyenand_plan *p)
+{
+    g_err[0] = 0;
+    if (!p) { fail(HYENAND_ERR_INVALID_ARG, "plan is NULL"); return -1; }
+    int v = 0;
+    if (cudaMemcpy(&v, p->dev_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        fail(HYENAND_ERR_CUDA, "reading the status word failed: %s", cudaGetErrorString(cudaGetLastError()));
+        return -1;
+    }
+    return v;
 }
 
 // ---- generic path scheduling -----------------------------------------------------------
@@ -314,6 +337,22 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
     return 0;
 }
 
+// arguments of the z core of the 3-D path for n slices starting at slice s0
+static AxisArgs planes3d_core_args(const hyenand_plan *p, long long n, bool shared, long long s0)
+{
+    const long long nc = (long long)p->XH * p->P[1];
+    AxisArgs a{};
+    a.in = p->ws_a; a.out = p->ws_a;
+    a.n_outer = n; a.in_outer = a.out_outer = (long long)p->L[0] * nc;
+    a.nc = (int)nc; a.n_in = p->L[0]; a.n_out = p->L[0]; a.shift = 0;
+    a.log2p = p->log2p[0]; a.prune_in = 1;
+    a.h = p->wh_a; a.h_outer = (long long)p->K[0] * nc; a.h_n_in = p->K[0]; a.h_shift = p->L[0] - 1;
+    a.h_mod = shared ? p->C : 0; a.h_off = shared ? s0 % p->C : 0;
+    a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
+    a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+    return a;
+}
+
 static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const char *v, const char *h,
                             bool shared, char *y, cudaStream_t st, int *launches)
 {
@@ -345,17 +384,12 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;
-        AxisArgs a{};
-        a.in = p->ws_a; a.out = p->ws_a;
-        a.n_outer = n; a.in_outer = a.out_outer = (long long)p->L[0] * nc;
-        a.nc = (int)nc; a.n_in = p->L[0]; a.n_out = p->L[0]; a.shift = 0;
-        a.log2p = p->log2p[0]; a.prune_in = 1;
-        a.h = p->wh_a; a.h_outer = (long long)p->K[0] * nc; a.h_n_in = p->K[0]; a.h_shift = p->L[0] - 1;
-        a.h_mod = shared ? p->C : 0; a.h_off = shared ? s0 % p->C : 0;
-        a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
-        a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        const AxisArgs a = planes3d_core_args(p, n, shared, s0);
         p->prof.begin(KID_CORE, st);
-        c = (core_w_supported(a.log2p) && !getenv("HYENAND_GENERIC_CORE")) ? launch_core_w(a, st) : launch_axis(a, AXIS_CORE, st);
+        c = -1;
+        if (p->tma.valid && !getenv("HYENAND_NO_TMA")) c = launch_core_tma(a, p->tma, p->dev_status, st);
+        if (c < 0)
+            c = (core_w_supported(a.log2p) && !getenv("HYENAND_GENERIC_CORE")) ? launch_core_w(a, st) : launch_axis(a, AXIS_CORE, st);
         p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;

@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         L.hyenand_destroy_plan.argtypes = [vp]
         L.hyenand_destroy_plan.restype = None
         L.hyenand_last_error.restype = ctypes.c_char_p
+        L.hyenand_plan_device_status.argtypes = [vp]
+        L.hyenand_plan_device_status.restype = ctypes.c_int
         L.hyenand_plan_workspace_bytes.argtypes = [vp]
         L.hyenand_plan_workspace_bytes.restype = ctypes.c_size_t
         L.hyenand_plan_fft_dims.argtypes = [vp, ip]
@@ -114,6 +116,11 @@ def hyenand_forward_ex(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stre
 def hyenand_forward_host(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stream=None) -> None:
     _check(lib().hyenand_forward_host(plan, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
                                       int(h_batch_stride_elems), y.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_plan_device_status(plan: int) -> int:
+    """0 unless a kernel of the plan gave up a bounded wait (synchronise the stream first)."""
+    return int(lib().hyenand_plan_device_status(plan))
 
 
 def hyenand_plan_workspace_bytes(plan: int) -> int:

@@ -114,6 +114,30 @@ def test_fused_2d_path(dims, dtype, shared):
     check(w, q, k, v, h)
 
 
+TMA_CORE_SHAPES = [(70, 40, 50), (128, 33, 64), (65, 64, 64), (100, 65, 70)]
+
+
+@pytest.mark.parametrize("dtype,shared", [("f32", False), ("bf16", False), ("f32", True)])
+@pytest.mark.parametrize("dims", TMA_CORE_SHAPES, ids=str)
+def test_plane_fused_3d_with_256_point_depth_axis(dims, dtype, shared):
+    """A depth axis padded to 256 points takes the spectral core whose tiles move as tensor (TMA)
+    copies; its bounded waits must not have given up (device status 0)."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem(dims, B=2, C=2, dtype=dtype, h_shared=shared, seed=27)
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    try:
+        assert hn.hyenand_plan_path(plan.handle) == "planes3d"
+        dq, dk, dv, dh = (t.cuda() for t in (q, k, v, h))
+        y = torch.full_like(dq, float("nan"))
+        plan.forward(dq, dk, dv, dh, y)
+        plan.forward(dq, dk, dv, dh, y)                     # a second pass over the same buffers
+        torch.cuda.synchronize()
+        assert hn.hyenand_plan_device_status(plan.handle) == 0
+    finally:
+        plan.close()
+    check(w, q, k, v, h)
+
+
 def test_plane_fused_3d_shared_filter():
     w, (q, k, v, h) = W.random_problem((3, 40, 50), B=3, C=2, dtype="f32", h_shared=True, seed=22)
     check(w, q, k, v, h)
