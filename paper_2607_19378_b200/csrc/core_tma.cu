@@ -1,16 +1,16 @@
-// Fused spectral core along a strided axis for 256-point lines, tiles moved by TMA.
+// Fused spectral core along a strided axis for 256- and 1024-point lines, tiles moved by TMA.
 //
 // Same arithmetic as core_w.cu (forward transform of the filter lines, forward transform of the
 // k*v lines, spectral product of Eq. 12 of the paper, inverse, cropped half written back in
-// place), but the tiles -- 16 adjacent bins by all rows of the axis -- travel as tensor copies:
+// place), but the tiles -- 16 (8 for 1024-point lines) adjacent bins by all rows of the axis -- travel as tensor copies:
 //
-//   cp.async.bulk.tensor loads   filter tile (two boxes of 128 rows: the wrapped placement of the
+//   cp.async.bulk.tensor loads   filter tile (boxes of up to 256 rows; the wrapped placement of the
 //                                taps is two row ranges) and k*v tile (one box; rows past the data
 //                                and bins past the end come back as zeros)
 //   cp.async.bulk.tensor store   the cropped result tile
 //
 // One elected thread issues them; nobody computes addresses or waits per element.  The boxes land
-// row-major (128 bytes per row) with the 128-byte swizzle, which spreads the 16 rows a group of
+// row-major (one 64- or 128-byte row per axis position) with the matching swizzle, which spreads the rows a group of
 // lanes reads at once over 8 bank groups.  A tile buffer is free again as soon as the first pass
 // has read it, so the next tile's copy runs under the rest of this tile's arithmetic.
 //
@@ -24,14 +24,32 @@
 
 namespace hn {
 
-constexpr int kTmaLog2 = 8;
-constexpr int kTmaN = 1 << kTmaLog2;                 // line length
 constexpr int kTmaThreads = 256;
-constexpr int kTmaTX = 16;                           // bins per tile (one 128-byte row)
-constexpr int kTmaHalf = kTmaN / 2;                  // rows per box
-constexpr unsigned kRowBytes = kTmaTX * 8;           // 128
-constexpr unsigned kBoxBytes = kTmaHalf * kRowBytes; // 16 KB
 constexpr int kWaitLimit = 1 << 22;                  // polls of a barrier before giving up
+
+// Geometry of a tile for LOG2P-point lines: one line per group of TPL lanes, so TX = 256 / TPL bins
+// per tile and TX * 8 bytes per tile row (128 for 256-point lines, 64 for 1024-point lines: the
+// swizzle span of the tensor maps).  A box holds at most 256 rows.
+template <int LOG2P> struct TmaGeo {
+    using F = WF<LOG2P, false>;
+    static constexpr int N = 1 << LOG2P, HALF = N / 2;
+    static constexpr int TX = kTmaThreads / F::TPL;
+    static constexpr unsigned ROWB = TX * 8;
+    static constexpr int BOXR = HALF < 256 ? HALF : 256;             // rows per box
+    static constexpr int NB = HALF / BOXR;                           // boxes per half line
+    static constexpr unsigned BOXB = BOXR * ROWB;
+    static constexpr unsigned HALFB = HALF * ROWB;
+    static constexpr int LS = TX >= 16 ? line_stride(N) : ((F::ph(N - 1) + 1 + 15) / 16 * 16 + 2);
+    static_assert(ROWB == 128 || ROWB == 64, "tile rows match a swizzle span");
+    // shared memory: tile buffers first (1024-byte aligned, as the swizzle pattern repeats every 1024 bytes)
+    static constexpr size_t TH = 0;                                  // filter tile, N rows
+    static constexpr size_t TU = TH + 2 * HALFB;                     // k*v tile, N/2 rows
+    static constexpr size_t TO = TU + HALFB;                         // result tile, N/2 rows
+    static constexpr size_t LINES = TO + HALFB;                      // one skewed line per group
+    static constexpr size_t TW = LINES + sizeof(float2) * TX * LS;
+    static constexpr size_t BARS = TW + sizeof(float2) * N;
+    static constexpr size_t TOTAL = BARS + 2 * sizeof(uint64_t) + 1024;    // + room to align the start
+};
 
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t *b, unsigned count)
@@ -83,40 +101,32 @@ struct CoreTmaParams {
     int *status;              // device word: 0 ok, else which wait gave up
 };
 
-// shared memory: tile buffers first (1024-byte aligned, as the swizzle pattern repeats every 8 rows)
-struct CoreTmaSmem {
-    static constexpr int LS = line_stride(kTmaN);
-    static constexpr size_t TH = 0;                                  // filter tile, 256 rows
-    static constexpr size_t TU = TH + 2 * kBoxBytes;                 // k*v tile, 128 rows
-    static constexpr size_t TO = TU + kBoxBytes;                     // result tile, 128 rows
-    static constexpr size_t LINES = TO + kBoxBytes;                  // one skewed line per group
-    static constexpr size_t TW = LINES + sizeof(float2) * kTmaTX * LS;
-    static constexpr size_t BARS = TW + sizeof(float2) * kTmaN;
-    static constexpr size_t TOTAL = BARS + 2 * sizeof(uint64_t) + 1024;    // + room to align the start
-};
-
-__global__ void __launch_bounds__(kTmaThreads, 2)
+template <int LOG2P>
+__global__ void __launch_bounds__(kTmaThreads, (LOG2P >= 10 ? 1 : 2))
 axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_h, CoreTmaParams p)
 {
-    using F = WF<kTmaLog2, false>;
-    using FI = WF<kTmaLog2, true>;
-    constexpr int N = kTmaN, TPL = F::TPL, NP = F::NP;
-    static_assert(TPL == 16 && NP == 2 && kTmaThreads / TPL == kTmaTX, "tile = one line per group of 16 lanes");
+    using G = TmaGeo<LOG2P>;
+    using F = WF<LOG2P, false>;
+    using FI = WF<LOG2P, true>;
+    constexpr int N = G::N, TPL = F::TPL, NP = F::NP;
+    static_assert(NP == 2 && F::radix(0) == F::radix(1), "two equal passes: one register set of twiddles serves both directions");
     using PL = typename F::template Pass<NP - 1>;
-    using PE = typename FI::template Pass<NP - 1>;
+    using P0 = typename F::template Pass<0>;
+    static_assert(P0::IPL == 1 && PL::IPL == 1, "one item per lane and pass");
+    constexpr int RSTEP = (N / P0::R) * (int)G::ROWB / 8;            // float2 between legs r and r+1 of a lane in a tile
     extern __shared__ __align__(1024) unsigned char smem_dyn[];
     // the swizzle pattern is a function of the shared-memory address: start on a 1024-byte boundary
     unsigned char *smem_raw = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
-    unsigned char *th = smem_raw + CoreTmaSmem::TH;
-    unsigned char *tu = smem_raw + CoreTmaSmem::TU;
-    unsigned char *to = smem_raw + CoreTmaSmem::TO;
-    float2 *lines = reinterpret_cast<float2 *>(smem_raw + CoreTmaSmem::LINES);
-    float2 *twt = reinterpret_cast<float2 *>(smem_raw + CoreTmaSmem::TW);
-    uint64_t *bar_h = reinterpret_cast<uint64_t *>(smem_raw + CoreTmaSmem::BARS);
+    unsigned char *th = smem_raw + G::TH;
+    unsigned char *tu = smem_raw + G::TU;
+    unsigned char *to = smem_raw + G::TO;
+    float2 *lines = reinterpret_cast<float2 *>(smem_raw + G::LINES);
+    float2 *twt = reinterpret_cast<float2 *>(smem_raw + G::TW);
+    uint64_t *bar_h = reinterpret_cast<uint64_t *>(smem_raw + G::BARS);
     uint64_t *bar_u = bar_h + 1;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
-    float2 *line = lines + gid * CoreTmaSmem::LS;
+    float2 *line = lines + gid * G::LS;
     for (int t = tid; t < N; t += kTmaThreads) twt[t] = p.gtw[t * (p.gtw_n / N)];
     if (tid == 0) {
         mbar_init(bar_h, 1);
@@ -124,28 +134,37 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
         fence_mbar_init();
     }
     __syncthreads();
-    PlaneTw<kTmaLog2, false> tw;
-    tw.init(l, twt, twt, tid, kTmaThreads);            // 16 x 16: twiddles live in registers, no table
-    static_assert(PlaneTw<kTmaLog2, false>::HOIST && PlaneTw<kTmaLog2, true>::HOIST, "register twiddles");
-    PlaneTw<kTmaLog2, true> twi;
-    twi.init(l, twt, twt, tid, kTmaThreads);
-    // Row z = l + 16 r of bin `gid` inside a swizzled tile: 128 bytes per row, the 16-byte chunk index
-    // is XORed with (z & 7) = (l & 7), so every r is the same per-lane offset plus r * 2048 bytes.
-    const unsigned tile_off = (unsigned)l * kRowBytes + ((((unsigned)gid >> 1) ^ ((unsigned)l & 7u)) << 4) + ((unsigned)gid & 1u) * 8u;
+    // two equal passes: the twiddles depend on the lane only and live in registers; the inverse uses the
+    // same values conjugated, so one set serves both directions
+    PlaneTw<LOG2P, false> tw;
+    static_assert(PlaneTw<LOG2P, false>::HOIST, "register twiddles");
+    tw.init(l, twt, twt, tid, kTmaThreads);
+    // Row z = l + TPL*r of bin `gid` inside a swizzled tile.  A row is ROWB bytes; the 16-byte chunk index
+    // of an address is XORed with address bits 7 and up (3 bits for the 128-byte swizzle, 2 for the 64-byte
+    // one), i.e. with a function of z that TPL*r does not change: every leg r is the same per-lane offset
+    // plus a constant.
+    constexpr unsigned ZSH = G::ROWB == 128 ? 0 : 1, ZMASK = G::ROWB == 128 ? 7u : 3u;
+    const unsigned tile_off = (unsigned)l * G::ROWB
+                            + ((((unsigned)gid >> 1) ^ (((unsigned)l >> ZSH) & ZMASK)) << 4) + ((unsigned)gid & 1u) * 8u;
     const long long tiles = p.n_outer * p.tiles_per_outer;
     auto issue_h = [&](long long t) {                  // one thread
         const long long o = t / p.tiles_per_outer;
-        const int x = (int)(t % p.tiles_per_outer) * kTmaTX * 2;          // in floats
+        const int x = (int)(t % p.tiles_per_outer) * G::TX * 2;          // in floats
         const long long oh = p.h_mod ? (o + p.h_off) % p.h_mod : o;
-        mbar_expect_tx(bar_h, 2 * kBoxBytes);
-        tma_load_3d(th, &map_h, bar_h, x, p.h_shift, (int)oh);                        // positions [0, 128)
-        tma_load_3d(th + kBoxBytes, &map_h, bar_h, x, p.h_shift - kTmaHalf, (int)oh); // positions [128, 256)
+        mbar_expect_tx(bar_h, 2 * G::HALFB);
+#pragma unroll
+        for (int b = 0; b < G::NB; ++b) {
+            // positions [0, N/2) hold filter rows from h_shift on, positions [N/2, N) the rows before it
+            tma_load_3d(th + b * G::BOXB, &map_h, bar_h, x, p.h_shift + b * G::BOXR, (int)oh);
+            tma_load_3d(th + G::HALFB + b * G::BOXB, &map_h, bar_h, x, p.h_shift - G::HALF + b * G::BOXR, (int)oh);
+        }
     };
     auto issue_u = [&](long long t) {
         const long long o = t / p.tiles_per_outer;
-        const int x = (int)(t % p.tiles_per_outer) * kTmaTX * 2;
-        mbar_expect_tx(bar_u, kBoxBytes);
-        tma_load_3d(tu, &map_u, bar_u, x, 0, (int)o);
+        const int x = (int)(t % p.tiles_per_outer) * G::TX * 2;
+        mbar_expect_tx(bar_u, G::HALFB);
+#pragma unroll
+        for (int b = 0; b < G::NB; ++b) tma_load_3d(tu + b * G::BOXB, &map_u, bar_u, x, b * G::BOXR, (int)o);
     };
     long long t = blockIdx.x;
     if (tid == 0 && t < tiles) { issue_h(t); issue_u(t); }
@@ -153,58 +172,59 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
     int failed = 0;
     for (; t < tiles; t += gridDim.x, phase ^= 1u) {
         const long long tn = t + gridDim.x;
-        float2 H[PL::IPL][PL::R];
+        float2 H[PL::R];
         // ---- filter lines: tile -> registers ------------------------------------------------------
         if (!mbar_wait(bar_h, phase)) failed = 1;
         {
             const float2 *src = reinterpret_cast<const float2 *>(th + tile_off);
             F::template pass<0, PRUNE_NONE>(l, tw,
-                [&](int, int r, int) { return src[r * (2048 / 8)]; },
+                [&](int, int r, int) { return src[r * RSTEP]; },
                 [&](int, int, int idx, float2 v) { line[F::ph(idx)] = v; });
         }
         if (__syncthreads_or(failed)) break;           // the filter tile buffer is free again
         if (tid == 0 && tn < tiles) issue_h(tn);
         F::template pass<NP - 1, PRUNE_NONE>(l, tw,
             [&](int, int, int idx) { return line[F::ph(idx)]; },
-            [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * p.scale); });
+            [&](int, int r, int, float2 v) { H[r] = make_float2(v.x * p.scale, v.y * p.scale); });
         __syncwarp(m);
         // ---- k*v lines: tile -> spectrum, product, inverse ----------------------------------------
         if (!mbar_wait(bar_u, phase)) failed = 2;
         {
             const float2 *src = reinterpret_cast<const float2 *>(tu + tile_off);
             F::template pass<0, PRUNE_IN>(l, tw,
-                [&](int, int r, int) { return src[r * (2048 / 8)]; },
+                [&](int, int r, int) { return src[r * RSTEP]; },
                 [&](int, int, int idx, float2 v) { line[F::ph(idx)] = v; });
         }
         if (tid == 0) tma_wait_read0();                // the previous result tile has left its buffer
         if (__syncthreads_or(failed)) break;           // the k*v tile buffer is free again
         if (tid == 0 && tn < tiles) issue_u(tn);
-        float2 Y[PL::IPL][PL::R];
+        float2 Y[PL::R];
         F::template pass<NP - 1, PRUNE_NONE>(l, tw,
             [&](int, int, int idx) { return line[F::ph(idx)]; },
-            [&](int i, int r, int, float2 v) { Y[i][r] = cmul(v, H[i][r]); });
+            [&](int, int r, int, float2 v) { Y[r] = cmul(v, H[r]); });
         __syncwarp(m);
-        FI::template pass<0, PRUNE_NONE>(l, twi,
-            [&](int i, int r, int) { return Y[i][r]; },
+        FI::template pass<0, PRUNE_NONE>(l, tw,
+            [&](int, int r, int) { return Y[r]; },
             [&](int, int, int idx, float2 v) { line[FI::ph(idx)] = v; });
         __syncwarp(m);
         {
             float2 *dst = reinterpret_cast<float2 *>(to + tile_off);
-            FI::template pass<NP - 1, PRUNE_OUT>(l, twi,
+            FI::template pass<NP - 1, PRUNE_OUT>(l, tw,
                 [&](int, int, int idx) { return line[FI::ph(idx)]; },
-                [&](int, int r, int, float2 v) { dst[r * (2048 / 8)] = v; });
+                [&](int, int r, int, float2 v) { dst[r * RSTEP] = v; });
         }
         __syncwarp(m);
         fence_async_smem();                            // generic-proxy writes visible to the copy engine
         __syncthreads();
         if (tid == 0) {
             const long long o = t / p.tiles_per_outer;
-            const int x = (int)(t % p.tiles_per_outer) * kTmaTX * 2;
-            tma_store_3d(&map_u, to, x, 0, (int)o);
+            const int x = (int)(t % p.tiles_per_outer) * G::TX * 2;
+#pragma unroll
+            for (int b = 0; b < G::NB; ++b) tma_store_3d(&map_u, to + b * G::BOXB, x, b * G::BOXR, (int)o);
             tma_commit();
         }
     }
-    if (failed || t < tiles) {
+    if (t < tiles) {
         // a wait gave up: say so, then give copies that may still be in flight a bounded time to land
         if (failed) atomicExch(p.status, failed);
         mbar_wait(bar_h, phase);
@@ -236,26 +256,32 @@ static EncodeTiledFn encode_fn()
     return fn;
 }
 
-// [outer][rows][nc] complex fp32, seen as fp32 with 2*nc entries per row; box = 32 floats x 128 rows
-static bool make_map(CUtensorMap *map, const float2 *base, long long outer, int rows, int nc, long long outer_stride_elems)
+// [outer][rows][nc] complex fp32, seen as fp32 with 2*nc entries per row; box = one tile row of 2*TX floats
+// by up to 256 rows, swizzled over the row's 64 or 128 bytes
+static bool make_map(CUtensorMap *map, const float2 *base, long long outer, int rows, int nc, long long outer_stride_elems,
+                     int tx, int box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)2 * nc, (cuuint64_t)rows, (cuuint64_t)outer};
     const cuuint64_t strides[2] = {(cuuint64_t)nc * 8, (cuuint64_t)outer_stride_elems * 8};
-    const cuuint32_t box[3] = {(cuuint32_t)kTmaTX * 2, (cuuint32_t)kTmaHalf, 1};
+    const cuuint32_t box[3] = {(cuuint32_t)tx * 2, (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     if ((strides[0] % 16) || (strides[1] % 16) || ((uintptr_t)base % 16)) return false;
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float2 *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_INTERLEAVE_NONE, tx * 8 == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+static bool tma_log2p_ok(int log2p) { return log2p == 8 || log2p == 10; }
 
 bool core_tma_supported(const AxisArgs &a)
 {
-    return a.log2p == kTmaLog2 && a.in == a.out && a.in_outer == a.out_outer && a.n_in == a.n_out &&
-           a.n_in >= 1 && a.n_in <= kTmaHalf && a.h_n_in >= 1 && a.h_n_in <= kTmaN && a.shift == 0 &&
-           a.h_shift >= 0 && a.h_shift < kTmaN && (a.nc % 2) == 0 && a.n_outer < (1ll << 31) && encode_fn() != nullptr;
+    if (!tma_log2p_ok(a.log2p)) return false;
+    const int n = 1 << a.log2p;
+    return a.in == a.out && a.in_outer == a.out_outer && a.n_in == a.n_out && a.n_in >= 1 && a.n_in <= n / 2 &&
+           a.h_n_in >= 1 && a.h_n_in <= n && a.shift == 0 && a.h_shift >= 0 && a.h_shift < n && (a.nc % 2) == 0 &&
+           a.n_outer < (1ll << 31) && encode_fn() != nullptr;
 }
 
 bool core_tma_make(CoreTmaMaps *m, const AxisArgs &a, long long max_outer, long long h_outer_count)
@@ -263,27 +289,21 @@ bool core_tma_make(CoreTmaMaps *m, const AxisArgs &a, long long max_outer, long 
     m->valid = false;
     if (!core_tma_supported(a)) return false;
     static_assert(sizeof(m->u) >= sizeof(CUtensorMap) && sizeof(m->h) >= sizeof(CUtensorMap), "room for a tensor map");
-    if (!make_map(reinterpret_cast<CUtensorMap *>(m->u), a.in, max_outer, a.n_in, a.nc, a.in_outer)) return false;
-    if (!make_map(reinterpret_cast<CUtensorMap *>(m->h), a.h, h_outer_count, a.h_n_in, a.nc, a.h_outer)) return false;
-    m->in = a.in; m->h_base = a.h; m->nc = a.nc; m->n_in = a.n_in; m->h_n_in = a.h_n_in;
+    const int tx = a.log2p == 8 ? TmaGeo<8>::TX : TmaGeo<10>::TX;
+    const int br = a.log2p == 8 ? TmaGeo<8>::BOXR : TmaGeo<10>::BOXR;
+    if (!make_map(reinterpret_cast<CUtensorMap *>(m->u), a.in, max_outer, a.n_in, a.nc, a.in_outer, tx, br)) return false;
+    if (!make_map(reinterpret_cast<CUtensorMap *>(m->h), a.h, h_outer_count, a.h_n_in, a.nc, a.h_outer, tx, br)) return false;
+    m->in = a.in; m->h_base = a.h; m->nc = a.nc; m->n_in = a.n_in; m->h_n_in = a.h_n_in; m->log2p = a.log2p;
     m->in_outer = a.in_outer; m->h_outer = a.h_outer; m->max_outer = max_outer; m->h_outer_count = h_outer_count;
     m->valid = true;
     return true;
 }
 
-int launch_core_tma(const AxisArgs &a, const CoreTmaMaps &m, int *status, cudaStream_t st)
+template <int LOG2P> static int launch_core_tma_t(const CoreTmaParams &p0, const CoreTmaMaps &m, int nc, cudaStream_t st)
 {
-    // the maps describe fixed buffers: refuse anything else
-    if (!m.valid || a.in != m.in || a.h != m.h_base || a.nc != m.nc || a.n_in != m.n_in || a.h_n_in != m.h_n_in ||
-        a.in_outer != m.in_outer || a.h_outer != m.h_outer || a.n_outer > m.max_outer || !core_tma_supported(a))
-        return -1;
-    const long long h_need = a.h_mod ? a.h_mod : a.n_outer;
-    if (h_need > m.h_outer_count) return -1;
-    CoreTmaParams p{};
-    p.n_outer = a.n_outer;
-    p.tiles_per_outer = (a.nc + kTmaTX - 1) / kTmaTX;
-    p.h_shift = a.h_shift; p.h_mod = a.h_mod; p.h_off = a.h_off;
-    p.scale = a.scale; p.gtw = a.gtw; p.gtw_n = a.gtw_n; p.status = status;
+    using G = TmaGeo<LOG2P>;
+    CoreTmaParams p = p0;
+    p.tiles_per_outer = (nc + G::TX - 1) / G::TX;
     static int sms = 0;
     if (!sms) {
         int dev = 0;
@@ -293,13 +313,30 @@ int launch_core_tma(const AxisArgs &a, const CoreTmaMaps &m, int *status, cudaSt
     }
     static DevOnce attr;
     if (attr.first())
-        cudaFuncSetAttribute(axis_core_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CoreTmaSmem::TOTAL);
+        cudaFuncSetAttribute(axis_core_tma_kernel<LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::TOTAL);
     const long long tiles = p.n_outer * p.tiles_per_outer;
-    const int grid = (int)(tiles < 2ll * sms ? tiles : 2ll * sms);
+    const long long res = (long long)sms * (LOG2P >= 10 ? 1 : 2);    // resident CTAs
+    const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
-    axis_core_tma_kernel<<<grid, kTmaThreads, CoreTmaSmem::TOTAL, st>>>(
+    axis_core_tma_kernel<LOG2P><<<grid, kTmaThreads, G::TOTAL, st>>>(
         *reinterpret_cast<const CUtensorMap *>(m.u), *reinterpret_cast<const CUtensorMap *>(m.h), p);
     return 1;
+}
+
+int launch_core_tma(const AxisArgs &a, const CoreTmaMaps &m, int *status, cudaStream_t st)
+{
+    // the maps describe fixed buffers: refuse anything else
+    if (!m.valid || a.log2p != m.log2p || a.in != m.in || a.h != m.h_base || a.nc != m.nc || a.n_in != m.n_in ||
+        a.h_n_in != m.h_n_in || a.in_outer != m.in_outer || a.h_outer != m.h_outer || a.n_outer > m.max_outer ||
+        !core_tma_supported(a))
+        return -1;
+    const long long h_need = a.h_mod ? a.h_mod : a.n_outer;
+    if (h_need > m.h_outer_count) return -1;
+    CoreTmaParams p{};
+    p.n_outer = a.n_outer;
+    p.h_shift = a.h_shift; p.h_mod = a.h_mod; p.h_off = a.h_off;
+    p.scale = a.scale; p.gtw = a.gtw; p.gtw_n = a.gtw_n; p.status = status;
+    return a.log2p == 8 ? launch_core_tma_t<8>(p, m, a.nc, st) : launch_core_tma_t<10>(p, m, a.nc, st);
 }
 
 }  // namespace hn

@@ -11,12 +11,12 @@ struct CoreTmaMaps {
     alignas(64) unsigned char u[128];
     alignas(64) unsigned char h[128];
     const float2 *in, *h_base;
-    int nc, n_in, h_n_in;
+    int nc, n_in, h_n_in, log2p;
     long long in_outer, h_outer, max_outer, h_outer_count;
     bool valid;
 };
 
-// true if `a` is a case the TMA core handles (256-point axis, in place, even number of bins) and the
+// true if `a` is a case the TMA core handles (256- or 1024-point axis, in place, even number of bins) and the
 // driver offers tensor-map encoding
 bool core_tma_supported(const AxisArgs &a);
 // builds the maps for buffers a.in (max_outer outer entries) and a.h (h_outer_count entries)

@@ -48,7 +48,7 @@ struct hyenand_plan {
     long long wh_slices;              // slices the filter workspace holds
     float2 *gtw;
     int gtw_n;
-    // 3-D path: tensor maps of the z core's workspace buffers (valid only if the TMA core applies)
+    // tensor maps of the fused core's workspace buffers (valid only where the TMA core applies)
     CoreTmaMaps tma;
     int *dev_status;                  // device word set by a kernel whose bounded wait gave up
     // long 1-D path
@@ -100,6 +100,7 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
 }
 
 static AxisArgs planes3d_core_args(const hyenand_plan *p, long long n, bool shared, long long s0);
+static AxisArgs generic_core_args(const hyenand_plan *p, long long n, bool shared, long long s0);
 
 extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype)
 {
@@ -199,8 +200,9 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     if (!e && cudaMemset(p->dev_status, 0, sizeof(int)) != cudaSuccess)
         e = fail(HYENAND_ERR_CUDA, "status word: %s", cudaGetErrorString(cudaGetLastError()));
     if (e) { hyenand_destroy_plan(p); return nullptr; }
-    if (p->path == PATH_PLANES3D)      // tensor maps of the z core's buffers; left invalid where the TMA core does not apply
-        core_tma_make(&p->tma, planes3d_core_args(p, spc, false, 0), spc, p->wh_slices);
+    // tensor maps of the fused core's buffers; left invalid where the TMA core does not apply
+    if (p->path == PATH_PLANES3D) core_tma_make(&p->tma, planes3d_core_args(p, spc, false, 0), spc, p->wh_slices);
+    if (p->path == PATH_ND_GENERIC) core_tma_make(&p->tma, generic_core_args(p, spc, false, 0), spc, p->wh_slices);
     return p;
 }
 
@@ -208,6 +210,7 @@ extern "C" int hyenand_plan_device_status(hyenand_plan *p)
 {
     g_err[0] = 0;
     if (!p) { fail(HYENAND_ERR_INVALID_ARG, "plan is NULL"); return -1; }
+    if (!p->dev_status) return 0;             // plans whose kernels make no such waits have no status word
     int v = 0;
     if (cudaMemcpy(&v, p->dev_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
         fail(HYENAND_ERR_CUDA, "reading the status word failed: %s", cudaGetErrorString(cudaGetLastError()));
@@ -253,6 +256,29 @@ static int filter_spectrum_generic(hyenand_plan *p, const char *h, long long n_s
     return 0;
 }
 
+// arguments of the fused core (last transformed axis) of the generic path for n slices starting at slice s0
+static AxisArgs generic_core_args(const hyenand_plan *p, long long n, bool shared, long long s0)
+{
+    const bool three = p->P[0] > 1;
+    AxisArgs a{};
+    const int ax = three ? 0 : 1;                       // core axis
+    const long long inner = three ? (long long)p->P[1] * p->XP : p->XP;
+    a.in = three ? p->ws_b : p->ws_a; a.out = (float2 *)a.in;
+    a.n_outer = n;
+    a.in_outer = a.out_outer = (long long)p->L[ax] * inner;
+    a.nc = (int)inner; a.n_in = p->L[ax]; a.n_out = p->L[ax]; a.shift = 0;
+    a.log2p = p->log2p[ax]; a.prune_in = 1;
+    a.h = three ? p->wh_b : p->wh_a;
+    a.h_outer = (long long)p->K[ax] * inner;
+    a.h_n_in = p->K[ax];
+    a.h_shift = p->causal ? 0 : p->L[ax] - 1;
+    a.h_mod = shared ? p->C : 0;
+    a.h_off = shared ? s0 % p->C : 0;
+    a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
+    a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+    return a;
+}
+
 static int forward_generic(hyenand_plan *p, const char *q, const char *k, const char *v, const char *h,
                            bool shared, char *y, cudaStream_t st, int *launches)
 {
@@ -288,24 +314,12 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             *launches += c;
         }
         {
-            AxisArgs a{};
-            const int ax = three ? 0 : 1;                       // core axis
-            const long long inner = three ? (long long)p->P[1] * p->XP : p->XP;
-            a.in = three ? p->ws_b : p->ws_a; a.out = (float2 *)a.in;
-            a.n_outer = n;
-            a.in_outer = a.out_outer = (long long)p->L[ax] * inner;
-            a.nc = (int)inner; a.n_in = p->L[ax]; a.n_out = p->L[ax]; a.shift = 0;
-            a.log2p = p->log2p[ax]; a.prune_in = 1;
-            a.h = three ? p->wh_b : p->wh_a;
-            a.h_outer = (long long)p->K[ax] * inner;
-            a.h_n_in = p->K[ax];
-            a.h_shift = p->causal ? 0 : p->L[ax] - 1;
-            a.h_mod = shared ? p->C : 0;
-            a.h_off = shared ? s0 % p->C : 0;
-            a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
-            a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+            const AxisArgs a = generic_core_args(p, n, shared, s0);
             p->prof.begin(KID_CORE, st);
-            c = (core_w_supported(a.log2p) && !getenv("HYENAND_GENERIC_CORE")) ? launch_core_w(a, st) : launch_axis(a, AXIS_CORE, st);
+            c = -1;
+            if (p->tma.valid && !getenv("HYENAND_NO_TMA")) c = launch_core_tma(a, p->tma, p->dev_status, st);
+            if (c < 0)
+                c = (core_w_supported(a.log2p) && !getenv("HYENAND_GENERIC_CORE")) ? launch_core_w(a, st) : launch_axis(a, AXIS_CORE, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;

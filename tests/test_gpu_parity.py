@@ -21,6 +21,7 @@ def run_gpu(w, q, k, v, h):
         y = torch.full_like(dq, float("nan"))
         plan.forward(dq, dk, dv, dh, y)
         torch.cuda.synchronize()
+        assert hn.hyenand_plan_device_status(plan.handle) == 0, "a kernel gave up a bounded wait"
         return y.cpu(), hn.hyenand_plan_path(plan.handle)
     finally:
         plan.close()
@@ -51,7 +52,7 @@ def check(w, q, k, v, h, full_direct=False):
 
 
 SHAPES_1D = [(1,), (2,), (3,), (5,), (17,), (64,), (200,), (400,), (1000,), (4096,)]
-SHAPES_ND = [(3, 5), (15, 14), (32, 32), (33, 70), (64, 64), (1, 9), (9, 1), (150, 200), (300, 129),
+SHAPES_ND = [(3, 5), (15, 14), (32, 32), (33, 70), (64, 64), (1, 9), (9, 1), (150, 200), (300, 129), (100, 40), (128, 512),
              (5, 3, 2), (7, 1, 4), (16, 16, 16), (20, 9, 12), (1, 1, 6)]
 
 
