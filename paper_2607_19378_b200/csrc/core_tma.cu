@@ -21,11 +21,11 @@
 #include "common.cuh"
 #include "plane_util.cuh"
 #include "core_tma.cuh"
+#include "tma_util.cuh"
 
 namespace hn {
 
 constexpr int kTmaThreads = 256;
-constexpr int kWaitLimit = 1 << 22;                  // polls of a barrier before giving up
 
 // Geometry of a tile for LOG2P-point lines: one line per group of TPL lanes, so TX = 256 / TPL bins
 // per tile and TX * 8 bytes per tile row (128 for 256-point lines, 64 for 1024-point lines: the
@@ -50,45 +50,6 @@ template <int LOG2P> struct TmaGeo {
     static constexpr size_t BARS = TW + sizeof(float2) * N;
     static constexpr size_t TOTAL = BARS + 2 * sizeof(uint64_t) + 1024;    // + room to align the start
 };
-
-__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t *b, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(b)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *b, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *b, unsigned parity)
-{
-    unsigned ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-                 : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// bounded wait; false if the phase did not complete
-__device__ __forceinline__ bool mbar_wait(uint64_t *b, unsigned parity)
-{
-    for (int i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(b, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z)
-{
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z) : "memory");
-}
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, const void *src, int x, int y, int z)
-{
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];\n"
-                 ::"l"(map), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z) : "memory");
-}
-__device__ __forceinline__ void tma_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
-__device__ __forceinline__ void tma_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
-__device__ __forceinline__ void tma_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
-__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
 
 struct CoreTmaParams {
     long long n_outer;
@@ -235,42 +196,15 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
 
 // ---- host side -------------------------------------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-        else
-            cudaGetLastError();
-    }
-    return fn;
-}
-
 // [outer][rows][nc] complex fp32, seen as fp32 with 2*nc entries per row; box = one tile row of 2*TX floats
 // by up to 256 rows, swizzled over the row's 64 or 128 bytes
 static bool make_map(CUtensorMap *map, const float2 *base, long long outer, int rows, int nc, long long outer_stride_elems,
                      int tx, int box_rows)
 {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)2 * nc, (cuuint64_t)rows, (cuuint64_t)outer};
-    const cuuint64_t strides[2] = {(cuuint64_t)nc * 8, (cuuint64_t)outer_stride_elems * 8};
-    const cuuint32_t box[3] = {(cuuint32_t)tx * 2, (cuuint32_t)box_rows, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    if ((strides[0] % 16) || (strides[1] % 16) || ((uintptr_t)base % 16)) return false;
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float2 *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, tx * 8 == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const unsigned long long dims[3] = {2ull * nc, (unsigned long long)rows, (unsigned long long)outer};
+    const unsigned long long strides[2] = {(unsigned long long)nc * 8, (unsigned long long)outer_stride_elems * 8};
+    const unsigned box[3] = {(unsigned)tx * 2, (unsigned)box_rows, 1};
+    return tma_encode_3d(map, base, /*bf16=*/false, dims, strides, box, tx * 8);
 }
 
 static bool tma_log2p_ok(int log2p) { return log2p == 8 || log2p == 10; }
@@ -281,7 +215,7 @@ bool core_tma_supported(const AxisArgs &a)
     const int n = 1 << a.log2p;
     return a.in == a.out && a.in_outer == a.out_outer && a.n_in == a.n_out && a.n_in >= 1 && a.n_in <= n / 2 &&
            a.h_n_in >= 1 && a.h_n_in <= n && a.shift == 0 && a.h_shift >= 0 && a.h_shift < n && (a.nc % 2) == 0 &&
-           a.n_outer < (1ll << 31) && encode_fn() != nullptr;
+           a.n_outer < (1ll << 31) && tma_available();
 }
 
 bool core_tma_make(CoreTmaMaps *m, const AxisArgs &a, long long max_outer, long long h_outer_count)

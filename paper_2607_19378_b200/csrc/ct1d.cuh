@@ -17,6 +17,7 @@ struct Ct1dPlan {
     float2 *tw1, *tw2;        // twiddle tables for P1 and P2
     float2 *twp_coarse, *twp_fine;   // W_P^j = coarse[j >> lo] * fine[j & (2^lo - 1)]
     int lo;
+    int *status;              // device word set when a bounded wait on a tensor copy gives up (owned by the plan)
     long long slices_per_chunk, wh_slices;
 };
 

@@ -12,7 +12,10 @@
 //   cols_inv_w   rebuild the mirrored half, inverse along f1 keeping t < P/2, crop, gate
 //                with q, coalesced store.
 #include <type_traits>
+#include <cstring>
+#include <cstdlib>
 #include "common.cuh"
+#include "tma_util.cuh"
 #include "ct1d.cuh"
 #include "plane_util.cuh"
 
@@ -50,13 +53,18 @@ struct ColsFwdWArgs {
     long long slices;
     long long in_slice;       // elements per slice of the input (multiple of 16 bytes)
     int len;                  // valid elements (<= P/2)
+    int *status;              // device word set when a bounded wait on a tensor copy gives up (may be NULL)
     int log2p2;
     const float2 *tw1;        // P1-point table
     TwoLevelW twp;
 };
 
-template <typename T, int LOG2P1, bool HAS_B>
-__global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_fwd_w_kernel(ColsFwdWArgs p)
+// TMA = true: the tile (all rows t1 of TX column pairs, for k and for v) arrives as tensor copies into
+// row-major swizzled buffers, issued by one thread as soon as the previous tile has been read; false: 8-byte
+// asynchronous copies per thread into padded rows.
+template <typename T, int LOG2P1, bool HAS_B, bool TMA>
+__global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4))
+ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b)
 {
     using F = WF<LOG2P1, false>;
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = F::TPL;
@@ -72,6 +80,13 @@ __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_fwd
     constexpr int PG = 8 / PAIRB;                          // column pairs per 8-byte copy
     constexpr int RS = TX * PAIRB + 8;                     // bytes per staged row
     unsigned char *raw = reinterpret_cast<unsigned char *>(twt + P1);
+    // tensor copies: rows of TX*PAIRB bytes (64 or 128: the swizzle span), 1024-byte aligned tile buffers
+    constexpr unsigned TROW = TX * PAIRB;
+    constexpr int TBOXR = HP1 < 256 ? HP1 : 256, TNB = HP1 / TBOXR;
+    constexpr unsigned TBYTES = HP1 * TROW;
+    static_assert(!TMA || TROW == 64 || TROW == 128, "tile rows match a swizzle span");
+    if constexpr (TMA) raw += (1024u - (smem_u32(raw) & 1023u)) & 1023u;
+    uint64_t *bar = reinterpret_cast<uint64_t *>(raw + 2 * TBYTES);
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     PassTw<LOG2P1, false>::build(twt, p.tw1, P1, tid, kCtThreads);
@@ -80,11 +95,34 @@ __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_fwd
     const int tpc = (P2 / 2) / TX;                         // tiles per slice (P2/2 is a multiple of TX)
     const long long tiles = p.slices * tpc;
     const unsigned char *ab = (const unsigned char *)p.a, *bb = (const unsigned char *)p.b;
-    for (long long t = blockIdx.x; t < tiles; t += gridDim.x) {
+    auto issue = [&](long long t) {                        // one thread
+        const long long s = t / tpc;
+        const int x = 2 * (int)(t % tpc) * TX;             // first column of the tile
+        mbar_expect_tx(bar, (HAS_B ? 2 : 1) * TBYTES);
+#pragma unroll
+        for (int b = 0; b < TNB; ++b) {
+            tma_load_3d(raw + b * TBOXR * TROW, &map_a, bar, x, b * TBOXR, (int)s);
+            if (HAS_B) tma_load_3d(raw + TBYTES + b * TBOXR * TROW, &map_b, bar, x, b * TBOXR, (int)s);
+        }
+    };
+    if constexpr (TMA) {
+        if (tid == 0) {
+            mbar_init(bar, 1);
+            fence_mbar_init();
+        }
+        __syncthreads();
+        if (tid == 0 && (long long)blockIdx.x < tiles) issue(blockIdx.x);
+    }
+    unsigned phase = 0;
+    int failed = 0;
+    for (long long t = blockIdx.x; t < tiles; t += gridDim.x, phase ^= 1u) {
         const long long s = t / tpc;
         const int c0 = (int)(t % tpc) * TX;
         const long long base = s * p.in_slice;
         __syncthreads();                                   // previous tile done with raw and lines
+        if constexpr (TMA) {
+            if (!mbar_wait(bar, phase)) failed = 1;
+        } else {
         for (int idx = tid; idx < HP1 * (TX / PG); idx += kCtThreads) {
             const int t1 = idx / (TX / PG), xg = idx % (TX / PG);
             const long long e0 = (long long)t1 * P2 + 2 * (c0 + PG * xg);
@@ -103,15 +141,21 @@ __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_fwd
         }
         cp_async_wait_all();
         __syncthreads();
+        }
         for (int x = gid; x < TX; x += NGRP) {
         float2 *line = lines + x * LS;
-        const unsigned char *ra = raw + (size_t)x * PAIRB;
-        const unsigned char *rb = ra + (size_t)HP1 * RS;
+        // TMA: the 16-byte chunk of pair x in row idx is XORed with a function of idx that the engine's strides
+        // (multiples of 8 rows) leave alone, so it depends on the lane only
+        constexpr unsigned RSTR = TMA ? TROW : (unsigned)RS;
+        const unsigned sw = TROW == 128 ? ((unsigned)l & 7u) : (((unsigned)l >> 1) & 3u);
+        const unsigned xo = TMA ? ((((unsigned)x * PAIRB >> 4) ^ sw) << 4) + (((unsigned)x * PAIRB) & 15u) : (unsigned)x * PAIRB;
+        const unsigned char *ra = raw + xo;
+        const unsigned char *rb = ra + (TMA ? (size_t)TBYTES : (size_t)HP1 * RS);
         F::template run_to_line<PRUNE_IN>(l, m, tw, line, [&](int, int, int idx) {
-            float a0 = staged<T>(ra + (size_t)idx * RS, 0, 0), a1 = staged<T>(ra + (size_t)idx * RS, 0, 1);
+            float a0 = staged<T>(ra + (size_t)idx * RSTR, 0, 0), a1 = staged<T>(ra + (size_t)idx * RSTR, 0, 1);
             if (HAS_B) {
-                a0 *= staged<T>(rb + (size_t)idx * RS, 0, 0);
-                a1 *= staged<T>(rb + (size_t)idx * RS, 0, 1);
+                a0 *= staged<T>(rb + (size_t)idx * RSTR, 0, 0);
+                a1 *= staged<T>(rb + (size_t)idx * RSTR, 0, 1);
             }
             return make_float2(a0, a1);
         });
@@ -141,12 +185,24 @@ __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_fwd
             }
         }
         }
-        __syncthreads();
+        if constexpr (TMA) {
+            if (__syncthreads_or(failed)) break;           // the tile buffers are free again
+            if (tid == 0 && t + gridDim.x < tiles) issue(t + gridDim.x);
+        } else {
+            __syncthreads();
+        }
         float2 *dst = p.out + s * (long long)F1 * P2 + 2 * c0;
         for (int idx = tid; idx < F1 * TX; idx += kCtThreads) {
             const int f1 = idx / TX, x = idx % TX;
             *reinterpret_cast<float4 *>(dst + (long long)f1 * P2 + 2 * x) =
                 *reinterpret_cast<const float4 *>(lines + x * LS + 2 * f1);
+        }
+    }
+    if constexpr (TMA) {
+        if (failed) {
+            // a wait gave up: say so, then give the copy a bounded time to land before the buffers go away
+            if (p.status) atomicExch(p.status, 7);
+            mbar_wait(bar, phase);
         }
     }
 }
@@ -382,6 +438,15 @@ bool ct1d_w_supported(int log2p1, int log2p2, int L, int K, int causal, int dtyp
     return true;
 }
 
+template <typename T, int LOG2P1, bool HAS_B, bool TMA>
+static void launch_cols_fwd_w_tt(const ColsFwdWArgs &a, const CUtensorMap &ma, const CUtensorMap &mb, int grid, size_t sm, cudaStream_t st)
+{
+    static DevOnce attr;
+    if (attr.first())
+        cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, HAS_B, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    ct_cols_fwd_w_kernel<T, LOG2P1, HAS_B, TMA><<<grid, kCtThreads, sm, st>>>(a, ma, mb);
+}
+
 template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWArgs &a, cudaStream_t st)
 {
     using F = WF<LOG2P1, false>;
@@ -392,15 +457,31 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
     const long long res = (LOG2P1 >= 9 ? 2ll : 4ll) * ctw_sms();   // resident CTAs
     const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
-    if (a.b) {
-        static DevOnce attr;
-        if (attr.first()) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }
-        ct_cols_fwd_w_kernel<T, LOG2P1, true><<<grid, kCtThreads, sm, st>>>(a);
-    } else {
-        static DevOnce attr;
-        if (attr.first()) { cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }
-        ct_cols_fwd_w_kernel<T, LOG2P1, false><<<grid, kCtThreads, sm, st>>>(a);
+    // Tensor copies need the slice to be a whole number of rows of P2 elements (then [slice][row][P2] is an
+    // exact view of the input and rows past the data read as zeros) and tile rows of 64 or 128 bytes.
+    alignas(64) CUtensorMap ma, mb;
+    memset(&ma, 0, sizeof(ma));
+    memset(&mb, 0, sizeof(mb));
+    constexpr unsigned TROW = TX * 2 * sizeof(T);
+    bool tma = (TROW == 64 || TROW == 128) && a.len % P2 == 0 && a.slices < (1ll << 31) && tma_available() &&
+               !getenv("HYENAND_NO_TMA");
+    if (tma) {
+        constexpr int HP1 = P1 / 2;
+        const unsigned long long dims[3] = {(unsigned long long)P2, (unsigned long long)(a.len / P2), (unsigned long long)a.slices};
+        const unsigned long long strides[2] = {(unsigned long long)P2 * sizeof(T), (unsigned long long)a.in_slice * sizeof(T)};
+        const unsigned box[3] = {2 * TX, (unsigned)(HP1 < 256 ? HP1 : 256), 1};
+        tma = tma_encode_3d(&ma, a.a, sizeof(T) == 2, dims, strides, box, (int)TROW);
+        if (tma && a.b) tma = tma_encode_3d(&mb, a.b, sizeof(T) == 2, dims, strides, box, (int)TROW);
     }
+    if constexpr (TROW == 64 || TROW == 128) {
+        if (tma) {
+            if (a.b) launch_cols_fwd_w_tt<T, LOG2P1, true, true>(a, ma, mb, grid, sm, st);
+            else launch_cols_fwd_w_tt<T, LOG2P1, false, true>(a, ma, mb, grid, sm, st);
+            return 1;
+        }
+    }
+    if (a.b) launch_cols_fwd_w_tt<T, LOG2P1, true, false>(a, ma, mb, grid, sm, st);
+    else launch_cols_fwd_w_tt<T, LOG2P1, false, false>(a, ma, mb, grid, sm, st);
     return 1;
 }
 
@@ -460,7 +541,7 @@ int ct1d_w_filter(Ct1dPlan *c, const void *h, long long n, bool staged_ok, cudaS
     const TwoLevelW twp{c->twp_coarse, c->twp_fine, c->lo};
     if (staged_ok) {
         ColsFwdWArgs a{};
-        a.a = h; a.b = nullptr; a.out = c->wh; a.slices = n; a.in_slice = c->K; a.len = c->K;
+        a.a = h; a.b = nullptr; a.out = c->wh; a.slices = n; a.in_slice = c->K; a.len = c->K; a.status = c->status;
         a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.twp = twp;
         prof->begin(KID_CT_COLS_H, st);
         int r = 0;
@@ -490,7 +571,7 @@ int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long l
 {
     const TwoLevelW twp{c->twp_coarse, c->twp_fine, c->lo};
     ColsFwdWArgs a{};
-    a.a = k; a.b = v; a.out = c->wu; a.slices = n; a.in_slice = c->L; a.len = c->L;
+    a.a = k; a.b = v; a.out = c->wu; a.slices = n; a.in_slice = c->L; a.len = c->L; a.status = c->status;
     a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.twp = twp;
     prof->begin(KID_CT_COLS_U, st);
     int r = 0;

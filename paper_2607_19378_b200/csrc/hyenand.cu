@@ -145,6 +145,11 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
             ct1d_free(&p->ct); delete p; return nullptr;
         }
         p->ws_bytes += bytes;
+        if (dev_alloc(p, (void **)&p->dev_status, sizeof(int)) || cudaMemset(p->dev_status, 0, sizeof(int)) != cudaSuccess) {
+            hyenand_destroy_plan(p);
+            return nullptr;
+        }
+        p->ct.status = p->dev_status;
         return p;
     }
     for (int a = 0; a < 3; ++a)
