@@ -164,15 +164,26 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
         {
             // W_P^(t2*f1) with f1 = l + i*TPL is the product of a per-lane factor W_P^(t2*l) (one
             // gathered lookup) and a per-line factor W_P^(t2*TPL*i) (the same address in all lanes)
+            // The per-line factor is looked up every fourth step and advanced by W_P^(t2*TPL) in between
+            // (at most three products after a table value).
             const float2 cl0 = twp_w(p.twp, t2 * (unsigned)l), cl1 = twp_w(p.twp, (t2 + 1u) * (unsigned)l);
+            const float2 st0 = twp_w(p.twp, t2 * (unsigned)TPL), st1 = twp_w(p.twp, (t2 + 1u) * (unsigned)TPL);
             float2 A0[(F1 + TPL - 1) / TPL], A1[(F1 + TPL - 1) / TPL];
+            float2 w0 = cl0, w1 = cl1;
 #pragma unroll
             for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
                 const int f1 = l + i * TPL;
+                if (i > 0) {
+                    if (i % 4 == 0) {
+                        w0 = cmul(cl0, twp_w(p.twp, t2 * (unsigned)(i * TPL)));
+                        w1 = cmul(cl1, twp_w(p.twp, (t2 + 1u) * (unsigned)(i * TPL)));
+                    } else {
+                        w0 = cmul(w0, st0);
+                        w1 = cmul(w1, st1);
+                    }
+                }
                 if (f1 < F1) {
                     const float2 z1 = line[F::ph(f1)], z2 = line[F::ph((P1 - f1) & (P1 - 1))];
-                    const float2 w0 = cmul(cl0, twp_w(p.twp, t2 * (unsigned)(i * TPL)));
-                    const float2 w1 = cmul(cl1, twp_w(p.twp, (t2 + 1u) * (unsigned)(i * TPL)));
                     A0[i] = cmul(make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y)), w0);
                     A1[i] = cmul(make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x)), w1);
                 }
@@ -310,11 +321,17 @@ __global__ void __launch_bounds__(256, 2) ct_core_w_kernel(CoreWArgs p)
         FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, line);
         // undo the inter-pass twiddle W_P^(t2*f1), t2 = l + TPL*q: per-lane factor W_P^(f1*l) times a
         // per-row factor W_P^(f1*TPL*q) whose address is the same in all lanes
+        // (the per-row factor is looked up every fourth leg and advanced by one leg's step in between)
         const float2 cl = twp_w(p.twp, (unsigned)f1 * (unsigned)l);
+        using PE = typename FI::LastPass;
+        const float2 stp = twp_w(p.twp, (unsigned)f1 * (unsigned)(P2 / PE::R));
+        float2 w = cl;
         FI::template pass<NP - 1, PRUNE_NONE>(l, twi,
             [&](int, int, int idx) { return line[FI::ph(idx)]; },
-            [&](int, int, int idx, float2 v) {
-                const float2 w = cmul(cl, twp_w(p.twp, (unsigned)f1 * (unsigned)(idx - l)));
+            [&](int, int r, int idx, float2 v) {
+                // legs of one item come in order r = 0, 1, ...: positions idx = l + i*TPL + r*(P2/R)
+                if (r % 4 == 0) w = cmul(cl, twp_w(p.twp, (unsigned)f1 * (unsigned)(idx - l)));
+                else w = cmul(w, stp);
                 row[idx] = cmulc(v, w);
             });
         __syncwarp(m);
