@@ -384,12 +384,17 @@ __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_inv
         __syncthreads();
         for (int x = gid; x < TX; x += NGRP) {
             float2 *line = lines + x * LS;
-            FI::template run_to_line<PRUNE_OUT, true>(l, m, tw, line, [&](int, int, int idx) {
-                const bool mirror = idx > HP1;
-                const int f1 = mirror ? P1 - idx : idx;
-                float4 ab = *reinterpret_cast<const float4 *>(line + 2 * f1);
-                if (mirror) { ab.y = -ab.y; ab.w = -ab.w; }
-                return make_float2(ab.x - ab.w, ab.y + ab.z);
+            // legs below half the first-pass radix read bins <= P1/2 directly, the others the mirrored bin
+            // conjugated: known per leg at compile time, except where a leg starts at bin P1/2 itself
+            constexpr int RH = FI::template Pass<0>::R / 2;
+            FI::template run_to_line<PRUNE_OUT, true>(l, m, tw, line, [&](int, int r, int idx) {
+                if (r < RH) {
+                    const float4 ab = *reinterpret_cast<const float4 *>(line + 2 * idx);
+                    return make_float2(ab.x - ab.w, ab.y + ab.z);
+                }
+                const float4 ab = *reinterpret_cast<const float4 *>(line + 2 * (P1 - idx));
+                const float sg = (r == RH && idx == HP1) ? 1.f : -1.f;
+                return make_float2(fmaf(-sg, ab.w, ab.x), fmaf(sg, ab.y, ab.z));
             });
         }
         __syncthreads();

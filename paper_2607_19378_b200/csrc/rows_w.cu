@@ -122,13 +122,20 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
         }
         cp_async_wait_all();
         __syncwarp(m);
-        FI::template run_to_line<PRUNE_OUT, true>(l, m, tw, line, [&](int, int, int idx) {
-            const bool mirror = idx > HP;
-            const int kx = mirror ? P - idx : idx;
-            float2 A = line[kx];
-            float2 B = has1 ? line[RS + kx] : make_float2(0.f, 0.f);
-            if (mirror) { A.y = -A.y; B.y = -B.y; }
-            return make_float2(A.x - B.y, A.y + B.x);
+        // Legs below half the first-pass radix read bins <= P/2 directly; the others read the mirrored bin
+        // conjugated.  Which case applies is known per leg at compile time, except for the leg that starts at
+        // P/2 (its first position is the unmirrored bin P/2 itself).
+        if (!has1) for (int c = l; c <= HP; c += TPL) line[RS + c] = make_float2(0.f, 0.f);
+        __syncwarp(m);
+        constexpr int RH = FI::template Pass<0>::R / 2;
+        FI::template run_to_line<PRUNE_OUT, true>(l, m, tw, line, [&](int, int r, int idx) {
+            if (r < RH) {
+                const float2 A = line[idx], B = line[RS + idx];
+                return make_float2(A.x - B.y, A.y + B.x);
+            }
+            const float2 A = line[P - idx], B = line[RS + P - idx];
+            const float sg = (r == RH && idx == HP) ? 1.f : -1.f;
+            return make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
         });
         for (int n = l; n < p.len; n += TPL) {
             const float2 z = line[FI::ph(n)];
