@@ -108,7 +108,7 @@ __device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, in
 // tables in shared memory.
 template <int LOG2P, bool INV> struct PlaneTw {
     using F = WF<LOG2P, INV>;
-    static constexpr bool HOIST = F::NP == 2 && WPlan<LOG2P>::R[0] == WPlan<LOG2P>::R[1];
+    static constexpr bool HOIST = F::NP == 2 && (WPlan<LOG2P>::R[0] == WPlan<LOG2P>::R[1] || (LOG2P == 7 && !INV));
     static constexpr int TABLE = HOIST ? 0 : PassTw<LOG2P, INV>::TOTAL;   // shared-memory entries needed
     typename F::template Hoist<F::NP - 1> hw;
     PassTw<LOG2P, INV> pt;
