@@ -27,6 +27,9 @@ constexpr int kCtThreads = 256;
 // 16-byte accesses of neighbouring lines (tile loads and stores run across lines) hit different banks
 __host__ __device__ constexpr int ct_ls(int n) { return (n + 15) / 16 * 16 + 2; }
 __host__ __device__ constexpr int ct_tx(int tpl) { return kCtThreads / tpl > 8 ? kCtThreads / tpl : 8; }
+// the inverse column kernel runs as CTAs of 4 warps: more, smaller tiles in flight per SM
+constexpr int kCtInvThreads = 128;
+__host__ __device__ constexpr int ct_inv_tx(int tpl) { return kCtInvThreads / tpl > 8 ? kCtInvThreads / tpl : 8; }
 
 template <int BYTES> __device__ __forceinline__ void cp_async_n(void *smem_dst, const void *gmem_src)
 {
@@ -351,19 +354,19 @@ struct ColsInvWArgs {
 };
 
 template <typename T, int LOG2P1>
-__global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_inv_w_kernel(ColsInvWArgs p)
+__global__ void __launch_bounds__(kCtInvThreads, (LOG2P1 >= 9 ? 4 : 8)) ct_cols_inv_w_kernel(ColsInvWArgs p)
 {
     using FI = WF<LOG2P1, true>;
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = FI::TPL;
-    constexpr int TX = ct_tx(TPL);
-    constexpr int NGRP = kCtThreads / TPL;
+    constexpr int TX = ct_inv_tx(TPL);
+    constexpr int NGRP = kCtInvThreads / TPL;
     constexpr int LS = ct_ls(phys_max(P1) + 2);
     extern __shared__ float2 smem[];
     float2 *lines = smem;
     float2 *twt = lines + TX * LS;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = FI::group_mask(tid);
-    PassTw<LOG2P1, true>::build(twt, p.tw1, P1, tid, kCtThreads);
+    PassTw<LOG2P1, true>::build(twt, p.tw1, P1, tid, kCtInvThreads);
     const PassTw<LOG2P1, true> tw{twt};
     const int P2 = 1 << p.log2p2;
     const int tpc = (P2 / 2) / TX;
@@ -376,7 +379,7 @@ __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_inv
         const float2 *src = p.in + s * (long long)F1 * P2 + 2 * c0;
         __syncthreads();
         // both bins of a column pair land side by side in slot f1 of that pair's line
-        for (int idx = tid; idx < F1 * TX; idx += kCtThreads) {
+        for (int idx = tid; idx < F1 * TX; idx += kCtInvThreads) {
             const int f1 = idx / TX, x = idx % TX;
             cp_async16(lines + x * LS + 2 * f1, src + (long long)f1 * P2 + 2 * x);
         }
@@ -401,13 +404,13 @@ __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4)) ct_cols_inv
         // line x now holds, at position t1 < P1/2, the two real outputs of columns 2x, 2x+1
         const long long base = s * (long long)p.len + 2 * c0;
         // gate values first (all requests in flight together), then products and stores
-        constexpr int NE = HP1 * TX / kCtThreads;
-        static_assert(HP1 * TX % kCtThreads == 0, "whole epilogue rounds");
+        constexpr int NE = HP1 * TX / kCtInvThreads;
+        static_assert(HP1 * TX % kCtInvThreads == 0, "whole epilogue rounds");
         // a half warp takes 8 pairs of two neighbouring rows: line stride and skew then spread its
         // 16 reads over all banks, and each row still receives whole 32-byte sectors
         const int x = (tid & 7) + 8 * ((tid >> 4) % (TX / 8));
         const int tb = ((tid >> 3) & 1) + 2 * ((tid >> 4) / (TX / 8));
-        constexpr int TSTEP = kCtThreads / TX;
+        constexpr int TSTEP = kCtInvThreads / TX;
         const long long ox = base + 2 * x;
         using Q2 = typename std::conditional<sizeof(T) == 4, float2, __nv_bfloat162>::type;
         Q2 qv[NE];
@@ -510,16 +513,16 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
 template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWArgs &a, cudaStream_t st)
 {
     using F = WF<LOG2P1, true>;
-    constexpr int P1 = 1 << LOG2P1, TX = ct_tx(F::TPL), LS = ct_ls(phys_max(P1) + 2);
+    constexpr int P1 = 1 << LOG2P1, TX = ct_inv_tx(F::TPL), LS = ct_ls(phys_max(P1) + 2);
     const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1);
     const int P2 = 1 << a.log2p2;
     const long long tiles = a.slices * ((P2 / 2) / TX);
-    const long long res = (LOG2P1 >= 9 ? 2ll : 4ll) * ctw_sms();   // resident CTAs
+    const long long res = (LOG2P1 >= 9 ? 4ll : 8ll) * ctw_sms();   // resident CTAs
     const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
     static DevOnce attr;
     if (attr.first()) { cudaFuncSetAttribute(ct_cols_inv_w_kernel<T, LOG2P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }
-    ct_cols_inv_w_kernel<T, LOG2P1><<<grid, kCtThreads, sm, st>>>(a);
+    ct_cols_inv_w_kernel<T, LOG2P1><<<grid, kCtInvThreads, sm, st>>>(a);
     return 1;
 }
 
