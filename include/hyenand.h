@@ -114,6 +114,12 @@ int hyenand_last_error_code(void);
  * no counterpart; it exists so that a failed copy is observable from the host. */
 int hyenand_plan_device_status(hyenand_plan *plan);
 
+/* Self-test of the mechanism behind hyenand_plan_device_status: launches one small CTA that waits, for at
+ * most `polls` polls (clamped to [1, 65536]), on a barrier that nothing ever completes.  The wait must run out
+ * and the kernel must report it: returns 9 (the code that kernel records), 0 if the wait wrongly succeeded,
+ * -1 on a CUDA error.  Blocking; allocates and frees 4 bytes of device memory.  No counterpart in the paper. */
+int hyenand_selftest_bounded_wait(int polls);
+
 /* Reporting helpers (host-only, no device work). */
 size_t hyenand_plan_workspace_bytes(const hyenand_plan *plan);        /* device bytes owned by the plan */
 int hyenand_plan_fft_dims(const hyenand_plan *plan, int *out_P);      /* writes ndim padded sizes P_n */

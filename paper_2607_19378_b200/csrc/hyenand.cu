@@ -13,6 +13,7 @@
 #include "ct1d.cuh"
 #include "planes.cuh"
 #include "core_tma.cuh"
+#include "tma_util.cuh"
 #include "fused2d.cuh"
 
 using namespace hn;
@@ -221,6 +222,14 @@ extern "C" int hyenand_plan_device_status(hyenand_plan *p)
         fail(HYENAND_ERR_CUDA, "reading the status word failed: %s", cudaGetErrorString(cudaGetLastError()));
         return -1;
     }
+    return v;
+}
+
+extern "C" int hyenand_selftest_bounded_wait(int polls)
+{
+    g_err[0] = 0;
+    const int v = tma_selftest_bounded_wait(polls);
+    if (v < 0) fail(HYENAND_ERR_CUDA, "bounded-wait self-test could not run: %s", cudaGetErrorString(cudaGetLastError()));
     return v;
 }
 

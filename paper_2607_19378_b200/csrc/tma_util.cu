@@ -42,4 +42,33 @@ bool tma_encode_3d(CUtensorMap *map, const void *base, bool bf16, const unsigned
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+__global__ void bounded_wait_selftest_kernel(int polls, int *status)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    // nobody arrives on `bar`: the wait must run out and report it
+    if (!mbar_wait(&bar, 0, polls)) {
+        if (threadIdx.x == 0) atomicExch(status, 9);
+    }
+}
+
+int tma_selftest_bounded_wait(int polls)
+{
+    int *d = nullptr, v = -1;
+    if (polls < 1) polls = 1;
+    if (polls > (1 << 16)) polls = 1 << 16;
+    if (cudaMalloc(&d, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return -1; }
+    bool ok = cudaMemset(d, 0, sizeof(int)) == cudaSuccess;
+    if (ok) {
+        bounded_wait_selftest_kernel<<<1, 64>>>(polls, d);
+        ok = cudaGetLastError() == cudaSuccess && cudaMemcpy(&v, d, sizeof(int), cudaMemcpyDeviceToHost) == cudaSuccess;
+    }
+    cudaFree(d);
+    return ok ? v : -1;
+}
+
 }  // namespace hn

@@ -25,10 +25,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *b, unsigned parity)
                  : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
     return ok != 0;
 }
-// bounded wait; false if the phase did not complete
-__device__ __forceinline__ bool mbar_wait(uint64_t *b, unsigned parity)
+// bounded wait; false if the phase did not complete within `limit` polls
+__device__ __forceinline__ bool mbar_wait(uint64_t *b, unsigned parity, int limit = kWaitLimit)
 {
-    for (int i = 0; i < kWaitLimit; ++i)
+    for (int i = 0; i < limit; ++i)
         if (mbar_try_wait(b, parity)) return true;
     return false;
 }
@@ -52,6 +52,10 @@ __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier
 // ---- host -----------------------------------------------------------------------------------------------------
 // true if the driver offers tensor-map encoding (looked up once through the runtime)
 bool tma_available();
+// Self-test of the bounded wait: one CTA waits, for at most `polls` polls, on a barrier that nothing ever
+// completes, and must come back with code 9 in the returned status word (0 would mean the wait "succeeded",
+// -1 a CUDA error).  Blocking; allocates and frees one device word.
+int tma_selftest_bounded_wait(int polls);
 // Encodes a 3-D tiled map of fp32 (bf16 = false) or bf16 elements: dims and box in elements (innermost first),
 // strides in bytes for dimensions 1 and 2, swizzle = bytes of one box row (64 or 128).  False if the arguments
 // break an alignment rule or the driver refuses.

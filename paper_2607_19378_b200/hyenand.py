@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         L.hyenand_destroy_plan.argtypes = [vp]
         L.hyenand_destroy_plan.restype = None
         L.hyenand_last_error.restype = ctypes.c_char_p
+        L.hyenand_selftest_bounded_wait.argtypes = [ctypes.c_int]
+        L.hyenand_selftest_bounded_wait.restype = ctypes.c_int
         L.hyenand_plan_device_status.argtypes = [vp]
         L.hyenand_plan_device_status.restype = ctypes.c_int
         L.hyenand_plan_workspace_bytes.argtypes = [vp]
@@ -116,6 +118,11 @@ def hyenand_forward_ex(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stre
 def hyenand_forward_host(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stream=None) -> None:
     _check(lib().hyenand_forward_host(plan, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
                                       int(h_batch_stride_elems), y.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_selftest_bounded_wait(polls: int = 1000) -> int:
+    """9 if a wait on a barrier that nothing completes ran out and was reported, as it must."""
+    return int(lib().hyenand_selftest_bounded_wait(int(polls)))
 
 
 def hyenand_plan_device_status(plan: int) -> int:

@@ -198,3 +198,12 @@ def test_scaled_named_workloads():
         w = W.WORKLOADS[name].scaled(B=B, C=C)
         q, k, v, h = W.make_inputs(w)
         check(w, q, k, v, h)
+
+
+def test_bounded_wait_runs_out_and_is_reported():
+    """The waits of the TMA kernels are bounded polls: a wait on a barrier that nothing ever completes must
+    come back and record its code instead of hanging (no fault, no trap: the kernel simply returns)."""
+    from paper_2607_19378_b200 import hyenand as hn
+    assert hn.hyenand_selftest_bounded_wait(200) == 9
+    # the device is still usable afterwards
+    assert float(torch.ones(8, device="cuda").sum().item()) == 8.0
