@@ -88,11 +88,18 @@ int hyenand_forward_ex(hyenand_plan *plan, const void *q, const void *k, const v
 
 /*
  * End-to-end variant: q, k, v, h, y are HOST pointers (pinned memory gives the
- * fastest copies but any host memory works).  Copies the inputs to device
- * staging buffers owned by the plan (allocated on the first call, which
- * therefore may synchronise), runs the same kernels as hyenand_forward_ex and
- * copies y back, all on cuda_stream; returns after y has arrived on the host
- * (the call synchronises the stream).
+ * fastest copies and is needed for the copies to overlap; any host memory
+ * works).  Copies the inputs to device staging buffers owned by the plan
+ * (allocated on the first call, which therefore may synchronise), runs the
+ * same kernels as hyenand_forward_ex and copies y back.  Problems above 64 MB
+ * are pipelined over up to eight groups of (b,c) slices: the inputs of the next
+ * group travel on a copy stream of the plan while the current group is computed
+ * on cuda_stream and the previous group's result travels back on a second copy
+ * stream (a filter shared over the batch is copied first, whole).  The copy
+ * streams start after the work already queued on cuda_stream.  The result is
+ * bit-identical to hyenand_forward_ex on device copies of the same tensors.
+ * Returns after y has arrived on the host (the call synchronises all three
+ * streams).
  */
 int hyenand_forward_host(hyenand_plan *plan, const void *q, const void *k, const void *v,
                          const void *h, long long h_batch_stride_elems, void *y, void *cuda_stream);

@@ -421,9 +421,9 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
     const TwoLevel twp{c->twp_coarse, c->twp_fine, c->lo};
     if (ct1d_uses_w(c)) {
         const bool staged_ok = c->causal != 0;
-        if (shared && ct1d_w_filter(c, h, c->C, staged_ok, st, launches, prof, filter_pass)) return -1;
-        for (long long s0 = 0; s0 < S; s0 += c->slices_per_chunk) {
-            const long long n = S - s0 < c->slices_per_chunk ? S - s0 : c->slices_per_chunk;
+        if (shared && c->r0 == 0 && ct1d_w_filter(c, h, c->C, staged_ok, st, launches, prof, filter_pass)) return -1;
+        for (long long s0 = c->r0; s0 < c->r1; s0 += c->slices_per_chunk) {
+            const long long n = c->r1 - s0 < c->slices_per_chunk ? c->r1 - s0 : c->slices_per_chunk;
             if (!shared && ct1d_w_filter(c, (const char *)h + (size_t)s0 * c->K * es, n, staged_ok, st, launches, prof, filter_pass))
                 return -1;
             if (ct1d_w_body(c, (const char *)q + (size_t)s0 * c->L * es, (const char *)k + (size_t)s0 * c->L * es,
@@ -433,9 +433,9 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
         }
         return 0;
     }
-    if (shared && filter_pass(c, (const char *)h, c->C, st, launches, prof)) return -1;
-    for (long long s0 = 0; s0 < S; s0 += c->slices_per_chunk) {
-        const long long n = S - s0 < c->slices_per_chunk ? S - s0 : c->slices_per_chunk;
+    if (shared && c->r0 == 0 && filter_pass(c, (const char *)h, c->C, st, launches, prof)) return -1;
+    for (long long s0 = c->r0; s0 < c->r1; s0 += c->slices_per_chunk) {
+        const long long n = c->r1 - s0 < c->slices_per_chunk ? c->r1 - s0 : c->slices_per_chunk;
         if (!shared && filter_pass(c, (const char *)h + (size_t)s0 * c->K * es, n, st, launches, prof)) return -1;
         ColsFwdArgs a{};
         a.a = (const char *)k + (size_t)s0 * c->L * es; a.b = (const char *)v + (size_t)s0 * c->L * es;

@@ -19,6 +19,7 @@ struct Ct1dPlan {
     int lo;
     int *status;              // device word set when a bounded wait on a tensor copy gives up (owned by the plan)
     long long slices_per_chunk, wh_slices;
+    long long r0, r1;         // slices [r0, r1) the next forward works on
 };
 
 int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, int dtype, size_t *bytes);

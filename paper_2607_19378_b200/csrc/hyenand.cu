@@ -52,6 +52,10 @@ struct hyenand_plan {
     // tensor maps of the fused core's workspace buffers (valid only where the TMA core applies)
     CoreTmaMaps tma;
     int *dev_status;                  // device word set by a kernel whose bounded wait gave up
+    // slices [r0, r1) the next forward works on (the whole batch except inside hyenand_forward_host's pipeline)
+    long long r0, r1;
+    cudaStream_t copy_in, copy_out;   // streams of hyenand_forward_host's pipeline (created on first use)
+    cudaEvent_t ev_in[2], ev_out;
     // long 1-D path
     Ct1dPlan ct;
     // host-staging for hyenand_forward_host
@@ -95,6 +99,10 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
     cudaFree(p->ws_a); cudaFree(p->ws_b); cudaFree(p->wh_a); cudaFree(p->wh_b); cudaFree(p->gtw); cudaFree(p->dev_status);
     ct1d_free(&p->ct);
     for (int i = 0; i < 5; ++i) cudaFree(p->stage[i]);
+    if (p->copy_in) cudaStreamDestroy(p->copy_in);
+    if (p->copy_out) cudaStreamDestroy(p->copy_out);
+    for (int i = 0; i < 2; ++i) if (p->ev_in[i]) cudaEventDestroy(p->ev_in[i]);
+    if (p->ev_out) cudaEventDestroy(p->ev_out);
     p->prof.destroy();
     if (cur != p->device) cudaSetDevice(cur);
     delete p;
@@ -118,6 +126,7 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     hyenand_plan *p = new hyenand_plan();
     memset(p, 0, sizeof(*p));
     p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype;
+    p->r0 = 0; p->r1 = (long long)B * C;
     cudaGetDevice(&p->device);
     p->vol = 1; p->kvol = 1;
     for (int a = 0; a < 3; ++a) { p->L[a] = 1; p->K[a] = 1; p->P[a] = 1; p->log2p[a] = 0; }
@@ -299,9 +308,9 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
     const long long S = (long long)p->B * p->C;
     const size_t es = elsize(p->dtype);
     const bool three = p->P[0] > 1;
-    if (shared && filter_spectrum_generic(p, h, p->C, st, launches)) return -1;
-    for (long long s0 = 0; s0 < S; s0 += p->slices_per_chunk) {
-        const long long n = S - s0 < p->slices_per_chunk ? S - s0 : p->slices_per_chunk;
+    if (shared && p->r0 == 0 && filter_spectrum_generic(p, h, p->C, st, launches)) return -1;
+    for (long long s0 = p->r0; s0 < p->r1; s0 += p->slices_per_chunk) {
+        const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter_spectrum_generic(p, h + (size_t)s0 * p->kvol * es, n, st, launches)) return -1;
         RowsArgs r{};
         r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = p->ws_a; r.pitch = p->XP;
@@ -399,9 +408,9 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         *launches += c;
         return 0;
     };
-    if (shared && filter(h, p->C)) return -1;
-    for (long long s0 = 0; s0 < S; s0 += p->slices_per_chunk) {
-        const long long n = S - s0 < p->slices_per_chunk ? S - s0 : p->slices_per_chunk;
+    if (shared && p->r0 == 0 && filter(h, p->C)) return -1;
+    for (long long s0 = p->r0; s0 < p->r1; s0 += p->slices_per_chunk) {
+        const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter(h + (size_t)s0 * p->kvol * es, n)) return -1;
         PlaneArgs u{};
         u.a = k + (size_t)s0 * p->vol * es; u.b = v + (size_t)s0 * p->vol * es; u.out = p->ws_a;
@@ -437,9 +446,12 @@ static int forward_fused2d(hyenand_plan *p, const void *q, const void *k, const 
                            bool shared, void *y, cudaStream_t st, int *launches)
 {
     Fused2dArgs a{};
-    a.q = q; a.k = k; a.v = v; a.h = h; a.y = y;
-    a.slices = (long long)p->B * p->C; a.lx = p->L[2]; a.ly = p->L[1];
-    a.h_mod = shared ? p->C : 0; a.h_off = 0;
+    const size_t es = elsize(p->dtype);
+    const size_t off = (size_t)p->r0 * p->vol * es;
+    a.q = (const char *)q + off; a.k = (const char *)k + off; a.v = (const char *)v + off; a.y = (char *)y + off;
+    a.h = shared ? h : (const void *)((const char *)h + (size_t)p->r0 * p->kvol * es);
+    a.slices = p->r1 - p->r0; a.lx = p->L[2]; a.ly = p->L[1];
+    a.h_mod = shared ? p->C : 0; a.h_off = shared ? p->r0 % p->C : 0;
     a.scale = (float)(1.0 / ((double)p->P[1] * p->P[2]));
     a.gtw = p->gtw; a.gtw_n = p->gtw_n;
     a.kv_elems = a.slices * p->vol;
@@ -462,7 +474,10 @@ static int run_forward(hyenand_plan *p, const void *q, const void *k, const void
         rc = forward_planes3d(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
                               (char *)y, st, launches);
     else if (p->path == PATH_CT1D)
+    {
+        p->ct.r0 = p->r0; p->ct.r1 = p->r1;
         rc = ct1d_forward(&p->ct, q, k, v, h, shared, y, st, launches, &p->prof);
+    }
     else
         rc = forward_generic(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
                              (char *)y, st, launches);
@@ -535,16 +550,51 @@ extern "C" int hyenand_forward_host(hyenand_plan *p, const void *q, const void *
             p->stage_bytes[i] = want[i];
         }
     }
-    const void *src[4] = {q, k, v, h};
-    for (int i = 0; i < 4; ++i)
-        if (cudaMemcpyAsync(p->stage[i], src[i], want[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return fail(HYENAND_ERR_CUDA, "host-to-device copy %d failed: %s", i, cudaGetErrorString(cudaGetLastError()));
+    // Pipeline over groups of slices: the inputs of group g+1 travel to the device (copy-in stream) while group g
+    // is computed (caller's stream) and the result of group g-1 travels back (copy-out stream).  A filter shared
+    // over the batch goes first, whole.  With one group this is copy, compute, copy.
+    if (!p->copy_in) {
+        if (cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p->ev_in[0], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p->ev_in[1], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&p->ev_out, cudaEventDisableTiming) != cudaSuccess)
+            return fail(HYENAND_ERR_CUDA, "pipeline streams: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+    const long long S = (long long)p->B * p->C;
+    const size_t sl = (size_t)p->vol * es, hsl = (size_t)p->kvol * es;       // bytes per slice
+    long long groups = S < 8 ? S : 8;
+    if (nbytes + hbytes < ((size_t)64 << 20)) groups = 1;                      // small problems: nothing to overlap
+    const long long per = (S + groups - 1) / groups;
     int launches = 0;
-    e = run_forward(p, p->stage[0], p->stage[1], p->stage[2], p->stage[3], shared, p->stage[4], st, &launches);
-    if (e) return e;
-    if (cudaMemcpyAsync(y, p->stage[4], nbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return fail(HYENAND_ERR_CUDA, "device-to-host copy failed: %s", cudaGetErrorString(cudaGetLastError()));
-    cudaError_t ce = cudaStreamSynchronize(st);
+    bool bad = false;
+    // the copy-in stream starts after whatever the caller's stream holds (the staging buffers may still be read)
+    bad |= cudaEventRecord(p->ev_out, st) != cudaSuccess || cudaStreamWaitEvent(p->copy_in, p->ev_out, 0) != cudaSuccess;
+    if (shared) bad |= cudaMemcpyAsync(p->stage[3], h, hbytes, cudaMemcpyHostToDevice, p->copy_in) != cudaSuccess;
+    int g = 0;
+    for (long long s0 = 0; s0 < S && !bad; s0 += per, ++g) {
+        const long long n = S - s0 < per ? S - s0 : per;
+        const void *src[3] = {k, v, q};
+        const int dsti[3] = {1, 2, 0};
+        if (!shared)
+            bad |= cudaMemcpyAsync((char *)p->stage[3] + s0 * hsl, (const char *)h + s0 * hsl, n * hsl, cudaMemcpyHostToDevice, p->copy_in) != cudaSuccess;
+        for (int i = 0; i < 3; ++i)
+            bad |= cudaMemcpyAsync((char *)p->stage[dsti[i]] + s0 * sl, (const char *)src[i] + s0 * sl, n * sl, cudaMemcpyHostToDevice, p->copy_in) != cudaSuccess;
+        cudaEvent_t ev = p->ev_in[g & 1];
+        // an event is reused every other group: by then the compute stream has long passed its previous wait
+        bad |= cudaEventRecord(ev, p->copy_in) != cudaSuccess || cudaStreamWaitEvent(st, ev, 0) != cudaSuccess;
+        if (bad) break;
+        p->r0 = s0; p->r1 = s0 + n;
+        e = run_forward(p, p->stage[0], p->stage[1], p->stage[2], p->stage[3], shared, p->stage[4], st, &launches);
+        p->r0 = 0; p->r1 = S;
+        if (e) return e;
+        bad |= cudaEventRecord(p->ev_out, st) != cudaSuccess || cudaStreamWaitEvent(p->copy_out, p->ev_out, 0) != cudaSuccess;
+        bad |= cudaMemcpyAsync((char *)y + s0 * sl, (char *)p->stage[4] + s0 * sl, n * sl, cudaMemcpyDeviceToHost, p->copy_out) != cudaSuccess;
+    }
+    if (bad) return fail(HYENAND_ERR_CUDA, "pipelined host copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+    cudaError_t ce = cudaStreamSynchronize(p->copy_out);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(p->copy_in);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
     if (ce != cudaSuccess) return fail(HYENAND_ERR_CUDA, "stream synchronise failed: %s", cudaGetErrorString(ce));
     return HYENAND_OK;
 }
@@ -763,6 +813,7 @@ extern "C" int hyenand_forward_noalloc(int ndim, const int *dims, int B, int C, 
     memset(&sp, 0, sizeof(sp));
     hyenand_plan *p = &sp;
     p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype;
+    p->r0 = 0; p->r1 = (long long)B * C;
     p->vol = 1; p->kvol = 1;
     for (int a = 0; a < 3; ++a) { p->L[a] = 1; p->K[a] = 1; p->P[a] = 1; p->log2p[a] = 0; }
     for (int a = 0; a < ndim; ++a) {

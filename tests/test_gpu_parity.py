@@ -207,3 +207,35 @@ def test_bounded_wait_runs_out_and_is_reported():
     assert hn.hyenand_selftest_bounded_wait(200) == 9
     # the device is still usable afterwards
     assert float(torch.ones(8, device="cuda").sum().item()) == 8.0
+
+
+HOST_CASES = [
+    ((512, 512), 2, 8, "f32", False, False),        # generic 2-D, eight groups of two slices
+    ((131072,), 4, 64, "bf16", True, True),         # long 1-D, filter shared over the batch
+    ((72, 64, 64), 1, 16, "bf16", False, False),    # plane-fused 3-D with the TMA core
+    ((64, 64), 16, 128, "bf16", False, False),      # fused 2-D
+    ((20, 30), 2, 3, "f32", False, True),           # small: a single group
+]
+
+
+@pytest.mark.parametrize("dims,B,C,dtype,causal,shared", HOST_CASES, ids=str)
+def test_host_forward_pipeline_matches_device_forward(dims, B, C, dtype, causal, shared):
+    """hyenand_forward_host (host buffers, copies pipelined over groups of slices inside the call) returns
+    exactly what hyenand_forward computes on device-resident copies of the same tensors."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w = W.Workload("host", dims, B, C, dtype, seed=3, causal=causal, h_shared=shared)
+    q, k, v, h = W.make_inputs(w, device="cpu")
+    plan = hn.Plan(w.dims, w.B, w.C, causal=causal, dtype=w.torch_dtype)
+    try:
+        dq, dk, dv, dh = (t.cuda() for t in (q, k, v, h))
+        y_dev = torch.full_like(dq, float("nan"))
+        plan.forward(dq, dk, dv, dh, y_dev)
+        torch.cuda.synchronize()
+        host = [t.contiguous().pin_memory() for t in (q, k, v, h)]
+        y_host = torch.full_like(q, float("nan")).pin_memory()
+        plan.forward_host(*host, y_host)
+        plan.forward_host(*host, y_host)                    # and again over the same staging buffers
+        assert hn.hyenand_plan_device_status(plan.handle) == 0
+    finally:
+        plan.close()
+    assert torch.equal(y_host, y_dev.cpu())
