@@ -416,7 +416,6 @@ static int filter_pass(Ct1dPlan *c, const char *h, long long n, cudaStream_t st,
 int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const void *h, bool shared,
                  void *y, cudaStream_t st, int *launches, Prof *prof)
 {
-    const long long S = (long long)c->B * c->C;
     const size_t es = c->dtype == 0 ? 4 : 2;
     const TwoLevel twp{c->twp_coarse, c->twp_fine, c->lo};
     if (ct1d_uses_w(c)) {

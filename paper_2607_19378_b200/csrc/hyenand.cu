@@ -305,7 +305,6 @@ static AxisArgs generic_core_args(const hyenand_plan *p, long long n, bool share
 static int forward_generic(hyenand_plan *p, const char *q, const char *k, const char *v, const char *h,
                            bool shared, char *y, cudaStream_t st, int *launches)
 {
-    const long long S = (long long)p->B * p->C;
     const size_t es = elsize(p->dtype);
     const bool three = p->P[0] > 1;
     if (shared && p->r0 == 0 && filter_spectrum_generic(p, h, p->C, st, launches)) return -1;
@@ -393,9 +392,7 @@ static AxisArgs planes3d_core_args(const hyenand_plan *p, long long n, bool shar
 static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const char *v, const char *h,
                             bool shared, char *y, cudaStream_t st, int *launches)
 {
-    const long long S = (long long)p->B * p->C;
     const size_t es = elsize(p->dtype);
-    const long long nc = (long long)p->XH * p->P[1];
     auto filter = [&](const char *hp, long long n) -> int {
         PlaneArgs a{};
         a.a = hp; a.out = p->wh_a; a.planes = n * p->K[0];

@@ -144,7 +144,6 @@ __global__ void __launch_bounds__(kThreads) rows_inv_kernel(RowsInvArgs p)
 {
     constexpr int N = 1 << LOG2P;
     constexpr int LS = line_stride(N);
-    constexpr int XH = N / 2 + 1;
     extern __shared__ float2 smem[];
     const int G = lines_per_chunk(LOG2P);
     float2 *buf = smem;
