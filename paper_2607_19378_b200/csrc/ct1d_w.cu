@@ -27,6 +27,13 @@ constexpr int kCtThreads = 256;
 // 16-byte accesses of neighbouring lines (tile loads and stores run across lines) hit different banks
 __host__ __device__ constexpr int ct_ls(int n) { return (n + 15) / 16 * 16 + 2; }
 __host__ __device__ constexpr int ct_tx(int tpl) { return kCtThreads / tpl > 8 ? kCtThreads / tpl : 8; }
+// result tile of the forward column kernel as tensor copies: F1 rows in one box, or in two boxes whose
+// starts stay on 1024-byte boundaries (rows per box a multiple of 8)
+__host__ __device__ constexpr int ct_out_boxes(int f1) { return (f1 + 7) / 8 * 8 > 256 ? 2 : 1; }
+__host__ __device__ constexpr int ct_out_box_rows(int f1)
+{
+    return ct_out_boxes(f1) == 1 ? (f1 + 7) / 8 * 8 : ((f1 + 1) / 2 + 7) / 8 * 8;
+}
 // the inverse column kernel runs as CTAs of 4 warps: more, smaller tiles in flight per SM
 constexpr int kCtInvThreads = 128;
 __host__ __device__ constexpr int ct_inv_tx(int tpl) { return kCtInvThreads / tpl > 8 ? kCtInvThreads / tpl : 8; }
@@ -67,7 +74,8 @@ struct ColsFwdWArgs {
 // asynchronous copies per thread into padded rows.
 template <typename T, int LOG2P1, bool HAS_B, bool TMA>
 __global__ void __launch_bounds__(kCtThreads, (LOG2P1 >= 9 ? 2 : 4))
-ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b)
+ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const __grid_constant__ CUtensorMap map_o)
 {
     using F = WF<LOG2P1, false>;
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = F::TPL;
@@ -90,6 +98,14 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
     static_assert(!TMA || TROW == 64 || TROW == 128, "tile rows match a swizzle span");
     if constexpr (TMA) raw += (1024u - (smem_u32(raw) & 1023u)) & 1023u;
     uint64_t *bar = reinterpret_cast<uint64_t *>(raw + 2 * TBYTES);
+    // Result tile as tensor copies too (one line per group): the separated bins are written row-major
+    // [f1][pair] into a swizzled staging area that reuses the lines, as two halves of 8 pairs (128-byte rows);
+    // boxes of 136 rows keep every box start on a 1024-byte boundary.
+    constexpr bool TSTORE = TMA && TX == 16 && NGRP == 16;
+    constexpr int ONB = ct_out_boxes(F1), OBOXR = ct_out_box_rows(F1), OHALF = ONB * OBOXR * 128;   // boxes, rows per box, bytes per half
+    static_assert(!TSTORE || (F1 <= ONB * OBOXR && 2 * OHALF + 1024 <= TX * LS * 8), "result staging fits the lines");
+    unsigned char *to0 = reinterpret_cast<unsigned char *>(lines);
+    if constexpr (TSTORE) to0 += (1024u - (smem_u32(to0) & 1023u)) & 1023u;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     PassTw<LOG2P1, false>::build(twt, p.tw1, P1, tid, kCtThreads);
@@ -122,6 +138,7 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
         const long long s = t / tpc;
         const int c0 = (int)(t % tpc) * TX;
         const long long base = s * p.in_slice;
+        if constexpr (TSTORE) { if (tid == 0) tma_wait_read0(); }   // the previous result tile has left the lines
         __syncthreads();                                   // previous tile done with raw and lines
         if constexpr (TMA) {
             if (!mbar_wait(bar, phase)) failed = 1;
@@ -145,6 +162,7 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
         cp_async_wait_all();
         __syncthreads();
         }
+        float2 A0[(F1 + TPL - 1) / TPL], A1[(F1 + TPL - 1) / TPL];
         for (int x = gid; x < TX; x += NGRP) {
         float2 *line = lines + x * LS;
         // TMA: the 16-byte chunk of pair x in row idx is XORed with a function of idx that the engine's strides
@@ -171,7 +189,6 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
             // (at most three products after a table value).
             const float2 cl0 = twp_w(p.twp, t2 * (unsigned)l), cl1 = twp_w(p.twp, (t2 + 1u) * (unsigned)l);
             const float2 st0 = twp_w(p.twp, t2 * (unsigned)TPL), st1 = twp_w(p.twp, (t2 + 1u) * (unsigned)TPL);
-            float2 A0[(F1 + TPL - 1) / TPL], A1[(F1 + TPL - 1) / TPL];
             float2 w0 = cl0, w1 = cl1;
 #pragma unroll
             for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
@@ -192,18 +209,41 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
                 }
             }
             __syncwarp(m);
+            if constexpr (!TSTORE) {
 #pragma unroll
-            for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
-                const int f1 = l + i * TPL;
-                if (f1 < F1) *reinterpret_cast<float4 *>(line + 2 * f1) = make_float4(A0[i].x, A0[i].y, A1[i].x, A1[i].y);
+                for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
+                    const int f1 = l + i * TPL;
+                    if (f1 < F1) *reinterpret_cast<float4 *>(line + 2 * f1) = make_float4(A0[i].x, A0[i].y, A1[i].x, A1[i].y);
+                }
             }
         }
         }
         if constexpr (TMA) {
-            if (__syncthreads_or(failed)) break;           // the tile buffers are free again
+            if (__syncthreads_or(failed)) break;           // the tile buffers are free again (and every line has been read)
             if (tid == 0 && t + gridDim.x < tiles) issue(t + gridDim.x);
         } else {
             __syncthreads();
+        }
+        if constexpr (TSTORE) {
+            // group gid holds pair x = gid: rows f1 = l + i*TPL, 16 bytes each, chunk index XORed with (f1 & 7)
+            unsigned char *th = to0 + (gid >> 3) * OHALF;
+#pragma unroll
+            for (int i = 0; i < (F1 + TPL - 1) / TPL; ++i) {
+                const int f1 = l + i * TPL;
+                if (f1 < F1)
+                    *reinterpret_cast<float4 *>(th + f1 * 128 + (((gid & 7) ^ (f1 & 7)) << 4)) = make_float4(A0[i].x, A0[i].y, A1[i].x, A1[i].y);
+            }
+            fence_async_smem();
+            __syncthreads();
+            if (tid == 0) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                    for (int rb = 0; rb < ONB; ++rb)
+                        tma_store_3d(&map_o, to0 + hh * OHALF + rb * OBOXR * 128, 4 * c0 + 32 * hh, rb * OBOXR, (int)s);
+                tma_commit();
+            }
+            continue;
         }
         float2 *dst = p.out + s * (long long)F1 * P2 + 2 * c0;
         for (int idx = tid; idx < F1 * TX; idx += kCtThreads) {
@@ -219,6 +259,7 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
             mbar_wait(bar, phase);
         }
     }
+    if constexpr (TSTORE) { if (tid == 0) tma_wait_all0(); }
 }
 
 // ---- filter rows: spectrum in place -----------------------------------------------------------------
@@ -464,12 +505,13 @@ bool ct1d_w_supported(int log2p1, int log2p2, int L, int K, int causal, int dtyp
 }
 
 template <typename T, int LOG2P1, bool HAS_B, bool TMA>
-static void launch_cols_fwd_w_tt(const ColsFwdWArgs &a, const CUtensorMap &ma, const CUtensorMap &mb, int grid, size_t sm, cudaStream_t st)
+static void launch_cols_fwd_w_tt(const ColsFwdWArgs &a, const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mo, int grid,
+                                size_t sm, cudaStream_t st)
 {
     static DevOnce attr;
     if (attr.first())
         cudaFuncSetAttribute(ct_cols_fwd_w_kernel<T, LOG2P1, HAS_B, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    ct_cols_fwd_w_kernel<T, LOG2P1, HAS_B, TMA><<<grid, kCtThreads, sm, st>>>(a, ma, mb);
+    ct_cols_fwd_w_kernel<T, LOG2P1, HAS_B, TMA><<<grid, kCtThreads, sm, st>>>(a, ma, mb, mo);
 }
 
 template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWArgs &a, cudaStream_t st)
@@ -484,9 +526,10 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
     if (grid <= 0) return 0;
     // Tensor copies need the slice to be a whole number of rows of P2 elements (then [slice][row][P2] is an
     // exact view of the input and rows past the data read as zeros) and tile rows of 64 or 128 bytes.
-    alignas(64) CUtensorMap ma, mb;
+    alignas(64) CUtensorMap ma, mb, mo;
     memset(&ma, 0, sizeof(ma));
     memset(&mb, 0, sizeof(mb));
+    memset(&mo, 0, sizeof(mo));
     constexpr unsigned TROW = TX * 2 * sizeof(T);
     bool tma = (TROW == 64 || TROW == 128) && a.len % P2 == 0 && a.slices < (1ll << 31) && tma_available() &&
                !getenv("HYENAND_NO_TMA");
@@ -497,16 +540,21 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
         const unsigned box[3] = {2 * TX, (unsigned)(HP1 < 256 ? HP1 : 256), 1};
         tma = tma_encode_3d(&ma, a.a, sizeof(T) == 2, dims, strides, box, (int)TROW);
         if (tma && a.b) tma = tma_encode_3d(&mb, a.b, sizeof(T) == 2, dims, strides, box, (int)TROW);
+        // results [slice][P1/2+1][P2] complex, as fp32: boxes of 8 column pairs (32 floats) by 136 rows
+        const unsigned long long od[3] = {2ull * P2, (unsigned long long)(HP1 + 1), (unsigned long long)a.slices};
+        const unsigned long long os[2] = {(unsigned long long)P2 * 8, (unsigned long long)(HP1 + 1) * P2 * 8};
+        const unsigned ob[3] = {32, (unsigned)ct_out_box_rows(HP1 + 1), 1};
+        if (tma) tma = tma_encode_3d(&mo, a.out, false, od, os, ob, 128);
     }
     if constexpr (TROW == 64 || TROW == 128) {
         if (tma) {
-            if (a.b) launch_cols_fwd_w_tt<T, LOG2P1, true, true>(a, ma, mb, grid, sm, st);
-            else launch_cols_fwd_w_tt<T, LOG2P1, false, true>(a, ma, mb, grid, sm, st);
+            if (a.b) launch_cols_fwd_w_tt<T, LOG2P1, true, true>(a, ma, mb, mo, grid, sm, st);
+            else launch_cols_fwd_w_tt<T, LOG2P1, false, true>(a, ma, mb, mo, grid, sm, st);
             return 1;
         }
     }
-    if (a.b) launch_cols_fwd_w_tt<T, LOG2P1, true, false>(a, ma, mb, grid, sm, st);
-    else launch_cols_fwd_w_tt<T, LOG2P1, false, false>(a, ma, mb, grid, sm, st);
+    if (a.b) launch_cols_fwd_w_tt<T, LOG2P1, true, false>(a, ma, mb, mo, grid, sm, st);
+    else launch_cols_fwd_w_tt<T, LOG2P1, false, false>(a, ma, mb, mo, grid, sm, st);
     return 1;
 }
 
