@@ -392,10 +392,14 @@ struct ColsInvWArgs {
     int len;                  // L (multiple of 16 bytes worth of elements)
     int log2p2;
     const float2 *tw1;
+    int *status;              // device word set when a bounded wait on a tensor copy gives up (may be NULL)
 };
 
-template <typename T, int LOG2P1>
-__global__ void __launch_bounds__(kCtInvThreads, (LOG2P1 >= 9 ? 4 : 8)) ct_cols_inv_w_kernel(ColsInvWArgs p)
+// TMA = true: the gate tile q arrives, and the result tile y leaves, as tensor copies ([t1][pair] rows of
+// TX pairs, no swizzle: a warp touches whole consecutive rows); false: per-thread loads and stores.
+template <typename T, int LOG2P1, bool TMA>
+__global__ void __launch_bounds__(kCtInvThreads, (LOG2P1 >= 9 ? 4 : 8))
+ct_cols_inv_w_kernel(ColsInvWArgs p, const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_y)
 {
     using FI = WF<LOG2P1, true>;
     constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, F1 = HP1 + 1, TPL = FI::TPL;
@@ -405,8 +409,23 @@ __global__ void __launch_bounds__(kCtInvThreads, (LOG2P1 >= 9 ? 4 : 8)) ct_cols_
     extern __shared__ float2 smem[];
     float2 *lines = smem;
     float2 *twt = lines + TX * LS;
+    // gate and result tiles: HP1 rows of TX pairs
+    constexpr unsigned QROW = TX * 2 * sizeof(T), QBYTES = HP1 * QROW;
+    constexpr int QBOXR = HP1 < 256 ? HP1 : 256, QNB = HP1 / QBOXR;
+    unsigned char *tq = reinterpret_cast<unsigned char *>(twt + P1);
+    if constexpr (TMA) tq += (128u - (smem_u32(tq) & 127u)) & 127u;
+    unsigned char *ty = tq + QBYTES;
+    uint64_t *bar = reinterpret_cast<uint64_t *>(ty + QBYTES);
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = FI::group_mask(tid);
+    if constexpr (TMA) {
+        if (tid == 0) {
+            mbar_init(bar, 1);
+            fence_mbar_init();
+        }
+    }
+    unsigned phase = 0;
+    int failed = 0;
     PassTw<LOG2P1, true>::build(twt, p.tw1, P1, tid, kCtInvThreads);
     const PassTw<LOG2P1, true> tw{twt};
     const int P2 = 1 << p.log2p2;
@@ -418,7 +437,15 @@ __global__ void __launch_bounds__(kCtInvThreads, (LOG2P1 >= 9 ? 4 : 8)) ct_cols_
         const long long s = t / tpc;
         const int c0 = (int)(t % tpc) * TX;
         const float2 *src = p.in + s * (long long)F1 * P2 + 2 * c0;
+        if constexpr (TMA) { if (tid == 0) tma_wait_read0(); }        // the previous result tile has left its buffer
         __syncthreads();
+        if constexpr (TMA) {
+            if (tid == 0) {
+                mbar_expect_tx(bar, QBYTES);
+#pragma unroll
+                for (int b = 0; b < QNB; ++b) tma_load_3d(tq + b * QBOXR * QROW, &map_q, bar, 2 * c0, b * QBOXR, (int)s);
+            }
+        }
         // both bins of a column pair land side by side in slot f1 of that pair's line
         for (int idx = tid; idx < F1 * TX; idx += kCtInvThreads) {
             const int f1 = idx / TX, x = idx % TX;
@@ -444,16 +471,38 @@ __global__ void __launch_bounds__(kCtInvThreads, (LOG2P1 >= 9 ? 4 : 8)) ct_cols_
         __syncthreads();
         // line x now holds, at position t1 < P1/2, the two real outputs of columns 2x, 2x+1
         const long long base = s * (long long)p.len + 2 * c0;
-        // gate values first (all requests in flight together), then products and stores
-        constexpr int NE = HP1 * TX / kCtInvThreads;
-        static_assert(HP1 * TX % kCtInvThreads == 0, "whole epilogue rounds");
         // a half warp takes 8 pairs of two neighbouring rows: line stride and skew then spread its
         // 16 reads over all banks, and each row still receives whole 32-byte sectors
+        constexpr int NE = HP1 * TX / kCtInvThreads;
+        static_assert(HP1 * TX % kCtInvThreads == 0, "whole epilogue rounds");
         const int x = (tid & 7) + 8 * ((tid >> 4) % (TX / 8));
         const int tb = ((tid >> 3) & 1) + 2 * ((tid >> 4) / (TX / 8));
         constexpr int TSTEP = kCtInvThreads / TX;
-        const long long ox = base + 2 * x;
         using Q2 = typename std::conditional<sizeof(T) == 4, float2, __nv_bfloat162>::type;
+        if constexpr (TMA) {
+            // gate values from the tile that arrived during the transforms; results into the staging tile
+            if (!mbar_wait(bar, phase)) failed = 1;
+            phase ^= 1u;
+#pragma unroll
+            for (int e = 0; e < NE; ++e) {
+                const int t1 = tb + e * TSTEP;
+                const float2 z = lines[x * LS + FI::ph(t1)];
+                const Q2 qv = *reinterpret_cast<const Q2 *>(tq + t1 * QROW + x * sizeof(Q2));
+                Q2 *o = reinterpret_cast<Q2 *>(ty + t1 * QROW + x * sizeof(Q2));
+                if constexpr (sizeof(T) == 4) *o = make_float2(z.x * qv.x, z.y * qv.y);
+                else *o = __floats2bfloat162_rn(z.x * __low2float(qv), z.y * __high2float(qv));
+            }
+            fence_async_smem();
+            if (__syncthreads_or(failed)) break;
+            if (tid == 0) {
+#pragma unroll
+                for (int b = 0; b < QNB; ++b) tma_store_3d(&map_y, ty + b * QBOXR * QROW, 2 * c0, b * QBOXR, (int)s);
+                tma_commit();
+            }
+            continue;
+        }
+        // gate values first (all requests in flight together), then products and stores
+        const long long ox = base + 2 * x;
         Q2 qv[NE];
 #pragma unroll
         for (int e = 0; e < NE; ++e) {
@@ -476,6 +525,13 @@ __global__ void __launch_bounds__(kCtInvThreads, (LOG2P1 >= 9 ? 4 : 8)) ct_cols_
                 }
             }
         }
+    }
+    if constexpr (TMA) {
+        if (failed) {
+            if (p.status) atomicExch(p.status, 8);
+            mbar_wait(bar, phase ^ 1u);
+        }
+        if (tid == 0) tma_wait_all0();
     }
 }
 
@@ -558,19 +614,40 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
     return 1;
 }
 
+template <typename T, int LOG2P1, bool TMA>
+static void launch_cols_inv_w_tt(const ColsInvWArgs &a, const CUtensorMap &mq, const CUtensorMap &my, int grid, size_t sm, cudaStream_t st)
+{
+    static DevOnce attr;
+    if (attr.first())
+        cudaFuncSetAttribute(ct_cols_inv_w_kernel<T, LOG2P1, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    ct_cols_inv_w_kernel<T, LOG2P1, TMA><<<grid, kCtInvThreads, sm, st>>>(a, mq, my);
+}
+
 template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWArgs &a, cudaStream_t st)
 {
     using F = WF<LOG2P1, true>;
-    constexpr int P1 = 1 << LOG2P1, TX = ct_inv_tx(F::TPL), LS = ct_ls(phys_max(P1) + 2);
-    const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1);
+    constexpr int P1 = 1 << LOG2P1, HP1 = P1 / 2, TX = ct_inv_tx(F::TPL), LS = ct_ls(phys_max(P1) + 2);
+    constexpr unsigned QROW = TX * 2 * sizeof(T);
+    // lines, twiddles, and (tensor-copy variant) gate tile, result tile, barrier, alignment slack
+    const size_t sm = sizeof(float2) * ((size_t)TX * LS + P1) + 2 * (size_t)HP1 * QROW + 8 + 128;
     const int P2 = 1 << a.log2p2;
     const long long tiles = a.slices * ((P2 / 2) / TX);
     const long long res = (LOG2P1 >= 9 ? 4ll : 8ll) * ctw_sms();   // resident CTAs
     const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
-    static DevOnce attr;
-    if (attr.first()) { cudaFuncSetAttribute(ct_cols_inv_w_kernel<T, LOG2P1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); }
-    ct_cols_inv_w_kernel<T, LOG2P1><<<grid, kCtInvThreads, sm, st>>>(a);
+    alignas(64) CUtensorMap mq, my;
+    memset(&mq, 0, sizeof(mq));
+    memset(&my, 0, sizeof(my));
+    // tensor copies need the slice to be a whole number of rows of P2 elements
+    bool tma = a.len % P2 == 0 && a.slices < (1ll << 31) && QROW % 16 == 0 && tma_available() && !getenv("HYENAND_NO_TMA");
+    if (tma) {
+        const unsigned long long dims[3] = {(unsigned long long)P2, (unsigned long long)(a.len / P2), (unsigned long long)a.slices};
+        const unsigned long long strides[2] = {(unsigned long long)P2 * sizeof(T), (unsigned long long)a.len * sizeof(T)};
+        const unsigned box[3] = {2 * TX, (unsigned)(HP1 < 256 ? HP1 : 256), 1};
+        tma = tma_encode_3d(&mq, a.q, sizeof(T) == 2, dims, strides, box, 0) && tma_encode_3d(&my, a.y, sizeof(T) == 2, dims, strides, box, 0);
+    }
+    if (tma) launch_cols_inv_w_tt<T, LOG2P1, true>(a, mq, my, grid, sm, st);
+    else launch_cols_inv_w_tt<T, LOG2P1, false>(a, mq, my, grid, sm, st);
     return 1;
 }
 
@@ -666,7 +743,7 @@ int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long l
     if (r < 0) return -1;
     *launches += r;
     ColsInvWArgs ci{};
-    ci.in = c->wu; ci.q = q; ci.y = y; ci.slices = n; ci.len = c->L; ci.log2p2 = c->log2p2; ci.tw1 = c->tw1;
+    ci.in = c->wu; ci.q = q; ci.y = y; ci.slices = n; ci.len = c->L; ci.log2p2 = c->log2p2; ci.tw1 = c->tw1; ci.status = c->status;
     prof->begin(KID_CT_COLS_INV, st);
 #define CALLF(L) r = launch_cols_inv_w_t<float, L>(ci, st)
 #define CALLB(L) r = launch_cols_inv_w_t<bf16, L>(ci, st)

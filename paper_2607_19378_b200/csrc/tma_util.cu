@@ -32,13 +32,14 @@ bool tma_encode_3d(CUtensorMap *map, const void *base, bool bf16, const unsigned
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     if ((strides[0] % 16) || (strides[1] % 16) || ((uintptr_t)base % 16)) return false;
-    if (swizzle_bytes != 64 && swizzle_bytes != 128) return false;
+    if (swizzle_bytes != 0 && swizzle_bytes != 64 && swizzle_bytes != 128) return false;
     const cuuint64_t d[3] = {dims[0], dims[1], dims[2]};
     const cuuint64_t s[2] = {strides[0], strides[1]};
     const cuuint32_t b[3] = {box[0], box[1], box[2]};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), d, s, b,
-              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

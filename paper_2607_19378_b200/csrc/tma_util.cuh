@@ -57,7 +57,7 @@ bool tma_available();
 // -1 a CUDA error).  Blocking; allocates and frees one device word.
 int tma_selftest_bounded_wait(int polls);
 // Encodes a 3-D tiled map of fp32 (bf16 = false) or bf16 elements: dims and box in elements (innermost first),
-// strides in bytes for dimensions 1 and 2, swizzle = bytes of one box row (64 or 128).  False if the arguments
+// strides in bytes for dimensions 1 and 2, swizzle = bytes of one box row (64 or 128) or 0 for none.  False if the arguments
 // break an alignment rule or the driver refuses.
 bool tma_encode_3d(CUtensorMap *map, const void *base, bool bf16, const unsigned long long dims[3],
                    const unsigned long long strides[2], const unsigned box[3], int swizzle_bytes);
