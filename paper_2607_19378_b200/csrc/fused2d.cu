@@ -15,7 +15,7 @@
 
 namespace hn {
 
-constexpr int kF2Threads = kPlaneThreads + 32;               // one extra warp for the packed column
+constexpr int kF2Threads = kPlaneThreads + 32;               // 68 groups of 8 lanes: one per column kx = 0 .. 64 of a 128-point plane
 
 template <int LOG2P> struct F2Cfg {
     static constexpr int P = 1 << LOG2P, HP = P / 2;
@@ -26,8 +26,11 @@ template <int LOG2P> struct F2Cfg {
     static constexpr int NGM = kPlaneThreads / F::TPL;       // groups of the 16 main warps
     static constexpr int NG = kF2Threads / F::TPL;           // all groups
     static constexpr int LS = plane_ls(P);
-    static constexpr size_t SMEM =
-        sizeof(float2) * ((size_t)HP * HCSS + 2 * (size_t)HP * UCSS + (size_t)NG * LS + 5 * P);
+    static constexpr int NCOL = HP + 1;                      // columns kx = 0 .. P/2, none packed
+    // entries per column store, rounded to an even count: what follows them (the lines, which receive 16-byte
+    // asynchronous copies) must start on a 16-byte boundary
+    static constexpr int HCSN = (NCOL * HCSS + 1) & ~1, UCSN = (NCOL * UCSS + 1) & ~1;
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HCSN + 2 * (size_t)UCSN + (size_t)NG * LS + 3 * P);
 };
 
 // Schedule per CTA (slices s0, s1, ... of this CTA):
@@ -46,11 +49,10 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
     constexpr int P = C::P, HP = C::HP, TPL = F::TPL, NP = F::NP, NGM = C::NGM;
     extern __shared__ float2 smem[];
     float2 *hcs = smem;
-    float2 *ucs0 = hcs + HP * C::HCSS;
-    float2 *wbuf = ucs0 + 2 * HP * C::UCSS;
-    float2 *x0 = wbuf + C::NG * C::LS;                       // packed column: filter bins kx = 0 ...
-    float2 *xn = x0 + P;                                     // ... and kx = P/2
-    float2 *tw = xn + P;
+    static_assert((C::HCSN + 2 * C::UCSN) % 2 == 0 && C::LS % 2 == 0, "lines start on 16-byte boundaries");
+    float2 *ucs0 = hcs + C::HCSN;
+    float2 *wbuf = ucs0 + 2 * C::UCSN;
+    float2 *tw = wbuf + C::NG * C::LS;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
@@ -77,18 +79,14 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
             const long long o0 = sp * vol + (long long)y0 * Lx, o1 = o0 + Lx;
             FI::template run<PRUNE_OUT>(l, m, twi, line,
                 [&](int, int, int idx) {
-                    // branch-free merge of two half spectra into one complex row (column 0 is packed)
+                    // branch-free merge of two half spectra into one complex row
                     const bool mirror = idx > HP;
                     const int kx = mirror ? P - idx : idx;
-                    const int col = kx == HP ? 0 : kx;
-                    const float2 A = ub[col * C::UCSS + y0];
-                    float2 B = ub[col * C::UCSS + y1];
+                    const float2 A = ub[kx * C::UCSS + y0];
+                    float2 B = ub[kx * C::UCSS + y1];
                     if (!has1) B = make_float2(0.f, 0.f);
                     const float sg = mirror ? -1.f : 1.f;
-                    float2 g = make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
-                    g = kx == 0 ? make_float2(A.x, B.x) : g;
-                    g = kx == HP ? make_float2(A.y, B.y) : g;
-                    return g;
+                    return make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
                 },
                 [&](int, int, int idx, float2 v) {
                     if (idx < Lx) {
@@ -103,7 +101,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
     int cur = 0;
     long long sprev = -1;
     for (long long s = blockIdx.x; s < p.slices; s += gridDim.x) {
-        float2 *ucs = ucs0 + cur * HP * C::UCSS;
+        float2 *ucs = ucs0 + cur * C::UCSN;
         const long long hs = p.h_mod ? (s + p.h_off) % p.h_mod : s;
         const long long sn = s + gridDim.x;
         if (sn < p.slices && tid < kPlaneThreads) {
@@ -141,10 +139,10 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
                         const int mx = (cw + i * TPL + r * (P / F::template Pass<0>::R)) & (P - 1);
                         return make_float2(staged<T>(s0, f0, mx), staged<T>(s1, f1, mx));
                     });
-                    separate_rows<LOG2P, C::HCSS>(line, hcs, yp0, yp1, l);
+                    separate_rows_full<LOG2P, C::HCSS>(line, hcs, yp0, yp1, l);
                     __syncwarp(m);
                 } else {
-                    for (int kx = l; kx < HP; kx += TPL) {
+                    for (int kx = l; kx <= HP; kx += TPL) {
                         hcs[kx * C::HCSS + yp0] = make_float2(0.f, 0.f);
                         hcs[kx * C::HCSS + yp1] = make_float2(0.f, 0.f);
                     }
@@ -181,19 +179,20 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
                             return make_float2(a, b);
                         });
                     }
-                    separate_rows<LOG2P, C::UCSS>(line, ucs, y0, y1, l);
+                    separate_rows_full<LOG2P, C::UCSS>(line, ucs, y0, y1, l);
                     __syncwarp(m);
                 }
             } else if (sprev >= 0) {
                 // ---- rows back of the previous slice (its columns were finished last iteration) ----
-                rows_back(sprev, ucs0 + (cur ^ 1) * HP * C::UCSS, gid - NGM / 2, NGM / 2);
+                rows_back(sprev, ucs0 + (cur ^ 1) * C::UCSN, gid - NGM / 2, NGM / 2);
             }
         }
         __syncthreads();
         // ---- columns: filter spectrum, k*v spectrum, product, inverse --------------------------
-        if (gid < NGM) {
-            for (int kx = spread_pair<8>(gid); kx < HP; kx += NGM) {
-                if (kx == 0) continue;                       // the packed column belongs to the extra warp
+        {
+            // every column kx = 0 .. P/2 has a group of its own (columns 0 and P/2 hold real data: their
+            // transforms are done as general complex ones, which keeps all groups on one code path)
+            for (int kx = spread_pair<8>(gid); kx <= HP; kx += C::NG) {
                 const float2 *hc = hcs + kx * C::HCSS;
                 float2 *uc = ucs + kx * C::UCSS;
                 float2 H[PL::IPL][PL::R];
@@ -216,40 +215,12 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
                     [&](int, int, int idx, float2 v) { uc[idx] = v; });
                 __syncwarp(m);
             }
-        } else if (gid < NGM + 2) {
-            // Column 0 carries the real bins kx = 0 and kx = P/2 of every row as one complex column:
-            // the spectra are split with the Hermitian symmetry, multiplied bin by bin and packed
-            // again.  Group NGM transforms and splits the filter part while group NGM+1 transforms
-            // the k*v part; they meet once, then group NGM+1 runs the inverse.
-            const unsigned m2 = (1u << (2 * TPL)) - 1u;      // lanes of the two groups (same warp)
-            if (gid == NGM) {
-                F::template run_to_line<PRUNE_NONE>(l, m, twf, line, [&](int, int, int idx) { return hcs[idx]; });
-                for (int ky = l; ky < P; ky += TPL) {
-                    const float2 c1 = line[F::ph(ky)], c2 = line[F::ph((P - ky) & (P - 1))];
-                    x0[ky] = make_float2(0.5f * p.scale * (c1.x + c2.x), 0.5f * p.scale * (c1.y - c2.y));
-                    xn[ky] = make_float2(0.5f * p.scale * (c1.y + c2.y), 0.5f * p.scale * (c2.x - c1.x));
-                }
-                __syncwarp(m2);
-            } else {
-                F::template run_to_line<PRUNE_IN>(l, m, twf, line,
-                    [&](int, int, int idx) { return idx < Ly ? ucs[idx] : make_float2(0.f, 0.f); });
-                __syncwarp(m2);
-                FI::template run<PRUNE_OUT, true>(l, m, twi, line,
-                    [&](int, int, int idx) {
-                        const float2 c1 = line[F::ph(idx)], c2 = line[F::ph((P - idx) & (P - 1))];
-                        const float2 u0 = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
-                        const float2 un = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
-                        const float2 y0 = cmul(u0, x0[idx]), yn = cmul(un, xn[idx]);
-                        return make_float2(y0.x - yn.y, y0.y + yn.x);
-                    },
-                    [&](int, int, int idx, float2 v) { ucs[idx] = v; });
-            }
         }
         __syncthreads();
         sprev = s;
         cur ^= 1;
     }
-    if (sprev >= 0 && gid < NGM) rows_back(sprev, ucs0 + (cur ^ 1) * HP * C::UCSS, gid, NGM);
+    if (sprev >= 0 && gid < NGM) rows_back(sprev, ucs0 + (cur ^ 1) * C::UCSN, gid, NGM);
 }
 
 template <typename T, int LOG2P> static int launch_fused2d_t(const Fused2dArgs &a, cudaStream_t st)
