@@ -34,7 +34,8 @@ template <int LOG2P> struct PlaneCfg {
     static constexpr int LS = plane_ls(P);
     static constexpr int LSH = plane_ls(HP);
     static constexpr int WBUF = (NG * LS > NGH * LSH) ? NG * LS : NGH * LSH;
-    static constexpr size_t SMEM = sizeof(float2) * ((size_t)HP * CSS + WBUF + P + HP + 2 * P);
+    static constexpr size_t TMP = (size_t)HP * CSS + WBUF + P + HP + 2 * P;     // P entries: raw transform of the packed column
+    static constexpr size_t SMEM = sizeof(float2) * (TMP + P);
 };
 
 template <int LOG2P> __device__ __forceinline__ void load_plane_twiddles(float2 *tw, float2 *twh, const float2 *gtw, int gtw_n, int tid)
@@ -58,6 +59,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
     float2 *wbuf = cs + HP * C::CSS;
     float2 *tw = wbuf + C::WBUF;
     float2 *twh = tw + P;
+    float2 *tmp = smem + C::TMP;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
@@ -117,16 +119,17 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
         float2 *dst = p.out + pl * (long long)C::XH * P;
         for (int kx = gid; kx < HP; kx += C::NG) {
             const float2 *col = cs + kx * C::CSS;
-            if (kx != 0) {
-                float2 *d = dst + (long long)kx * P;
-                F::template run<PRUNE_IN>(l, m, twp, line,
-                    [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); },
-                    [&](int, int, int idx, float2 v) { d[idx] = v; });
-            } else {
-                F::template run_to_line<PRUNE_IN>(l, m, twp, line,
-                    [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); });
+            // Every column runs the same transform (the group that shares a warp with column 0 must not wait
+            // for a second, different code path): column 0, which packs bins kx = 0 and kx = P/2, only sends
+            // its raw transform to a shared-memory line instead of global memory and unpacks it afterwards.
+            float2 *d = kx != 0 ? dst + (long long)kx * P : tmp;
+            F::template run<PRUNE_IN>(l, m, twp, line,
+                [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); },
+                [&](int, int, int idx, float2 v) { d[idx] = v; });
+            if (kx == 0) {
+                __syncwarp(m);
                 for (int ky = l; ky < P; ky += TPL) {
-                    const float2 c1 = line[F::ph(ky)], c2 = line[F::ph((P - ky) & (P - 1))];
+                    const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
                     dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
                     dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                 }
@@ -174,6 +177,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     float2 *wbuf = cs + HP * C::CSS;
     float2 *tw = wbuf + C::WBUF;
     float2 *twh = tw + P;
+    float2 *tmp = smem + C::TMP;
     const int tid = threadIdx.x;
     const int l = tid % TPL, gid = tid / TPL;
     const int lh = tid % TPLH, gidh = tid / TPLH;
@@ -262,17 +266,17 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
             // columns: P-point transforms over y of the bins kx = 2k + e
             for (int k = gid; k < QP; k += C::NG) {
                 const float2 *col = cs + k * CSH;
-                if (e == 1 || k != 0) {
-                    float2 *d = dst + (long long)(2 * k + e) * P;
-                    F::template run<PRUNE_NONE>(l, m, twp, line,
-                        [&](int, int, int idx) { return col[idx]; },
-                        [&](int, int, int idx, float2 v) { d[idx] = v; });
-                } else {
-                    // column 0 of the even half carries bins kx = 0 and kx = P/2 of every row
-                    F::template run_to_line<PRUNE_NONE>(l, m, twp, line,
-                        [&](int, int, int idx) { return col[idx]; });
+                // one code path for all columns; column 0 of the even half (bins kx = 0 and kx = P/2 of every
+                // row, packed) sends its raw transform to a shared-memory line and is unpacked afterwards
+                const bool packed = e == 0 && k == 0;
+                float2 *d = packed ? tmp : dst + (long long)(2 * k + e) * P;
+                F::template run<PRUNE_NONE>(l, m, twp, line,
+                    [&](int, int, int idx) { return col[idx]; },
+                    [&](int, int, int idx, float2 v) { d[idx] = v; });
+                if (packed) {
+                    __syncwarp(m);
                     for (int ky = l; ky < P; ky += TPL) {
-                        const float2 c1 = line[F::ph(ky)], c2 = line[F::ph((P - ky) & (P - 1))];
+                        const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
                         dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
                         dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                     }
@@ -298,6 +302,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
     float2 *wbuf = cs + HP * C::CSS;
     float2 *tw = wbuf + C::WBUF;
     float2 *twh = tw + P;
+    float2 *tmp = smem + C::TMP;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = FI::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
@@ -323,28 +328,29 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
 #pragma unroll
                 for (int r = 0; r < P0::R; ++r) pre[i][r] = __ldcg(s + i * TPL + r * (P / P0::R));
         };
-        if (gid != 0 && gid < HP) fetch(gid);
+        if (gid < HP) fetch(gid);
+        if (gid == 0) {
+            // column 0 packs bins kx = 0 and kx = P/2: line 0 + i * line P/2, combined as the values arrive; the
+            // transform itself is the same code for every column, so the group sharing this warp is not held up
+            const float2 *sn = src + (long long)HP * P + l;
+#pragma unroll
+            for (int i = 0; i < P0::IPL; ++i)
+#pragma unroll
+                for (int r = 0; r < P0::R; ++r) {
+                    const float2 gn = __ldcg(sn + i * TPL + r * (P / P0::R));
+                    pre[i][r] = make_float2(pre[i][r].x - gn.y, pre[i][r].y + gn.x);
+                }
+        }
         for (int kx = gid; kx < HP; kx += C::NG) {
             float2 *col = cs + kx * C::CSS;
-            if (kx != 0) {
-                FI::template pass<0, PRUNE_NONE>(l, twp,
-                    [&](int i, int r, int) { return pre[i][r]; },
-                    [&](int, int, int idx, float2 v) { line[FI::ph(idx)] = v; });
-                __syncwarp(m);
-                if (kx + C::NG < HP) fetch(kx + C::NG);
-                FI::template pass<1, PRUNE_OUT>(l, twp,
-                    [&](int, int, int idx) { return line[FI::ph(idx)]; },
-                    [&](int, int, int idx, float2 v) { col[idx] = v; });
-            } else {
-                const float2 *sn = src + (long long)HP * P;
-                FI::template run<PRUNE_OUT>(l, m, twp, line,
-                    [&](int, int, int idx) {
-                        const float2 g0 = src[idx], gn = sn[idx];
-                        return make_float2(g0.x - gn.y, g0.y + gn.x);
-                    },
-                    [&](int, int, int idx, float2 v) { col[idx] = v; });
-                if (kx + C::NG < HP) fetch(kx + C::NG);
-            }
+            FI::template pass<0, PRUNE_NONE>(l, twp,
+                [&](int i, int r, int) { return pre[i][r]; },
+                [&](int, int, int idx, float2 v) { line[FI::ph(idx)] = v; });
+            __syncwarp(m);
+            if (kx + C::NG < HP) fetch(kx + C::NG);
+            FI::template pass<1, PRUNE_OUT>(l, twp,
+                [&](int, int, int idx) { return line[FI::ph(idx)]; },
+                [&](int, int, int idx, float2 v) { col[idx] = v; });
             __syncwarp(m);
         }
         __syncthreads();
