@@ -199,8 +199,6 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const long long ib = pl * (long long)Ky * Kx;
         float2 *dst = p.out + pl * (long long)C::XH * P;
-        if (pl + gridDim.x < p.planes)
-            prefetch_l2(hb + (pl + gridDim.x) * (long long)Ky * Kx * sizeof(T), (long long)Ky * Kx * sizeof(T), tid);
         for (int e = 0; e < 2; ++e) {
             // rows: padded row y holds tap row (y + Ly - 1) mod P; two rows per transform
             // the two groups of a half warp take rows 8 apart, so their column-store writes (one
