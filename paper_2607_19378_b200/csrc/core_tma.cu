@@ -127,7 +127,15 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
 #pragma unroll
         for (int b = 0; b < G::NB; ++b) tma_load_3d(tu + b * G::BOXB, &map_u, bar_u, x, b * G::BOXR, (int)o);
     };
-    long long t = blockIdx.x;
+    auto store_tile = [&](long long t) {               // one thread
+        const long long o = t / p.tiles_per_outer;
+        const int x = (int)(t % p.tiles_per_outer) * G::TX * 2;
+#pragma unroll
+        for (int b = 0; b < G::NB; ++b) tma_store_3d(&map_u, to + b * G::BOXB, x, b * G::BOXR, (int)o);
+        tma_commit();
+    };
+    long long t = blockIdx.x, tprev = 0;
+    bool have_prev = false;
     if (tid == 0 && t < tiles) { issue_h(t); issue_u(t); }
     unsigned phase = 0;
     int failed = 0;
@@ -142,8 +150,11 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
                 [&](int, int r, int) { return src[r * RSTEP]; },
                 [&](int, int, int idx, float2 v) { line[F::ph(idx)] = v; });
         }
-        if (__syncthreads_or(failed)) break;           // the filter tile buffer is free again
-        if (tid == 0 && tn < tiles) issue_h(tn);
+        if (__syncthreads_or(failed)) break;           // the filter tile buffer is free again; the previous result tile is complete
+        if (tid == 0) {
+            if (have_prev) store_tile(tprev);          // (its writers fenced before this barrier)
+            if (tn < tiles) issue_h(tn);
+        }
         F::template pass<NP - 1, PRUNE_NONE>(l, tw,
             [&](int, int, int idx) { return line[F::ph(idx)]; },
             [&](int, int r, int, float2 v) { H[r] = make_float2(v.x * p.scale, v.y * p.scale); });
@@ -176,14 +187,14 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
         }
         __syncwarp(m);
         fence_async_smem();                            // generic-proxy writes visible to the copy engine
+        // the tile is sent after the next barrier every thread passes (the first one of the next tile, or the
+        // one after the loop): no barrier of its own
+        tprev = t;
+        have_prev = true;
+    }
+    if (t >= tiles) {
         __syncthreads();
-        if (tid == 0) {
-            const long long o = t / p.tiles_per_outer;
-            const int x = (int)(t % p.tiles_per_outer) * G::TX * 2;
-#pragma unroll
-            for (int b = 0; b < G::NB; ++b) tma_store_3d(&map_u, to + b * G::BOXB, x, b * G::BOXR, (int)o);
-            tma_commit();
-        }
+        if (tid == 0 && have_prev) store_tile(tprev);
     }
     if (t < tiles) {
         // a wait gave up: say so, then give copies that may still be in flight a bounded time to land
