@@ -209,6 +209,39 @@ def test_bounded_wait_runs_out_and_is_reported():
     assert float(torch.ones(8, device="cuda").sum().item()) == 8.0
 
 
+def test_forward_rejects_bad_arguments_and_launches_nothing():
+    """Host-side precondition checks of the forward calls: a misaligned pointer, an output that overlaps an input,
+    a filter stride that is neither 0 nor C*K, a NULL pointer.  Each returns INVALID_ARG and leaves y untouched."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem((15, 14), B=2, C=3, dtype="f32", seed=21)
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    try:
+        dq, dk, dv, dh = (t.cuda() for t in (q, k, v, h))
+        big = torch.full((dq.numel() + 8,), 7.0, device="cuda")
+        y = big[:dq.numel()].view_as(dq)
+        stride = w.C * h[0, 0].numel()
+
+        def rejected(*args):
+            with pytest.raises(hn.HyenaNDError) as ei:
+                hn.hyenand_forward_ex(plan.handle, *args)
+            assert ei.value.code == 1 and hn.hyenand_last_error()
+            torch.cuda.synchronize()
+            assert bool((big == 7.0).all()), "a rejected call wrote to y"
+
+        rejected(dq, dk, dv, dh, stride, big[1:1 + dq.numel()])         # y 4 bytes off a 16-byte boundary
+        rejected(dq, dk, big[4:4 + dq.numel()], dh, stride, y)          # y overlaps v
+        rejected(dq, dk, dv, dh, stride - 1, y)                         # stride neither 0 nor C*K
+        L = hn.lib()
+        assert L.hyenand_forward_ex(plan.handle, dq.data_ptr(), None, dv.data_ptr(), dh.data_ptr(), stride,
+                                    y.data_ptr(), None) == 1
+        # the same plan still runs a valid call afterwards
+        hn.hyenand_forward_ex(plan.handle, dq, dk, dv, dh, stride, y)
+        torch.cuda.synchronize()
+        assert oracle.rel_l2(y.cpu(), oracle.conv_fft(q, k, v, h, "linear")) <= TOL["f32"]
+    finally:
+        plan.close()
+
+
 HOST_CASES = [
     ((512, 512), 2, 8, "f32", False, False),        # generic 2-D, eight groups of two slices
     ((131072,), 4, 64, "bf16", True, True),         # long 1-D, filter shared over the batch
