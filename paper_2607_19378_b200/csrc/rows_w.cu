@@ -67,6 +67,16 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
                 const int mm = (cw + i * TPL + r * (P / F::template Pass<0>::R)) & (P - 1);
                 return make_float2(staged<T>(s, f0, mm), staged<T>(s + SLOT, f1, mm));
             });
+        } else if (p.len == HP && has1) {
+            // full rows: no bounds tests in the input functor
+            F::template run_to_line<PR, true>(l, m, tw, line, [&](int, int, int idx) {
+                float a = staged<T>(s, f0, idx), b = staged<T>(s + SLOT, f1, idx);
+                if (MODE == 0) {
+                    a *= staged<T>(s + 2 * SLOT, fb0, idx);
+                    b *= staged<T>(s + 3 * SLOT, fb1, idx);
+                }
+                return make_float2(a, b);
+            });
         } else {
             F::template run_to_line<PR, true>(l, m, tw, line, [&](int, int, int idx) {
                 float a = 0.f, b = 0.f;
@@ -120,6 +130,11 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
             cp_async16(line + 2 * c, i0 + 2 * c);
             if (has1) cp_async16(line + RS + 2 * c, i1 + 2 * c);
         }
+        if (p.len == HP && has1 && l == 0) {
+            // the two gate rows of the pair (contiguous, a multiple of 16 bytes from a 16-byte boundary)
+            const unsigned long long qa = (unsigned long long)(pq + r0 * HP);
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(qa), "r"((unsigned)(2 * HP * sizeof(T))) : "memory");
+        }
         cp_async_wait_all();
         __syncwarp(m);
         // Legs below half the first-pass radix read bins <= P/2 directly; the others read the mirrored bin
@@ -137,10 +152,26 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
             const float sg = (r == RH && idx == HP) ? 1.f : -1.f;
             return make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
         });
-        for (int n = l; n < p.len; n += TPL) {
-            const float2 z = line[FI::ph(n)];
-            IO<T>::st(py, r0 * p.len + n, z.x * IO<T>::ld(pq, r0 * p.len + n));
-            if (has1) IO<T>::st(py, r1 * p.len + n, z.y * IO<T>::ld(pq, r1 * p.len + n));
+        if (p.len == HP && has1) {
+            // full rows: all gate loads of the pair are in flight together (they were asked into L2 above)
+            float qa[HP / TPL], qb[HP / TPL];
+#pragma unroll
+            for (int t = 0; t < HP / TPL; ++t) {
+                qa[t] = IO<T>::ld(pq, r0 * HP + l + t * TPL);
+                qb[t] = IO<T>::ld(pq, r1 * HP + l + t * TPL);
+            }
+#pragma unroll
+            for (int t = 0; t < HP / TPL; ++t) {
+                const float2 z = line[FI::ph(l + t * TPL)];
+                IO<T>::st(py, r0 * HP + l + t * TPL, z.x * qa[t]);
+                IO<T>::st(py, r1 * HP + l + t * TPL, z.y * qb[t]);
+            }
+        } else {
+            for (int n = l; n < p.len; n += TPL) {
+                const float2 z = line[FI::ph(n)];
+                IO<T>::st(py, r0 * p.len + n, z.x * IO<T>::ld(pq, r0 * p.len + n));
+                if (has1) IO<T>::st(py, r1 * p.len + n, z.y * IO<T>::ld(pq, r1 * p.len + n));
+            }
         }
         __syncwarp(m);
     }
