@@ -14,6 +14,13 @@ namespace hn {
 constexpr int kRowThreads = 256;
 
 // MODE 0: k*v rows (upper half zero), 1: filter rows with wrapped placement, 2: causal filter rows
+// One lane asks the memory system to bring [lo, hi) of an array into L2, trimmed inwards to 16-byte granules.
+__device__ __forceinline__ void prefetch_rows_l2(const unsigned char *lo, const unsigned char *hi)
+{
+    const unsigned long long a0 = ((unsigned long long)lo + 15ull) & ~15ull, a1 = (unsigned long long)hi & ~15ull;
+    if (a1 > a0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(a0), "r"((unsigned)(a1 - a0)) : "memory");
+}
+
 template <typename T, int LOG2P, int MODE>
 __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
 {
@@ -53,6 +60,15 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
             if (has1) stage_row<TPL>(s + 3 * SLOT, h1, rowb, bb, bhi, l);
             fb0 = (int)((unsigned long long)h0 & 15ull);
             fb1 = (int)((unsigned long long)h1 & 15ull);
+        }
+        if (MODE != 1 && l == 0) {
+            // the k and v rows this group takes next travel to L2 while it works on these (measured: a gain for
+            // the short k*v rows, none for the long filter rows)
+            const long long rn = 2 * (rp + (long long)gridDim.x * G);
+            if (rn + 1 < p.rows) {
+                prefetch_rows_l2(ab + rn * rowb, ab + (rn + 2) * rowb);
+                if (MODE == 0) prefetch_rows_l2(bb + rn * rowb, bb + (rn + 2) * rowb);
+            }
         }
         cp_async_wait_all();
         __syncwarp(m);
