@@ -55,6 +55,26 @@ __device__ __forceinline__ void stage_row(unsigned char *dst, const unsigned cha
         }
     }
 }
+// The same copy for rows of at most MAXB bytes: the chunk loop has a compile-time trip count, so every copy is one
+// predicated instruction with constant offsets.
+template <int TPL, int MAXB>
+__device__ __forceinline__ void stage_row_u(unsigned char *dst, const unsigned char *src, int n,
+                                            const unsigned char *lo, const unsigned char *hi, int l)
+{
+    const unsigned char *a = src - ((unsigned long long)src & 15ull);
+    const int nch = (int)((src + n - a + 15) >> 4);
+    if (a >= lo && a + 16 * nch <= hi) {
+        constexpr int MAXCH = (MAXB + 15) / 16 + 1;
+        unsigned char *d = dst + 16 * l;
+        const unsigned char *g = a + 16 * l;
+        const int left = nch - l;
+#pragma unroll
+        for (int t = 0; t < (MAXCH + TPL - 1) / TPL; ++t)
+            if (t * TPL < left) cp_async16(d + 16 * TPL * t, g + 16 * TPL * t);
+        return;
+    }
+    stage_row<TPL>(dst, src, n, lo, hi, l);
+}
 template <typename T> __device__ __forceinline__ float staged(const unsigned char *row, int off, int i)
 {
     if constexpr (sizeof(T) == 4) return *reinterpret_cast<const float *>(row + off + 4 * i);

@@ -51,13 +51,13 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
         const bool has1 = r1 < p.rows;
         unsigned char *s = reinterpret_cast<unsigned char *>(line);
         const unsigned char *g0 = ab + r0 * rowb, *g1 = ab + r1 * rowb;
-        stage_row<TPL>(s, g0, rowb, ab, ahi, l);
-        if (has1) stage_row<TPL>(s + SLOT, g1, rowb, ab, ahi, l);
+        stage_row_u<TPL, ROWMAX>(s, g0, rowb, ab, ahi, l);
+        if (has1) stage_row_u<TPL, ROWMAX>(s + SLOT, g1, rowb, ab, ahi, l);
         int fb0 = 0, fb1 = 0;
         if (MODE == 0) {
             const unsigned char *h0 = bb + r0 * rowb, *h1 = bb + r1 * rowb;
-            stage_row<TPL>(s + 2 * SLOT, h0, rowb, bb, bhi, l);
-            if (has1) stage_row<TPL>(s + 3 * SLOT, h1, rowb, bb, bhi, l);
+            stage_row_u<TPL, ROWMAX>(s + 2 * SLOT, h0, rowb, bb, bhi, l);
+            if (has1) stage_row_u<TPL, ROWMAX>(s + 3 * SLOT, h1, rowb, bb, bhi, l);
             fb0 = (int)((unsigned long long)h0 & 15ull);
             fb1 = (int)((unsigned long long)h1 & 15ull);
         }
