@@ -200,6 +200,45 @@ def test_scaled_named_workloads():
         check(w, q, k, v, h)
 
 
+REPEAT_CASES = [
+    ((40, 48, 72), 1, 3, "bf16", False),     # plane-fused 3-D, TMA core
+    ((200, 300), 2, 2, "f32", False),        # generic 2-D, TMA core
+    ((64, 64), 3, 5, "bf16", False),         # fused 2-D
+    ((65536,), 2, 4, "bf16", True),          # long 1-D
+    ((1000,), 2, 3, "f32", True),            # short 1-D
+]
+
+
+@pytest.mark.parametrize("dims,B,C,dtype,causal", REPEAT_CASES, ids=lambda c: str(c))
+def test_repeated_forwards_are_bit_identical(dims, B, C, dtype, causal):
+    """No kernel accumulates with atomics or depends on scheduling order: the same plan run three times on the same
+    inputs, with another problem run in between on a second plan, returns the same bits each time, and leaves the
+    inputs untouched."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem(dims, B=B, C=C, dtype=dtype, causal=causal, seed=31)
+    w2, t2 = W.random_problem((33, 70), B=1, C=2, dtype=dtype, seed=32)
+    plan = hn.Plan(w.dims, w.B, w.C, causal=w.causal, dtype=w.torch_dtype)
+    other = hn.Plan(w2.dims, w2.B, w2.C, dtype=w2.torch_dtype)
+    try:
+        dq, dk, dv, dh = (t.cuda() for t in (q, k, v, h))
+        d2 = [t.cuda() for t in t2]
+        outs = []
+        for _ in range(3):
+            y = torch.full_like(dq, float("nan"))
+            plan.forward(dq, dk, dv, dh, y)
+            other.forward(*d2, torch.empty_like(d2[0]))
+            torch.cuda.synchronize()
+            outs.append(y.cpu())
+        assert hn.hyenand_plan_device_status(plan.handle) == 0
+        for y in outs[1:]:
+            assert torch.equal(y.view(torch.uint8), outs[0].view(torch.uint8))
+        for d, t in zip((dq, dk, dv, dh), (q, k, v, h)):
+            assert torch.equal(d.cpu().view(torch.uint8), t.view(torch.uint8)), "an input was modified"
+    finally:
+        plan.close()
+        other.close()
+
+
 def test_bounded_wait_runs_out_and_is_reported():
     """The waits of the TMA kernels are bounded polls: a wait on a barrier that nothing ever completes must
     come back and record its code instead of hanging (no fault, no trap: the kernel simply returns)."""
