@@ -5,6 +5,8 @@ CUDA graph, the caller sits inside its allocator's critical section, or all devi
 handed out at start-up).  hyenand_forward_noalloc serves them from a fixed 16 MiB array inside the
 library.  Here it is called through the C ABI twice in a row and compared with the regular
 plan-based entry point on the same inputs, with the tolerances the parity tests use."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -37,6 +39,7 @@ def test_noalloc_matches_plan_based_forward_twice(dims, B, C, dtype, causal, sha
     before = torch.cuda.memory_allocated()
     for attempt in range(2):
         y = torch.full_like(dq, float("nan"))
+        gc.collect()                                            # garbage of earlier tests must not be freed mid-call
         before = torch.cuda.memory_allocated()
         hn.hyenand_forward_noalloc(w.dims, B, C, int(causal), code, dq, dk, dv, dh, stride, y)
         torch.cuda.synchronize()
