@@ -154,15 +154,20 @@ def time_workload(w: W.Workload, steps: int, warmup: int, dist, device, want_ker
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.time()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps - 1)]
     e0.record(stream)
-    for _ in range(steps):
+    for i in range(steps):
         plan.forward(q, k, v, h, y)
+        if i < steps - 1:
+            marks[i].record(stream)               # per-step times for the median and the minimum
     e1.record(stream)
     torch.cuda.synchronize()
     t1 = time.time()
     if dist is not None:
         dist.barrier()
     ms = e0.elapsed_time(e1) / steps
+    seq = [e0] + marks + [e1]
+    per_step = sorted(a.elapsed_time(b) for a, b in zip(seq[:-1], seq[1:]))
     clocks = sampler.stop(t0, t1) if sampler is not None else None
     kernels = []
     if want_kernels:
@@ -174,7 +179,7 @@ def time_workload(w: W.Workload, steps: int, warmup: int, dist, device, want_ker
                                 "ms_per_launch": tot_ms / n, "bytes_per_launch": nbytes / launches,
                                 "flops_per_launch": flops / launches})
         hn.hyenand_plan_set_timing(plan.handle, False)
-    res = {"ms": ms, "clocks": clocks, "kernels": kernels,
+    res = {"ms": ms, "ms_median": per_step[len(per_step) // 2], "ms_min": per_step[0], "clocks": clocks, "kernels": kernels,
            "launches": hn.hyenand_plan_launches(plan.handle, w.h_shared),
            "path": hn.hyenand_plan_path(plan.handle),
            "workspace_bytes": hn.hyenand_plan_workspace_bytes(plan.handle)}
@@ -365,6 +370,7 @@ def main_ours(args):
     out = {
         "metric": METRIC, "value": aggregate_throughput(w.elements, world, ms), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+        "ms_per_step_median": res["ms_median"], "ms_per_step_min": res["ms_min"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "dims": list(w.dims), "B": w.B, "C": w.C, "causal": w.causal,
@@ -460,8 +466,8 @@ def main_reference(args):
 if __name__ == "__main__":
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.WORKLOADS))
     ap.add_argument("--batch", type=int, default=None, help="override B (profiling on a smaller case)")
