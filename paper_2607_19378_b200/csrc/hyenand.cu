@@ -151,7 +151,8 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
         size_t bytes = 0;
         int e = ct1d_init(&p->ct, p->L[2], p->K[2], p->log2p[2], B, C, causal, dtype, &bytes);
         if (e != HYENAND_OK) {
-            fail(e, "long 1-D path: workspace allocation of %zu bytes failed", bytes);
+            fail(e, "long 1-D path: workspace allocation failed (%zu bytes were allocated before): %s", bytes,
+                 cudaGetErrorString(cudaGetLastError()));
             ct1d_free(&p->ct); delete p; return nullptr;
         }
         p->ws_bytes += bytes;
