@@ -20,6 +20,7 @@
 #include "planes.cuh"
 #include "wfft.cuh"
 #include "plane_util.cuh"
+#include "tmem_util.cuh"
 
 namespace hn {
 
@@ -35,7 +36,7 @@ template <int LOG2P> struct PlaneCfg {
     static constexpr int LSH = plane_ls(HP);
     static constexpr int WBUF = (NG * LS > NGH * LSH) ? NG * LS : NGH * LSH;
     static constexpr size_t TMP = (size_t)HP * CSS + WBUF + P + HP + 2 * P;     // P entries: raw transform of the packed column
-    static constexpr size_t SMEM = sizeof(float2) * (TMP + P);
+    static constexpr size_t SMEM = sizeof(float2) * (TMP + P + 2);      // + the slot that receives the tensor-memory base
 };
 
 template <int LOG2P> __device__ __forceinline__ void load_plane_twiddles(float2 *tw, float2 *twh, const float2 *gtw, int gtw_n, int tid)
@@ -163,6 +164,9 @@ __device__ __forceinline__ void separate_rows_odd(const float2 *line, float2 *cs
 // of a row are the half-length transform of f[x] + f[x + P/2], the odd bins that of
 // (f[x] - f[x + P/2]) W_P^x.  Each half (e = 0: even kx, e = 1: odd kx) fills a column store of
 // P/4 columns by P rows, whose columns are then transformed along y and written out as whole lines.
+// The tap rows are fetched and unpacked once per plane: while a thread prepares the even half it also forms its
+// inputs of the odd half, f[x] - f[x + P/2], and parks them in tensor memory (its own lane, 2 * points-per-thread
+// columns per row pair); the odd half reads them back instead of staging the rows again.
 template <typename T, int LOG2P>
 __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
 {
@@ -184,8 +188,20 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     const unsigned m = F::group_mask(tid), mh = FH::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
     float2 *lineh = wbuf + gidh * C::LSH;
+    using PH0 = typename FH::template Pass<0>;
+    constexpr int NPT = 2 * PH0::IPL * PH0::R;               // parked values per thread and row pair
+    constexpr int ROUNDS = HP / C::NGH;                      // row pairs per lane group and half
+    constexpr int TCOLS = 4 * ROUNDS * NPT;                  // four warps share each 32-lane quadrant
+    static_assert(HP % C::NGH == 0 && TCOLS >= 32 && TCOLS <= 512 && (TCOLS & (TCOLS - 1)) == 0, "tensor-memory columns");
+    const int warp = tid >> 5;
+    unsigned *tslot = reinterpret_cast<unsigned *>(smem + C::TMP + P);
+    if (warp == 0) tmem_alloc((unsigned)__cvta_generic_to_shared(tslot), TCOLS);
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
+    tmem_fence_before_sync();
     __syncthreads();
+    tmem_fence_after_sync();
+    const unsigned tbase = *tslot;
+    const unsigned tpark = tmem_addr(tbase, warp, (warp >> 2) * ROUNDS * NPT);
     PlaneTw<LOG2P, false> twp;
     twp.init(l, tw, twh + HP, tid, kPlaneThreads);
     PassTw<LOG2P - 1, false> twr;                            // half-length rows
@@ -203,57 +219,82 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
             // rows: padded row y holds tap row (y + Ly - 1) mod P; two rows per transform
             // the two groups of a half warp take rows 8 apart, so their column-store writes (one
             // row per group, consecutive columns per lane) fall into different banks
-            for (int rp = spread_pair<4>(gidh); rp < HP; rp += C::NGH) {
+            int round = 0;
+            for (int rp = spread_pair<4>(gidh); rp < HP; rp += C::NGH, ++round) {
                 const int y0 = 2 * rp, y1 = y0 + 1;
                 const int my0 = (y0 + Ly - 1) & (P - 1), my1 = (y1 + Ly - 1) & (P - 1);
-                const bool v0 = my0 < Ky, v1 = my1 < Ky;
-                if (v0 || v1) {
-                    // STAGED: both tap rows are fetched with 16-byte copies into the line itself, which
-                    // the first pass reads before anything is written to it; 4-byte taps do not fit the
-                    // half-length line and are read from global memory (L2) directly
-                    constexpr bool STAGED = sizeof(T) == 2;
-                    constexpr int SLOT = ((C::P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;   // bytes kept per staged row
-                    static_assert(!STAGED || 2 * SLOT + 32 <= C::LSH * 8, "staged rows must fit the line");
-                    // the four lines of a warp start 0, 64, 0, 64 bytes into the 128-byte bank row:
-                    // lines 2 and 3 stage 32 bytes further in, so the narrow tap loads do not collide
-                    unsigned char *s0 = reinterpret_cast<unsigned char *>(lineh) + 16 * (gidh & 2), *s1 = s0 + SLOT;
-                    const unsigned char *g0 = hb + (ib + (long long)my0 * Kx) * sizeof(T);
-                    const unsigned char *g1 = hb + (ib + (long long)my1 * Kx) * sizeof(T);
-                    const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
-                    if constexpr (STAGED) {
-                        if (v0) stage_row<TPLH>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
-                        if (v1) stage_row<TPLH>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
-                        cp_async_wait_all();
-                        __syncwarp(mh);
-                        // blank the padding taps (and a missing row) once: the input functors are branch-free
-                        zero_staged<T, TPLH>(s0, f0, v0 ? Kx : 0, P, lh);
-                        zero_staged<T, TPLH>(s1, f1, v1 ? Kx : 0, P, lh);
-                        __syncwarp(mh);
+                const bool v0 = my0 < Ky, v1 = my1 < Ky, valid = v0 || v1;
+                // STAGED: both tap rows are fetched with 16-byte copies into the line itself, which
+                // the first pass reads before anything is written to it; 4-byte taps do not fit the
+                // half-length line and are read from global memory (L2) directly
+                constexpr bool STAGED = sizeof(T) == 2;
+                constexpr int SLOT = ((C::P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;   // bytes kept per staged row
+                static_assert(!STAGED || 2 * SLOT + 32 <= C::LSH * 8, "staged rows must fit the line");
+                // the four lines of a warp start 0, 64, 0, 64 bytes into the 128-byte bank row:
+                // lines 2 and 3 stage 32 bytes further in, so the narrow tap loads do not collide
+                unsigned char *s0 = reinterpret_cast<unsigned char *>(lineh) + 16 * (gidh & 2), *s1 = s0 + SLOT;
+                const unsigned char *g0 = hb + (ib + (long long)my0 * Kx) * sizeof(T);
+                const unsigned char *g1 = hb + (ib + (long long)my1 * Kx) * sizeof(T);
+                const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
+                const int n0 = v0 ? Kx : 0, n1 = v1 ? Kx : 0;
+                auto tap0 = [&](int mx) -> float {
+                    if constexpr (STAGED) return staged<T>(s0, f0, mx);
+                    else return mx < n0 ? IO<T>::ld(reinterpret_cast<const T *>(g0), mx) : 0.f;
+                };
+                auto tap1 = [&](int mx) -> float {
+                    if constexpr (STAGED) return staged<T>(s1, f1, mx);
+                    else return mx < n1 ? IO<T>::ld(reinterpret_cast<const T *>(g1), mx) : 0.f;
+                };
+                float dd[NPT];                                // this thread's inputs of the odd half, before the twiddle
+                const unsigned tcol = tpark + round * NPT;
+                if (e == 0) {
+                    if (valid) {
+                        if constexpr (STAGED) {
+                            if (v0) stage_row<TPLH>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
+                            if (v1) stage_row<TPLH>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
+                            cp_async_wait_all();
+                            __syncwarp(mh);
+                            // blank the padding taps (and a missing row) once: the input functors are branch-free
+                            zero_staged<T, TPLH>(s0, f0, v0 ? Kx : 0, P, lh);
+                            zero_staged<T, TPLH>(s1, f1, v1 ? Kx : 0, P, lh);
+                            __syncwarp(mh);
+                        }
+#pragma unroll
+                        for (int i = 0; i < PH0::IPL; ++i)
+#pragma unroll
+                            for (int r = 0; r < R0; ++r) {
+                                const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
+                                dd[2 * (i * R0 + r)] = tap0(ma) - tap0(mb);
+                                dd[2 * (i * R0 + r) + 1] = tap1(ma) - tap1(mb);
+                            }
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < NPT; ++t) dd[t] = 0.f;
                     }
-                    const int n0 = v0 ? Kx : 0, n1 = v1 ? Kx : 0;
-                    auto tap0 = [&](int mx) -> float {
-                        if constexpr (STAGED) return staged<T>(s0, f0, mx);
-                        else return mx < n0 ? IO<T>::ld(reinterpret_cast<const T *>(g0), mx) : 0.f;
-                    };
-                    auto tap1 = [&](int mx) -> float {
-                        if constexpr (STAGED) return staged<T>(s1, f1, mx);
-                        else return mx < n1 ? IO<T>::ld(reinterpret_cast<const T *>(g1), mx) : 0.f;
-                    };
-                    if (e == 0) {
+                    __syncwarp();                             // the whole warp parks together
+                    TmemIO<NPT>::st(tcol, dd);
+                    tmem_wait_st();
+                    if (valid) {
                         FH::template run_to_line<PRUNE_NONE, STAGED>(lh, mh, twr, lineh, [&](int i, int r, int) {
                             const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
                             return make_float2(tap0(ma) + tap0(mb), tap1(ma) + tap1(mb));
                         });
                         separate_rows<LOG2P - 1, CSH>(lineh, cs, y0, y1, lh);
-                    } else {
-                        FH::template run_to_line<PRUNE_NONE, STAGED>(lh, mh, twr, lineh, [&](int i, int r, int idx) {
-                            const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
-                            return cmul(make_float2(tap0(ma) - tap0(mb), tap1(ma) - tap1(mb)), tw[idx]);
+                        __syncwarp(mh);
+                    }
+                } else {
+                    __syncwarp();
+                    TmemIO<NPT>::ld(dd, tcol);
+                    tmem_wait_ld();
+                    if (valid) {
+                        FH::template run_to_line<PRUNE_NONE, false>(lh, mh, twr, lineh, [&](int i, int r, int idx) {
+                            return cmul(make_float2(dd[2 * (i * R0 + r)], dd[2 * (i * R0 + r) + 1]), tw[idx]);
                         });
                         separate_rows_odd<LOG2P - 1, CSH>(lineh, cs, y0, y1, lh);
+                        __syncwarp(mh);
                     }
-                    __syncwarp(mh);
-                } else {
+                }
+                if (!valid) {
                     for (int k = lh; k < QP; k += TPLH) {
                         cs[k * CSH + y0] = make_float2(0.f, 0.f);
                         cs[k * CSH + y1] = make_float2(0.f, 0.f);
@@ -284,6 +325,10 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
             __syncthreads();
         }
     }
+    // every warp's last tensor-memory read was waited for before the barrier above; the allocating warp frees
+    tmem_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tbase, TCOLS);
 }
 
 
