@@ -246,6 +246,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                     else return mx < n1 ? IO<T>::ld(reinterpret_cast<const T *>(g1), mx) : 0.f;
                 };
                 float dd[NPT];                                // this thread's inputs of the odd half, before the twiddle
+                float ss[NPT];                                // and of the even half
                 const unsigned tcol = tpark + round * NPT;
                 if (e == 0) {
                     if (valid) {
@@ -264,8 +265,11 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
 #pragma unroll
                             for (int r = 0; r < R0; ++r) {
                                 const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
-                                dd[2 * (i * R0 + r)] = tap0(ma) - tap0(mb);
-                                dd[2 * (i * R0 + r) + 1] = tap1(ma) - tap1(mb);
+                                const float a0 = tap0(ma), b0 = tap0(mb), a1 = tap1(ma), b1 = tap1(mb);
+                                ss[2 * (i * R0 + r)] = a0 + b0;
+                                ss[2 * (i * R0 + r) + 1] = a1 + b1;
+                                dd[2 * (i * R0 + r)] = a0 - b0;
+                                dd[2 * (i * R0 + r) + 1] = a1 - b1;
                             }
                     } else {
 #pragma unroll
@@ -275,9 +279,9 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                     TmemIO<NPT>::st(tcol, dd);
                     tmem_wait_st();
                     if (valid) {
-                        FH::template run_to_line<PRUNE_NONE, STAGED>(lh, mh, twr, lineh, [&](int i, int r, int) {
-                            const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
-                            return make_float2(tap0(ma) + tap0(mb), tap1(ma) + tap1(mb));
+                        // (every lane of the group has read its taps from the line before the barrier above)
+                        FH::template run_to_line<PRUNE_NONE, false>(lh, mh, twr, lineh, [&](int i, int r, int) {
+                            return make_float2(ss[2 * (i * R0 + r)], ss[2 * (i * R0 + r) + 1]);
                         });
                         separate_rows<LOG2P - 1, CSH>(lineh, cs, y0, y1, lh);
                         __syncwarp(mh);
