@@ -74,6 +74,31 @@ template <int T, bool INV> __device__ __forceinline__ float2 mul_w16(float2 a)
     }
 }
 
+// W_16^T split as rho * c * (1 + i tau): rho a power of -i (free), c in {1, cos(pi/8), sqrt(1/2)} and
+// tau in {0, +-tan(pi/8), +-1}.  w16_unscaled returns rho (1 + i tau) a (two fused multiply-adds at most); the factor
+// c is left to the butterfly that consumes the value, where it turns an addition into a fused multiply-add.
+#define HN_T8 0.41421356237309504880f   // tan(pi/8)
+template <int T> __host__ __device__ constexpr float w16_scale()
+{
+    constexpr int t = T & 15;
+    return (t % 4 == 0) ? 1.f : (t % 2 == 0 ? HN_SQ2 : HN_C8);
+}
+template <int T, bool INV> __device__ __forceinline__ float2 w16_unscaled(float2 a)
+{
+    constexpr int t = T & 15;
+    // forward factor exp(-2 pi i t / 16): quarter turns q (rho = (-i)^q) and tau
+    constexpr int qf = (t == 0 || t == 1 || t == 2 || t == 15) ? 0 : (t >= 3 && t <= 6) ? 1 : (t >= 7 && t <= 10) ? 2 : 3;
+    constexpr float tf = (t % 4 == 0) ? 0.f : (t % 4 == 2) ? -1.f : (t % 4 == 1) ? -HN_T8 : HN_T8;
+    constexpr int q = INV ? ((4 - qf) & 3) : qf;
+    constexpr float tau = INV ? -tf : tf;
+    float2 v = a;
+    if constexpr (tau != 0.f) v = make_float2(fmaf(-tau, a.y, a.x), fmaf(tau, a.x, a.y));
+    if constexpr (q == 0) return v;
+    else if constexpr (q == 1) return make_float2(v.y, -v.x);
+    else if constexpr (q == 2) return make_float2(-v.x, -v.y);
+    else return make_float2(-v.y, v.x);
+}
+
 // ---- register DFTs, natural order in and out ------------------------------------
 
 template <bool INV, int PR> __device__ __forceinline__ void dft2(float2 &a, float2 &b)
@@ -97,6 +122,25 @@ __device__ __forceinline__ void dft4(float2 &a0, float2 &a1, float2 &a2, float2 
         a0 = cadd(t0, t2);
         a1 = cadd(t1, t3);
         if constexpr (PR != PRUNE_OUT) { a2 = csub(t0, t2); a3 = csub(t1, t3); }
+    }
+}
+
+// 4-point transform of a0, W^T1 a1, W^T2 a2, W^T3 a3 (W = W_16): the scale factors of the twiddles ride on the
+// butterflies' fused multiply-adds.
+template <bool INV, int PR, int T1, int T2, int T3>
+__device__ __forceinline__ void dft4_tw(float2 &a0, float2 &a1, float2 &a2, float2 &a3)
+{
+    constexpr float s1 = w16_scale<T1>(), s2 = w16_scale<T2>(), s3 = w16_scale<T3>(), s31 = s3 / s1;
+    const float2 m1 = w16_unscaled<T1, INV>(a1), m2 = w16_unscaled<T2, INV>(a2), m3 = w16_unscaled<T3, INV>(a3);
+    const float2 t0 = make_float2(fmaf(s2, m2.x, a0.x), fmaf(s2, m2.y, a0.y));
+    const float2 t1 = make_float2(fmaf(-s2, m2.x, a0.x), fmaf(-s2, m2.y, a0.y));
+    const float2 u2 = make_float2(fmaf(s31, m3.x, m1.x), fmaf(s31, m3.y, m1.y));
+    const float2 r3 = rot90<INV>(make_float2(fmaf(-s31, m3.x, m1.x), fmaf(-s31, m3.y, m1.y)));
+    a0 = make_float2(fmaf(s1, u2.x, t0.x), fmaf(s1, u2.y, t0.y));
+    a1 = make_float2(fmaf(s1, r3.x, t1.x), fmaf(s1, r3.y, t1.y));
+    if constexpr (PR != PRUNE_OUT) {
+        a2 = make_float2(fmaf(-s1, u2.x, t0.x), fmaf(-s1, u2.y, t0.y));
+        a3 = make_float2(fmaf(-s1, r3.x, t1.x), fmaf(-s1, r3.y, t1.y));
     }
 }
 
@@ -129,12 +173,13 @@ template <bool INV, int PR> __device__ __forceinline__ void dft16(float2 (&x)[16
         a[n2][0] = x[n2]; a[n2][1] = x[n2 + 4]; a[n2][2] = x[n2 + 8]; a[n2][3] = x[n2 + 12];
         dft4<INV, PIN>(a[n2][0], a[n2][1], a[n2][2], a[n2][3]);
     }
-    a[1][1] = mul_w16<1, INV>(a[1][1]); a[1][2] = mul_w16<2, INV>(a[1][2]); a[1][3] = mul_w16<3, INV>(a[1][3]);
-    a[2][1] = mul_w16<2, INV>(a[2][1]); a[2][2] = mul_w16<4, INV>(a[2][2]); a[2][3] = mul_w16<6, INV>(a[2][3]);
-    a[3][1] = mul_w16<3, INV>(a[3][1]); a[3][2] = mul_w16<6, INV>(a[3][2]); a[3][3] = mul_w16<9, INV>(a[3][3]);
+    // column k1 takes a[n2][k1] W16^(n2*k1), n2 = 1..3
+    dft4<INV, POUT>(a[0][0], a[1][0], a[2][0], a[3][0]);
+    dft4_tw<INV, POUT, 1, 2, 3>(a[0][1], a[1][1], a[2][1], a[3][1]);
+    dft4_tw<INV, POUT, 2, 4, 6>(a[0][2], a[1][2], a[2][2], a[3][2]);
+    dft4_tw<INV, POUT, 3, 6, 9>(a[0][3], a[1][3], a[2][3], a[3][3]);
 #pragma unroll
     for (int k1 = 0; k1 < 4; ++k1) {
-        dft4<INV, POUT>(a[0][k1], a[1][k1], a[2][k1], a[3][k1]);
         x[k1] = a[0][k1]; x[k1 + 4] = a[1][k1];
         if constexpr (PR != PRUNE_OUT) { x[k1 + 8] = a[2][k1]; x[k1 + 12] = a[3][k1]; }
     }
