@@ -12,6 +12,7 @@
 // lower half of every inverse.  PRUNE_IN drops the arithmetic on the zero half
 // in the first pass, PRUNE_OUT skips the unused outputs of the last pass.
 #pragma once
+#include <type_traits>
 #include <cuda_runtime.h>
 
 namespace hn {
@@ -212,6 +213,53 @@ template <int T, bool INV> __device__ __forceinline__ float2 mul_w32(float2 a)
     }
 }
 
+// W_32^T split as rho * c * (1 + i tau) like the W_16 factors above: T = 8 q + r with r in (-4, 4], rho = (-i)^q,
+// c = cos(r pi/16), tau = -tan(r pi/16) (forward sign; conjugate for INV).
+template <int T> __host__ __device__ constexpr int w32_res() { return (((T & 31) + 3) & 7) - 3; }
+template <int T> __host__ __device__ constexpr float w32_scale() { return w32_cos(w32_res<T>()); }
+template <int T, bool INV> __device__ __forceinline__ float2 w32_unscaled(float2 a)
+{
+    constexpr int r = w32_res<T>();
+    constexpr int qf = ((((T & 31) - r) / 8) & 3);
+    constexpr float tf = r == 0 ? 0.f : r == 4 ? -1.f : -w32_sin(r) / w32_cos(r);
+    constexpr int q = INV ? ((4 - qf) & 3) : qf;
+    constexpr float tau = INV ? -tf : tf;
+    float2 v = a;
+    if constexpr (tau != 0.f) v = make_float2(fmaf(-tau, a.y, a.x), fmaf(tau, a.x, a.y));
+    if constexpr (q == 0) return v;
+    else if constexpr (q == 1) return make_float2(v.y, -v.x);
+    else if constexpr (q == 2) return make_float2(-v.x, -v.y);
+    else return make_float2(-v.y, v.x);
+}
+
+__device__ __forceinline__ float2 fma2(float s, float2 a, float2 b) { return make_float2(fmaf(s, a.x, b.x), fmaf(s, a.y, b.y)); }
+
+// 8-point transform of c[n] W_32^(n K1), n = 0..7: every scale factor (of the outer twiddles and of the two
+// sqrt(1/2) twiddles inside) rides on a fused multiply-add of the butterflies.
+template <bool INV, int PR, int K1> __device__ __forceinline__ void dft8_tw(float2 (&c)[8])
+{
+    constexpr float s1 = w32_scale<K1>(), s2 = w32_scale<2 * K1>(), s3 = w32_scale<3 * K1>(), s4 = w32_scale<4 * K1>(),
+                    s5 = w32_scale<5 * K1>(), s6 = w32_scale<6 * K1>(), s7 = w32_scale<7 * K1>();
+    const float2 m0 = c[0];
+    const float2 m1 = w32_unscaled<K1, INV>(c[1]), m2 = w32_unscaled<2 * K1, INV>(c[2]), m3 = w32_unscaled<3 * K1, INV>(c[3]),
+                 m4 = w32_unscaled<4 * K1, INV>(c[4]), m5 = w32_unscaled<5 * K1, INV>(c[5]), m6 = w32_unscaled<6 * K1, INV>(c[6]),
+                 m7 = w32_unscaled<7 * K1, INV>(c[7]);
+    // evens: true values
+    const float2 t0 = fma2(s4, m4, m0), t1 = fma2(-s4, m4, m0);
+    const float2 u2 = fma2(s6 / s2, m6, m2), r3 = rot90<INV>(fma2(-s6 / s2, m6, m2));
+    const float2 e0 = fma2(s2, u2, t0), e1 = fma2(s2, r3, t1), e2 = fma2(-s2, u2, t0), e3 = fma2(-s2, r3, t1);
+    // odds: values divided by s1
+    const float2 v0 = fma2(s5 / s1, m5, m1), v1 = fma2(-s5 / s1, m5, m1);
+    const float2 w2 = fma2(s7 / s3, m7, m3), w3 = rot90<INV>(fma2(-s7 / s3, m7, m3));
+    const float2 o0 = fma2(s3 / s1, w2, v0), o1 = fma2(s3 / s1, w3, v1), o2 = fma2(-s3 / s1, w2, v0), o3 = fma2(-s3 / s1, w3, v1);
+    const float2 p1 = w16_unscaled<2, INV>(o1), p2 = w16_unscaled<4, INV>(o2), p3 = w16_unscaled<6, INV>(o3);
+    constexpr float sq = s1 * HN_SQ2;
+    c[0] = fma2(s1, o0, e0); c[1] = fma2(sq, p1, e1); c[2] = fma2(s1, p2, e2); c[3] = fma2(sq, p3, e3);
+    if constexpr (PR != PRUNE_OUT) {
+        c[4] = fma2(-s1, o0, e0); c[5] = fma2(-sq, p1, e1); c[6] = fma2(-s1, p2, e2); c[7] = fma2(-sq, p3, e3);
+    }
+}
+
 template <int N2, bool INV> __device__ __forceinline__ void tw32_row(float2 (&a)[4])
 {
     a[1] = mul_w32<N2, INV>(a[1]); a[2] = mul_w32<2 * N2, INV>(a[2]); a[3] = mul_w32<3 * N2, INV>(a[3]);
@@ -229,17 +277,17 @@ template <bool INV, int PR> __device__ __forceinline__ void dft32(float2 (&x)[32
         a[n2][0] = x[n2]; a[n2][1] = x[n2 + 8]; a[n2][2] = x[n2 + 16]; a[n2][3] = x[n2 + 24];
         dft4<INV, PIN>(a[n2][0], a[n2][1], a[n2][2], a[n2][3]);
     }
-    tw32_row<1, INV>(a[1]); tw32_row<2, INV>(a[2]); tw32_row<3, INV>(a[3]); tw32_row<4, INV>(a[4]);
-    tw32_row<5, INV>(a[5]); tw32_row<6, INV>(a[6]); tw32_row<7, INV>(a[7]);
-#pragma unroll
-    for (int k1 = 0; k1 < 4; ++k1) {
+    auto column = [&](auto k1c) {
+        constexpr int k1 = decltype(k1c)::value;
         float2 c[8];
 #pragma unroll
         for (int n2 = 0; n2 < 8; ++n2) c[n2] = a[n2][k1];
-        dft8<INV, POUT>(c);
+        dft8_tw<INV, POUT, k1>(c);                  // the twiddles W32^(n2*k1) are applied inside
 #pragma unroll
         for (int k2 = 0; k2 < (PR == PRUNE_OUT ? 4 : 8); ++k2) x[k1 + 4 * k2] = c[k2];
-    }
+    };
+    column(std::integral_constant<int, 0>{}); column(std::integral_constant<int, 1>{});
+    column(std::integral_constant<int, 2>{}); column(std::integral_constant<int, 3>{});
 }
 
 template <int R, bool INV, int PR> __device__ __forceinline__ void dft(float2 (&x)[R])
