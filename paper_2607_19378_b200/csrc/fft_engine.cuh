@@ -100,6 +100,8 @@ template <int T, bool INV> __device__ __forceinline__ float2 w16_unscaled(float2
     else return make_float2(-v.y, v.x);
 }
 
+__device__ __forceinline__ float2 fma2(float s, float2 a, float2 b) { return make_float2(fmaf(s, a.x, b.x), fmaf(s, a.y, b.y)); }
+
 // ---- register DFTs, natural order in and out ------------------------------------
 
 template <bool INV, int PR> __device__ __forceinline__ void dft2(float2 &a, float2 &b)
@@ -153,12 +155,13 @@ template <bool INV, int PR> __device__ __forceinline__ void dft8(float2 (&x)[8])
     float2 o0 = x[1], o1 = x[3], o2 = x[5], o3 = x[7];
     dft4<INV, P4>(e0, e1, e2, e3);
     dft4<INV, P4>(o0, o1, o2, o3);
-    o1 = mul_w16<2, INV>(o1);
+    // W8^1 and W8^3 without their factor sqrt(1/2), which rides on the last additions
+    o1 = w16_unscaled<2, INV>(o1);
     o2 = mul_w16<4, INV>(o2);
-    o3 = mul_w16<6, INV>(o3);
-    x[0] = cadd(e0, o0); x[1] = cadd(e1, o1); x[2] = cadd(e2, o2); x[3] = cadd(e3, o3);
+    o3 = w16_unscaled<6, INV>(o3);
+    x[0] = cadd(e0, o0); x[1] = fma2(HN_SQ2, o1, e1); x[2] = cadd(e2, o2); x[3] = fma2(HN_SQ2, o3, e3);
     if constexpr (PR != PRUNE_OUT) {
-        x[4] = csub(e0, o0); x[5] = csub(e1, o1); x[6] = csub(e2, o2); x[7] = csub(e3, o3);
+        x[4] = csub(e0, o0); x[5] = fma2(-HN_SQ2, o1, e1); x[6] = csub(e2, o2); x[7] = fma2(-HN_SQ2, o3, e3);
     }
 }
 
@@ -231,8 +234,6 @@ template <int T, bool INV> __device__ __forceinline__ float2 w32_unscaled(float2
     else if constexpr (q == 2) return make_float2(-v.x, -v.y);
     else return make_float2(-v.y, v.x);
 }
-
-__device__ __forceinline__ float2 fma2(float s, float2 a, float2 b) { return make_float2(fmaf(s, a.x, b.x), fmaf(s, a.y, b.y)); }
 
 // 8-point transform of c[n] W_32^(n K1), n = 0..7: every scale factor (of the outer twiddles and of the two
 // sqrt(1/2) twiddles inside) rides on a fused multiply-add of the butterflies.
