@@ -10,7 +10,8 @@
 //   hplane     filter plane, which has twice the rows and columns: the even and the odd
 //              bins along x are produced one after the other (one radix-2
 //              decimation-in-frequency step applied to the taps as they are read), each
-//              half filling a column store of the size of a k*v plane's.
+//              half filling a column store of the size of a k*v plane's.  The tap rows are
+//              fetched once: the odd half's inputs wait in tensor memory meanwhile.
 //   plane_inv  inverse along y (keeping the cropped rows), inverse complex-to-real
 //              along x, crop, output gate q, store.
 //
