@@ -139,16 +139,12 @@ def time_workload(w: W.Workload, steps: int, warmup: int, dist, device, want_ker
     for _ in range(max(warmup, 3)):
         plan.forward(q, k, v, h, y)
     torch.cuda.synchronize()
-    if want_kernels:
-        hn.hyenand_plan_set_timing(plan.handle, True)
     sampler = ClockSampler(sampler_device) if sampler_device is not None else None
     if sampler is not None:
         time.sleep(0.6)                       # let nvidia-smi start sampling
         for _ in range(3):                    # re-warm after the pause
             plan.forward(q, k, v, h, y)
         torch.cuda.synchronize()
-        if want_kernels:
-            hn.hyenand_plan_set_timing(plan.handle, True)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
@@ -168,8 +164,17 @@ def time_workload(w: W.Workload, steps: int, warmup: int, dist, device, want_ker
     ms = e0.elapsed_time(e1) / steps
     seq = [e0] + marks + [e1]
     per_step = sorted(a.elapsed_time(b) for a, b in zip(seq[:-1], seq[1:]))
-    clocks = sampler.stop(t0, t1) if sampler is not None else None
     kernels = []
+    if want_kernels:
+        # Per-kernel durations: the same K forwards once more, every launch bracketed by CUDA events on its
+        # stream; a plan with several lanes enqueues its groups one after the other meanwhile (mode 2), so a
+        # kernel's duration is not stretched by another lane's kernels sharing the GPU.
+        hn.hyenand_plan_set_timing(plan.handle, 2)
+        for i in range(steps):
+            plan.forward(q, k, v, h, y)
+        torch.cuda.synchronize()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
     if want_kernels:
         for kid in range(hn.hyenand_plan_kernel_count(plan.handle)):
             name, launches, nbytes, flops = hn.hyenand_plan_kernel_info(plan.handle, kid, w.h_shared)
@@ -179,7 +184,14 @@ def time_workload(w: W.Workload, steps: int, warmup: int, dist, device, want_ker
                                 "ms_per_launch": tot_ms / n, "bytes_per_launch": nbytes / launches,
                                 "flops_per_launch": flops / launches})
         hn.hyenand_plan_set_timing(plan.handle, False)
+    status = hn.hyenand_plan_device_status(plan.handle)
+    damage = hn.hyenand_plan_guard_damage(plan.handle)
+    if status != 0 or damage != 0:
+        raise SystemExit(f"{w.name}: device status {status} (a bounded wait gave up) / {damage} damaged guard bytes: "
+                         "the timing is void")
+    group, lanes = hn.hyenand_plan_groups(plan.handle)
     res = {"ms": ms, "ms_median": per_step[len(per_step) // 2], "ms_min": per_step[0], "clocks": clocks, "kernels": kernels,
+           "device_status": status, "guard_damage": damage, "slices_per_group": group, "lanes": lanes,
            "launches": hn.hyenand_plan_launches(plan.handle, w.h_shared),
            "path": hn.hyenand_plan_path(plan.handle),
            "workspace_bytes": hn.hyenand_plan_workspace_bytes(plan.handle)}
@@ -329,8 +341,35 @@ def aggregate_throughput(elements_per_rank: int, world: int, ms: float) -> float
     return elements_per_rank * world / (ms * 1e-3) / 1e9
 
 
+def spawn_command(args, port: int):
+    """argv that runs this benchmark as args.gpus ranks on this node (one process per GPU)."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__),
+           "--gpus", str(args.gpus), "--steps", str(args.steps), "--warmup", str(args.warmup),
+           "--workload", args.workload, "--impl", args.impl]
+    if args.batch is not None:
+        cmd += ["--batch", str(args.batch)]
+    if args.channels is not None:
+        cmd += ["--channels", str(args.channels)]
+    for flag, on in (("--no-all", args.no_all), ("--no-cpu", args.no_cpu), ("--no-cufft", args.no_cufft)):
+        if on:
+            cmd.append(flag)
+    return cmd
+
+
 def main_ours(args):
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # called without a launcher: start the ranks ourselves
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} but only {torch.cuda.device_count()} CUDA device(s) are visible")
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        raise SystemExit(subprocess.call(spawn_command(args, port)))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} does not match WORLD_SIZE={world}")
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
@@ -376,7 +415,10 @@ def main_ours(args):
         "config": {"workload": w.name, "dims": list(w.dims), "B": w.B, "C": w.C, "causal": w.causal,
                    "h_shared_over_batch": w.h_shared, "padded_points_per_slice": P,
                    "l2": "inputs larger than L2 (no flush needed)" if nbytes > 126e6 else "fits L2; latency-bound",
-                   "path": res["path"], "per_gpu_batch": "fixed (each rank runs the full workload)"},
+                   "path": res["path"], "slices_per_group": res["slices_per_group"], "lanes": res["lanes"],
+                   "per_gpu_batch": "fixed (each rank runs the full workload)"},
+        "device_status": res["device_status"], "guard_damage": res["guard_damage"],
+        "kernel_timing": "CUDA events around every launch in a second pass of the same K forwards, lanes serialised",
         "clocks": res["clocks"],
         "e2e": {"value": aggregate_throughput(w.elements, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

@@ -64,13 +64,13 @@ enum {
  * tables on the current device (this call may synchronise).  Returns NULL on
  * failure, reason in hyenand_last_error().
  * Limits: for ndim >= 2 each padded axis P_n <= 8192; for ndim == 1,
- * P_1 <= 2^26.
+ * P_1 <= 2^24 (L_1 <= 8388608; the parity tests run up to that length).
  */
 hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype);
 
 /*
- * One forward pass, one kernel per (b,c) as in Section 3.2.2 ("B different
- * convolutional kernels, one for each of the inputs in a batch").
+ * One forward pass with one filter per (b,c): the input-dependent kernels of
+ * Section 3.2.2, one per sample of the batch and per channel.
  * q, k, v, h, y: DEVICE pointers, 16-byte aligned, y must not alias an input.
  * cuda_stream: a cudaStream_t (NULL = the legacy default stream).
  */
@@ -121,6 +121,13 @@ int hyenand_last_error_code(void);
  * no counterpart; it exists so that a failed copy is observable from the host. */
 int hyenand_plan_device_status(hyenand_plan *plan);
 
+/* Guard bands.  Every device allocation of a plan (workspace sets, twiddle tables, status word) sits between two
+ * bands of 4096 bytes filled with a fixed byte when the plan is created.  Returns how many of those bytes no
+ * longer hold it, i.e. 0 unless a kernel wrote outside the plan's workspace; -1 on error.  Blocking (copies the
+ * bands to the host): call it after synchronising the stream.  The paper has no counterpart; it stands in for a
+ * memory checker on machines where none can be run. */
+long long hyenand_plan_guard_damage(hyenand_plan *plan);
+
 /* Self-test of the mechanism behind hyenand_plan_device_status: launches one small CTA that waits, for at
  * most `polls` polls (clamped to [1, 65536]), on a barrier that nothing ever completes.  The wait must run out
  * and the kernel must report it: returns 9 (the code that kernel records), 0 if the wait wrongly succeeded,
@@ -132,6 +139,9 @@ size_t hyenand_plan_workspace_bytes(const hyenand_plan *plan);        /* device 
 int hyenand_plan_fft_dims(const hyenand_plan *plan, int *out_P);      /* writes ndim padded sizes P_n */
 int hyenand_plan_launches(const hyenand_plan *plan, int h_shared);    /* kernels enqueued by one forward */
 const char *hyenand_plan_path(const hyenand_plan *plan);              /* name of the kernel path chosen */
+/* How the batch is scheduled: slices per group and the number of lanes (workspace sets with a stream each; 1 =
+ * everything on the caller's stream).  Either pointer may be NULL. */
+int hyenand_plan_groups(const hyenand_plan *plan, long long *slices_per_group, int *lanes);
 
 
 /*
@@ -143,14 +153,16 @@ const char *hyenand_plan_path(const hyenand_plan *plan);              /* name of
  * geometry is passed with every call, and the workspace (twiddle table and half spectra, the same
  * passes as the general N-D path) lives in a fixed array of hyenand_noalloc_max_bytes() bytes
  * (16 MiB) inside the library image, which every GPU that loads the library holds until the
- * process exits.  Arguments as hyenand_create_plan + hyenand_forward_ex; q, k, v, h, y are DEVICE
- * pointers owned by the caller.  Work is enqueued on cuda_stream; the call does not synchronise.
+ * process exits.  Arguments and checks as hyenand_create_plan + hyenand_forward_ex (y must not overlap an
+ * input); q, k, v, h, y are DEVICE pointers owned by the caller.  Work is enqueued on cuda_stream; the call
+ * does not synchronise.
  *
  * Limits: every dims[n] <= 4096; one (b,c) slice's spectra (plus, when the filter is shared over
  * the batch, all C filter spectra) must fit the array, else HYENAND_ERR_UNSUPPORTED with the
  * sizes in hyenand_last_error().  Larger batches are processed in as many passes as needed.
- * The first call on a device resolves the array's device address (cudaGetSymbolAddress) and
- * should therefore come before any stream capture.  All calls share the one array, which keeps
+ * The first call on a device resolves the array's device address (cudaGetSymbolAddress), and the
+ * first call for a new geometry or dtype loads the kernels it needs and sets their attributes: make one
+ * warm-up call per geometry and dtype before any stream capture.  All calls share the one array, which keeps
  * the previous call's contents (nothing in it needs to start at zero): calls that overlap on
  * the GPU (different streams, or different host threads) race and give wrong results; calls
  * on one stream are safe.  Neither cudaMalloc, cudaFree nor any allocating library routine is
@@ -172,7 +184,10 @@ int hyenand_forward_noalloc(int ndim, const int *dims, int B, int C, int causal,
  * spectra.  A kernel this plan never launches reports zeros.
  * hyenand_plan_set_timing(plan, 1) makes every later forward bracket each
  * kernel launch with CUDA events on the launching stream (and clears the
- * totals); hyenand_plan_kernel_time returns the accumulated device time and
+ * totals); with 2 instead of 1 the groups of a plan with several lanes are
+ * additionally enqueued one after the other on the caller's stream, so that a
+ * kernel's duration is its own and not stretched by another lane's kernels
+ * sharing the GPU; 0 switches timing off. hyenand_plan_kernel_time returns the accumulated device time and
  * launch count of one kernel and must only be called after the stream has
  * been synchronised.  At most 4096 launches are recorded between two calls of
  * hyenand_plan_kernel_time.

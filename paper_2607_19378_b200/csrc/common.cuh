@@ -90,6 +90,29 @@ struct DevOnce {
     }
 };
 
+// Development switches (environment variables HYENAND_FORCE_GENERIC, HYENAND_GENERIC_ROWS, HYENAND_GENERIC_CORE,
+// HYENAND_NO_TMA select the older kernel variants for A/B runs and tests).  They are read once, when a plan is
+// created, and travel with the plan: a forward call never looks at the environment.
+struct Switches {
+    bool force_generic, generic_rows, generic_core, no_tma;
+};
+Switches read_switches();
+
+// Device allocations of a plan, each between two guard bands of kGuardBytes filled with a fixed byte.  A kernel
+// that writes outside its workspace damages a band; guard_damage() counts the damaged bytes (blocking copies
+// of the bands to the host).  This stands in for a memory checker on machines where none can run.
+constexpr size_t kGuardBytes = 4096;
+constexpr int kMaxGuarded = 24;
+struct GuardedAllocs {
+    struct Rec { unsigned char *base; size_t bytes; };
+    Rec recs[kMaxGuarded];
+    int n = 0;
+};
+// cudaMalloc of bytes + two bands; *ptr is the first usable byte (256-byte aligned).  cudaSuccess or the error.
+cudaError_t guarded_alloc(GuardedAllocs *g, void **ptr, size_t bytes);
+void guarded_free_all(GuardedAllocs *g);
+long long guard_damage(const GuardedAllocs *g);       // damaged guard bytes, -1 if a copy failed
+
 constexpr int kMaxLineLog2 = 13;          // longest line transformed in shared memory: 8192 points
 constexpr int kThreads = 256;             // threads per CTA of the generic kernels
 

@@ -346,7 +346,7 @@ static int launch_cols_inv(const ColsInvArgs &a, int log2p1, int dtype, cudaStre
     return n;
 }
 
-static float2 *upload_table(int n, double denom, double mult, size_t *bytes)
+static float2 *upload_table(GuardedAllocs *g, int n, double denom, double mult, size_t *bytes)
 {
     std::vector<float2> t(n);
     for (int i = 0; i < n; ++i) {
@@ -354,16 +354,18 @@ static float2 *upload_table(int n, double denom, double mult, size_t *bytes)
         t[i] = make_float2((float)cos(ang), (float)sin(ang));
     }
     float2 *d = nullptr;
-    if (cudaMalloc(&d, sizeof(float2) * n) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (guarded_alloc(g, (void **)&d, sizeof(float2) * n) != cudaSuccess) { cudaGetLastError(); return nullptr; }
     if (cudaMemcpy(d, t.data(), sizeof(float2) * n, cudaMemcpyHostToDevice) != cudaSuccess) {
-        cudaGetLastError(); cudaFree(d); return nullptr;
+        cudaGetLastError(); return nullptr;          // the allocation stays on the plan's list and is freed with it
     }
     *bytes += sizeof(float2) * n;
     return d;
 }
 
-int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, int dtype, size_t *bytes)
+int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, int dtype, const Switches &sw,
+              GuardedAllocs *g, size_t *bytes)
 {
+    c->sw = sw;
     c->L = L; c->K = K; c->log2p = log2p; c->B = B; c->C = C; c->causal = causal; c->dtype = dtype;
     c->log2p1 = log2p / 2;
     c->log2p2 = log2p - c->log2p1;
@@ -377,25 +379,18 @@ int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, in
     c->wh_slices = spc > C ? spc : C;
     *bytes = 0;
     c->lo = log2p / 2;
-    c->tw1 = upload_table(P1, (double)P1, 1.0, bytes);
-    c->tw2 = upload_table(P2, (double)P2, 1.0, bytes);
-    c->twp_fine = upload_table(1 << c->lo, ldexp(1.0, log2p), 1.0, bytes);
-    c->twp_coarse = upload_table(1 << (log2p - c->lo), ldexp(1.0, log2p), ldexp(1.0, c->lo), bytes);
+    c->tw1 = upload_table(g, P1, (double)P1, 1.0, bytes);
+    c->tw2 = upload_table(g, P2, (double)P2, 1.0, bytes);
+    c->twp_fine = upload_table(g, 1 << c->lo, ldexp(1.0, log2p), 1.0, bytes);
+    c->twp_coarse = upload_table(g, 1 << (log2p - c->lo), ldexp(1.0, log2p), ldexp(1.0, c->lo), bytes);
     if (!c->tw1 || !c->tw2 || !c->twp_fine || !c->twp_coarse) return 3;
     size_t need = sizeof(float2) * per_slice * spc;
-    if (cudaMalloc(&c->wu, need) != cudaSuccess) { cudaGetLastError(); *bytes = need; return 3; }
+    if (guarded_alloc(g, (void **)&c->wu, need) != cudaSuccess) { cudaGetLastError(); *bytes = need; return 3; }
     *bytes += need;
     need = sizeof(float2) * per_slice * c->wh_slices;
-    if (cudaMalloc(&c->wh, need) != cudaSuccess) { cudaGetLastError(); *bytes = need; return 3; }
+    if (guarded_alloc(g, (void **)&c->wh, need) != cudaSuccess) { cudaGetLastError(); *bytes = need; return 3; }
     *bytes += need;
     return 0;
-}
-
-void ct1d_free(Ct1dPlan *c)
-{
-    cudaFree(c->wu); cudaFree(c->wh); cudaFree(c->tw1); cudaFree(c->tw2);
-    cudaFree(c->twp_fine); cudaFree(c->twp_coarse);
-    c->wu = c->wh = c->tw1 = c->tw2 = c->twp_fine = c->twp_coarse = nullptr;
 }
 
 static int filter_pass(Ct1dPlan *c, const char *h, long long n, cudaStream_t st, int *launches, Prof *prof)
@@ -469,7 +464,7 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
 
 bool ct1d_uses_w(const Ct1dPlan *c)
 {
-    return ct1d_w_supported(c->log2p1, c->log2p2, c->L, c->K, c->causal, c->dtype) && !getenv("HYENAND_FORCE_GENERIC");
+    return ct1d_w_supported(c->log2p1, c->log2p2, c->L, c->K, c->causal, c->dtype) && !c->sw.force_generic;
 }
 
 int ct1d_launches(const Ct1dPlan *c, bool shared)

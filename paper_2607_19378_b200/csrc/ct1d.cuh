@@ -18,12 +18,14 @@ struct Ct1dPlan {
     float2 *twp_coarse, *twp_fine;   // W_P^j = coarse[j >> lo] * fine[j & (2^lo - 1)]
     int lo;
     int *status;              // device word set when a bounded wait on a tensor copy gives up (owned by the plan)
+    Switches sw;              // development switches, read when the plan was created
     long long slices_per_chunk, wh_slices;
     long long r0, r1;         // slices [r0, r1) the next forward works on
 };
 
-int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, int dtype, size_t *bytes);
-void ct1d_free(Ct1dPlan *c);
+// allocations go on the plan's guarded list `g` and are freed with it
+int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, int dtype, const Switches &sw,
+              GuardedAllocs *g, size_t *bytes);
 int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const void *h, bool shared,
                  void *y, cudaStream_t st, int *launches, Prof *prof);
 int ct1d_launches(const Ct1dPlan *c, bool shared);

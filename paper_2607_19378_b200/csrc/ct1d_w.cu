@@ -67,6 +67,7 @@ struct ColsFwdWArgs {
     int log2p2;
     const float2 *tw1;        // P1-point table
     TwoLevelW twp;
+    bool no_tma;              // development switch: per-thread copies even where tensor copies apply
 };
 
 // TMA = true: the tile (all rows t1 of TX column pairs, for k and for v) arrives as tensor copies into
@@ -393,6 +394,7 @@ struct ColsInvWArgs {
     int log2p2;
     const float2 *tw1;
     int *status;              // device word set when a bounded wait on a tensor copy gives up (may be NULL)
+    bool no_tma;              // development switch: per-thread copies even where tensor copies apply
 };
 
 // TMA = true: the gate tile q arrives, and the result tile y leaves, as tensor copies ([t1][pair] rows of
@@ -587,8 +589,7 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
     memset(&mb, 0, sizeof(mb));
     memset(&mo, 0, sizeof(mo));
     constexpr unsigned TROW = TX * 2 * sizeof(T);
-    bool tma = (TROW == 64 || TROW == 128) && a.len % P2 == 0 && a.slices < (1ll << 31) && tma_available() &&
-               !getenv("HYENAND_NO_TMA");
+    bool tma = (TROW == 64 || TROW == 128) && a.len % P2 == 0 && a.slices < (1ll << 31) && tma_available() && !a.no_tma;
     if (tma) {
         constexpr int HP1 = P1 / 2;
         const unsigned long long dims[3] = {(unsigned long long)P2, (unsigned long long)(a.len / P2), (unsigned long long)a.slices};
@@ -639,7 +640,7 @@ template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWA
     memset(&mq, 0, sizeof(mq));
     memset(&my, 0, sizeof(my));
     // tensor copies need the slice to be a whole number of rows of P2 elements
-    bool tma = a.len % P2 == 0 && a.slices < (1ll << 31) && QROW % 16 == 0 && tma_available() && !getenv("HYENAND_NO_TMA");
+    bool tma = a.len % P2 == 0 && a.slices < (1ll << 31) && QROW % 16 == 0 && tma_available() && !a.no_tma;
     if (tma) {
         const unsigned long long dims[3] = {(unsigned long long)P2, (unsigned long long)(a.len / P2), (unsigned long long)a.slices};
         const unsigned long long strides[2] = {(unsigned long long)P2 * sizeof(T), (unsigned long long)a.len * sizeof(T)};
@@ -691,7 +692,7 @@ int ct1d_w_filter(Ct1dPlan *c, const void *h, long long n, bool staged_ok, cudaS
     const TwoLevelW twp{c->twp_coarse, c->twp_fine, c->lo};
     if (staged_ok) {
         ColsFwdWArgs a{};
-        a.a = h; a.b = nullptr; a.out = c->wh; a.slices = n; a.in_slice = c->K; a.len = c->K; a.status = c->status;
+        a.a = h; a.b = nullptr; a.out = c->wh; a.slices = n; a.in_slice = c->K; a.len = c->K; a.status = c->status; a.no_tma = c->sw.no_tma;
         a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.twp = twp;
         prof->begin(KID_CT_COLS_H, st);
         int r = 0;
@@ -721,7 +722,7 @@ int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long l
 {
     const TwoLevelW twp{c->twp_coarse, c->twp_fine, c->lo};
     ColsFwdWArgs a{};
-    a.a = k; a.b = v; a.out = c->wu; a.slices = n; a.in_slice = c->L; a.len = c->L; a.status = c->status;
+    a.a = k; a.b = v; a.out = c->wu; a.slices = n; a.in_slice = c->L; a.len = c->L; a.status = c->status; a.no_tma = c->sw.no_tma;
     a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.twp = twp;
     prof->begin(KID_CT_COLS_U, st);
     int r = 0;
@@ -743,7 +744,7 @@ int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long l
     if (r < 0) return -1;
     *launches += r;
     ColsInvWArgs ci{};
-    ci.in = c->wu; ci.q = q; ci.y = y; ci.slices = n; ci.len = c->L; ci.log2p2 = c->log2p2; ci.tw1 = c->tw1; ci.status = c->status;
+    ci.in = c->wu; ci.q = q; ci.y = y; ci.slices = n; ci.len = c->L; ci.log2p2 = c->log2p2; ci.tw1 = c->tw1; ci.status = c->status; ci.no_tma = c->sw.no_tma;
     prof->begin(KID_CT_COLS_INV, st);
 #define CALLF(L) r = launch_cols_inv_w_t<float, L>(ci, st)
 #define CALLB(L) r = launch_cols_inv_w_t<bf16, L>(ci, st)

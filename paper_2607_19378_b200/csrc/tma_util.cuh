@@ -7,7 +7,10 @@
 
 namespace hn {
 
-constexpr int kWaitLimit = 1 << 22;                  // polls of a barrier before giving up
+// A wait on a barrier gives up after kWaitLimitNs of device time (read from the global nanosecond timer every
+// 256 polls) or after kWaitLimit polls, whichever comes first.  A tile copy completes in microseconds.
+constexpr int kWaitLimit = 1 << 22;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;      // one second
 
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t *b, unsigned count)
@@ -25,11 +28,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *b, unsigned parity)
                  : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
     return ok != 0;
 }
-// bounded wait; false if the phase did not complete within `limit` polls
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    return t;
+}
+// bounded wait; false if the phase did not complete within `limit` polls or kWaitLimitNs nanoseconds
 __device__ __forceinline__ bool mbar_wait(uint64_t *b, unsigned parity, int limit = kWaitLimit)
 {
-    for (int i = 0; i < limit; ++i)
+    if (mbar_try_wait(b, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (int i = 1; i < limit; ++i) {
         if (mbar_try_wait(b, parity)) return true;
+        if ((i & 255) == 0 && globaltimer_ns() - t0 > kWaitLimitNs) return false;
+    }
     return false;
 }
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z)

@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
         L.hyenand_plan_launches.argtypes = [vp, ctypes.c_int]
         L.hyenand_plan_path.argtypes = [vp]
         L.hyenand_plan_path.restype = ctypes.c_char_p
+        L.hyenand_plan_groups.argtypes = [vp, ctypes.POINTER(ll), ip]
+        L.hyenand_plan_guard_damage.argtypes = [vp]
+        L.hyenand_plan_guard_damage.restype = ll
         dpp = ctypes.POINTER(ctypes.c_double)
         L.hyenand_plan_kernel_count.argtypes = [vp]
         L.hyenand_plan_kernel_info.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_char_p),
@@ -148,6 +151,18 @@ def hyenand_plan_path(plan: int) -> str:
     return lib().hyenand_plan_path(plan).decode()
 
 
+def hyenand_plan_groups(plan: int):
+    """(slices per group, lanes): how one forward schedules the batch."""
+    n, lanes = ctypes.c_longlong(), ctypes.c_int()
+    _check(lib().hyenand_plan_groups(plan, ctypes.byref(n), ctypes.byref(lanes)))
+    return int(n.value), int(lanes.value)
+
+
+def hyenand_plan_guard_damage(plan: int) -> int:
+    """Bytes of the guard bands around the plan's device allocations that a kernel overwrote (0 = none)."""
+    return int(lib().hyenand_plan_guard_damage(plan))
+
+
 def hyenand_plan_kernel_count(plan: int) -> int:
     return int(lib().hyenand_plan_kernel_count(plan))
 
@@ -161,8 +176,9 @@ def hyenand_plan_kernel_info(plan: int, kernel_id: int, h_shared: bool):
     return name.value.decode(), n.value, b.value, f.value
 
 
-def hyenand_plan_set_timing(plan: int, enable: bool) -> None:
-    _check(lib().hyenand_plan_set_timing(plan, 1 if enable else 0))
+def hyenand_plan_set_timing(plan: int, enable) -> None:
+    """0/False: off; 1/True: time every launch; 2: the same with the plan's lanes run one after the other."""
+    _check(lib().hyenand_plan_set_timing(plan, int(enable)))
 
 
 def hyenand_plan_kernel_time(plan: int, kernel_id: int):

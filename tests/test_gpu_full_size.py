@@ -1,16 +1,20 @@
-"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times: the
-oracle evaluates the defining sum (O1) at seeded sample positions of a few whole slices; the
-whole output must be finite."""
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+Three layers, all on the output of ONE forward over the whole batch:
+  * every element finite, guard bands around y and around the plan's workspace untouched;
+  * the defining sum (oracle O1) at seeded sample positions of six slices;
+  * whole slices (the first, the last, two seeded ones; every slice for vision2d) against the oracle's FFT
+    path (O2), with the whole-tensor gate, the per-slice gate and the element-wise bound of parity_util."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
 from paper_2607_19378_b200 import workloads as W
+from parity_util import TOL, assert_guards, assert_parity, guarded_output
 
 pytestmark = pytest.mark.gpu
 
-TOL = {"f32": 1e-5, "bf16": 2e-3}
 SAMPLES_PER_SLICE = 48
 
 
@@ -21,25 +25,36 @@ def test_named_workload_at_full_size(name):
     dev = torch.device("cuda", 0)
     q, k, v, h = W.make_inputs(w, device=dev)
     plan = hn.Plan(w.dims, w.B, w.C, causal=w.causal, dtype=w.torch_dtype)
-    y = torch.full_like(q, float("nan"))
+    big, y = guarded_output(q)
     plan.forward(q, k, v, h, y)
     torch.cuda.synchronize()
     status = hn.hyenand_plan_device_status(plan.handle)
+    damage = hn.hyenand_plan_guard_damage(plan.handle)
     plan.close()
     assert status == 0, "a kernel gave up a bounded wait"
+    assert damage == 0, "a kernel wrote outside the plan's workspace"
+    assert_guards(big, q.numel(), name)
     assert bool(torch.isfinite(y.float()).all()), "non-finite output"
     S = w.B * w.C
     rng = np.random.default_rng(w.seed)
     slices = sorted({0, S // 2, S - 1} | set(int(s) for s in rng.integers(0, S, size=3)))
     L = int(np.prod(w.dims))
     mode = "causal" if w.causal else "linear"
+
+    def one(t, s):
+        b, c = divmod(s, w.C)
+        return t[b, c].cpu()[None, None]
+
+    def filt(s):
+        b, c = divmod(s, w.C)
+        return (h[c] if w.h_shared else h[b, c]).cpu()[None, None]
+
+    # O1 at sampled positions
     got, ref = [], []
     for s in slices:
         b, c = divmod(s, w.C)
-        hs = h[c] if w.h_shared else h[b, c]
-        qs, ks, vs = (t[b, c].cpu()[None, None] for t in (q, k, v))
         idx = rng.integers(0, L, size=SAMPLES_PER_SLICE)
-        ref.append(oracle.conv_direct_at(qs, ks, vs, hs.cpu()[None, None], idx, mode))
+        ref.append(oracle.conv_direct_at(one(q, s), one(k, s), one(v, s), filt(s), idx, mode))
         got.append(oracle.to_f64(y[b, c].reshape(-1)[torch.from_numpy(idx).to(dev)]))
     got, ref = np.concatenate(got), np.concatenate(ref)
     err = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
@@ -50,3 +65,20 @@ def test_named_workload_at_full_size(name):
         assert err <= 1.1 * rounding + 1e-6, f"{name}: {err:.3e} vs rounding {rounding:.3e}"
         tol = max(tol, 1.1 * rounding)
     assert err <= tol, f"{name}: sampled rel-L2 {err:.3e}"
+
+    # O2 on whole slices, out of the full launch
+    if name in ("vision2d", "tiny2d"):
+        whole = list(range(S))
+    else:
+        whole = sorted({0, S - 1} | set(int(s) for s in rng.integers(0, S, size=2)))
+    if len(whole) == S:
+        hq = (t.cpu() for t in (q, k, v, h))
+        qh, kh, vh, hh = hq
+        ref2 = oracle.conv_fft(qh, kh, vh, hh, mode)
+        assert_parity(y.cpu(), ref2, qh, w, what="whole tensor vs O2")
+    else:
+        for s in whole:
+            b, c = divmod(s, w.C)
+            ws = W.Workload(w.name, w.dims, 1, 1, w.dtype, causal=w.causal)
+            ref2 = oracle.conv_fft(one(q, s), one(k, s), one(v, s), filt(s), mode)
+            assert_parity(y[b, c].cpu()[None, None], ref2, one(q, s), ws, what=f"slice {s} vs O2")

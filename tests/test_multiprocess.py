@@ -67,3 +67,18 @@ def test_single_process_helpers():
     assert abs(flops - 192 * 2.5 * 2 ** 24 * 24) < 1
     nbytes, flops, P = bench.op_algorithmic(W.WORKLOADS["genomics1d"])
     assert P == 2 ** 19 and abs(flops - 1280 * 2.5 * 2 ** 19 * 19) < 1
+
+
+def test_gpus_flag_spawns_one_rank_per_gpu_when_no_launcher_is_present():
+    """`bench.py --gpus N` without torchrun around it starts its N ranks itself: the command it builds is the
+    launcher the multi-rank path expects (one process per GPU, loopback rendezvous) and carries every option on."""
+    import argparse
+    import bench
+    args = argparse.Namespace(gpus=4, steps=7, warmup=3, workload="pde2d", impl="ours", batch=None, channels=16,
+                              no_all=True, no_cpu=False, no_cufft=True)
+    cmd = bench.spawn_command(args, 29512)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29512"
+    tail = cmd[cmd.index(os.path.join(ROOT, "bench.py")) + 1:]
+    assert tail == ["--gpus", "4", "--steps", "7", "--warmup", "3", "--workload", "pde2d", "--impl", "ours",
+                    "--channels", "16", "--no-all", "--no-cufft"]

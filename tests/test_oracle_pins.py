@@ -310,3 +310,23 @@ def test_argument_errors():
         oracle.conv_direct(rnd(1, 1, 4), rnd(1, 1, 4), rnd(1, 1, 4), rnd(1, 1, 6))
     with pytest.raises(ValueError):
         oracle.conv_direct(rnd(1, 1, 4, 4), rnd(1, 1, 4, 4), rnd(1, 1, 4, 4), rnd(1, 1, 4, 4), "causal")
+
+
+LARGE_PADDED = [((32768,), "linear"), ((32768,), "causal"), ((128, 128), "linear"), ((32, 64, 64), "linear")]
+
+
+@pytest.mark.parametrize("dims,mode", LARGE_PADDED, ids=str)
+def test_o2_agrees_with_sampled_o1_at_large_padded_sizes(dims, mode):
+    """Convolution theorem at the sizes the GPU tests rely on O2 for (padded 2^16, 256 x 256, 64 x 128 x 128):
+    the FFT path against the defining sum evaluated at seeded output positions, per-sample and shared filters."""
+    rng = np.random.default_rng(7)
+    B, C = 2, 2
+    taps = tuple(L if mode == "causal" else 2 * L - 1 for L in dims)
+    q, k, v = (rng.standard_normal((B, C) + dims) for _ in range(3))
+    for shared in (False, True):
+        h = rng.standard_normal(((C,) if shared else (B, C)) + taps)
+        full = oracle.conv_fft(q, k, v, h, mode)
+        idx = rng.integers(0, full.size, size=96)
+        at = oracle.conv_direct_at(q, k, v, h, idx, mode)
+        scale = np.sqrt(np.mean(full * full))
+        assert np.max(np.abs(full.ravel()[idx] - at)) <= 1e-11 * scale
