@@ -34,6 +34,7 @@ import torch  # noqa: E402
 
 from paper_2607_19378_b200 import workloads as W  # noqa: E402
 
+ALL_WORKLOADS = {**W.WORKLOADS, **W.EXTRA_WORKLOADS}
 METRIC = "hyenand_forward_throughput"
 UNIT = "Gelem/s"
 DEFAULT_WORKLOAD = "volume3d"
@@ -56,6 +57,11 @@ def fp32_peak_tflops(sm_count: int, sm_max_mhz: float) -> float:
     return 2.0 * FP32_LANES_PER_SM * sm_count * sm_max_mhz * 1e6 / 1e12
 
 
+def padded_dims(w: W.Workload):
+    """Transform size per axis: the grid itself with periodic boundaries, else the next power of two >= 2L-1."""
+    return [L if w.circular else 1 << max(0, (2 * L - 2).bit_length()) for L in w.dims]
+
+
 def op_algorithmic(w: W.Workload):
     """Minimal bytes (q,k,v,h,y once) and nominal flops (2.5 P log2 P per real transform:
     k*v forward and the inverse per slice, h forward per filter) of one forward."""
@@ -63,9 +69,7 @@ def op_algorithmic(w: W.Workload):
     E = w.elements
     hcount = w.C if w.h_shared else w.B * w.C
     hbytes = hcount * math.prod(w.taps) * s
-    P = 1
-    for L in w.dims:
-        P *= 1 << max(0, (2 * L - 2).bit_length())
+    P = math.prod(padded_dims(w))
     transforms = 2 * w.B * w.C + hcount
     flops = transforms * 2.5 * P * math.log2(P) if P > 1 else 0.0
     return 4 * E * s + hbytes, flops, P
@@ -134,7 +138,7 @@ def time_workload(w: W.Workload, steps: int, warmup: int, dist, device, want_ker
     from paper_2607_19378_b200 import hyenand as hn
     q, k, v, h = W.make_inputs(w, device=device)
     y = torch.empty_like(q)
-    plan = hn.Plan(w.dims, w.B, w.C, causal=w.causal, dtype=w.torch_dtype)
+    plan = hn.Plan(w.dims, w.B, w.C, causal=w.causal, dtype=w.torch_dtype, circular=w.circular)
     stream = torch.cuda.current_stream()
     for _ in range(max(warmup, 3)):
         plan.forward(q, k, v, h, y)
@@ -226,7 +230,7 @@ def cufft_composition(w: W.Workload, tensors, reps: int = 3):
     Returns its time per forward and its error against our result."""
     q, k, v, h, y = tensors
     nd = len(w.dims)
-    P = [1 << max(0, (2 * L - 2)).bit_length() if L > 1 else 1 for L in w.dims]
+    P = padded_dims(w)
     S = w.B * w.C
     axes = tuple(range(1, nd + 1))
     qf, kf, vf = (t.reshape(S, *w.dims) for t in (q, k, v))
@@ -234,7 +238,7 @@ def cufft_composition(w: W.Workload, tensors, reps: int = 3):
     per_slice = 4 * 6 * int(torch.tensor(P).prod())           # bytes of fp32 work arrays per slice, roughly
     chunk = max(1, min(S, int(4e9) // max(per_slice, 1)))
     out = torch.empty_like(qf)
-    crop0 = [0 if w.causal else L - 1 for L in w.dims]
+    crop0 = [0 if (w.causal or w.circular) else L - 1 for L in w.dims]
 
     def run():
         for s0 in range(0, S, chunk):
@@ -275,7 +279,7 @@ def cpu_oracle_sample(w: W.Workload, budget_s: float = 15.0):
     """Times the oracle (as it stands) on a bounded sample of slices of the workload."""
     import oracle
     threads = oracle.threads()
-    mode = "causal" if w.causal else "linear"
+    mode = w.mode
 
     def run(n_slices):
         ws = w.scaled(B=1, C=n_slices)
@@ -380,7 +384,7 @@ def main_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
-    w = W.WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
+    w = ALL_WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
     w = workload_for_rank(w, rank, world)
     hbm_gbs, peak_src, sm_max = measured_peaks()
     props = torch.cuda.get_device_properties(local)
@@ -412,7 +416,7 @@ def main_ours(args):
         "ms_per_step_median": res["ms_median"], "ms_per_step_min": res["ms_min"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
-        "config": {"workload": w.name, "dims": list(w.dims), "B": w.B, "C": w.C, "causal": w.causal,
+        "config": {"workload": w.name, "dims": list(w.dims), "B": w.B, "C": w.C, "causal": w.causal, "circular": w.circular,
                    "h_shared_over_batch": w.h_shared, "padded_points_per_slice": P,
                    "l2": "inputs larger than L2 (no flush needed)" if nbytes > 126e6 else "fits L2; latency-bound",
                    "path": res["path"], "slices_per_group": res["slices_per_group"], "lanes": res["lanes"],
@@ -469,9 +473,9 @@ def main_reference(args):
     if rank != 0:
         return
     import oracle
-    w = W.WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
+    w = ALL_WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
     threads = oracle.threads()
-    mode = "causal" if w.causal else "linear"
+    mode = w.mode
     S = w.B * w.C
     # size one step at roughly 2 s of oracle time: probe with one slice per thread first
     n = min(S, threads)
@@ -511,7 +515,7 @@ if __name__ == "__main__":
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(ALL_WORKLOADS))
     ap.add_argument("--batch", type=int, default=None, help="override B (profiling on a smaller case)")
     ap.add_argument("--channels", type=int, default=None, help="override C (profiling on a smaller case)")
     ap.add_argument("--no-all", action="store_true", help="skip the table over the other workloads")

@@ -69,6 +69,18 @@ enum {
 hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype);
 
 /*
+ * Same with the boundary handling named explicitly (Section 3.2.1, circular and non-circular convolutions):
+ *   HYENAND_MODE_LINEAR    zero-padded, non-causal: the kernel lives on (2 L_1 - 1) x ... x (2 L_N - 1)
+ *   HYENAND_MODE_CAUSAL    1-D only (Appendix A.3): K_1 = L_1, negative displacements carry no weight
+ *   HYENAND_MODE_CIRCULAR  periodic boundaries: the kernel lives on the grid itself, K_n = L_n, tap index
+ *                          m_n = (i_n - j_n) mod L_n, and the transforms run on L_n points with no padding.
+ *                          Every L_n must be a power of two and at most 8192 (HYENAND_ERR_UNSUPPORTED otherwise).
+ * hyenand_create_plan(..., causal, ...) is this call with mode = causal ? CAUSAL : LINEAR.
+ */
+enum { HYENAND_MODE_LINEAR = 0, HYENAND_MODE_CAUSAL = 1, HYENAND_MODE_CIRCULAR = 2 };
+hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int B, int C, int mode, int dtype);
+
+/*
  * One forward pass with one filter per (b,c): the input-dependent kernels of
  * Section 3.2.2, one per sample of the batch and per channel.
  * q, k, v, h, y: DEVICE pointers, 16-byte aligned, y must not alias an input.

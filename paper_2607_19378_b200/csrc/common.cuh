@@ -134,6 +134,7 @@ struct RowsArgs {
     int prune_in;         // 1: all valid positions are < P/2 (u, causal h)
     const float2 *gtw;    // global twiddle table, gtw_n points
     int gtw_n;
+    int full_in;          // 1: circular mode, k*v rows fill the whole line (len == P): nothing to prune
 };
 
 struct RowsInvArgs {
@@ -146,6 +147,7 @@ struct RowsInvArgs {
     int log2p;
     const float2 *gtw;
     int gtw_n;
+    int full_out;         // 1: circular mode, all P outputs of a row are kept (len == P)
 };
 
 // A family of strided lines: line (o, c), element a at base[o*outer + a*nc + c].
@@ -173,6 +175,7 @@ struct AxisArgs {
     float scale;              // applied to the product (1/P_total)
     const float2 *gtw;
     int gtw_n;
+    int full;                 // 1: circular mode (n_in == n_out == P): no pruned input half, all outputs kept
 };
 
 enum AxisMode { AXIS_FWD = 0, AXIS_INV = 1, AXIS_CORE = 2 };

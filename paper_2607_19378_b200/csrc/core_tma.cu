@@ -39,7 +39,9 @@ template <int LOG2P> struct TmaGeo {
     static constexpr int NB = HALF / BOXR;                           // boxes per half line
     static constexpr unsigned BOXB = BOXR * ROWB;
     static constexpr unsigned HALFB = HALF * ROWB;
-    static constexpr int LS = TX >= 16 ? line_stride(N) : ((F::ph(N - 1) + 1 + 15) / 16 * 16 + 2);
+    // 16-lane groups (two lines per warp): the lanes of a half warp belong to both lines (see the kernel), whose
+    // strides are therefore 8 mod 16 entries, i.e. half a bank row apart
+    static constexpr int LS = TX >= 16 ? plane_ls(N) : ((F::ph(N - 1) + 1 + 15) / 16 * 16 + 2);
     static_assert(ROWB == 128 || ROWB == 64, "tile rows match a swizzle span");
     // shared memory: tile buffers first (1024-byte aligned, as the swizzle pattern repeats every 1024 bytes)
     static constexpr size_t TH = 0;                                  // filter tile, N rows
@@ -85,8 +87,14 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
     float2 *twt = reinterpret_cast<float2 *>(smem_raw + G::TW);
     uint64_t *bar_h = reinterpret_cast<uint64_t *>(smem_raw + G::BARS);
     uint64_t *bar_u = bar_h + 1;
-    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
-    const unsigned m = F::group_mask(tid);
+    // Lanes of a warp: with one line per warp (32 lanes per line) lane = position.  With two lines per warp the
+    // two are interleaved in blocks of 8 lanes (lanes 0-7 and 16-23 work on the first line, 8-15 and 24-31 on the
+    // second): an 8-byte shared-memory access is served per half warp, and a half warp then reads 8 rows of BOTH
+    // bins of a 16-byte tile chunk, 16 distinct 8-byte slots, instead of 16 rows of one bin, which share 8 slots.
+    const int tid = threadIdx.x;
+    const int l = TPL == 16 ? ((tid & 7) | ((tid >> 1) & 8)) : tid % TPL;
+    const int gid = TPL == 16 ? ((tid >> 5) * 2 + ((tid >> 3) & 1)) : tid / TPL;
+    const unsigned m = TPL == 16 ? (0x00ff00ffu << (tid & 8)) : F::group_mask(tid);
     float2 *line = lines + gid * G::LS;
     for (int t = tid; t < N; t += kTmaThreads) twt[t] = p.gtw[t * (p.gtw_n / N)];
     if (tid == 0) {

@@ -41,7 +41,8 @@ template <int LOG2P> __host__ __device__ constexpr int core_ls()
     return n;
 }
 
-template <int LOG2P>
+// FULL (circular mode: n_in == n_out == N): the k*v lines have no zero half and every output is kept.
+template <int LOG2P, bool FULL>
 __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) axis_core_w_kernel(AxisArgs p)
 {
     constexpr int kCoreThreads = core_threads(LOG2P);
@@ -116,7 +117,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
         int pos = r0;
 #pragma unroll 4
         for (; pos < nin; pos += RPS, src += step) cp_async8_s(bu_x + 8u * (unsigned)F::ph(pos), src);
-        for (; pos < N / 2; pos += RPS) bu[x * LS + F::ph(pos)] = make_float2(0.f, 0.f);
+        for (; pos < (FULL ? N : N / 2); pos += RPS) bu[x * LS + F::ph(pos)] = make_float2(0.f, 0.f);
     };
     long long t = blockIdx.x;
     if (t < tiles) { issue_h(t); }
@@ -145,7 +146,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
         }
         __syncthreads();
         {
-            F::template mid<0, NP - 1, PRUNE_IN>(l, m, tw, uline);
+            F::template mid<0, NP - 1, FULL ? PRUNE_NONE : PRUNE_IN>(l, m, tw, uline);
             float2 Y[PL::IPL][PL::R];
             F::template pass<NP - 1, PRUNE_NONE>(l, tw,
                 [&](int, int, int idx) { return uline[F::ph(idx)]; },
@@ -164,7 +165,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
             FI::template mid<1, NP - 1, PRUNE_NONE>(l, m, twi, uline);
             using PE = typename FI::template Pass<NP - 1>;
             float2 keep[PE::IPL][PE::R];
-            FI::template pass<NP - 1, PRUNE_OUT>(l, twi,
+            FI::template pass<NP - 1, FULL ? PRUNE_NONE : PRUNE_OUT>(l, twi,
                 [&](int, int, int idx) { return uline[FI::ph(idx)]; },
                 [&](int i, int r, int, float2 v) { keep[i][r] = v; });
             __syncwarp(m);
@@ -172,7 +173,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
 #pragma unroll
                 for (int i = 0; i < PE::IPL; ++i)
 #pragma unroll
-                    for (int r = 0; r < PE::R / 2; ++r)
+                    for (int r = 0; r < (FULL ? PE::R : PE::R / 2); ++r)
                         uline[FI::ph(l + i * TPL + r * (N / PE::R))] = keep[i][r];
             }
         }
@@ -197,7 +198,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
     cp_async_wait<0>();
 }
 
-template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t st)
+template <int LOG2P, bool FULL> static int launch_core_w_t(const AxisArgs &a, cudaStream_t st)
 {
     using F = WF<LOG2P, false>;
     constexpr int kCoreThreads = core_threads(LOG2P);
@@ -211,12 +212,12 @@ template <int LOG2P> static int launch_core_w_t(const AxisArgs &a, cudaStream_t 
         if (sms <= 0) sms = 148;
     }
     static DevOnce attr;
-    if (attr.first()) cudaFuncSetAttribute(axis_core_w_kernel<LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (attr.first()) cudaFuncSetAttribute(axis_core_w_kernel<LOG2P, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     const long long tiles = a.n_outer * ((a.nc + TX - 1) / TX);
     const long long res = (long long)sms * 2;
     const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
-    axis_core_w_kernel<LOG2P><<<grid, kCoreThreads, sm, st>>>(a);
+    axis_core_w_kernel<LOG2P, FULL><<<grid, kCoreThreads, sm, st>>>(a);
     return 1;
 }
 
@@ -225,11 +226,11 @@ bool core_w_supported(int log2p) { return log2p >= 6 && log2p <= 10; }
 int launch_core_w(const AxisArgs &a, cudaStream_t st)
 {
     switch (a.log2p) {
-    case 6: return launch_core_w_t<6>(a, st);
-    case 7: return launch_core_w_t<7>(a, st);
-    case 8: return launch_core_w_t<8>(a, st);
-    case 9: return launch_core_w_t<9>(a, st);
-    case 10: return launch_core_w_t<10>(a, st);
+    case 6: return a.full ? launch_core_w_t<6, true>(a, st) : launch_core_w_t<6, false>(a, st);
+    case 7: return a.full ? launch_core_w_t<7, true>(a, st) : launch_core_w_t<7, false>(a, st);
+    case 8: return a.full ? launch_core_w_t<8, true>(a, st) : launch_core_w_t<8, false>(a, st);
+    case 9: return a.full ? launch_core_w_t<9, true>(a, st) : launch_core_w_t<9, false>(a, st);
+    case 10: return a.full ? launch_core_w_t<10, true>(a, st) : launch_core_w_t<10, false>(a, st);
     default: return -1;
     }
 }

@@ -36,6 +36,7 @@ constexpr int kMaxLanes = 4;
 
 struct hyenand_plan {
     int ndim, B, C, causal, dtype;
+    bool circular;                    // periodic boundaries: K_n = P_n = L_n
     int dims[3];
     int L[3], K[3], P[3], log2p[3];   // internal 3-axis form (leading axes of extent 1)
     int XH;                           // half-spectrum bins along the contiguous axis
@@ -130,19 +131,36 @@ static void choose_groups(hyenand_plan *p, long long per_slice_elems);
 
 extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype)
 {
+    if (causal != 0 && causal != 1) { g_err[0] = 0; fail(HYENAND_ERR_INVALID_ARG, "causal must be 0 or 1"); return nullptr; }
+    return hyenand_create_plan_mode(ndim, dims, B, C, causal ? HYENAND_MODE_CAUSAL : HYENAND_MODE_LINEAR, dtype);
+}
+
+extern "C" hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int B, int C, int mode, int dtype)
+{
     g_err[0] = 0;
+    if (mode != HYENAND_MODE_LINEAR && mode != HYENAND_MODE_CAUSAL && mode != HYENAND_MODE_CIRCULAR) {
+        fail(HYENAND_ERR_INVALID_ARG, "unknown boundary mode %d", mode);
+        return nullptr;
+    }
+    const int causal = mode == HYENAND_MODE_CAUSAL;
+    const bool circular = mode == HYENAND_MODE_CIRCULAR;
     if (ndim < 1 || ndim > 3) { fail(HYENAND_ERR_INVALID_ARG, "ndim must be 1, 2 or 3 (got %d)", ndim); return nullptr; }
     if (!dims) { fail(HYENAND_ERR_INVALID_ARG, "dims is NULL"); return nullptr; }
     if (B < 1 || C < 1) { fail(HYENAND_ERR_INVALID_ARG, "B and C must be >= 1 (got %d, %d)", B, C); return nullptr; }
     if (dtype != HYENAND_F32 && dtype != HYENAND_BF16) { fail(HYENAND_ERR_INVALID_ARG, "unknown dtype %d", dtype); return nullptr; }
-    if (causal != 0 && causal != 1) { fail(HYENAND_ERR_INVALID_ARG, "causal must be 0 or 1"); return nullptr; }
     for (int a = 0; a < ndim; ++a)
         if (dims[a] < 1) { fail(HYENAND_ERR_INVALID_ARG, "dims[%d] = %d must be >= 1", a, dims[a]); return nullptr; }
     if (causal && ndim != 1) { fail(HYENAND_ERR_UNSUPPORTED, "causal kernels are defined for 1-D grids only"); return nullptr; }
+    if (circular)
+        for (int a = 0; a < ndim; ++a)
+            if (dims[a] & (dims[a] - 1)) {
+                fail(HYENAND_ERR_UNSUPPORTED, "circular mode transforms the grid itself: dims[%d] = %d is not a power of two", a, dims[a]);
+                return nullptr;
+            }
 
     hyenand_plan *p = new hyenand_plan();
     memset(p, 0, sizeof(*p));
-    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype;
+    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->circular = circular; p->dtype = dtype;
     p->r0 = 0; p->r1 = (long long)B * C;
     cudaGetDevice(&p->device);
     p->sw = read_switches();
@@ -154,8 +172,8 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
         p->dims[a] = dims[a];
         if ((long long)dims[a] > (1ll << 25)) { fail(HYENAND_ERR_UNSUPPORTED, "dims[%d] too long", a); delete p; return nullptr; }
         p->L[ia] = dims[a];
-        p->K[ia] = causal ? dims[a] : 2 * dims[a] - 1;
-        p->log2p[ia] = next_pow2_log(2 * dims[a] - 1);
+        p->K[ia] = (causal || circular) ? dims[a] : 2 * dims[a] - 1;
+        p->log2p[ia] = circular ? next_pow2_log(dims[a]) : next_pow2_log(2 * dims[a] - 1);
         p->P[ia] = 1 << p->log2p[ia];
         p->vol *= dims[a];
         p->kvol *= p->K[ia];
@@ -163,8 +181,13 @@ extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, i
     p->XH = p->P[2] / 2 + 1;
     p->XP = (p->XH + 1) & ~1;
     const long long S = (long long)B * C;
+    if (circular) {
+        // periodic boundaries run on the general N-D passes, which transform whole lines here (nothing is
+        // padded, so there is no zero half to prune and no half to crop); no plane, fused or tensor-copy kernels
+        p->sw.force_generic = p->sw.no_tma = true;
+    }
 
-    if (ndim == 1 && p->log2p[2] > kMaxLineLog2) {
+    if (ndim == 1 && p->log2p[2] > kMaxLineLog2 && !circular) {
         p->path = PATH_CT1D;
         if (p->log2p[2] > 24) { fail(HYENAND_ERR_UNSUPPORTED, "1-D grid too long (padded size 2^%d > 2^24)", p->log2p[2]); delete p; return nullptr; }
         size_t bytes = 0;
@@ -359,9 +382,10 @@ static int filter_spectrum_generic(hyenand_plan *p, int l, const char *h, long l
     r.a = h; r.b = nullptr; r.out = ln.wh_a; r.pitch = p->XP;
     r.rows = n_slices * p->K[0] * p->K[1];
     r.len = p->K[2];
-    r.shift = p->causal ? 0 : p->L[2] - 1;
+    r.shift = (p->causal || p->circular) ? 0 : p->L[2] - 1;
     r.log2p = p->log2p[2];
     r.prune_in = p->causal && p->P[2] >= 2;
+    r.full_in = p->circular;
     r.gtw = p->gtw; r.gtw_n = p->gtw_n;
     p->prof.begin(KID_ROWS_H, st);
     const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
@@ -376,7 +400,7 @@ static int filter_spectrum_generic(hyenand_plan *p, int l, const char *h, long l
         a.in_outer = (long long)p->K[1] * p->XP;
         a.out_outer = (long long)p->P[1] * p->XP;
         a.nc = p->XP; a.n_in = p->K[1]; a.n_out = p->P[1];
-        a.shift = p->L[1] - 1; a.log2p = p->log2p[1]; a.prune_in = 0;
+        a.shift = p->circular ? 0 : p->L[1] - 1; a.log2p = p->log2p[1]; a.prune_in = 0;
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         p->prof.begin(KID_AXIS_H, st);
         n = launch_axis(a, AXIS_FWD, st);
@@ -400,11 +424,11 @@ static AxisArgs generic_core_args(const hyenand_plan *p, int l, long long n, boo
     a.n_outer = n;
     a.in_outer = a.out_outer = (long long)p->L[ax] * inner;
     a.nc = (int)inner; a.n_in = p->L[ax]; a.n_out = p->L[ax]; a.shift = 0;
-    a.log2p = p->log2p[ax]; a.prune_in = 1;
+    a.log2p = p->log2p[ax]; a.prune_in = 1; a.full = p->circular;
     a.h = three ? lh.wh_b : lh.wh_a;
     a.h_outer = (long long)p->K[ax] * inner;
     a.h_n_in = p->K[ax];
-    a.h_shift = p->causal ? 0 : p->L[ax] - 1;
+    a.h_shift = (p->causal || p->circular) ? 0 : p->L[ax] - 1;
     a.h_mod = shared ? p->C : 0;
     a.h_off = shared ? s0 % p->C : 0;
     a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
@@ -442,7 +466,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         RowsArgs r{};
         r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = ln.ws_a; r.pitch = p->XP;
         r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
-        r.prune_in = 1; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
+        r.prune_in = 1; r.full_in = p->circular; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
         p->prof.begin(KID_ROWS_U, st);
         const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
         int c = roww ? launch_rows_fwd_w(r, p->dtype, st) : launch_rows_fwd(r, p->dtype, st);
@@ -455,7 +479,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.n_outer = n * p->L[0];
             a.in_outer = (long long)p->L[1] * p->XP; a.out_outer = (long long)p->P[1] * p->XP;
             a.nc = p->XP; a.n_in = p->L[1]; a.n_out = p->P[1]; a.shift = 0;
-            a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2;
+            a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2 && !p->circular;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
             p->prof.begin(KID_AXIS_U, st);
             c = launch_axis(a, AXIS_FWD, st);
@@ -477,7 +501,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.n_outer = n * p->L[0];
             a.in_outer = (long long)p->P[1] * p->XP; a.out_outer = (long long)p->L[1] * p->XP;
             a.nc = p->XP; a.n_in = p->P[1]; a.n_out = p->L[1]; a.shift = 0;
-            a.log2p = p->log2p[1]; a.prune_in = 0;
+            a.log2p = p->log2p[1]; a.prune_in = 0; a.full = p->circular;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
             p->prof.begin(KID_AXIS_INV, st);
             c = launch_axis(a, AXIS_INV, st);
@@ -488,7 +512,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         RowsInvArgs ri{};
         ri.in = ln.ws_a; ri.pitch = p->XP; ri.q = q + (size_t)s0 * p->vol * es; ri.y = y + (size_t)s0 * p->vol * es;
         ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
-        ri.gtw = p->gtw; ri.gtw_n = p->gtw_n;
+        ri.gtw = p->gtw; ri.gtw_n = p->gtw_n; ri.full_out = p->circular;
         p->prof.begin(KID_ROWS_INV, st);
         c = roww ? launch_rows_inv_w(ri, p->dtype, st) : launch_rows_inv(ri, p->dtype, st);
         p->prof.end(st);

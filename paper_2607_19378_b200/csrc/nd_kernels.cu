@@ -109,7 +109,8 @@ static int launch_rows_fwd_t(const RowsArgs &a, cudaStream_t st)
         }                                                                                       \
         rows_fwd_kernel<T, LOG2P, HASB, PR><<<grid, kThreads, sm, st>>>(a);                     \
     } while (0)
-    if (a.b) HN_LAUNCH(true, true);
+    if (a.b && a.full_in) HN_LAUNCH(true, false);
+    else if (a.b) HN_LAUNCH(true, true);
     else if (a.prune_in) HN_LAUNCH(false, true);
     else HN_LAUNCH(false, false);
 #undef HN_LAUNCH
@@ -139,7 +140,7 @@ int launch_rows_fwd(const RowsArgs &a, int dtype, cudaStream_t st)
 
 // ---- rows, inverse + crop + output gate ----------------------------------------------
 
-template <typename T, int LOG2P>
+template <typename T, int LOG2P, bool FULL>
 __global__ void __launch_bounds__(kThreads) rows_inv_kernel(RowsInvArgs p)
 {
     constexpr int N = 1 << LOG2P;
@@ -167,7 +168,7 @@ __global__ void __launch_bounds__(kThreads) rows_inv_kernel(RowsInvArgs p)
             buf[g * LS + phys(pos)] = make_float2(A.x - B.y, A.y + B.x);
         }
         __syncthreads();
-        fft_lines<LOG2P, true, PRUNE_OUT, kThreads>(buf, G, LS, tw, tid);
+        fft_lines<LOG2P, true, FULL ? PRUNE_NONE : PRUNE_OUT, kThreads>(buf, G, LS, tw, tid);
         for (int idx = tid; idx < G * p.len; idx += kThreads) {
             const int g = idx / p.len, n = idx % p.len;
             const long long r0 = 2 * (ch * G + g), r1 = r0 + 1;
@@ -188,11 +189,10 @@ static int launch_rows_inv_t(const RowsInvArgs &a, cudaStream_t st)
     const long long chunks = (pairs + G - 1) / G;
     const int grid = (int)(chunks < (long long)sm_count() * 8 ? chunks : (long long)sm_count() * 8);
     if (grid <= 0) return 0;
-    static DevOnce attr;
-    if (attr.first()) {
-        cudaFuncSetAttribute(rows_inv_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    }
-    rows_inv_kernel<T, LOG2P><<<grid, kThreads, sm, st>>>(a);
+    static DevOnce attr[2];
+    void (*fn)(RowsInvArgs) = a.full_out ? rows_inv_kernel<T, LOG2P, true> : rows_inv_kernel<T, LOG2P, false>;
+    if (attr[a.full_out ? 1 : 0].first()) cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    fn<<<grid, kThreads, sm, st>>>(a);
     return 1;
 }
 
@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(kThreads) axis_kernel(AxisArgs p)
         }
         __syncthreads();
         if (MODE == AXIS_INV) {
-            fft_lines<LOG2P, true, PRUNE_OUT, kThreads>(bu, TX, LS, tw, tid);
+            fft_lines<LOG2P, true, PRUNE ? PRUNE_OUT : PRUNE_NONE, kThreads>(bu, TX, LS, tw, tid);
         } else {
             fft_lines<LOG2P, false, PRUNE ? PRUNE_IN : PRUNE_NONE, kThreads>(bu, TX, LS, tw, tid);
         }
@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(kThreads) axis_kernel(AxisArgs p)
                 bu[a] = make_float2(w.x * p.scale, w.y * p.scale);
             }
             __syncthreads();
-            fft_lines<LOG2P, true, PRUNE_OUT, kThreads>(bu, TX, LS, tw, tid);
+            fft_lines<LOG2P, true, PRUNE ? PRUNE_OUT : PRUNE_NONE, kThreads>(bu, TX, LS, tw, tid);
         }
         float2 *dst = p.out + o * p.out_outer + c0;
         for (int idx = tid; idx < TX * p.n_out; idx += kThreads) {
@@ -295,16 +295,23 @@ int launch_axis(const AxisArgs &a, int mode, cudaStream_t st)
     int n = 0;
 #define CALL_FP(L) n = launch_axis_t<AXIS_FWD, L, true>(a, st)
 #define CALL_FN(L) n = launch_axis_t<AXIS_FWD, L, false>(a, st)
-#define CALL_I(L) n = launch_axis_t<AXIS_INV, L, false>(a, st)
+    // inverse and core: the flag selects the cropped (pruned) output half, or the whole line in circular mode
+#define CALL_I(L) n = launch_axis_t<AXIS_INV, L, true>(a, st)
+#define CALL_IF(L) n = launch_axis_t<AXIS_INV, L, false>(a, st)
 #define CALL_C(L) n = launch_axis_t<AXIS_CORE, L, true>(a, st)
+#define CALL_CF(L) n = launch_axis_t<AXIS_CORE, L, false>(a, st)
     if (mode == AXIS_FWD && a.prune_in) { HN_SWITCH_LOG2P(a.log2p, CALL_FP) }
     else if (mode == AXIS_FWD) { HN_SWITCH_LOG2P(a.log2p, CALL_FN) }
+    else if (mode == AXIS_INV && a.full) { HN_SWITCH_LOG2P(a.log2p, CALL_IF) }
     else if (mode == AXIS_INV) { HN_SWITCH_LOG2P(a.log2p, CALL_I) }
+    else if (a.full) { HN_SWITCH_LOG2P(a.log2p, CALL_CF) }
     else { HN_SWITCH_LOG2P(a.log2p, CALL_C) }
 #undef CALL_FP
 #undef CALL_FN
 #undef CALL_I
+#undef CALL_IF
 #undef CALL_C
+#undef CALL_CF
     return n;
 }
 

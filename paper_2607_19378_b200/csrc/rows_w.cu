@@ -13,7 +13,9 @@ namespace hn {
 
 constexpr int kRowThreads = 256;
 
-// MODE 0: k*v rows (upper half zero), 1: filter rows with wrapped placement, 2: causal filter rows
+// MODE 0: k*v rows (upper half zero), 1: filter rows with wrapped placement, 2: causal filter rows,
+// 3: circular mode, rows of exactly P elements (k*v when b is given, else the filter): power-of-two, aligned rows
+// that are read straight from global memory (no staging of misaligned odd-length rows is needed)
 // One lane asks the memory system to bring [lo, hi) of an array into L2, trimmed inwards to 16-byte granules.
 __device__ __forceinline__ void prefetch_rows_l2(const unsigned char *lo, const unsigned char *hi)
 {
@@ -26,7 +28,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
 {
     using F = WF<LOG2P, false>;
     constexpr int P = 1 << LOG2P, HP = P / 2, TPL = F::TPL, G = kRowThreads / TPL, LS = plane_ls(P);
-    constexpr int PR = MODE == 1 ? PRUNE_NONE : PRUNE_IN;
+    constexpr int PR = (MODE == 1 || MODE == 3) ? PRUNE_NONE : PRUNE_IN;
     constexpr int NT = MODE == 0 ? 2 : 1;                                       // tensors per row
     constexpr int ROWMAX = (MODE == 1 ? P - 1 : HP) * (int)sizeof(T);           // longest row in bytes
     constexpr int SLOT = (ROWMAX + 15) / 16 * 16 + 16;
@@ -49,6 +51,25 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
     for (long long rp = (long long)blockIdx.x * G + gid; rp < pairs; rp += (long long)gridDim.x * G) {
         const long long r0 = 2 * rp, r1 = r0 + 1;
         const bool has1 = r1 < p.rows;
+        if constexpr (MODE == 3) {
+            const T *a0 = (const T *)p.a + r0 * P, *a1 = (const T *)p.a + (has1 ? r1 : r0) * P;
+            const T *b0 = (const T *)p.b + r0 * P, *b1 = (const T *)p.b + (has1 ? r1 : r0) * P;
+            const bool gated = p.b != nullptr;
+            const float keep1 = has1 ? 1.f : 0.f;
+            F::template run_to_line<PR, false>(l, m, tw, line, [&](int, int, int idx) {
+                float a = IO<T>::ld(a0, idx), b = IO<T>::ld(a1, idx) * keep1;
+                if (gated) { a *= IO<T>::ld(b0, idx); b *= IO<T>::ld(b1, idx); }
+                return make_float2(a, b);
+            });
+            float2 *o0 = p.out + r0 * p.pitch, *o1 = p.out + r1 * p.pitch;
+            for (int kx = l; kx <= HP; kx += TPL) {
+                const float2 z1 = line[F::ph(kx)], z2 = line[F::ph((P - kx) & (P - 1))];
+                o0[kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
+                if (has1) o1[kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
+            }
+            __syncwarp(m);
+            continue;
+        }
         unsigned char *s = reinterpret_cast<unsigned char *>(line);
         const unsigned char *g0 = ab + r0 * rowb, *g1 = ab + r1 * rowb;
         stage_row_u<TPL, ROWMAX>(s, g0, rowb, ab, ahi, l);
@@ -117,7 +138,8 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
     }
 }
 
-template <typename T, int LOG2P>
+// FULL (circular mode): all P outputs of a row are kept.
+template <typename T, int LOG2P, bool FULL>
 __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs p)
 {
     using FI = WF<LOG2P, true>;
@@ -146,7 +168,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
             cp_async16(line + 2 * c, i0 + 2 * c);
             if (has1) cp_async16(line + RS + 2 * c, i1 + 2 * c);
         }
-        if (p.len == HP && has1 && l == 0) {
+        if (!FULL && p.len == HP && has1 && l == 0) {
             // the two gate rows of the pair (contiguous, a multiple of 16 bytes from a 16-byte boundary)
             const unsigned long long qa = (unsigned long long)(pq + r0 * HP);
             asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(qa), "r"((unsigned)(2 * HP * sizeof(T))) : "memory");
@@ -159,7 +181,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
         if (!has1) for (int c = l; c <= HP; c += TPL) line[RS + c] = make_float2(0.f, 0.f);
         __syncwarp(m);
         constexpr int RH = FI::template Pass<0>::R / 2;
-        FI::template run_to_line<PRUNE_OUT, true>(l, m, tw, line, [&](int, int r, int idx) {
+        FI::template run_to_line<FULL ? PRUNE_NONE : PRUNE_OUT, true>(l, m, tw, line, [&](int, int r, int idx) {
             if (r < RH) {
                 const float2 A = line[idx], B = line[RS + idx];
                 return make_float2(A.x - B.y, A.y + B.x);
@@ -168,7 +190,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
             const float sg = (r == RH && idx == HP) ? 1.f : -1.f;
             return make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
         });
-        if (p.len == HP && has1) {
+        if (!FULL && p.len == HP && has1) {
             // full rows: all gate loads of the pair are in flight together (they were asked into L2 above)
             float qa[HP / TPL], qb[HP / TPL];
 #pragma unroll
@@ -223,7 +245,8 @@ template <typename T, int LOG2P> static int launch_rows_fwd_w_t(const RowsArgs &
         }                                                                                                \
         rows_fwd_w_kernel<T, LOG2P, MODE><<<grid, kRowThreads, sm, st>>>(a);                             \
     } while (0)
-    if (a.b) HN_LAUNCH(0);
+    if (a.full_in) HN_LAUNCH(3);
+    else if (a.b) HN_LAUNCH(0);
     else if (a.prune_in) HN_LAUNCH(2);
     else HN_LAUNCH(1);
 #undef HN_LAUNCH
@@ -238,11 +261,10 @@ template <typename T, int LOG2P> static int launch_rows_inv_w_t(const RowsInvArg
     const long long want = ((a.rows + 1) / 2 + G - 1) / G;
     const int grid = (int)(want < 2ll * rows_sms() ? want : 2ll * rows_sms());
     if (grid <= 0) return 0;
-    static DevOnce attr;
-    if (attr.first()) {
-        cudaFuncSetAttribute(rows_inv_w_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    }
-    rows_inv_w_kernel<T, LOG2P><<<grid, kRowThreads, sm, st>>>(a);
+    static DevOnce attr[2];
+    void (*fn)(RowsInvArgs) = a.full_out ? rows_inv_w_kernel<T, LOG2P, true> : rows_inv_w_kernel<T, LOG2P, false>;
+    if (attr[a.full_out ? 1 : 0].first()) cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    fn<<<grid, kRowThreads, sm, st>>>(a);
     return 1;
 }
 

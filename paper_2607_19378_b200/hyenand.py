@@ -17,6 +17,9 @@ LIB_PATH = os.path.join(_HERE, "libhyenand.so")
 
 HYENAND_F32 = 0
 HYENAND_BF16 = 1
+HYENAND_MODE_LINEAR = 0
+HYENAND_MODE_CAUSAL = 1
+HYENAND_MODE_CIRCULAR = 2
 HYENAND_OK = 0
 HYENAND_ERR_INVALID_ARG = 1
 HYENAND_ERR_UNSUPPORTED = 2
@@ -43,6 +46,8 @@ def lib() -> ctypes.CDLL:
         vp, ip, ll = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.c_longlong
         L.hyenand_create_plan.restype = vp
         L.hyenand_create_plan.argtypes = [ctypes.c_int, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        L.hyenand_create_plan_mode.restype = vp
+        L.hyenand_create_plan_mode.argtypes = [ctypes.c_int, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int]
         L.hyenand_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.hyenand_forward_ex.argtypes = [vp, vp, vp, vp, vp, ll, vp, vp]
         L.hyenand_forward_host.argtypes = [vp, vp, vp, vp, vp, ll, vp, vp]
@@ -91,6 +96,16 @@ def _check(code: int):
 def hyenand_create_plan(ndim: int, dims, B: int, C: int, causal: int, dtype: int) -> int:
     arr = (ctypes.c_int * max(1, len(dims)))(*[int(d) for d in dims])
     h = lib().hyenand_create_plan(int(ndim), arr, int(B), int(C), int(causal), int(dtype))
+    if not h:
+        msg = hyenand_last_error()
+        code = hyenand_last_error_code() or HYENAND_ERR_INVALID_ARG
+        raise HyenaNDError(code, msg)
+    return h
+
+
+def hyenand_create_plan_mode(ndim: int, dims, B: int, C: int, mode: int, dtype: int) -> int:
+    arr = (ctypes.c_int * max(1, len(dims)))(*[int(d) for d in dims])
+    h = lib().hyenand_create_plan_mode(int(ndim), arr, int(B), int(C), int(mode), int(dtype))
     if not h:
         msg = hyenand_last_error()
         code = hyenand_last_error_code() or HYENAND_ERR_INVALID_ARG
@@ -205,13 +220,18 @@ def hyenand_forward_noalloc(dims, B: int, C: int, causal: int, dtype: int, q, k,
 class Plan:
     """Convenience owner of a plan handle (create on construction, destroy on close)."""
 
-    def __init__(self, dims, B: int, C: int, causal: bool = False, dtype=torch.float32):
+    def __init__(self, dims, B: int, C: int, causal: bool = False, dtype=torch.float32, circular: bool = False):
         self.dims = tuple(int(d) for d in dims)
-        self.B, self.C, self.causal, self.dtype = B, C, bool(causal), dtype
-        self.handle = hyenand_create_plan(len(self.dims), self.dims, B, C, int(self.causal), _DTYPES[dtype])
+        self.B, self.C, self.causal, self.dtype, self.circular = B, C, bool(causal), dtype, bool(circular)
+        if self.circular:
+            if self.causal:
+                raise ValueError("a plan is causal or circular, not both")
+            self.handle = hyenand_create_plan_mode(len(self.dims), self.dims, B, C, HYENAND_MODE_CIRCULAR, _DTYPES[dtype])
+        else:
+            self.handle = hyenand_create_plan(len(self.dims), self.dims, B, C, int(self.causal), _DTYPES[dtype])
 
     def _stride(self, h) -> int:
-        taps = tuple(L if self.causal else 2 * L - 1 for L in self.dims)
+        taps = tuple(L if (self.causal or self.circular) else 2 * L - 1 for L in self.dims)
         if tuple(h.shape) == (self.C,) + taps:
             return 0
         if tuple(h.shape) == (self.B, self.C) + taps:

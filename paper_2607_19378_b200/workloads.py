@@ -43,6 +43,7 @@ class Workload:
     filt: str = "radial"  # "l1" | "causal_exp" | "radial" | "spectral"
     alpha: Tuple[float, float] = (0.05, 1.0)
     field: str = "normal"  # "normal" | "spectral"
+    circular: bool = False  # periodic boundaries: the filter lives on the grid itself (K_n = L_n)
 
     @property
     def ndim(self) -> int:
@@ -50,7 +51,12 @@ class Workload:
 
     @property
     def taps(self) -> Tuple[int, ...]:
-        return tuple(L if self.causal else 2 * L - 1 for L in self.dims)
+        return tuple(L if (self.causal or self.circular) else 2 * L - 1 for L in self.dims)
+
+    @property
+    def mode(self) -> str:
+        """Boundary handling in the oracle's vocabulary."""
+        return "causal" if self.causal else "circular" if self.circular else "linear"
 
     @property
     def elements(self) -> int:
@@ -74,6 +80,14 @@ WORKLOADS = {
     "pde2d": Workload("pde2d", (512, 512), 4, 128, "f32", seed=4, filt="spectral", field="spectral"),
     "volume3d": Workload("volume3d", (128, 128, 128), 1, 64, "bf16", seed=5, filt="radial",
                          alpha=(0.05, 0.5)),
+}
+
+# Workloads of the rows built after the five above (not part of the default benchmark table):
+#   periodic2d  2-D 512x512 smooth fields with periodic boundaries, fp32: the circular mode of Section 3.2.1,
+#               shaped like the periodic PDE fields of Section 5.4
+EXTRA_WORKLOADS = {
+    "periodic2d": Workload("periodic2d", (512, 512), 4, 128, "f32", seed=6, filt="radial", alpha=(0.02, 0.3),
+                           field="spectral", circular=True),
 }
 
 
@@ -102,9 +116,13 @@ def _smooth_field(shape, g, device):
     return out
 
 
-def _offsets(L, causal, device):
+def _offsets(L, causal, device, circular=False):
     if causal:
         return torch.arange(L, device=device, dtype=torch.float32)
+    if circular:
+        # tap m is the displacement m mod L: its length on the periodic grid is min(m, L - m)
+        m = torch.arange(L, device=device, dtype=torch.float32)
+        return torch.minimum(m, L - m)
     return torch.arange(-(L - 1), L, device=device, dtype=torch.float32)
 
 
@@ -115,7 +133,7 @@ def make_filter(w: Workload, device="cpu") -> torch.Tensor:
     ga = _gen(w.seed, 5, device)
     alpha = torch.rand((w.C,), generator=ga, device=device) * (w.alpha[1] - w.alpha[0]) + w.alpha[0]
     alpha = alpha.reshape((w.C,) + (1,) * w.ndim)
-    offs = [_offsets(L, w.causal, device) for L in w.dims]
+    offs = [_offsets(L, w.causal, device, w.circular) for L in w.dims]
     if w.filt == "spectral":
         # same low-passed construction as the fields, built on the padded torus and cropped
         P = tuple(2 * L for L in w.dims)
@@ -164,9 +182,9 @@ def make_inputs(w: Workload, device="cpu"):
     return q, k, v, make_filter(w, device)
 
 
-def random_problem(dims, B=2, C=3, dtype="f32", causal=False, h_shared=False, seed=0, device="cpu"):
+def random_problem(dims, B=2, C=3, dtype="f32", causal=False, h_shared=False, seed=0, device="cpu", circular=False):
     """A small problem of arbitrary shape with N(0,1) inputs and a radially decaying filter."""
     w = Workload("random", tuple(int(d) for d in dims), B, C, dtype, causal=causal,
                  h_shared=h_shared, seed=seed,
-                 filt="causal_exp" if causal else "radial", alpha=(0.05, 1.0))
+                 filt="causal_exp" if causal else "radial", alpha=(0.05, 1.0), circular=circular)
     return w, make_inputs(w, device)

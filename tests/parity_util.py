@@ -47,7 +47,7 @@ def run_gpu(w, q, k, v, h, stream=None, env=None):
         old[key] = os.environ.get(key)
         os.environ[key] = val
     try:
-        plan = hn.Plan(w.dims, w.B, w.C, causal=w.causal, dtype=w.torch_dtype)
+        plan = hn.Plan(w.dims, w.B, w.C, causal=w.causal, dtype=w.torch_dtype, circular=w.circular)
     finally:
         for key, val in old.items():
             if val is None:
@@ -108,6 +108,5 @@ def assert_parity(y, ref, q, w, what=""):
 
 def check(w, q, k, v, h, full_direct=False, stream=None, env=None):
     y, path = run_gpu(w, q, k, v, h, stream=stream, env=env)
-    mode = "causal" if w.causal else "linear"
-    ref = (oracle.conv_direct if full_direct else oracle.conv_fft)(q, k, v, h, mode)
+    ref = (oracle.conv_direct if full_direct else oracle.conv_fft)(q, k, v, h, w.mode)
     return assert_parity(y, ref, q, w, what=f"path={path}")

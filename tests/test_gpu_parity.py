@@ -224,6 +224,45 @@ def test_plan_of_another_device_is_rejected():
         plan.close()
 
 
+CIRCULAR_SHAPES = [(1,), (2,), (64,), (1024,), (8192,), (4, 8), (32, 32), (64, 128), (256, 64), (1, 16), (16, 1),
+                   (2, 4, 8), (16, 16, 16), (8, 1, 32), (4, 64, 64)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shared", [False, True])
+@pytest.mark.parametrize("dims", CIRCULAR_SHAPES, ids=str)
+def test_circular_mode(dims, dtype, shared):
+    """Periodic boundaries (Section 3.2.1): the filter lives on the grid itself and the transforms run on
+    L_n points with nothing padded, pruned or cropped."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem(dims, B=2, C=3, dtype=dtype, h_shared=shared, seed=51, circular=True)
+    assert h.shape[-len(dims):] == tuple(dims)
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype, circular=True)
+    assert hn.hyenand_plan_fft_dims(plan.handle, len(dims)) == tuple(dims)
+    plan.close()
+    check(w, q, k, v, h, full_direct=int(np.prod(dims)) <= 4096)
+
+
+def test_circular_mode_wraps_around_and_rejects_other_sizes():
+    """A shifted delta filter rolls the gated input around the torus (no zero fill at the edges); grids that are
+    not powers of two, or longer than one line, are refused."""
+    from paper_2607_19378_b200 import hyenand as hn
+    dims = (8, 16)
+    w, (q, k, v, h) = W.random_problem(dims, B=1, C=2, dtype="f32", seed=52, circular=True)
+    h = torch.zeros_like(h)
+    h[..., 3, 14] = 1.0                                   # displacement (+3, -2)
+    y, _ = run_gpu(w, q, k, v, h)
+    expect = q.double() * torch.roll((k * v).double(), shifts=(3, -2), dims=(-2, -1))
+    assert oracle.rel_l2(y, expect.numpy()) < 1e-6
+    for bad in [(12,), (8, 6), (16384,)]:
+        with pytest.raises(hn.HyenaNDError) as e:
+            hn.hyenand_create_plan_mode(len(bad), bad, 1, 1, hn.HYENAND_MODE_CIRCULAR, hn.HYENAND_F32)
+        assert e.value.code == hn.HYENAND_ERR_UNSUPPORTED
+    with pytest.raises(hn.HyenaNDError) as e:
+        hn.hyenand_create_plan_mode(1, (8,), 1, 1, 3, hn.HYENAND_F32)
+    assert e.value.code == hn.HYENAND_ERR_INVALID_ARG
+
+
 def test_tiny2d_workload_full():
     w = W.WORKLOADS["tiny2d"]
     q, k, v, h = W.make_inputs(w)
