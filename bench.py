@@ -466,6 +466,77 @@ def main_ours(args):
         dist.destroy_process_group()
 
 
+# ---- the full operator of Eq. 2 (pointwise stages + long convolution) ------------------------------------
+
+def main_mixer(args):
+    """`--op mixer`: times hyenand_mixer_forward (Eq. 2) on the workload, inputs resident in HBM.  The long
+    convolution inside runs on an fp32 plan; its kernels are timed by the library, the pointwise stages are the
+    remainder."""
+    from paper_2607_19378_b200 import hyenand as hn
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    w = ALL_WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
+    q, k, v, h = W.make_inputs(w, device=device)
+    g_in = torch.ones(w.C, device=device)
+    g_out = torch.ones(w.C, device=device)
+    y = torch.empty_like(q)
+    mx = hn.Mixer(w.dims, w.B, w.C, mode=w.mode, dtype=w.torch_dtype, eps=1e-6)
+    for _ in range(max(args.warmup, 3)):
+        mx.forward(q, k, v, h, g_in, g_out, y)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    time.sleep(0.6)
+    for _ in range(3):
+        mx.forward(q, k, v, h, g_in, g_out, y)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        mx.forward(q, k, v, h, g_in, g_out, y)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    inner = hn.hyenand_mixer_plan(mx.handle)
+    hn.hyenand_plan_set_timing(inner, 2)
+    for _ in range(args.steps):
+        mx.forward(q, k, v, h, g_in, g_out, y)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    conv_ms = 0.0
+    kernels = []
+    for kid in range(hn.hyenand_plan_kernel_count(inner)):
+        name = hn.hyenand_plan_kernel_info(inner, kid, w.h_shared)[0]
+        tot, n = hn.hyenand_plan_kernel_time(inner, kid)
+        if n > 0:
+            kernels.append({"name": name, "ms_per_step": tot / args.steps, "launches_per_step": n / args.steps})
+            conv_ms += tot / args.steps
+    hn.hyenand_plan_set_timing(inner, 0)
+    status = hn.hyenand_plan_device_status(inner)
+    damage = hn.hyenand_mixer_guard_damage(mx.handle)
+    if status != 0 or damage != 0:
+        raise SystemExit(f"mixer: device status {status} / {damage} damaged guard bytes: the timing is void")
+    mx.close()
+    hbm_gbs, peak_src, sm_max = measured_peaks()
+    fp32_tf = fp32_peak_tflops(torch.cuda.get_device_properties(0).multi_processor_count, sm_max)
+    nbytes, flops, P = op_algorithmic(w)
+    t_hbm, t_alu = nbytes / (hbm_gbs * 1e9) * 1e3, flops / (fp32_tf * 1e12) * 1e3
+    print(json.dumps({
+        "metric": "hyenand_mixer_throughput", "value": w.elements / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "op": "Eq. 2: RMSNorm(Sigmoid(v) * (K conv RMSNorm(l2(q) * SiLU(k))))",
+                   "dims": list(w.dims), "B": w.B, "C": w.C, "mode": w.mode},
+        "stages": {"long_convolution_ms": conv_ms, "pointwise_and_widening_ms": ms - conv_ms, "conv_kernels": kernels},
+        "op_roofline": {"t_hbm_ms": t_hbm, "t_fp32_ms": t_alu, "roofline_ms": max(t_hbm, t_alu),
+                        "frac": max(t_hbm, t_alu) / ms,
+                        "note": "minimal bytes and transform flops of the long convolution; the pointwise stages add no minimal traffic"},
+        "clocks": clocks, "device_status": status, "guard_damage": damage}))
+
+
 # ---- reference arm: the CPU oracle ----------------------------------------------------------------
 
 def main_reference(args):
@@ -521,8 +592,12 @@ if __name__ == "__main__":
     ap.add_argument("--no-all", action="store_true", help="skip the table over the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-cufft", action="store_true", help="skip the torch.fft (cuFFT) composition reference point")
+    ap.add_argument("--op", default="conv", choices=["conv", "mixer"],
+                    help="conv: the gated long convolution (default, the benchmark line); mixer: the full operator of Eq. 2")
     a = ap.parse_args()
     if a.impl == "reference":
         main_reference(a)
+    elif a.op == "mixer":
+        main_mixer(a)
     else:
         main_ours(a)

@@ -157,6 +157,31 @@ int hyenand_plan_groups(const hyenand_plan *plan, long long *slices_per_group, i
 
 
 /*
+ * The full HyenaND operator, Eq. 2 (Section 3.2):
+ *
+ *     y = RMSNorm_out( Sigmoid(v) * ( K conv RMSNorm_in( l2(q) * SiLU(k) ) ) )
+ *
+ * q, k, v are the projected inputs [B][C][L_1]..[L_N], h the kernel K laid out as for hyenand_forward_ex, g_in and
+ * g_out the C fp32 weights of the two RMSNorms (device pointers).  l2 and both RMSNorms act per token (one grid
+ * position of one batch entry) across the C channels: l2(q) = q / max(||q||_2, 1e-12); RMSNorm(x) = x /
+ * sqrt(mean_c(x^2) + eps) * g, eps as given at creation (>= 0).  The pointwise stages are kernels of their own before
+ * and after the long convolution; everything between the first read of q, k, v and the store of y stays fp32 (the
+ * convolution runs on an fp32 plan even when the I/O type is bf16, with h widened once per call), so y carries one
+ * rounding.  mode: HYENAND_MODE_*.  The object owns an fp32 plan and fp32 scratch for at most 2 GiB worth of batch
+ * entries per pass; hyenand_mixer_plan exposes the inner plan for the reporting helpers (do not destroy it).
+ * Errors and stream semantics as hyenand_forward_ex.  hyenand_mixer_guard_damage: as hyenand_plan_guard_damage, over
+ * the scratch and the inner plan.
+ */
+typedef struct hyenand_mixer hyenand_mixer;
+hyenand_mixer *hyenand_mixer_create(int ndim, const int *dims, int B, int C, int mode, int dtype, float eps);
+int hyenand_mixer_forward(hyenand_mixer *mixer, const void *q, const void *k, const void *v, const void *h,
+                          long long h_batch_stride_elems, const float *g_in, const float *g_out, void *y,
+                          void *cuda_stream);
+hyenand_plan *hyenand_mixer_plan(hyenand_mixer *mixer);
+long long hyenand_mixer_guard_damage(hyenand_mixer *mixer);
+void hyenand_mixer_destroy(hyenand_mixer *mixer);
+
+/*
  * Forward pass that allocates nothing (no counterpart in the paper: an integration aid).
  *
  * For callers that cannot allocate device memory when they need the operator -- host code running

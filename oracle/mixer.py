@@ -40,8 +40,10 @@ def rms_norm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
     return x / np.sqrt(ms + eps) * g.reshape(shape)
 
 
-def hyena_mixer(q, k, v, h, g_in, g_out, eps: float = 1e-6, mode: str = "linear", direct: bool = False) -> np.ndarray:
-    """Eq. 2 on [B, C, L_1..L_N] tensors; h as for the convolution oracle; g_in, g_out: [C]."""
+def hyena_mixer(q, k, v, h, g_in, g_out, eps: float = 1e-6, mode: str = "linear", direct: bool = False,
+                parts: bool = False):
+    """Eq. 2 on [B, C, L_1..L_N] tensors; h as for the convolution oracle; g_in, g_out: [C].
+    parts=True also returns the gated convolution (the argument of the last RMSNorm), for error bounds in tests."""
     q, k, v = (to_f64(t) for t in (q, k, v))
     g_in, g_out = to_f64(g_in), to_f64(g_out)
     inner = l2_normalise(q) * silu(k)                       # l2(q) * SiLU(k)
@@ -49,4 +51,5 @@ def hyena_mixer(q, k, v, h, g_in, g_out, eps: float = 1e-6, mode: str = "linear"
     one = np.ones_like(z)
     conv = (conv_direct if direct else conv_fft)(one, z, one, h, mode)     # K conv z  (gates of the conv oracle = 1)
     gated = sigmoid(v) * conv                               # outer gate
-    return rms_norm(gated, g_out, eps)                      # RMSNorm before the residual addition
+    y = rms_norm(gated, g_out, eps)                         # RMSNorm before the residual addition
+    return (y, gated) if parts else y

@@ -15,6 +15,7 @@
 #include "core_tma.cuh"
 #include "tma_util.cuh"
 #include "fused2d.cuh"
+#include "mixer.cuh"
 
 using namespace hn;
 
@@ -950,6 +951,143 @@ extern "C" int hyenand_plan_kernel_time(hyenand_plan *p, int kid, double *total_
     *total_ms = p->prof.ms[kid];
     *launches = (double)p->prof.launches[kid];
     return HYENAND_OK;
+}
+
+// ---- the full HyenaND operator (Eq. 2): pointwise stages around the long convolution -----------------
+//
+// The long convolution runs on an fp32 plan whatever the I/O type, so that nothing between the first read of
+// q, k, v and the final store of y is rounded below fp32: the pre-stage writes its three results in fp32, the
+// kernel h is widened once per call when the I/O type is bf16, and the post-stage reads the gated convolution
+// in fp32.  Batches are worked off in groups of batch entries that bound the fp32 scratch.
+
+struct hyenand_mixer {
+    hyenand_plan *plan;               // fp32 plan over nb batch entries
+    int B, C, dtype, nb;              // nb: batch entries per pass
+    long long L, kvol;
+    float eps;
+    float *qz, *kz, *vz, *oz, *h32;   // scratch, fp32 (h32 only for bf16 I/O)
+    GuardedAllocs allocs;
+    int device;
+};
+
+extern "C" void hyenand_mixer_destroy(hyenand_mixer *m)
+{
+    if (!m) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != m->device) cudaSetDevice(m->device);
+    hyenand_destroy_plan(m->plan);
+    guarded_free_all(&m->allocs);
+    if (cur != m->device) cudaSetDevice(cur);
+    delete m;
+}
+
+extern "C" hyenand_mixer *hyenand_mixer_create(int ndim, const int *dims, int B, int C, int mode, int dtype, float eps)
+{
+    g_err[0] = 0;
+    if (dtype != HYENAND_F32 && dtype != HYENAND_BF16) { fail(HYENAND_ERR_INVALID_ARG, "unknown dtype %d", dtype); return nullptr; }
+    if (!(eps >= 0.f)) { fail(HYENAND_ERR_INVALID_ARG, "eps must be >= 0"); return nullptr; }
+    if (ndim < 1 || ndim > 3 || !dims || B < 1 || C < 1) { fail(HYENAND_ERR_INVALID_ARG, "bad geometry"); return nullptr; }
+    long long L = 1;
+    for (int a = 0; a < ndim; ++a) {
+        if (dims[a] < 1) { fail(HYENAND_ERR_INVALID_ARG, "dims[%d] = %d must be >= 1", a, dims[a]); return nullptr; }
+        L *= dims[a];
+    }
+    // batch entries per pass: four fp32 tensors of nb*C*L elements, at most 2 GiB together
+    long long nb = (2ll << 30) / (16ll * C * L);
+    if (const char *e = getenv("HYENAND_MIXER_MAX_BATCH")) { const long long v = atoll(e); if (v > 0 && v < nb) nb = v; }   // development aid
+    if (nb < 1) nb = 1;
+    if (nb > B) nb = B;
+    hyenand_plan *plan = hyenand_create_plan_mode(ndim, dims, (int)nb, C, mode, HYENAND_F32);
+    if (!plan) return nullptr;
+    hyenand_mixer *m = new hyenand_mixer();
+    memset(m, 0, sizeof(*m));
+    m->plan = plan; m->B = B; m->C = C; m->dtype = dtype; m->nb = (int)nb; m->L = L; m->kvol = plan->kvol; m->eps = eps;
+    m->device = plan->device;
+    const size_t n = (size_t)nb * C * L * sizeof(float);
+    cudaError_t e = guarded_alloc(&m->allocs, (void **)&m->qz, n);
+    if (e == cudaSuccess) e = guarded_alloc(&m->allocs, (void **)&m->kz, n);
+    if (e == cudaSuccess) e = guarded_alloc(&m->allocs, (void **)&m->vz, n);
+    if (e == cudaSuccess) e = guarded_alloc(&m->allocs, (void **)&m->oz, n);
+    if (e == cudaSuccess && dtype == HYENAND_BF16)
+        e = guarded_alloc(&m->allocs, (void **)&m->h32, (size_t)nb * C * m->kvol * sizeof(float));
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        fail(HYENAND_ERR_ALLOC, "scratch of the pointwise stages: %s", cudaGetErrorString(e));
+        hyenand_mixer_destroy(m);
+        return nullptr;
+    }
+    return m;
+}
+
+extern "C" int hyenand_mixer_forward(hyenand_mixer *m, const void *q, const void *k, const void *v, const void *h,
+                                     long long h_batch_stride_elems, const float *g_in, const float *g_out, void *y,
+                                     void *cuda_stream)
+{
+    g_err[0] = 0;
+    if (!m) return fail(HYENAND_ERR_INVALID_ARG, "mixer is NULL");
+    if (!q || !k || !v || !h || !y || !g_in || !g_out) return fail(HYENAND_ERR_INVALID_ARG, "q, k, v, h, g_in, g_out, y must be non-NULL");
+    const void *ptrs[5] = {q, k, v, h, y};
+    for (int i = 0; i < 5; ++i)
+        if (((uintptr_t)ptrs[i]) & 15) return fail(HYENAND_ERR_INVALID_ARG, "pointer %d is not 16-byte aligned", i);
+    hyenand_plan *p = m->plan;
+    bool shared = false;
+    int e = check_stride(p, h_batch_stride_elems, &shared);
+    if (!e) e = check_device(p);
+    if (e) return e;
+    const size_t es = elsize(m->dtype);
+    {
+        // y must not overlap an input (geometry of the whole batch, in the I/O type)
+        const size_t nbytes = (size_t)m->B * m->C * m->L * es, hbytes = (size_t)(shared ? 1 : m->B) * m->C * m->kvol * es;
+        const char *yb = (const char *)y;
+        const void *ins[4] = {q, k, v, h};
+        for (int i = 0; i < 4; ++i) {
+            const char *ib = (const char *)ins[i];
+            const size_t ilen = i == 3 ? hbytes : nbytes;
+            if (yb < ib + ilen && ib < yb + nbytes) return fail(HYENAND_ERR_INVALID_ARG, "y overlaps input %d", i);
+        }
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t slab = (size_t)m->C * m->L;                        // elements per batch entry
+    const float *hf = (const float *)h;
+    if (m->dtype == HYENAND_BF16 && shared) {
+        launch_widen(h, m->dtype, (long long)m->C * m->kvol, m->h32, st);
+        hf = m->h32;
+    }
+    for (int b0 = 0; b0 < m->B; b0 += m->nb) {
+        const int n = m->B - b0 < m->nb ? m->B - b0 : m->nb;
+        const char *qb = (const char *)q + (size_t)b0 * slab * es, *kb = (const char *)k + (size_t)b0 * slab * es,
+                   *vb = (const char *)v + (size_t)b0 * slab * es;
+        launch_mixer_pre(qb, kb, vb, g_in, m->eps, m->dtype, n, m->C, m->L, m->qz, m->kz, m->vz, st);
+        const float *hb = hf;
+        if (!shared) {
+            if (m->dtype == HYENAND_BF16) {
+                launch_widen((const char *)h + (size_t)b0 * m->C * m->kvol * es, m->dtype, (long long)n * m->C * m->kvol, m->h32, st);
+                hb = m->h32;
+            } else {
+                hb = (const float *)h + (size_t)b0 * m->C * m->kvol;
+            }
+        }
+        int launches = 0;
+        p->r0 = 0; p->r1 = (long long)n * m->C;
+        e = run_forward(p, m->qz, m->kz, m->vz, hb, shared, m->oz, st, &launches);
+        p->r0 = 0; p->r1 = (long long)p->B * p->C;
+        if (e) return e;
+        launch_mixer_post(m->oz, g_out, m->eps, m->dtype, n, m->C, m->L, (char *)y + (size_t)b0 * slab * es, st);
+    }
+    cudaError_t ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(HYENAND_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(ce));
+    return HYENAND_OK;
+}
+
+extern "C" hyenand_plan *hyenand_mixer_plan(hyenand_mixer *m) { return m ? m->plan : nullptr; }
+
+extern "C" long long hyenand_mixer_guard_damage(hyenand_mixer *m)
+{
+    g_err[0] = 0;
+    if (!m) { fail(HYENAND_ERR_INVALID_ARG, "mixer is NULL"); return -1; }
+    const long long a = guard_damage(&m->allocs), b = guard_damage(&m->plan->allocs);
+    return (a < 0 || b < 0) ? -1 : a + b;
 }
 
 // ---- forward without any device allocation --------------------------------------------------

@@ -74,6 +74,16 @@ def lib() -> ctypes.CDLL:
         L.hyenand_noalloc_max_bytes.restype = ctypes.c_size_t
         L.hyenand_forward_noalloc.argtypes = [ctypes.c_int, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                               vp, vp, vp, vp, ll, vp, vp]
+        fp = ctypes.POINTER(ctypes.c_float)
+        L.hyenand_mixer_create.restype = vp
+        L.hyenand_mixer_create.argtypes = [ctypes.c_int, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_float]
+        L.hyenand_mixer_forward.argtypes = [vp, vp, vp, vp, vp, ll, vp, vp, vp, vp]
+        L.hyenand_mixer_plan.restype = vp
+        L.hyenand_mixer_plan.argtypes = [vp]
+        L.hyenand_mixer_guard_damage.restype = ll
+        L.hyenand_mixer_guard_damage.argtypes = [vp]
+        L.hyenand_mixer_destroy.restype = None
+        L.hyenand_mixer_destroy.argtypes = [vp]
         L.hyenand_plan_set_timing.argtypes = [vp, ctypes.c_int]
         L.hyenand_plan_kernel_time.argtypes = [vp, ctypes.c_int, dpp, dpp]
         _lib = L
@@ -215,6 +225,72 @@ def hyenand_forward_noalloc(dims, B: int, C: int, causal: int, dtype: int, q, k,
     _check(lib().hyenand_forward_noalloc(len(dims), arr, int(B), int(C), int(causal), int(dtype),
                                          q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
                                          int(h_batch_stride_elems), y.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_mixer_create(ndim: int, dims, B: int, C: int, mode: int, dtype: int, eps: float) -> int:
+    arr = (ctypes.c_int * max(1, len(dims)))(*[int(d) for d in dims])
+    h = lib().hyenand_mixer_create(int(ndim), arr, int(B), int(C), int(mode), int(dtype), float(eps))
+    if not h:
+        raise HyenaNDError(hyenand_last_error_code() or HYENAND_ERR_INVALID_ARG, hyenand_last_error())
+    return h
+
+
+def hyenand_mixer_forward(mixer: int, q, k, v, h, h_batch_stride_elems: int, g_in, g_out, y, stream=None) -> None:
+    _check(lib().hyenand_mixer_forward(mixer, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
+                                       int(h_batch_stride_elems), g_in.data_ptr(), g_out.data_ptr(), y.data_ptr(),
+                                       _stream_ptr(stream)))
+
+
+def hyenand_mixer_plan(mixer: int) -> int:
+    return lib().hyenand_mixer_plan(mixer)
+
+
+def hyenand_mixer_guard_damage(mixer: int) -> int:
+    return int(lib().hyenand_mixer_guard_damage(mixer))
+
+
+def hyenand_mixer_destroy(mixer: int) -> None:
+    lib().hyenand_mixer_destroy(mixer)
+
+
+class Mixer:
+    """Owner of a hyenand_mixer handle: the full operator of Eq. 2 (pointwise stages + long convolution)."""
+
+    def __init__(self, dims, B: int, C: int, mode: str = "linear", dtype=torch.float32, eps: float = 1e-6):
+        self.dims = tuple(int(d) for d in dims)
+        self.B, self.C, self.mode, self.dtype = B, C, mode, dtype
+        code = {"linear": HYENAND_MODE_LINEAR, "causal": HYENAND_MODE_CAUSAL, "circular": HYENAND_MODE_CIRCULAR}[mode]
+        self.handle = hyenand_mixer_create(len(self.dims), self.dims, B, C, code, _DTYPES[dtype], eps)
+
+    def forward(self, q, k, v, h, g_in, g_out, y=None, stream=None):
+        taps = tuple(2 * L - 1 if self.mode == "linear" else L for L in self.dims)
+        if tuple(h.shape) == (self.C,) + taps:
+            stride = 0
+        elif tuple(h.shape) == (self.B, self.C) + taps:
+            stride = self.C * h[0, 0].numel()
+        else:
+            raise ValueError(f"h has shape {tuple(h.shape)}")
+        for t in (q, k, v, h):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == self.dtype):
+                raise ValueError("inputs must be contiguous CUDA tensors of the mixer's dtype")
+        for g in (g_in, g_out):
+            if not (g.is_cuda and g.is_contiguous() and g.dtype == torch.float32 and g.numel() == self.C):
+                raise ValueError("g_in, g_out must be contiguous fp32 CUDA tensors of C elements")
+        if y is None:
+            y = torch.empty_like(q)
+        hyenand_mixer_forward(self.handle, q, k, v, h, stride, g_in, g_out, y, stream)
+        return y
+
+    def close(self):
+        if self.handle:
+            hyenand_mixer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class Plan:
