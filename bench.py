@@ -537,6 +537,71 @@ def main_mixer(args):
         "clocks": clocks, "device_status": status, "guard_damage": damage}))
 
 
+# ---- kernel synthesis ---------------------------------------------------------------------------------------
+
+def main_synth(args):
+    """`--op synth`: times hyenand_synthesize_kernel for the workload's kernel grid (SIREN of `--hidden` units and
+    `--layers` hidden layers, FiLM-modulated per batch entry when the kernel is per sample).  Bound: FP32 ALUs
+    (one fused multiply-add per weight and tap), reported against the derived FP32 peak."""
+    from paper_2607_19378_b200 import hyenand as hn
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = ALL_WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
+    N, Hf, J = w.ndim, args.hidden, args.layers
+    Bk = 1 if w.h_shared else w.B
+    g = torch.Generator(device=dev).manual_seed(w.seed)
+    r = lambda *shape: torch.rand(shape, generator=g, device=dev) * 2 - 1
+    W1, b1, om = r(Hf, N) / math.sqrt(N), r(Hf) * 0.5, (r(Hf) + 1) * 15 + 1
+    Wh, bh = r(max(J - 1, 1), Hf, Hf) * math.sqrt(6 / Hf), r(max(J - 1, 1), Hf) * 0.3
+    Wout, bout = r(w.C, Hf) * math.sqrt(6 / Hf), r(w.C) * 0.1
+    gamma, beta = (1 + 0.3 * r(Bk, J, Hf), 0.3 * r(Bk, J, Hf)) if not w.h_shared else (None, None)
+    window = (r(w.C) + 1.5) if w.causal else torch.exp(r(N, w.C))
+    h = torch.empty((Bk, w.C) + w.taps, dtype=w.torch_dtype, device=dev)
+    mode = {"linear": 0, "causal": 1, "circular": 2}[w.mode]
+    code = hn.HYENAND_F32 if w.dtype == "f32" else hn.HYENAND_BF16
+
+    def run():
+        hn.hyenand_synthesize_kernel(w.dims, mode, Bk, w.C, Hf, J, W1, b1, om, Wh if J > 1 else None, bh if J > 1 else None,
+                                     Wout, bout, gamma, beta, window, code, h)
+    for _ in range(max(args.warmup, 3)):
+        run()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    time.sleep(0.6)
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1) / args.steps
+    clocks = sampler.stop(t0, t1)
+    taps = Bk * math.prod(w.taps)
+    flops = 2.0 * taps * (Hf * (N + 1) + (J - 1) * Hf * (Hf + 1) + w.C * (Hf + 1))
+    hbm_gbs, peak_src, sm_max = measured_peaks()
+    fp32_tf = fp32_peak_tflops(torch.cuda.get_device_properties(0).multi_processor_count, sm_max)
+    out_bytes = taps * w.C * (4 if w.dtype == "f32" else 2)
+    ach = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "hyenand_kernel_synthesis_throughput", "value": taps * w.C / (ms * 1e-3) / 1e9, "unit": "Gtap/s (taps x channels)",
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "op": "K(x) = window * SIREN(coordinates; FiLM)", "dims": list(w.dims), "taps": list(w.taps),
+                   "kernels": Bk, "C": w.C, "hidden": Hf, "layers": J, "mode": w.mode},
+        "roofline": {"kernel": "synth", "bound": "alu", "achieved": ach, "peak": fp32_tf, "unit": "TFLOP/s", "frac": ach / fp32_tf,
+                     "traffic": None, "peak_source": "derived: 2 x 128 FP32 lanes x SMs x max SM clock",
+                     "flops": "2 per weight and tap (fused multiply-adds of the three layer kinds); sines and exponentials not counted",
+                     "t_hbm_ms_for_the_output": out_bytes / (hbm_gbs * 1e9) * 1e3},
+        "clocks": clocks}))
+
+
 # ---- reference arm: the CPU oracle ----------------------------------------------------------------
 
 def main_reference(args):
@@ -592,12 +657,17 @@ if __name__ == "__main__":
     ap.add_argument("--no-all", action="store_true", help="skip the table over the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-cufft", action="store_true", help="skip the torch.fft (cuFFT) composition reference point")
-    ap.add_argument("--op", default="conv", choices=["conv", "mixer"],
-                    help="conv: the gated long convolution (default, the benchmark line); mixer: the full operator of Eq. 2")
+    ap.add_argument("--op", default="conv", choices=["conv", "mixer", "synth"],
+                    help="conv: the gated long convolution (default, the benchmark line); mixer: the full operator of Eq. 2; "
+                         "synth: the kernel synthesis K(x)")
+    ap.add_argument("--hidden", type=int, default=32, help="--op synth: width of the SIREN")
+    ap.add_argument("--layers", type=int, default=2, help="--op synth: hidden layers of the SIREN")
     a = ap.parse_args()
     if a.impl == "reference":
         main_reference(a)
     elif a.op == "mixer":
         main_mixer(a)
+    elif a.op == "synth":
+        main_synth(a)
     else:
         main_ours(a)

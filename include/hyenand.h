@@ -182,6 +182,32 @@ long long hyenand_mixer_guard_damage(hyenand_mixer *mixer);
 void hyenand_mixer_destroy(hyenand_mixer *mixer);
 
 /*
+ * Kernel synthesis: evaluates the input-dependent convolution kernel of Section 3.2.1 / 3.2.2,
+ *
+ *     K(x)[b][c][i] = w_c(c_i) * f_theta(c_i; gamma_b, beta_b)[c],
+ *
+ * on the tap grid and writes it as h in the layout hyenand_forward reads ([B][C][K_1]..[K_N], I/O dtype).
+ * f_theta is the SIREN of Eq. 3 with `layers` hidden layers of width `hidden` and a frequency VECTOR omega0,
+ * FiLM-modulated after every sine (Eq. 4):
+ *     a_1 = gamma_1 * sin(omega0 * (W1 c_i + b1)) + beta_1,   a_j = gamma_j * sin(Wh_j a_{j-1} + bh_j) + beta_j,
+ *     f = Wout a_J + bout.
+ * Eq. 3 prints no biases: pass zeros for it.  gamma, beta ([B][layers][hidden]) are what the FiLM network makes of
+ * the control variable z(x) (that small per-sample network is the caller's); NULL for both = identity modulation,
+ * the static kernel.  w is the Gaussian window of Eq. 6 with window = sigma [N][C] (per axis and channel), or, for
+ * mode CAUSAL, exp(-alpha_c |c_i|) with window = alpha [C] (Appendix A.3; taps exist only for displacements >= 0).
+ * Coordinates per axis: LINEAR displacement d in [-(L-1), L-1] -> d/(L-1); CAUSAL t -> t/(L-1); CIRCULAR tap m ->
+ * (m <= L/2 ? m : m - L) / (L/2); 0 when L = 1.  Window and SIREN share them.
+ * All parameter arrays are fp32 DEVICE pointers, row-major: W1 [hidden][N], b1 [hidden], omega0 [hidden],
+ * Wh [layers-1][hidden][hidden], bh [layers-1][hidden], Wout [C][hidden], bout [C].  hidden <= 64, layers <= 8.
+ * fp32 arithmetic with accurate sine and exponential; the error of the first sine grows with |omega0 (W1 c + b1)|
+ * (fp32 carries relative precision), about 1e-7 per radian.  Enqueues one kernel on cuda_stream; no allocation.
+ */
+int hyenand_synthesize_kernel(int ndim, const int *dims, int mode, int B, int C, int hidden, int layers,
+                              const float *W1, const float *b1, const float *omega0, const float *Wh, const float *bh,
+                              const float *Wout, const float *bout, const float *gamma, const float *beta,
+                              const float *window, int dtype, void *h, void *cuda_stream);
+
+/*
  * Forward pass that allocates nothing (no counterpart in the paper: an integration aid).
  *
  * For callers that cannot allocate device memory when they need the operator -- host code running

@@ -17,8 +17,10 @@ NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v"]
 # --use_fast_math only affects division/transcendental intrinsics and denormal flushing;
-# the kernels use neither divisions nor sin/cos on the data path (twiddles come from
-# tables computed in double on the host).
+# the transform kernels use neither divisions nor sin/cos on the data path (twiddles come from
+# tables computed in double on the host).  Sources that evaluate sines and exponentials of the data
+# (kernel synthesis) are compiled without it.
+PRECISE = {"synth.cu"}
 
 
 def _sources():
@@ -48,7 +50,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     def compile_one(job):
         s, o = job
-        r = subprocess.run([NVCC] + FLAGS + ["-c", s, "-o", o], capture_output=True, text=True)
+        flags = [f for f in FLAGS if not (f == "--use_fast_math" and os.path.basename(s) in PRECISE)]
+        r = subprocess.run([NVCC] + flags + ["-c", s, "-o", o], capture_output=True, text=True)
         with open(o[:-2] + ".ptxas.log", "w") as f:
             f.write(r.stderr)
         if r.returncode != 0:

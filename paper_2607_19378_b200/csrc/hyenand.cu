@@ -16,6 +16,7 @@
 #include "tma_util.cuh"
 #include "fused2d.cuh"
 #include "mixer.cuh"
+#include "synth.cuh"
 
 using namespace hn;
 
@@ -1088,6 +1089,42 @@ extern "C" long long hyenand_mixer_guard_damage(hyenand_mixer *m)
     if (!m) { fail(HYENAND_ERR_INVALID_ARG, "mixer is NULL"); return -1; }
     const long long a = guard_damage(&m->allocs), b = guard_damage(&m->plan->allocs);
     return (a < 0 || b < 0) ? -1 : a + b;
+}
+
+// ---- kernel synthesis ---------------------------------------------------------------------------------
+
+extern "C" int hyenand_synthesize_kernel(int ndim, const int *dims, int mode, int B, int C, int hidden, int layers,
+                                         const float *W1, const float *b1, const float *omega0, const float *Wh,
+                                         const float *bh, const float *Wout, const float *bout, const float *gamma,
+                                         const float *beta, const float *window, int dtype, void *h, void *cuda_stream)
+{
+    g_err[0] = 0;
+    if (ndim < 1 || ndim > 3 || !dims) return fail(HYENAND_ERR_INVALID_ARG, "ndim must be 1, 2 or 3 and dims non-NULL");
+    if (mode != HYENAND_MODE_LINEAR && mode != HYENAND_MODE_CAUSAL && mode != HYENAND_MODE_CIRCULAR)
+        return fail(HYENAND_ERR_INVALID_ARG, "unknown boundary mode %d", mode);
+    if (mode == HYENAND_MODE_CAUSAL && ndim != 1) return fail(HYENAND_ERR_UNSUPPORTED, "causal kernels are defined for 1-D grids only");
+    if (B < 1 || C < 1) return fail(HYENAND_ERR_INVALID_ARG, "B and C must be >= 1");
+    if (dtype != HYENAND_F32 && dtype != HYENAND_BF16) return fail(HYENAND_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (!synth_supported(hidden, layers))
+        return fail(HYENAND_ERR_UNSUPPORTED, "hidden width must be 1..64 and the number of hidden layers 1..8 (got %d, %d)", hidden, layers);
+    if (!W1 || !b1 || !omega0 || !Wout || !bout || !window || !h || (layers > 1 && (!Wh || !bh)))
+        return fail(HYENAND_ERR_INVALID_ARG, "a parameter pointer is NULL");
+    if ((gamma == nullptr) != (beta == nullptr)) return fail(HYENAND_ERR_INVALID_ARG, "gamma and beta are given together or not at all");
+    if (((uintptr_t)h) & 15) return fail(HYENAND_ERR_INVALID_ARG, "h is not 16-byte aligned");
+    SynthArgs a{};
+    a.ndim = ndim; a.mode = mode; a.B = B; a.C = C; a.hidden = hidden; a.layers = layers;
+    for (int x = 0; x < 3; ++x) { a.L[x] = 1; a.K[x] = 1; }
+    for (int x = 0; x < ndim; ++x) {
+        if (dims[x] < 1) return fail(HYENAND_ERR_INVALID_ARG, "dims[%d] = %d must be >= 1", x, dims[x]);
+        a.L[3 - ndim + x] = dims[x];
+        a.K[3 - ndim + x] = mode == HYENAND_MODE_LINEAR ? 2 * dims[x] - 1 : dims[x];
+    }
+    a.W1 = W1; a.b1 = b1; a.omega0 = omega0; a.Wh = Wh; a.bh = bh; a.Wout = Wout; a.bout = bout;
+    a.gamma = gamma; a.beta = beta; a.window = window; a.h = h; a.dtype = dtype;
+    if (launch_synth(a, (cudaStream_t)cuda_stream) < 0) return fail(HYENAND_ERR_UNSUPPORTED, "kernel grid too large for one launch");
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(HYENAND_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    return HYENAND_OK;
 }
 
 // ---- forward without any device allocation --------------------------------------------------

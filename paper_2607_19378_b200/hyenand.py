@@ -84,6 +84,7 @@ def lib() -> ctypes.CDLL:
         L.hyenand_mixer_guard_damage.argtypes = [vp]
         L.hyenand_mixer_destroy.restype = None
         L.hyenand_mixer_destroy.argtypes = [vp]
+        L.hyenand_synthesize_kernel.argtypes = [ctypes.c_int, ip] + [ctypes.c_int] * 5 + [vp] * 10 + [ctypes.c_int, vp, vp]
         L.hyenand_plan_set_timing.argtypes = [vp, ctypes.c_int]
         L.hyenand_plan_kernel_time.argtypes = [vp, ctypes.c_int, dpp, dpp]
         _lib = L
@@ -251,6 +252,17 @@ def hyenand_mixer_guard_damage(mixer: int) -> int:
 
 def hyenand_mixer_destroy(mixer: int) -> None:
     lib().hyenand_mixer_destroy(mixer)
+
+
+def hyenand_synthesize_kernel(dims, mode: int, B: int, C: int, hidden: int, layers: int, W1, b1, omega0, Wh, bh, Wout,
+                              bout, gamma, beta, window, dtype: int, h, stream=None) -> None:
+    """K(x) on the tap grid of `dims` into h (device tensor [B, C, K..]); parameters: fp32 device tensors, gamma and
+    beta may both be None (static kernel), Wh and bh may be None when layers == 1."""
+    arr = (ctypes.c_int * max(1, len(dims)))(*[int(d) for d in dims])
+    ptr = lambda t: None if t is None else t.data_ptr()
+    _check(lib().hyenand_synthesize_kernel(len(dims), arr, int(mode), int(B), int(C), int(hidden), int(layers),
+                                           ptr(W1), ptr(b1), ptr(omega0), ptr(Wh), ptr(bh), ptr(Wout), ptr(bout),
+                                           ptr(gamma), ptr(beta), ptr(window), int(dtype), h.data_ptr(), _stream_ptr(stream)))
 
 
 class Mixer:

@@ -1,0 +1,136 @@
+"""GPU parity of the kernel synthesis (hyenand_synthesize_kernel) against oracle/kernel_synthesis.py, and the
+synthesised kernel fed straight into the long convolution.
+
+Gates on K(x): whole-tensor rel-L2 against the unrounded fp64 oracle <= 1e-5 (fp32 output), <= 2e-3 and 1.1 x the
+output rounding (bf16 output); element-wise |K - ref| <= R |ref| + 2e-5 * max|f| * w (fp32 network arithmetic: the
+first sine takes arguments of up to about 40 radians here, 1e-7 per radian, then two or three more layers)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import kernel_synthesis as ks
+from parity_util import ELEM_R, TOL
+
+pytestmark = pytest.mark.gpu
+
+MODES = {"linear": 0, "causal": 1, "circular": 2}
+
+
+def make_params(N, Hf, J, C, B, mode, seed, film=True):
+    g = np.random.default_rng(seed)
+    p = dict(W1=g.uniform(-1, 1, (Hf, N)) / math.sqrt(N), b1=g.uniform(-0.5, 0.5, Hf), omega0=g.uniform(1, 30, Hf),
+             Wh=g.uniform(-1, 1, (max(J - 1, 0), Hf, Hf)) * math.sqrt(6 / Hf), bh=g.uniform(-0.3, 0.3, (max(J - 1, 0), Hf)),
+             Wout=g.uniform(-1, 1, (C, Hf)) * math.sqrt(6 / Hf), bout=g.uniform(-0.1, 0.1, C))
+    if film:
+        p["gamma"] = 1 + 0.3 * g.standard_normal((B, J, Hf))
+        p["beta"] = 0.3 * g.standard_normal((B, J, Hf))
+    else:
+        p["gamma"] = p["beta"] = None
+    p["window"] = g.uniform(0.5, 4.0, C) if mode == "causal" else np.exp(g.uniform(math.log(0.1), math.log(2.0), (N, C)))
+    # the oracle sees exactly the fp32 values the GPU gets
+    return {k: (None if v is None else np.asarray(v, dtype=np.float32)) for k, v in p.items()}
+
+
+def gpu_synthesize(dims, mode, B, C, Hf, J, p, dtype):
+    from paper_2607_19378_b200 import hyenand as hn
+    dev = {k: (None if v is None else torch.from_numpy(v).contiguous().cuda()) for k, v in p.items()}
+    taps = tuple(2 * L - 1 if mode == "linear" else L for L in dims)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    n = B * C * int(np.prod(taps))
+    big = torch.full((n + 512,), 7.0, dtype=tdt, device="cuda")
+    h = big[256:256 + n].view((B, C) + taps)
+    h.fill_(float("nan"))
+    hn.hyenand_synthesize_kernel(dims, MODES[mode], B, C, Hf, J, dev["W1"], dev["b1"], dev["omega0"], dev["Wh"] if J > 1 else None,
+                                 dev["bh"] if J > 1 else None, dev["Wout"], dev["bout"], dev["gamma"], dev["beta"], dev["window"],
+                                 hn.HYENAND_F32 if dtype == "f32" else hn.HYENAND_BF16, h)
+    torch.cuda.synchronize()
+    assert bool((big[:256] == 7.0).all()) and bool((big[256 + n:] == 7.0).all()), "the kernel wrote outside h"
+    return h
+
+
+def oracle_synthesize(dims, mode, B, J, Hf, p):
+    gamma = p["gamma"] if p["gamma"] is not None else np.ones((B, J, Hf))
+    beta = p["beta"] if p["beta"] is not None else np.zeros((B, J, Hf))
+    return ks.synthesize(dims, mode, p["W1"], p["b1"], p["omega0"], p["Wh"], p["bh"], p["Wout"], p["bout"], gamma, beta, p["window"])
+
+
+CASES = [((300,), "causal", 2, 5, 16, 2), ((1000,), "linear", 1, 3, 32, 3), ((17, 20), "linear", 2, 4, 16, 2),
+         ((32, 32), "circular", 2, 3, 8, 1), ((64, 64), "linear", 2, 40, 32, 2), ((9, 10, 11), "linear", 2, 3, 24, 3),
+         ((5, 3, 2), "linear", 3, 70, 64, 2), ((1,), "linear", 1, 2, 4, 1), ((2, 1, 3), "linear", 1, 1, 33, 4)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dims,mode,B,C,Hf,J", CASES, ids=str)
+def test_synthesis_matches_the_oracle(dims, mode, B, C, Hf, J, dtype):
+    p = make_params(len(dims), Hf, J, C, B, mode, seed=71)
+    h = gpu_synthesize(dims, mode, B, C, Hf, J, p, dtype)
+    ref = oracle_synthesize(dims, mode, B, J, Hf, p)
+    err = oracle.rel_l2(h.cpu(), ref)
+    tol = TOL[dtype]
+    if dtype == "bf16":
+        rounding = oracle.rel_l2(torch.from_numpy(ref).bfloat16(), ref)
+        assert err <= 1.1 * rounding + 1e-6, f"rel-L2 {err:.3e} vs rounding {rounding:.3e}"
+        if ref.size < 4096:
+            tol = max(tol, 1.1 * rounding)
+    assert np.isfinite(err) and err <= tol, f"rel-L2 {err:.3e}"
+    # element-wise: the window multiplies an fp32 network output whose absolute error is relative to the network's range
+    coords = ks.coordinates(dims, mode).reshape(-1, len(dims))
+    if mode == "causal":
+        win = np.exp(-p["window"].astype(np.float64)[None, :] * np.abs(coords[:, :1]))
+    else:
+        win = np.exp(-0.5 * np.sum((coords[:, :, None] / p["window"].astype(np.float64)[None]) ** 2, axis=1))
+    win = win.T.reshape((1, C) + ref.shape[2:])
+    fmax = float(np.max(np.abs(ref) / np.maximum(win, 1e-300) * (win > 1e-30)))
+    bound = ELEM_R[dtype] * np.abs(ref) + 2e-5 * fmax * win + 1e-37
+    ex = float(np.max(np.abs(oracle.to_f64(h.cpu()) - ref) / bound))
+    assert ex <= 1.0, f"an element is off by {ex:.2f} x its bound"
+
+
+def test_static_kernel_and_argument_checks():
+    from paper_2607_19378_b200 import hyenand as hn
+    dims, B, C, Hf, J = (12, 9), 2, 3, 10, 2
+    p = make_params(2, Hf, J, C, B, "linear", seed=72, film=False)
+    h = gpu_synthesize(dims, "linear", B, C, Hf, J, p, "f32")
+    ref = oracle_synthesize(dims, "linear", B, J, Hf, p)
+    assert oracle.rel_l2(h.cpu(), ref) <= 1e-5
+    assert torch.equal(h[0], h[1])                        # identity modulation: the same kernel for every sample
+    t = torch.zeros(64, device="cuda")
+    L = hn.lib()
+    arr = (__import__("ctypes").c_int * 1)(8)
+    args = lambda hidden, layers, mode, ndim: (ndim, arr, mode, 1, 1, hidden, layers) + (t.data_ptr(),) * 10 + (0, t.data_ptr(), None)
+    assert L.hyenand_synthesize_kernel(*args(65, 2, 0, 1)) == hn.HYENAND_ERR_UNSUPPORTED
+    assert L.hyenand_synthesize_kernel(*args(8, 9, 0, 1)) == hn.HYENAND_ERR_UNSUPPORTED
+    assert L.hyenand_synthesize_kernel(*args(8, 2, 5, 1)) == hn.HYENAND_ERR_INVALID_ARG
+    assert L.hyenand_synthesize_kernel(*args(8, 2, 0, 4)) == hn.HYENAND_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_synthesised_kernel_feeds_the_convolution(dtype):
+    """K(x) written by the synthesis kernel is consumed by hyenand_forward without passing through the host; the
+    result equals the oracle's convolution with the oracle's kernel (rounded to the I/O type where the GPU rounds it)."""
+    from paper_2607_19378_b200 import hyenand as hn
+    from paper_2607_19378_b200 import workloads as W
+    dims, B, C, Hf, J = (40, 48), 2, 6, 16, 2
+    w, (q, k, v, _) = W.random_problem(dims, B=B, C=C, dtype=dtype, seed=73)
+    p = make_params(2, Hf, J, C, B, "linear", seed=73)
+    h = gpu_synthesize(dims, "linear", B, C, Hf, J, p, dtype)
+    plan = hn.Plan(dims, B, C, dtype=w.torch_dtype)
+    y = plan.forward(q.cuda(), k.cuda(), v.cuda(), h.contiguous())
+    torch.cuda.synchronize()
+    plan.close()
+    href = oracle_synthesize(dims, "linear", B, J, Hf, p)
+    href_io = torch.from_numpy(href).to(w.torch_dtype)    # h is an I/O tensor of the convolution: one rounding there
+    ref = oracle.conv_fft(q, k, v, href_io, "linear")
+    err = oracle.rel_l2(y.cpu(), ref)
+    if dtype == "bf16":
+        # a tap whose fp32 value sits next to a bf16 rounding boundary may round the other way than the oracle's:
+        # compare against the convolution with the GPU's own h as well
+        ref_own = oracle.conv_fft(q, k, v, h.cpu(), "linear")
+        rounding = oracle.rel_l2(torch.from_numpy(ref_own).bfloat16(), ref_own)
+        assert oracle.rel_l2(y.cpu(), ref_own) <= 1.1 * rounding + 1e-6
+        assert err <= 1.5 * TOL[dtype]
+    else:
+        assert err <= 2e-5
