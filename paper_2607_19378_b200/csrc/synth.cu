@@ -8,8 +8,10 @@
 // registers, the weights are read from shared memory as 16-byte broadcasts (every lane reads the same address), so
 // each loaded weight feeds NC fused multiply-adds.  The output layer runs over chunks of channels whose weights are
 // staged in shared memory in turn; for a fixed channel a warp stores 32*NC neighbouring taps (coalesced).
-// This translation unit is compiled WITHOUT fast-math: the first sine takes arguments of tens of radians, where
-// the fast sine's error would exceed the fp32 gate.
+// Sines: the first layer's arguments reach tens of radians, where the hardware sine alone loses accuracy, so every
+// argument is first reduced to [-pi, pi] with a two-term 2*pi (exact to fp32 rounding for the multiples that occur);
+// the hardware sine's absolute error on that interval is 2^-21.4.  This translation unit is compiled without
+// fast-math so that nothing else (divisions, the reduction) is replaced by approximations.
 #include "common.cuh"
 #include "synth.cuh"
 
@@ -17,6 +19,14 @@ namespace hn {
 
 constexpr int kSynThreads = 128;
 constexpr int kSynChanChunk = 32;        // output channels whose weights sit in shared memory at a time
+
+__device__ __forceinline__ float sin_reduced(float x)
+{
+    const float k = rintf(x * 0.15915494309189535f);
+    float r = fmaf(-k, 6.2831854820251465f, x);           // float(2 pi)
+    r = fmaf(k, 1.7484555e-7f, r);                        // float(2 pi) - 2 pi
+    return __sinf(r);
+}
 
 __device__ __forceinline__ float axis_coord(int m, int L, int mode)
 {
@@ -85,7 +95,7 @@ __global__ void __launch_bounds__(kSynThreads) synth_kernel(SynthArgs p)
 #pragma unroll
         for (int n = 0; n < NC; ++n) {
             const float pre = fmaf(w.x, cx[n][0], fmaf(w.y, cx[n][1], fmaf(w.z, cx[n][2], w.w)));
-            act[n][i] = fmaf(ga, sinf(om * pre), be);
+            act[n][i] = fmaf(ga, sin_reduced(om * pre), be);
         }
     }
     for (int j = 1; j < J; ++j) {
@@ -105,7 +115,7 @@ __global__ void __launch_bounds__(kSynThreads) synth_kernel(SynthArgs p)
             }
             const float ga = sFi[(j * 2) * HF + i], be = sFi[(j * 2 + 1) * HF + i];
 #pragma unroll
-            for (int n = 0; n < NC; ++n) nxt[n][i] = fmaf(ga, sinf(s[n]), be);
+            for (int n = 0; n < NC; ++n) nxt[n][i] = fmaf(ga, sin_reduced(s[n]), be);
         }
 #pragma unroll
         for (int i = 0; i < HF; ++i)
@@ -149,10 +159,10 @@ __global__ void __launch_bounds__(kSynThreads) synth_kernel(SynthArgs p)
 #pragma unroll
             for (int n = 0; n < NC; ++n) {
                 float win;
-                if (p.mode == 1) win = expf(-w2 * fabsf(cx[n][2]));
+                if (p.mode == 1) win = __expf(-w2 * fabsf(cx[n][2]));
                 else {
                     const float a0 = cx[n][0] * w0, a1 = cx[n][1] * w1, a2 = cx[n][2] * w2;
-                    win = expf(-0.5f * (a0 * a0 + a1 * a1 + a2 * a2));
+                    win = __expf(-0.5f * (a0 * a0 + a1 * a1 + a2 * a2));
                 }
                 if (t0 + n < taps) IO<T>::st(out, (long long)(c0 + c) * taps + t0 + n, win * s[n]);
             }
