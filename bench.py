@@ -537,6 +537,65 @@ def main_mixer(args):
         "clocks": clocks, "device_status": status, "guard_damage": damage}))
 
 
+# ---- backward pass ------------------------------------------------------------------------------------------
+
+def main_backward(args):
+    """`--op backward`: times hyenand_backward (dq, dk, dv, dh) on the workload, inputs resident in HBM.  Roofline:
+    the minimal traffic of the gradient (q, k, v, h, dy in; dq, dk, dv, dh out) and the transforms a direct spectral
+    formulation needs (k v, dy q and h forward; dq, du, dh inverse), charged like the forward's."""
+    from paper_2607_19378_b200 import hyenand as hn
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    w = ALL_WORKLOADS[args.workload].scaled(B=args.batch, C=args.channels)
+    q, k, v, h = W.make_inputs(w, device=device)
+    dy = torch.randn(q.shape, device=device, generator=torch.Generator(device=device).manual_seed(w.seed)).to(q.dtype)
+    bw = hn.Backward(w.dims, w.B, w.C, mode=w.mode, dtype=w.torch_dtype)
+    for _ in range(max(args.warmup, 3)):
+        bw(q, k, v, h, dy)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    time.sleep(0.6)
+    bw(q, k, v, h, dy)
+    torch.cuda.synchronize()
+    outs = [torch.empty_like(q), torch.empty_like(q), torch.empty_like(q), torch.empty_like(h)]
+    stride = 0 if w.h_shared else w.C * h[0, 0].numel()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        hn.hyenand_backward(bw.handle, q, k, v, h, stride, dy, *outs)
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1) / args.steps
+    clocks = sampler.stop(t0, t1)
+    damage = hn.hyenand_backward_guard_damage(bw.handle)
+    if damage != 0:
+        raise SystemExit(f"backward: {damage} damaged guard bytes: the timing is void")
+    bw.close()
+    hbm_gbs, peak_src, sm_max = measured_peaks()
+    fp32_tf = fp32_peak_tflops(torch.cuda.get_device_properties(0).multi_processor_count, sm_max)
+    sbytes = 4 if w.dtype == "f32" else 2
+    hcount = w.C if w.h_shared else w.B * w.C
+    nbytes = 7 * w.elements * sbytes + 2 * hcount * math.prod(w.taps) * sbytes
+    P = math.prod(padded_dims(w))
+    transforms = 5 * w.B * w.C + hcount
+    flops = transforms * 2.5 * P * math.log2(P) if P > 1 else 0.0
+    t_hbm, t_alu = nbytes / (hbm_gbs * 1e9) * 1e3, flops / (fp32_tf * 1e12) * 1e3
+    print(json.dumps({
+        "metric": "hyenand_backward_throughput", "value": w.elements / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "op": "dq, dk, dv, dh of y = q * (h conv (k v))", "dims": list(w.dims), "B": w.B,
+                   "C": w.C, "mode": w.mode, "h_shared_over_batch": w.h_shared},
+        "op_roofline": {"t_hbm_ms": t_hbm, "t_fp32_ms": t_alu, "roofline_ms": max(t_hbm, t_alu), "frac": max(t_hbm, t_alu) / ms,
+                        "min_bytes": nbytes, "nominal_flops": flops,
+                        "note": "six transforms per slice (five when the kernel is shared over the batch) at 2.5 P log2 P"},
+        "clocks": clocks, "guard_damage": damage}))
+
+
 # ---- kernel synthesis ---------------------------------------------------------------------------------------
 
 def main_synth(args):
@@ -657,9 +716,9 @@ if __name__ == "__main__":
     ap.add_argument("--no-all", action="store_true", help="skip the table over the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-cufft", action="store_true", help="skip the torch.fft (cuFFT) composition reference point")
-    ap.add_argument("--op", default="conv", choices=["conv", "mixer", "synth"],
+    ap.add_argument("--op", default="conv", choices=["conv", "mixer", "synth", "backward"],
                     help="conv: the gated long convolution (default, the benchmark line); mixer: the full operator of Eq. 2; "
-                         "synth: the kernel synthesis K(x)")
+                         "synth: the kernel synthesis K(x); backward: dq, dk, dv, dh")
     ap.add_argument("--hidden", type=int, default=32, help="--op synth: width of the SIREN")
     ap.add_argument("--layers", type=int, default=2, help="--op synth: hidden layers of the SIREN")
     a = ap.parse_args()
@@ -669,5 +728,7 @@ if __name__ == "__main__":
         main_mixer(a)
     elif a.op == "synth":
         main_synth(a)
+    elif a.op == "backward":
+        main_backward(a)
     else:
         main_ours(a)

@@ -182,6 +182,28 @@ long long hyenand_mixer_guard_damage(hyenand_mixer *mixer);
 void hyenand_mixer_destroy(hyenand_mixer *mixer);
 
 /*
+ * Backward pass of the gated long convolution (the paper defines and benchmarks the forward only, Appendix B.4;
+ * this is the derivative of Definition A.3).  With y = q * (h conv (k v)) and dy given:
+ *     dq = dy * (h conv (k v));   du = h' conv (dy q) with h'[d] = h[-d];   dk = du * v;   dv = du * k;
+ *     dh[d] = sum_i (dy q)_i (k v)_{i-d} for every displacement d that has a tap, summed over the batch as well when
+ *     the kernel is shared (h_batch_stride_elems = 0; dh then has the shape of h, [C][K..]).
+ * q, k, v, dy, dq, dk, dv: [B][C][L..]; h, dh: as hyenand_forward_ex; all DEVICE pointers of the one I/O dtype,
+ * 16-byte aligned; outputs must not overlap inputs.  Every gradient is computed on fp32 plans and fp32 scratch (bf16
+ * inputs are widened once) and rounded once, at its store.  The gradients are long convolutions themselves and run on
+ * the forward's kernels: three to five forward passes per call (dq; du; dh as one circular convolution on the padded
+ * grid, or, for 1-D grids whose padded length exceeds 8192, one or two causal convolutions of reversed signals).
+ * The handle owns up to four fp32 plans and the scratch (about 4 GiB for the batch groups, 2 GiB for the dh groups).
+ * Limits: as the forward's; circular mode needs power-of-two grids.  Errors and stream semantics as hyenand_forward_ex.
+ */
+typedef struct hyenand_grad hyenand_grad;
+hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int B, int C, int mode, int dtype);
+int hyenand_backward(hyenand_grad *grad, const void *q, const void *k, const void *v, const void *h,
+                     long long h_batch_stride_elems, const void *dy, void *dq, void *dk, void *dv, void *dh,
+                     void *cuda_stream);
+long long hyenand_backward_guard_damage(hyenand_grad *grad);
+void hyenand_backward_destroy(hyenand_grad *grad);
+
+/*
  * Kernel synthesis: evaluates the input-dependent convolution kernel of Section 3.2.1 / 3.2.2,
  *
  *     K(x)[b][c][i] = w_c(c_i) * f_theta(c_i; gamma_b, beta_b)[c],

@@ -17,6 +17,7 @@
 #include "fused2d.cuh"
 #include "mixer.cuh"
 #include "synth.cuh"
+#include "backward.cuh"
 
 using namespace hn;
 
@@ -1089,6 +1090,297 @@ extern "C" long long hyenand_mixer_guard_damage(hyenand_mixer *m)
     if (!m) { fail(HYENAND_ERR_INVALID_ARG, "mixer is NULL"); return -1; }
     const long long a = guard_damage(&m->allocs), b = guard_damage(&m->plan->allocs);
     return (a < 0 || b < 0) ? -1 : a + b;
+}
+
+// ---- backward pass ----------------------------------------------------------------------------------------
+//
+// Forward: y = q * w, w = h conv u, u = k * v.  With g = dy * q:
+//     dq = dy * w                         one forward with the outer gate dy
+//     du = h' conv g, h'[d] = h[-d]       one forward with the kernel re-indexed to the opposite displacement
+//     dk = du * v, dv = du * k
+//     dh[d] = sum_i g_i u_{i-d}           a correlation of two grid signals whose result lives on the TAP grid:
+//         - transforms up to 8192 points per axis: one circular convolution on the padded grid P (which holds every
+//           displacement without wrap-around) of the zero-padded g with the zero-padded u at the opposite
+//           displacement; the taps are read back from the ring;
+//         - circular operators: the same on the grid itself;
+//         - long 1-D: the causal forward applied to reversed signals (one call per sign of the displacement).
+// Everything runs on fp32 plans and fp32 scratch (bf16 inputs are widened once), each gradient is rounded once, at
+// its final store.  Batches are worked off in groups of batch entries, the dh correlation in groups of slices.
+
+struct hyenand_grad {
+    int ndim, B, C, mode, dtype, device;
+    int dims[3];
+    int L[3], K[3], P[3];             // internal 3-axis form
+    long long vol, kvol, pvol, kopp;  // elements per slice: grid, taps, padded ring, taps of the opposite kernel
+    bool long1d;
+    int nb;                           // batch entries per pass
+    long long ns;                     // slices per pass of the dh correlation (ring path)
+    hyenand_plan *main, *adj, *ring, *caus;
+    float *q32, *k32, *v32, *dy32, *ones, *t32, *h32, *hopp;      // per pass of nb entries
+    float *rk, *rv, *rh, *rones, *rt;                            // ring path, ns slices each
+    float *aux;                       // nb*C slices: reversed signals of the long 1-D path
+    float *dhs;                       // nb*C slices of taps: per-slice kernel gradients before the sum over the batch
+    float *dh32;                      // accumulated kernel gradient (shared kernel: [C][kvol]; else [nb*C][kvol])
+    GuardedAllocs allocs;
+};
+
+extern "C" void hyenand_backward_destroy(hyenand_grad *g)
+{
+    if (!g) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != g->device) cudaSetDevice(g->device);
+    if (g->adj && g->adj != g->main) hyenand_destroy_plan(g->adj);
+    if (g->caus && g->caus != g->main) hyenand_destroy_plan(g->caus);
+    hyenand_destroy_plan(g->ring);
+    hyenand_destroy_plan(g->main);
+    guarded_free_all(&g->allocs);
+    if (cur != g->device) cudaSetDevice(cur);
+    delete g;
+}
+
+extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int B, int C, int mode, int dtype)
+{
+    g_err[0] = 0;
+    if (dtype != HYENAND_F32 && dtype != HYENAND_BF16) { fail(HYENAND_ERR_INVALID_ARG, "unknown dtype %d", dtype); return nullptr; }
+    if (ndim < 1 || ndim > 3 || !dims || B < 1 || C < 1) { fail(HYENAND_ERR_INVALID_ARG, "bad geometry"); return nullptr; }
+    for (int a = 0; a < ndim; ++a)
+        if (dims[a] < 1) { fail(HYENAND_ERR_INVALID_ARG, "dims[%d] = %d must be >= 1", a, dims[a]); return nullptr; }
+    hyenand_grad *g = new hyenand_grad();
+    memset(g, 0, sizeof(*g));
+    cudaGetDevice(&g->device);
+    g->ndim = ndim; g->B = B; g->C = C; g->mode = mode; g->dtype = dtype;
+    g->vol = g->kvol = g->pvol = 1;
+    for (int a = 0; a < 3; ++a) { g->L[a] = g->K[a] = g->P[a] = 1; }
+    int pdims[3] = {1, 1, 1};
+    bool ring_ok = true;
+    for (int a = 0; a < ndim; ++a) {
+        const int ia = 3 - ndim + a;
+        g->dims[a] = dims[a];
+        g->L[ia] = dims[a];
+        g->K[ia] = mode == HYENAND_MODE_LINEAR ? 2 * dims[a] - 1 : dims[a];
+        g->P[ia] = mode == HYENAND_MODE_CIRCULAR ? dims[a] : 1 << next_pow2_log(2 * dims[a] - 1);
+        pdims[a] = g->P[ia];
+        if (g->P[ia] > (1 << kMaxLineLog2)) ring_ok = false;
+        g->vol *= dims[a]; g->kvol *= g->K[ia]; g->pvol *= g->P[ia];
+    }
+    g->kopp = mode == HYENAND_MODE_CAUSAL ? 2ll * g->L[2] - 1 : g->kvol;
+    g->long1d = !ring_ok;
+    if (g->long1d && (ndim != 1 || mode == HYENAND_MODE_CIRCULAR)) {
+        fail(HYENAND_ERR_UNSUPPORTED, "a padded axis exceeds %d points (only 1-D linear and causal grids may)", 1 << kMaxLineLog2);
+        delete g; return nullptr;
+    }
+    // batch entries per pass: nine fp32 tensors of nb*C*vol elements (+ kernels) within about 4 GiB
+    long long nb = (4ll << 30) / (4ll * C * (8 * g->vol + g->kopp + 3 * g->kvol));
+    if (const char *e = getenv("HYENAND_BACKWARD_MAX_BATCH")) { const long long v = atoll(e); if (v > 0 && v < nb) nb = v; }   // development aid
+    if (nb < 1) nb = 1;
+    if (nb > B) nb = B;
+    g->nb = (int)nb;
+    const long long S = nb * C;
+    g->main = hyenand_create_plan_mode(ndim, dims, (int)nb, C, mode, HYENAND_F32);
+    if (!g->main) { delete g; return nullptr; }
+    g->adj = g->main;
+    if (mode == HYENAND_MODE_CAUSAL) {
+        g->adj = hyenand_create_plan_mode(ndim, dims, (int)nb, C, HYENAND_MODE_LINEAR, HYENAND_F32);
+        if (!g->adj) { g->adj = g->main; hyenand_backward_destroy(g); return nullptr; }
+    }
+    if (g->long1d) {
+        g->caus = g->main;
+        if (mode != HYENAND_MODE_CAUSAL) {
+            g->caus = hyenand_create_plan_mode(ndim, dims, (int)nb, C, HYENAND_MODE_CAUSAL, HYENAND_F32);
+            if (!g->caus) { hyenand_backward_destroy(g); return nullptr; }
+        }
+    } else if (mode != HYENAND_MODE_CIRCULAR) {
+        // ring path: five fp32 tensors of ns*pvol elements within about 2 GiB
+        long long ns = (2ll << 30) / (20ll * g->pvol);
+        if (const char *e = getenv("HYENAND_BACKWARD_RING_SLICES")) { const long long v = atoll(e); if (v > 0 && v < ns) ns = v; }   // development aid
+        if (ns < 1) ns = 1;
+        if (ns > S) ns = S;
+        g->ns = ns;
+        g->ring = hyenand_create_plan_mode(ndim, pdims, 1, (int)ns, HYENAND_MODE_CIRCULAR, HYENAND_F32);
+        if (!g->ring) { hyenand_backward_destroy(g); return nullptr; }
+    }
+    const bool widen = dtype == HYENAND_BF16;
+    cudaError_t e = cudaSuccess;
+    auto get = [&](float **ptr, long long elems) {
+        if (e == cudaSuccess) e = guarded_alloc(&g->allocs, (void **)ptr, (size_t)elems * sizeof(float));
+    };
+    if (widen) { get(&g->q32, S * g->vol); get(&g->k32, S * g->vol); get(&g->v32, S * g->vol); get(&g->dy32, S * g->vol); get(&g->h32, S * g->kvol); }
+    get(&g->ones, S * g->vol); get(&g->t32, S * g->vol); get(&g->hopp, S * g->kopp);
+    get(&g->aux, S * g->vol); get(&g->dhs, S * g->kvol); get(&g->dh32, S * g->kvol);
+    if (g->ring) { get(&g->rk, g->ns * g->pvol); get(&g->rv, g->ns * g->pvol); get(&g->rh, g->ns * g->pvol);
+                   get(&g->rones, g->ns * g->pvol); get(&g->rt, g->ns * g->pvol); }
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        fail(HYENAND_ERR_ALLOC, "scratch of the backward pass: %s", cudaGetErrorString(e));
+        hyenand_backward_destroy(g);
+        return nullptr;
+    }
+    launch_fill(g->ones, 1.f, S * g->vol, 0);
+    if (g->ring) launch_fill(g->rones, 1.f, g->ns * g->pvol, 0);
+    if (cudaDeviceSynchronize() != cudaSuccess) {
+        fail(HYENAND_ERR_CUDA, "filling the constant tensors failed: %s", cudaGetErrorString(cudaGetLastError()));
+        hyenand_backward_destroy(g);
+        return nullptr;
+    }
+    return g;
+}
+
+// one forward of `n` slices on an inner fp32 plan (a plan of more slices runs the first n)
+static int grad_forward(hyenand_plan *p, long long n, const float *q, const float *k, const float *v, const float *h,
+                        bool shared, float *y, cudaStream_t st)
+{
+    int launches = 0;
+    p->r0 = 0; p->r1 = n;
+    const int e = run_forward(p, q, k, v, h, shared, y, st, &launches);
+    p->r0 = 0; p->r1 = (long long)p->B * p->C;
+    return e;
+}
+
+extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, const void *v, const void *h,
+                                long long h_batch_stride_elems, const void *dy, void *dq, void *dk, void *dv, void *dh,
+                                void *cuda_stream)
+{
+    g_err[0] = 0;
+    if (!g) return fail(HYENAND_ERR_INVALID_ARG, "handle is NULL");
+    const void *ptrs[9] = {q, k, v, h, dy, dq, dk, dv, dh};
+    for (int i = 0; i < 9; ++i) {
+        if (!ptrs[i]) return fail(HYENAND_ERR_INVALID_ARG, "pointer %d is NULL", i);
+        if (((uintptr_t)ptrs[i]) & 15) return fail(HYENAND_ERR_INVALID_ARG, "pointer %d is not 16-byte aligned", i);
+    }
+    bool shared = false;
+    if (h_batch_stride_elems == 0) shared = true;
+    else if (h_batch_stride_elems != (long long)g->C * g->kvol)
+        return fail(HYENAND_ERR_INVALID_ARG, "h_batch_stride_elems must be 0 or C*K_1*..*K_N = %lld", (long long)g->C * g->kvol);
+    int e = check_device(g->main);
+    if (e) return e;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t es = elsize(g->dtype);
+    const bool widen = g->dtype == HYENAND_BF16;
+    const long long C = g->C, vol = g->vol, kvol = g->kvol;
+    const int *L = g->L, *K = g->K, *P = g->P;
+    const float *hsh = (const float *)h;                       // shared kernel, fp32 view
+    if (shared && widen) { launch_widen(h, g->dtype, C * kvol, g->h32, st); hsh = g->h32; }
+    for (int b0 = 0; b0 < g->B; b0 += g->nb) {
+        const long long n = g->B - b0 < g->nb ? g->B - b0 : g->nb, S = n * C, off = (long long)b0 * C * vol;
+        const float *q32 = (const float *)q + off, *k32 = (const float *)k + off, *v32 = (const float *)v + off, *dy32 = (const float *)dy + off;
+        if (widen) {
+            launch_widen((const char *)q + off * es, g->dtype, S * vol, g->q32, st); q32 = g->q32;
+            launch_widen((const char *)k + off * es, g->dtype, S * vol, g->k32, st); k32 = g->k32;
+            launch_widen((const char *)v + off * es, g->dtype, S * vol, g->v32, st); v32 = g->v32;
+            launch_widen((const char *)dy + off * es, g->dtype, S * vol, g->dy32, st); dy32 = g->dy32;
+        }
+        const float *h32 = hsh;
+        if (!shared) {
+            h32 = (const float *)h + (long long)b0 * C * kvol;
+            if (widen) { launch_widen((const char *)h + (long long)b0 * C * kvol * es, g->dtype, S * kvol, g->h32, st); h32 = g->h32; }
+        }
+        const long long Sh = shared ? C : S;
+        // dq = dy * (h conv (k v))
+        if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st))) return e;
+        launch_mul_cast(g->t32, nullptr, S * vol, g->dtype, (char *)dq + off * es, st);
+        // the kernel at the opposite displacement
+        {
+            RemapArgs r{};
+            r.a = h32; r.b = nullptr; r.out = g->hopp; r.slices = Sh;
+            for (int a = 0; a < 3; ++a) {
+                r.Ls[a] = K[a]; r.G[a] = K[a];
+                r.mode[a] = g->mode == HYENAND_MODE_CIRCULAR ? REMAP_NEG : REMAP_REV;
+            }
+            if (g->mode == HYENAND_MODE_CAUSAL) r.G[2] = 2 * L[2] - 1;       // causal taps as the negative half of a non-causal kernel
+            launch_remap(r, st);
+        }
+        // du = h' conv (dy q);  dk = du v, dv = du k
+        if ((e = grad_forward(g->adj, S, g->ones, dy32, q32, g->hopp, shared, g->t32, st))) return e;
+        launch_mul_cast(g->t32, v32, S * vol, g->dtype, (char *)dk + off * es, st);
+        launch_mul_cast(g->t32, k32, S * vol, g->dtype, (char *)dv + off * es, st);
+        // dh
+        float *dhS = shared ? g->dhs : g->dh32;                  // per-slice kernel gradients of this pass
+        if (g->mode == HYENAND_MODE_CIRCULAR) {
+            // dh[m] = sum_i g_i u_{(i-m) mod L}: circular convolution of g with u read at the opposite displacement
+            // (hopp is free again: the forward that consumed the opposite kernel precedes this on the stream)
+            RemapArgs r{};
+            r.a = k32; r.b = v32; r.out = g->hopp; r.slices = S;
+            for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = REMAP_NEG; }
+            launch_remap(r, st);
+            if ((e = grad_forward(g->main, S, g->ones, dy32, q32, g->hopp, false, dhS, st))) return e;
+            if (shared) launch_batch_sum(dhS, n, C, kvol, b0 == 0, g->dh32, st);
+        } else if (g->long1d) {
+            const int Ln = L[2];
+            // Displacements d >= 0: dh[d] = sum_s g_{s+d} u_s.  The causal forward with the reversed g as its kernel gives
+            // c[n] = sum_{s<=n} g[L-1-(n-s)] u_s, and c[L-1-d] is that sum.
+            RemapArgs r{};
+            r.a = dy32; r.b = q32; r.out = g->aux; r.slices = S;
+            for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
+            launch_remap(r, st);
+            if ((e = grad_forward(g->caus, S, g->ones, k32, v32, g->aux, false, g->t32, st))) return e;
+            if (g->mode == HYENAND_MODE_CAUSAL) {
+                RemapArgs w{};                                 // tap t <- c[L-1-t]
+                w.a = g->t32; w.out = dhS; w.slices = S;
+                for (int a = 0; a < 3; ++a) { w.Ls[a] = L[a]; w.G[a] = K[a]; w.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
+                launch_remap(w, st);
+            } else {
+                // Displacements -t < 0: dh[-t] = sum_s u_{s+t} g_s, the same form with g and u exchanged: c'[L-1-t].
+                // Tap m = d + L-1: the lower taps m = 0..L-1 are c'[m] (a plain copy), the upper taps m = L..2L-2 are
+                // c[2(L-1)-m], the reversed c from its second entry on.
+                r.a = k32; r.b = v32;
+                launch_remap(r, st);                           // reversed u (the forward that read aux precedes this on the stream)
+                float *neg = g->hopp;                          // S*(2L-1) floats, free again
+                if ((e = grad_forward(g->caus, S, g->ones, dy32, q32, g->aux, false, neg, st))) return e;
+                RemapArgs lo{};
+                lo.a = neg; lo.out = dhS; lo.slices = S;
+                for (int a = 0; a < 3; ++a) { lo.Ls[a] = L[a]; lo.G[a] = K[a]; lo.mode[a] = REMAP_PAD; }
+                launch_remap(lo, st);
+                RemapArgs rv{};
+                rv.a = g->t32; rv.out = g->aux; rv.slices = S;
+                for (int a = 0; a < 3; ++a) { rv.Ls[a] = L[a]; rv.G[a] = L[a]; rv.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
+                launch_remap(rv, st);                          // aux[j] = c[L-1-j] = dh[d = j]
+                if (Ln > 1 &&
+                    cudaMemcpy2DAsync(dhS + Ln, (size_t)kvol * sizeof(float), g->aux + 1, (size_t)vol * sizeof(float),
+                                      (size_t)(Ln - 1) * sizeof(float), (size_t)S, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                    return fail(HYENAND_ERR_CUDA, "copy of the upper taps failed: %s", cudaGetErrorString(cudaGetLastError()));
+            }
+            if (shared) launch_batch_sum(dhS, n, C, kvol, b0 == 0, g->dh32, st);
+        } else {
+            // ring path, ns slices at a time
+            for (long long s0 = 0; s0 < S; s0 += g->ns) {
+                const long long m = S - s0 < g->ns ? S - s0 : g->ns;
+                RemapArgs pad{};
+                pad.slices = m;
+                for (int a = 0; a < 3; ++a) { pad.Ls[a] = L[a]; pad.G[a] = P[a]; pad.mode[a] = REMAP_PAD; }
+                pad.a = dy32 + s0 * vol; pad.out = g->rk; launch_remap(pad, st);
+                pad.a = q32 + s0 * vol; pad.out = g->rv; launch_remap(pad, st);
+                RemapArgs opp = pad;
+                for (int a = 0; a < 3; ++a) opp.mode[a] = REMAP_NEG;
+                opp.a = k32 + s0 * vol; opp.b = v32 + s0 * vol; opp.out = g->rh; launch_remap(opp, st);
+                if ((e = grad_forward(g->ring, m, g->rones, g->rk, g->rv, g->rh, false, g->rt, st))) return e;
+                RemapArgs tap{};
+                tap.a = g->rt; tap.out = dhS + s0 * kvol; tap.slices = m;
+                for (int a = 0; a < 3; ++a) {
+                    tap.Ls[a] = P[a]; tap.G[a] = K[a]; tap.mode[a] = REMAP_WRAP;
+                    tap.shift[a] = g->mode == HYENAND_MODE_LINEAR ? L[a] - 1 : 0;      // tap m is displacement m - (L-1), or m when causal
+                }
+                launch_remap(tap, st);
+            }
+            if (shared) launch_batch_sum(dhS, n, C, kvol, b0 == 0, g->dh32, st);
+        }
+        if (!shared) launch_mul_cast(g->dh32, nullptr, S * kvol, g->dtype, (char *)dh + (long long)b0 * C * kvol * es, st);
+    }
+    if (shared) launch_mul_cast(g->dh32, nullptr, C * kvol, g->dtype, dh, st);
+    cudaError_t ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(HYENAND_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(ce));
+    return HYENAND_OK;
+}
+
+extern "C" long long hyenand_backward_guard_damage(hyenand_grad *g)
+{
+    g_err[0] = 0;
+    if (!g) { fail(HYENAND_ERR_INVALID_ARG, "handle is NULL"); return -1; }
+    long long bad = guard_damage(&g->allocs);
+    hyenand_plan *plans[4] = {g->main, g->adj != g->main ? g->adj : nullptr, g->ring, (g->caus && g->caus != g->main) ? g->caus : nullptr};
+    for (int i = 0; i < 4 && bad >= 0; ++i)
+        if (plans[i]) { const long long b = guard_damage(&plans[i]->allocs); bad = b < 0 ? -1 : bad + b; }
+    return bad;
 }
 
 // ---- kernel synthesis ---------------------------------------------------------------------------------

@@ -84,6 +84,13 @@ def lib() -> ctypes.CDLL:
         L.hyenand_mixer_guard_damage.argtypes = [vp]
         L.hyenand_mixer_destroy.restype = None
         L.hyenand_mixer_destroy.argtypes = [vp]
+        L.hyenand_backward_create.restype = vp
+        L.hyenand_backward_create.argtypes = [ctypes.c_int, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+        L.hyenand_backward.argtypes = [vp, vp, vp, vp, vp, ll, vp, vp, vp, vp, vp, vp]
+        L.hyenand_backward_guard_damage.restype = ll
+        L.hyenand_backward_guard_damage.argtypes = [vp]
+        L.hyenand_backward_destroy.restype = None
+        L.hyenand_backward_destroy.argtypes = [vp]
         L.hyenand_synthesize_kernel.argtypes = [ctypes.c_int, ip] + [ctypes.c_int] * 5 + [vp] * 10 + [ctypes.c_int, vp, vp]
         L.hyenand_plan_set_timing.argtypes = [vp, ctypes.c_int]
         L.hyenand_plan_kernel_time.argtypes = [vp, ctypes.c_int, dpp, dpp]
@@ -263,6 +270,63 @@ def hyenand_synthesize_kernel(dims, mode: int, B: int, C: int, hidden: int, laye
     _check(lib().hyenand_synthesize_kernel(len(dims), arr, int(mode), int(B), int(C), int(hidden), int(layers),
                                            ptr(W1), ptr(b1), ptr(omega0), ptr(Wh), ptr(bh), ptr(Wout), ptr(bout),
                                            ptr(gamma), ptr(beta), ptr(window), int(dtype), h.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_backward_create(ndim: int, dims, B: int, C: int, mode: int, dtype: int) -> int:
+    arr = (ctypes.c_int * max(1, len(dims)))(*[int(d) for d in dims])
+    h = lib().hyenand_backward_create(int(ndim), arr, int(B), int(C), int(mode), int(dtype))
+    if not h:
+        raise HyenaNDError(hyenand_last_error_code() or HYENAND_ERR_INVALID_ARG, hyenand_last_error())
+    return h
+
+
+def hyenand_backward(grad: int, q, k, v, h, h_batch_stride_elems: int, dy, dq, dk, dv, dh, stream=None) -> None:
+    _check(lib().hyenand_backward(grad, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(), int(h_batch_stride_elems),
+                                  dy.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), dh.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_backward_guard_damage(grad: int) -> int:
+    return int(lib().hyenand_backward_guard_damage(grad))
+
+
+def hyenand_backward_destroy(grad: int) -> None:
+    lib().hyenand_backward_destroy(grad)
+
+
+class Backward:
+    """Owner of a hyenand_grad handle: dq, dk, dv, dh of the gated long convolution."""
+
+    def __init__(self, dims, B: int, C: int, mode: str = "linear", dtype=torch.float32):
+        self.dims = tuple(int(d) for d in dims)
+        self.B, self.C, self.mode, self.dtype = B, C, mode, dtype
+        code = {"linear": HYENAND_MODE_LINEAR, "causal": HYENAND_MODE_CAUSAL, "circular": HYENAND_MODE_CIRCULAR}[mode]
+        self.handle = hyenand_backward_create(len(self.dims), self.dims, B, C, code, _DTYPES[dtype])
+
+    def __call__(self, q, k, v, h, dy, stream=None):
+        taps = tuple(2 * L - 1 if self.mode == "linear" else L for L in self.dims)
+        if tuple(h.shape) == (self.C,) + taps:
+            stride = 0
+        elif tuple(h.shape) == (self.B, self.C) + taps:
+            stride = self.C * h[0, 0].numel()
+        else:
+            raise ValueError(f"h has shape {tuple(h.shape)}")
+        for t in (q, k, v, h, dy):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == self.dtype):
+                raise ValueError("inputs must be contiguous CUDA tensors of the handle's dtype")
+        dq, dk, dv, dh = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q), torch.empty_like(h)
+        hyenand_backward(self.handle, q, k, v, h, stride, dy, dq, dk, dv, dh, stream)
+        return dq, dk, dv, dh
+
+    def close(self):
+        if self.handle:
+            hyenand_backward_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class Mixer:
