@@ -68,7 +68,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     listed = open(manifest).read() if os.path.exists(manifest) else ""
     if jobs or stale or listed != "\n".join(objs):
         tmp = LIB + ".tmp.%d" % os.getpid()
-        subprocess.check_call([NVCC, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs + ["-lcudart"])
+        subprocess.check_call([NVCC, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs + ["-lcudart", "-ldl"])
         os.replace(tmp, LIB)
         with open(manifest, "w") as f:
             f.write("\n".join(objs))

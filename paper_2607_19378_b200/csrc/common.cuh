@@ -29,8 +29,15 @@ enum KernelId {
     KID_CT_COLS_H, KID_CT_COLS_U, KID_CT_CORE, KID_CT_COLS_INV, KID_PLANE_H, KID_PLANE_U, KID_PLANE_INV, KID_FUSED2D, KID_CT_HSPEC, KID_COUNT
 };
 
+// names of the KernelId entries (hyenand.cu)
+extern const char *const kKernelNames[];
+// NVTX range around a launch (a no-op unless a profiler that consumes NVTX is attached)
+void nvtx_push(const char *name);
+void nvtx_pop();
+
 struct Prof {
     bool on = false;
+    bool nvtx = false;                // HYENAND_NVTX at plan creation: one NVTX range per kernel launch
     struct Rec { cudaEvent_t a, b; int kid; };
     Rec recs[4096];
     int created = 0, used = 0;
@@ -38,6 +45,7 @@ struct Prof {
     long long launches[KID_COUNT] = {0};
     void begin(int kid, cudaStream_t st)
     {
+        if (nvtx) nvtx_push(kKernelNames[kid]);
         if (!on || used >= 4096) return;
         if (used == created) {
             cudaEventCreate(&recs[created].a);
@@ -49,6 +57,7 @@ struct Prof {
     }
     void end(cudaStream_t st)
     {
+        if (nvtx) nvtx_pop();
         if (!on || used >= 4096) return;
         cudaEventRecord(recs[used].b, st);
         ++used;
@@ -95,6 +104,7 @@ struct DevOnce {
 // created, and travel with the plan: a forward call never looks at the environment.
 struct Switches {
     bool force_generic, generic_rows, generic_core, no_tma;
+    bool nvtx;                        // HYENAND_NVTX: name every kernel launch with an NVTX range
 };
 Switches read_switches();
 

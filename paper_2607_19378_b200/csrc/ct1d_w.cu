@@ -595,13 +595,13 @@ template <typename T, int LOG2P1> static int launch_cols_fwd_w_t(const ColsFwdWA
         const unsigned long long dims[3] = {(unsigned long long)P2, (unsigned long long)(a.len / P2), (unsigned long long)a.slices};
         const unsigned long long strides[2] = {(unsigned long long)P2 * sizeof(T), (unsigned long long)a.in_slice * sizeof(T)};
         const unsigned box[3] = {2 * TX, (unsigned)(HP1 < 256 ? HP1 : 256), 1};
-        tma = tma_encode_3d(&ma, a.a, sizeof(T) == 2, dims, strides, box, (int)TROW);
-        if (tma && a.b) tma = tma_encode_3d(&mb, a.b, sizeof(T) == 2, dims, strides, box, (int)TROW);
+        tma = tma_encode_3d_cached(&ma, a.a, sizeof(T) == 2, dims, strides, box, (int)TROW);
+        if (tma && a.b) tma = tma_encode_3d_cached(&mb, a.b, sizeof(T) == 2, dims, strides, box, (int)TROW);
         // results [slice][P1/2+1][P2] complex, as fp32: boxes of 8 column pairs (32 floats) by 136 rows
         const unsigned long long od[3] = {2ull * P2, (unsigned long long)(HP1 + 1), (unsigned long long)a.slices};
         const unsigned long long os[2] = {(unsigned long long)P2 * 8, (unsigned long long)(HP1 + 1) * P2 * 8};
         const unsigned ob[3] = {32, (unsigned)ct_out_box_rows(HP1 + 1), 1};
-        if (tma) tma = tma_encode_3d(&mo, a.out, false, od, os, ob, 128);
+        if (tma) tma = tma_encode_3d_cached(&mo, a.out, false, od, os, ob, 128);
     }
     if constexpr (TROW == 64 || TROW == 128) {
         if (tma) {
@@ -645,7 +645,7 @@ template <typename T, int LOG2P1> static int launch_cols_inv_w_t(const ColsInvWA
         const unsigned long long dims[3] = {(unsigned long long)P2, (unsigned long long)(a.len / P2), (unsigned long long)a.slices};
         const unsigned long long strides[2] = {(unsigned long long)P2 * sizeof(T), (unsigned long long)a.len * sizeof(T)};
         const unsigned box[3] = {2 * TX, (unsigned)(HP1 < 256 ? HP1 : 256), 1};
-        tma = tma_encode_3d(&mq, a.q, sizeof(T) == 2, dims, strides, box, 0) && tma_encode_3d(&my, a.y, sizeof(T) == 2, dims, strides, box, 0);
+        tma = tma_encode_3d_cached(&mq, a.q, sizeof(T) == 2, dims, strides, box, 0) && tma_encode_3d_cached(&my, a.y, sizeof(T) == 2, dims, strides, box, 0);
     }
     if (tma) launch_cols_inv_w_tt<T, LOG2P1, true>(a, mq, my, grid, sm, st);
     else launch_cols_inv_w_tt<T, LOG2P1, false>(a, mq, my, grid, sm, st);

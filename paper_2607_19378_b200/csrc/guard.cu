@@ -4,6 +4,8 @@
 
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace hn {
@@ -17,8 +19,12 @@ Switches read_switches()
     s.generic_rows = getenv("HYENAND_GENERIC_ROWS") != nullptr;
     s.generic_core = getenv("HYENAND_GENERIC_CORE") != nullptr;
     s.no_tma = getenv("HYENAND_NO_TMA") != nullptr;
+    s.nvtx = getenv("HYENAND_NVTX") != nullptr;
     return s;
 }
+
+void nvtx_push(const char *name) { nvtxRangePushA(name); }
+void nvtx_pop() { nvtxRangePop(); }
 
 cudaError_t guarded_alloc(GuardedAllocs *g, void **ptr, size_t bytes)
 {

@@ -167,6 +167,7 @@ extern "C" hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int
     p->r0 = 0; p->r1 = (long long)B * C;
     cudaGetDevice(&p->device);
     p->sw = read_switches();
+    p->prof.nvtx = p->sw.nvtx;
     p->n_lanes = 1;
     p->vol = 1; p->kvol = 1;
     for (int a = 0; a < 3; ++a) { p->L[a] = 1; p->K[a] = 1; p->P[a] = 1; p->log2p[a] = 0; }
@@ -818,7 +819,7 @@ extern "C" const char *hyenand_plan_path(const hyenand_plan *p)
 
 // ---- per-kernel accounting (reporting only) ---------------------------------------------
 
-static const char *kKernelNames[KID_COUNT] = {
+const char *const hn::kKernelNames[KID_COUNT] = {
     "rows_fwd(h)", "axis_fwd(h)", "rows_fwd(k*v)", "axis_fwd(k*v)", "axis_core", "axis_inv", "rows_inv",
     "ct_cols_fwd(h)", "ct_cols_fwd(k*v)", "ct_core", "ct_cols_inv", "plane_fwd(h)", "plane_fwd(k*v)", "plane_inv", "fused2d", "ct_hspec"};
 

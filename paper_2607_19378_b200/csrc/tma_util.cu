@@ -1,4 +1,5 @@
 // Tensor-map encoding for the kernels that use TMA (host side of tma_util.cuh).
+#include <cstring>
 #include "tma_util.cuh"
 
 namespace hn {
@@ -41,6 +42,32 @@ bool tma_encode_3d(CUtensorMap *map, const void *base, bool bf16, const unsigned
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tma_encode_3d_cached(CUtensorMap *map, const void *base, bool bf16, const unsigned long long dims[3],
+                          const unsigned long long strides[2], const unsigned box[3], int swizzle_bytes)
+{
+    struct Key {
+        const void *base;
+        unsigned long long dims[3], strides[2];
+        unsigned box[3];
+        int swizzle, bf16;
+    };
+    struct Entry { Key key; CUtensorMap map; bool used; };
+    constexpr int kEntries = 16;
+    static thread_local Entry cache[kEntries];
+    Key k;
+    memset(&k, 0, sizeof(k));
+    k.base = base; k.swizzle = swizzle_bytes; k.bf16 = bf16 ? 1 : 0;
+    for (int i = 0; i < 3; ++i) { k.dims[i] = dims[i]; k.box[i] = box[i]; }
+    k.strides[0] = strides[0]; k.strides[1] = strides[1];
+    unsigned long long h = (unsigned long long)(uintptr_t)base * 0x9E3779B97F4A7C15ull ^ dims[0] * 31 ^ dims[1] * 131 ^ dims[2] * 1031 ^
+                           (unsigned long long)box[0] * 7 ^ (unsigned long long)box[1] * 13 ^ (unsigned long long)swizzle_bytes;
+    Entry &e = cache[(h >> 7) % kEntries];
+    if (e.used && memcmp(&e.key, &k, sizeof(k)) == 0) { *map = e.map; return true; }
+    if (!tma_encode_3d(map, base, bf16, dims, strides, box, swizzle_bytes)) return false;
+    e.key = k; e.map = *map; e.used = true;
+    return true;
 }
 
 __global__ void bounded_wait_selftest_kernel(int polls, int *status)

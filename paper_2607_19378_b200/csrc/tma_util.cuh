@@ -74,5 +74,10 @@ int tma_selftest_bounded_wait(int polls);
 // break an alignment rule or the driver refuses.
 bool tma_encode_3d(CUtensorMap *map, const void *base, bool bf16, const unsigned long long dims[3],
                    const unsigned long long strides[2], const unsigned box[3], int swizzle_bytes);
+// The same through a small per-thread cache keyed by every argument: callers that pass the same tensors call after
+// call (a training loop's fixed buffers) skip the driver's encoding.  Encoding reads no device memory, so a cached map
+// stays valid as long as the key matches.
+bool tma_encode_3d_cached(CUtensorMap *map, const void *base, bool bf16, const unsigned long long dims[3],
+                          const unsigned long long strides[2], const unsigned box[3], int swizzle_bytes);
 
 }  // namespace hn
