@@ -165,6 +165,11 @@ __device__ __forceinline__ void separate_rows_odd(const float2 *line, float2 *cs
 // of a row are the half-length transform of f[x] + f[x + P/2], the odd bins that of
 // (f[x] - f[x + P/2]) W_P^x.  Each half (e = 0: even kx, e = 1: odd kx) fills a column store of
 // P/4 columns by P rows, whose columns are then transformed along y and written out as whole lines.
+// The two real rows that share a complex row transform are NOT separated after it: the raw transform Z of every row
+// pair goes straight from the last pass's registers into the store [bin k][row pair], and the column transform of bin k
+// separates them as it loads (it reads Z[k] and the mirrored bin of each row pair: the same number of shared-memory
+// wavefronts as reading separated values, no separation pass and no extra trip of the row results through the line).
+// Separated values come out at twice their value (the factor 1/2 of the separation is left to the spectral core's scale).
 // The tap rows are fetched and unpacked once per plane: while a thread prepares the even half it also forms its
 // inputs of the odd half, f[x] - f[x + P/2], and parks them in tensor memory (its own lane, 2 * points-per-thread
 // columns per row pair); the odd half reads them back instead of staging the rows again.
@@ -175,8 +180,8 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     using F = typename C::F;
     using FH = typename C::FH;
     constexpr int P = C::P, HP = C::HP, QP = P / 4, TPL = F::TPL, TPLH = FH::TPL;
-    constexpr int CSH = P + 1;                               // column-store stride (odd): QP columns of P rows
-    static_assert(QP * CSH <= HP * C::CSS, "column store of a half fits the plane buffer");
+    constexpr int CS2 = HP + 1;                              // store stride (odd): HP bins of HP row pairs, raw row transforms
+    static_assert(HP * CS2 <= HP * C::CSS, "store of a half fits the plane buffer");
     extern __shared__ float2 smem[];
     float2 *cs = smem;
     float2 *wbuf = cs + HP * C::CSS;
@@ -218,10 +223,10 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
         float2 *dst = p.out + pl * (long long)C::XH * P;
         for (int e = 0; e < 2; ++e) {
             // rows: padded row y holds tap row (y + Ly - 1) mod P; two rows per transform
-            // the two groups of a half warp take rows 8 apart, so their column-store writes (one
-            // row per group, consecutive columns per lane) fall into different banks
             int round = 0;
-            for (int rp = spread_pair<4>(gidh); rp < HP; rp += C::NGH, ++round) {
+            // the two groups of a half warp take row pairs 8 apart, so their stores (one row pair per group, consecutive
+            // bins per lane) fall into different banks
+            for (int rp = spread_pair<8>(gidh); rp < HP; rp += C::NGH, ++round) {
                 const int y0 = 2 * rp, y1 = y0 + 1;
                 const int my0 = (y0 + Ly - 1) & (P - 1), my1 = (y1 + Ly - 1) & (P - 1);
                 const bool v0 = my0 < Ky, v1 = my1 < Ky, valid = v0 || v1;
@@ -281,10 +286,9 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                     tmem_wait_st();
                     if (valid) {
                         // (every lane of the group has read its taps from the line before the barrier above)
-                        FH::template run_to_line<PRUNE_NONE, false>(lh, mh, twr, lineh, [&](int i, int r, int) {
-                            return make_float2(ss[2 * (i * R0 + r)], ss[2 * (i * R0 + r) + 1]);
-                        });
-                        separate_rows<LOG2P - 1, CSH>(lineh, cs, y0, y1, lh);
+                        FH::template run<PRUNE_NONE, false>(lh, mh, twr, lineh,
+                            [&](int i, int r, int) { return make_float2(ss[2 * (i * R0 + r)], ss[2 * (i * R0 + r) + 1]); },
+                            [&](int, int, int kk, float2 z) { cs[kk * CS2 + rp] = z; });
                         __syncwarp(mh);
                     }
                 } else {
@@ -292,30 +296,39 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                     TmemIO<NPT>::ld(dd, tcol);
                     tmem_wait_ld();
                     if (valid) {
-                        FH::template run_to_line<PRUNE_NONE, false>(lh, mh, twr, lineh, [&](int i, int r, int idx) {
-                            return cmul(make_float2(dd[2 * (i * R0 + r)], dd[2 * (i * R0 + r) + 1]), tw[idx]);
-                        });
-                        separate_rows_odd<LOG2P - 1, CSH>(lineh, cs, y0, y1, lh);
+                        FH::template run<PRUNE_NONE, false>(lh, mh, twr, lineh,
+                            [&](int i, int r, int idx) { return cmul(make_float2(dd[2 * (i * R0 + r)], dd[2 * (i * R0 + r) + 1]), tw[idx]); },
+                            [&](int, int, int kk, float2 z) { cs[kk * CS2 + rp] = z; });
                         __syncwarp(mh);
                     }
                 }
                 if (!valid) {
-                    for (int k = lh; k < QP; k += TPLH) {
-                        cs[k * CSH + y0] = make_float2(0.f, 0.f);
-                        cs[k * CSH + y1] = make_float2(0.f, 0.f);
-                    }
+                    for (int kk = lh; kk < HP; kk += TPLH) cs[kk * CS2 + rp] = make_float2(0.f, 0.f);
                 }
             }
             __syncthreads();
             // columns: P-point transforms over y of the bins kx = 2k + e
             for (int k = gid; k < QP; k += C::NG) {
-                const float2 *col = cs + k * CSH;
-                // one code path for all columns; column 0 of the even half (bins kx = 0 and kx = P/2 of every
-                // row, packed) sends its raw transform to a shared-memory line and is unpacked afterwards
+                // Row y = 2 rp + par of bin k: with Z = F_y0 + i F_y1 the raw transform of row pair rp,
+                //   2 F_y0[k] = Z[k] + conj Z[k'],  2 F_y1[k] = -i (Z[k] - conj Z[k']),
+                // k' the mirrored bin of the half-length transform ((H - k) mod H in the even half, H - 1 - k in the odd one).
+                // A lane's rows y = l + 16 r all have the parity of l.
+                // Column 0 of the even half packs the two purely real bins kx = 0 and kx = P/2 of every row as one
+                // complex number (2 F_y[0], 2 F_y[P/2]); it sends its raw transform to a shared-memory line and is
+                // unpacked afterwards.  One transform code path for all columns.
                 const bool packed = e == 0 && k == 0;
+                const int km = packed ? HP / 2 : (e == 0 ? ((HP - k) & (HP - 1)) : HP - 1 - k);
+                const float2 *ca = cs + k * CS2, *cb = cs + km * CS2;
+                const bool par = l & 1;
                 float2 *d = packed ? tmp : dst + (long long)(2 * k + e) * P;
                 F::template run<PRUNE_NONE>(l, m, twp, line,
-                    [&](int, int, int idx) { return col[idx]; },
+                    [&](int, int, int idx) {
+                        const float2 za = ca[idx >> 1], zm = cb[idx >> 1];
+                        const float a = par ? za.y : za.x, b = par ? zm.y : zm.x;
+                        if (packed) return make_float2(a + a, b + b);
+                        const float c = par ? -za.x : za.y, dd2 = par ? -zm.x : zm.y;
+                        return make_float2(a + b, c - dd2);
+                    },
                     [&](int, int, int idx, float2 v) { d[idx] = v; });
                 if (packed) {
                     __syncwarp(m);
