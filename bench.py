@@ -458,6 +458,31 @@ def main_ours(args):
                 table.append({"workload": name, "ms": r_ms, "gelem_s": ww.elements / (r_ms * 1e-3) / 1e9,
                               "t_hbm_ms": th, "t_fp32_ms": ta, "roofline_frac": max(th, ta) / r_ms, "path": path})
             out["all_workloads"] = table
+            # the rows built around the hot path, each timed on its own benchmark mode (few steps: reported, not the headline)
+            import copy
+            rows = []
+            for op, wl, fn in (("conv (circular mode)", "periodic2d", None), ("mixer", "volume3d", measure_mixer),
+                               ("synth", "volume3d", measure_synth), ("backward", "volume3d", measure_backward)):
+                try:
+                    if fn is None:
+                        r, p2, tens = time_workload(ALL_WORKLOADS[wl], 5, 3, None, device, False)
+                        p2.close()
+                        del tens, p2
+                        nb, fl, _ = op_algorithmic(ALL_WORKLOADS[wl])
+                        th, ta = nb / (hbm_gbs * 1e9) * 1e3, fl / (fp32_tf * 1e12) * 1e3
+                        rows.append({"op": op, "workload": wl, "ms": r["ms"], "roofline_frac": max(th, ta) / r["ms"]})
+                    else:
+                        a2 = copy.copy(args)
+                        a2.workload, a2.steps, a2.warmup, a2.batch, a2.channels = wl, 3, 3, None, None
+                        if not hasattr(a2, "hidden"):
+                            a2.hidden, a2.layers = 32, 2
+                        d = fn(a2, sample_clocks=False)
+                        frac = d.get("op_roofline", d.get("roofline", {})).get("frac")
+                        rows.append({"op": op, "workload": wl, "ms": d["ms_per_step"], "roofline_frac": frac})
+                    torch.cuda.empty_cache()
+                except Exception as exc:                          # reported rows: never fail the benchmark line
+                    rows.append({"op": op, "workload": wl, "unavailable": repr(exc)[:200]})
+            out["next_rows"] = rows
         if not args.no_cpu:
             out["cpu_baseline"] = cpu_oracle_sample(w)
     if rank == 0:
@@ -468,7 +493,7 @@ def main_ours(args):
 
 # ---- the full operator of Eq. 2 (pointwise stages + long convolution) ------------------------------------
 
-def main_mixer(args):
+def measure_mixer(args, sample_clocks=True):
     """`--op mixer`: times hyenand_mixer_forward (Eq. 2) on the workload, inputs resident in HBM.  The long
     convolution inside runs on an fp32 plan; its kernels are timed by the library, the pointwise stages are the
     remainder."""
@@ -486,8 +511,9 @@ def main_mixer(args):
     for _ in range(max(args.warmup, 3)):
         mx.forward(q, k, v, h, g_in, g_out, y)
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
-    time.sleep(0.6)
+    sampler = ClockSampler(0) if sample_clocks else None
+    if sampler is not None:
+        time.sleep(0.6)
     for _ in range(3):
         mx.forward(q, k, v, h, g_in, g_out, y)
     torch.cuda.synchronize()
@@ -505,7 +531,7 @@ def main_mixer(args):
         mx.forward(q, k, v, h, g_in, g_out, y)
     torch.cuda.synchronize()
     t1 = time.time()
-    clocks = sampler.stop(t0, t1)
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
     conv_ms = 0.0
     kernels = []
     for kid in range(hn.hyenand_plan_kernel_count(inner)):
@@ -524,7 +550,7 @@ def main_mixer(args):
     fp32_tf = fp32_peak_tflops(torch.cuda.get_device_properties(0).multi_processor_count, sm_max)
     nbytes, flops, P = op_algorithmic(w)
     t_hbm, t_alu = nbytes / (hbm_gbs * 1e9) * 1e3, flops / (fp32_tf * 1e12) * 1e3
-    print(json.dumps({
+    return {
         "metric": "hyenand_mixer_throughput", "value": w.elements / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
         "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
@@ -534,12 +560,12 @@ def main_mixer(args):
         "op_roofline": {"t_hbm_ms": t_hbm, "t_fp32_ms": t_alu, "roofline_ms": max(t_hbm, t_alu),
                         "frac": max(t_hbm, t_alu) / ms,
                         "note": "minimal bytes and transform flops of the long convolution; the pointwise stages add no minimal traffic"},
-        "clocks": clocks, "device_status": status, "guard_damage": damage}))
+        "clocks": clocks, "device_status": status, "guard_damage": damage}
 
 
 # ---- backward pass ------------------------------------------------------------------------------------------
 
-def main_backward(args):
+def measure_backward(args, sample_clocks=True):
     """`--op backward`: times hyenand_backward (dq, dk, dv, dh) on the workload, inputs resident in HBM.  Roofline:
     the minimal traffic of the gradient (q, k, v, h, dy in; dq, dk, dv, dh out) and the transforms a direct spectral
     formulation needs (k v, dy q and h forward; dq, du, dh inverse), charged like the forward's."""
@@ -555,8 +581,9 @@ def main_backward(args):
     for _ in range(max(args.warmup, 3)):
         bw(q, k, v, h, dy)
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
-    time.sleep(0.6)
+    sampler = ClockSampler(0) if sample_clocks else None
+    if sampler is not None:
+        time.sleep(0.6)
     bw(q, k, v, h, dy)
     torch.cuda.synchronize()
     outs = [torch.empty_like(q), torch.empty_like(q), torch.empty_like(q), torch.empty_like(h)]
@@ -570,7 +597,7 @@ def main_backward(args):
     torch.cuda.synchronize()
     t1 = time.time()
     ms = e0.elapsed_time(e1) / args.steps
-    clocks = sampler.stop(t0, t1)
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
     damage = hn.hyenand_backward_guard_damage(bw.handle)
     if damage != 0:
         raise SystemExit(f"backward: {damage} damaged guard bytes: the timing is void")
@@ -584,7 +611,7 @@ def main_backward(args):
     transforms = 5 * w.B * w.C + hcount
     flops = transforms * 2.5 * P * math.log2(P) if P > 1 else 0.0
     t_hbm, t_alu = nbytes / (hbm_gbs * 1e9) * 1e3, flops / (fp32_tf * 1e12) * 1e3
-    print(json.dumps({
+    return {
         "metric": "hyenand_backward_throughput", "value": w.elements / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
         "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
@@ -593,12 +620,12 @@ def main_backward(args):
         "op_roofline": {"t_hbm_ms": t_hbm, "t_fp32_ms": t_alu, "roofline_ms": max(t_hbm, t_alu), "frac": max(t_hbm, t_alu) / ms,
                         "min_bytes": nbytes, "nominal_flops": flops,
                         "note": "six transforms per slice (five when the kernel is shared over the batch) at 2.5 P log2 P"},
-        "clocks": clocks, "guard_damage": damage}))
+        "clocks": clocks, "guard_damage": damage}
 
 
 # ---- kernel synthesis ---------------------------------------------------------------------------------------
 
-def main_synth(args):
+def measure_synth(args, sample_clocks=True):
     """`--op synth`: times hyenand_synthesize_kernel for the workload's kernel grid (SIREN of `--hidden` units and
     `--layers` hidden layers, FiLM-modulated per batch entry when the kernel is per sample).  Bound: FP32 ALUs
     (one fused multiply-add per weight and tap), reported against the derived FP32 peak."""
@@ -627,8 +654,9 @@ def main_synth(args):
     for _ in range(max(args.warmup, 3)):
         run()
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
-    time.sleep(0.6)
+    sampler = ClockSampler(0) if sample_clocks else None
+    if sampler is not None:
+        time.sleep(0.6)
     for _ in range(3):
         run()
     torch.cuda.synchronize()
@@ -641,14 +669,14 @@ def main_synth(args):
     torch.cuda.synchronize()
     t1 = time.time()
     ms = e0.elapsed_time(e1) / args.steps
-    clocks = sampler.stop(t0, t1)
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
     taps = Bk * math.prod(w.taps)
     flops = 2.0 * taps * (Hf * (N + 1) + (J - 1) * Hf * (Hf + 1) + w.C * (Hf + 1))
     hbm_gbs, peak_src, sm_max = measured_peaks()
     fp32_tf = fp32_peak_tflops(torch.cuda.get_device_properties(0).multi_processor_count, sm_max)
     out_bytes = taps * w.C * (4 if w.dtype == "f32" else 2)
     ach = flops / (ms * 1e-3) / 1e12
-    print(json.dumps({
+    return {
         "metric": "hyenand_kernel_synthesis_throughput", "value": taps * w.C / (ms * 1e-3) / 1e9, "unit": "Gtap/s (taps x channels)",
         "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
         "dtype": "f32", "io_dtype": w.dtype, "data": "synthetic",
@@ -658,7 +686,7 @@ def main_synth(args):
                      "traffic": None, "peak_source": "derived: 2 x 128 FP32 lanes x SMs x max SM clock",
                      "flops": "2 per weight and tap (fused multiply-adds of the three layer kinds); sines and exponentials not counted",
                      "t_hbm_ms_for_the_output": out_bytes / (hbm_gbs * 1e9) * 1e3},
-        "clocks": clocks}))
+        "clocks": clocks}
 
 
 # ---- reference arm: the CPU oracle ----------------------------------------------------------------
@@ -725,10 +753,10 @@ if __name__ == "__main__":
     if a.impl == "reference":
         main_reference(a)
     elif a.op == "mixer":
-        main_mixer(a)
+        print(json.dumps(measure_mixer(a)))
     elif a.op == "synth":
-        main_synth(a)
+        print(json.dumps(measure_synth(a)))
     elif a.op == "backward":
-        main_backward(a)
+        print(json.dumps(measure_backward(a)))
     else:
         main_ours(a)

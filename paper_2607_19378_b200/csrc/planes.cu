@@ -144,22 +144,6 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
 
 // ---- filter planes ----------------------------------------------------------------------------------
 
-// Spectra of two real rows packed in one half-length transform of the ODD bins (kx = 2k+1): the
-// partner of bin k is bin HP-1-k.  Results go to column k of the column store, rows y0 and y1.
-template <int LOG2H, int CSS>
-__device__ __forceinline__ void separate_rows_odd(const float2 *line, float2 *cs, int y0, int y1, int l)
-{
-    constexpr int H = 1 << LOG2H, TPL = WF<LOG2H, false>::TPL;
-#pragma unroll
-    for (int t = 0; t < H / 2 / TPL; ++t) {
-        const int k = l + t * TPL;
-        const float2 z1 = line[WF<LOG2H, false>::ph(k)];
-        const float2 z2 = line[WF<LOG2H, false>::ph(H - 1 - k)];
-        cs[k * CSS + y0] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
-        cs[k * CSS + y1] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
-    }
-}
-
 // A filter plane has P rows of P taps: twice the rows and columns of a k*v plane, too much for one
 // column store.  The transform along x is split by one decimation-in-frequency step: the even bins
 // of a row are the half-length transform of f[x] + f[x + P/2], the odd bins that of

@@ -417,3 +417,50 @@ def test_host_forward_pipeline_matches_device_forward(dims, B, C, dtype, causal,
     finally:
         plan.close()
     assert torch.equal(y_host, y_dev.cpu())
+
+
+def test_reporting_helpers_and_nvtx_switch(monkeypatch):
+    """hyenand_plan_groups reports how a forward schedules the batch; the NVTX switch (a range per kernel launch,
+    read at plan creation) does not change results."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem((70, 40, 50), B=3, C=3, dtype="bf16", seed=91)
+    monkeypatch.setenv("HYENAND_GROUP_SLICES", "2")
+    monkeypatch.setenv("HYENAND_LANES", "3")
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    assert hn.hyenand_plan_groups(plan.handle) == (2, 3)
+    assert hn.hyenand_plan_launches(plan.handle, False) == 5 * 4          # five groups of four kernels
+    y0 = plan.forward(q.cuda(), k.cuda(), v.cuda(), h.cuda()).cpu()
+    plan.close()
+    monkeypatch.setenv("HYENAND_NVTX", "1")
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    y1 = plan.forward(q.cuda(), k.cuda(), v.cuda(), h.cuda()).cpu()
+    plan.close()
+    assert torch.equal(y0.view(torch.uint8), y1.view(torch.uint8))
+    fused = hn.Plan((32, 32), 1, 2)
+    assert hn.hyenand_plan_groups(fused.handle) == (2, 1)
+    fused.close()
+
+
+def test_long_1d_tensor_maps_follow_the_callers_buffers():
+    """The long 1-D path encodes tensor maps for the caller's q, k, v, h, y and caches them per thread: calls that
+    alternate between two sets of buffers (and a third call with the first set's pointers holding new data) must each
+    see their own tensors."""
+    from paper_2607_19378_b200 import hyenand as hn
+    wa, ta = W.random_problem((65536,), B=1, C=2, dtype="bf16", causal=True, seed=92)
+    wb, tb = W.random_problem((65536,), B=1, C=2, dtype="bf16", causal=True, seed=93)
+    plan = hn.Plan(wa.dims, wa.B, wa.C, causal=True, dtype=wa.torch_dtype)
+    da, db = [t.cuda() for t in ta], [t.cuda() for t in tb]
+    ya, yb = torch.empty_like(da[0]), torch.empty_like(db[0])
+    for _ in range(2):
+        plan.forward(*da, ya)
+        plan.forward(*db, yb)
+    torch.cuda.synchronize()
+    ra, rb = oracle.conv_fft(*ta, "causal"), oracle.conv_fft(*tb, "causal")
+    assert oracle.rel_l2(ya.cpu(), ra) <= TOL["bf16"] and oracle.rel_l2(yb.cpu(), rb) <= TOL["bf16"]
+    for d, t in zip(da, tb):
+        d.copy_(t)                                        # same pointers, other data
+    plan.forward(*da, ya)
+    torch.cuda.synchronize()
+    assert hn.hyenand_plan_device_status(plan.handle) == 0
+    plan.close()
+    assert oracle.rel_l2(ya.cpu(), rb) <= TOL["bf16"]
