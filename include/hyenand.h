@@ -140,6 +140,22 @@ int hyenand_plan_device_status(hyenand_plan *plan);
  * memory checker on machines where none can be run. */
 long long hyenand_plan_guard_damage(hyenand_plan *plan);
 
+/* Checked build.  libhyenand_debug.so is this library compiled with -DHYENAND_DEBUG: every load, store, asynchronous
+ * copy and L2 prefetch a kernel makes to global memory is first compared with the address ranges the call may touch
+ * (the caller's tensors and the device allocations of the objects involved; tensor copies are bounded by their
+ * tensor maps and shared-memory indices are not checked).  An access outside all ranges is counted; it is still made.
+ * hyenand_debug_build returns 1 in that library, 0 in the product library.  hyenand_debug_violations synchronises the
+ * device and returns the number of such accesses since the last call (clearing the count), with the address, source
+ * line and source file of the first one; -1 in the product library.  The paper has no counterpart; it stands in for
+ * a memory checker on machines where none can be run.  Every call of the checked library synchronises the device. */
+int hyenand_debug_build(void);
+long long hyenand_debug_violations(unsigned long long *first_address, int *first_line, const char **file);
+/* Self-test of the checked build: fills a registered and an unregistered device buffer of 1000 floats (both valid
+ * allocations, so nothing faults) and returns the number of accesses the checker counted for the second one
+ * (1000 when it works); -1 in the product library, -2 when memory could not be had, -3 when the registered buffer
+ * was flagged, -4 when the reported address lies outside the unregistered buffer. */
+long long hyenand_debug_selftest(void);
+
 /* Self-test of the mechanism behind hyenand_plan_device_status: launches one small CTA that waits, for at
  * most `polls` polls (clamped to [1, 65536]), on a barrier that nothing ever completes.  The wait must run out
  * and the kernel must report it: returns 9 (the code that kernel records), 0 if the wait wrongly succeeded,

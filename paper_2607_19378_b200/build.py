@@ -36,7 +36,10 @@ def _newest_header():
     return t
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compiles and links the library; debug=True builds the checked variant (-DHYENAND_DEBUG) as libhyenand_debug.so."""
+    OBJ = os.path.join(HERE, "build_debug" if debug else "build")
+    LIB = os.path.join(HERE, "libhyenand_debug.so" if debug else "libhyenand.so")
     os.makedirs(OBJ, exist_ok=True)
     hdr = _newest_header()
     jobs = []
@@ -51,6 +54,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     def compile_one(job):
         s, o = job
         flags = [f for f in FLAGS if not (f == "--use_fast_math" and os.path.basename(s) in PRECISE)]
+        if debug:
+            flags = flags + ["-DHYENAND_DEBUG"]
         r = subprocess.run([NVCC] + flags + ["-c", s, "-o", o], capture_output=True, text=True)
         with open(o[:-2] + ".ptxas.log", "w") as f:
             f.write(r.stderr)
@@ -76,4 +81,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

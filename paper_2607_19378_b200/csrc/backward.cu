@@ -48,30 +48,34 @@ __global__ void __launch_bounds__(kBwdThreads) remap_kernel(RemapArgs r)
         float val = 0.f;
         if (j0 >= 0 && j0 < r.Ls[0] && j1 >= 0 && j1 < r.Ls[1] && j2 >= 0 && j2 < r.Ls[2]) {
             const long long src = s * svol + ((long long)j0 * r.Ls[1] + j1) * r.Ls[2] + j2;
+            HN_G(r.a + src, 4);
+            if (r.b) HN_G(r.b + src, 4);
             val = __ldg(r.a + src);
             if (r.b) val *= __ldg(r.b + src);
         }
+        HN_G(r.out + e, 4);
         r.out[e] = val;
     }
 }
 
 __global__ void fill_kernel(float *dst, float value, long long n)
 {
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) dst[i] = value;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) { HN_G(dst + i, 4); dst[i] = value; }
 }
 
 template <typename T> __global__ void mul_cast_kernel(const float *a, const float *b, long long n, T *dst)
 {
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
-        IO<T>::st(dst, i, b ? a[i] * b[i] : a[i]);
+        { HN_G(a + i, 4); if (b) HN_G(b + i, 4); IO<T>::st(dst, i, b ? a[i] * b[i] : a[i]); }
 }
 
 __global__ void batch_sum_kernel(const float *src, long long nb, long long C, long long kvol, int set, float *acc)
 {
     const long long total = C * kvol;
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+        HN_G(acc + e, 4);
         float s = set ? 0.f : acc[e];
-        for (long long b = 0; b < nb; ++b) s += src[b * total + e];      // fixed order: the result does not depend on scheduling
+        for (long long b = 0; b < nb; ++b) { HN_G(src + b * total + e, 4); s += src[b * total + e]; }      // fixed order: the result does not depend on scheduling
         acc[e] = s;
     }
 }

@@ -8,17 +8,72 @@ namespace hn {
 
 typedef __nv_bfloat16 bf16;
 
+// ---- checked build -----------------------------------------------------------------------------------------
+// With -DHYENAND_DEBUG (libhyenand_debug.so) every access to global memory that a kernel makes through its own
+// instructions (loads, stores, asynchronous copies, L2 prefetches; tensor copies are bounded by their tensor maps) is
+// first compared with the list of address ranges the call may touch: the caller's tensors and the device allocations
+// of the objects involved.  An access outside all of them is counted, with its address and source line; the access
+// itself is still made (the checked build must behave like the product build).  It stands in for a memory checker
+// on machines where none can be run.  Each translation unit holds its own copy of the list and of the counters
+// (no relocatable device code), kept in step by hooks registered at load time.
+constexpr int kDbgRanges = 96;
+struct DbgRanges {
+    unsigned long long lo[kDbgRanges], hi[kDbgRanges];
+    int n;
+};
+struct DbgReport {
+    unsigned long long count, first_address;
+    int first_line;
+    const char *file;
+};
+typedef void (*DbgHook)(const DbgRanges *set, unsigned long long *collect);
+void dbg_register(DbgHook hook, const char *file);
+void dbg_set_ranges(const DbgRanges &r);           // uploads to every translation unit
+DbgReport dbg_collect();                           // sums and clears the counters of every translation unit
+}  // namespace hn
+
+#ifdef HYENAND_DEBUG
+static __device__ hn::DbgRanges hn_dbg_ranges;
+static __device__ unsigned long long hn_dbg_bad[4];        // count, first address, first line
+namespace hn {
+__device__ __forceinline__ void dbg_check(const void *p, unsigned bytes, int line)
+{
+    if (!__isGlobal(p)) return;                            // generic pointers into shared memory are not this check's business
+    const unsigned long long a = (unsigned long long)p;
+    bool ok = false;
+    for (int i = 0; i < hn_dbg_ranges.n; ++i) ok |= a >= hn_dbg_ranges.lo[i] && a + bytes <= hn_dbg_ranges.hi[i];
+    if (!ok && atomicAdd(&hn_dbg_bad[0], 1ull) == 0) { hn_dbg_bad[1] = a; hn_dbg_bad[2] = (unsigned long long)line; }
+}
+}  // namespace hn
+static void hn_dbg_hook(const hn::DbgRanges *set, unsigned long long *collect)
+{
+    if (set) cudaMemcpyToSymbol(hn_dbg_ranges, set, sizeof(*set));
+    if (collect) {
+        cudaMemcpyFromSymbol(collect, hn_dbg_bad, sizeof(unsigned long long) * 4);
+        const unsigned long long zero[4] = {0, 0, 0, 0};
+        cudaMemcpyToSymbol(hn_dbg_bad, zero, sizeof(zero));
+    }
+}
+namespace { struct HnDbgRegistrar { HnDbgRegistrar() { hn::dbg_register(hn_dbg_hook, __BASE_FILE__); } } hn_dbg_registrar; }
+#define HN_G(p, bytes) hn::dbg_check((p), (unsigned)(bytes), __LINE__)
+#else
+#define HN_G(p, bytes) ((void)0)
+#endif
+
+namespace hn {
+
 template <typename T> struct IO;
 template <> struct IO<float> {
-    static __device__ __forceinline__ float ld(const float *p, long long i) { return __ldg(p + i); }
-    static __device__ __forceinline__ void st(float *p, long long i, float v) { p[i] = v; }
+    static __device__ __forceinline__ float ld(const float *p, long long i) { HN_G(p + i, 4); return __ldg(p + i); }
+    static __device__ __forceinline__ void st(float *p, long long i, float v) { HN_G(p + i, 4); p[i] = v; }
 };
 template <> struct IO<bf16> {
     static __device__ __forceinline__ float ld(const bf16 *p, long long i)
     {
+        HN_G(p + i, 2);
         return __bfloat162float(__ldg(p + i));
     }
-    static __device__ __forceinline__ void st(bf16 *p, long long i, float v) { p[i] = __float2bfloat16_rn(v); }
+    static __device__ __forceinline__ void st(bf16 *p, long long i, float v) { HN_G(p + i, 2); p[i] = __float2bfloat16_rn(v); }
 };
 
 // Optional per-kernel timing: when enabled, every kernel launch of a forward is

@@ -96,7 +96,7 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
     const int gid = TPL == 16 ? ((tid >> 5) * 2 + ((tid >> 3) & 1)) : tid / TPL;
     const unsigned m = TPL == 16 ? (0x00ff00ffu << (tid & 8)) : F::group_mask(tid);
     float2 *line = lines + gid * G::LS;
-    for (int t = tid; t < N; t += kTmaThreads) twt[t] = p.gtw[t * (p.gtw_n / N)];
+    for (int t = tid; t < N; t += kTmaThreads) { HN_G(p.gtw + t * (p.gtw_n / N), 8); twt[t] = p.gtw[t * (p.gtw_n / N)]; }
     if (tid == 0) {
         mbar_init(bar_h, 1);
         mbar_init(bar_u, 1);

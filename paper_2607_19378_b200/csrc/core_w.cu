@@ -18,10 +18,12 @@ __host__ __device__ constexpr int core_threads(int) { return 256; }
 __device__ __forceinline__ void cp_async8(void *smem_dst, const void *gmem_src)
 {
     const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    HN_G(gmem_src, 8);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(d), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async8_s(unsigned smem_addr, const void *gmem_src)
 {
+    HN_G(gmem_src, 8);
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(smem_addr), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
@@ -60,7 +62,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
     const unsigned m = F::group_mask(tid);
     float2 *uline = bu + gid * LS;
     float2 *hline = bh + gid * LS;
-    for (int t = tid; t < N; t += kCoreThreads) twt[t] = p.gtw[t * (p.gtw_n / N)];
+    for (int t = tid; t < N; t += kCoreThreads) { HN_G(p.gtw + t * (p.gtw_n / N), 8); twt[t] = p.gtw[t * (p.gtw_n / N)]; }
     __syncthreads();
     // twiddles: registers when both passes are equal (they depend on the lane only), else
     // per-pass tables
@@ -188,7 +190,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
             float2 *dst = p.out + o * p.out_outer + c0 + x + (long long)r0 * p.nc;
             const long long step = (long long)RPS * p.nc;
             if (c0 + x < p.nc)
-                for (int pos = r0; pos < p.n_out; pos += RPS, dst += step) *dst = bu[x * LS + FI::ph(pos)];
+                for (int pos = r0; pos < p.n_out; pos += RPS, dst += step) { HN_G(dst, 8); *dst = bu[x * LS + FI::ph(pos)]; }
         }
         __syncthreads();
         if (tn < tiles) issue_u(tn);

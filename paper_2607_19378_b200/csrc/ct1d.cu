@@ -47,6 +47,8 @@ struct TwoLevel {
 };
 __device__ __forceinline__ float2 twiddle_p(const TwoLevel &t, unsigned j)
 {
+    HN_G(t.coarse + (j >> t.lo), 8);
+    HN_G(t.fine + (j & ((1u << t.lo) - 1)), 8);
     const float2 c = __ldg(t.coarse + (j >> t.lo));
     const float2 f = __ldg(t.fine + (j & ((1u << t.lo) - 1)));
     return cmul(c, f);
@@ -118,6 +120,7 @@ __global__ void __launch_bounds__(kThreads) ct_cols_fwd_kernel(ColsFwdArgs p)
             const unsigned t2 = 2u * (c0 + x);
             A0 = cmul(A0, twiddle_p(p.twp, t2 * (unsigned)f1));
             A1 = cmul(A1, twiddle_p(p.twp, (t2 + 1u) * (unsigned)f1));
+            HN_G(dst + (long long)f1 * P2 + t2, 16);
             *reinterpret_cast<float4 *>(dst + (long long)f1 * P2 + t2) = make_float4(A0.x, A0.y, A1.x, A1.y);
         }
         __syncthreads();
@@ -158,6 +161,8 @@ __global__ void __launch_bounds__(kThreads) ct_core_kernel(CoreArgs p)
                 const long long s = r / p.f1n;
                 const int f1 = (int)(r % p.f1n);
                 const long long hs = p.h_mod ? (s + p.h_off) % p.h_mod : s;
+                HN_G(p.u + r * P2 + t2, 8);
+                HN_G(p.h + (hs * p.f1n + f1) * P2 + t2, 8);
                 a = p.u[r * P2 + t2];
                 b = __ldg(p.h + (hs * p.f1n + f1) * P2 + t2);
             }
@@ -181,6 +186,7 @@ __global__ void __launch_bounds__(kThreads) ct_core_kernel(CoreArgs p)
             if (r >= rows) continue;
             const int f1 = (int)(r % p.f1n);
             const float2 w = twiddle_p(p.twp, (unsigned)t2 * (unsigned)f1);
+            HN_G(p.u + r * P2 + t2, 8);
             p.u[r * P2 + t2] = cmulc(bu[g * LS + phys(t2)], w);
         }
         __syncthreads();
@@ -225,6 +231,7 @@ __global__ void __launch_bounds__(kThreads) ct_cols_inv_kernel(ColsInvArgs p)
             if (x < width) {
                 const bool mirror = pos > P1 / 2;
                 const int f1 = mirror ? P1 - pos : pos;
+                HN_G(src + (long long)f1 * P2 + 2 * (c0 + x), 16);
                 float4 ab = *reinterpret_cast<const float4 *>(src + (long long)f1 * P2 + 2 * (c0 + x));
                 if (mirror) { ab.y = -ab.y; ab.w = -ab.w; }
                 c = make_float2(ab.x - ab.w, ab.y + ab.z);

@@ -41,6 +41,7 @@ __host__ __device__ constexpr int ct_inv_tx(int tpl) { return kCtInvThreads / tp
 template <int BYTES> __device__ __forceinline__ void cp_async_n(void *smem_dst, const void *gmem_src)
 {
     const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    HN_G(gmem_src, BYTES);
     asm volatile("cp.async.ca.shared.global [%0], [%1], %2;\n" ::"r"(d), "l"(gmem_src), "n"(BYTES) : "memory");
 }
 
@@ -50,6 +51,8 @@ struct TwoLevelW {
 };
 __device__ __forceinline__ float2 twp_w(const TwoLevelW &t, unsigned j)
 {
+    HN_G(t.coarse + (j >> t.lo), 8);
+    HN_G(t.fine + (j & ((1u << t.lo) - 1)), 8);
     const float2 c = __ldg(t.coarse + (j >> t.lo));
     const float2 f = __ldg(t.fine + (j & ((1u << t.lo) - 1)));
     return cmul(c, f);
@@ -154,6 +157,8 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
             } else {
                 for (int e = 0; e < 2 * PG; ++e) {
                     const bool ok = e0 + e < p.len;
+                    if (ok) HN_G(reinterpret_cast<const T *>(ab) + base + e0 + e, sizeof(T));
+                    if (ok && HAS_B) HN_G(reinterpret_cast<const T *>(bb) + base + e0 + e, sizeof(T));
                     reinterpret_cast<T *>(d)[e] = ok ? reinterpret_cast<const T *>(ab)[base + e0 + e] : T(0.f);
                     if (HAS_B)
                         reinterpret_cast<T *>(d + (size_t)HP1 * RS)[e] = ok ? reinterpret_cast<const T *>(bb)[base + e0 + e] : T(0.f);
@@ -249,6 +254,7 @@ ct_cols_fwd_w_kernel(ColsFwdWArgs p, const __grid_constant__ CUtensorMap map_a, 
         float2 *dst = p.out + s * (long long)F1 * P2 + 2 * c0;
         for (int idx = tid; idx < F1 * TX; idx += kCtThreads) {
             const int f1 = idx / TX, x = idx % TX;
+            HN_G(dst + (long long)f1 * P2 + 2 * x, 16);
             *reinterpret_cast<float4 *>(dst + (long long)f1 * P2 + 2 * x) =
                 *reinterpret_cast<const float4 *>(lines + x * LS + 2 * f1);
         }
@@ -288,8 +294,8 @@ __global__ void __launch_bounds__(256, 2) ct_hspec_w_kernel(HspecArgs p)
     for (long long r = (long long)blockIdx.x * G + gid; r < p.rows; r += (long long)gridDim.x * G) {
         float2 *row = p.h + r * P2;
         F::template run<PRUNE_NONE>(l, m, tw, line,
-            [&](int, int, int idx) { return row[idx]; },
-            [&](int, int, int idx, float2 v) { row[idx] = make_float2(v.x * p.scale, v.y * p.scale); });
+            [&](int, int, int idx) { HN_G(row + idx, 8); return row[idx]; },
+            [&](int, int, int idx, float2 v) { HN_G(row + idx, 8); row[idx] = make_float2(v.x * p.scale, v.y * p.scale); });
         __syncwarp(m);
     }
 }
@@ -357,7 +363,10 @@ __global__ void __launch_bounds__(256, 2) ct_core_w_kernel(CoreWArgs p)
 #pragma unroll
         for (int i = 0; i < PL::IPL; ++i)
 #pragma unroll
-            for (int rr = 0; rr < PL::R; ++rr) Y[i][rr] = cmul(Y[i][rr], __ldg(hrow + F::last_pos(l, i, rr)));
+            for (int rr = 0; rr < PL::R; ++rr) {
+                HN_G(hrow + F::last_pos(l, i, rr), 8);
+                Y[i][rr] = cmul(Y[i][rr], __ldg(hrow + F::last_pos(l, i, rr)));
+            }
         __syncwarp(m);
         FI::template pass<0, PRUNE_NONE>(l, twi,
             [&](int i, int rr, int) { return Y[i][rr]; },
@@ -377,6 +386,7 @@ __global__ void __launch_bounds__(256, 2) ct_core_w_kernel(CoreWArgs p)
                 // legs of one item come in order r = 0, 1, ...: positions idx = l + i*TPL + r*(P2/R)
                 if (r % 4 == 0) w = cmul(cl, twp_w(p.twp, (unsigned)f1 * (unsigned)(idx - l)));
                 else w = cmul(w, stp);
+                HN_G(row + idx, 8);
                 row[idx] = cmulc(v, w);
             });
         __syncwarp(m);
@@ -510,6 +520,7 @@ ct_cols_inv_w_kernel(ColsInvWArgs p, const __grid_constant__ CUtensorMap map_q, 
         for (int e = 0; e < NE; ++e) {
             const int t1 = tb + e * TSTEP;
             const long long tt = (long long)t1 * P2 + 2 * (c0 + x);
+            if (tt < p.len) HN_G(pq + ox + (long long)t1 * P2, 2 * sizeof(T));
             if (tt < p.len) qv[e] = __ldg(reinterpret_cast<const Q2 *>(pq + ox + (long long)t1 * P2));
         }
 #pragma unroll
@@ -519,6 +530,7 @@ ct_cols_inv_w_kernel(ColsInvWArgs p, const __grid_constant__ CUtensorMap map_q, 
             if (tt < p.len) {
                 const float2 z = lines[x * LS + FI::ph(t1)];
                 const long long o = ox + (long long)t1 * P2;
+                HN_G(py + o, 2 * sizeof(T));
                 if constexpr (sizeof(T) == 4) {
                     *reinterpret_cast<float2 *>(py + o) = make_float2(z.x * qv[e].x, z.y * qv[e].y);
                 } else {

@@ -14,6 +14,7 @@
 #pragma once
 #include <type_traits>
 #include <cuda_runtime.h>
+#include "common.cuh"
 
 namespace hn {
 
@@ -397,7 +398,7 @@ __device__ __forceinline__ void fft_lines(float2 *buf, int G, int LS, const floa
 __device__ __forceinline__ void load_twiddles(float2 *tw, const float2 *gt, int N, int NT, int tid, int T)
 {
     const int step = NT / N;
-    for (int t = tid; t < N / 2; t += T) tw[t] = gt[t * step];
+    for (int t = tid; t < N / 2; t += T) { HN_G(gt + t * step, 8); tw[t] = gt[t * step]; }
 }
 
 }  // namespace hn

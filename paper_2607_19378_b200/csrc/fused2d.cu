@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
-    for (int t = tid; t < P; t += kF2Threads) tw[t] = p.gtw[t * (p.gtw_n >> LOG2P)];
+    for (int t = tid; t < P; t += kF2Threads) { HN_G(p.gtw + t * (p.gtw_n >> LOG2P), 8); tw[t] = p.gtw[t * (p.gtw_n >> LOG2P)]; }
     __syncthreads();
     PlaneTw<LOG2P, false> twf;
     twf.init(l, tw, tw + P, tid, kF2Threads);

@@ -23,6 +23,33 @@ Switches read_switches()
     return s;
 }
 
+// ---- checked build: hooks of the translation units ----------------------------------------------------------
+static DbgHook g_dbg_hooks[32];
+static const char *g_dbg_files[32];
+static int g_dbg_n = 0;
+
+void dbg_register(DbgHook hook, const char *file)
+{
+    if (g_dbg_n < 32) { g_dbg_hooks[g_dbg_n] = hook; g_dbg_files[g_dbg_n] = file; ++g_dbg_n; }
+}
+
+void dbg_set_ranges(const DbgRanges &r)
+{
+    for (int i = 0; i < g_dbg_n; ++i) g_dbg_hooks[i](&r, nullptr);
+}
+
+DbgReport dbg_collect()
+{
+    DbgReport rep{0, 0, 0, nullptr};
+    for (int i = 0; i < g_dbg_n; ++i) {
+        unsigned long long c[4] = {0, 0, 0, 0};
+        g_dbg_hooks[i](nullptr, c);
+        if (c[0] && !rep.count) { rep.first_address = c[1]; rep.first_line = (int)c[2]; rep.file = g_dbg_files[i]; }
+        rep.count += c[0];
+    }
+    return rep;
+}
+
 void nvtx_push(const char *name) { nvtxRangePushA(name); }
 void nvtx_pop() { nvtxRangePop(); }
 

@@ -34,6 +34,87 @@ static int fail(int code, const char *fmt, ...)
     return code;
 }
 
+// Checked build: the address ranges a call may touch (the caller's tensors, the device allocations of the objects
+// involved), handed to every translation unit before the call's kernels are enqueued.
+struct DbgScope {
+#ifdef HYENAND_DEBUG
+    DbgRanges r;
+    DbgScope() { r.n = 0; }
+    void add(const void *ptr, size_t bytes)
+    {
+        if (ptr && bytes && r.n < kDbgRanges) { r.lo[r.n] = (unsigned long long)ptr; r.hi[r.n] = r.lo[r.n] + bytes; ++r.n; }
+    }
+    void add(const GuardedAllocs &g)
+    {
+        for (int i = 0; i < g.n; ++i) add(g.recs[i].base + kGuardBytes, g.recs[i].bytes);
+    }
+    void commit()
+    {
+        cudaDeviceSynchronize();               // kernels of earlier calls still compare against the previous list
+        dbg_set_ranges(r);
+    }
+#else
+    void add(const void *, size_t) {}
+    void add(const GuardedAllocs &) {}
+    void commit() {}
+#endif
+};
+
+extern "C" int hyenand_debug_build(void)
+{
+#ifdef HYENAND_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+extern "C" long long hyenand_debug_violations(unsigned long long *first_address, int *first_line, const char **file)
+{
+#ifdef HYENAND_DEBUG
+    cudaDeviceSynchronize();
+    const DbgReport rep = dbg_collect();
+    if (first_address) *first_address = rep.first_address;
+    if (first_line) *first_line = rep.first_line;
+    if (file) *file = rep.file ? rep.file : "";
+    return (long long)rep.count;
+#else
+    if (first_address) *first_address = 0;
+    if (first_line) *first_line = 0;
+    if (file) *file = "";
+    return -1;
+#endif
+}
+
+extern "C" long long hyenand_debug_selftest(void)
+{
+#ifdef HYENAND_DEBUG
+    // Two valid buffers; only the first is registered.  Filling the first must count nothing, filling the second
+    // must count every element: no access leaves allocated memory, so nothing faults.
+    float *a = nullptr, *b = nullptr;
+    const long long n = 1000;
+    if (cudaMalloc(&a, n * sizeof(float)) != cudaSuccess) return -2;
+    if (cudaMalloc(&b, n * sizeof(float)) != cudaSuccess) { cudaFree(a); return -2; }
+    cudaDeviceSynchronize();
+    (void)dbg_collect();
+    DbgScope d;
+    d.add(a, n * sizeof(float));
+    d.commit();
+    launch_fill(a, 1.f, n, nullptr);
+    cudaDeviceSynchronize();
+    const DbgReport clean = dbg_collect();
+    launch_fill(b, 1.f, n, nullptr);
+    cudaDeviceSynchronize();
+    const DbgReport dirty = dbg_collect();
+    cudaFree(a); cudaFree(b);
+    if (clean.count != 0) return -3;
+    if (dirty.first_address < (unsigned long long)b || dirty.first_address >= (unsigned long long)(b + n)) return -4;
+    return (long long)dirty.count;
+#else
+    return -1;
+#endif
+}
+
 enum Path { PATH_ND_GENERIC = 0, PATH_CT1D = 1, PATH_PLANES3D = 2, PATH_FUSED2D = 3 };
 constexpr int kMaxLanes = 4;
 
@@ -690,6 +771,14 @@ extern "C" int hyenand_forward_ex(hyenand_plan *p, const void *q, const void *k,
     if (!e) e = check_overlap(p, shared, q, k, v, h, y);
     if (!e) e = check_device(p);
     if (e) return e;
+    {
+        DbgScope d;
+        const size_t nbytes = (size_t)p->B * p->C * p->vol * elsize(p->dtype);
+        d.add(q, nbytes); d.add(k, nbytes); d.add(v, nbytes); d.add(y, nbytes);
+        d.add(h, (size_t)(shared ? 1 : p->B) * p->C * p->kvol * elsize(p->dtype));
+        d.add(p->allocs);
+        d.commit();
+    }
     int launches = 0;
     return run_forward(p, q, k, v, h, shared, y, (cudaStream_t)cuda_stream, &launches);
 }
@@ -729,6 +818,12 @@ extern "C" int hyenand_forward_host(hyenand_plan *p, const void *q, const void *
             p->ws_bytes += want[i];
             p->stage_bytes[i] = want[i];
         }
+    }
+    {
+        DbgScope d;
+        for (int i = 0; i < 5; ++i) d.add(p->stage[i], p->stage_bytes[i]);
+        d.add(p->allocs);
+        d.commit();
     }
     // Pipeline over groups of slices: the inputs of group g+1 travel to the device (copy-in stream) while group g
     // is computed (caller's stream) and the result of group g-1 travels back (copy-out stream).  A filter shared
@@ -1051,6 +1146,15 @@ extern "C" int hyenand_mixer_forward(hyenand_mixer *m, const void *q, const void
             if (yb < ib + ilen && ib < yb + nbytes) return fail(HYENAND_ERR_INVALID_ARG, "y overlaps input %d", i);
         }
     }
+    {
+        DbgScope d;
+        const size_t nbytes = (size_t)m->B * m->C * m->L * es;
+        d.add(q, nbytes); d.add(k, nbytes); d.add(v, nbytes); d.add(y, nbytes);
+        d.add(h, (size_t)(shared ? 1 : m->B) * m->C * m->kvol * es);
+        d.add(g_in, (size_t)m->C * sizeof(float)); d.add(g_out, (size_t)m->C * sizeof(float));
+        d.add(m->allocs); d.add(p->allocs);
+        d.commit();
+    }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const size_t slab = (size_t)m->C * m->L;                        // elements per batch entry
     const float *hf = (const float *)h;
@@ -1218,6 +1322,7 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
         hyenand_backward_destroy(g);
         return nullptr;
     }
+    { DbgScope d; d.add(g->allocs); d.commit(); }
     launch_fill(g->ones, 1.f, S * g->vol, 0);
     if (g->ring) launch_fill(g->rones, 1.f, g->ns * g->pvol, 0);
     if (cudaDeviceSynchronize() != cudaSuccess) {
@@ -1256,6 +1361,18 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
         return fail(HYENAND_ERR_INVALID_ARG, "h_batch_stride_elems must be 0 or C*K_1*..*K_N = %lld", (long long)g->C * g->kvol);
     int e = check_device(g->main);
     if (e) return e;
+    {
+        DbgScope d;
+        const size_t nbytes = (size_t)g->B * g->C * g->vol * elsize(g->dtype);
+        const size_t hbytes = (size_t)(shared ? 1 : g->B) * g->C * g->kvol * elsize(g->dtype);
+        d.add(q, nbytes); d.add(k, nbytes); d.add(v, nbytes); d.add(dy, nbytes); d.add(dq, nbytes); d.add(dk, nbytes); d.add(dv, nbytes);
+        d.add(h, hbytes); d.add(dh, hbytes);
+        d.add(g->allocs); d.add(g->main->allocs);
+        if (g->adj != g->main) d.add(g->adj->allocs);
+        if (g->ring) d.add(g->ring->allocs);
+        if (g->caus && g->caus != g->main) d.add(g->caus->allocs);
+        d.commit();
+    }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const size_t es = elsize(g->dtype);
     const bool widen = g->dtype == HYENAND_BF16;
@@ -1415,6 +1532,17 @@ extern "C" int hyenand_synthesize_kernel(int ndim, const int *dims, int mode, in
     }
     a.W1 = W1; a.b1 = b1; a.omega0 = omega0; a.Wh = Wh; a.bh = bh; a.Wout = Wout; a.bout = bout;
     a.gamma = gamma; a.beta = beta; a.window = window; a.h = h; a.dtype = dtype;
+    {
+        DbgScope d;
+        const size_t f = sizeof(float);
+        d.add(W1, f * hidden * ndim); d.add(b1, f * hidden); d.add(omega0, f * hidden);
+        d.add(Wh, f * (size_t)(layers - 1) * hidden * hidden); d.add(bh, f * (size_t)(layers - 1) * hidden);
+        d.add(Wout, f * (size_t)C * hidden); d.add(bout, f * C);
+        d.add(gamma, f * (size_t)B * layers * hidden); d.add(beta, f * (size_t)B * layers * hidden);
+        d.add(window, f * (size_t)(mode == HYENAND_MODE_CAUSAL ? C : ndim * C));
+        d.add(h, (size_t)B * C * a.K[0] * a.K[1] * a.K[2] * elsize(dtype));
+        d.commit();
+    }
     if (launch_synth(a, (cudaStream_t)cuda_stream) < 0) return fail(HYENAND_ERR_UNSUPPORTED, "kernel grid too large for one launch");
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(HYENAND_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
@@ -1539,6 +1667,14 @@ extern "C" int hyenand_forward_noalloc(int ndim, const int *dims, int B, int C, 
     ln.wh_a = (float2 *)(base + off); off += ha * (unsigned long long)ln.wh_slices;
     ln.wh_b = three ? (float2 *)(base + off) : nullptr; off += hb2 * (unsigned long long)ln.wh_slices;
     // the per-slice strides used by the kernels are the unrounded ones; the carve only has to be large enough
+    {
+        DbgScope d;
+        const size_t nbytes = (size_t)B * C * p->vol * elsize(dtype);
+        d.add(q, nbytes); d.add(k, nbytes); d.add(v, nbytes); d.add(y, nbytes);
+        d.add(h, (size_t)(shared ? 1 : B) * C * p->kvol * elsize(dtype));
+        d.add(base, HYENAND_NOALLOC_MAX_BYTES);
+        d.commit();
+    }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     noalloc_twiddle_kernel<<<(p->gtw_n + 255) / 256, 256, 0, st>>>(p->gtw, p->gtw_n);
     int launches = 1;

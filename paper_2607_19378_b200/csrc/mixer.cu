@@ -39,6 +39,7 @@ __global__ void __launch_bounds__(kMixThreads) mixer_pre_kernel(const T *q, cons
         const float scale = inv_norm * rsqrtf(s2 * inv_norm * inv_norm / (float)C + eps);
         for (int c = 0; c < C; ++c) {
             const float qc = IO<T>::ld(q, base + c * L), kc = IO<T>::ld(k, base + c * L), vc = IO<T>::ld(v, base + c * L);
+            HN_G(g_in + c, 4); HN_G(kz + base + c * L, 4); HN_G(vz + base + c * L, 4); HN_G(qz + base + c * L, 4);
             kz[base + c * L] = qc * scale * __ldg(g_in + c);
             vz[base + c * L] = kc * sigmoidf_(kc);
             qz[base + c * L] = sigmoidf_(vc);
@@ -56,18 +57,19 @@ __global__ void __launch_bounds__(kMixThreads) mixer_post_kernel(const float *o,
         const long long base = b * C * L + i;
         float s = 0.f;
         for (int c = 0; c < C; ++c) {
+            HN_G(o + base + c * L, 4);
             const float oc = __ldg(o + base + c * L);
             s = fmaf(oc, oc, s);
         }
         const float scale = rsqrtf(s / (float)C + eps);
-        for (int c = 0; c < C; ++c) IO<T>::st(y, base + c * L, __ldg(o + base + c * L) * scale * __ldg(g_out + c));
+        for (int c = 0; c < C; ++c) { HN_G(g_out + c, 4); IO<T>::st(y, base + c * L, __ldg(o + base + c * L) * scale * __ldg(g_out + c)); }
     }
 }
 
 template <typename T> __global__ void widen_kernel(const T *src, long long n, float *dst)
 {
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
-        dst[i] = IO<T>::ld(src, i);
+        { HN_G(dst + i, 4); dst[i] = IO<T>::ld(src, i); }
 }
 
 static int mix_grid(long long items)

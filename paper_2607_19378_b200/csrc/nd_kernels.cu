@@ -84,8 +84,8 @@ __global__ void __launch_bounds__(kThreads) rows_fwd_kernel(RowsArgs p)
             const long long r0 = 2 * (ch * G + g), r1 = r0 + 1;
             const float2 z1 = buf[g * LS + phys(kx)];
             const float2 z2 = buf[g * LS + phys((N - kx) & (N - 1))];
-            if (r0 < p.rows) p.out[r0 * p.pitch + kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
-            if (r1 < p.rows) p.out[r1 * p.pitch + kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
+            if (r0 < p.rows) { HN_G(p.out + r0 * p.pitch + kx, 8); p.out[r0 * p.pitch + kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y)); }
+            if (r1 < p.rows) { HN_G(p.out + r1 * p.pitch + kx, 8); p.out[r1 * p.pitch + kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x)); }
         }
         __syncthreads();
     }
@@ -162,8 +162,8 @@ __global__ void __launch_bounds__(kThreads) rows_inv_kernel(RowsInvArgs p)
             const bool mirror = pos > N / 2;
             const int kx = mirror ? N - pos : pos;
             float2 A = make_float2(0.f, 0.f), B = A;
-            if (r0 < p.rows) A = p.in[r0 * p.pitch + kx];
-            if (r1 < p.rows) B = p.in[r1 * p.pitch + kx];
+            if (r0 < p.rows) { HN_G(p.in + r0 * p.pitch + kx, 8); A = p.in[r0 * p.pitch + kx]; }
+            if (r1 < p.rows) { HN_G(p.in + r1 * p.pitch + kx, 8); B = p.in[r1 * p.pitch + kx]; }
             if (mirror) { A.y = -A.y; B.y = -B.y; }
             buf[g * LS + phys(pos)] = make_float2(A.x - B.y, A.y + B.x);
         }
@@ -219,7 +219,7 @@ __device__ __forceinline__ void fill_tile(float2 *buf, int LS, int TX, const flo
         const int x = idx % TX, pos = idx / TX;
         const int m = (pos + shift) & (N - 1);
         float2 val = make_float2(0.f, 0.f);
-        if (m < n_in && x < width) val = src[(long long)m * nc + x];
+        if (m < n_in && x < width) { HN_G(src + (long long)m * nc + x, 8); val = src[(long long)m * nc + x]; }
         buf[x * LS + phys(pos)] = val;
     }
 }
@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kThreads) axis_kernel(AxisArgs p)
         float2 *dst = p.out + o * p.out_outer + c0;
         for (int idx = tid; idx < TX * p.n_out; idx += kThreads) {
             const int x = idx % TX, a = idx / TX;
-            if (x < width) dst[(long long)a * p.nc + x] = bu[x * LS + phys(a)];
+            if (x < width) { HN_G(dst + (long long)a * p.nc + x, 8); dst[(long long)a * p.nc + x] = bu[x * LS + phys(a)]; }
         }
         __syncthreads();
     }

@@ -20,6 +20,7 @@ __device__ __forceinline__ void prefetch_l2(const void *ptr, long long bytes, in
     constexpr unsigned long long CH = 4096;
     for (unsigned long long a = a0 + (unsigned long long)tid * CH; a < a1; a += (unsigned long long)kPlaneThreads * CH) {
         const unsigned sz = (unsigned)(a1 - a < CH ? a1 - a : CH);
+        HN_G((const void *)a, sz);
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(a), "r"(sz) : "memory");
     }
 }
@@ -27,6 +28,7 @@ __device__ __forceinline__ void prefetch_l2(const void *ptr, long long bytes, in
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
 {
     const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    HN_G(gmem_src, 16);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
@@ -50,8 +52,10 @@ __device__ __forceinline__ void stage_row(unsigned char *dst, const unsigned cha
         if (g >= lo && g + 16 <= hi) cp_async16(dst + 16 * c, g);
         else {
             for (int b = 0; b < 16; b += 2)
-                if (g + b >= src && g + b < src + n)
+                if (g + b >= src && g + b < src + n) {
+                    HN_G(g + b, 2);
                     *reinterpret_cast<unsigned short *>(dst + 16 * c + b) = *reinterpret_cast<const unsigned short *>(g + b);
+                }
         }
     }
 }

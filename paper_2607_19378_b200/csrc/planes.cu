@@ -44,8 +44,8 @@ template <int LOG2P> __device__ __forceinline__ void load_plane_twiddles(float2 
 {
     constexpr int P = 1 << LOG2P;
     const int step = gtw_n >> LOG2P;
-    for (int t = tid; t < P; t += kPlaneThreads) tw[t] = gtw[t * step];
-    for (int t = tid; t < P / 2; t += kPlaneThreads) twh[t] = gtw[2 * t * step];
+    for (int t = tid; t < P; t += kPlaneThreads) { HN_G(gtw + t * step, 8); tw[t] = gtw[t * step]; }
+    for (int t = tid; t < P / 2; t += kPlaneThreads) { HN_G(gtw + 2 * t * step, 8); twh[t] = gtw[2 * t * step]; }
 }
 
 // ---- k*v planes ---------------------------------------------------------------------------------
@@ -127,11 +127,13 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
             float2 *d = kx != 0 ? dst + (long long)kx * P : tmp;
             F::template run<PRUNE_IN>(l, m, twp, line,
                 [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); },
-                [&](int, int, int idx, float2 v) { d[idx] = v; });
+                [&](int, int, int idx, float2 v) { HN_G(d + idx, 8); d[idx] = v; });
             if (kx == 0) {
                 __syncwarp(m);
                 for (int ky = l; ky < P; ky += TPL) {
                     const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
+                    HN_G(dst + ky, 8);
+                    HN_G(dst + (long long)HP * P + ky, 8);
                     dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
                     dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                 }
@@ -313,11 +315,13 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                         const float c = par ? -za.x : za.y, dd2 = par ? -zm.x : zm.y;
                         return make_float2(a + b, c - dd2);
                     },
-                    [&](int, int, int idx, float2 v) { d[idx] = v; });
+                    [&](int, int, int idx, float2 v) { HN_G(d + idx, 8); d[idx] = v; });
                 if (packed) {
                     __syncwarp(m);
                     for (int ky = l; ky < P; ky += TPL) {
                         const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
+                        HN_G(dst + ky, 8);
+                        HN_G(dst + (long long)HP * P + ky, 8);
                         dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
                         dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
                     }
@@ -371,7 +375,10 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
 #pragma unroll
             for (int i = 0; i < P0::IPL; ++i)
 #pragma unroll
-                for (int r = 0; r < P0::R; ++r) pre[i][r] = __ldcg(s + i * TPL + r * (P / P0::R));
+                for (int r = 0; r < P0::R; ++r) {
+                    HN_G(s + i * TPL + r * (P / P0::R), 8);
+                    pre[i][r] = __ldcg(s + i * TPL + r * (P / P0::R));
+                }
         };
         if (gid < HP) fetch(gid);
         if (gid == 0) {
@@ -382,6 +389,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
             for (int i = 0; i < P0::IPL; ++i)
 #pragma unroll
                 for (int r = 0; r < P0::R; ++r) {
+                    HN_G(sn + i * TPL + r * (P / P0::R), 8);
                     const float2 gn = __ldcg(sn + i * TPL + r * (P / P0::R));
                     pre[i][r] = make_float2(pre[i][r].x - gn.y, pre[i][r].y + gn.x);
                 }
@@ -418,6 +426,8 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
 #pragma unroll
                 for (int r = 0; r < PE::R / 2; ++r) {
                     const int idx = FI::last_pos(l, i, r);
+                    if (idx < Lx) HN_G(pq + o0 + idx, sizeof(T));
+                    if (idx < Lx && has1) HN_G(pq + o1 + idx, sizeof(T));
                     q0[i * (PE::R / 2) + r] = idx < Lx ? __ldg(pq + o0 + idx) : T(0.f);
                     q1[i * (PE::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
                 }

@@ -20,6 +20,7 @@ constexpr int kRowThreads = 256;
 __device__ __forceinline__ void prefetch_rows_l2(const unsigned char *lo, const unsigned char *hi)
 {
     const unsigned long long a0 = ((unsigned long long)lo + 15ull) & ~15ull, a1 = (unsigned long long)hi & ~15ull;
+    if (a1 > a0) HN_G((const void *)a0, a1 - a0);
     if (a1 > a0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(a0), "r"((unsigned)(a1 - a0)) : "memory");
 }
 
@@ -38,7 +39,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = F::group_mask(tid);
     float2 *line = smem + gid * LS;
-    for (int t = tid; t < P; t += kRowThreads) twt[t] = p.gtw[t * (p.gtw_n >> LOG2P)];
+    for (int t = tid; t < P; t += kRowThreads) { HN_G(p.gtw + t * (p.gtw_n >> LOG2P), 8); twt[t] = p.gtw[t * (p.gtw_n >> LOG2P)]; }
     __syncthreads();
     PlaneTw<LOG2P, false> tw;
     tw.init(l, twt, twt + P, tid, kRowThreads);
@@ -64,6 +65,8 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
             float2 *o0 = p.out + r0 * p.pitch, *o1 = p.out + r1 * p.pitch;
             for (int kx = l; kx <= HP; kx += TPL) {
                 const float2 z1 = line[F::ph(kx)], z2 = line[F::ph((P - kx) & (P - 1))];
+                HN_G(o0 + kx, 8);
+                if (has1) HN_G(o1 + kx, 8);
                 o0[kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
                 if (has1) o1[kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
             }
@@ -131,6 +134,8 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_fwd_w_kernel(RowsArgs p)
         float2 *o0 = p.out + r0 * p.pitch, *o1 = p.out + r1 * p.pitch;
         for (int kx = l; kx <= HP; kx += TPL) {
             const float2 z1 = line[F::ph(kx)], z2 = line[F::ph((P - kx) & (P - 1))];
+            HN_G(o0 + kx, 8);
+            if (has1) HN_G(o1 + kx, 8);
             o0[kx] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
             if (has1) o1[kx] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
         }
@@ -151,7 +156,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
     const unsigned m = FI::group_mask(tid);
     float2 *line = smem + gid * LS;
-    for (int t = tid; t < P; t += kRowThreads) twt[t] = p.gtw[t * (p.gtw_n >> LOG2P)];
+    for (int t = tid; t < P; t += kRowThreads) { HN_G(p.gtw + t * (p.gtw_n >> LOG2P), 8); twt[t] = p.gtw[t * (p.gtw_n >> LOG2P)]; }
     __syncthreads();
     PlaneTw<LOG2P, true> tw;
     tw.init(l, twt, twt + P, tid, kRowThreads);
@@ -171,6 +176,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
         if (!FULL && p.len == HP && has1 && l == 0) {
             // the two gate rows of the pair (contiguous, a multiple of 16 bytes from a 16-byte boundary)
             const unsigned long long qa = (unsigned long long)(pq + r0 * HP);
+            HN_G((const void *)qa, 2 * HP * sizeof(T));
             asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(qa), "r"((unsigned)(2 * HP * sizeof(T))) : "memory");
         }
         cp_async_wait_all();

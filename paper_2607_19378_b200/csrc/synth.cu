@@ -17,6 +17,9 @@
 
 namespace hn {
 
+// parameter loads (checked in the checked build)
+#define SYN_LD(ptr, idx) (HN_G((ptr) + (idx), 4), (ptr)[idx])
+
 constexpr int kSynThreads = 128;
 constexpr int kSynChanChunk = 32;        // output channels whose weights sit in shared memory at a time
 
@@ -59,19 +62,19 @@ __global__ void __launch_bounds__(kSynThreads) synth_kernel(SynthArgs p)
         // coefficients of the internal axes (0, 1, 2) = the last N of them carry the grid
         for (int a = 0; a < 3; ++a) {
             const int ua = a - (3 - N);                   // user axis
-            sW1[i * 4 + a] = (in && ua >= 0) ? p.W1[i * N + ua] : 0.f;
+            sW1[i * 4 + a] = (in && ua >= 0) ? SYN_LD(p.W1, i * N + ua) : 0.f;
         }
-        sW1[i * 4 + 3] = in ? p.b1[i] : 0.f;
-        sOm[i] = in ? p.omega0[i] : 0.f;
+        sW1[i * 4 + 3] = in ? SYN_LD(p.b1, i) : 0.f;
+        sOm[i] = in ? SYN_LD(p.omega0, i) : 0.f;
         for (int j = 0; j < J; ++j) {
-            sFi[(j * 2 + 0) * HF + i] = in ? (p.gamma ? p.gamma[((long long)b * J + j) * H + i] : 1.f) : 0.f;
-            sFi[(j * 2 + 1) * HF + i] = in ? (p.beta ? p.beta[((long long)b * J + j) * H + i] : 0.f) : 0.f;
+            sFi[(j * 2 + 0) * HF + i] = in ? (p.gamma ? SYN_LD(p.gamma, ((long long)b * J + j) * H + i) : 1.f) : 0.f;
+            sFi[(j * 2 + 1) * HF + i] = in ? (p.beta ? SYN_LD(p.beta, ((long long)b * J + j) * H + i) : 0.f) : 0.f;
         }
-        for (int j = 0; j + 1 < J; ++j) sBh[j * HF + i] = in ? p.bh[j * H + i] : 0.f;
+        for (int j = 0; j + 1 < J; ++j) sBh[j * HF + i] = in ? SYN_LD(p.bh, j * H + i) : 0.f;
     }
     for (int e = tid; e < (J - 1) * HF * HF; e += kSynThreads) {
         const int j = e / (HF * HF), r = (e / HF) % HF, c = e % HF;
-        sWh[e] = (r < H && c < H) ? p.Wh[((long long)j * H + r) * H + c] : 0.f;
+        sWh[e] = (r < H && c < H) ? SYN_LD(p.Wh, ((long long)j * H + r) * H + c) : 0.f;
     }
     __syncthreads();
     const long long taps = (long long)p.K[0] * p.K[1] * p.K[2];
@@ -129,16 +132,16 @@ __global__ void __launch_bounds__(kSynThreads) synth_kernel(SynthArgs p)
         const int nc = p.C - c0 < kSynChanChunk ? p.C - c0 : kSynChanChunk;
         for (int e = tid; e < kSynChanChunk * HF; e += kSynThreads) {
             const int c = e / HF, i = e % HF;
-            sWo[e] = (c < nc && i < H) ? p.Wout[(long long)(c0 + c) * H + i] : 0.f;
+            sWo[e] = (c < nc && i < H) ? SYN_LD(p.Wout, (long long)(c0 + c) * H + i) : 0.f;
         }
         for (int c = tid; c < kSynChanChunk; c += kSynThreads) {
-            sBo[c] = c < nc ? p.bout[c0 + c] : 0.f;
+            sBo[c] = c < nc ? SYN_LD(p.bout, c0 + c) : 0.f;
             for (int a = 0; a < 3; ++a) {
                 const int ua = a - (3 - N);
                 float wv = 0.f;                            // Gaussian: 1 / sigma per axis; causal: alpha in slot 2
                 if (c < nc) {
-                    if (p.mode == 1) wv = a == 2 ? p.window[c0 + c] : 0.f;
-                    else if (ua >= 0) wv = 1.f / p.window[(long long)ua * p.C + c0 + c];
+                    if (p.mode == 1) wv = a == 2 ? SYN_LD(p.window, c0 + c) : 0.f;
+                    else if (ua >= 0) wv = 1.f / SYN_LD(p.window, (long long)ua * p.C + c0 + c);
                 }
                 sWin[a * kSynChanChunk + c] = wv;
             }

@@ -227,6 +227,7 @@ template <int LOG2N, bool INV> struct PassTw {
             const int ns = F::ns(s), rad = F::radix(s), off = offset(s);
             for (int e = tid; e < (rad - 1) * ns; e += nthr) {
                 const int r = e / ns + 1, k = e % ns;
+                HN_G(gtw + r * k * (N / (ns * rad)) * step, 8);
                 dst[off + e] = gtw[r * k * (N / (ns * rad)) * step];
             }
         }

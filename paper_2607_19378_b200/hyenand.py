@@ -13,7 +13,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libhyenand.so")
+# HYENAND_LIB=debug selects the checked build (libhyenand_debug.so, see hyenand_debug_build in the header)
+LIB_PATH = os.path.join(_HERE, "libhyenand_debug.so" if os.environ.get("HYENAND_LIB") == "debug" else "libhyenand.so")
 
 HYENAND_F32 = 0
 HYENAND_BF16 = 1
@@ -54,6 +55,10 @@ def lib() -> ctypes.CDLL:
         L.hyenand_destroy_plan.argtypes = [vp]
         L.hyenand_destroy_plan.restype = None
         L.hyenand_last_error.restype = ctypes.c_char_p
+        L.hyenand_debug_build.restype = ctypes.c_int
+        L.hyenand_debug_violations.restype = ll
+        L.hyenand_debug_violations.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), ip, ctypes.POINTER(ctypes.c_char_p)]
+        L.hyenand_debug_selftest.restype = ll
         L.hyenand_selftest_bounded_wait.argtypes = [ctypes.c_int]
         L.hyenand_selftest_bounded_wait.restype = ctypes.c_int
         L.hyenand_plan_device_status.argtypes = [vp]
@@ -154,6 +159,22 @@ def hyenand_forward_ex(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stre
 def hyenand_forward_host(plan: int, q, k, v, h, h_batch_stride_elems: int, y, stream=None) -> None:
     _check(lib().hyenand_forward_host(plan, q.data_ptr(), k.data_ptr(), v.data_ptr(), h.data_ptr(),
                                       int(h_batch_stride_elems), y.data_ptr(), _stream_ptr(stream)))
+
+
+def hyenand_debug_build() -> bool:
+    return bool(lib().hyenand_debug_build())
+
+
+def hyenand_debug_violations():
+    """(count, first address, first line, first file) of the checked build's out-of-range accesses since the last call;
+    count is -1 in the product library."""
+    addr, line, name = ctypes.c_ulonglong(), ctypes.c_int(), ctypes.c_char_p()
+    n = lib().hyenand_debug_violations(ctypes.byref(addr), ctypes.byref(line), ctypes.byref(name))
+    return int(n), int(addr.value), int(line.value), (name.value or b"").decode()
+
+
+def hyenand_debug_selftest() -> int:
+    return int(lib().hyenand_debug_selftest())
 
 
 def hyenand_selftest_bounded_wait(polls: int = 1000) -> int:
