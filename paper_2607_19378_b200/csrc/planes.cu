@@ -151,14 +151,27 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
 // of a row are the half-length transform of f[x] + f[x + P/2], the odd bins that of
 // (f[x] - f[x + P/2]) W_P^x.  Each half (e = 0: even kx, e = 1: odd kx) fills a column store of
 // P/4 columns by P rows, whose columns are then transformed along y and written out as whole lines.
-// The two real rows that share a complex row transform are NOT separated after it: the raw transform Z of every row
-// pair goes straight from the last pass's registers into the store [bin k][row pair], and the column transform of bin k
-// separates them as it loads (it reads Z[k] and the mirrored bin of each row pair: the same number of shared-memory
-// wavefronts as reading separated values, no separation pass and no extra trip of the row results through the line).
-// Separated values come out at twice their value (the factor 1/2 of the separation is left to the spectral core's scale).
-// The tap rows are fetched and unpacked once per plane: while a thread prepares the even half it also forms its
-// inputs of the odd half, f[x] - f[x + P/2], and parks them in tensor memory (its own lane, 2 * points-per-thread
+//
+// Two real rows share one complex row transform: padded rows y and y + P/2 (row pair p = y mod P/2).  They are NOT
+// separated after it: the raw transform Z of every row pair goes straight from the last pass's registers into the
+// store [bin k][row pair], and the column transform of bin k separates them as it loads.  A lane's first-pass inputs
+// y = j + r P/R come from the row pairs p = j + r P/R, r < R/2, both members each, so one pair of loads (Z[k] and the
+// mirrored bin Z[k']) yields two inputs:
+//   2 F_y[k] = Z[k] + conj Z[k'],   2 F_{y+P/2}[k] = -i (Z[k] - conj Z[k']),
+// k' = (H - k) mod H in the even half, H - 1 - k in the odd one (H = P/2 bins per half).  Separated values come out at
+// twice their value (the factor 1/2 is left to the spectral core's scale).
+//
+// Tap rows are staged so that no index wraps: padded position x holds tap (x + Lx - 1) mod P, so the P positions of
+// a row are a window W of P consecutive tap indices starting at -(P/2 + 1 - Lx), with zeros outside [0, Kx):
+// position x + P/2 is W[x], position x is W[x + P/2] (x < P/2).  A thread's taps sit at constant offsets from one
+// address.  The tap rows are fetched and unpacked once per plane: while a thread prepares the even half it also forms
+// its inputs of the odd half, f[x] - f[x + P/2], and parks them in tensor memory (its own lane, 2 * points-per-thread
 // columns per row pair); the odd half reads them back instead of staging the rows again.
+//
+// The purely real bins kx = 0 and kx = P/2 of every row travel as one complex column (column 0 of the even half): its
+// store entries are rewritten by the row phase so that the common separation formulas deliver (2 F_y[0], 2 F_y[P/2])
+// for it; its raw transform goes to a shared-memory line, which the whole CTA unpacks into lines 0 and P/2 of the
+// output after the column phase.
 template <typename T, int LOG2P>
 __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
 {
@@ -177,14 +190,16 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     const int tid = threadIdx.x;
     const int l = tid % TPL, gid = tid / TPL;
     const int lh = tid % TPLH, gidh = tid / TPLH;
-    const unsigned m = F::group_mask(tid), mh = FH::group_mask(tid);
+    constexpr unsigned FULL = 0xffffffffu;                   // every warp runs the loops below in step: whole-warp barriers
     float2 *line = wbuf + gid * C::LS;
     float2 *lineh = wbuf + gidh * C::LSH;
     using PH0 = typename FH::template Pass<0>;
+    using PC0 = typename F::template Pass<0>;
     constexpr int NPT = 2 * PH0::IPL * PH0::R;               // parked values per thread and row pair
     constexpr int ROUNDS = HP / C::NGH;                      // row pairs per lane group and half
     constexpr int TCOLS = 4 * ROUNDS * NPT;                  // four warps share each 32-lane quadrant
     static_assert(HP % C::NGH == 0 && TCOLS >= 32 && TCOLS <= 512 && (TCOLS & (TCOLS - 1)) == 0, "tensor-memory columns");
+    static_assert(QP % C::NG == 0 || C::NG % QP == 0, "whole warps take part in the column loop");
     const int warp = tid >> 5;
     unsigned *tslot = reinterpret_cast<unsigned *>(smem + C::TMP + P);
     if (warp == 0) tmem_alloc((unsigned)__cvta_generic_to_shared(tslot), TCOLS);
@@ -202,131 +217,144 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     __syncthreads();
     const unsigned char *hb = (const unsigned char *)p.a;
     const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
-    constexpr int R0 = FH::template Pass<0>::R;
-    const int c0 = (lh + Lx - 1) & (P - 1);                  // tap of padded position x: (x + Lx - 1) mod P
+    constexpr int R0 = PH0::R;
+    const int J0 = HP + 1 - Lx;                              // window position of tap 0
+    const int RU = (J0 * (int)sizeof(T) + 15) & ~15;         // bytes kept free before the first copied chunk
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const long long ib = pl * (long long)Ky * Kx;
         float2 *dst = p.out + pl * (long long)C::XH * P;
         for (int e = 0; e < 2; ++e) {
-            // rows: padded row y holds tap row (y + Ly - 1) mod P; two rows per transform
+            // the next plane's taps travel to L2 during the second half, when this plane's are on chip
+            if (e == 1 && pl + gridDim.x < p.planes)
+                prefetch_l2(hb + (pl + gridDim.x) * (long long)Ky * Kx * sizeof(T), (long long)Ky * Kx * sizeof(T), tid);
+            if (e == 1 && tid < P) {
+                // the raw transform C of the packed column (bins kx = 0 and kx = P/2 of every row) waits in a shared-memory
+                // line since the column phase that has just ended: the two bins are (C[ky] + conj C[-ky]) / 2 and
+                // -i (C[ky] - conj C[-ky]) / 2.  (The line is next written two CTA barriers from here.)
+                const int ky = tid;
+                const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
+                float2 *dn = dst + (long long)HP * P;
+                HN_G(dst + ky, 8);
+                HN_G(dn + ky, 8);
+                dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
+                dn[ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
+            }
+            // rows: padded row y holds tap row (y + Ly - 1) mod P; rows y and y + P/2 share a transform (at most one
+            // of the two lies in the zero band, which is shorter than P/2 rows)
             int round = 0;
             // the two groups of a half warp take row pairs 8 apart, so their stores (one row pair per group, consecutive
             // bins per lane) fall into different banks
             for (int rp = spread_pair<8>(gidh); rp < HP; rp += C::NGH, ++round) {
-                const int y0 = 2 * rp, y1 = y0 + 1;
-                const int my0 = (y0 + Ly - 1) & (P - 1), my1 = (y1 + Ly - 1) & (P - 1);
-                const bool v0 = my0 < Ky, v1 = my1 < Ky, valid = v0 || v1;
+                const int my0 = (rp + Ly - 1) & (P - 1), my1 = my0 ^ HP;
+                const bool v0 = my0 < Ky, v1 = my1 < Ky;
                 // STAGED: both tap rows are fetched with 16-byte copies into the line itself, which
                 // the first pass reads before anything is written to it; 4-byte taps do not fit the
                 // half-length line and are read from global memory (L2) directly
                 constexpr bool STAGED = sizeof(T) == 2;
-                constexpr int SLOT = ((C::P - 1) * (int)sizeof(T) + 15) / 16 * 16 + 16;   // bytes kept per staged row
+                constexpr int SLOT = 4 * HP + 48;            // bytes kept per staged row: window, alignment slack, last chunk
                 static_assert(!STAGED || 2 * SLOT + 32 <= C::LSH * 8, "staged rows must fit the line");
                 // the four lines of a warp start 0, 64, 0, 64 bytes into the 128-byte bank row:
                 // lines 2 and 3 stage 32 bytes further in, so the narrow tap loads do not collide
                 unsigned char *s0 = reinterpret_cast<unsigned char *>(lineh) + 16 * (gidh & 2), *s1 = s0 + SLOT;
                 const unsigned char *g0 = hb + (ib + (long long)my0 * Kx) * sizeof(T);
                 const unsigned char *g1 = hb + (ib + (long long)my1 * Kx) * sizeof(T);
-                const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
                 const int n0 = v0 ? Kx : 0, n1 = v1 ? Kx : 0;
-                auto tap0 = [&](int mx) -> float {
-                    if constexpr (STAGED) return staged<T>(s0, f0, mx);
-                    else return mx < n0 ? IO<T>::ld(reinterpret_cast<const T *>(g0), mx) : 0.f;
-                };
-                auto tap1 = [&](int mx) -> float {
-                    if constexpr (STAGED) return staged<T>(s1, f1, mx);
-                    else return mx < n1 ? IO<T>::ld(reinterpret_cast<const T *>(g1), mx) : 0.f;
-                };
                 float dd[NPT];                                // this thread's inputs of the odd half, before the twiddle
                 float ss[NPT];                                // and of the even half
                 const unsigned tcol = tpark + round * NPT;
                 if (e == 0) {
-                    if (valid) {
-                        if constexpr (STAGED) {
-                            if (v0) stage_row<TPLH>(s0, g0, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
-                            if (v1) stage_row<TPLH>(s1, g1, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
-                            cp_async_wait_all();
-                            __syncwarp(mh);
-                            // blank the padding taps (and a missing row) once: the input functors are branch-free
-                            zero_staged<T, TPLH>(s0, f0, v0 ? Kx : 0, P, lh);
-                            zero_staged<T, TPLH>(s1, f1, v1 ? Kx : 0, P, lh);
-                            __syncwarp(mh);
+                    if constexpr (STAGED) {
+                        const int f0 = (int)((unsigned long long)g0 & 15ull), f1 = (int)((unsigned long long)g1 & 15ull);
+                        if (v0) stage_row_u<TPLH, (2 * HP - 1) * (int)sizeof(T)>(s0 + RU, g0, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
+                        if (v1) stage_row_u<TPLH, (2 * HP - 1) * (int)sizeof(T)>(s1 + RU, g1, Kx * (int)sizeof(T), hb, hb + p.a_elems * sizeof(T), lh);
+                        cp_async_wait_all();
+                        __syncwarp();
+                        // window element j sits at w + 2 j; blank what lies outside the row once, so the tap loads
+                        // need no bounds test
+                        unsigned char *w0 = s0 + RU + f0 - J0 * (int)sizeof(T), *w1 = s1 + RU + f1 - J0 * (int)sizeof(T);
+                        for (int j = lh; j < J0; j += TPLH) {
+                            *reinterpret_cast<T *>(w0 + j * sizeof(T)) = T(0.f);
+                            *reinterpret_cast<T *>(w1 + j * sizeof(T)) = T(0.f);
                         }
+                        for (int j = J0 + n0 + lh; j < P; j += TPLH) *reinterpret_cast<T *>(w0 + j * sizeof(T)) = T(0.f);
+                        for (int j = J0 + n1 + lh; j < P; j += TPLH) *reinterpret_cast<T *>(w1 + j * sizeof(T)) = T(0.f);
+                        __syncwarp();
+                        const T *t0 = reinterpret_cast<const T *>(w0) + lh, *t1 = reinterpret_cast<const T *>(w1) + lh;
 #pragma unroll
                         for (int i = 0; i < PH0::IPL; ++i)
 #pragma unroll
                             for (int r = 0; r < R0; ++r) {
-                                const int ma = (c0 + i * TPLH + r * (HP / R0)) & (P - 1), mb = ma ^ HP;
-                                const float a0 = tap0(ma), b0 = tap0(mb), a1 = tap1(ma), b1 = tap1(mb);
+                                const int x = i * TPLH + r * (HP / R0);          // + lh: position of this input
+                                const float a0 = (float)t0[x + HP], b0 = (float)t0[x], a1 = (float)t1[x + HP], b1 = (float)t1[x];
                                 ss[2 * (i * R0 + r)] = a0 + b0;
                                 ss[2 * (i * R0 + r) + 1] = a1 + b1;
                                 dd[2 * (i * R0 + r)] = a0 - b0;
                                 dd[2 * (i * R0 + r) + 1] = a1 - b1;
                             }
                     } else {
+                        const T *r0 = reinterpret_cast<const T *>(g0), *r1 = reinterpret_cast<const T *>(g1);
 #pragma unroll
-                        for (int t = 0; t < NPT; ++t) dd[t] = 0.f;
+                        for (int i = 0; i < PH0::IPL; ++i)
+#pragma unroll
+                            for (int r = 0; r < R0; ++r) {
+                                const int x = lh + i * TPLH + r * (HP / R0);
+                                const int ta = x + Lx - 1, tb = x - J0;          // tap indices of positions x and x + P/2
+                                const float a0 = ta < n0 ? IO<T>::ld(r0, ta) : 0.f, a1 = ta < n1 ? IO<T>::ld(r1, ta) : 0.f;
+                                const float b0 = (tb >= 0 && tb < n0) ? IO<T>::ld(r0, tb) : 0.f;
+                                const float b1 = (tb >= 0 && tb < n1) ? IO<T>::ld(r1, tb) : 0.f;
+                                ss[2 * (i * R0 + r)] = a0 + b0;
+                                ss[2 * (i * R0 + r) + 1] = a1 + b1;
+                                dd[2 * (i * R0 + r)] = a0 - b0;
+                                dd[2 * (i * R0 + r) + 1] = a1 - b1;
+                            }
                     }
-                    __syncwarp();                             // the whole warp parks together
+                    __syncwarp();                             // the whole warp parks together; every lane has read its taps
                     TmemIO<NPT>::st(tcol, dd);
                     tmem_wait_st();
-                    if (valid) {
-                        // (every lane of the group has read its taps from the line before the barrier above)
-                        FH::template run<PRUNE_NONE, false>(lh, mh, twr, lineh,
-                            [&](int i, int r, int) { return make_float2(ss[2 * (i * R0 + r)], ss[2 * (i * R0 + r) + 1]); },
-                            [&](int, int, int kk, float2 z) { cs[kk * CS2 + rp] = z; });
-                        __syncwarp(mh);
+                    float2 z0 = make_float2(0.f, 0.f), zh = z0;
+                    FH::template run<PRUNE_NONE, false>(lh, FULL, twr, lineh,
+                        [&](int i, int r, int) { return make_float2(ss[2 * (i * R0 + r)], ss[2 * (i * R0 + r) + 1]); },
+                        [&](int, int r, int kk, float2 z) {
+                            cs[kk * CS2 + rp] = z;
+                            if (r == 0) z0 = z;                                  // lane 0: bins 0 and H/2
+                            if (r == FH::LastPass::R / 2) zh = z;
+                        });
+                    if (lh == 0) {
+                        // Bins 0 and H/2 (both held by lane 0) are the real bins kx = 0 and kx = P/2 of the two rows:
+                        // Z[0] = (F_y[0], F_y'[0]), Z[H/2] = (F_y[P/2], F_y'[P/2]).  They travel as one column (k = 0, mirrored
+                        // bin H/2): with a = (Z0.x - Zh.y, Z0.y + Zh.x), b = (Z0.x + Zh.y, Z0.y - Zh.x) the column phase's
+                        // separation gives a + conj b = 2 (Z0.x, Zh.x) and -i (a - conj b) = 2 (Z0.y, Zh.y).
+                        static_assert(FH::LastPass::IPL == 1 && (HP / 2) % (HP / FH::LastPass::R) == 0, "lane 0 holds bins 0 and H/2");
+                        cs[rp] = make_float2(z0.x - zh.y, z0.y + zh.x);
+                        cs[(HP / 2) * CS2 + rp] = make_float2(z0.x + zh.y, z0.y - zh.x);
                     }
                 } else {
                     __syncwarp();
                     TmemIO<NPT>::ld(dd, tcol);
                     tmem_wait_ld();
-                    if (valid) {
-                        FH::template run<PRUNE_NONE, false>(lh, mh, twr, lineh,
-                            [&](int i, int r, int idx) { return cmul(make_float2(dd[2 * (i * R0 + r)], dd[2 * (i * R0 + r) + 1]), tw[idx]); },
-                            [&](int, int, int kk, float2 z) { cs[kk * CS2 + rp] = z; });
-                        __syncwarp(mh);
-                    }
+                    FH::template run<PRUNE_NONE, false>(lh, FULL, twr, lineh,
+                        [&](int i, int r, int idx) { return cmul(make_float2(dd[2 * (i * R0 + r)], dd[2 * (i * R0 + r) + 1]), tw[idx]); },
+                        [&](int, int, int kk, float2 z) { cs[kk * CS2 + rp] = z; });
                 }
-                if (!valid) {
-                    for (int kk = lh; kk < HP; kk += TPLH) cs[kk * CS2 + rp] = make_float2(0.f, 0.f);
-                }
+                __syncwarp();
             }
             __syncthreads();
             // columns: P-point transforms over y of the bins kx = 2k + e
             for (int k = gid; k < QP; k += C::NG) {
-                // Row y = 2 rp + par of bin k: with Z = F_y0 + i F_y1 the raw transform of row pair rp,
-                //   2 F_y0[k] = Z[k] + conj Z[k'],  2 F_y1[k] = -i (Z[k] - conj Z[k']),
-                // k' the mirrored bin of the half-length transform ((H - k) mod H in the even half, H - 1 - k in the odd one).
-                // A lane's rows y = l + 16 r all have the parity of l.
-                // Column 0 of the even half packs the two purely real bins kx = 0 and kx = P/2 of every row as one
-                // complex number (2 F_y[0], 2 F_y[P/2]); it sends its raw transform to a shared-memory line and is
-                // unpacked afterwards.  One transform code path for all columns.
                 const bool packed = e == 0 && k == 0;
                 const int km = packed ? HP / 2 : (e == 0 ? ((HP - k) & (HP - 1)) : HP - 1 - k);
                 const float2 *ca = cs + k * CS2, *cb = cs + km * CS2;
-                const bool par = l & 1;
                 float2 *d = packed ? tmp : dst + (long long)(2 * k + e) * P;
-                F::template run<PRUNE_NONE>(l, m, twp, line,
-                    [&](int, int, int idx) {
-                        const float2 za = ca[idx >> 1], zm = cb[idx >> 1];
-                        const float a = par ? za.y : za.x, b = par ? zm.y : zm.x;
-                        if (packed) return make_float2(a + a, b + b);
-                        const float c = par ? -za.x : za.y, dd2 = par ? -zm.x : zm.y;
-                        return make_float2(a + b, c - dd2);
+                float2 second[PC0::IPL][PC0::R / 2];          // inputs y + P/2, formed with their partners y
+                F::template run<PRUNE_NONE>(l, FULL, twp, line,
+                    [&](int i, int r, int idx) {
+                        if (r >= PC0::R / 2) return second[i][r - PC0::R / 2];
+                        const float2 za = ca[idx], zm = cb[idx];
+                        second[i][r] = make_float2(za.y + zm.y, zm.x - za.x);
+                        return make_float2(za.x + zm.x, za.y - zm.y);
                     },
                     [&](int, int, int idx, float2 v) { HN_G(d + idx, 8); d[idx] = v; });
-                if (packed) {
-                    __syncwarp(m);
-                    for (int ky = l; ky < P; ky += TPL) {
-                        const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
-                        HN_G(dst + ky, 8);
-                        HN_G(dst + (long long)HP * P + ky, 8);
-                        dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
-                        dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
-                    }
-                }
-                __syncwarp(m);
+                __syncwarp();
             }
             __syncthreads();
         }
