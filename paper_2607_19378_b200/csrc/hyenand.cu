@@ -619,8 +619,8 @@ static AxisArgs planes3d_core_args(const hyenand_plan *p, int l, long long n, bo
     a.log2p = p->log2p[0]; a.prune_in = 1;
     a.h = lh.wh_a; a.h_outer = (long long)p->K[0] * nc; a.h_n_in = p->K[0]; a.h_shift = p->L[0] - 1;
     a.h_mod = shared ? p->C : 0; a.h_off = shared ? s0 % p->C : 0;
-    // 1/P of the inverse transforms, and the factor 1/2 the filter-plane kernel leaves out of its row separation
-    a.scale = (float)(0.5 / ((double)p->P[0] * p->P[1] * p->P[2]));
+    // 1/P of the inverse transforms, and the factors 1/2 the two forward plane kernels leave out of their row separations
+    a.scale = (float)(0.25 / ((double)p->P[0] * p->P[1] * p->P[2]));
     a.gtw = p->gtw; a.gtw_n = p->gtw_n;
     return a;
 }

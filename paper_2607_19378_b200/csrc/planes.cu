@@ -5,8 +5,9 @@
 // shared memory the same way for 1-D and 2-D; it describes no 3-D kernel):
 //
 //   uplane     k*v plane: gate, zero-pad, real-to-complex along x (two real rows
-//              per complex transform), transpose through a shared-memory column
-//              store, complex transform along y.  Output lines are [kx][ky].
+//              per complex transform, separated by the column transform as it loads),
+//              transpose through a shared-memory column store, complex transform
+//              along y.  Output lines are [kx][ky], at twice their value.
 //   hplane     filter plane, which has twice the rows and columns: the even and the odd
 //              bins along x are produced one after the other (one radix-2
 //              decimation-in-frequency step applied to the taps as they are read), each
@@ -36,7 +37,9 @@ template <int LOG2P> struct PlaneCfg {
     static constexpr int LS = plane_ls(P);
     static constexpr int LSH = plane_ls(HP);
     static constexpr int WBUF = (NG * LS > NGH * LSH) ? NG * LS : NGH * LSH;
-    static constexpr size_t TMP = (size_t)HP * CSS + WBUF + P + HP + 2 * P;     // P entries: raw transform of the packed column
+    static constexpr int CSU = P / 4 + 1;                    // k*v planes: P bins of P/4 row pairs (odd stride)
+    static constexpr int CSN = (HP * CSS > P * CSU) ? HP * CSS : P * CSU;       // column store, entries
+    static constexpr size_t TMP = (size_t)CSN + WBUF + P + HP + 2 * P;          // P entries: raw transform of the packed column
     static constexpr size_t SMEM = sizeof(float2) * (TMP + P + 2);      // + the slot that receives the tensor-memory base
 };
 
@@ -55,15 +58,18 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
 {
     using C = PlaneCfg<LOG2P>;
     using F = typename C::F;
-    constexpr int P = C::P, HP = C::HP, TPL = F::TPL;
+    using PC0 = typename F::template Pass<0>;
+    constexpr int P = C::P, HP = C::HP, QP = P / 4, TPL = F::TPL, CSU = C::CSU;
+    constexpr unsigned FULL = 0xffffffffu;                   // every warp runs the loops below in step: whole-warp barriers
+    static_assert(QP % C::NG == 0 || C::NG % QP == 0, "whole warps take part in the row loop");
+    static_assert(HP % C::NG == 0 || C::NG % HP == 0, "whole warps take part in the column loop");
     extern __shared__ float2 smem[];
     float2 *cs = smem;
-    float2 *wbuf = cs + HP * C::CSS;
+    float2 *wbuf = cs + C::CSN;
     float2 *tw = wbuf + C::WBUF;
     float2 *twh = tw + P;
     float2 *tmp = smem + C::TMP;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
-    const unsigned m = F::group_mask(tid);
     float2 *line = wbuf + gid * C::LS;
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
@@ -73,6 +79,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
     const T *pk = (const T *)p.a;
     const T *pv = (const T *)p.b;
     const unsigned char *kb = (const unsigned char *)p.a, *vb = (const unsigned char *)p.b;
+    const unsigned char *ke = kb + p.a_elems * sizeof(T), *ve = vb + p.a_elems * sizeof(T);
     const int Lx = p.lx, Ly = p.ly;
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const long long ib = pl * (long long)Ly * Lx;
@@ -81,66 +88,102 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
             prefetch_l2(pk + nb, (long long)Ly * Lx * sizeof(T), tid);
             prefetch_l2(pv + nb, (long long)Ly * Lx * sizeof(T), tid);
         }
-        for (int rp = gid; 2 * rp < HP; rp += C::NG) {
-            const int y0 = 2 * rp, y1 = y0 + 1;
-            if (y0 < Ly) {
-                const bool has1 = y1 < Ly;
-                // the two rows of k and of v (consecutive in memory) are fetched with 16-byte copies
-                // into the line itself, which the first pass reads before anything is written to it
-                const int nrow = (has1 ? 2 : 1) * Lx * (int)sizeof(T);
-                const unsigned char *gk = kb + (ib + (long long)y0 * Lx) * sizeof(T);
-                const unsigned char *gv = vb + (ib + (long long)y0 * Lx) * sizeof(T);
-                unsigned char *sk = reinterpret_cast<unsigned char *>(line);
-                unsigned char *sv = sk + C::LS * 4;                       // second half of the line
-                stage_row<TPL>(sk, gk, nrow, kb, kb + p.a_elems * sizeof(T), l);
-                stage_row<TPL>(sv, gv, nrow, vb, vb + p.a_elems * sizeof(T), l);
-                cp_async_wait_all();
-                __syncwarp(m);
-                const int ok = (int)((unsigned long long)gk & 15ull), ov = (int)((unsigned long long)gv & 15ull);
-                if (Lx == HP && has1) {
-                    // full rows: no bounds tests in the input functor
-                    F::template run_to_line<PRUNE_IN, true>(l, m, twp, line, [&](int, int, int idx) {
-                        return make_float2(staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx),
-                                           staged<T>(sk, ok, HP + idx) * staged<T>(sv, ov, HP + idx));
-                    });
-                } else {
-                    F::template run_to_line<PRUNE_IN, true>(l, m, twp, line, [&](int, int, int idx) {
-                        float a = 0.f, b = 0.f;
-                        if (idx < Lx) {
-                            a = staged<T>(sk, ok, idx) * staged<T>(sv, ov, idx);
-                            if (has1) b = staged<T>(sk, ok, Lx + idx) * staged<T>(sv, ov, Lx + idx);
-                        }
-                        return make_float2(a, b);
-                    });
-                }
-                separate_rows<LOG2P, C::CSS>(line, cs, y0, y1, l);
-                __syncwarp(m);
+        // rows: y and y + P/4 share a transform (rows P/4 .. Ly-1 exist, Ly > P/4; a missing partner is a zero row)
+        for (int rp = gid; rp < QP; rp += C::NG) {
+            const int y1 = rp + QP;
+            const bool has1 = y1 < Ly;
+            // the rows of k and of v are fetched with 16-byte copies into the line itself, which the first pass reads
+            // before anything is written to it
+            constexpr int SLOT = HP * (int)sizeof(T) + 32;
+            static_assert(4 * SLOT <= C::LS * 8, "staged rows must fit the line");
+            unsigned char *sk0 = reinterpret_cast<unsigned char *>(line), *sk1 = sk0 + SLOT, *sv0 = sk1 + SLOT, *sv1 = sv0 + SLOT;
+            const int rowb = Lx * (int)sizeof(T);
+            const unsigned char *gk0 = kb + (ib + (long long)rp * Lx) * sizeof(T), *gk1 = gk0 + (long long)QP * rowb;
+            const unsigned char *gv0 = vb + (ib + (long long)rp * Lx) * sizeof(T), *gv1 = gv0 + (long long)QP * rowb;
+            stage_row_u<TPL, HP * (int)sizeof(T)>(sk0, gk0, rowb, kb, ke, l);
+            stage_row_u<TPL, HP * (int)sizeof(T)>(sv0, gv0, rowb, vb, ve, l);
+            if (has1) {
+                stage_row_u<TPL, HP * (int)sizeof(T)>(sk1, gk1, rowb, kb, ke, l);
+                stage_row_u<TPL, HP * (int)sizeof(T)>(sv1, gv1, rowb, vb, ve, l);
             }
+            cp_async_wait_all();
+            __syncwarp();
+            const T *k0 = reinterpret_cast<const T *>(sk0 + ((unsigned long long)gk0 & 15ull)) + l;
+            const T *v0 = reinterpret_cast<const T *>(sv0 + ((unsigned long long)gv0 & 15ull)) + l;
+            const T *k1 = reinterpret_cast<const T *>(sk1 + ((unsigned long long)gk1 & 15ull)) + l;
+            const T *v1 = reinterpret_cast<const T *>(sv1 + ((unsigned long long)gv1 & 15ull)) + l;
+            float2 z0 = make_float2(0.f, 0.f), zh = z0;
+            // The raw transform Z of the row pair goes straight into the store [bin][row pair]; the column transform
+            // separates the two rows as it loads.
+            auto keep = [&](int, int r, int kk, float2 z) {
+                cs[kk * CSU + rp] = z;
+                if (r == 0) z0 = z;                           // lane 0: bins 0 and P/2
+                if (r == F::LastPass::R / 2) zh = z;
+            };
+            if (Lx == HP && has1) {
+                // full rows: no bounds tests in the input functor
+                F::template run<PRUNE_IN, true>(l, FULL, twp, line, [&](int i, int r, int) {
+                    const int x = i * TPL + r * (P / PC0::R);                   // + l
+                    return make_float2((float)k0[x] * (float)v0[x], (float)k1[x] * (float)v1[x]);
+                }, keep);
+            } else {
+                F::template run<PRUNE_IN, true>(l, FULL, twp, line, [&](int i, int r, int idx) {
+                    const int x = i * TPL + r * (P / PC0::R);
+                    float a = 0.f, b = 0.f;
+                    if (idx < Lx) {
+                        a = (float)k0[x] * (float)v0[x];
+                        if (has1) b = (float)k1[x] * (float)v1[x];
+                    }
+                    return make_float2(a, b);
+                }, keep);
+            }
+            if (l == 0) {
+                // Bins 0 and P/2 (both held by lane 0) are the real bins of the two rows: Z[0] = (F_y[0], F_y'[0]),
+                // Z[P/2] = (F_y[P/2], F_y'[P/2]).  They travel as one column (kx = 0, mirrored bin P/2): with
+                // a = (Z0.x - Zh.y, Z0.y + Zh.x), b = (Z0.x + Zh.y, Z0.y - Zh.x) the column phase's separation
+                // gives a + conj b = 2 (Z0.x, Zh.x) and -i (a - conj b) = 2 (Z0.y, Zh.y).
+                static_assert(F::LastPass::IPL == 1 && HP % (P / F::LastPass::R) == 0, "lane 0 holds bins 0 and P/2");
+                cs[rp] = make_float2(z0.x - zh.y, z0.y + zh.x);
+                cs[HP * CSU + rp] = make_float2(z0.x + zh.y, z0.y - zh.x);
+            }
+            __syncwarp();
         }
         __syncthreads();
+        // columns: with Z the raw transform of row pair (y, y + P/4),
+        //   2 F_y[kx] = Z[kx] + conj Z[P - kx],   2 F_{y+P/4}[kx] = -i (Z[kx] - conj Z[P - kx]);
+        // a lane's first-pass inputs y = j + r P/R, r < R/2 (the rest is padding), come from the row pairs of r < R/4,
+        // both members each.  Values leave at twice their size (the factor 1/2 is left to the spectral core's scale).
         float2 *dst = p.out + pl * (long long)C::XH * P;
         for (int kx = gid; kx < HP; kx += C::NG) {
-            const float2 *col = cs + kx * C::CSS;
-            // Every column runs the same transform (the group that shares a warp with column 0 must not wait
-            // for a second, different code path): column 0, which packs bins kx = 0 and kx = P/2, only sends
-            // its raw transform to a shared-memory line instead of global memory and unpacks it afterwards.
-            float2 *d = kx != 0 ? dst + (long long)kx * P : tmp;
-            F::template run<PRUNE_IN>(l, m, twp, line,
-                [&](int, int, int idx) { return idx < Ly ? col[idx] : make_float2(0.f, 0.f); },
+            // Column 0 packs bins kx = 0 and kx = P/2 of every row as one complex number; it runs the same transform as
+            // every other column (the group that shares its warp does not wait for a second code path), its raw transform
+            // goes to a shared-memory line and is unpacked after the column phase.
+            const bool packed = kx == 0;
+            const float2 *ca = cs + kx * CSU, *cb = cs + (packed ? HP : P - kx) * CSU;
+            float2 *d = packed ? tmp : dst + (long long)kx * P;
+            float2 second[PC0::IPL][PC0::R / 4];
+            F::template run<PRUNE_IN>(l, FULL, twp, line,
+                [&](int i, int r, int idx) {
+                    if (r >= PC0::R / 4) return second[i][r - PC0::R / 4];
+                    const float2 za = ca[idx], zm = cb[idx];
+                    second[i][r] = make_float2(za.y + zm.y, zm.x - za.x);
+                    return make_float2(za.x + zm.x, za.y - zm.y);
+                },
                 [&](int, int, int idx, float2 v) { HN_G(d + idx, 8); d[idx] = v; });
-            if (kx == 0) {
-                __syncwarp(m);
-                for (int ky = l; ky < P; ky += TPL) {
-                    const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
-                    HN_G(dst + ky, 8);
-                    HN_G(dst + (long long)HP * P + ky, 8);
-                    dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
-                    dst[(long long)HP * P + ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
-                }
-            }
-            __syncwarp(m);
+            __syncwarp();
         }
         __syncthreads();
+        if (tid < P) {
+            // C = raw transform of the packed column: bins kx = 0 and kx = P/2 are (C[ky] + conj C[-ky]) / 2 and
+            // -i (C[ky] - conj C[-ky]) / 2.  (The line is next written after the next CTA barrier.)
+            const int ky = tid;
+            const float2 c1 = tmp[ky], c2 = tmp[(P - ky) & (P - 1)];
+            float2 *dn = dst + (long long)HP * P;
+            HN_G(dst + ky, 8);
+            HN_G(dn + ky, 8);
+            dst[ky] = make_float2(0.5f * (c1.x + c2.x), 0.5f * (c1.y - c2.y));
+            dn[ky] = make_float2(0.5f * (c1.y + c2.y), 0.5f * (c2.x - c1.x));
+        }
     }
 }
 
@@ -183,7 +226,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
     static_assert(HP * CS2 <= HP * C::CSS, "store of a half fits the plane buffer");
     extern __shared__ float2 smem[];
     float2 *cs = smem;
-    float2 *wbuf = cs + HP * C::CSS;
+    float2 *wbuf = cs + C::CSN;
     float2 *tw = wbuf + C::WBUF;
     float2 *twh = tw + P;
     float2 *tmp = smem + C::TMP;
@@ -376,7 +419,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
     constexpr int P = C::P, HP = C::HP, TPL = FI::TPL;
     extern __shared__ float2 smem[];
     float2 *cs = smem;
-    float2 *wbuf = cs + HP * C::CSS;
+    float2 *wbuf = cs + C::CSN;
     float2 *tw = wbuf + C::WBUF;
     float2 *twh = tw + P;
     float2 *tmp = smem + C::TMP;
