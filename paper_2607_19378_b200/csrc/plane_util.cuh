@@ -11,17 +11,16 @@ constexpr int kPlaneThreads = 512;
 // neighbouring lines do not share banks: stride = 8 mod 16 complex numbers
 __host__ __device__ constexpr int plane_ls(int n) { return ((phys_max(n) + 1 + 7) / 16) * 16 + 8; }
 
-// Ask the memory system to bring [ptr, ptr + bytes) into L2 (bulk prefetch, 16-byte granules);
-// the CTA issues it for the plane it will work on next, so that plane's loads hit L2.
+// Ask the memory system to bring [ptr, ptr + bytes) into L2, one prefetch per 128-byte line, the lines dealt out to
+// the CTA's threads (a handful of plain prefetch instructions per thread; a bulk prefetch per thread is executed lane
+// by lane and held the issuing warps up for thousands of cycles).  The CTA issues it for the plane it will work on
+// next, so that plane's loads hit L2.
 __device__ __forceinline__ void prefetch_l2(const void *ptr, long long bytes, int tid)
 {
-    const unsigned long long a0 = (unsigned long long)ptr & ~15ull;
-    const unsigned long long a1 = ((unsigned long long)ptr + (unsigned long long)bytes + 15ull) & ~15ull;
-    constexpr unsigned long long CH = 4096;
-    for (unsigned long long a = a0 + (unsigned long long)tid * CH; a < a1; a += (unsigned long long)kPlaneThreads * CH) {
-        const unsigned sz = (unsigned)(a1 - a < CH ? a1 - a : CH);
-        HN_G((const void *)a, sz);
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(a), "r"(sz) : "memory");
+    const char *b = reinterpret_cast<const char *>(ptr);
+    for (long long o = (long long)tid * 128; o < bytes; o += (long long)kPlaneThreads * 128) {
+        HN_G(b + o, 1);
+        asm volatile("prefetch.global.L2 [%0];\n" ::"l"(b + o) : "memory");
     }
 }
 

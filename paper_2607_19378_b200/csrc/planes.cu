@@ -13,7 +13,8 @@
 //              decimation-in-frequency step applied to the taps as they are read), each
 //              half filling a column store of the size of a k*v plane's.  The tap rows are
 //              fetched once: the odd half's inputs wait in tensor memory meanwhile.
-//   plane_inv  inverse along y (keeping the cropped rows), inverse complex-to-real
+//   plane_inv  inverse along y (keeping the cropped rows; two rows combined into one
+//              complex row as they leave the registers), inverse complex-to-real
 //              along x, crop, output gate q, store.
 //
 // Column 0 of the column store carries the two purely real bins of every row (kx = 0 and
@@ -83,11 +84,6 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
     const int Lx = p.lx, Ly = p.ly;
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const long long ib = pl * (long long)Ly * Lx;
-        if (pl + gridDim.x < p.planes) {
-            const long long nb = (pl + gridDim.x) * (long long)Ly * Lx;
-            prefetch_l2(pk + nb, (long long)Ly * Lx * sizeof(T), tid);
-            prefetch_l2(pv + nb, (long long)Ly * Lx * sizeof(T), tid);
-        }
         // rows: y and y + P/4 share a transform (rows P/4 .. Ly-1 exist, Ly > P/4; a missing partner is a zero row)
         for (int rp = gid; rp < QP; rp += C::NG) {
             const int y1 = rp + QP;
@@ -154,6 +150,12 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
         // a lane's first-pass inputs y = j + r P/R, r < R/2 (the rest is padding), come from the row pairs of r < R/4,
         // both members each.  Values leave at twice their size (the factor 1/2 is left to the spectral core's scale).
         float2 *dst = p.out + pl * (long long)C::XH * P;
+        if (pl + gridDim.x < p.planes) {
+            // the next plane's rows travel to L2 during the column phase, which loads nothing from global memory
+            const long long nb = (pl + gridDim.x) * (long long)Ly * Lx;
+            prefetch_l2(pk + nb, (long long)Ly * Lx * sizeof(T), tid);
+            prefetch_l2(pv + nb, (long long)Ly * Lx * sizeof(T), tid);
+        }
         for (int kx = gid; kx < HP; kx += C::NG) {
             // Column 0 packs bins kx = 0 and kx = P/2 of every row as one complex number; it runs the same transform as
             // every other column (the group that shares its warp does not wait for a second code path), its raw transform
@@ -416,15 +418,15 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
 {
     using C = PlaneCfg<LOG2P>;
     using FI = typename C::FI;
-    constexpr int P = C::P, HP = C::HP, TPL = FI::TPL;
+    constexpr int P = C::P, HP = C::HP, QP = P / 4, TPL = FI::TPL, CSI = C::CSU;
     extern __shared__ float2 smem[];
     float2 *cs = smem;
     float2 *wbuf = cs + C::CSN;
     float2 *tw = wbuf + C::WBUF;
     float2 *twh = tw + P;
-    float2 *tmp = smem + C::TMP;
     const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
-    const unsigned m = FI::group_mask(tid);
+    constexpr unsigned m = 0xffffffffu;                      // every warp runs the loops below in step: whole-warp barriers
+    static_assert((HP % C::NG == 0 || C::NG % HP == 0) && (QP % C::NG == 0 || C::NG % QP == 0), "whole warps take part in both loops");
     float2 *line = wbuf + gid * C::LS;
     load_plane_twiddles<LOG2P>(tw, twh, p.gtw, p.gtw_n, tid);
     __syncthreads();
@@ -465,62 +467,87 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
                     pre[i][r] = make_float2(pre[i][r].x - gn.y, pre[i][r].y + gn.x);
                 }
         }
+        // Rows y and y + P/4 leave as one complex row transform (real part row y, imaginary part row y + P/4).  With A, B
+        // the values of column kx at the two rows, that transform's input is G[kx] = A + iB at bin kx and
+        // G[P - kx] = conj A + i conj B at the mirrored bin: the column transform forms both from its last pass's
+        // registers (legs r and r + R/4 of a lane are a row pair) and stores the whole line G of every row pair, so the
+        // row transform loads one value per point.  The packed column (kx = 0 with kx = P/2) stores the same two
+        // combinations at bins 0 and P/2; the row phase turns them into (A.x, B.x) and (A.y, B.y).
+        using P1 = typename FI::template Pass<1>;
         for (int kx = gid; kx < HP; kx += C::NG) {
-            float2 *col = cs + kx * C::CSS;
+            float2 *lo = cs + kx * CSI, *hi = cs + (kx == 0 ? HP : P - kx) * CSI;
             FI::template pass<0, PRUNE_NONE>(l, twp,
                 [&](int i, int r, int) { return pre[i][r]; },
                 [&](int, int, int idx, float2 v) { line[FI::ph(idx)] = v; });
             __syncwarp(m);
             if (kx + C::NG < HP) fetch(kx + C::NG);
+            float2 first[P1::IPL][P1::R / 4];
             FI::template pass<1, PRUNE_OUT>(l, twp,
                 [&](int, int, int idx) { return line[FI::ph(idx)]; },
-                [&](int, int, int idx, float2 v) { col[idx] = v; });
+                [&](int i, int r, int idx, float2 B) {
+                    if (r < P1::R / 4) { first[i][r] = B; return; }
+                    const float2 A = first[i][r - P1::R / 4];
+                    lo[idx - QP] = make_float2(A.x - B.y, A.y + B.x);
+                    hi[idx - QP] = make_float2(A.x + B.y, B.x - A.y);
+                });
             __syncwarp(m);
         }
-        __syncthreads();
+        // The gate values of all of this lane's outputs are requested before anything else of the row phase (before
+        // the barrier, and before the prefetch below, whose burst of requests would otherwise sit in front of them).
         const long long ob = pl * (long long)Ly * Lx;
-        if (pl + gridDim.x < p.planes) {
-            // while the rows are transformed, bring the next plane's spectra and gate into L2
-            prefetch_l2(p.in + (pl + gridDim.x) * (long long)C::XH * P, (long long)C::XH * P * sizeof(float2), tid);
-            prefetch_l2(pq + (pl + gridDim.x) * (long long)Ly * Lx, (long long)Ly * Lx * sizeof(T), tid);
-        }
-        for (int rp = gid; 2 * rp < Ly; rp += C::NG) {
-            const int y0 = 2 * rp, y1 = y0 + 1;
-            const bool has1 = y1 < Ly;
-            const long long o0 = ob + (long long)y0 * Lx, o1 = o0 + Lx;
-            // the gate values of this lane's outputs are requested before the transform starts
-            using PE = typename FI::LastPass;
-            constexpr int NQ = PE::IPL * (PE::R / 2);
-            T q0[NQ], q1[NQ];
+        using PE = typename FI::LastPass;
+        constexpr int NQ = PE::IPL * (PE::R / 2);
+        constexpr int RIT = QP > C::NG ? QP / C::NG : 1;      // row pairs per lane group
+        T q0[RIT][NQ], q1[RIT][NQ];
+#pragma unroll
+        for (int it = 0; it < RIT; ++it) {
+            const int rp = gid + it * C::NG, y1 = rp + QP;
+            const bool has0 = rp < QP, has1 = has0 && y1 < Ly;
+            const long long o0 = ob + (long long)rp * Lx, o1 = ob + (long long)y1 * Lx;
 #pragma unroll
             for (int i = 0; i < PE::IPL; ++i)
 #pragma unroll
                 for (int r = 0; r < PE::R / 2; ++r) {
                     const int idx = FI::last_pos(l, i, r);
-                    if (idx < Lx) HN_G(pq + o0 + idx, sizeof(T));
+                    if (idx < Lx && has0) HN_G(pq + o0 + idx, sizeof(T));
                     if (idx < Lx && has1) HN_G(pq + o1 + idx, sizeof(T));
-                    q0[i * (PE::R / 2) + r] = idx < Lx ? __ldg(pq + o0 + idx) : T(0.f);
-                    q1[i * (PE::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
+                    q0[it][i * (PE::R / 2) + r] = (idx < Lx && has0) ? __ldg(pq + o0 + idx) : T(0.f);
+                    q1[it][i * (PE::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
                 }
+        }
+        __syncthreads();
+        if (pl + gridDim.x < p.planes) {
+            // while the rows are transformed, bring the next plane's spectra and gate into L2
+            prefetch_l2(p.in + (pl + gridDim.x) * (long long)C::XH * P, (long long)C::XH * P * sizeof(float2), tid);
+            prefetch_l2(pq + (pl + gridDim.x) * (long long)Ly * Lx, (long long)Ly * Lx * sizeof(T), tid);
+        }
+#pragma unroll
+        for (int it = 0; it < RIT; ++it) {
+            const int rp = gid + it * C::NG;
+            if (rp >= QP) break;
+            const int y1 = rp + QP;
+            const bool has1 = y1 < Ly;
+            const long long o0 = ob + (long long)rp * Lx, o1 = ob + (long long)y1 * Lx;
+            static_assert(P0::IPL == 1, "lane 0 holds bins 0 and P/2 of a row");
+            const float2 *g = cs + l * CSI + rp;
+            float2 nyq = make_float2(0.f, 0.f);
             FI::template run<PRUNE_OUT>(l, m, twp, line,
-                [&](int, int, int idx) {
-                    // branch-free merge of two half spectra into one complex row (column 0 is packed)
-                    const bool mirror = idx > HP;
-                    const int kx = mirror ? P - idx : idx;
-                    const int col = kx == HP ? 0 : kx;
-                    const float2 A = cs[col * C::CSS + y0];
-                    float2 B = cs[col * C::CSS + y1];
-                    if (!has1) B = make_float2(0.f, 0.f);
-                    const float sg = mirror ? -1.f : 1.f;
-                    float2 g = make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
-                    g = kx == 0 ? make_float2(A.x, B.x) : g;
-                    g = kx == HP ? make_float2(A.y, B.y) : g;
-                    return g;
+                [&](int, int r, int) {
+                    float2 v = g[r * (P / P0::R) * CSI];
+                    if (r == 0 && l == 0) {
+                        // bins 0 and P/2 hold A + iB and conj A + i conj B of the packed column, A = (X_0[y], X_{P/2}[y]):
+                        // the row transform wants (A.x, B.x) at bin 0 and (A.y, B.y) at bin P/2
+                        const float2 w = g[HP * CSI];
+                        nyq = make_float2(0.5f * (v.y - w.y), 0.5f * (w.x - v.x));
+                        v = make_float2(0.5f * (v.x + w.x), 0.5f * (v.y + w.y));
+                    }
+                    if (r == P0::R / 2 && l == 0) v = nyq;
+                    return v;
                 },
                 [&](int i, int r, int idx, float2 v) {
                     if (idx < Lx) {
-                        IO<T>::st(py, o0 + idx, v.x * (float)q0[i * (PE::R / 2) + r]);
-                        if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[i * (PE::R / 2) + r]);
+                        IO<T>::st(py, o0 + idx, v.x * (float)q0[it][i * (PE::R / 2) + r]);
+                        if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[it][i * (PE::R / 2) + r]);
                     }
                 });
             __syncwarp(m);
