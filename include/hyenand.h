@@ -163,7 +163,10 @@ long long hyenand_debug_selftest(void);
 int hyenand_selftest_bounded_wait(int polls);
 
 /* Reporting helpers (host-only, no device work). */
-size_t hyenand_plan_workspace_bytes(const hyenand_plan *plan);        /* device bytes owned by the plan */
+size_t hyenand_plan_workspace_bytes(const hyenand_plan *plan);        /* device bytes owned by the plan: workspace, plus the
+                                                                       * staging copies once hyenand_forward_host has run, plus
+                                                                       * room for C filter spectra once a filter shared over the
+                                                                       * batch has been used (allocated by that first call) */
 int hyenand_plan_fft_dims(const hyenand_plan *plan, int *out_P);      /* writes ndim padded sizes P_n */
 int hyenand_plan_launches(const hyenand_plan *plan, int h_shared);    /* kernels enqueued by one forward */
 const char *hyenand_plan_path(const hyenand_plan *plan);              /* name of the kernel path chosen */

@@ -28,7 +28,8 @@ struct DbgReport {
 };
 typedef void (*DbgHook)(const DbgRanges *set, unsigned long long *collect);
 void dbg_register(DbgHook hook, const char *file);
-void dbg_set_ranges(const DbgRanges &r);           // uploads to every translation unit
+void dbg_set_ranges(const DbgRanges &r);
+void dbg_append_range(const void *ptr, size_t bytes);     // one more range for the call in progress           // uploads to every translation unit
 DbgReport dbg_collect();                           // sums and clears the counters of every translation unit
 }  // namespace hn
 

@@ -33,9 +33,21 @@ void dbg_register(DbgHook hook, const char *file)
     if (g_dbg_n < 32) { g_dbg_hooks[g_dbg_n] = hook; g_dbg_files[g_dbg_n] = file; ++g_dbg_n; }
 }
 
+static DbgRanges g_dbg_last;
+
 void dbg_set_ranges(const DbgRanges &r)
 {
+    g_dbg_last = r;
     for (int i = 0; i < g_dbg_n; ++i) g_dbg_hooks[i](&r, nullptr);
+}
+
+void dbg_append_range(const void *ptr, size_t bytes)
+{
+    if (!ptr || !bytes || g_dbg_last.n >= kDbgRanges) return;
+    g_dbg_last.lo[g_dbg_last.n] = (unsigned long long)ptr;
+    g_dbg_last.hi[g_dbg_last.n] = (unsigned long long)ptr + bytes;
+    ++g_dbg_last.n;
+    dbg_set_ranges(g_dbg_last);
 }
 
 DbgReport dbg_collect()

@@ -210,6 +210,7 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
 }
 
 static AxisArgs planes3d_core_args(const hyenand_plan *p, int lane, long long n, bool shared, long long s0);
+static void make_core_maps(hyenand_plan *p);
 static AxisArgs generic_core_args(const hyenand_plan *p, int lane, long long n, bool shared, long long s0);
 static void choose_groups(hyenand_plan *p, long long per_slice_elems);
 
@@ -331,7 +332,7 @@ extern "C" hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int
     int e = dev_alloc(p, (void **)&p->gtw, sizeof(float2) * p->gtw_n);
     for (int l = 0; l < p->n_lanes && !e; ++l) {
         hyenand_plan::Lane &ln = p->lane[l];
-        ln.wh_slices = (l == 0 && C > spc) ? C : spc;       // lane 0 has room for all channels when the filter is shared
+        ln.wh_slices = spc;                                 // (a filter shared over the batch gets room for all channels on first use)
         e = dev_alloc(p, (void **)&ln.ws_a, sizeof(float2) * p->ws_a_slice * spc);
         if (!e && p->ws_b_slice) e = dev_alloc(p, (void **)&ln.ws_b, sizeof(float2) * p->ws_b_slice * spc);
         if (!e) e = dev_alloc(p, (void **)&ln.wh_a, sizeof(float2) * p->wh_a_slice * ln.wh_slices);
@@ -350,21 +351,48 @@ extern "C" hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int
         if (!ok) e = fail(HYENAND_ERR_CUDA, "lane streams: %s", cudaGetErrorString(cudaGetLastError()));
     }
     if (e) { hyenand_destroy_plan(p); return nullptr; }
-    // tensor maps of the fused core's buffers; left invalid where the TMA core does not apply
-    if (p->path != PATH_FUSED2D && !p->sw.no_tma) {
-        for (int l = 0; l < p->n_lanes; ++l) {
-            hyenand_plan::Lane &ln = p->lane[l];
-            const AxisArgs own = p->path == PATH_PLANES3D ? planes3d_core_args(p, l, spc, false, 0)
-                                                          : generic_core_args(p, l, spc, false, 0);
-            core_tma_make(&ln.tma, own, spc, ln.wh_slices);
-            if (l > 0) {
-                const AxisArgs sh = p->path == PATH_PLANES3D ? planes3d_core_args(p, l, spc, true, 0)
-                                                             : generic_core_args(p, l, spc, true, 0);
-                core_tma_make(&ln.tma_sh, sh, spc, p->lane[0].wh_slices);
-            }
+    make_core_maps(p);
+    return p;
+}
+
+// tensor maps of the fused core's buffers; left invalid where the TMA core does not apply
+static void make_core_maps(hyenand_plan *p)
+{
+    if (p->path != PATH_PLANES3D && p->path != PATH_ND_GENERIC) return;
+    if (p->sw.no_tma) return;
+    const long long spc = p->slices_per_chunk;
+    for (int l = 0; l < p->n_lanes; ++l) {
+        hyenand_plan::Lane &ln = p->lane[l];
+        const AxisArgs own = p->path == PATH_PLANES3D ? planes3d_core_args(p, l, spc, false, 0)
+                                                      : generic_core_args(p, l, spc, false, 0);
+        core_tma_make(&ln.tma, own, spc, ln.wh_slices);
+        if (l > 0) {
+            const AxisArgs sh = p->path == PATH_PLANES3D ? planes3d_core_args(p, l, spc, true, 0)
+                                                         : generic_core_args(p, l, spc, true, 0);
+            core_tma_make(&ln.tma_sh, sh, spc, p->lane[0].wh_slices);
         }
     }
-    return p;
+}
+
+// A filter shared over the batch is transformed once per forward, all C channels into lane 0's filter workspace,
+// which therefore needs room for C slices instead of one group's: it is enlarged the first time such a forward is
+// asked for (plans used with per-sample filters never pay for it).
+static int ensure_shared_filter_room(hyenand_plan *p)
+{
+    hyenand_plan::Lane &ln = p->lane[0];
+    if (ln.wh_slices >= p->C) return 0;
+    float2 *a = nullptr, *b = nullptr;
+    int e = dev_alloc(p, (void **)&a, sizeof(float2) * p->wh_a_slice * p->C);
+    if (!e && p->wh_b_slice) e = dev_alloc(p, (void **)&b, sizeof(float2) * p->wh_b_slice * p->C);
+    if (e) return e;
+    ln.wh_a = a; ln.wh_b = b; ln.wh_slices = p->C;       // (the smaller buffers stay with the plan until it is destroyed)
+#ifdef HYENAND_DEBUG
+    cudaDeviceSynchronize();
+    dbg_append_range(a, sizeof(float2) * p->wh_a_slice * p->C);
+    if (b) dbg_append_range(b, sizeof(float2) * p->wh_b_slice * p->C);
+#endif
+    make_core_maps(p);
+    return 0;
 }
 
 // Group size and number of lanes.  HYENAND_GROUP_SLICES / HYENAND_LANES override the choice (development aids,
@@ -539,6 +567,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
 {
     const size_t es = elsize(p->dtype);
     const bool three = p->P[0] > 1;
+    if (shared && ensure_shared_filter_room(p)) return -2;
     if (shared && p->r0 == 0 && filter_spectrum_generic(p, 0, h, p->C, st0, launches)) return -1;
     if (lanes_fork(p, st0)) return -1;
     int g = 0;
@@ -641,6 +670,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         *launches += c;
         return 0;
     };
+    if (shared && ensure_shared_filter_room(p)) return -2;
     if (shared && p->r0 == 0 && filter(0, h, p->C, st0)) return -1;
     if (lanes_fork(p, st0)) return -1;
     int g = 0;
@@ -716,6 +746,7 @@ static int run_forward(hyenand_plan *p, const void *q, const void *k, const void
     else
         rc = forward_generic(p, (const char *)q, (const char *)k, (const char *)v, (const char *)h, shared,
                              (char *)y, st, launches);
+    if (rc == -2) return HYENAND_ERR_ALLOC;              // (message already recorded by the allocation)
     if (rc) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(HYENAND_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
