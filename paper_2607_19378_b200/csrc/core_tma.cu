@@ -2,7 +2,7 @@
 //
 // Same arithmetic as core_w.cu (forward transform of the filter lines, forward transform of the
 // k*v lines, spectral product of Eq. 12 of the paper, inverse, cropped half written back in
-// place), but the tiles -- 16 (8 for 1024-point lines) adjacent bins by all rows of the axis -- travel as tensor copies:
+// place), but the tiles -- 8 adjacent bins by all rows of the axis -- travel as tensor copies:
 //
 //   cp.async.bulk.tensor loads   filter tile (boxes of up to 256 rows; the wrapped placement of the
 //                                taps is two row ranges) and k*v tile (one box; rows past the data
@@ -10,8 +10,8 @@
 //   cp.async.bulk.tensor store   the cropped result tile
 //
 // One elected thread issues them; nobody computes addresses or waits per element.  The boxes land
-// row-major (one 64- or 128-byte row per axis position) with the matching swizzle, which spreads the rows a group of
-// lanes reads at once over 8 bank groups.  A tile buffer is free again as soon as the first pass
+// row-major (one 64-byte row per axis position; the code also covers 128-byte rows) with the matching swizzle, which
+// spreads the rows a group of lanes reads at once over the banks.  A tile buffer is free again as soon as the first pass
 // has read it, so the next tile's copy runs under the rest of this tile's arithmetic.
 //
 // Every wait on a copy is bounded: if a barrier does not complete, the CTA records it in the
@@ -25,15 +25,22 @@
 
 namespace hn {
 
-constexpr int kTmaThreads = 256;
+// Threads per CTA: 256-point lines run as 4 CTAs of 128 threads per SM (8 lines per tile), 1024-point lines as one
+// CTA of 256 threads (8 lines per tile).  A CTA synchronises at two barriers per tile; more, smaller CTAs per SM
+// keep the schedulers busy while one of them waits.
+template <int LOG2P> struct TmaCta {
+    static constexpr int THREADS = LOG2P >= 10 ? 256 : 128;
+    static constexpr int PER_SM = LOG2P >= 10 ? 1 : 4;
+};
 
-// Geometry of a tile for LOG2P-point lines: one line per group of TPL lanes, so TX = 256 / TPL bins
-// per tile and TX * 8 bytes per tile row (128 for 256-point lines, 64 for 1024-point lines: the
-// swizzle span of the tensor maps).  A box holds at most 256 rows.
+// Geometry of a tile for LOG2P-point lines: one line per group of TPL lanes, so TX = THREADS / TPL bins
+// per tile and TX * 8 bytes per tile row (64 here: the swizzle span of the tensor maps).  A box holds at
+// most 256 rows.
 template <int LOG2P> struct TmaGeo {
     using F = WF<LOG2P, false>;
     static constexpr int N = 1 << LOG2P, HALF = N / 2;
-    static constexpr int TX = kTmaThreads / F::TPL;
+    static constexpr int THREADS = TmaCta<LOG2P>::THREADS;
+    static constexpr int TX = THREADS / F::TPL;
     static constexpr unsigned ROWB = TX * 8;
     static constexpr int BOXR = HALF < 256 ? HALF : 256;             // rows per box
     static constexpr int NB = HALF / BOXR;                           // boxes per half line
@@ -41,7 +48,7 @@ template <int LOG2P> struct TmaGeo {
     static constexpr unsigned HALFB = HALF * ROWB;
     // 16-lane groups (two lines per warp): the lanes of a half warp belong to both lines (see the kernel), whose
     // strides are therefore 8 mod 16 entries, i.e. half a bank row apart
-    static constexpr int LS = TX >= 16 ? plane_ls(N) : ((F::ph(N - 1) + 1 + 15) / 16 * 16 + 2);
+    static constexpr int LS = F::TPL == 16 ? plane_ls(N) : ((F::ph(N - 1) + 1 + 15) / 16 * 16 + 2);
     static_assert(ROWB == 128 || ROWB == 64, "tile rows match a swizzle span");
     // shared memory: tile buffers first (1024-byte aligned, as the swizzle pattern repeats every 1024 bytes)
     static constexpr size_t TH = 0;                                  // filter tile, N rows
@@ -55,7 +62,7 @@ template <int LOG2P> struct TmaGeo {
 
 struct CoreTmaParams {
     long long n_outer;
-    int tiles_per_outer;      // ceil(nc / 16)
+    int tiles_per_outer;      // ceil(nc / TX)
     int h_shift;              // filter row (pos + h_shift) mod N sits at position pos
     long long h_mod, h_off;   // filter outer index = h_mod ? (o + h_off) % h_mod : o
     float scale;
@@ -65,13 +72,13 @@ struct CoreTmaParams {
 };
 
 template <int LOG2P>
-__global__ void __launch_bounds__(kTmaThreads, (LOG2P >= 10 ? 1 : 2))
+__global__ void __launch_bounds__(TmaCta<LOG2P>::THREADS, TmaCta<LOG2P>::PER_SM)
 axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_constant__ CUtensorMap map_h, CoreTmaParams p)
 {
     using G = TmaGeo<LOG2P>;
     using F = WF<LOG2P, false>;
     using FI = WF<LOG2P, true>;
-    constexpr int N = G::N, TPL = F::TPL, NP = F::NP;
+    constexpr int N = G::N, TPL = F::TPL, NP = F::NP, kTmaThreads = G::THREADS;
     static_assert(NP == 2 && F::radix(0) == F::radix(1), "two equal passes: one register set of twiddles serves both directions");
     using PL = typename F::template Pass<NP - 1>;
     using P0 = typename F::template Pass<0>;
@@ -268,10 +275,10 @@ template <int LOG2P> static int launch_core_tma_t(const CoreTmaParams &p0, const
     if (attr.first())
         cudaFuncSetAttribute(axis_core_tma_kernel<LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::TOTAL);
     const long long tiles = p.n_outer * p.tiles_per_outer;
-    const long long res = (long long)sms * (LOG2P >= 10 ? 1 : 2);    // resident CTAs
+    const long long res = (long long)sms * TmaCta<LOG2P>::PER_SM;    // resident CTAs
     const int grid = (int)(tiles < res ? tiles : res);
     if (grid <= 0) return 0;
-    axis_core_tma_kernel<LOG2P><<<grid, kTmaThreads, G::TOTAL, st>>>(
+    axis_core_tma_kernel<LOG2P><<<grid, G::THREADS, G::TOTAL, st>>>(
         *reinterpret_cast<const CUtensorMap *>(m.u), *reinterpret_cast<const CUtensorMap *>(m.h), p);
     return 1;
 }
