@@ -158,6 +158,7 @@ struct hyenand_plan {
     // host-staging for hyenand_forward_host
     void *stage[5];
     size_t stage_bytes[5];
+    int h_dtype;                      // element type of the filter taps (differs from dtype only inside the mixer)
     size_t ws_bytes;
     Prof prof;
 };
@@ -245,7 +246,7 @@ extern "C" hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int
 
     hyenand_plan *p = new hyenand_plan();
     memset(p, 0, sizeof(*p));
-    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->circular = circular; p->dtype = dtype;
+    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->circular = circular; p->dtype = dtype; p->h_dtype = dtype;
     p->r0 = 0; p->r1 = (long long)B * C;
     cudaGetDevice(&p->device);
     p->sw = read_switches();
@@ -372,6 +373,17 @@ static void make_core_maps(hyenand_plan *p)
             core_tma_make(&ln.tma_sh, sh, spc, p->lane[0].wh_slices);
         }
     }
+}
+
+// The multi-kernel paths transform the filter in kernels of their own, which take the taps' element type per launch:
+// a plan of fp32 tensors can read bf16 taps there (the mixer's inner plan: q, k, v come out of its fp32 pointwise
+// stage, the kernel arrives in the caller's type).  False where the path has one element type for everything.
+static bool plan_set_filter_dtype(hyenand_plan *p, int dtype)
+{
+    if (dtype == p->dtype) { p->h_dtype = dtype; return true; }
+    if (p->path != PATH_PLANES3D && p->path != PATH_ND_GENERIC) return false;
+    p->h_dtype = dtype;
+    return true;
 }
 
 // A filter shared over the batch is transformed once per forward, all C channels into lane 0's filter workspace,
@@ -502,7 +514,7 @@ static int filter_spectrum_generic(hyenand_plan *p, int l, const char *h, long l
     r.gtw = p->gtw; r.gtw_n = p->gtw_n;
     p->prof.begin(KID_ROWS_H, st);
     const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
-    int n = roww ? launch_rows_fwd_w(r, p->dtype, st) : launch_rows_fwd(r, p->dtype, st);
+    int n = roww ? launch_rows_fwd_w(r, p->h_dtype, st) : launch_rows_fwd(r, p->h_dtype, st);
     p->prof.end(st);
     if (n < 0) return -1;
     *launches += n;
@@ -576,7 +588,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         hyenand_plan::Lane &ln = p->lane[l];
         cudaStream_t st = lane_stream(p, l, st0);
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
-        if (!shared && filter_spectrum_generic(p, l, h + (size_t)s0 * p->kvol * es, n, st, launches)) return -1;
+        if (!shared && filter_spectrum_generic(p, l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st, launches)) return -1;
         RowsArgs r{};
         r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = ln.ws_a; r.pitch = p->XP;
         r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
@@ -664,7 +676,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         a.a_elems = n * p->kvol;
         a.lx = p->L[2]; a.ly = p->L[1]; a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         p->prof.begin(KID_PLANE_H, st);
-        int c = launch_plane(a, PLANE_H, p->log2p[2], p->dtype, st);
+        int c = launch_plane(a, PLANE_H, p->log2p[2], p->h_dtype, st);
         p->prof.end(st);
         if (c < 0) return -1;
         *launches += c;
@@ -679,7 +691,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         hyenand_plan::Lane &ln = p->lane[l];
         cudaStream_t st = lane_stream(p, l, st0);
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
-        if (!shared && filter(l, h + (size_t)s0 * p->kvol * es, n, st)) return -1;
+        if (!shared && filter(l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st)) return -1;
         PlaneArgs u{};
         u.a = k + (size_t)s0 * p->vol * es; u.b = v + (size_t)s0 * p->vol * es; u.out = ln.ws_a;
         u.a_elems = n * p->vol;
@@ -1095,7 +1107,8 @@ struct hyenand_mixer {
     int B, C, dtype, nb;              // nb: batch entries per pass
     long long L, kvol;
     float eps;
-    float *qz, *kz, *vz, *oz, *h32;   // scratch, fp32 (h32 only for bf16 I/O)
+    float *qz, *kz, *vz, *oz, *h32;   // scratch, fp32 (h32: widened bf16 taps, only where the inner plan cannot read them itself)
+    bool h_native;                    // the inner plan reads the taps in the caller's element type
     GuardedAllocs allocs;
     int device;
 };
@@ -1134,12 +1147,13 @@ extern "C" hyenand_mixer *hyenand_mixer_create(int ndim, const int *dims, int B,
     memset(m, 0, sizeof(*m));
     m->plan = plan; m->B = B; m->C = C; m->dtype = dtype; m->nb = (int)nb; m->L = L; m->kvol = plan->kvol; m->eps = eps;
     m->device = plan->device;
+    m->h_native = plan_set_filter_dtype(plan, dtype);      // else bf16 taps are widened into h32 first
     const size_t n = (size_t)nb * C * L * sizeof(float);
     cudaError_t e = guarded_alloc(&m->allocs, (void **)&m->qz, n);
     if (e == cudaSuccess) e = guarded_alloc(&m->allocs, (void **)&m->kz, n);
     if (e == cudaSuccess) e = guarded_alloc(&m->allocs, (void **)&m->vz, n);
     if (e == cudaSuccess) e = guarded_alloc(&m->allocs, (void **)&m->oz, n);
-    if (e == cudaSuccess && dtype == HYENAND_BF16)
+    if (e == cudaSuccess && dtype == HYENAND_BF16 && !m->h_native)
         e = guarded_alloc(&m->allocs, (void **)&m->h32, (size_t)nb * C * m->kvol * sizeof(float));
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -1188,8 +1202,9 @@ extern "C" int hyenand_mixer_forward(hyenand_mixer *m, const void *q, const void
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const size_t slab = (size_t)m->C * m->L;                        // elements per batch entry
+    const bool widen_h = m->dtype == HYENAND_BF16 && !m->h_native;
     const float *hf = (const float *)h;
-    if (m->dtype == HYENAND_BF16 && shared) {
+    if (widen_h && shared) {
         launch_widen(h, m->dtype, (long long)m->C * m->kvol, m->h32, st);
         hf = m->h32;
     }
@@ -1200,11 +1215,11 @@ extern "C" int hyenand_mixer_forward(hyenand_mixer *m, const void *q, const void
         launch_mixer_pre(qb, kb, vb, g_in, m->eps, m->dtype, n, m->C, m->L, m->qz, m->kz, m->vz, st);
         const float *hb = hf;
         if (!shared) {
-            if (m->dtype == HYENAND_BF16) {
+            if (widen_h) {
                 launch_widen((const char *)h + (size_t)b0 * m->C * m->kvol * es, m->dtype, (long long)n * m->C * m->kvol, m->h32, st);
                 hb = m->h32;
             } else {
-                hb = (const float *)h + (size_t)b0 * m->C * m->kvol;
+                hb = (const float *)((const char *)h + (size_t)b0 * m->C * m->kvol * es);      // taps in the caller's type
             }
         }
         int launches = 0;
