@@ -206,14 +206,14 @@ struct RowsArgs {
 struct RowsInvArgs {
     const float2 *in;     // [rows][pitch]
     int pitch;
-    const void *q;        // [rows][len]
+    const void *q;        // [rows][len]; nullptr: no gate
     void *y;              // [rows][len]
     long long rows;
     int len;              // L3
     int log2p;
     const float2 *gtw;
     int gtw_n;
-    int full_out;         // 1: circular mode, all P outputs of a row are kept (len == P)
+    int full_out;         // 1: no output half is cropped away, the first len <= P outputs of a row are kept (circular mode: len == P)
 };
 
 // A family of strided lines: line (o, c), element a at base[o*outer + a*nc + c].

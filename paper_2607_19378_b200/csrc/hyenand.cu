@@ -1266,10 +1266,10 @@ struct hyenand_grad {
     long long vol, kvol, pvol, kopp;  // elements per slice: grid, taps, padded ring, taps of the opposite kernel
     bool long1d;
     int nb;                           // batch entries per pass
-    long long ns;                     // slices per pass of the dh correlation (ring path)
-    hyenand_plan *main, *adj, *ring, *caus;
+    long long ns;                     // slices per pass of the dh correlation (0: not on that path)
+    hyenand_plan *main, *adj, *caus;
     float *q32, *k32, *v32, *dy32, *ones, *t32, *h32, *hopp;      // per pass of nb entries
-    float *rk, *rv, *rh, *rones, *rt;                            // ring path, ns slices each
+    float2 *cga, *cgb, *cua, *cub, *cwc, *cwd;                   // dh correlation: spectra of ns slices (see corr_dh)
     float *aux;                       // nb*C slices: reversed signals of the long 1-D path
     float *dhs;                       // nb*C slices of taps: per-slice kernel gradients before the sum over the batch
     float *dh32;                      // accumulated kernel gradient (shared kernel: [C][kvol]; else [nb*C][kvol])
@@ -1284,11 +1284,116 @@ extern "C" void hyenand_backward_destroy(hyenand_grad *g)
     if (cur != g->device) cudaSetDevice(g->device);
     if (g->adj && g->adj != g->main) hyenand_destroy_plan(g->adj);
     if (g->caus && g->caus != g->main) hyenand_destroy_plan(g->caus);
-    hyenand_destroy_plan(g->ring);
     hyenand_destroy_plan(g->main);
     guarded_free_all(&g->allocs);
     if (cur != g->device) cudaSetDevice(cur);
     delete g;
+}
+
+// ---- dh as a correlation on the general N-D kernels --------------------------------------------------------------
+// dh[d + L-1] = sum_t g[t] u[t - d] with g = dy q and u = k v is the full linear convolution of g with u reversed
+// along every axis: both operands have L points per axis (the zero half of their padded lines is pruned from the
+// forward transforms, like the k*v side of a forward), all 2L-1 outputs per axis are kept.  The stages are those of
+// the general path -- rows, [middle axis in 3-D], fused core along the last transformed axis, [middle axis back],
+// rows back -- on spectra of this handle's own (nothing padded is ever materialised; the first version ran a
+// circular convolution over padded copies of all three tensors, 55 of the 71 ms of a volume3d backward).
+struct CorrGeo {
+    long long rows_in;      // [L0][L1][XP]   row spectra of an operand
+    long long mid;          // [L0][P1][XP]   after the middle axis (3-D only)
+    long long core_out;     // [K0][P1][XP]   (3-D) or [K1][XP] (1-D, 2-D): after the core
+    long long inv_out;      // [K0][K1][XP]   (3-D only): after the middle axis back
+};
+
+static CorrGeo corr_geo(const hyenand_grad *g)
+{
+    const hyenand_plan *p = g->main;
+    const long long XP = p->XP;
+    const long long K0 = 2ll * g->L[0] - 1, K1 = 2ll * g->L[1] - 1;
+    const bool three = g->P[0] > 1;
+    CorrGeo c{};
+    c.rows_in = (long long)g->L[0] * g->L[1] * XP;
+    c.mid = three ? (long long)g->L[0] * g->P[1] * XP : 0;
+    c.core_out = three ? K0 * g->P[1] * XP : K1 * XP;
+    c.inv_out = three ? K0 * K1 * XP : 0;
+    return c;
+}
+
+static long long corr_slice_elems(const hyenand_grad *g)
+{
+    const CorrGeo c = corr_geo(g);
+    return 2 * c.rows_in + 2 * c.mid + c.core_out + c.inv_out;
+}
+
+// m slices: gy, gq (their product is g), ur (u reversed) -> out [m][2L0-1][2L1-1][2L2-1]
+static int corr_dh(hyenand_grad *g, long long m, const float *gy, const float *gq, const float *ur, float *out, cudaStream_t st)
+{
+    hyenand_plan *p = g->main;                          // geometry, twiddles, switches
+    const int *L = g->L, *P = g->P;
+    const int K0 = 2 * L[0] - 1, K1 = 2 * L[1] - 1, K2 = 2 * L[2] - 1;
+    const bool three = P[0] > 1;
+    const int XP = p->XP;
+    int c = 0;
+    auto rows = [&](const float *a, const float *b, float2 *dst) {
+        RowsArgs r{};
+        r.a = a; r.b = b; r.out = dst; r.pitch = XP;
+        r.rows = m * L[0] * L[1]; r.len = L[2]; r.shift = 0; r.log2p = p->log2p[2];
+        r.prune_in = p->P[2] >= 2; r.full_in = 0; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
+        const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
+        return roww ? launch_rows_fwd_w(r, HYENAND_F32, st) : launch_rows_fwd(r, HYENAND_F32, st);
+    };
+    auto middle = [&](const float2 *src, float2 *dst) {
+        AxisArgs a{};
+        a.in = src; a.out = dst;
+        a.n_outer = m * L[0];
+        a.in_outer = (long long)L[1] * XP; a.out_outer = (long long)P[1] * XP;
+        a.nc = XP; a.n_in = L[1]; a.n_out = P[1]; a.shift = 0;
+        a.log2p = p->log2p[1]; a.prune_in = P[1] >= 2;
+        a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        return launch_axis(a, AXIS_FWD, st);
+    };
+    if ((c = rows(gy, gq, g->cga)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    if ((c = rows(ur, nullptr, g->cua)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    if (three) {
+        if ((c = middle(g->cga, g->cgb)) < 0 || (c = middle(g->cua, g->cub)) < 0)
+            return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    }
+    {
+        const int ax = three ? 0 : 1;                   // core axis
+        const int Kax = three ? K0 : K1;
+        const long long inner = three ? (long long)P[1] * XP : XP;
+        AxisArgs a{};
+        a.in = three ? g->cgb : g->cga; a.out = g->cwc;
+        a.n_outer = m;
+        a.in_outer = (long long)L[ax] * inner; a.out_outer = (long long)Kax * inner;
+        a.nc = (int)inner; a.n_in = L[ax]; a.n_out = Kax; a.shift = 0;
+        a.log2p = p->log2p[ax]; a.prune_in = 0; a.full = 1;
+        a.h = three ? g->cub : g->cua; a.h_outer = (long long)L[ax] * inner; a.h_n_in = L[ax]; a.h_shift = 0;
+        a.h_mod = 0; a.h_off = 0;
+        a.scale = (float)(1.0 / ((double)P[0] * P[1] * P[2]));
+        a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        c = (core_w_supported(a.log2p) && !p->sw.generic_core) ? launch_core_w(a, st) : launch_axis(a, AXIS_CORE, st);
+        if (c < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    }
+    if (three) {
+        AxisArgs a{};
+        a.in = g->cwc; a.out = g->cwd;
+        a.n_outer = m * K0;
+        a.in_outer = (long long)P[1] * XP; a.out_outer = (long long)K1 * XP;
+        a.nc = XP; a.n_in = P[1]; a.n_out = K1; a.shift = 0;
+        a.log2p = p->log2p[1]; a.prune_in = 0; a.full = 1;
+        a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+        if ((c = launch_axis(a, AXIS_INV, st)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    }
+    {
+        RowsInvArgs ri{};
+        ri.in = three ? g->cwd : g->cwc; ri.pitch = XP; ri.q = nullptr; ri.y = out;
+        ri.rows = m * K0 * K1; ri.len = K2; ri.log2p = p->log2p[2];
+        ri.gtw = p->gtw; ri.gtw_n = p->gtw_n; ri.full_out = 1;
+        const bool roww = rows_w_supported(ri.log2p) && !p->sw.generic_rows;
+        c = roww ? launch_rows_inv_w(ri, HYENAND_F32, st) : launch_rows_inv(ri, HYENAND_F32, st);
+        if (c < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    }
+    return HYENAND_OK;
 }
 
 extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int B, int C, int mode, int dtype)
@@ -1304,7 +1409,6 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     g->ndim = ndim; g->B = B; g->C = C; g->mode = mode; g->dtype = dtype;
     g->vol = g->kvol = g->pvol = 1;
     for (int a = 0; a < 3; ++a) { g->L[a] = g->K[a] = g->P[a] = 1; }
-    int pdims[3] = {1, 1, 1};
     bool ring_ok = true;
     for (int a = 0; a < ndim; ++a) {
         const int ia = 3 - ndim + a;
@@ -1312,7 +1416,6 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
         g->L[ia] = dims[a];
         g->K[ia] = mode == HYENAND_MODE_LINEAR ? 2 * dims[a] - 1 : dims[a];
         g->P[ia] = mode == HYENAND_MODE_CIRCULAR ? dims[a] : 1 << next_pow2_log(2 * dims[a] - 1);
-        pdims[a] = g->P[ia];
         if (g->P[ia] > (1 << kMaxLineLog2)) ring_ok = false;
         g->vol *= dims[a]; g->kvol *= g->K[ia]; g->pvol *= g->P[ia];
     }
@@ -1343,14 +1446,12 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
             if (!g->caus) { hyenand_backward_destroy(g); return nullptr; }
         }
     } else if (mode != HYENAND_MODE_CIRCULAR) {
-        // ring path: five fp32 tensors of ns*pvol elements within about 2 GiB
-        long long ns = (2ll << 30) / (20ll * g->pvol);
+        // dh correlation: the spectra of ns slices within about 2 GiB
+        long long ns = (2ll << 30) / (8ll * corr_slice_elems(g));
         if (const char *e = getenv("HYENAND_BACKWARD_RING_SLICES")) { const long long v = atoll(e); if (v > 0 && v < ns) ns = v; }   // development aid
         if (ns < 1) ns = 1;
         if (ns > S) ns = S;
         g->ns = ns;
-        g->ring = hyenand_create_plan_mode(ndim, pdims, 1, (int)ns, HYENAND_MODE_CIRCULAR, HYENAND_F32);
-        if (!g->ring) { hyenand_backward_destroy(g); return nullptr; }
     }
     const bool widen = dtype == HYENAND_BF16;
     cudaError_t e = cudaSuccess;
@@ -1360,8 +1461,12 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     if (widen) { get(&g->q32, S * g->vol); get(&g->k32, S * g->vol); get(&g->v32, S * g->vol); get(&g->dy32, S * g->vol); get(&g->h32, S * g->kvol); }
     get(&g->ones, S * g->vol); get(&g->t32, S * g->vol); get(&g->hopp, S * g->kopp);
     get(&g->aux, S * g->vol); get(&g->dhs, S * g->kvol); get(&g->dh32, S * g->kvol);
-    if (g->ring) { get(&g->rk, g->ns * g->pvol); get(&g->rv, g->ns * g->pvol); get(&g->rh, g->ns * g->pvol);
-                   get(&g->rones, g->ns * g->pvol); get(&g->rt, g->ns * g->pvol); }
+    if (g->ns) {
+        const CorrGeo c = corr_geo(g);
+        auto get2 = [&](float2 **ptr, long long elems) { if (elems) get((float **)ptr, 2 * elems * g->ns); };
+        get2(&g->cga, c.rows_in); get2(&g->cua, c.rows_in); get2(&g->cgb, c.mid); get2(&g->cub, c.mid);
+        get2(&g->cwc, c.core_out); get2(&g->cwd, c.inv_out);
+    }
     if (e != cudaSuccess) {
         cudaGetLastError();
         fail(HYENAND_ERR_ALLOC, "scratch of the backward pass: %s", cudaGetErrorString(e));
@@ -1370,7 +1475,6 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     }
     { DbgScope d; d.add(g->allocs); d.commit(); }
     launch_fill(g->ones, 1.f, S * g->vol, 0);
-    if (g->ring) launch_fill(g->rones, 1.f, g->ns * g->pvol, 0);
     if (cudaDeviceSynchronize() != cudaSuccess) {
         fail(HYENAND_ERR_CUDA, "filling the constant tensors failed: %s", cudaGetErrorString(cudaGetLastError()));
         hyenand_backward_destroy(g);
@@ -1415,7 +1519,6 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
         d.add(h, hbytes); d.add(dh, hbytes);
         d.add(g->allocs); d.add(g->main->allocs);
         if (g->adj != g->main) d.add(g->adj->allocs);
-        if (g->ring) d.add(g->ring->allocs);
         if (g->caus && g->caus != g->main) d.add(g->caus->allocs);
         d.commit();
     }
@@ -1507,26 +1610,23 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             }
             if (shared) launch_batch_sum(dhS, n, C, kvol, b0 == 0, g->dh32, st);
         } else {
-            // ring path, ns slices at a time
+            // dh[m] = sum_t g_t u_{t - d}, m = d + L-1: the full linear convolution of g = dy q with the reversed u = k v,
+            // ns slices at a time
+            {
+                RemapArgs r{};
+                r.a = k32; r.b = v32; r.out = g->aux; r.slices = S;
+                for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = REMAP_REV; }
+                launch_remap(r, st);
+            }
+            float *full = g->mode == HYENAND_MODE_CAUSAL ? g->hopp : dhS;     // all 2L-1 taps per slice
             for (long long s0 = 0; s0 < S; s0 += g->ns) {
                 const long long m = S - s0 < g->ns ? S - s0 : g->ns;
-                RemapArgs pad{};
-                pad.slices = m;
-                for (int a = 0; a < 3; ++a) { pad.Ls[a] = L[a]; pad.G[a] = P[a]; pad.mode[a] = REMAP_PAD; }
-                pad.a = dy32 + s0 * vol; pad.out = g->rk; launch_remap(pad, st);
-                pad.a = q32 + s0 * vol; pad.out = g->rv; launch_remap(pad, st);
-                RemapArgs opp = pad;
-                for (int a = 0; a < 3; ++a) opp.mode[a] = REMAP_NEG;
-                opp.a = k32 + s0 * vol; opp.b = v32 + s0 * vol; opp.out = g->rh; launch_remap(opp, st);
-                if ((e = grad_forward(g->ring, m, g->rones, g->rk, g->rv, g->rh, false, g->rt, st))) return e;
-                RemapArgs tap{};
-                tap.a = g->rt; tap.out = dhS + s0 * kvol; tap.slices = m;
-                for (int a = 0; a < 3; ++a) {
-                    tap.Ls[a] = P[a]; tap.G[a] = K[a]; tap.mode[a] = REMAP_WRAP;
-                    tap.shift[a] = g->mode == HYENAND_MODE_LINEAR ? L[a] - 1 : 0;      // tap m is displacement m - (L-1), or m when causal
-                }
-                launch_remap(tap, st);
+                if ((e = corr_dh(g, m, dy32 + s0 * vol, q32 + s0 * vol, g->aux + s0 * vol, full + s0 * g->kopp, st))) return e;
             }
+            if (g->mode == HYENAND_MODE_CAUSAL &&
+                cudaMemcpy2DAsync(dhS, (size_t)kvol * sizeof(float), g->hopp + (L[2] - 1), (size_t)g->kopp * sizeof(float),
+                                  (size_t)kvol * sizeof(float), (size_t)S, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return fail(HYENAND_ERR_CUDA, "copy of the causal taps failed: %s", cudaGetErrorString(cudaGetLastError()));
             if (shared) launch_batch_sum(dhS, n, C, kvol, b0 == 0, g->dh32, st);
         }
         if (!shared) launch_mul_cast(g->dh32, nullptr, S * kvol, g->dtype, (char *)dh + (long long)b0 * C * kvol * es, st);
@@ -1542,7 +1642,7 @@ extern "C" long long hyenand_backward_guard_damage(hyenand_grad *g)
     g_err[0] = 0;
     if (!g) { fail(HYENAND_ERR_INVALID_ARG, "handle is NULL"); return -1; }
     long long bad = guard_damage(&g->allocs);
-    hyenand_plan *plans[4] = {g->main, g->adj != g->main ? g->adj : nullptr, g->ring, (g->caus && g->caus != g->main) ? g->caus : nullptr};
+    hyenand_plan *plans[4] = {g->main, g->adj != g->main ? g->adj : nullptr, nullptr, (g->caus && g->caus != g->main) ? g->caus : nullptr};
     for (int i = 0; i < 4 && bad >= 0; ++i)
         if (plans[i]) { const long long b = guard_damage(&plans[i]->allocs); bad = b < 0 ? -1 : bad + b; }
     return bad;

@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
             cp_async16(line + 2 * c, i0 + 2 * c);
             if (has1) cp_async16(line + RS + 2 * c, i1 + 2 * c);
         }
-        if (!FULL && p.len == HP && has1 && l == 0) {
+        if (!FULL && p.len == HP && has1 && l == 0 && pq) {
             // the two gate rows of the pair (contiguous, a multiple of 16 bytes from a 16-byte boundary)
             const unsigned long long qa = (unsigned long long)(pq + r0 * HP);
             HN_G((const void *)qa, 2 * HP * sizeof(T));
@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
             const float sg = (r == RH && idx == HP) ? 1.f : -1.f;
             return make_float2(fmaf(-sg, B.y, A.x), fmaf(sg, A.y, B.x));
         });
-        if (!FULL && p.len == HP && has1) {
+        if (!FULL && p.len == HP && has1 && pq) {
             // full rows: all gate loads of the pair are in flight together (they were asked into L2 above)
             float qa[HP / TPL], qb[HP / TPL];
 #pragma unroll
@@ -213,8 +213,9 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
         } else {
             for (int n = l; n < p.len; n += TPL) {
                 const float2 z = line[FI::ph(n)];
-                IO<T>::st(py, r0 * p.len + n, z.x * IO<T>::ld(pq, r0 * p.len + n));
-                if (has1) IO<T>::st(py, r1 * p.len + n, z.y * IO<T>::ld(pq, r1 * p.len + n));
+                // (no gate tensor: the rows leave as they are)
+                IO<T>::st(py, r0 * p.len + n, pq ? z.x * IO<T>::ld(pq, r0 * p.len + n) : z.x);
+                if (has1) IO<T>::st(py, r1 * p.len + n, pq ? z.y * IO<T>::ld(pq, r1 * p.len + n) : z.y);
             }
         }
         __syncwarp(m);
