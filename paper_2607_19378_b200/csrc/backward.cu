@@ -48,13 +48,24 @@ __global__ void __launch_bounds__(kBwdThreads) remap_kernel(RemapArgs r)
         float val = 0.f;
         if (j0 >= 0 && j0 < r.Ls[0] && j1 >= 0 && j1 < r.Ls[1] && j2 >= 0 && j2 < r.Ls[2]) {
             const long long src = s * svol + ((long long)j0 * r.Ls[1] + j1) * r.Ls[2] + j2;
-            HN_G(r.a + src, 4);
-            if (r.b) HN_G(r.b + src, 4);
-            val = __ldg(r.a + src);
-            if (r.b) val *= __ldg(r.b + src);
+            if (r.a_bf16) {
+                const bf16 *ab = reinterpret_cast<const bf16 *>(r.a);
+                HN_G(ab + src, 2);
+                val = __bfloat162float(ab[src]);
+            } else {
+                HN_G(r.a + src, 4);
+                val = __ldg(r.a + src);
+            }
+            if (r.b) { HN_G(r.b + src, 4); val *= __ldg(r.b + src); }
         }
-        HN_G(r.out + e, 4);
-        r.out[e] = val;
+        if (r.out_bf16) {
+            bf16 *ob = reinterpret_cast<bf16 *>(r.out);
+            HN_G(ob + e, 2);
+            ob[e] = __float2bfloat16_rn(val);
+        } else {
+            HN_G(r.out + e, 4);
+            r.out[e] = val;
+        }
     }
 }
 

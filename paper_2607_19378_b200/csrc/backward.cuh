@@ -17,6 +17,7 @@ struct RemapArgs {
     float *out;               // [slices][G0][G1][G2]
     long long slices;
     int G[3], Ls[3], mode[3], shift[3];
+    int a_bf16, out_bf16;     // a (with b == NULL) and/or out hold bf16 instead of fp32 (a re-indexed copy of bf16 taps is exact)
 };
 
 // out[s][i] = a[s][j(i)] * (b ? b[s][j(i)] : 1), zero where an axis index falls outside the source

@@ -1265,6 +1265,7 @@ struct hyenand_grad {
     int L[3], K[3], P[3];             // internal 3-axis form
     long long vol, kvol, pvol, kopp;  // elements per slice: grid, taps, padded ring, taps of the opposite kernel
     bool long1d;
+    bool h_native;                    // bf16 I/O: the forwards for dq and du read bf16 taps themselves (no widened kernel)
     int nb;                           // batch entries per pass
     long long ns;                     // slices per pass of the dh correlation (0: not on that path)
     hyenand_plan *main, *adj, *caus;
@@ -1454,11 +1455,13 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
         g->ns = ns;
     }
     const bool widen = dtype == HYENAND_BF16;
+    auto reads_bf16 = [](const hyenand_plan *q) { return q->path == PATH_PLANES3D || q->path == PATH_ND_GENERIC; };
+    g->h_native = widen && reads_bf16(g->main) && reads_bf16(g->adj);
     cudaError_t e = cudaSuccess;
     auto get = [&](float **ptr, long long elems) {
         if (e == cudaSuccess) e = guarded_alloc(&g->allocs, (void **)ptr, (size_t)elems * sizeof(float));
     };
-    if (widen) { get(&g->q32, S * g->vol); get(&g->k32, S * g->vol); get(&g->v32, S * g->vol); get(&g->dy32, S * g->vol); get(&g->h32, S * g->kvol); }
+    if (widen) { get(&g->q32, S * g->vol); get(&g->k32, S * g->vol); get(&g->v32, S * g->vol); get(&g->dy32, S * g->vol); if (!g->h_native) get(&g->h32, S * g->kvol); }
     get(&g->ones, S * g->vol); get(&g->t32, S * g->vol); get(&g->hopp, S * g->kopp);
     get(&g->aux, S * g->vol); get(&g->dhs, S * g->kvol); get(&g->dh32, S * g->kvol);
     if (g->ns) {
@@ -1484,13 +1487,15 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
 }
 
 // one forward of `n` slices on an inner fp32 plan (a plan of more slices runs the first n)
-static int grad_forward(hyenand_plan *p, long long n, const float *q, const float *k, const float *v, const float *h,
-                        bool shared, float *y, cudaStream_t st)
+static int grad_forward(hyenand_plan *p, long long n, const float *q, const float *k, const float *v, const void *h,
+                        bool shared, float *y, cudaStream_t st, int h_dtype = HYENAND_F32)
 {
     int launches = 0;
+    if (!plan_set_filter_dtype(p, h_dtype)) return fail(HYENAND_ERR_UNSUPPORTED, "filter element type on this path");
     p->r0 = 0; p->r1 = n;
     const int e = run_forward(p, q, k, v, h, shared, y, st, &launches);
     p->r0 = 0; p->r1 = (long long)p->B * p->C;
+    p->h_dtype = p->dtype;
     return e;
 }
 
@@ -1527,8 +1532,10 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
     const bool widen = g->dtype == HYENAND_BF16;
     const long long C = g->C, vol = g->vol, kvol = g->kvol;
     const int *L = g->L, *K = g->K, *P = g->P;
+    const bool nat = widen && g->h_native;                     // bf16 taps go to the transforms as they are
+    const int hdt = nat ? HYENAND_BF16 : HYENAND_F32;
     const float *hsh = (const float *)h;                       // shared kernel, fp32 view
-    if (shared && widen) { launch_widen(h, g->dtype, C * kvol, g->h32, st); hsh = g->h32; }
+    if (shared && widen && !nat) { launch_widen(h, g->dtype, C * kvol, g->h32, st); hsh = g->h32; }
     for (int b0 = 0; b0 < g->B; b0 += g->nb) {
         const long long n = g->B - b0 < g->nb ? g->B - b0 : g->nb, S = n * C, off = (long long)b0 * C * vol;
         const float *q32 = (const float *)q + off, *k32 = (const float *)k + off, *v32 = (const float *)v + off, *dy32 = (const float *)dy + off;
@@ -1538,19 +1545,20 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             launch_widen((const char *)v + off * es, g->dtype, S * vol, g->v32, st); v32 = g->v32;
             launch_widen((const char *)dy + off * es, g->dtype, S * vol, g->dy32, st); dy32 = g->dy32;
         }
-        const float *h32 = hsh;
+        const float *h32 = hsh;                                  // (bf16 taps when nat)
         if (!shared) {
-            h32 = (const float *)h + (long long)b0 * C * kvol;
-            if (widen) { launch_widen((const char *)h + (long long)b0 * C * kvol * es, g->dtype, S * kvol, g->h32, st); h32 = g->h32; }
+            h32 = (const float *)((const char *)h + (long long)b0 * C * kvol * es);
+            if (widen && !nat) { launch_widen((const char *)h + (long long)b0 * C * kvol * es, g->dtype, S * kvol, g->h32, st); h32 = g->h32; }
         }
         const long long Sh = shared ? C : S;
         // dq = dy * (h conv (k v))
-        if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st))) return e;
+        if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
         launch_mul_cast(g->t32, nullptr, S * vol, g->dtype, (char *)dq + off * es, st);
         // the kernel at the opposite displacement
         {
             RemapArgs r{};
             r.a = h32; r.b = nullptr; r.out = g->hopp; r.slices = Sh;
+            r.a_bf16 = r.out_bf16 = nat;
             for (int a = 0; a < 3; ++a) {
                 r.Ls[a] = K[a]; r.G[a] = K[a];
                 r.mode[a] = g->mode == HYENAND_MODE_CIRCULAR ? REMAP_NEG : REMAP_REV;
@@ -1559,7 +1567,7 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             launch_remap(r, st);
         }
         // du = h' conv (dy q);  dk = du v, dv = du k
-        if ((e = grad_forward(g->adj, S, g->ones, dy32, q32, g->hopp, shared, g->t32, st))) return e;
+        if ((e = grad_forward(g->adj, S, g->ones, dy32, q32, g->hopp, shared, g->t32, st, hdt))) return e;
         launch_mul_cast(g->t32, v32, S * vol, g->dtype, (char *)dk + off * es, st);
         launch_mul_cast(g->t32, k32, S * vol, g->dtype, (char *)dv + off * es, st);
         // dh
