@@ -247,6 +247,13 @@ int hyenand_synthesize_kernel(int ndim, const int *dims, int mode, int B, int C,
                               const float *W1, const float *b1, const float *omega0, const float *Wh, const float *bh,
                               const float *Wout, const float *bout, const float *gamma, const float *beta,
                               const float *window, int dtype, void *h, void *cuda_stream);
+/* The hidden and output layers of the network run on the tensor cores (tcgen05.mma, tf32 operands split in two so
+ * that the products keep fp32 accuracy) wherever the operands fit in shared memory; the one wait of that kernel is
+ * bounded.  Returns 0, or 1 once such a wait has given up since the library was loaded (the call that met it stored
+ * an incomplete kernel), -1 if the word cannot be read.  Synchronises the device.  HYENAND_SYNTH_ALU in the
+ * environment (read at the first call) selects the version without tensor cores. */
+int hyenand_synth_device_status(void);
+
 
 /*
  * Forward pass that allocates nothing (no counterpart in the paper: an integration aid).

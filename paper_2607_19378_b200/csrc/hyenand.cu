@@ -1658,6 +1658,9 @@ extern "C" long long hyenand_backward_guard_damage(hyenand_grad *g)
 
 // ---- kernel synthesis ---------------------------------------------------------------------------------
 
+extern "C" int hyenand_synth_device_status(void) { return synth_device_status(); }
+
+
 extern "C" int hyenand_synthesize_kernel(int ndim, const int *dims, int mode, int B, int C, int hidden, int layers,
                                          const float *W1, const float *b1, const float *omega0, const float *Wh,
                                          const float *bh, const float *Wout, const float *bout, const float *gamma,
@@ -1686,6 +1689,8 @@ extern "C" int hyenand_synthesize_kernel(int ndim, const int *dims, int mode, in
     }
     a.W1 = W1; a.b1 = b1; a.omega0 = omega0; a.Wh = Wh; a.bh = bh; a.Wout = Wout; a.bout = bout;
     a.gamma = gamma; a.beta = beta; a.window = window; a.h = h; a.dtype = dtype;
+    static const bool alu_only = getenv("HYENAND_SYNTH_ALU") != nullptr;     // development switch, read once
+    a.no_tensor_cores = alu_only;
     {
         DbgScope d;
         const size_t f = sizeof(float);

@@ -14,6 +14,8 @@
 // fast-math so that nothing else (divisions, the reduction) is replaced by approximations.
 #include "common.cuh"
 #include "synth.cuh"
+#include "tma_util.cuh"
+#include "tmem_util.cuh"
 
 namespace hn {
 
@@ -25,7 +27,9 @@ constexpr int kSynChanChunk = 32;        // output channels whose weights sit in
 
 __device__ __forceinline__ float sin_reduced(float x)
 {
-    const float k = rintf(x * 0.15915494309189535f);
+    // nearest integer of x / 2 pi by adding and subtracting 1.5 * 2^23 (two full-rate additions; the rounding
+    // instruction runs on the quarter-rate pipe the sine itself needs); exact for |x / 2 pi| < 2^22
+    const float k = (fmaf(x, 0.15915494309189535f, 12582912.f)) - 12582912.f;
     float r = fmaf(-k, 6.2831854820251465f, x);           // float(2 pi)
     r = fmaf(k, 1.7484555e-7f, r);                        // float(2 pi) - 2 pi
     return __sinf(r);
@@ -173,6 +177,277 @@ __global__ void __launch_bounds__(kSynThreads) synth_kernel(SynthArgs p)
     }
 }
 
+// ---- tensor-core version ---------------------------------------------------------------------------------------
+// The hidden layers and the output layer are dense contractions: per tile of 128 taps, [128 x HF] activations times
+// [HF x HF] (or [HF x 32 channels]) weights.  They run on the tensor cores: one thread issues tcgen05.mma
+// (cta_group::1, kind::tf32, M = 128, N = HF or 32, K = 8 per instruction), the operands sit in shared memory in the
+// canonical K-major layout without swizzle (8-row x 16-byte core matrices, 128 bytes apart along K, HF/4 * 128 bytes
+// apart along M/N), the accumulator [128 lanes x N columns] sits in tensor memory, tap t of the tile in lane t, and
+// every thread reads its own tap's row back with tcgen05.ld for the bias, the FiLM modulation and the sine, which
+// stay on the ALUs.  fp32 accuracy from tf32 products: activations and weights are split x = hi + lo (hi = x rounded
+// to tf32, lo = the remainder, of which the tensor cores read the leading tf32 bits) and every contraction is three accumulating products
+// hi*hi + hi*lo + lo*hi (the dropped lo*lo term is 2^-22 of the product).  The first layer (N coordinates in, sines of
+// arguments of tens of radians) and the window stay in fp32 on the ALUs.  A CTA is persistent over tiles; its weights
+// are split and staged once.  The one wait on the tensor cores (mbarrier armed by tcgen05.commit) is bounded: if it
+// gives up, the CTA raises the module's status word, stores nothing more and returns.
+static __device__ int hn_synth_status;
+
+constexpr int kTcThreads = 128;                          // = taps per tile = rows of the accumulator
+constexpr int kTcChan = 32;                              // output channels per contraction
+
+// x rounded to the nearest tf32 (10 explicit mantissa bits) with integer arithmetic: the conversion instruction runs
+// on the quarter-rate pipe, which the sines already fill
+__device__ __forceinline__ float to_tf32(float x)
+{
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
+}
+
+// K-major operand tile without swizzle: element (row, k) of a [rows x HF] tile
+template <int HF> __device__ __forceinline__ int tc_off(int row, int k)
+{
+    return (row >> 3) * (HF / 4) * 32 + (k >> 2) * 32 + (row & 7) * 4 + (k & 3);        // in floats
+}
+
+template <int HF> __device__ __forceinline__ unsigned long long tc_desc(unsigned smem_addr)
+{
+    constexpr unsigned long long LBO = 128 >> 4, SBO = ((HF / 4) * 128) >> 4;
+    return (unsigned long long)((smem_addr & 0x3ffffu) >> 4) | (LBO << 16) | (SBO << 32) | (1ull << 46);
+}
+
+__device__ __forceinline__ void tc_mma_tf32(unsigned tmem_d, unsigned long long da, unsigned long long db, unsigned idesc, unsigned accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n}\n"
+                 ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+
+template <int HF> constexpr size_t synth_tc_smem(int layers)
+{
+    // A hi/lo, hidden-layer weights hi/lo, output chunk hi/lo, small parameters, barrier + tensor-memory slot
+    return sizeof(float) * ((size_t)2 * kTcThreads * HF + (size_t)(layers - 1) * 2 * HF * HF + (size_t)2 * kTcChan * HF +
+                            (size_t)HF * 4 + HF + (size_t)(layers - 1) * HF + (size_t)layers * 2 * HF + kTcChan + 3 * kTcChan) + 64;
+}
+
+template <typename T, int HF>
+__global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
+{
+    extern __shared__ float4 smem4[];
+    float *sm = reinterpret_cast<float *>(smem4);
+    const int J = p.layers, H = p.hidden, N = p.ndim;
+    constexpr int TA = kTcThreads * HF, TB = HF * HF, TO = kTcChan * HF;
+    float *sA = sm;                                        // [2][128 x HF]  activations, hi then lo
+    float *sB = sA + 2 * TA;                               // [J-1][2][HF x HF]
+    float *sO = sB + (J - 1) * 2 * TB;                     // [2][32 x HF]   output-layer chunk
+    float *sW1 = sO + 2 * TO;
+    float *sOm = sW1 + HF * 4;
+    float *sBh = sOm + HF;
+    float *sFi = sBh + (J - 1) * HF;
+    float *sBo = sFi + J * 2 * HF;
+    float *sWin = sBo + kTcChan;                           // [3][32]
+    uint64_t *bar = reinterpret_cast<uint64_t *>(sWin + 3 * kTcChan);
+    unsigned *tslot = reinterpret_cast<unsigned *>(bar + 1);
+    const int tid = threadIdx.x, warp = tid >> 5, b = blockIdx.y;
+    constexpr unsigned TCOLS = HF > kTcChan ? HF : kTcChan;                   // 32 or 64: a power of two >= 32
+    if (warp == 0) tmem_alloc(smem_u32(tslot), TCOLS);
+    if (tid == 0) { mbar_init(bar, 1); fence_mbar_init(); }
+    for (int i = tid; i < HF; i += kTcThreads) {
+        const bool in = i < H;
+        for (int a = 0; a < 3; ++a) {
+            const int ua = a - (3 - N);
+            sW1[i * 4 + a] = (in && ua >= 0) ? SYN_LD(p.W1, i * N + ua) : 0.f;
+        }
+        sW1[i * 4 + 3] = in ? SYN_LD(p.b1, i) : 0.f;
+        sOm[i] = in ? SYN_LD(p.omega0, i) : 0.f;
+        for (int j = 0; j < J; ++j) {
+            sFi[(j * 2 + 0) * HF + i] = in ? (p.gamma ? SYN_LD(p.gamma, ((long long)b * J + j) * H + i) : 1.f) : 0.f;
+            sFi[(j * 2 + 1) * HF + i] = in ? (p.beta ? SYN_LD(p.beta, ((long long)b * J + j) * H + i) : 0.f) : 0.f;
+        }
+        for (int j = 0; j + 1 < J; ++j) sBh[j * HF + i] = in ? SYN_LD(p.bh, j * H + i) : 0.f;
+    }
+    // hidden-layer weights W[out n][in k], split and laid out as the B operand (N rows, K-major)
+    for (int e = tid; e < (J - 1) * TB; e += kTcThreads) {
+        const int j = e / TB, n = (e / HF) % HF, k = e % HF;
+        const float w = (n < H && k < H) ? SYN_LD(p.Wh, ((long long)j * H + n) * H + k) : 0.f;
+        const float hi = to_tf32(w);
+        sB[(j * 2 + 0) * TB + tc_off<HF>(n, k)] = hi;
+        sB[(j * 2 + 1) * TB + tc_off<HF>(n, k)] = to_tf32(w - hi);
+    }
+    tmem_fence_before_sync();
+    __syncthreads();
+    tmem_fence_after_sync();
+    const unsigned tbase = *tslot;
+    const unsigned trow = tmem_addr(tbase, warp, 0);       // this thread's lane, column 0
+    const unsigned aA = smem_u32(sA), aB = smem_u32(sB), aO = smem_u32(sO);
+    constexpr unsigned IDESC_H = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(HF >> 3) << 17) | ((unsigned)(kTcThreads >> 4) << 24);
+    constexpr unsigned IDESC_O = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(kTcChan >> 3) << 17) | ((unsigned)(kTcThreads >> 4) << 24);
+    const long long taps = (long long)p.K[0] * p.K[1] * p.K[2];
+    const long long tiles = (taps + kTcThreads - 1) / kTcThreads;
+    T *out = (T *)p.h + (long long)b * p.C * taps;
+    unsigned phase = 0;
+    bool failed = false;
+    // one contraction: A (activations in sA) times the B operand at shared address ab (hi at ab, lo at ab + tb bytes)
+    auto contract = [&](unsigned ab, unsigned tb, unsigned idesc) {
+        if (tid == 0) {
+            tmem_fence_after_sync();
+#pragma unroll
+            for (int ks = 0; ks < HF / 8; ++ks) {
+                const unsigned long long ah = tc_desc<HF>(aA + ks * 256), al = tc_desc<HF>(aA + TA * 4 + ks * 256);
+                const unsigned long long bh = tc_desc<HF>(ab + ks * 256), bl = tc_desc<HF>(ab + tb + ks * 256);
+                tc_mma_tf32(tbase, ah, bh, idesc, ks != 0);
+                tc_mma_tf32(tbase, ah, bl, idesc, 1);
+                tc_mma_tf32(tbase, al, bh, idesc, 1);
+            }
+            tc_commit(bar);
+        }
+        const bool ok = mbar_wait(bar, phase);
+        failed = __syncthreads_or(!ok) != 0;                // one decision for the whole CTA
+        phase ^= 1u;
+        tmem_fence_after_sync();
+    };
+    // this thread's activations -> row tid of the A operand, split
+    auto put_acts = [&](const float (&act)[HF]) {
+#pragma unroll
+        for (int kc = 0; kc < HF / 4; ++kc) {
+            float4 hi, lo;
+            hi.x = to_tf32(act[4 * kc]); hi.y = to_tf32(act[4 * kc + 1]); hi.z = to_tf32(act[4 * kc + 2]); hi.w = to_tf32(act[4 * kc + 3]);
+            // the remainder goes in as it is: the tensor cores read its leading tf32 bits (2^-11 of 2^-11 is dropped)
+            lo.x = act[4 * kc] - hi.x; lo.y = act[4 * kc + 1] - hi.y;
+            lo.z = act[4 * kc + 2] - hi.z; lo.w = act[4 * kc + 3] - hi.w;
+            *reinterpret_cast<float4 *>(sA + tc_off<HF>(tid, 4 * kc)) = hi;
+            *reinterpret_cast<float4 *>(sA + TA + tc_off<HF>(tid, 4 * kc)) = lo;
+        }
+        fence_async_smem();                                // generic-proxy writes visible to the tensor cores
+        tmem_fence_before_sync();                          // (and this thread's tensor-memory reads precede the next product)
+        __syncthreads();
+    };
+    for (long long tile = blockIdx.x; tile < tiles && !failed; tile += gridDim.x) {
+        long long t = tile * kTcThreads + tid;
+        const bool live = t < taps;
+        if (!live) t = taps - 1;                           // clamped: computed, never stored
+        const int m2 = (int)(t % p.K[2]), m1 = (int)((t / p.K[2]) % p.K[1]), m0 = (int)(t / ((long long)p.K[2] * p.K[1]));
+        const float cx0 = axis_coord(m0, p.L[0], p.mode), cx1 = axis_coord(m1, p.L[1], p.mode), cx2 = axis_coord(m2, p.L[2], p.mode);
+        float act[HF];
+#pragma unroll
+        for (int i = 0; i < HF; ++i) {
+            const float4 w = *reinterpret_cast<const float4 *>(sW1 + 4 * i);
+            const float pre = fmaf(w.x, cx0, fmaf(w.y, cx1, fmaf(w.z, cx2, w.w)));
+            act[i] = fmaf(sFi[i], sin_reduced(sOm[i] * pre), sFi[HF + i]);
+        }
+        for (int j = 1; j < J; ++j) {
+            put_acts(act);
+            contract(aB + (j - 1) * 2 * TB * 4, TB * 4, IDESC_H);
+            if (failed) break;
+#pragma unroll
+            for (int c0 = 0; c0 < HF; c0 += 16) {
+                float acc[16];
+                TmemIO<16>::ld(acc, trow + c0);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    act[c0 + i] = fmaf(sFi[(j * 2) * HF + c0 + i], sin_reduced(acc[i] + sBh[(j - 1) * HF + c0 + i]), sFi[(j * 2 + 1) * HF + c0 + i]);
+            }
+        }
+        if (failed) break;
+        put_acts(act);                                      // operand of every output chunk
+        for (int c0 = 0; c0 < p.C; c0 += kTcChan) {
+            const int nc = p.C - c0 < kTcChan ? p.C - c0 : kTcChan;
+            // output weights of this chunk (one chunk: staged once per CTA; more: once per tile and chunk)
+            if (tile == (long long)blockIdx.x || p.C > kTcChan) {
+                for (int e = tid; e < TO; e += kTcThreads) {
+                    const int c = e / HF, k = e % HF;
+                    const float w = (c < nc && k < H) ? SYN_LD(p.Wout, (long long)(c0 + c) * H + k) : 0.f;
+                    const float hi = to_tf32(w);
+                    sO[tc_off<HF>(c, k)] = hi;
+                    sO[TO + tc_off<HF>(c, k)] = to_tf32(w - hi);
+                }
+                for (int c = tid; c < kTcChan; c += kTcThreads) {
+                    sBo[c] = c < nc ? SYN_LD(p.bout, c0 + c) : 0.f;
+                    for (int a = 0; a < 3; ++a) {
+                        const int ua = a - (3 - N);
+                        float wv = 0.f;                    // Gaussian: 1 / sigma per axis; causal: alpha in slot 2
+                        if (c < nc) {
+                            if (p.mode == 1) wv = a == 2 ? SYN_LD(p.window, c0 + c) : 0.f;
+                            else if (ua >= 0) wv = 1.f / SYN_LD(p.window, (long long)ua * p.C + c0 + c);
+                        }
+                        sWin[a * kTcChan + c] = wv;
+                    }
+                }
+                fence_async_smem();
+                tmem_fence_before_sync();
+                __syncthreads();
+            }
+            contract(aO, TO * 4, IDESC_O);
+            if (failed) break;
+#pragma unroll
+            for (int q0 = 0; q0 < kTcChan; q0 += 16) {
+                float acc[16];
+                TmemIO<16>::ld(acc, trow + q0);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int c = q0 + i;
+                    float win;
+                    if (p.mode == 1) win = __expf(-sWin[2 * kTcChan + c] * fabsf(cx2));
+                    else {
+                        const float a0 = cx0 * sWin[c], a1 = cx1 * sWin[kTcChan + c], a2 = cx2 * sWin[2 * kTcChan + c];
+                        win = __expf(-0.5f * (a0 * a0 + a1 * a1 + a2 * a2));
+                    }
+                    if (live && c < nc) IO<T>::st(out, (long long)(c0 + c) * taps + t, win * (acc[i] + sBo[c]));
+                }
+            }
+            if (p.C > kTcChan) {
+                // the next chunk's weights overwrite sO and the next product overwrites the accumulator
+                tmem_fence_before_sync();
+                __syncthreads();
+            }
+        }
+    }
+    if (failed) atomicExch(&hn_synth_status, 1);
+    tmem_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tbase, TCOLS);
+}
+
+int synth_device_status()
+{
+    int v = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(&v, hn_synth_status, sizeof(int)) != cudaSuccess) return -1;
+    return v;
+}
+
+template <typename T, int HF> static int launch_synth_tc_t(const SynthArgs &a, cudaStream_t st)
+{
+    const long long taps = (long long)a.K[0] * a.K[1] * a.K[2];
+    const long long tiles = (taps + kTcThreads - 1) / kTcThreads;
+    const size_t sm = synth_tc_smem<HF>(a.layers);
+    if (tiles <= 0 || a.B > 65535 || sm > 160 * 1024) return -1;
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms <= 0) sms = 148;
+    }
+    static DevOnce attr;
+    if (attr.first()) cudaFuncSetAttribute(synth_tc_kernel<T, HF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    // persistent CTAs: as many as fit (shared memory, 512 tensor-memory columns per SM), at most one per tile
+    long long per_sm = (220 * 1024) / (long long)(sm + 1024);
+    const long long by_tmem = 512 / (HF > kTcChan ? HF : kTcChan);
+    if (per_sm > by_tmem) per_sm = by_tmem;
+    if (per_sm > 8) per_sm = 8;
+    if (per_sm < 1) per_sm = 1;
+    long long grid = (long long)sms * per_sm / (a.B < sms * per_sm ? a.B : 1);
+    if (grid < 1) grid = 1;
+    if (grid > tiles) grid = tiles;
+    synth_tc_kernel<T, HF><<<dim3((unsigned)grid, (unsigned)a.B), kTcThreads, sm, st>>>(a);
+    return 1;
+}
+
 bool synth_supported(int hidden, int layers) { return hidden >= 1 && hidden <= 64 && layers >= 1 && layers <= 8; }
 
 template <typename T, int HF, int NC> static int launch_synth_t(const SynthArgs &a, cudaStream_t st)
@@ -193,6 +468,14 @@ template <typename T, int HF, int NC> static int launch_synth_t(const SynthArgs 
 int launch_synth(const SynthArgs &a, cudaStream_t st)
 {
     if (!synth_supported(a.hidden, a.layers)) return -1;
+    // tensor-core version for 17 .. 64 hidden units wherever its operands fit in shared memory (else the ALU version)
+    if (!a.no_tensor_cores) {
+        int n = -1;
+        if (a.hidden <= 16) n = -1;                        // 16 units: the products are too small to pay for the round trips
+        else if (a.hidden <= 32) n = a.dtype == 0 ? launch_synth_tc_t<float, 32>(a, st) : launch_synth_tc_t<bf16, 32>(a, st);
+        else n = a.dtype == 0 ? launch_synth_tc_t<float, 64>(a, st) : launch_synth_tc_t<bf16, 64>(a, st);
+        if (n >= 0) return n;
+    }
 #define HN_SYN(T)                                                                   \
     do {                                                                            \
         if (a.hidden <= 16) return launch_synth_t<T, 16, 2>(a, st);                 \

@@ -15,9 +15,12 @@ struct SynthArgs {
     const float *window;               // Gaussian: sigma [ndim][C]; causal: alpha [C]
     void *h;                           // [B][C][K...] in the I/O dtype
     int dtype;
+    int no_tensor_cores;               // 1: the ALU version (development switch HYENAND_SYNTH_ALU)
 };
 
 bool synth_supported(int hidden, int layers);
 int launch_synth(const SynthArgs &a, cudaStream_t st);
+// 0, or 1 once a bounded wait on the tensor cores has given up (synchronises the device); -1 if it cannot be read
+int synth_device_status();
 
 }  // namespace hn

@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.hyenand_debug_violations.restype = ll
         L.hyenand_debug_violations.argtypes = [ctypes.POINTER(ctypes.c_ulonglong), ip, ctypes.POINTER(ctypes.c_char_p)]
         L.hyenand_debug_selftest.restype = ll
+        L.hyenand_synth_device_status.restype = ctypes.c_int
         L.hyenand_selftest_bounded_wait.argtypes = [ctypes.c_int]
         L.hyenand_selftest_bounded_wait.restype = ctypes.c_int
         L.hyenand_plan_device_status.argtypes = [vp]
@@ -171,6 +172,10 @@ def hyenand_debug_violations():
     addr, line, name = ctypes.c_ulonglong(), ctypes.c_int(), ctypes.c_char_p()
     n = lib().hyenand_debug_violations(ctypes.byref(addr), ctypes.byref(line), ctypes.byref(name))
     return int(n), int(addr.value), int(line.value), (name.value or b"").decode()
+
+
+def hyenand_synth_device_status() -> int:
+    return int(lib().hyenand_synth_device_status())
 
 
 def hyenand_debug_selftest() -> int:

@@ -134,3 +134,26 @@ def test_synthesised_kernel_feeds_the_convolution(dtype):
         assert err <= 1.5 * TOL[dtype]
     else:
         assert err <= 2e-5
+
+
+def test_tensor_core_wait_never_gave_up():
+    """The tensor-core version (17 .. 64 hidden units) has one bounded wait; none of the calls of this process met its
+    limit."""
+    from paper_2607_19378_b200 import hyenand as hn
+    p = make_params(2, 32, 3, 40, 2, "linear", seed=74)
+    gpu_synthesize((48, 40), "linear", 2, 40, 32, 3, p, "f32")
+    assert hn.hyenand_synth_device_status() == 0
+
+
+def test_version_without_tensor_cores_behind_its_switch():
+    """HYENAND_SYNTH_ALU is read once per process: the parity cases run again in a child process that sets it."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    if os.environ.get("HYENAND_SYNTH_ALU"):
+        pytest.skip("already running with the switch")
+    env = dict(os.environ, HYENAND_SYNTH_ALU="1")
+    r = subprocess.run([sys.executable, "-m", "pytest", "-m", "gpu", "-x", "-q", "-p", "no:cacheprovider", "-k", "matches_the_oracle",
+                        "tests/test_gpu_synthesis.py"], cwd=root, env=env, capture_output=True, text=True, timeout=1500)
+    assert r.returncode == 0, (r.stdout[-3000:], r.stderr[-2000:])
