@@ -1753,7 +1753,7 @@ extern "C" int hyenand_forward_noalloc(int ndim, const int *dims, int B, int C, 
     static thread_local hyenand_plan sp;
     memset(&sp, 0, sizeof(sp));
     hyenand_plan *p = &sp;
-    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype;
+    p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype; p->h_dtype = dtype;
     p->r0 = 0; p->r1 = (long long)B * C;
     p->vol = 1; p->kvol = 1;
     for (int a = 0; a < 3; ++a) { p->L[a] = 1; p->K[a] = 1; p->P[a] = 1; p->log2p[a] = 0; }
