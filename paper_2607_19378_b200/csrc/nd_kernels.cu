@@ -169,13 +169,23 @@ __global__ void __launch_bounds__(kThreads) rows_inv_kernel(RowsInvArgs p)
         }
         __syncthreads();
         fft_lines<LOG2P, true, FULL ? PRUNE_NONE : PRUNE_OUT, kThreads>(buf, G, LS, tw, tid);
-        for (int idx = tid; idx < G * p.len; idx += kThreads) {
-            const int g = idx / p.len, n = idx % p.len;
-            const long long r0 = 2 * (ch * G + g), r1 = r0 + 1;
-            const float2 z = buf[g * LS + phys(n)];
-            // (no gate tensor: the rows leave as they are)
-            if (r0 < p.rows) IO<T>::st(py, r0 * p.len + n, pq ? z.x * IO<T>::ld(pq, r0 * p.len + n) : z.x);
-            if (r1 < p.rows) IO<T>::st(py, r1 * p.len + n, pq ? z.y * IO<T>::ld(pq, r1 * p.len + n) : z.y);
+        if (pq) {
+            for (int idx = tid; idx < G * p.len; idx += kThreads) {
+                const int g = idx / p.len, n = idx % p.len;
+                const long long r0 = 2 * (ch * G + g), r1 = r0 + 1;
+                const float2 z = buf[g * LS + phys(n)];
+                if (r0 < p.rows) IO<T>::st(py, r0 * p.len + n, z.x * IO<T>::ld(pq, r0 * p.len + n));
+                if (r1 < p.rows) IO<T>::st(py, r1 * p.len + n, z.y * IO<T>::ld(pq, r1 * p.len + n));
+            }
+        } else {
+            // no gate tensor: the rows leave as they are
+            for (int idx = tid; idx < G * p.len; idx += kThreads) {
+                const int g = idx / p.len, n = idx % p.len;
+                const long long r0 = 2 * (ch * G + g), r1 = r0 + 1;
+                const float2 z = buf[g * LS + phys(n)];
+                if (r0 < p.rows) IO<T>::st(py, r0 * p.len + n, z.x);
+                if (r1 < p.rows) IO<T>::st(py, r1 * p.len + n, z.y);
+            }
         }
         __syncthreads();
     }

@@ -211,11 +211,20 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
                 IO<T>::st(py, r1 * HP + l + t * TPL, z.y * qb[t]);
             }
         } else {
-            for (int n = l; n < p.len; n += TPL) {
-                const float2 z = line[FI::ph(n)];
-                // (no gate tensor: the rows leave as they are)
-                IO<T>::st(py, r0 * p.len + n, pq ? z.x * IO<T>::ld(pq, r0 * p.len + n) : z.x);
-                if (has1) IO<T>::st(py, r1 * p.len + n, pq ? z.y * IO<T>::ld(pq, r1 * p.len + n) : z.y);
+            if (pq) {
+                // (a loop of its own: the read-only gate loads of several iterations go out together)
+                for (int n = l; n < p.len; n += TPL) {
+                    const float2 z = line[FI::ph(n)];
+                    IO<T>::st(py, r0 * p.len + n, z.x * IO<T>::ld(pq, r0 * p.len + n));
+                    if (has1) IO<T>::st(py, r1 * p.len + n, z.y * IO<T>::ld(pq, r1 * p.len + n));
+                }
+            } else {
+                // no gate tensor: the rows leave as they are
+                for (int n = l; n < p.len; n += TPL) {
+                    const float2 z = line[FI::ph(n)];
+                    IO<T>::st(py, r0 * p.len + n, z.x);
+                    if (has1) IO<T>::st(py, r1 * p.len + n, z.y);
+                }
             }
         }
         __syncwarp(m);
