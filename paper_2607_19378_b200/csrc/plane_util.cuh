@@ -101,54 +101,6 @@ template <int D> __host__ __device__ __forceinline__ constexpr int spread_pair(i
     return ((g >> 1) & (D - 1)) | ((g & 1) * D) | (g & ~(2 * D - 1));
 }
 
-// Separate the spectra of the two real rows packed in one complex transform (results in
-// `line`, natural order) and scatter them into column store rows y0, y1.
-template <int LOG2P, int CSS>
-__device__ __forceinline__ void separate_rows(const float2 *line, float2 *cs, int y0, int y1, int l)
-{
-    using FW = WF<LOG2P, false>;
-    constexpr int P = 1 << LOG2P, HP = P / 2, TPL = FW::TPL;
-    // bins 1 .. HP-1 (lane 0's first entry, bin 0, is overwritten below)
-#pragma unroll
-    for (int t = 0; t < HP / TPL; ++t) {
-        const int kx = l + t * TPL;
-        const float2 z1 = line[FW::ph(kx)];
-        const float2 z2 = line[FW::ph((P - kx) & (P - 1))];
-        cs[kx * CSS + y0] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
-        cs[kx * CSS + y1] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
-    }
-    __syncwarp(WF<LOG2P, false>::group_mask(threadIdx.x));
-    if (l == 0) {
-        // the two purely real bins (kx = 0 and kx = P/2) of each row share column 0
-        const float2 z0 = line[FW::ph(0)], zh = line[FW::ph(HP)];
-        cs[y0] = make_float2(z0.x, zh.x);
-        cs[y1] = make_float2(z0.y, zh.y);
-    }
-}
-
-// Same separation, but the two purely real bins of a row (kx = 0 and kx = P/2) get columns of their own
-// (0 and P/2) as ordinary complex entries with zero imaginary part: P/2 + 1 columns, no packing.
-template <int LOG2P, int CSS>
-__device__ __forceinline__ void separate_rows_full(const float2 *line, float2 *cs, int y0, int y1, int l)
-{
-    using FW = WF<LOG2P, false>;
-    constexpr int P = 1 << LOG2P, HP = P / 2, TPL = FW::TPL;
-#pragma unroll
-    for (int t = 0; t < HP / TPL; ++t) {
-        const int kx = l + t * TPL;
-        const float2 z1 = line[FW::ph(kx)];
-        const float2 z2 = line[FW::ph((P - kx) & (P - 1))];
-        // for kx = 0 both reads are bin 0 and the formulas give (z.x, 0) and (z.y, 0), as they must
-        cs[kx * CSS + y0] = make_float2(0.5f * (z1.x + z2.x), 0.5f * (z1.y - z2.y));
-        cs[kx * CSS + y1] = make_float2(0.5f * (z1.y + z2.y), 0.5f * (z2.x - z1.x));
-    }
-    if (l == 0) {
-        const float2 zh = line[FW::ph(HP)];
-        cs[HP * CSS + y0] = make_float2(zh.x, 0.f);
-        cs[HP * CSS + y1] = make_float2(zh.y, 0.f);
-    }
-}
-
 // Twiddle source of the P-point transforms of a plane kernel: registers when the plan has two
 // equal passes (the twiddles of the second pass then depend on the lane only), else per-pass
 // tables in shared memory.

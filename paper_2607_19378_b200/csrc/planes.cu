@@ -13,12 +13,14 @@
 //              decimation-in-frequency step applied to the taps as they are read), each
 //              half filling a column store of the size of a k*v plane's.  The tap rows are
 //              fetched once: the odd half's inputs wait in tensor memory meanwhile.
+//              Output at twice its value as well (the core's scale carries both factors).
 //   plane_inv  inverse along y (keeping the cropped rows; two rows combined into one
 //              complex row as they leave the registers), inverse complex-to-real
 //              along x, crop, output gate q, store.
 //
-// Column 0 of the column store carries the two purely real bins of every row (kx = 0 and
-// kx = P/2) as one complex number, so a plane has exactly P/2 columns.
+// The stores hold the RAW transforms of the row pairs, [bin][row pair]; a column reads its bin and the mirrored one.
+// The two purely real bins of every row (kx = 0 and kx = P/2) travel as one complex column, so a plane has
+// exactly P/2 columns.
 #include "common.cuh"
 #include "planes.cuh"
 #include "wfft.cuh"
@@ -29,10 +31,10 @@ namespace hn {
 
 template <int LOG2P> struct PlaneCfg {
     static constexpr int P = 1 << LOG2P, HP = P / 2, XH = HP + 1;
-    static constexpr int CSS = HP + 1;                       // column-store stride (odd)
+    static constexpr int CSS = HP + 1;                       // filter planes: store stride (odd), P/2 bins of P/2 row pairs per half
     using F = WF<LOG2P, false>;
     using FI = WF<LOG2P, true>;
-    using FH = WF<LOG2P - 1, false>;                         // half-length columns of hplane
+    using FH = WF<LOG2P - 1, false>;                         // half-length rows of hplane
     static constexpr int NG = kPlaneThreads / F::TPL;        // groups working on P-point lines
     static constexpr int NGH = kPlaneThreads / FH::TPL;      // groups working on P/2-point lines
     static constexpr int LS = plane_ls(P);
