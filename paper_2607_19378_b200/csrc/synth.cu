@@ -16,6 +16,7 @@
 #include "synth.cuh"
 #include "tma_util.cuh"
 #include "tmem_util.cuh"
+#include <type_traits>
 
 namespace hn {
 
@@ -180,11 +181,12 @@ __global__ void __launch_bounds__(kSynThreads) synth_kernel(SynthArgs p)
 // ---- tensor-core version ---------------------------------------------------------------------------------------
 // The hidden layers and the output layer are dense contractions: per tile of 128 taps, [128 x HF] activations times
 // [HF x HF] (or [HF x 32 channels]) weights.  They run on the tensor cores: one thread issues tcgen05.mma
-// (cta_group::1, kind::tf32, M = 128, N = HF or 32, K = 8 per instruction), the operands sit in shared memory in the
-// canonical K-major layout without swizzle (8-row x 16-byte core matrices, 128 bytes apart along K, HF/4 * 128 bytes
-// apart along M/N), the accumulator [128 lanes x N columns] sits in tensor memory, tap t of the tile in lane t, and
-// every thread reads its own tap's row back with tcgen05.ld for the bias, the FiLM modulation and the sine, which
-// stay on the ALUs.  fp32 accuracy from tf32 products: activations and weights are split x = hi + lo (hi = x rounded
+// (cta_group::1, kind::tf32, M = 128, K = 8 per instruction).  Tap t of a tile is thread t is lane t of tensor memory:
+// the activations (the A operand) are written there by their own threads with tcgen05.st, the weights (the B operand)
+// sit in shared memory in the K-major layout with the 128-byte swizzle, the accumulator [128 lanes x N columns] sits
+// in tensor memory as well, and every thread reads its own tap's row back with tcgen05.ld for the bias, the FiLM
+// modulation and the sine, which stay on the ALUs.  (With the activations in shared memory the tensor pipe spent its
+// time fetching them: 250 cycles per instruction, 60% of the kernel.)  fp32 accuracy from tf32 products: activations and weights are split x = hi + lo (hi = x rounded
 // to tf32, lo = the remainder, of which the tensor cores read the leading tf32 bits) and every contraction is three accumulating products
 // hi*hi + hi*lo + lo*hi (the dropped lo*lo term is 2^-22 of the product).  The first layer (N coordinates in, sines of
 // arguments of tens of radians) and the window stay in fp32 on the ALUs.  A CTA is persistent over tiles; its weights
@@ -202,16 +204,21 @@ __device__ __forceinline__ float to_tf32(float x)
     return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
 }
 
-// K-major operand tile without swizzle: element (row, k) of a [rows x HF] tile
-template <int HF> __device__ __forceinline__ int tc_off(int row, int k)
+// K-major operand tile in the 128-byte swizzle: a row holds 32 tf32 values of one K block (128 bytes), 8 rows make a
+// 1024-byte group, the 16-byte chunk index inside a row is XORed with the row's index in its group, and K blocks
+// (columns 32.., for 64 hidden units) follow one another as whole tiles.  Byte offset of element (row, k) of a tile
+// of ROWS rows.  (The layout without swizzle, 8 x 16-byte core matrices, puts every row group on the same banks: the
+// products then took 200 cycles per instruction and 60% of the kernel's time.)
+template <int ROWS> __device__ __forceinline__ int tc_off(int row, int k)
 {
-    return (row >> 3) * (HF / 4) * 32 + (k >> 2) * 32 + (row & 7) * 4 + (k & 3);        // in floats
+    return (k >> 5) * (ROWS * 128) + (row >> 3) * 1024 + (row & 7) * 128 + (((((k & 31) >> 2) ^ (row & 7))) << 4) + (k & 3) * 4;
 }
 
-template <int HF> __device__ __forceinline__ unsigned long long tc_desc(unsigned smem_addr)
+// descriptor of the 8-value K step ks (K block ks / 4) of a tile of ROWS rows, starting at row r0 (a multiple of 8)
+template <int ROWS> __device__ __forceinline__ unsigned long long tc_desc(unsigned tile_addr, int ks, int r0 = 0)
 {
-    constexpr unsigned long long LBO = 128 >> 4, SBO = ((HF / 4) * 128) >> 4;
-    return (unsigned long long)((smem_addr & 0x3ffffu) >> 4) | (LBO << 16) | (SBO << 32) | (1ull << 46);
+    const unsigned a = tile_addr + (unsigned)((ks >> 2) * (ROWS * 128) + (r0 >> 3) * 1024 + (ks & 3) * 32);
+    return (unsigned long long)((a & 0x3ffffu) >> 4) | (1ull << 16) | ((unsigned long long)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
 __device__ __forceinline__ void tc_mma_tf32(unsigned tmem_d, unsigned long long da, unsigned long long db, unsigned idesc, unsigned accumulate)
@@ -220,6 +227,13 @@ __device__ __forceinline__ void tc_mma_tf32(unsigned tmem_d, unsigned long long 
                  " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n}\n"
                  ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
 }
+// the same with the A operand in tensor memory ([128 lanes x 8 columns] at ta: row m of the tile is lane m)
+__device__ __forceinline__ void tc_mma_tf32_ts(unsigned tmem_d, unsigned ta, unsigned long long db, unsigned idesc, unsigned accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n}\n"
+                 ::"r"(tmem_d), "r"(ta), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u) : "memory");
+}
 __device__ __forceinline__ void tc_commit(uint64_t *bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar)) : "memory");
@@ -227,22 +241,23 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar)
 
 template <int HF> constexpr size_t synth_tc_smem(int layers)
 {
-    // A hi/lo, hidden-layer weights hi/lo, output chunk hi/lo, small parameters, barrier + tensor-memory slot
-    return sizeof(float) * ((size_t)2 * kTcThreads * HF + (size_t)(layers - 1) * 2 * HF * HF + (size_t)2 * kTcChan * HF +
-                            (size_t)HF * 4 + HF + (size_t)(layers - 1) * HF + (size_t)layers * 2 * HF + kTcChan + 3 * kTcChan) + 64;
+    // weight tiles (per hidden layer [2 HF x HF] = hi rows then lo rows; output chunk [64 x HF]), room to start them
+    // on a 1024-byte boundary, small parameters, barrier + tensor-memory slot (the activations live in tensor memory)
+    return (size_t)(layers - 1) * 2 * HF * HF * 4 + (size_t)2 * kTcChan * HF * 4 + 1024 +
+           sizeof(float) * ((size_t)HF * 4 + HF + (size_t)(layers - 1) * HF + (size_t)layers * 2 * HF + kTcChan + 3 * kTcChan) + 64;
 }
 
 template <typename T, int HF>
 __global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
 {
-    extern __shared__ float4 smem4[];
-    float *sm = reinterpret_cast<float *>(smem4);
+    extern __shared__ __align__(1024) unsigned char smem_dyn[];
+    // the swizzle pattern is a function of the shared-memory address: tiles start on 1024-byte boundaries
+    unsigned char *sm = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
     const int J = p.layers, H = p.hidden, N = p.ndim;
-    constexpr int TA = kTcThreads * HF, TB = HF * HF, TO = kTcChan * HF;
-    float *sA = sm;                                        // [2][128 x HF]  activations, hi then lo
-    float *sB = sA + 2 * TA;                               // [J-1][2][HF x HF]
-    float *sO = sB + (J - 1) * 2 * TB;                     // [2][32 x HF]   output-layer chunk
-    float *sW1 = sO + 2 * TO;
+    constexpr int TB = 2 * HF * HF * 4, TO = 2 * kTcChan * HF * 4;      // bytes
+    unsigned char *sB = sm;                                // [J-1] tiles of [2 HF x HF]: rows 0..HF-1 hi, HF..2HF-1 lo
+    unsigned char *sO = sB + (J - 1) * TB;                 // [64 x HF]: rows 0..31 hi, 32..63 lo of the output chunk
+    float *sW1 = reinterpret_cast<float *>(sO + TO);
     float *sOm = sW1 + HF * 4;
     float *sBh = sOm + HF;
     float *sFi = sBh + (J - 1) * HF;
@@ -251,7 +266,9 @@ __global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
     uint64_t *bar = reinterpret_cast<uint64_t *>(sWin + 3 * kTcChan);
     unsigned *tslot = reinterpret_cast<unsigned *>(bar + 1);
     const int tid = threadIdx.x, warp = tid >> 5, b = blockIdx.y;
-    constexpr unsigned TCOLS = HF > kTcChan ? HF : kTcChan;                   // 32 or 64: a power of two >= 32
+    // tensor memory: accumulator (hi*hi and hi*lo side by side), then this tile's activations, hi and lo: row = lane
+    constexpr unsigned DCOLS = 2 * (HF > kTcChan ? HF : kTcChan), TCOLS = DCOLS + 2 * HF;       // 128 or 256 columns
+    static_assert((TCOLS & (TCOLS - 1)) == 0 && TCOLS <= 512, "a power of two");
     if (warp == 0) tmem_alloc(smem_u32(tslot), TCOLS);
     if (tid == 0) { mbar_init(bar, 1); fence_mbar_init(); }
     for (int i = tid; i < HF; i += kTcThreads) {
@@ -269,38 +286,40 @@ __global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
         for (int j = 0; j + 1 < J; ++j) sBh[j * HF + i] = in ? SYN_LD(p.bh, j * H + i) : 0.f;
     }
     // hidden-layer weights W[out n][in k], split and laid out as the B operand (N rows, K-major)
-    for (int e = tid; e < (J - 1) * TB; e += kTcThreads) {
-        const int j = e / TB, n = (e / HF) % HF, k = e % HF;
+    for (int e = tid; e < (J - 1) * HF * HF; e += kTcThreads) {
+        const int j = e / (HF * HF), n = (e / HF) % HF, k = e % HF;
         const float w = (n < H && k < H) ? SYN_LD(p.Wh, ((long long)j * H + n) * H + k) : 0.f;
         const float hi = to_tf32(w);
-        sB[(j * 2 + 0) * TB + tc_off<HF>(n, k)] = hi;
-        sB[(j * 2 + 1) * TB + tc_off<HF>(n, k)] = to_tf32(w - hi);
+        *reinterpret_cast<float *>(sB + j * TB + tc_off<2 * HF>(n, k)) = hi;
+        *reinterpret_cast<float *>(sB + j * TB + tc_off<2 * HF>(HF + n, k)) = w - hi;
     }
+    fence_async_smem();                                    // generic-proxy writes visible to the tensor cores
     tmem_fence_before_sync();
     __syncthreads();
     tmem_fence_after_sync();
     const unsigned tbase = *tslot;
     const unsigned trow = tmem_addr(tbase, warp, 0);       // this thread's lane, column 0
-    const unsigned aA = smem_u32(sA), aB = smem_u32(sB), aO = smem_u32(sO);
-    constexpr unsigned IDESC_H = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(HF >> 3) << 17) | ((unsigned)(kTcThreads >> 4) << 24);
-    constexpr unsigned IDESC_O = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(kTcChan >> 3) << 17) | ((unsigned)(kTcThreads >> 4) << 24);
+    const unsigned aB = smem_u32(sB), aO = smem_u32(sO);
+    constexpr unsigned IDESC = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(kTcThreads >> 4) << 24);      // f32 out, tf32 in, K-major, M = 128
+    auto idesc_n = [](int n) { return IDESC | ((unsigned)(n >> 3) << 17); };
     const long long taps = (long long)p.K[0] * p.K[1] * p.K[2];
     const long long tiles = (taps + kTcThreads - 1) / kTcThreads;
     T *out = (T *)p.h + (long long)b * p.C * taps;
     unsigned phase = 0;
     bool failed = false;
-    // one contraction: A (activations in sA) times the B operand at shared address ab (hi at ab, lo at ab + tb bytes)
-    auto contract = [&](unsigned ab, unsigned tb, unsigned idesc) {
+    // One contraction of the activations (in tensor memory) with a weight tile of 2 NB rows (NB hi rows, then NB lo rows):
+    // A_hi x [B_hi; B_lo] fills accumulator columns [0, 2 NB) with hi*hi | hi*lo, A_lo x B_hi adds lo*hi to columns
+    // [0, NB): 2 * HF / 8 instructions.  The caller adds the two halves when it reads its row.
+    auto contract = [&](unsigned ab, auto nb_tag) {
+        constexpr int NB = decltype(nb_tag)::value;
         if (tid == 0) {
             tmem_fence_after_sync();
 #pragma unroll
-            for (int ks = 0; ks < HF / 8; ++ks) {
-                const unsigned long long ah = tc_desc<HF>(aA + ks * 256), al = tc_desc<HF>(aA + TA * 4 + ks * 256);
-                const unsigned long long bh = tc_desc<HF>(ab + ks * 256), bl = tc_desc<HF>(ab + tb + ks * 256);
-                tc_mma_tf32(tbase, ah, bh, idesc, ks != 0);
-                tc_mma_tf32(tbase, ah, bl, idesc, 1);
-                tc_mma_tf32(tbase, al, bh, idesc, 1);
-            }
+            for (int ks = 0; ks < HF / 8; ++ks)
+                tc_mma_tf32_ts(tbase, tbase + DCOLS + ks * 8, tc_desc<2 * NB>(ab, ks), idesc_n(2 * NB), ks != 0);
+#pragma unroll
+            for (int ks = 0; ks < HF / 8; ++ks)
+                tc_mma_tf32_ts(tbase, tbase + DCOLS + HF + ks * 8, tc_desc<2 * NB>(ab, ks), idesc_n(NB), 1);
             tc_commit(bar);
         }
         const bool ok = mbar_wait(bar, phase);
@@ -308,20 +327,21 @@ __global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
         phase ^= 1u;
         tmem_fence_after_sync();
     };
-    // this thread's activations -> row tid of the A operand, split
+    // this thread's activations -> its lane of the A operand in tensor memory, split
     auto put_acts = [&](const float (&act)[HF]) {
 #pragma unroll
-        for (int kc = 0; kc < HF / 4; ++kc) {
-            float4 hi, lo;
-            hi.x = to_tf32(act[4 * kc]); hi.y = to_tf32(act[4 * kc + 1]); hi.z = to_tf32(act[4 * kc + 2]); hi.w = to_tf32(act[4 * kc + 3]);
-            // the remainder goes in as it is: the tensor cores read its leading tf32 bits (2^-11 of 2^-11 is dropped)
-            lo.x = act[4 * kc] - hi.x; lo.y = act[4 * kc + 1] - hi.y;
-            lo.z = act[4 * kc + 2] - hi.z; lo.w = act[4 * kc + 3] - hi.w;
-            *reinterpret_cast<float4 *>(sA + tc_off<HF>(tid, 4 * kc)) = hi;
-            *reinterpret_cast<float4 *>(sA + TA + tc_off<HF>(tid, 4 * kc)) = lo;
+        for (int c0 = 0; c0 < HF; c0 += 16) {
+            float hi[16], lo[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                hi[i] = to_tf32(act[c0 + i]);
+                lo[i] = act[c0 + i] - hi[i];               // the tensor cores read its leading tf32 bits (2^-11 of 2^-11 is dropped)
+            }
+            TmemIO<16>::st(trow + DCOLS + c0, hi);
+            TmemIO<16>::st(trow + DCOLS + HF + c0, lo);
         }
-        fence_async_smem();                                // generic-proxy writes visible to the tensor cores
-        tmem_fence_before_sync();                          // (and this thread's tensor-memory reads precede the next product)
+        tmem_wait_st();
+        tmem_fence_before_sync();                          // (this thread's tensor-memory reads and writes precede the next product)
         __syncthreads();
     };
     for (long long tile = blockIdx.x; tile < tiles && !failed; tile += gridDim.x) {
@@ -339,16 +359,17 @@ __global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
         }
         for (int j = 1; j < J; ++j) {
             put_acts(act);
-            contract(aB + (j - 1) * 2 * TB * 4, TB * 4, IDESC_H);
+            contract(aB + (j - 1) * TB, std::integral_constant<int, HF>{});
             if (failed) break;
 #pragma unroll
             for (int c0 = 0; c0 < HF; c0 += 16) {
-                float acc[16];
+                float acc[16], acl[16];
                 TmemIO<16>::ld(acc, trow + c0);
+                TmemIO<16>::ld(acl, trow + HF + c0);
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                    act[c0 + i] = fmaf(sFi[(j * 2) * HF + c0 + i], sin_reduced(acc[i] + sBh[(j - 1) * HF + c0 + i]), sFi[(j * 2 + 1) * HF + c0 + i]);
+                    act[c0 + i] = fmaf(sFi[(j * 2) * HF + c0 + i], sin_reduced((acc[i] + acl[i]) + sBh[(j - 1) * HF + c0 + i]), sFi[(j * 2 + 1) * HF + c0 + i]);
             }
         }
         if (failed) break;
@@ -357,12 +378,12 @@ __global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
             const int nc = p.C - c0 < kTcChan ? p.C - c0 : kTcChan;
             // output weights of this chunk (one chunk: staged once per CTA; more: once per tile and chunk)
             if (tile == (long long)blockIdx.x || p.C > kTcChan) {
-                for (int e = tid; e < TO; e += kTcThreads) {
+                for (int e = tid; e < kTcChan * HF; e += kTcThreads) {
                     const int c = e / HF, k = e % HF;
                     const float w = (c < nc && k < H) ? SYN_LD(p.Wout, (long long)(c0 + c) * H + k) : 0.f;
                     const float hi = to_tf32(w);
-                    sO[tc_off<HF>(c, k)] = hi;
-                    sO[TO + tc_off<HF>(c, k)] = to_tf32(w - hi);
+                    *reinterpret_cast<float *>(sO + tc_off<2 * kTcChan>(c, k)) = hi;
+                    *reinterpret_cast<float *>(sO + tc_off<2 * kTcChan>(kTcChan + c, k)) = w - hi;
                 }
                 for (int c = tid; c < kTcChan; c += kTcThreads) {
                     sBo[c] = c < nc ? SYN_LD(p.bout, c0 + c) : 0.f;
@@ -380,13 +401,16 @@ __global__ void __launch_bounds__(kTcThreads) synth_tc_kernel(SynthArgs p)
                 tmem_fence_before_sync();
                 __syncthreads();
             }
-            contract(aO, TO * 4, IDESC_O);
+            contract(aO, std::integral_constant<int, kTcChan>{});
             if (failed) break;
 #pragma unroll
             for (int q0 = 0; q0 < kTcChan; q0 += 16) {
-                float acc[16];
+                float acc[16], acl[16];
                 TmemIO<16>::ld(acc, trow + q0);
+                TmemIO<16>::ld(acl, trow + kTcChan + q0);
                 tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] += acl[i];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     const int c = q0 + i;
@@ -437,7 +461,7 @@ template <typename T, int HF> static int launch_synth_tc_t(const SynthArgs &a, c
     if (attr.first()) cudaFuncSetAttribute(synth_tc_kernel<T, HF>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
     // persistent CTAs: as many as fit (shared memory, 512 tensor-memory columns per SM), at most one per tile
     long long per_sm = (220 * 1024) / (long long)(sm + 1024);
-    const long long by_tmem = 512 / (HF > kTcChan ? HF : kTcChan);
+    const long long by_tmem = 512 / (2 * (HF > kTcChan ? HF : kTcChan) + 2 * HF);
     if (per_sm > by_tmem) per_sm = by_tmem;
     if (per_sm > 8) per_sm = 8;
     if (per_sm < 1) per_sm = 1;
