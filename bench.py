@@ -685,7 +685,11 @@ def measure_synth(args, sample_clocks=True):
         "roofline": {"kernel": "synth", "bound": "alu", "achieved": ach, "peak": fp32_tf, "unit": "TFLOP/s", "frac": ach / fp32_tf,
                      "traffic": None, "peak_source": "derived: 2 x 128 FP32 lanes x SMs x max SM clock",
                      "flops": "2 per weight and tap (fused multiply-adds of the three layer kinds); sines and exponentials not counted",
-                     "t_hbm_ms_for_the_output": out_bytes / (hbm_gbs * 1e9) * 1e3},
+                     "t_hbm_ms_for_the_output": out_bytes / (hbm_gbs * 1e9) * 1e3,
+                     "contractions_on": ("tensor cores (tcgen05.mma, tf32 operands split in two, three products: the "
+                                         "fraction is the equivalent FP32 rate against the ALU peak)")
+                                        if 16 < Hf <= 64 and not os.environ.get("HYENAND_SYNTH_ALU") else "FP32 ALUs"},
+        "synth_device_status": hn.hyenand_synth_device_status(),
         "clocks": clocks}
 
 

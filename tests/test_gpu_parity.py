@@ -78,6 +78,30 @@ def test_fused_2d_path(dims, dtype, shared):
     check(w, q, k, v, h)
 
 
+def _seeded_fused_shapes():
+    """Eight seeded shapes inside the domains of the plane-fused 3-D and the fused 2-D kernels (both inner padded axes
+    equal: extents in (P/4, P/2]), with seeded batch, channel, dtype and filter-sharing choices."""
+    g = np.random.default_rng(20261125)
+    cases = []
+    for i in range(8):
+        P = int(g.choice([128, 256] if i < 5 else [64, 128]))
+        ly, lx = (int(g.integers(P // 4 + 1, P // 2 + 1)) for _ in range(2))
+        dims = (int(g.integers(1, 9)) + 1, ly, lx) if i < 5 else (ly, lx)
+        cases.append((dims, int(g.integers(1, 4)), int(g.integers(1, 4)), ["f32", "bf16"][i % 2], bool(g.integers(0, 2))))
+    return cases
+
+
+@pytest.mark.parametrize("dims,B,C,dtype,shared", _seeded_fused_shapes(), ids=str)
+def test_seeded_shapes_on_the_fused_paths(dims, B, C, dtype, shared):
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem(dims, B=B, C=C, dtype=dtype, h_shared=shared, seed=29)
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    path = hn.hyenand_plan_path(plan.handle)
+    plan.close()
+    assert path == ("planes3d" if len(dims) == 3 else "fused2d")
+    check(w, q, k, v, h)
+
+
 TMA_CORE_SHAPES = [(70, 40, 50), (128, 33, 64), (65, 64, 64), (100, 65, 70)]
 
 
