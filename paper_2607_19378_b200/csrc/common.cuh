@@ -258,5 +258,7 @@ int launch_axis(const AxisArgs &a, int mode, cudaStream_t st);
 // warp-engine version of AXIS_CORE (core_w.cu); needs n_in <= P/2, h_n_in <= P, n_out <= P/2
 bool core_w_supported(int log2p);
 int launch_core_w(const AxisArgs &a, cudaStream_t st);
+// warp-engine version of AXIS_FWD / AXIS_INV for 64- to 1024-point axes (core_w.cu); -1 where it does not apply
+int launch_axis_w(const AxisArgs &a, bool inverse, cudaStream_t st);
 
 }  // namespace hn

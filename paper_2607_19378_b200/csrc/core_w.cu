@@ -223,6 +223,114 @@ template <int LOG2P, bool FULL> static int launch_core_w_t(const AxisArgs &a, cu
     return 1;
 }
 
+// ---- one transform along a strided axis (the middle axis of 3-D grids on the general path) ------------------------
+// Same tiles and lane groups as the core above, one transform per line: forward (PRUNE: the upper half of the padded
+// input is zero) from n_in entries, placed at (m - shift) mod N, to n_out <= N bins; or inverse from n_in <= N bins to
+// n_out entries (PRUNE: only the lower half is produced, n_out <= N/2).  Lines are read from `in` and written to `out`
+// (different buffers, their own outer strides).
+template <int LOG2P, bool INV, bool PRUNE>
+__global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) axis_w_kernel(AxisArgs p)
+{
+    constexpr int kCoreThreads = core_threads(LOG2P);
+    using F = WF<LOG2P, INV>;
+    constexpr int N = 1 << LOG2P, TPL = F::TPL;
+    constexpr int TX = kCoreThreads / TPL;
+    constexpr int LS = core_ls<LOG2P>();
+    extern __shared__ float2 smem[];
+    float2 *bu = smem;
+    float2 *twt = smem + TX * LS;
+    const int tid = threadIdx.x, l = tid % TPL, gid = tid / TPL;
+    const unsigned m = F::group_mask(tid);
+    float2 *line = bu + gid * LS;
+    for (int t = tid; t < N; t += kCoreThreads) { HN_G(p.gtw + t * (p.gtw_n / N), 8); twt[t] = p.gtw[t * (p.gtw_n / N)]; }
+    __syncthreads();
+    PlaneTw<LOG2P, INV> tw;
+    tw.init(l, twt, twt + N, tid, kCoreThreads);
+    __syncthreads();
+    const long long tpo = (p.nc + TX - 1) / TX;
+    const long long tiles = p.n_outer * tpo;
+    constexpr int RPS = kCoreThreads / TX;                 // rows per step
+    const int x = tid % TX, r0 = tid / TX;
+    const unsigned bu_x = (unsigned)__cvta_generic_to_shared(bu + x * LS);
+    constexpr int NFILL = (!INV && PRUNE) ? N / 2 : N;     // positions the first pass reads
+    for (long long t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const long long o = t / tpo;
+        const int c0 = (int)(t % tpo) * TX;
+        const bool inside = c0 + x < p.nc;
+        const float2 *us = p.in + o * p.in_outer + c0 + x;
+        const long long step = (long long)RPS * p.nc;
+        if (inside) {
+            // position pos holds entry (pos + shift) mod N: entries [shift, n_in) sit at [0, n_in - shift), entries
+            // [0, shift) at [N - shift, N), the gap is zero
+            const int head = p.n_in - p.shift, tail0 = N - p.shift;
+            const float2 *src = us + (long long)(p.shift + r0) * p.nc;
+            for (int pos = r0; pos < head && pos < NFILL; pos += RPS, src += step) cp_async8_s(bu_x + 8u * (unsigned)F::ph(pos), src);
+            if (p.shift) {
+                int pos = tail0 + ((r0 - tail0) & (RPS - 1));
+                src = us + (long long)(pos - tail0) * p.nc;
+                for (; pos < NFILL; pos += RPS, src += step) cp_async8_s(bu_x + 8u * (unsigned)F::ph(pos), src);
+            }
+            const int z1 = p.shift ? tail0 : N;
+            for (int z = (head > 0 ? head : 0) + ((r0 - (head > 0 ? head : 0)) & (RPS - 1)); z < z1 && z < NFILL; z += RPS)
+                bu[x * LS + F::ph(z)] = make_float2(0.f, 0.f);
+        } else {
+            for (int pos = r0; pos < NFILL; pos += RPS) bu[x * LS + F::ph(pos)] = make_float2(0.f, 0.f);
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        constexpr int PR = PRUNE ? (INV ? PRUNE_OUT : PRUNE_IN) : PRUNE_NONE;
+        F::template run_to_line<PR, true>(l, m, tw, line, [&](int, int, int idx) { return line[F::ph(idx)]; });
+        __syncthreads();
+        if (inside) {
+            float2 *dst = p.out + o * p.out_outer + c0 + x + (long long)r0 * p.nc;
+            for (int pos = r0; pos < p.n_out; pos += RPS, dst += step) { HN_G(dst, 8); *dst = bu[x * LS + F::ph(pos)]; }
+        }
+        __syncthreads();
+    }
+}
+
+template <int LOG2P, bool INV, bool PRUNE> static int launch_axis_w_t(const AxisArgs &a, cudaStream_t st)
+{
+    using F = WF<LOG2P, INV>;
+    constexpr int kCoreThreads = core_threads(LOG2P);
+    constexpr int N = 1 << LOG2P, TX = kCoreThreads / F::TPL;
+    const size_t sm = sizeof(float2) * ((size_t)TX * core_ls<LOG2P>() + N + PlaneTw<LOG2P, INV>::TABLE);
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms <= 0) sms = 148;
+    }
+    static DevOnce attr;
+    if (attr.first()) cudaFuncSetAttribute(axis_w_kernel<LOG2P, INV, PRUNE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    const long long tiles = a.n_outer * ((a.nc + TX - 1) / TX);
+    const long long res = (long long)sms * (LOG2P >= 10 ? 1 : 4);
+    const int grid = (int)(tiles < res ? tiles : res);
+    if (grid <= 0) return 0;
+    axis_w_kernel<LOG2P, INV, PRUNE><<<grid, kCoreThreads, sm, st>>>(a);
+    return 1;
+}
+
+// forward: a.prune_in selects the pruned first pass; inverse: a.full keeps every output, else the lower half
+int launch_axis_w(const AxisArgs &a, bool inverse, cudaStream_t st)
+{
+    const int n = 1 << a.log2p;
+    if (a.in == a.out) return -1;
+    if (!inverse && (a.n_in > (a.prune_in ? n / 2 : n) || a.n_out > n || a.shift < 0 || a.shift >= n || (a.prune_in && a.shift))) return -1;
+    if (inverse && (a.n_in > n || a.shift || a.n_out > (a.full ? n : n / 2))) return -1;
+#define HN_AXW(L)                                                                                       \
+    case L:                                                                                             \
+        if (!inverse) return a.prune_in ? launch_axis_w_t<L, false, true>(a, st) : launch_axis_w_t<L, false, false>(a, st); \
+        return a.full ? launch_axis_w_t<L, true, false>(a, st) : launch_axis_w_t<L, true, true>(a, st);
+    switch (a.log2p) {
+        HN_AXW(6) HN_AXW(7) HN_AXW(8) HN_AXW(9) HN_AXW(10)
+    default: return -1;
+    }
+#undef HN_AXW
+}
+
 bool core_w_supported(int log2p) { return log2p >= 6 && log2p <= 10; }
 
 int launch_core_w(const AxisArgs &a, cudaStream_t st)

@@ -499,6 +499,16 @@ static int lanes_join(hyenand_plan *p, cudaStream_t st)
     return 0;
 }
 
+// one transform along the middle axis: warp-engine kernel where it applies, else the block-wide one
+static int launch_axis_any(const Switches &sw, const AxisArgs &a, int mode, cudaStream_t st)
+{
+    if (core_w_supported(a.log2p) && !sw.generic_core) {
+        const int c = launch_axis_w(a, mode == AXIS_INV, st);
+        if (c >= 0) return c;
+    }
+    return launch_axis(a, mode, st);
+}
+
 static int filter_spectrum_generic(hyenand_plan *p, int l, const char *h, long long n_slices, cudaStream_t st, int *launches)
 {
     hyenand_plan::Lane &ln = p->lane[l];
@@ -528,7 +538,7 @@ static int filter_spectrum_generic(hyenand_plan *p, int l, const char *h, long l
         a.shift = p->circular ? 0 : p->L[1] - 1; a.log2p = p->log2p[1]; a.prune_in = 0;
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         p->prof.begin(KID_AXIS_H, st);
-        n = launch_axis(a, AXIS_FWD, st);
+        n = launch_axis_any(p->sw, a, AXIS_FWD, st);
         p->prof.end(st);
         if (n < 0) return -1;
         *launches += n;
@@ -608,7 +618,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2 && !p->circular;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
             p->prof.begin(KID_AXIS_U, st);
-            c = launch_axis(a, AXIS_FWD, st);
+            c = launch_axis_any(p->sw, a, AXIS_FWD, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
@@ -630,7 +640,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             a.log2p = p->log2p[1]; a.prune_in = 0; a.full = p->circular;
             a.gtw = p->gtw; a.gtw_n = p->gtw_n;
             p->prof.begin(KID_AXIS_INV, st);
-            c = launch_axis(a, AXIS_INV, st);
+            c = launch_axis_any(p->sw, a, AXIS_INV, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
@@ -1350,7 +1360,7 @@ static int corr_dh(hyenand_grad *g, long long m, const float *gy, const float *g
         a.nc = XP; a.n_in = L[1]; a.n_out = P[1]; a.shift = 0;
         a.log2p = p->log2p[1]; a.prune_in = P[1] >= 2;
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
-        return launch_axis(a, AXIS_FWD, st);
+        return launch_axis_any(p->sw, a, AXIS_FWD, st);
     };
     if ((c = rows(gy, gq, g->cga)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
     if ((c = rows(ur, nullptr, g->cua)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
@@ -1383,7 +1393,7 @@ static int corr_dh(hyenand_grad *g, long long m, const float *gy, const float *g
         a.nc = XP; a.n_in = P[1]; a.n_out = K1; a.shift = 0;
         a.log2p = p->log2p[1]; a.prune_in = 0; a.full = 1;
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
-        if ((c = launch_axis(a, AXIS_INV, st)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+        if ((c = launch_axis_any(p->sw, a, AXIS_INV, st)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
     }
     {
         RowsInvArgs ri{};

@@ -78,6 +78,21 @@ def test_fused_2d_path(dims, dtype, shared):
     check(w, q, k, v, h)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shared", [False, True])
+@pytest.mark.parametrize("dims", [(6, 40, 20), (3, 100, 300), (2, 300, 40), (5, 17, 33)], ids=str)
+def test_general_3d_path_with_a_long_middle_axis(dims, dtype, shared):
+    """3-D grids whose inner padded axes differ run on the general path; a middle axis padded to 64 .. 1024 points
+    takes the warp-engine axis kernel (forward with the filter's wrapped placement, pruned forward, cropped inverse)."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem(dims, B=2, C=2, dtype=dtype, h_shared=shared, seed=31)
+    plan = hn.Plan(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    path = hn.hyenand_plan_path(plan.handle)
+    plan.close()
+    assert path == "nd_generic"
+    check(w, q, k, v, h)
+
+
 def _seeded_fused_shapes():
     """Eight seeded shapes inside the domains of the plane-fused 3-D and the fused 2-D kernels (both inner padded axes
     equal: extents in (P/4, P/2]), with seeded batch, channel, dtype and filter-sharing choices."""
