@@ -415,7 +415,42 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
 
 // ---- inverse planes ------------------------------------------------------------------------------------
 
-template <typename T, int LOG2P>
+// 16 bytes of gate values or results: VEC elements of T
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+    static constexpr int VEC = 4;
+    static __device__ __forceinline__ void unpack(const uint4 &u, float (&f)[4])
+    {
+        f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[4])
+    {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+    }
+};
+template <> struct Vec16<bf16> {
+    static constexpr int VEC = 8;
+    static __device__ __forceinline__ void unpack(const uint4 &u, float (&f)[8])
+    {
+        const unsigned w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[8])
+    {
+        unsigned w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+            w[i] = *reinterpret_cast<const unsigned *>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// VST: rows are whole numbers of 16-byte vectors and q, y are 16-byte aligned: the cropped rows go through the line
+// once more and leave as 16-byte stores (gate values arrive as 16-byte loads); else one element per lane and leg.
+template <typename T, int LOG2P, bool VST>
 __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p)
 {
     using C = PlaneCfg<LOG2P>;
@@ -500,12 +535,24 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
         using PE = typename FI::LastPass;
         constexpr int NQ = PE::IPL * (PE::R / 2);
         constexpr int RIT = QP > C::NG ? QP / C::NG : 1;      // row pairs per lane group
-        T q0[RIT][NQ], q1[RIT][NQ];
+        constexpr int VEC = Vec16<T>::VEC, NV = (HP / VEC + TPL - 1) / TPL;      // vectors per row and lane
+        T q0[VST ? 1 : RIT][VST ? 1 : NQ], q1[VST ? 1 : RIT][VST ? 1 : NQ];
+        uint4 qv0[VST ? RIT : 1][VST ? NV : 1], qv1[VST ? RIT : 1][VST ? NV : 1];
 #pragma unroll
         for (int it = 0; it < RIT; ++it) {
             const int rp = gid + it * C::NG, y1 = rp + QP;
             const bool has0 = rp < QP, has1 = has0 && y1 < Ly;
             const long long o0 = ob + (long long)rp * Lx, o1 = ob + (long long)y1 * Lx;
+            if constexpr (VST) {
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    const int x0 = (l + j * TPL) * VEC;
+                    qv0[it][j] = qv1[it][j] = make_uint4(0u, 0u, 0u, 0u);
+                    if (x0 < Lx && has0) { HN_G(pq + o0 + x0, 16); qv0[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o0 + x0)); }
+                    if (x0 < Lx && has1) { HN_G(pq + o1 + x0, 16); qv1[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o1 + x0)); }
+                }
+                continue;
+            }
 #pragma unroll
             for (int i = 0; i < PE::IPL; ++i)
 #pragma unroll
@@ -533,8 +580,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
             static_assert(P0::IPL == 1, "lane 0 holds bins 0 and P/2 of a row");
             const float2 *g = cs + l * CSI + rp;
             float2 nyq = make_float2(0.f, 0.f);
-            FI::template run<PRUNE_OUT>(l, m, twp, line,
-                [&](int, int r, int) {
+            auto spectrum = [&](int, int r, int) {
                     float2 v = g[r * (P / P0::R) * CSI];
                     if (r == 0 && l == 0) {
                         // bins 0 and P/2 hold A + iB and conj A + i conj B of the packed column, A = (X_0[y], X_{P/2}[y]):
@@ -545,13 +591,37 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
                     }
                     if (r == P0::R / 2 && l == 0) v = nyq;
                     return v;
-                },
-                [&](int i, int r, int idx, float2 v) {
-                    if (idx < Lx) {
-                        IO<T>::st(py, o0 + idx, v.x * (float)q0[it][i * (PE::R / 2) + r]);
-                        if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[it][i * (PE::R / 2) + r]);
+                };
+            if constexpr (VST) {
+                // results to the line in natural order; a lane then takes VEC neighbouring outputs of both rows
+                FI::template run_to_line<PRUNE_OUT>(l, m, twp, line, spectrum);
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    const int x0 = (l + j * TPL) * VEC;
+                    if (x0 < Lx) {
+                        float a[VEC], b[VEC], ga[VEC], gb[VEC];
+                        Vec16<T>::unpack(qv0[it][j], ga);
+                        Vec16<T>::unpack(qv1[it][j], gb);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) {
+                            const float2 z = line[FI::ph(x0 + e)];
+                            a[e] = z.x * ga[e];
+                            b[e] = z.y * gb[e];
+                        }
+                        HN_G(py + o0 + x0, 16);
+                        *reinterpret_cast<uint4 *>(py + o0 + x0) = Vec16<T>::pack(a);
+                        if (has1) { HN_G(py + o1 + x0, 16); *reinterpret_cast<uint4 *>(py + o1 + x0) = Vec16<T>::pack(b); }
                     }
-                });
+                }
+            } else {
+                FI::template run<PRUNE_OUT>(l, m, twp, line, spectrum,
+                    [&](int i, int r, int idx, float2 v) {
+                        if (idx < Lx) {
+                            IO<T>::st(py, o0 + idx, v.x * (float)q0[it][i * (PE::R / 2) + r]);
+                            if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[it][i * (PE::R / 2) + r]);
+                        }
+                    });
+            }
             __syncwarp(m);
         }
         __syncthreads();
@@ -583,9 +653,13 @@ template <typename T, int LOG2P> static int launch_plane_t(const PlaneArgs &a, i
     using C = PlaneCfg<LOG2P>;
     const int grid = plane_grid(a.planes);
     if (grid <= 0) return 0;
-    static DevOnce attr[3];
+    static DevOnce attr[4];
+    // 16-byte gate loads and result stores where every row is a whole number of vectors on a 16-byte boundary
+    const bool vst = which == PLANE_INV && a.lx % Vec16<T>::VEC == 0 && (((uintptr_t)a.a | (uintptr_t)a.y) & 15) == 0;
     void (*fn)(PlaneArgs) = which == PLANE_U ? uplane_kernel<T, LOG2P>
-                          : which == PLANE_H ? hplane_kernel<T, LOG2P> : plane_inv_kernel<T, LOG2P>;
+                          : which == PLANE_H ? hplane_kernel<T, LOG2P>
+                          : vst ? plane_inv_kernel<T, LOG2P, true> : plane_inv_kernel<T, LOG2P, false>;
+    if (vst) which = 3;
     if (attr[which].first()) {
         cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
     }
