@@ -42,7 +42,9 @@ template <int LOG2P> struct F2Cfg {
 //   phase 2  one group per column kx = 0 .. P/2 (the extra warp takes the last one); columns 0 and P/2 hold
 //            real data and run as general complex transforms, which keeps all groups on one code path
 // so every phase keeps all groups busy; the k*v store is double buffered.
-template <typename T, int LOG2P>
+// VST: rows are whole numbers of 16-byte vectors and q, y are 16-byte aligned: gate values arrive as 16-byte loads, the
+// cropped rows go through the line once more and leave as 16-byte stores; else one element per lane and leg.
+template <typename T, int LOG2P, bool VST>
 __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)     // 96 registers: one scheduler hosts 5 of the 17 warps
 {
     using C = F2Cfg<LOG2P>;
@@ -90,26 +92,57 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)  
             const long long o0 = sp * vol + (long long)rp * Lx, o1 = sp * vol + (long long)y1 * Lx;
             // the gate values of this lane's outputs are requested before the transform starts
             constexpr int NQ = PIL::IPL * (PIL::R / 2);
-            T q0[NQ], q1[NQ];
-#pragma unroll
-            for (int i = 0; i < PIL::IPL; ++i)
-#pragma unroll
-                for (int r = 0; r < PIL::R / 2; ++r) {
-                    const int idx = FI::last_pos(l, i, r);
-                    if (idx < Lx) HN_G(pq + o0 + idx, ES);
-                    if (idx < Lx && has1) HN_G(pq + o1 + idx, ES);
-                    q0[i * (PIL::R / 2) + r] = idx < Lx ? __ldg(pq + o0 + idx) : T(0.f);
-                    q1[i * (PIL::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
-                }
+            constexpr int VEC = Vec16<T>::VEC, NV = (HP / VEC + TPL - 1) / TPL;       // vectors per row and lane
             const float2 *g = ub + l * UCS + rp;
-            FI::template run<PRUNE_OUT>(l, m, twi, line,
-                [&](int i, int r, int) { return g[(i * TPL + r * (P / PI0::R)) * UCS]; },
-                [&](int i, int r, int idx, float2 v) {
-                    if (idx < Lx) {
-                        IO<T>::st(py, o0 + idx, v.x * (float)q0[i * (PIL::R / 2) + r]);
-                        if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[i * (PIL::R / 2) + r]);
+            auto spectrum = [&](int i, int r, int) { return g[(i * TPL + r * (P / PI0::R)) * UCS]; };
+            if constexpr (VST) {
+                uint4 qv0[NV], qv1[NV];
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    const int x0 = (l + j * TPL) * VEC;
+                    qv0[j] = qv1[j] = make_uint4(0u, 0u, 0u, 0u);
+                    if (x0 < Lx) { HN_G(pq + o0 + x0, 16); qv0[j] = __ldg(reinterpret_cast<const uint4 *>(pq + o0 + x0)); }
+                    if (x0 < Lx && has1) { HN_G(pq + o1 + x0, 16); qv1[j] = __ldg(reinterpret_cast<const uint4 *>(pq + o1 + x0)); }
+                }
+                FI::template run_to_line<PRUNE_OUT>(l, m, twi, line, spectrum);
+#pragma unroll
+                for (int j = 0; j < NV; ++j) {
+                    const int x0 = (l + j * TPL) * VEC;
+                    if (x0 < Lx) {
+                        float a[VEC], b[VEC], ga[VEC], gb[VEC];
+                        Vec16<T>::unpack(qv0[j], ga);
+                        Vec16<T>::unpack(qv1[j], gb);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) {
+                            const float2 z = line[FI::ph(x0 + e)];
+                            a[e] = z.x * ga[e];
+                            b[e] = z.y * gb[e];
+                        }
+                        HN_G(py + o0 + x0, 16);
+                        *reinterpret_cast<uint4 *>(py + o0 + x0) = Vec16<T>::pack(a);
+                        if (has1) { HN_G(py + o1 + x0, 16); *reinterpret_cast<uint4 *>(py + o1 + x0) = Vec16<T>::pack(b); }
                     }
-                });
+                }
+            } else {
+                T q0[NQ], q1[NQ];
+#pragma unroll
+                for (int i = 0; i < PIL::IPL; ++i)
+#pragma unroll
+                    for (int r = 0; r < PIL::R / 2; ++r) {
+                        const int idx = FI::last_pos(l, i, r);
+                        if (idx < Lx) HN_G(pq + o0 + idx, ES);
+                        if (idx < Lx && has1) HN_G(pq + o1 + idx, ES);
+                        q0[i * (PIL::R / 2) + r] = idx < Lx ? __ldg(pq + o0 + idx) : T(0.f);
+                        q1[i * (PIL::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
+                    }
+                FI::template run<PRUNE_OUT>(l, m, twi, line, spectrum,
+                    [&](int i, int r, int idx, float2 v) {
+                        if (idx < Lx) {
+                            IO<T>::st(py, o0 + idx, v.x * (float)q0[i * (PIL::R / 2) + r]);
+                            if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[i * (PIL::R / 2) + r]);
+                        }
+                    });
+            }
             __syncwarp(m);
         }
     };
@@ -287,11 +320,14 @@ template <typename T, int LOG2P> static int launch_fused2d_t(const Fused2dArgs &
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms <= 0) sms = 148;
     }
-    static DevOnce attr;
-    if (attr.first()) cudaFuncSetAttribute(fused2d_kernel<T, LOG2P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+    // 16-byte gate loads and result stores where every row is a whole number of vectors on a 16-byte boundary
+    const bool vst = a.lx % Vec16<T>::VEC == 0 && (((uintptr_t)a.q | (uintptr_t)a.y) & 15) == 0;
+    static DevOnce attr[2];
+    void (*fn)(Fused2dArgs) = vst ? fused2d_kernel<T, LOG2P, true> : fused2d_kernel<T, LOG2P, false>;
+    if (attr[vst ? 1 : 0].first()) cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
     const int grid = (int)(a.slices < sms ? a.slices : sms);
     if (grid <= 0) return 0;
-    fused2d_kernel<T, LOG2P><<<grid, kF2Threads, C::SMEM, st>>>(a);
+    fn<<<grid, kF2Threads, C::SMEM, st>>>(a);
     return 1;
 }
 

@@ -415,39 +415,6 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
 
 // ---- inverse planes ------------------------------------------------------------------------------------
 
-// 16 bytes of gate values or results: VEC elements of T
-template <typename T> struct Vec16;
-template <> struct Vec16<float> {
-    static constexpr int VEC = 4;
-    static __device__ __forceinline__ void unpack(const uint4 &u, float (&f)[4])
-    {
-        f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&f)[4])
-    {
-        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
-    }
-};
-template <> struct Vec16<bf16> {
-    static constexpr int VEC = 8;
-    static __device__ __forceinline__ void unpack(const uint4 &u, float (&f)[8])
-    {
-        const unsigned w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&f)[8])
-    {
-        unsigned w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-            w[i] = *reinterpret_cast<const unsigned *>(&h);
-        }
-        return make_uint4(w[0], w[1], w[2], w[3]);
-    }
-};
-
 // VST: rows are whole numbers of 16-byte vectors and q, y are 16-byte aligned: the cropped rows go through the line
 // once more and leave as 16-byte stores (gate values arrive as 16-byte loads); else one element per lane and leg.
 template <typename T, int LOG2P, bool VST>
