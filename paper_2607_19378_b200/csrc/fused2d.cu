@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)  
             float2 *ua = ucs + kx * UCS, *um = ucs + km * UCS;
             float2 H[PL::IPL][PL::R];
             {
-                float2 second[PF0::IPL][PF0::R / 2];          // rows y + P/2, formed with their partners y
+                float2 second[PF0::IPL][PF0::R / 2] = {};     // rows y + P/2, formed with their partners y
                 F::template run<PRUNE_NONE>(l, m, twf, line,
                     [&](int i, int r, int idx) {
                         if (r >= PF0::R / 2) return second[i][r - PF0::R / 2];
@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)  
             __syncwarp(m);
             float2 Y[PL::IPL][PL::R];
             {
-                float2 second[PF0::IPL][PF0::R / 4];          // rows y + P/4 (the upper half of the column is padding)
+                float2 second[PF0::IPL][PF0::R / 4] = {};     // rows y + P/4 (the upper half of the column is padding)
                 F::template run<PRUNE_IN>(l, m, twf, line,
                     [&](int i, int r, int idx) {
                         if (r >= PF0::R / 4) return second[i][r - PF0::R / 4];

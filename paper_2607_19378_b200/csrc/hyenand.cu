@@ -267,7 +267,6 @@ extern "C" hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int
     }
     p->XH = p->P[2] / 2 + 1;
     p->XP = (p->XH + 1) & ~1;
-    const long long S = (long long)B * C;
     if (circular) {
         // periodic boundaries run on the general N-D passes, which transform whole lines here (nothing is
         // padded, so there is no zero half to prune and no half to crop); no plane, fused or tensor-copy kernels
@@ -1541,7 +1540,7 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
     const size_t es = elsize(g->dtype);
     const bool widen = g->dtype == HYENAND_BF16;
     const long long C = g->C, vol = g->vol, kvol = g->kvol;
-    const int *L = g->L, *K = g->K, *P = g->P;
+    const int *L = g->L, *K = g->K;
     const bool nat = widen && g->h_native;                     // bf16 taps go to the transforms as they are
     const int hdt = nat ? HYENAND_BF16 : HYENAND_F32;
     const float *hsh = (const float *)h;                       // shared kernel, fp32 view

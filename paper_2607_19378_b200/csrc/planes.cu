@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) uplane_kernel(PlaneArgs p)
             const bool packed = kx == 0;
             const float2 *ca = cs + kx * CSU, *cb = cs + (packed ? HP : P - kx) * CSU;
             float2 *d = packed ? tmp : dst + (long long)kx * P;
-            float2 second[PC0::IPL][PC0::R / 4];
+            float2 second[PC0::IPL][PC0::R / 4] = {};
             F::template run<PRUNE_IN>(l, FULL, twp, line,
                 [&](int i, int r, int idx) {
                     if (r >= PC0::R / 4) return second[i][r - PC0::R / 4];
@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
                 const int km = packed ? HP / 2 : (e == 0 ? ((HP - k) & (HP - 1)) : HP - 1 - k);
                 const float2 *ca = cs + k * CS2, *cb = cs + km * CS2;
                 float2 *d = packed ? tmp : dst + (long long)(2 * k + e) * P;
-                float2 second[PC0::IPL][PC0::R / 2];          // inputs y + P/2, formed with their partners y
+                float2 second[PC0::IPL][PC0::R / 2] = {};     // inputs y + P/2, formed with their partners y
                 F::template run<PRUNE_NONE>(l, FULL, twp, line,
                     [&](int i, int r, int idx) {
                         if (r >= PC0::R / 2) return second[i][r - PC0::R / 2];
@@ -518,18 +518,18 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
                     if (x0 < Lx && has0) { HN_G(pq + o0 + x0, 16); qv0[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o0 + x0)); }
                     if (x0 < Lx && has1) { HN_G(pq + o1 + x0, 16); qv1[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o1 + x0)); }
                 }
-                continue;
+            } else {
+#pragma unroll
+                for (int i = 0; i < PE::IPL; ++i)
+#pragma unroll
+                    for (int r = 0; r < PE::R / 2; ++r) {
+                        const int idx = FI::last_pos(l, i, r);
+                        if (idx < Lx && has0) HN_G(pq + o0 + idx, sizeof(T));
+                        if (idx < Lx && has1) HN_G(pq + o1 + idx, sizeof(T));
+                        q0[it][i * (PE::R / 2) + r] = (idx < Lx && has0) ? __ldg(pq + o0 + idx) : T(0.f);
+                        q1[it][i * (PE::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
+                    }
             }
-#pragma unroll
-            for (int i = 0; i < PE::IPL; ++i)
-#pragma unroll
-                for (int r = 0; r < PE::R / 2; ++r) {
-                    const int idx = FI::last_pos(l, i, r);
-                    if (idx < Lx && has0) HN_G(pq + o0 + idx, sizeof(T));
-                    if (idx < Lx && has1) HN_G(pq + o1 + idx, sizeof(T));
-                    q0[it][i * (PE::R / 2) + r] = (idx < Lx && has0) ? __ldg(pq + o0 + idx) : T(0.f);
-                    q1[it][i * (PE::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
-                }
         }
         __syncthreads();
         if (pl + gridDim.x < p.planes) {
