@@ -242,6 +242,8 @@ struct AxisArgs {
     const float2 *gtw;
     int gtw_n;
     int full;                 // 1: circular mode (n_in == n_out == P): no pruned input half, all outputs kept
+    int h_conj;               // core only, 1: the product takes the conjugate of the filter spectrum (the kernel read at the
+                              // opposite displacement, h'[d] = h[-d]: the filter of the backward pass's input gradient)
 };
 
 enum AxisMode { AXIS_FWD = 0, AXIS_INV = 1, AXIS_CORE = 2 };

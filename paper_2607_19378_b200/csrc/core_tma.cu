@@ -66,6 +66,7 @@ struct CoreTmaParams {
     int h_shift;              // filter row (pos + h_shift) mod N sits at position pos
     long long h_mod, h_off;   // filter outer index = h_mod ? (o + h_off) % h_mod : o
     float scale;
+    float scale_im;           // scale, or -scale where the product takes the conjugate of the filter spectrum
     const float2 *gtw;
     int gtw_n;
     int *status;              // device word: 0 ok, else which wait gave up
@@ -172,7 +173,7 @@ axis_core_tma_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
         }
         F::template pass<NP - 1, PRUNE_NONE>(l, tw,
             [&](int, int, int idx) { return line[F::ph(idx)]; },
-            [&](int, int r, int, float2 v) { H[r] = make_float2(v.x * p.scale, v.y * p.scale); });
+            [&](int, int r, int, float2 v) { H[r] = make_float2(v.x * p.scale, v.y * p.scale_im); });
         __syncwarp(m);
         // ---- k*v lines: tile -> spectrum, product, inverse ----------------------------------------
         if (!mbar_wait(bar_u, phase)) failed = 2;
@@ -295,7 +296,7 @@ int launch_core_tma(const AxisArgs &a, const CoreTmaMaps &m, int *status, cudaSt
     CoreTmaParams p{};
     p.n_outer = a.n_outer;
     p.h_shift = a.h_shift; p.h_mod = a.h_mod; p.h_off = a.h_off;
-    p.scale = a.scale; p.gtw = a.gtw; p.gtw_n = a.gtw_n; p.status = status;
+    p.scale = a.scale; p.scale_im = a.h_conj ? -a.scale : a.scale; p.gtw = a.gtw; p.gtw_n = a.gtw_n; p.status = status;
     return a.log2p == 8 ? launch_core_tma_t<8>(p, m, a.nc, st) : launch_core_tma_t<10>(p, m, a.nc, st);
 }
 

@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
             F::template mid<0, NP - 1, PRUNE_NONE>(l, m, tw, hline);
             F::template pass<NP - 1, PRUNE_NONE>(l, tw,
                 [&](int, int, int idx) { return hline[F::ph(idx)]; },
-                [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * p.scale); });
+                [&](int i, int r, int, float2 v) { H[i][r] = make_float2(v.x * p.scale, v.y * (p.h_conj ? -p.scale : p.scale)); });
             __syncthreads();                               // filter lines are free again
             if (tn < tiles) issue_h(tn);
             cp_async_commit();
@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(core_threads(LOG2P), (LOG2P >= 10 ? 1 : 2)) ax
                     if constexpr (HREG) Y[i][r] = cmul(v, H[i][r]);
                     else {
                         const float2 hh = hline[F::ph(idx)];
-                        Y[i][r] = cmul(v, make_float2(hh.x * p.scale, hh.y * p.scale));
+                        Y[i][r] = cmul(v, make_float2(hh.x * p.scale, hh.y * (p.h_conj ? -p.scale : p.scale)));
                     }
                 });
             __syncwarp(m);

@@ -159,6 +159,11 @@ struct hyenand_plan {
     void *stage[5];
     size_t stage_bytes[5];
     int h_dtype;                      // element type of the filter taps (differs from dtype only inside the mixer)
+    // Second signal side of the multi-kernel paths (backward pass): after y = q (h conv (k v)) every group also
+    // computes y2 = q2 (h' conv (k2 v2)) with h'[d] = h[-d], whose spectrum is the conjugate of the filter spectrum
+    // the group has just computed.  Unused (nullptr) in an ordinary forward.
+    const char *q2, *k2, *v2;
+    char *y2;
     size_t ws_bytes;
     Prof prof;
 };
@@ -210,9 +215,9 @@ extern "C" void hyenand_destroy_plan(hyenand_plan *p)
     delete p;
 }
 
-static AxisArgs planes3d_core_args(const hyenand_plan *p, int lane, long long n, bool shared, long long s0);
+static AxisArgs planes3d_core_args(const hyenand_plan *p, int lane, long long n, bool shared, long long s0, bool conj = false);
 static void make_core_maps(hyenand_plan *p);
-static AxisArgs generic_core_args(const hyenand_plan *p, int lane, long long n, bool shared, long long s0);
+static AxisArgs generic_core_args(const hyenand_plan *p, int lane, long long n, bool shared, long long s0, bool conj = false);
 static void choose_groups(hyenand_plan *p, long long per_slice_elems);
 
 extern "C" hyenand_plan *hyenand_create_plan(int ndim, const int *dims, int B, int C, int causal, int dtype)
@@ -547,7 +552,7 @@ static int filter_spectrum_generic(hyenand_plan *p, int l, const char *h, long l
 
 // arguments of the fused core (last transformed axis) of the generic path for n slices starting at slice s0,
 // in the workspace of lane l (a filter shared over the batch sits in lane 0's filter workspace)
-static AxisArgs generic_core_args(const hyenand_plan *p, int l, long long n, bool shared, long long s0)
+static AxisArgs generic_core_args(const hyenand_plan *p, int l, long long n, bool shared, long long s0, bool conj)
 {
     const hyenand_plan::Lane &ln = p->lane[l], &lh = p->lane[shared ? 0 : l];
     const bool three = p->P[0] > 1;
@@ -567,6 +572,7 @@ static AxisArgs generic_core_args(const hyenand_plan *p, int l, long long n, boo
     a.h_off = shared ? s0 % p->C : 0;
     a.scale = (float)(1.0 / ((double)p->P[0] * p->P[1] * p->P[2]));
     a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+    a.h_conj = conj;
     return a;
 }
 
@@ -598,67 +604,73 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         cudaStream_t st = lane_stream(p, l, st0);
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter_spectrum_generic(p, l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st, launches)) return -1;
-        RowsArgs r{};
-        r.a = k + (size_t)s0 * p->vol * es; r.b = v + (size_t)s0 * p->vol * es; r.out = ln.ws_a; r.pitch = p->XP;
-        r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
-        r.prune_in = 1; r.full_in = p->circular; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
-        p->prof.begin(KID_ROWS_U, st);
-        const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
-        int c = roww ? launch_rows_fwd_w(r, p->dtype, st) : launch_rows_fwd(r, p->dtype, st);
-        p->prof.end(st);
-        if (c < 0) return -1;
-        *launches += c;
-        if (three) {
-            AxisArgs a{};
-            a.in = ln.ws_a; a.out = ln.ws_b;
-            a.n_outer = n * p->L[0];
-            a.in_outer = (long long)p->L[1] * p->XP; a.out_outer = (long long)p->P[1] * p->XP;
-            a.nc = p->XP; a.n_in = p->L[1]; a.n_out = p->P[1]; a.shift = 0;
-            a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2 && !p->circular;
-            a.gtw = p->gtw; a.gtw_n = p->gtw_n;
-            p->prof.begin(KID_AXIS_U, st);
-            c = launch_axis_any(p->sw, a, AXIS_FWD, st);
+        // one signal side: rows, [middle axis], core against the group's filter spectrum (or its conjugate), back
+        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj) -> int {
+            RowsArgs r{};
+            r.a = sk + (size_t)s0 * p->vol * es; r.b = sv + (size_t)s0 * p->vol * es; r.out = ln.ws_a; r.pitch = p->XP;
+            r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
+            r.prune_in = 1; r.full_in = p->circular; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
+            p->prof.begin(KID_ROWS_U, st);
+            const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
+            int c = roww ? launch_rows_fwd_w(r, p->dtype, st) : launch_rows_fwd(r, p->dtype, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
-        }
-        {
-            const AxisArgs a = generic_core_args(p, l, n, shared, s0);
-            p->prof.begin(KID_CORE, st);
-            c = launch_core_any(p, l, a, shared, st);
+            if (three) {
+                AxisArgs a{};
+                a.in = ln.ws_a; a.out = ln.ws_b;
+                a.n_outer = n * p->L[0];
+                a.in_outer = (long long)p->L[1] * p->XP; a.out_outer = (long long)p->P[1] * p->XP;
+                a.nc = p->XP; a.n_in = p->L[1]; a.n_out = p->P[1]; a.shift = 0;
+                a.log2p = p->log2p[1]; a.prune_in = p->P[1] >= 2 && !p->circular;
+                a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+                p->prof.begin(KID_AXIS_U, st);
+                c = launch_axis_any(p->sw, a, AXIS_FWD, st);
+                p->prof.end(st);
+                if (c < 0) return -1;
+                *launches += c;
+            }
+            {
+                const AxisArgs a = generic_core_args(p, l, n, shared, s0, conj);
+                p->prof.begin(KID_CORE, st);
+                c = launch_core_any(p, l, a, shared, st);
+                p->prof.end(st);
+                if (c < 0) return -1;
+                *launches += c;
+            }
+            if (three) {
+                AxisArgs a{};
+                a.in = ln.ws_b; a.out = ln.ws_a;
+                a.n_outer = n * p->L[0];
+                a.in_outer = (long long)p->P[1] * p->XP; a.out_outer = (long long)p->L[1] * p->XP;
+                a.nc = p->XP; a.n_in = p->P[1]; a.n_out = p->L[1]; a.shift = 0;
+                a.log2p = p->log2p[1]; a.prune_in = 0; a.full = p->circular;
+                a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+                p->prof.begin(KID_AXIS_INV, st);
+                c = launch_axis_any(p->sw, a, AXIS_INV, st);
+                p->prof.end(st);
+                if (c < 0) return -1;
+                *launches += c;
+            }
+            RowsInvArgs ri{};
+            ri.in = ln.ws_a; ri.pitch = p->XP; ri.q = sq + (size_t)s0 * p->vol * es; ri.y = sy + (size_t)s0 * p->vol * es;
+            ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
+            ri.gtw = p->gtw; ri.gtw_n = p->gtw_n; ri.full_out = p->circular;
+            p->prof.begin(KID_ROWS_INV, st);
+            c = roww ? launch_rows_inv_w(ri, p->dtype, st) : launch_rows_inv(ri, p->dtype, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
-        }
-        if (three) {
-            AxisArgs a{};
-            a.in = ln.ws_b; a.out = ln.ws_a;
-            a.n_outer = n * p->L[0];
-            a.in_outer = (long long)p->P[1] * p->XP; a.out_outer = (long long)p->L[1] * p->XP;
-            a.nc = p->XP; a.n_in = p->P[1]; a.n_out = p->L[1]; a.shift = 0;
-            a.log2p = p->log2p[1]; a.prune_in = 0; a.full = p->circular;
-            a.gtw = p->gtw; a.gtw_n = p->gtw_n;
-            p->prof.begin(KID_AXIS_INV, st);
-            c = launch_axis_any(p->sw, a, AXIS_INV, st);
-            p->prof.end(st);
-            if (c < 0) return -1;
-            *launches += c;
-        }
-        RowsInvArgs ri{};
-        ri.in = ln.ws_a; ri.pitch = p->XP; ri.q = q + (size_t)s0 * p->vol * es; ri.y = y + (size_t)s0 * p->vol * es;
-        ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
-        ri.gtw = p->gtw; ri.gtw_n = p->gtw_n; ri.full_out = p->circular;
-        p->prof.begin(KID_ROWS_INV, st);
-        c = roww ? launch_rows_inv_w(ri, p->dtype, st) : launch_rows_inv(ri, p->dtype, st);
-        p->prof.end(st);
-        if (c < 0) return -1;
-        *launches += c;
+            return 0;
+        };
+        if (side(q, k, v, y, false)) return -1;
+        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true)) return -1;
     }
     return lanes_join(p, st0);
 }
 
 // arguments of the z core of the 3-D path for n slices starting at slice s0, in the workspace of lane l
-static AxisArgs planes3d_core_args(const hyenand_plan *p, int l, long long n, bool shared, long long s0)
+static AxisArgs planes3d_core_args(const hyenand_plan *p, int l, long long n, bool shared, long long s0, bool conj)
 {
     const hyenand_plan::Lane &ln = p->lane[l], &lh = p->lane[shared ? 0 : l];
     const long long nc = (long long)p->XH * p->P[1];
@@ -672,6 +684,7 @@ static AxisArgs planes3d_core_args(const hyenand_plan *p, int l, long long n, bo
     // 1/P of the inverse transforms, and the factors 1/2 the two forward plane kernels leave out of their row separations
     a.scale = (float)(0.25 / ((double)p->P[0] * p->P[1] * p->P[2]));
     a.gtw = p->gtw; a.gtw_n = p->gtw_n;
+    a.h_conj = conj;
     return a;
 }
 
@@ -701,29 +714,35 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         cudaStream_t st = lane_stream(p, l, st0);
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter(l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st)) return -1;
-        PlaneArgs u{};
-        u.a = k + (size_t)s0 * p->vol * es; u.b = v + (size_t)s0 * p->vol * es; u.out = ln.ws_a;
-        u.a_elems = n * p->vol;
-        u.planes = n * p->L[0]; u.lx = p->L[2]; u.ly = p->L[1]; u.gtw = p->gtw; u.gtw_n = p->gtw_n;
-        p->prof.begin(KID_PLANE_U, st);
-        int c = launch_plane(u, PLANE_U, p->log2p[2], p->dtype, st);
-        p->prof.end(st);
-        if (c < 0) return -1;
-        *launches += c;
-        const AxisArgs a = planes3d_core_args(p, l, n, shared, s0);
-        p->prof.begin(KID_CORE, st);
-        c = launch_core_any(p, l, a, shared, st);
-        p->prof.end(st);
-        if (c < 0) return -1;
-        *launches += c;
-        PlaneArgs iv{};
-        iv.a = q + (size_t)s0 * p->vol * es; iv.y = y + (size_t)s0 * p->vol * es; iv.in = ln.ws_a;
-        iv.planes = n * p->L[0]; iv.lx = p->L[2]; iv.ly = p->L[1]; iv.gtw = p->gtw; iv.gtw_n = p->gtw_n;
-        p->prof.begin(KID_PLANE_INV, st);
-        c = launch_plane(iv, PLANE_INV, p->log2p[2], p->dtype, st);
-        p->prof.end(st);
-        if (c < 0) return -1;
-        *launches += c;
+        // one signal side: k v planes, z core against the group's filter spectrum (or its conjugate), planes back
+        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj) -> int {
+            PlaneArgs u{};
+            u.a = sk + (size_t)s0 * p->vol * es; u.b = sv + (size_t)s0 * p->vol * es; u.out = ln.ws_a;
+            u.a_elems = n * p->vol;
+            u.planes = n * p->L[0]; u.lx = p->L[2]; u.ly = p->L[1]; u.gtw = p->gtw; u.gtw_n = p->gtw_n;
+            p->prof.begin(KID_PLANE_U, st);
+            int c = launch_plane(u, PLANE_U, p->log2p[2], p->dtype, st);
+            p->prof.end(st);
+            if (c < 0) return -1;
+            *launches += c;
+            const AxisArgs a = planes3d_core_args(p, l, n, shared, s0, conj);
+            p->prof.begin(KID_CORE, st);
+            c = launch_core_any(p, l, a, shared, st);
+            p->prof.end(st);
+            if (c < 0) return -1;
+            *launches += c;
+            PlaneArgs iv{};
+            iv.a = sq + (size_t)s0 * p->vol * es; iv.y = sy + (size_t)s0 * p->vol * es; iv.in = ln.ws_a;
+            iv.planes = n * p->L[0]; iv.lx = p->L[2]; iv.ly = p->L[1]; iv.gtw = p->gtw; iv.gtw_n = p->gtw_n;
+            p->prof.begin(KID_PLANE_INV, st);
+            c = launch_plane(iv, PLANE_INV, p->log2p[2], p->dtype, st);
+            p->prof.end(st);
+            if (c < 0) return -1;
+            *launches += c;
+            return 0;
+        };
+        if (side(q, k, v, y, false)) return -1;
+        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true)) return -1;
     }
     return lanes_join(p, st0);
 }
@@ -1275,6 +1294,7 @@ struct hyenand_grad {
     long long vol, kvol, pvol, kopp;  // elements per slice: grid, taps, padded ring, taps of the opposite kernel
     bool long1d;
     bool h_native;                    // bf16 I/O: the forwards for dq and du read bf16 taps themselves (no widened kernel)
+    bool pair;                        // dq and du come out of one pass over the groups (one filter spectrum serves both)
     int nb;                           // batch entries per pass
     long long ns;                     // slices per pass of the dh correlation (0: not on that path)
     hyenand_plan *main, *adj, *caus;
@@ -1445,7 +1465,8 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     g->main = hyenand_create_plan_mode(ndim, dims, (int)nb, C, mode, HYENAND_F32);
     if (!g->main) { delete g; return nullptr; }
     g->adj = g->main;
-    if (mode == HYENAND_MODE_CAUSAL) {
+    g->pair = g->main->path == PATH_PLANES3D || g->main->path == PATH_ND_GENERIC;
+    if (mode == HYENAND_MODE_CAUSAL && !g->pair) {
         g->adj = hyenand_create_plan_mode(ndim, dims, (int)nb, C, HYENAND_MODE_LINEAR, HYENAND_F32);
         if (!g->adj) { g->adj = g->main; hyenand_backward_destroy(g); return nullptr; }
     }
@@ -1508,6 +1529,20 @@ static int grad_forward(hyenand_plan *p, long long n, const float *q, const floa
     return e;
 }
 
+// y = q (h conv (k v)) and y2 = q2 (h' conv (k2 v2)), h'[d] = h[-d], in one pass over the groups of the plan (multi-kernel
+// paths): the spectrum of h' is the conjugate of the spectrum of h under the wrapped tap placement (real taps), so the
+// second signal side reuses the filter spectrum its group has just computed.  In causal mode h' is the anti-causal
+// kernel: supports [0, L) and [-(L-1), 0] on a ring of P >= 2L-1 points still do not wrap into the kept outputs.
+static int grad_forward_pair(hyenand_plan *p, long long n, const float *q, const float *k, const float *v, float *y,
+                             const float *q2, const float *k2, const float *v2, float *y2, const void *h, bool shared,
+                             cudaStream_t st, int h_dtype)
+{
+    p->q2 = (const char *)q2; p->k2 = (const char *)k2; p->v2 = (const char *)v2; p->y2 = (char *)y2;
+    const int e = grad_forward(p, n, q, k, v, h, shared, y, st, h_dtype);
+    p->q2 = p->k2 = p->v2 = nullptr; p->y2 = nullptr;
+    return e;
+}
+
 extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, const void *v, const void *h,
                                 long long h_batch_stride_elems, const void *dy, void *dq, void *dk, void *dv, void *dh,
                                 void *cuda_stream)
@@ -1560,25 +1595,33 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             if (widen && !nat) { launch_widen((const char *)h + (long long)b0 * C * kvol * es, g->dtype, S * kvol, g->h32, st); h32 = g->h32; }
         }
         const long long Sh = shared ? C : S;
-        // dq = dy * (h conv (k v))
-        if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
-        launch_mul_cast(g->t32, nullptr, S * vol, g->dtype, (char *)dq + off * es, st);
-        // the kernel at the opposite displacement
-        {
-            RemapArgs r{};
-            r.a = h32; r.b = nullptr; r.out = g->hopp; r.slices = Sh;
-            r.a_bf16 = r.out_bf16 = nat;
-            for (int a = 0; a < 3; ++a) {
-                r.Ls[a] = K[a]; r.G[a] = K[a];
-                r.mode[a] = g->mode == HYENAND_MODE_CIRCULAR ? REMAP_NEG : REMAP_REV;
+        if (g->pair) {
+            // dq = dy * (h conv (k v)) and du = h' conv (dy q) from one pass over the groups; dk = du v, dv = du k
+            if ((e = grad_forward_pair(g->main, S, dy32, k32, v32, g->t32, g->ones, dy32, q32, g->aux, h32, shared, st, hdt))) return e;
+            launch_mul_cast(g->t32, nullptr, S * vol, g->dtype, (char *)dq + off * es, st);
+            launch_mul_cast(g->aux, v32, S * vol, g->dtype, (char *)dk + off * es, st);
+            launch_mul_cast(g->aux, k32, S * vol, g->dtype, (char *)dv + off * es, st);
+        } else {
+            // dq = dy * (h conv (k v))
+            if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
+            launch_mul_cast(g->t32, nullptr, S * vol, g->dtype, (char *)dq + off * es, st);
+            // the kernel at the opposite displacement
+            {
+                RemapArgs r{};
+                r.a = h32; r.b = nullptr; r.out = g->hopp; r.slices = Sh;
+                r.a_bf16 = r.out_bf16 = nat;
+                for (int a = 0; a < 3; ++a) {
+                    r.Ls[a] = K[a]; r.G[a] = K[a];
+                    r.mode[a] = g->mode == HYENAND_MODE_CIRCULAR ? REMAP_NEG : REMAP_REV;
+                }
+                if (g->mode == HYENAND_MODE_CAUSAL) r.G[2] = 2 * L[2] - 1;       // causal taps as the negative half of a non-causal kernel
+                launch_remap(r, st);
             }
-            if (g->mode == HYENAND_MODE_CAUSAL) r.G[2] = 2 * L[2] - 1;       // causal taps as the negative half of a non-causal kernel
-            launch_remap(r, st);
+            // du = h' conv (dy q);  dk = du v, dv = du k
+            if ((e = grad_forward(g->adj, S, g->ones, dy32, q32, g->hopp, shared, g->t32, st, hdt))) return e;
+            launch_mul_cast(g->t32, v32, S * vol, g->dtype, (char *)dk + off * es, st);
+            launch_mul_cast(g->t32, k32, S * vol, g->dtype, (char *)dv + off * es, st);
         }
-        // du = h' conv (dy q);  dk = du v, dv = du k
-        if ((e = grad_forward(g->adj, S, g->ones, dy32, q32, g->hopp, shared, g->t32, st, hdt))) return e;
-        launch_mul_cast(g->t32, v32, S * vol, g->dtype, (char *)dk + off * es, st);
-        launch_mul_cast(g->t32, k32, S * vol, g->dtype, (char *)dv + off * es, st);
         // dh
         float *dhS = shared ? g->dhs : g->dh32;                  // per-slice kernel gradients of this pass
         if (g->mode == HYENAND_MODE_CIRCULAR) {

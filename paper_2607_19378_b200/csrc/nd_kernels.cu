@@ -270,7 +270,7 @@ __global__ void __launch_bounds__(kThreads) axis_kernel(AxisArgs p)
             for (int idx = tid; idx < TX * N; idx += kThreads) {
                 const int x = idx / N, pos = idx % N;
                 const int a = x * LS + phys(pos);
-                float2 w = cmul(bu[a], bh[a]);
+                float2 w = p.h_conj ? cmulc(bu[a], bh[a]) : cmul(bu[a], bh[a]);
                 bu[a] = make_float2(w.x * p.scale, w.y * p.scale);
             }
             __syncthreads();
