@@ -86,7 +86,17 @@ __global__ void __launch_bounds__(kBwdThreads) remap_kernel(RemapArgs r)
             if (r.b) {
 #pragma unroll
                 for (int k = 0; k < kRemapRows; ++k)
-                    if (row_in[k] && col_in) { HN_G(r.b + sbase[k] + j2, 4); val[k] *= __ldg(r.b + sbase[k] + j2); }
+                    if (row_in[k] && col_in) {
+                        const long long src = sbase[k] + j2;
+                        if (r.a_bf16) {
+                            const bf16 *bb = reinterpret_cast<const bf16 *>(r.b);
+                            HN_G(bb + src, 2);
+                            val[k] *= __bfloat162float(bb[src]);
+                        } else {
+                            HN_G(r.b + src, 4);
+                            val[k] *= __ldg(r.b + src);
+                        }
+                    }
             }
 #pragma unroll
             for (int k = 0; k < kRemapRows; ++k) {
@@ -112,7 +122,7 @@ __global__ void __launch_bounds__(kBwdThreads) remap_kernel(RemapArgs r)
 constexpr int kRevUnroll = 16;
 
 template <typename TA, typename TO>
-__global__ void __launch_bounds__(kBwdThreads) reverse_kernel(const TA *a, const float *b, TO *out, long long n)
+__global__ void __launch_bounds__(kBwdThreads) reverse_kernel(const TA *a, const TA *b, TO *out, long long n)
 {
     const long long base = (long long)blockIdx.y * n;
     const long long e0 = (long long)blockIdx.x * (kBwdThreads * kRevUnroll) + threadIdx.x;
@@ -127,7 +137,7 @@ __global__ void __launch_bounds__(kBwdThreads) reverse_kernel(const TA *a, const
 #pragma unroll
         for (int u = 0; u < kRevUnroll; ++u) {
             const long long e = e0 + (long long)u * kBwdThreads;
-            if (e < n) { const long long src = base + n - 1 - e; HN_G(b + src, 4); val[u] *= __ldg(b + src); }
+            if (e < n) { const long long src = base + n - 1 - e; HN_G(b + src, sizeof(TA)); val[u] *= IO<TA>::ld(b, src); }
         }
     }
 #pragma unroll
@@ -142,7 +152,7 @@ __global__ void fill_kernel(float *dst, float value, long long n)
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) { HN_G(dst + i, 4); dst[i] = value; }
 }
 
-template <typename T> __global__ void mul_cast_kernel(const float *a, const float *b, long long n, T *dst)
+template <typename T, typename TB> __global__ void mul_cast_kernel(const float *a, const TB *b, long long n, T *dst)
 {
     // eight elements per thread and round, all loads before the first store
     constexpr int U = 8;
@@ -159,7 +169,7 @@ template <typename T> __global__ void mul_cast_kernel(const float *a, const floa
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const long long i = i0 + (long long)u * blockDim.x;
-                if (i < n) { HN_G(b + i, 4); v[u] *= b[i]; }
+                if (i < n) { HN_G(b + i, sizeof(TB)); v[u] *= IO<TB>::ld(b, i); }
             }
         }
 #pragma unroll
@@ -191,8 +201,8 @@ int launch_remap(const RemapArgs &r, cudaStream_t st)
         const long long n = (long long)r.G[0] * r.G[1] * r.G[2];
         const long long per = (long long)kBwdThreads * kRevUnroll;
         const dim3 grid((unsigned)((n + per - 1) / per), (unsigned)r.slices);
-        if (r.a_bf16 && r.out_bf16) reverse_kernel<bf16, bf16><<<grid, kBwdThreads, 0, st>>>((const bf16 *)r.a, r.b, (bf16 *)r.out, n);
-        else if (r.a_bf16) reverse_kernel<bf16, float><<<grid, kBwdThreads, 0, st>>>((const bf16 *)r.a, r.b, r.out, n);
+        if (r.a_bf16 && r.out_bf16) reverse_kernel<bf16, bf16><<<grid, kBwdThreads, 0, st>>>((const bf16 *)r.a, (const bf16 *)r.b, (bf16 *)r.out, n);
+        else if (r.a_bf16) reverse_kernel<bf16, float><<<grid, kBwdThreads, 0, st>>>((const bf16 *)r.a, (const bf16 *)r.b, r.out, n);
         else if (r.out_bf16) reverse_kernel<float, bf16><<<grid, kBwdThreads, 0, st>>>(r.a, r.b, (bf16 *)r.out, n);
         else reverse_kernel<float, float><<<grid, kBwdThreads, 0, st>>>(r.a, r.b, r.out, n);
         return 1;
@@ -212,12 +222,15 @@ int launch_fill(float *dst, float value, long long n, cudaStream_t st)
     return 1;
 }
 
-int launch_mul_cast(const float *a, const float *b, long long n, int dtype, void *dst, cudaStream_t st)
+int launch_mul_cast(const float *a, const void *b, int b_dtype, long long n, int dtype, void *dst, cudaStream_t st)
 {
     const int grid = bwd_grid((n + 7) / 8);
     if (grid <= 0) return 0;
-    if (dtype == 0) mul_cast_kernel<float><<<grid, kBwdThreads, 0, st>>>(a, b, n, (float *)dst);
-    else mul_cast_kernel<bf16><<<grid, kBwdThreads, 0, st>>>(a, b, n, (bf16 *)dst);
+    const bool bh = b && b_dtype != 0;
+    if (dtype == 0 && !bh) mul_cast_kernel<float, float><<<grid, kBwdThreads, 0, st>>>(a, (const float *)b, n, (float *)dst);
+    else if (dtype == 0) mul_cast_kernel<float, bf16><<<grid, kBwdThreads, 0, st>>>(a, (const bf16 *)b, n, (float *)dst);
+    else if (!bh) mul_cast_kernel<bf16, float><<<grid, kBwdThreads, 0, st>>>(a, (const float *)b, n, (bf16 *)dst);
+    else mul_cast_kernel<bf16, bf16><<<grid, kBwdThreads, 0, st>>>(a, (const bf16 *)b, n, (bf16 *)dst);
     return 1;
 }
 

@@ -17,14 +17,14 @@ struct RemapArgs {
     float *out;               // [slices][G0][G1][G2]
     long long slices;
     int G[3], Ls[3], mode[3], shift[3];
-    int a_bf16, out_bf16;     // a (with b == NULL) and/or out hold bf16 instead of fp32 (a re-indexed copy of bf16 taps is exact)
+    int a_bf16, out_bf16;     // the sources (a, and b when there is one) and/or out hold bf16 instead of fp32
 };
 
 // out[s][i] = a[s][j(i)] * (b ? b[s][j(i)] : 1), zero where an axis index falls outside the source
 int launch_remap(const RemapArgs &r, cudaStream_t st);
 int launch_fill(float *dst, float value, long long n, cudaStream_t st);
-// dst (I/O dtype) = a * (b ? b : 1)
-int launch_mul_cast(const float *a, const float *b, long long n, int dtype, void *dst, cudaStream_t st);
+// dst (I/O dtype) = a * (b ? b : 1); b holds elements of b_dtype (0: fp32, else bf16)
+int launch_mul_cast(const float *a, const void *b, int b_dtype, long long n, int dtype, void *dst, cudaStream_t st);
 // acc[c][t] (+)= sum over nb of src[(b * C + c)][t]   (set = true overwrites)
 int launch_batch_sum(const float *src, long long nb, long long C, long long kvol, bool set, float *acc, cudaStream_t st);
 

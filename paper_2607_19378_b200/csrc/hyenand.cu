@@ -159,6 +159,10 @@ struct hyenand_plan {
     void *stage[5];
     size_t stage_bytes[5];
     int h_dtype;                      // element type of the filter taps (differs from dtype only inside the mixer)
+    // Element types per signal side on the multi-kernel paths, which take them per launch (the backward pass reads the
+    // caller's bf16 tensors and writes a bf16 gradient on one side, an fp32 intermediate on the other): k and v are
+    // `in`, the gate q and the result y are `out`.  Equal to dtype everywhere else.
+    int dt_in, dt_out, dt_in2, dt_out2;
     // Second signal side of the multi-kernel paths (backward pass): after y = q (h conv (k v)) every group also
     // computes y2 = q2 (h' conv (k2 v2)) with h'[d] = h[-d], whose spectrum is the conjugate of the filter spectrum
     // the group has just computed.  Unused (nullptr) in an ordinary forward.
@@ -252,6 +256,7 @@ extern "C" hyenand_plan *hyenand_create_plan_mode(int ndim, const int *dims, int
     hyenand_plan *p = new hyenand_plan();
     memset(p, 0, sizeof(*p));
     p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->circular = circular; p->dtype = dtype; p->h_dtype = dtype;
+    p->dt_in = p->dt_out = p->dt_in2 = p->dt_out2 = dtype;
     p->r0 = 0; p->r1 = (long long)B * C;
     cudaGetDevice(&p->device);
     p->sw = read_switches();
@@ -605,14 +610,15 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter_spectrum_generic(p, l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st, launches)) return -1;
         // one signal side: rows, [middle axis], core against the group's filter spectrum (or its conjugate), back
-        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj) -> int {
+        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj, int dt_in, int dt_out) -> int {
+            const size_t ei = elsize(dt_in), eo = elsize(dt_out);
             RowsArgs r{};
-            r.a = sk + (size_t)s0 * p->vol * es; r.b = sv + (size_t)s0 * p->vol * es; r.out = ln.ws_a; r.pitch = p->XP;
+            r.a = sk + (size_t)s0 * p->vol * ei; r.b = sv + (size_t)s0 * p->vol * ei; r.out = ln.ws_a; r.pitch = p->XP;
             r.rows = n * p->L[0] * p->L[1]; r.len = p->L[2]; r.shift = 0; r.log2p = p->log2p[2];
             r.prune_in = 1; r.full_in = p->circular; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
             p->prof.begin(KID_ROWS_U, st);
             const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
-            int c = roww ? launch_rows_fwd_w(r, p->dtype, st) : launch_rows_fwd(r, p->dtype, st);
+            int c = roww ? launch_rows_fwd_w(r, dt_in, st) : launch_rows_fwd(r, dt_in, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
@@ -653,18 +659,18 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
                 *launches += c;
             }
             RowsInvArgs ri{};
-            ri.in = ln.ws_a; ri.pitch = p->XP; ri.q = sq + (size_t)s0 * p->vol * es; ri.y = sy + (size_t)s0 * p->vol * es;
+            ri.in = ln.ws_a; ri.pitch = p->XP; ri.q = sq ? sq + (size_t)s0 * p->vol * eo : nullptr; ri.y = sy + (size_t)s0 * p->vol * eo;
             ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
             ri.gtw = p->gtw; ri.gtw_n = p->gtw_n; ri.full_out = p->circular;
             p->prof.begin(KID_ROWS_INV, st);
-            c = roww ? launch_rows_inv_w(ri, p->dtype, st) : launch_rows_inv(ri, p->dtype, st);
+            c = roww ? launch_rows_inv_w(ri, dt_out, st) : launch_rows_inv(ri, dt_out, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
             return 0;
         };
-        if (side(q, k, v, y, false)) return -1;
-        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true)) return -1;
+        if (side(q, k, v, y, false, p->dt_in, p->dt_out)) return -1;
+        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true, p->dt_in2, p->dt_out2)) return -1;
     }
     return lanes_join(p, st0);
 }
@@ -715,13 +721,14 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter(l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st)) return -1;
         // one signal side: k v planes, z core against the group's filter spectrum (or its conjugate), planes back
-        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj) -> int {
+        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj, int dt_in, int dt_out) -> int {
+            const size_t ei = elsize(dt_in), eo = elsize(dt_out);
             PlaneArgs u{};
-            u.a = sk + (size_t)s0 * p->vol * es; u.b = sv + (size_t)s0 * p->vol * es; u.out = ln.ws_a;
+            u.a = sk + (size_t)s0 * p->vol * ei; u.b = sv + (size_t)s0 * p->vol * ei; u.out = ln.ws_a;
             u.a_elems = n * p->vol;
             u.planes = n * p->L[0]; u.lx = p->L[2]; u.ly = p->L[1]; u.gtw = p->gtw; u.gtw_n = p->gtw_n;
             p->prof.begin(KID_PLANE_U, st);
-            int c = launch_plane(u, PLANE_U, p->log2p[2], p->dtype, st);
+            int c = launch_plane(u, PLANE_U, p->log2p[2], dt_in, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
@@ -732,17 +739,17 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
             if (c < 0) return -1;
             *launches += c;
             PlaneArgs iv{};
-            iv.a = sq + (size_t)s0 * p->vol * es; iv.y = sy + (size_t)s0 * p->vol * es; iv.in = ln.ws_a;
+            iv.a = sq ? sq + (size_t)s0 * p->vol * eo : nullptr; iv.y = sy + (size_t)s0 * p->vol * eo; iv.in = ln.ws_a;     // no gate: y = the convolution
             iv.planes = n * p->L[0]; iv.lx = p->L[2]; iv.ly = p->L[1]; iv.gtw = p->gtw; iv.gtw_n = p->gtw_n;
             p->prof.begin(KID_PLANE_INV, st);
-            c = launch_plane(iv, PLANE_INV, p->log2p[2], p->dtype, st);
+            c = launch_plane(iv, PLANE_INV, p->log2p[2], dt_out, st);
             p->prof.end(st);
             if (c < 0) return -1;
             *launches += c;
             return 0;
         };
-        if (side(q, k, v, y, false)) return -1;
-        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true)) return -1;
+        if (side(q, k, v, y, false, p->dt_in, p->dt_out)) return -1;
+        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true, p->dt_in2, p->dt_out2)) return -1;
     }
     return lanes_join(p, st0);
 }
@@ -1295,6 +1302,8 @@ struct hyenand_grad {
     bool long1d;
     bool h_native;                    // bf16 I/O: the forwards for dq and du read bf16 taps themselves (no widened kernel)
     bool pair;                        // dq and du come out of one pass over the groups (one filter spectrum serves both)
+    bool native;                      // bf16 I/O on the multi-kernel paths: every kernel reads the caller's bf16 tensors itself and
+                                      // dq leaves its pass as bf16 (no widened copies of q, k, v, dy)
     int nb;                           // batch entries per pass
     long long ns;                     // slices per pass of the dh correlation (0: not on that path)
     hyenand_plan *main, *adj, *caus;
@@ -1354,8 +1363,10 @@ static long long corr_slice_elems(const hyenand_grad *g)
     return 2 * c.rows_in + 2 * c.mid + c.core_out + c.inv_out;
 }
 
-// m slices: gy, gq (their product is g), ur (u reversed) -> out [m][2L0-1][2L1-1][2L2-1]
-static int corr_dh(hyenand_grad *g, long long m, const float *gy, const float *gq, const float *ur, float *out, cudaStream_t st)
+// m slices: gy, gq (elements of g_dtype; their product is g), ur (u reversed, fp32) -> out [m][2L0-1][2L1-1][2L2-1],
+// elements of type out_dtype
+static int corr_dh(hyenand_grad *g, long long m, const void *gy, const void *gq, int g_dtype, const float *ur, void *out,
+                   int out_dtype, cudaStream_t st)
 {
     hyenand_plan *p = g->main;                          // geometry, twiddles, switches
     const int *L = g->L, *P = g->P;
@@ -1363,13 +1374,13 @@ static int corr_dh(hyenand_grad *g, long long m, const float *gy, const float *g
     const bool three = P[0] > 1;
     const int XP = p->XP;
     int c = 0;
-    auto rows = [&](const float *a, const float *b, float2 *dst) {
+    auto rows = [&](const void *a, const void *b, int dt, float2 *dst) {
         RowsArgs r{};
         r.a = a; r.b = b; r.out = dst; r.pitch = XP;
         r.rows = m * L[0] * L[1]; r.len = L[2]; r.shift = 0; r.log2p = p->log2p[2];
         r.prune_in = p->P[2] >= 2; r.full_in = 0; r.gtw = p->gtw; r.gtw_n = p->gtw_n;
         const bool roww = rows_w_supported(r.log2p) && !p->sw.generic_rows;
-        return roww ? launch_rows_fwd_w(r, HYENAND_F32, st) : launch_rows_fwd(r, HYENAND_F32, st);
+        return roww ? launch_rows_fwd_w(r, dt, st) : launch_rows_fwd(r, dt, st);
     };
     auto middle = [&](const float2 *src, float2 *dst) {
         AxisArgs a{};
@@ -1381,8 +1392,8 @@ static int corr_dh(hyenand_grad *g, long long m, const float *gy, const float *g
         a.gtw = p->gtw; a.gtw_n = p->gtw_n;
         return launch_axis_any(p->sw, a, AXIS_FWD, st);
     };
-    if ((c = rows(gy, gq, g->cga)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
-    if ((c = rows(ur, nullptr, g->cua)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    if ((c = rows(gy, gq, g_dtype, g->cga)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
+    if ((c = rows(ur, nullptr, HYENAND_F32, g->cua)) < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
     if (three) {
         if ((c = middle(g->cga, g->cgb)) < 0 || (c = middle(g->cua, g->cub)) < 0)
             return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
@@ -1420,7 +1431,7 @@ static int corr_dh(hyenand_grad *g, long long m, const float *gy, const float *g
         ri.rows = m * K0 * K1; ri.len = K2; ri.log2p = p->log2p[2];
         ri.gtw = p->gtw; ri.gtw_n = p->gtw_n; ri.full_out = 1;
         const bool roww = rows_w_supported(ri.log2p) && !p->sw.generic_rows;
-        c = roww ? launch_rows_inv_w(ri, HYENAND_F32, st) : launch_rows_inv(ri, HYENAND_F32, st);
+        c = roww ? launch_rows_inv_w(ri, out_dtype, st) : launch_rows_inv(ri, out_dtype, st);
         if (c < 0) return fail(HYENAND_ERR_CUDA, "internal launch dispatch failed");
     }
     return HYENAND_OK;
@@ -1487,12 +1498,15 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     const bool widen = dtype == HYENAND_BF16;
     auto reads_bf16 = [](const hyenand_plan *q) { return q->path == PATH_PLANES3D || q->path == PATH_ND_GENERIC; };
     g->h_native = widen && reads_bf16(g->main) && reads_bf16(g->adj);
+    g->native = widen && g->pair && mode != HYENAND_MODE_CIRCULAR && !g->long1d;
     cudaError_t e = cudaSuccess;
     auto get = [&](float **ptr, long long elems) {
         if (e == cudaSuccess) e = guarded_alloc(&g->allocs, (void **)ptr, (size_t)elems * sizeof(float));
     };
-    if (widen) { get(&g->q32, S * g->vol); get(&g->k32, S * g->vol); get(&g->v32, S * g->vol); get(&g->dy32, S * g->vol); if (!g->h_native) get(&g->h32, S * g->kvol); }
-    get(&g->ones, S * g->vol); get(&g->t32, S * g->vol); get(&g->hopp, S * g->kopp);
+    if (widen && !g->native) { get(&g->q32, S * g->vol); get(&g->k32, S * g->vol); get(&g->v32, S * g->vol); get(&g->dy32, S * g->vol); }
+    if (widen && !g->h_native) get(&g->h32, S * g->kvol);
+    if (!g->native) { get(&g->ones, S * g->vol); get(&g->t32, S * g->vol); }
+    get(&g->hopp, S * g->kopp);
     get(&g->aux, S * g->vol); get(&g->dhs, S * g->kvol); get(&g->dh32, S * g->kvol);
     if (g->ns) {
         const CorrGeo c = corr_geo(g);
@@ -1507,7 +1521,7 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
         return nullptr;
     }
     { DbgScope d; d.add(g->allocs); d.commit(); }
-    launch_fill(g->ones, 1.f, S * g->vol, 0);
+    if (g->ones) launch_fill(g->ones, 1.f, S * g->vol, 0);
     if (cudaDeviceSynchronize() != cudaSuccess) {
         fail(HYENAND_ERR_CUDA, "filling the constant tensors failed: %s", cudaGetErrorString(cudaGetLastError()));
         hyenand_backward_destroy(g);
@@ -1526,6 +1540,7 @@ static int grad_forward(hyenand_plan *p, long long n, const float *q, const floa
     const int e = run_forward(p, q, k, v, h, shared, y, st, &launches);
     p->r0 = 0; p->r1 = (long long)p->B * p->C;
     p->h_dtype = p->dtype;
+    p->dt_in = p->dt_out = p->dt_in2 = p->dt_out2 = p->dtype;
     return e;
 }
 
@@ -1533,12 +1548,14 @@ static int grad_forward(hyenand_plan *p, long long n, const float *q, const floa
 // paths): the spectrum of h' is the conjugate of the spectrum of h under the wrapped tap placement (real taps), so the
 // second signal side reuses the filter spectrum its group has just computed.  In causal mode h' is the anti-causal
 // kernel: supports [0, L) and [-(L-1), 0] on a ring of P >= 2L-1 points still do not wrap into the kept outputs.
-static int grad_forward_pair(hyenand_plan *p, long long n, const float *q, const float *k, const float *v, float *y,
-                             const float *q2, const float *k2, const float *v2, float *y2, const void *h, bool shared,
-                             cudaStream_t st, int h_dtype)
+static int grad_forward_pair(hyenand_plan *p, long long n, const void *q, const void *k, const void *v, void *y,
+                             const void *q2, const void *k2, const void *v2, void *y2, const void *h, bool shared,
+                             cudaStream_t st, int h_dtype, int dt_in = HYENAND_F32, int dt_out = HYENAND_F32,
+                             int dt_in2 = HYENAND_F32, int dt_out2 = HYENAND_F32)
 {
     p->q2 = (const char *)q2; p->k2 = (const char *)k2; p->v2 = (const char *)v2; p->y2 = (char *)y2;
-    const int e = grad_forward(p, n, q, k, v, h, shared, y, st, h_dtype);
+    p->dt_in = dt_in; p->dt_out = dt_out; p->dt_in2 = dt_in2; p->dt_out2 = dt_out2;
+    const int e = grad_forward(p, n, (const float *)q, (const float *)k, (const float *)v, h, shared, (float *)y, st, h_dtype);
     p->q2 = p->k2 = p->v2 = nullptr; p->y2 = nullptr;
     return e;
 }
@@ -1583,7 +1600,7 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
     for (int b0 = 0; b0 < g->B; b0 += g->nb) {
         const long long n = g->B - b0 < g->nb ? g->B - b0 : g->nb, S = n * C, off = (long long)b0 * C * vol;
         const float *q32 = (const float *)q + off, *k32 = (const float *)k + off, *v32 = (const float *)v + off, *dy32 = (const float *)dy + off;
-        if (widen) {
+        if (widen && !g->native) {
             launch_widen((const char *)q + off * es, g->dtype, S * vol, g->q32, st); q32 = g->q32;
             launch_widen((const char *)k + off * es, g->dtype, S * vol, g->k32, st); k32 = g->k32;
             launch_widen((const char *)v + off * es, g->dtype, S * vol, g->v32, st); v32 = g->v32;
@@ -1595,16 +1612,26 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             if (widen && !nat) { launch_widen((const char *)h + (long long)b0 * C * kvol * es, g->dtype, S * kvol, g->h32, st); h32 = g->h32; }
         }
         const long long Sh = shared ? C : S;
-        if (g->pair) {
+        // the caller's tensors of this pass, in their own element type
+        const char *qn = (const char *)q + off * es, *kn = (const char *)k + off * es, *vn = (const char *)v + off * es,
+                   *dyn = (const char *)dy + off * es;
+        if (g->native) {
+            // as below, on the caller's bf16 tensors: the first side is a bf16 forward with dy as its gate and dq as its
+            // result, the second reads dy and q and leaves du in fp32 without a gate
+            if ((e = grad_forward_pair(g->main, S, dyn, kn, vn, (char *)dq + off * es, nullptr, dyn, qn, g->aux, h32, shared, st, hdt,
+                                       HYENAND_BF16, HYENAND_BF16, HYENAND_BF16, HYENAND_F32))) return e;
+            launch_mul_cast(g->aux, vn, g->dtype, S * vol, g->dtype, (char *)dk + off * es, st);
+            launch_mul_cast(g->aux, kn, g->dtype, S * vol, g->dtype, (char *)dv + off * es, st);
+        } else if (g->pair) {
             // dq = dy * (h conv (k v)) and du = h' conv (dy q) from one pass over the groups; dk = du v, dv = du k
             if ((e = grad_forward_pair(g->main, S, dy32, k32, v32, g->t32, g->ones, dy32, q32, g->aux, h32, shared, st, hdt))) return e;
-            launch_mul_cast(g->t32, nullptr, S * vol, g->dtype, (char *)dq + off * es, st);
-            launch_mul_cast(g->aux, v32, S * vol, g->dtype, (char *)dk + off * es, st);
-            launch_mul_cast(g->aux, k32, S * vol, g->dtype, (char *)dv + off * es, st);
+            launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
+            launch_mul_cast(g->aux, v32, 0, S * vol, g->dtype, (char *)dk + off * es, st);
+            launch_mul_cast(g->aux, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
         } else {
             // dq = dy * (h conv (k v))
             if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
-            launch_mul_cast(g->t32, nullptr, S * vol, g->dtype, (char *)dq + off * es, st);
+            launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
             // the kernel at the opposite displacement
             {
                 RemapArgs r{};
@@ -1619,11 +1646,12 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             }
             // du = h' conv (dy q);  dk = du v, dv = du k
             if ((e = grad_forward(g->adj, S, g->ones, dy32, q32, g->hopp, shared, g->t32, st, hdt))) return e;
-            launch_mul_cast(g->t32, v32, S * vol, g->dtype, (char *)dk + off * es, st);
-            launch_mul_cast(g->t32, k32, S * vol, g->dtype, (char *)dv + off * es, st);
+            launch_mul_cast(g->t32, v32, 0, S * vol, g->dtype, (char *)dk + off * es, st);
+            launch_mul_cast(g->t32, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
         }
         // dh
         float *dhS = shared ? g->dhs : g->dh32;                  // per-slice kernel gradients of this pass
+        bool dh_direct = false;                                  // this pass's dh is already in the caller's tensor
         if (g->mode == HYENAND_MODE_CIRCULAR) {
             // dh[m] = sum_i g_i u_{(i-m) mod L}: circular convolution of g with u read at the opposite displacement
             // (hopp is free again: the forward that consumed the opposite kernel precedes this on the stream)
@@ -1675,13 +1703,23 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             {
                 RemapArgs r{};
                 r.a = k32; r.b = v32; r.out = g->aux; r.slices = S;
+                if (g->native) { r.a = (const float *)kn; r.b = (const float *)vn; r.a_bf16 = 1; }
                 for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = REMAP_REV; }
                 launch_remap(r, st);
             }
+            // Per-sample kernels without a causal crop: the last stage writes the caller's dh itself (one rounding of the
+            // fp32 sums either way), else fp32 taps that are cropped and/or summed over the batch below.
+            dh_direct = !shared && g->mode != HYENAND_MODE_CAUSAL;
+            char *dh_pass = (char *)dh + (long long)b0 * C * kvol * es;
             float *full = g->mode == HYENAND_MODE_CAUSAL ? g->hopp : dhS;     // all 2L-1 taps per slice
             for (long long s0 = 0; s0 < S; s0 += g->ns) {
                 const long long m = S - s0 < g->ns ? S - s0 : g->ns;
-                if ((e = corr_dh(g, m, dy32 + s0 * vol, q32 + s0 * vol, g->aux + s0 * vol, full + s0 * g->kopp, st))) return e;
+                void *dst = dh_direct ? (void *)(dh_pass + s0 * kvol * es) : (void *)(full + s0 * g->kopp);
+                const void *gy = g->native ? (const void *)(dyn + s0 * vol * es) : (const void *)(dy32 + s0 * vol);
+                const void *gq = g->native ? (const void *)(qn + s0 * vol * es) : (const void *)(q32 + s0 * vol);
+                if ((e = corr_dh(g, m, gy, gq, g->native ? g->dtype : HYENAND_F32, g->aux + s0 * vol, dst,
+                                 dh_direct ? g->dtype : HYENAND_F32, st)))
+                    return e;
             }
             if (g->mode == HYENAND_MODE_CAUSAL &&
                 cudaMemcpy2DAsync(dhS, (size_t)kvol * sizeof(float), g->hopp + (L[2] - 1), (size_t)g->kopp * sizeof(float),
@@ -1689,9 +1727,9 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
                 return fail(HYENAND_ERR_CUDA, "copy of the causal taps failed: %s", cudaGetErrorString(cudaGetLastError()));
             if (shared) launch_batch_sum(dhS, n, C, kvol, b0 == 0, g->dh32, st);
         }
-        if (!shared) launch_mul_cast(g->dh32, nullptr, S * kvol, g->dtype, (char *)dh + (long long)b0 * C * kvol * es, st);
+        if (!shared && !dh_direct) launch_mul_cast(g->dh32, nullptr, 0, S * kvol, g->dtype, (char *)dh + (long long)b0 * C * kvol * es, st);
     }
-    if (shared) launch_mul_cast(g->dh32, nullptr, C * kvol, g->dtype, dh, st);
+    if (shared) launch_mul_cast(g->dh32, nullptr, 0, C * kvol, g->dtype, dh, st);
     cudaError_t ce = cudaGetLastError();
     if (ce != cudaSuccess) return fail(HYENAND_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(ce));
     return HYENAND_OK;
@@ -1806,6 +1844,7 @@ extern "C" int hyenand_forward_noalloc(int ndim, const int *dims, int B, int C, 
     memset(&sp, 0, sizeof(sp));
     hyenand_plan *p = &sp;
     p->ndim = ndim; p->B = B; p->C = C; p->causal = causal; p->dtype = dtype; p->h_dtype = dtype;
+    p->dt_in = p->dt_out = p->dt_in2 = p->dt_out2 = dtype;
     p->r0 = 0; p->r1 = (long long)B * C;
     p->vol = 1; p->kvol = 1;
     for (int a = 0; a < 3; ++a) { p->L[a] = 1; p->K[a] = 1; p->P[a] = 1; p->log2p[a] = 0; }

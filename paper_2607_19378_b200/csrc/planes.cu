@@ -440,6 +440,15 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
     const T *pq = (const T *)p.a;
     T *py = (T *)p.y;
     const int Lx = p.lx, Ly = p.ly;
+    const bool gated = pq != nullptr;                        // no gate tensor: the convolution itself is written (gate 1)
+    const T qfill = gated ? T(0.f) : T(1.f);
+    uint4 qvfill;
+    {
+        float f[Vec16<T>::VEC];
+#pragma unroll
+        for (int e = 0; e < Vec16<T>::VEC; ++e) f[e] = gated ? 0.f : 1.f;
+        qvfill = Vec16<T>::pack(f);
+    }
     for (long long pl = blockIdx.x; pl < p.planes; pl += gridDim.x) {
         const float2 *src = p.in + pl * (long long)C::XH * P;
         // Column kx + NG is requested (into registers) between the two passes of column kx: the loads
@@ -514,9 +523,9 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
 #pragma unroll
                 for (int j = 0; j < NV; ++j) {
                     const int x0 = (l + j * TPL) * VEC;
-                    qv0[it][j] = qv1[it][j] = make_uint4(0u, 0u, 0u, 0u);
-                    if (x0 < Lx && has0) { HN_G(pq + o0 + x0, 16); qv0[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o0 + x0)); }
-                    if (x0 < Lx && has1) { HN_G(pq + o1 + x0, 16); qv1[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o1 + x0)); }
+                    qv0[it][j] = qv1[it][j] = qvfill;
+                    if (x0 < Lx && has0 && gated) { HN_G(pq + o0 + x0, 16); qv0[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o0 + x0)); }
+                    if (x0 < Lx && has1 && gated) { HN_G(pq + o1 + x0, 16); qv1[it][j] = __ldg(reinterpret_cast<const uint4 *>(pq + o1 + x0)); }
                 }
             } else {
 #pragma unroll
@@ -524,10 +533,10 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
 #pragma unroll
                     for (int r = 0; r < PE::R / 2; ++r) {
                         const int idx = FI::last_pos(l, i, r);
-                        if (idx < Lx && has0) HN_G(pq + o0 + idx, sizeof(T));
-                        if (idx < Lx && has1) HN_G(pq + o1 + idx, sizeof(T));
-                        q0[it][i * (PE::R / 2) + r] = (idx < Lx && has0) ? __ldg(pq + o0 + idx) : T(0.f);
-                        q1[it][i * (PE::R / 2) + r] = (idx < Lx && has1) ? __ldg(pq + o1 + idx) : T(0.f);
+                        if (idx < Lx && has0 && gated) HN_G(pq + o0 + idx, sizeof(T));
+                        if (idx < Lx && has1 && gated) HN_G(pq + o1 + idx, sizeof(T));
+                        q0[it][i * (PE::R / 2) + r] = (idx < Lx && has0 && gated) ? __ldg(pq + o0 + idx) : qfill;
+                        q1[it][i * (PE::R / 2) + r] = (idx < Lx && has1 && gated) ? __ldg(pq + o1 + idx) : qfill;
                     }
             }
         }
@@ -535,7 +544,7 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
         if (pl + gridDim.x < p.planes) {
             // while the rows are transformed, bring the next plane's spectra and gate into L2
             prefetch_l2(p.in + (pl + gridDim.x) * (long long)C::XH * P, (long long)C::XH * P * sizeof(float2), tid);
-            prefetch_l2(pq + (pl + gridDim.x) * (long long)Ly * Lx, (long long)Ly * Lx * sizeof(T), tid);
+            if (gated) prefetch_l2(pq + (pl + gridDim.x) * (long long)Ly * Lx, (long long)Ly * Lx * sizeof(T), tid);
         }
 #pragma unroll
         for (int it = 0; it < RIT; ++it) {

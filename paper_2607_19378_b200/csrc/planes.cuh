@@ -8,7 +8,7 @@ namespace hn {
 enum PlaneKind { PLANE_U = 0, PLANE_H = 1, PLANE_INV = 2 };
 
 struct PlaneArgs {
-    const void *a;        // k (PLANE_U), h (PLANE_H), q (PLANE_INV)
+    const void *a;        // k (PLANE_U), h (PLANE_H), q (PLANE_INV; NULL: no gate, the convolution itself is written)
     const void *b;        // v (PLANE_U)
     float2 *out;          // spectra [plane][P/2+1][P] written by PLANE_U / PLANE_H
     const float2 *in;     // spectra read by PLANE_INV

@@ -80,7 +80,7 @@ def check_backward(w, q, k, v, h, seed, direct=False):
 
 SHAPES = [((1,), False), ((5,), False), ((300,), False), ((1000,), True), ((4096,), True), ((5000,), False),
           ((9001,), True), ((15, 14), False), ((40, 50), False), ((64, 64), False), ((130, 70), False),
-          ((5, 3, 2), False), ((20, 24, 30), False)]
+          ((5, 3, 2), False), ((20, 24, 30), False), ((32, 32, 32), False), ((8, 40, 48), False), ((6, 36, 43), False)]
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
