@@ -196,7 +196,8 @@ int launch_remap(const RemapArgs &r, cudaStream_t st)
     const long long rows = r.slices * r.G[0] * r.G[1];
     if (rows <= 0 || r.G[2] <= 0) return 0;
     bool flat_rev = r.slices <= 65535;
-    for (int x = 0; x < 3; ++x) flat_rev = flat_rev && r.mode[x] == REMAP_REV && r.G[x] == r.Ls[x];
+    for (int x = 0; x < 3; ++x)                            // an axis of one point maps 0 -> 0 in every mode but WRAP
+        flat_rev = flat_rev && r.G[x] == r.Ls[x] && (r.mode[x] == REMAP_REV || (r.G[x] == 1 && r.mode[x] != REMAP_WRAP));
     if (flat_rev) {
         const long long n = (long long)r.G[0] * r.G[1] * r.G[2];
         const long long per = (long long)kBwdThreads * kRevUnroll;

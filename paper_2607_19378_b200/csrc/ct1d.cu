@@ -373,6 +373,7 @@ int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, in
               GuardedAllocs *g, size_t *bytes)
 {
     c->sw = sw;
+    c->keep_filter = 0;
     c->L = L; c->K = K; c->log2p = log2p; c->B = B; c->C = C; c->causal = causal; c->dtype = dtype;
     c->log2p1 = log2p / 2;
     c->log2p2 = log2p - c->log2p1;
@@ -422,7 +423,7 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
     const TwoLevel twp{c->twp_coarse, c->twp_fine, c->lo};
     if (ct1d_uses_w(c)) {
         const bool staged_ok = c->causal != 0;
-        if (shared && c->r0 == 0 && ct1d_w_filter(c, h, c->C, staged_ok, st, launches, prof, filter_pass)) return -1;
+        if (shared && c->r0 == 0 && !c->keep_filter && ct1d_w_filter(c, h, c->C, staged_ok, st, launches, prof, filter_pass)) return -1;
         for (long long s0 = c->r0; s0 < c->r1; s0 += c->slices_per_chunk) {
             const long long n = c->r1 - s0 < c->slices_per_chunk ? c->r1 - s0 : c->slices_per_chunk;
             if (!shared && ct1d_w_filter(c, (const char *)h + (size_t)s0 * c->K * es, n, staged_ok, st, launches, prof, filter_pass))
@@ -434,7 +435,7 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
         }
         return 0;
     }
-    if (shared && c->r0 == 0 && filter_pass(c, (const char *)h, c->C, st, launches, prof)) return -1;
+    if (shared && c->r0 == 0 && !c->keep_filter && filter_pass(c, (const char *)h, c->C, st, launches, prof)) return -1;
     for (long long s0 = c->r0; s0 < c->r1; s0 += c->slices_per_chunk) {
         const long long n = c->r1 - s0 < c->slices_per_chunk ? c->r1 - s0 : c->slices_per_chunk;
         if (!shared && filter_pass(c, (const char *)h + (size_t)s0 * c->K * es, n, st, launches, prof)) return -1;

@@ -21,6 +21,8 @@ struct Ct1dPlan {
     Switches sw;              // development switches, read when the plan was created
     long long slices_per_chunk, wh_slices;
     long long r0, r1;         // slices [r0, r1) the next forward works on
+    int keep_filter;          // 1: the spectrum of the shared filter is still in wh from this plan's previous forward
+                              // (same taps): the next forward does not transform it again
 };
 
 // allocations go on the plan's guarded list `g` and are freed with it

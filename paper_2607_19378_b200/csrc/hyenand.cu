@@ -1477,7 +1477,8 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     if (!g->main) { delete g; return nullptr; }
     g->adj = g->main;
     g->pair = g->main->path == PATH_PLANES3D || g->main->path == PATH_ND_GENERIC;
-    if (mode == HYENAND_MODE_CAUSAL && !g->pair) {
+    // (a long causal 1-D grid gets du from the causal plan and reversed signals, see hyenand_backward)
+    if (mode == HYENAND_MODE_CAUSAL && !g->pair && !g->long1d) {
         g->adj = hyenand_create_plan_mode(ndim, dims, (int)nb, C, HYENAND_MODE_LINEAR, HYENAND_F32);
         if (!g->adj) { g->adj = g->main; hyenand_backward_destroy(g); return nullptr; }
     }
@@ -1628,6 +1629,28 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
             launch_mul_cast(g->aux, v32, 0, S * vol, g->dtype, (char *)dk + off * es, st);
             launch_mul_cast(g->aux, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
+        } else if (g->long1d && g->mode == HYENAND_MODE_CAUSAL) {
+            // dq = dy * (h conv (k v))
+            if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
+            launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
+            // du[t] = sum_{s >= t} h[s - t] g[s], g = dy q, is the anti-causal convolution; read backwards in time it is
+            // the causal one, rev(du) = h conv rev(g): the causal plan (and its faster kernels) serves, with two
+            // reversals at the copy rate, instead of a non-causal plan with a kernel of 2L-1 taps, half of them zero.
+            // aux = rev(g) stays for the dh stage below.
+            RemapArgs r{};
+            r.a = dy32; r.b = q32; r.out = g->aux; r.slices = S;
+            for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
+            launch_remap(r, st);
+            g->main->ct.keep_filter = shared;                       // same taps as the forward for dq just before
+            e = grad_forward(g->main, S, g->ones, g->aux, g->ones, h32, shared, g->t32, st, hdt);
+            g->main->ct.keep_filter = 0;
+            if (e) return e;
+            RemapArgs rv{};
+            rv.a = g->t32; rv.out = g->hopp; rv.slices = S;          // hopp: S*(2L-1) floats, du takes the first S*L
+            for (int a = 0; a < 3; ++a) { rv.Ls[a] = L[a]; rv.G[a] = L[a]; rv.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
+            launch_remap(rv, st);
+            launch_mul_cast(g->hopp, v32, 0, S * vol, g->dtype, (char *)dk + off * es, st);
+            launch_mul_cast(g->hopp, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
         } else {
             // dq = dy * (h conv (k v))
             if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
@@ -1668,7 +1691,7 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             RemapArgs r{};
             r.a = dy32; r.b = q32; r.out = g->aux; r.slices = S;
             for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
-            launch_remap(r, st);
+            if (g->mode != HYENAND_MODE_CAUSAL) launch_remap(r, st);       // (causal: aux holds the reversed g already)
             if ((e = grad_forward(g->caus, S, g->ones, k32, v32, g->aux, false, g->t32, st))) return e;
             if (g->mode == HYENAND_MODE_CAUSAL) {
                 RemapArgs w{};                                 // tap t <- c[L-1-t]
