@@ -44,7 +44,8 @@ template <int LOG2P> struct F2Cfg {
 // so every phase keeps all groups busy; the k*v store is double buffered.
 // VST: rows are whole numbers of 16-byte vectors and q, y are 16-byte aligned: gate values arrive as 16-byte loads, the
 // cropped rows go through the line once more and leave as 16-byte stores; else one element per lane and leg.
-template <typename T, int LOG2P, bool VST>
+// TWO: a second gate and result, y2 = q2 * (the same convolution) (the backward pass: dk = v du and dv = k du).
+template <typename T, int LOG2P, bool VST, bool TWO>
 __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)     // 96 registers: one scheduler hosts 5 of the 17 warps
 {
     using C = F2Cfg<LOG2P>;
@@ -73,6 +74,8 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)  
     const unsigned char *ke = kb + p.kv_elems * sizeof(T), *ve = vb + p.kv_elems * sizeof(T), *he = hb + p.h_elems * sizeof(T);
     const T *pq = (const T *)p.q;
     T *py = (T *)p.y;
+    const T *pq2 = (const T *)p.q2;
+    T *py2 = (T *)p.y2;
     const int Lx = p.lx, Ly = p.ly, Kx = 2 * Lx - 1, Ky = 2 * Ly - 1;
     const long long vol = (long long)Lx * Ly, kvol = (long long)Kx * Ky;
     using PL = typename F::LastPass;
@@ -123,6 +126,28 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)  
                         if (has1) { HN_G(py + o1 + x0, 16); *reinterpret_cast<uint4 *>(py + o1 + x0) = Vec16<T>::pack(b); }
                     }
                 }
+                if constexpr (TWO) {
+#pragma unroll
+                    for (int j = 0; j < NV; ++j) {
+                        const int x0 = (l + j * TPL) * VEC;
+                        if (x0 < Lx) {
+                            float a[VEC], b[VEC], ga[VEC], gb[VEC];
+                            HN_G(pq2 + o0 + x0, 16);
+                            Vec16<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(pq2 + o0 + x0)), ga);
+                            if (has1) HN_G(pq2 + o1 + x0, 16);
+                            Vec16<T>::unpack(has1 ? __ldg(reinterpret_cast<const uint4 *>(pq2 + o1 + x0)) : make_uint4(0u, 0u, 0u, 0u), gb);
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) {
+                                const float2 z = line[FI::ph(x0 + e)];
+                                a[e] = z.x * ga[e];
+                                b[e] = z.y * gb[e];
+                            }
+                            HN_G(py2 + o0 + x0, 16);
+                            *reinterpret_cast<uint4 *>(py2 + o0 + x0) = Vec16<T>::pack(a);
+                            if (has1) { HN_G(py2 + o1 + x0, 16); *reinterpret_cast<uint4 *>(py2 + o1 + x0) = Vec16<T>::pack(b); }
+                        }
+                    }
+                }
             } else {
                 T q0[NQ], q1[NQ];
 #pragma unroll
@@ -140,6 +165,11 @@ __global__ void __launch_bounds__(kF2Threads, 1) fused2d_kernel(Fused2dArgs p)  
                         if (idx < Lx) {
                             IO<T>::st(py, o0 + idx, v.x * (float)q0[i * (PIL::R / 2) + r]);
                             if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[i * (PIL::R / 2) + r]);
+                            if constexpr (TWO) {
+                                HN_G(pq2 + o0 + idx, ES);
+                                IO<T>::st(py2, o0 + idx, v.x * IO<T>::ld(pq2, o0 + idx));
+                                if (has1) { HN_G(pq2 + o1 + idx, ES); IO<T>::st(py2, o1 + idx, v.y * IO<T>::ld(pq2, o1 + idx)); }
+                            }
                         }
                     });
             }
@@ -321,10 +351,13 @@ template <typename T, int LOG2P> static int launch_fused2d_t(const Fused2dArgs &
         if (sms <= 0) sms = 148;
     }
     // 16-byte gate loads and result stores where every row is a whole number of vectors on a 16-byte boundary
-    const bool vst = a.lx % Vec16<T>::VEC == 0 && (((uintptr_t)a.q | (uintptr_t)a.y) & 15) == 0;
-    static DevOnce attr[2];
-    void (*fn)(Fused2dArgs) = vst ? fused2d_kernel<T, LOG2P, true> : fused2d_kernel<T, LOG2P, false>;
-    if (attr[vst ? 1 : 0].first()) cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
+    const bool two = a.q2 != nullptr && a.y2 != nullptr;
+    const bool vst = a.lx % Vec16<T>::VEC == 0 &&
+                     (((uintptr_t)a.q | (uintptr_t)a.y | (uintptr_t)a.q2 | (uintptr_t)a.y2) & 15) == 0;
+    static DevOnce attr[4];
+    void (*fn)(Fused2dArgs) = two ? (vst ? fused2d_kernel<T, LOG2P, true, true> : fused2d_kernel<T, LOG2P, false, true>)
+                                  : (vst ? fused2d_kernel<T, LOG2P, true, false> : fused2d_kernel<T, LOG2P, false, false>);
+    if (attr[(two ? 2 : 0) + (vst ? 1 : 0)].first()) cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
     const int grid = (int)(a.slices < sms ? a.slices : sms);
     if (grid <= 0) return 0;
     fn<<<grid, kF2Threads, C::SMEM, st>>>(a);

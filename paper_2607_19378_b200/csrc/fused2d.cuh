@@ -7,6 +7,8 @@ namespace hn {
 struct Fused2dArgs {
     const void *q, *k, *v, *h;
     void *y;
+    const void *q2;           // optional second gate and result of the same convolution: y2 = q2 * (h conv (k v)); both or none
+    void *y2;
     long long slices;         // B*C
     int lx, ly;               // grid extent along x (contiguous) and y
     long long h_mod, h_off;   // filter slice = h_mod ? (s + h_off) % h_mod : s

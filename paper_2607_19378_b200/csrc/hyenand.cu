@@ -168,6 +168,8 @@ struct hyenand_plan {
     // the group has just computed.  Unused (nullptr) in an ordinary forward.
     const char *q2, *k2, *v2;
     char *y2;
+    const char *qg2;                  // fused 2-D path: a second gate and result of the same convolution (see Fused2dArgs)
+    char *yg2;
     size_t ws_bytes;
     Prof prof;
 };
@@ -765,6 +767,7 @@ static int forward_fused2d(hyenand_plan *p, const void *q, const void *k, const 
     a.slices = p->r1 - p->r0; a.lx = p->L[2]; a.ly = p->L[1];
     a.h_mod = shared ? p->C : 0; a.h_off = shared ? p->r0 % p->C : 0;
     a.scale = (float)(1.0 / ((double)p->P[1] * p->P[2]));
+    if (p->yg2) { a.q2 = p->qg2 + off; a.y2 = p->yg2 + off; }
     a.gtw = p->gtw; a.gtw_n = p->gtw_n;
     a.kv_elems = a.slices * p->vol;
     a.h_elems = (shared ? p->C : a.slices) * p->kvol;
@@ -1302,7 +1305,9 @@ struct hyenand_grad {
     bool long1d;
     bool h_native;                    // bf16 I/O: the forwards for dq and du read bf16 taps themselves (no widened kernel)
     bool pair;                        // dq and du come out of one pass over the groups (one filter spectrum serves both)
-    bool native;                      // bf16 I/O on the multi-kernel paths: every kernel reads the caller's bf16 tensors itself and
+    bool two_gate;                    // fused 2-D path, linear mode: the plan runs in the caller's element type; dq is a forward
+                                      // gated by dy, dk and dv are the two results of one forward gated by v and by k
+    bool native;                      // bf16 I/O on the multi-kernel paths and with two_gate: every kernel reads the caller's bf16 tensors itself and
                                       // dq leaves its pass as bf16 (no widened copies of q, k, v, dy)
     int nb;                           // batch entries per pass
     long long ns;                     // slices per pass of the dh correlation (0: not on that path)
@@ -1475,6 +1480,12 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     const long long S = nb * C;
     g->main = hyenand_create_plan_mode(ndim, dims, (int)nb, C, mode, HYENAND_F32);
     if (!g->main) { delete g; return nullptr; }
+    g->two_gate = g->main->path == PATH_FUSED2D && mode == HYENAND_MODE_LINEAR;
+    if (g->two_gate && dtype != HYENAND_F32) {
+        hyenand_destroy_plan(g->main);
+        g->main = hyenand_create_plan_mode(ndim, dims, (int)nb, C, mode, dtype);
+        if (!g->main) { delete g; return nullptr; }
+    }
     g->adj = g->main;
     g->pair = g->main->path == PATH_PLANES3D || g->main->path == PATH_ND_GENERIC;
     // (a long causal 1-D grid gets du from the causal plan and reversed signals, see hyenand_backward)
@@ -1498,8 +1509,8 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     }
     const bool widen = dtype == HYENAND_BF16;
     auto reads_bf16 = [](const hyenand_plan *q) { return q->path == PATH_PLANES3D || q->path == PATH_ND_GENERIC; };
-    g->h_native = widen && reads_bf16(g->main) && reads_bf16(g->adj);
-    g->native = widen && g->pair && mode != HYENAND_MODE_CIRCULAR && !g->long1d;
+    g->h_native = widen && ((reads_bf16(g->main) && reads_bf16(g->adj)) || g->two_gate);
+    g->native = widen && ((g->pair && mode != HYENAND_MODE_CIRCULAR && !g->long1d) || g->two_gate);
     cudaError_t e = cudaSuccess;
     auto get = [&](float **ptr, long long elems) {
         if (e == cudaSuccess) e = guarded_alloc(&g->allocs, (void **)ptr, (size_t)elems * sizeof(float));
@@ -1616,7 +1627,22 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
         // the caller's tensors of this pass, in their own element type
         const char *qn = (const char *)q + off * es, *kn = (const char *)k + off * es, *vn = (const char *)v + off * es,
                    *dyn = (const char *)dy + off * es;
-        if (g->native) {
+        if (g->two_gate) {
+            // the plan runs in the caller's element type: dq = dy * (h conv (k v)) is a forward gated by dy; the forward of
+            // dy q against the kernel at the opposite displacement leaves through two gates, dk = v * du and dv = k * du
+            char *dqn = (char *)dq + off * es, *dkn = (char *)dk + off * es, *dvn = (char *)dv + off * es;
+            if ((e = grad_forward(g->main, S, (const float *)dyn, (const float *)kn, (const float *)vn, h32, shared, (float *)dqn, st, g->dtype)))
+                return e;
+            RemapArgs r{};
+            r.a = h32; r.b = nullptr; r.out = g->hopp; r.slices = Sh;
+            r.a_bf16 = r.out_bf16 = widen;
+            for (int a = 0; a < 3; ++a) { r.Ls[a] = K[a]; r.G[a] = K[a]; r.mode[a] = REMAP_REV; }
+            launch_remap(r, st);
+            g->main->qg2 = kn; g->main->yg2 = dvn;
+            e = grad_forward(g->main, S, (const float *)vn, (const float *)dyn, (const float *)qn, g->hopp, shared, (float *)dkn, st, g->dtype);
+            g->main->qg2 = nullptr; g->main->yg2 = nullptr;
+            if (e) return e;
+        } else if (g->native) {
             // as below, on the caller's bf16 tensors: the first side is a bf16 forward with dy as its gate and dq as its
             // result, the second reads dy and q and leaves du in fp32 without a gate
             if ((e = grad_forward_pair(g->main, S, dyn, kn, vn, (char *)dq + off * es, nullptr, dyn, qn, g->aux, h32, shared, st, hdt,
