@@ -207,11 +207,15 @@ void hyenand_mixer_destroy(hyenand_mixer *mixer);
  *     dh[d] = sum_i (dy q)_i (k v)_{i-d} for every displacement d that has a tap, summed over the batch as well when
  *     the kernel is shared (h_batch_stride_elems = 0; dh then has the shape of h, [C][K..]).
  * q, k, v, dy, dq, dk, dv: [B][C][L..]; h, dh: as hyenand_forward_ex; all DEVICE pointers of the one I/O dtype,
- * 16-byte aligned; outputs must not overlap inputs.  Every gradient is computed on fp32 plans and fp32 scratch (bf16
- * inputs are widened once) and rounded once, at its store.  The gradients are long convolutions themselves and run on
- * the forward's kernels: three to five forward passes per call (dq; du; dh as one circular convolution on the padded
- * grid, or, for 1-D grids whose padded length exceeds 8192, one or two causal convolutions of reversed signals).
- * The handle owns up to four fp32 plans and the scratch (about 4 GiB for the batch groups, 2 GiB for the dh groups).
+ * 16-byte aligned; no output may overlap an input or another output (checked: HYENAND_ERR_INVALID_ARG, nothing is
+ * launched).  Every gradient is accumulated in fp32 and rounded once, at its store.  The gradients are long
+ * convolutions themselves and run on the forward's kernels: dq is a forward gated by dy; du is a forward of dy q against
+ * the kernel at the opposite displacement, leaving through the two gates v and k as dk and dv where the path's last
+ * kernel takes a second gate (else through an fp32 du); dh is the full linear convolution of dy q with the reversed
+ * k v on the general N-D kernels (circular mode: one circular convolution; 1-D grids whose padded length exceeds 8192:
+ * one or two causal convolutions of reversed signals).  With bf16 I/O the kernels read the caller's tensors themselves
+ * wherever the path takes an element type per launch; elsewhere the inputs are widened once.
+ * The handle owns up to three plans and the scratch (about 4 GiB for the batch groups, 2 GiB for the dh groups).
  * Limits: as the forward's; circular mode needs power-of-two grids.  Errors and stream semantics as hyenand_forward_ex.
  */
 typedef struct hyenand_grad hyenand_grad;

@@ -208,6 +208,8 @@ struct RowsInvArgs {
     int pitch;
     const void *q;        // [rows][len]; nullptr: no gate
     void *y;              // [rows][len]
+    const void *q2;       // optional second gate and result of the same rows: y2 = q2 * rows (both or none; the backward
+    void *y2;             // pass: dk = v du and dv = k du leave one kernel, du is never stored)
     long long rows;
     int len;              // L3
     int log2p;

@@ -168,8 +168,8 @@ struct hyenand_plan {
     // the group has just computed.  Unused (nullptr) in an ordinary forward.
     const char *q2, *k2, *v2;
     char *y2;
-    const char *qg2;                  // fused 2-D path: a second gate and result of the same convolution (see Fused2dArgs)
-    char *yg2;
+    const char *qg2;                  // a second gate and result of the same convolution, yg2 = qg2 * (h conv (k v)): of the one
+    char *yg2;                        // forward on the fused 2-D path, of the second signal side on the multi-kernel paths
     size_t ws_bytes;
     Prof prof;
 };
@@ -612,7 +612,8 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter_spectrum_generic(p, l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st, launches)) return -1;
         // one signal side: rows, [middle axis], core against the group's filter spectrum (or its conjugate), back
-        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj, int dt_in, int dt_out) -> int {
+        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj, int dt_in, int dt_out,
+                        const char *sq2, char *sy2) -> int {
             const size_t ei = elsize(dt_in), eo = elsize(dt_out);
             RowsArgs r{};
             r.a = sk + (size_t)s0 * p->vol * ei; r.b = sv + (size_t)s0 * p->vol * ei; r.out = ln.ws_a; r.pitch = p->XP;
@@ -662,6 +663,7 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             }
             RowsInvArgs ri{};
             ri.in = ln.ws_a; ri.pitch = p->XP; ri.q = sq ? sq + (size_t)s0 * p->vol * eo : nullptr; ri.y = sy + (size_t)s0 * p->vol * eo;
+            if (sy2) { ri.q2 = sq2 + (size_t)s0 * p->vol * eo; ri.y2 = sy2 + (size_t)s0 * p->vol * eo; }
             ri.rows = n * p->L[0] * p->L[1]; ri.len = p->L[2]; ri.log2p = p->log2p[2];
             ri.gtw = p->gtw; ri.gtw_n = p->gtw_n; ri.full_out = p->circular;
             p->prof.begin(KID_ROWS_INV, st);
@@ -671,8 +673,8 @@ static int forward_generic(hyenand_plan *p, const char *q, const char *k, const 
             *launches += c;
             return 0;
         };
-        if (side(q, k, v, y, false, p->dt_in, p->dt_out)) return -1;
-        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true, p->dt_in2, p->dt_out2)) return -1;
+        if (side(q, k, v, y, false, p->dt_in, p->dt_out, nullptr, nullptr)) return -1;
+        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true, p->dt_in2, p->dt_out2, p->qg2, p->yg2)) return -1;
     }
     return lanes_join(p, st0);
 }
@@ -723,7 +725,8 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
         const long long n = p->r1 - s0 < p->slices_per_chunk ? p->r1 - s0 : p->slices_per_chunk;
         if (!shared && filter(l, h + (size_t)s0 * p->kvol * elsize(p->h_dtype), n, st)) return -1;
         // one signal side: k v planes, z core against the group's filter spectrum (or its conjugate), planes back
-        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj, int dt_in, int dt_out) -> int {
+        auto side = [&](const char *sq, const char *sk, const char *sv, char *sy, bool conj, int dt_in, int dt_out,
+                        const char *sq2, char *sy2) -> int {
             const size_t ei = elsize(dt_in), eo = elsize(dt_out);
             PlaneArgs u{};
             u.a = sk + (size_t)s0 * p->vol * ei; u.b = sv + (size_t)s0 * p->vol * ei; u.out = ln.ws_a;
@@ -742,6 +745,7 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
             *launches += c;
             PlaneArgs iv{};
             iv.a = sq ? sq + (size_t)s0 * p->vol * eo : nullptr; iv.y = sy + (size_t)s0 * p->vol * eo; iv.in = ln.ws_a;     // no gate: y = the convolution
+            if (sy2) { iv.q2 = sq2 + (size_t)s0 * p->vol * eo; iv.y2 = sy2 + (size_t)s0 * p->vol * eo; }
             iv.planes = n * p->L[0]; iv.lx = p->L[2]; iv.ly = p->L[1]; iv.gtw = p->gtw; iv.gtw_n = p->gtw_n;
             p->prof.begin(KID_PLANE_INV, st);
             c = launch_plane(iv, PLANE_INV, p->log2p[2], dt_out, st);
@@ -750,8 +754,8 @@ static int forward_planes3d(hyenand_plan *p, const char *q, const char *k, const
             *launches += c;
             return 0;
         };
-        if (side(q, k, v, y, false, p->dt_in, p->dt_out)) return -1;
-        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true, p->dt_in2, p->dt_out2)) return -1;
+        if (side(q, k, v, y, false, p->dt_in, p->dt_out, nullptr, nullptr)) return -1;
+        if (p->y2 && side(p->q2, p->k2, p->v2, p->y2, true, p->dt_in2, p->dt_out2, p->qg2, p->yg2)) return -1;
     }
     return lanes_join(p, st0);
 }
@@ -1590,6 +1594,18 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
     int e = check_device(g->main);
     if (e) return e;
     {
+        // no output may overlap an input or another output: the kernels write the gradients while they read the inputs
+        const size_t nb_ = (size_t)g->B * g->C * g->vol * elsize(g->dtype);
+        const size_t hb_ = (size_t)(shared ? 1 : g->B) * g->C * g->kvol * elsize(g->dtype);
+        const size_t len[9] = {nb_, nb_, nb_, hb_, nb_, nb_, nb_, nb_, hb_};
+        for (int o = 5; o < 9; ++o)
+            for (int i = 0; i < o; ++i) {
+                const char *a = (const char *)ptrs[o], *b = (const char *)ptrs[i];
+                if (a < b + len[i] && b < a + len[o])
+                    return fail(HYENAND_ERR_INVALID_ARG, "output %d overlaps pointer %d", o, i);
+            }
+    }
+    {
         DbgScope d;
         const size_t nbytes = (size_t)g->B * g->C * g->vol * elsize(g->dtype);
         const size_t hbytes = (size_t)(shared ? 1 : g->B) * g->C * g->kvol * elsize(g->dtype);
@@ -1644,17 +1660,26 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             if (e) return e;
         } else if (g->native) {
             // as below, on the caller's bf16 tensors: the first side is a bf16 forward with dy as its gate and dq as its
-            // result, the second reads dy and q and leaves du in fp32 without a gate
-            if ((e = grad_forward_pair(g->main, S, dyn, kn, vn, (char *)dq + off * es, nullptr, dyn, qn, g->aux, h32, shared, st, hdt,
-                                       HYENAND_BF16, HYENAND_BF16, HYENAND_BF16, HYENAND_F32))) return e;
-            launch_mul_cast(g->aux, vn, g->dtype, S * vol, g->dtype, (char *)dk + off * es, st);
-            launch_mul_cast(g->aux, kn, g->dtype, S * vol, g->dtype, (char *)dv + off * es, st);
+            // result, the second reads dy and q and leaves through two gates, dk = v * du and dv = k * du
+            g->main->qg2 = kn; g->main->yg2 = (char *)dv + off * es;
+            e = grad_forward_pair(g->main, S, dyn, kn, vn, (char *)dq + off * es, vn, dyn, qn, (char *)dk + off * es, h32, shared, st, hdt,
+                                  HYENAND_BF16, HYENAND_BF16, HYENAND_BF16, HYENAND_BF16);
+            g->main->qg2 = nullptr; g->main->yg2 = nullptr;
+            if (e) return e;
         } else if (g->pair) {
             // dq = dy * (h conv (k v)) and du = h' conv (dy q) from one pass over the groups; dk = du v, dv = du k
-            if ((e = grad_forward_pair(g->main, S, dy32, k32, v32, g->t32, g->ones, dy32, q32, g->aux, h32, shared, st, hdt))) return e;
-            launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
-            launch_mul_cast(g->aux, v32, 0, S * vol, g->dtype, (char *)dk + off * es, st);
-            launch_mul_cast(g->aux, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
+            if (!widen) {
+                // fp32 I/O: every gradient is written in place, the second side leaves through two gates (dk = v du, dv = k du)
+                g->main->qg2 = (const char *)k32; g->main->yg2 = (char *)((float *)dv + off);
+                e = grad_forward_pair(g->main, S, dy32, k32, v32, (float *)dq + off, v32, dy32, q32, (float *)dk + off, h32, shared, st, hdt);
+                g->main->qg2 = nullptr; g->main->yg2 = nullptr;
+                if (e) return e;
+            } else {
+                if ((e = grad_forward_pair(g->main, S, dy32, k32, v32, g->t32, nullptr, dy32, q32, g->aux, h32, shared, st, hdt))) return e;
+                launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
+                launch_mul_cast(g->aux, v32, 0, S * vol, g->dtype, (char *)dk + off * es, st);
+                launch_mul_cast(g->aux, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
+            }
         } else if (g->long1d && g->mode == HYENAND_MODE_CAUSAL) {
             // dq = dy * (h conv (k v))
             if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;

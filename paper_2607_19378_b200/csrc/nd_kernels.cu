@@ -187,6 +187,18 @@ __global__ void __launch_bounds__(kThreads) rows_inv_kernel(RowsInvArgs p)
                 if (r1 < p.rows) IO<T>::st(py, r1 * p.len + n, z.y);
             }
         }
+        if (p.y2) {
+            // second gate and result: the rows are still in the buffer
+            const T *pq2 = (const T *)p.q2;
+            T *py2 = (T *)p.y2;
+            for (int idx = tid; idx < G * p.len; idx += kThreads) {
+                const int g = idx / p.len, n = idx % p.len;
+                const long long r0 = 2 * (ch * G + g), r1 = r0 + 1;
+                const float2 z = buf[g * LS + phys(n)];
+                if (r0 < p.rows) IO<T>::st(py2, r0 * p.len + n, z.x * IO<T>::ld(pq2, r0 * p.len + n));
+                if (r1 < p.rows) IO<T>::st(py2, r1 * p.len + n, z.y * IO<T>::ld(pq2, r1 * p.len + n));
+            }
+        }
         __syncthreads();
     }
 }

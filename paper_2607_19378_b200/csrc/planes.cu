@@ -417,7 +417,8 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) hplane_kernel(PlaneArgs p)
 
 // VST: rows are whole numbers of 16-byte vectors and q, y are 16-byte aligned: the cropped rows go through the line
 // once more and leave as 16-byte stores (gate values arrive as 16-byte loads); else one element per lane and leg.
-template <typename T, int LOG2P, bool VST>
+// TWO: a second gate and result of the same planes, y2 = q2 * planes (the backward pass: dk = v du, dv = k du)
+template <typename T, int LOG2P, bool VST, bool TWO>
 __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p)
 {
     using C = PlaneCfg<LOG2P>;
@@ -439,6 +440,8 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
     __syncthreads();
     const T *pq = (const T *)p.a;
     T *py = (T *)p.y;
+    const T *pq2 = (const T *)p.q2;
+    T *py2 = (T *)p.y2;
     const int Lx = p.lx, Ly = p.ly;
     const bool gated = pq != nullptr;                        // no gate tensor: the convolution itself is written (gate 1)
     const T qfill = gated ? T(0.f) : T(1.f);
@@ -589,12 +592,38 @@ __global__ void __launch_bounds__(kPlaneThreads, 1) plane_inv_kernel(PlaneArgs p
                         if (has1) { HN_G(py + o1 + x0, 16); *reinterpret_cast<uint4 *>(py + o1 + x0) = Vec16<T>::pack(b); }
                     }
                 }
+                if constexpr (TWO) {
+#pragma unroll
+                    for (int j = 0; j < NV; ++j) {
+                        const int x0 = (l + j * TPL) * VEC;
+                        if (x0 < Lx) {
+                            float a[VEC], b[VEC], ga[VEC], gb[VEC];
+                            HN_G(pq2 + o0 + x0, 16);
+                            Vec16<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(pq2 + o0 + x0)), ga);
+                            if (has1) HN_G(pq2 + o1 + x0, 16);
+                            Vec16<T>::unpack(has1 ? __ldg(reinterpret_cast<const uint4 *>(pq2 + o1 + x0)) : make_uint4(0u, 0u, 0u, 0u), gb);
+#pragma unroll
+                            for (int e = 0; e < VEC; ++e) {
+                                const float2 z = line[FI::ph(x0 + e)];
+                                a[e] = z.x * ga[e];
+                                b[e] = z.y * gb[e];
+                            }
+                            HN_G(py2 + o0 + x0, 16);
+                            *reinterpret_cast<uint4 *>(py2 + o0 + x0) = Vec16<T>::pack(a);
+                            if (has1) { HN_G(py2 + o1 + x0, 16); *reinterpret_cast<uint4 *>(py2 + o1 + x0) = Vec16<T>::pack(b); }
+                        }
+                    }
+                }
             } else {
                 FI::template run<PRUNE_OUT>(l, m, twp, line, spectrum,
                     [&](int i, int r, int idx, float2 v) {
                         if (idx < Lx) {
                             IO<T>::st(py, o0 + idx, v.x * (float)q0[it][i * (PE::R / 2) + r]);
                             if (has1) IO<T>::st(py, o1 + idx, v.y * (float)q1[it][i * (PE::R / 2) + r]);
+                            if constexpr (TWO) {
+                                IO<T>::st(py2, o0 + idx, v.x * IO<T>::ld(pq2, o0 + idx));
+                                if (has1) IO<T>::st(py2, o1 + idx, v.y * IO<T>::ld(pq2, o1 + idx));
+                            }
                         }
                     });
             }
@@ -629,13 +658,17 @@ template <typename T, int LOG2P> static int launch_plane_t(const PlaneArgs &a, i
     using C = PlaneCfg<LOG2P>;
     const int grid = plane_grid(a.planes);
     if (grid <= 0) return 0;
-    static DevOnce attr[4];
+    static DevOnce attr[6];
     // 16-byte gate loads and result stores where every row is a whole number of vectors on a 16-byte boundary
-    const bool vst = which == PLANE_INV && a.lx % Vec16<T>::VEC == 0 && (((uintptr_t)a.a | (uintptr_t)a.y) & 15) == 0;
+    const bool two = which == PLANE_INV && a.q2 != nullptr && a.y2 != nullptr;
+    const bool vst = which == PLANE_INV && a.lx % Vec16<T>::VEC == 0 &&
+                     (((uintptr_t)a.a | (uintptr_t)a.y | (uintptr_t)a.q2 | (uintptr_t)a.y2) & 15) == 0;
     void (*fn)(PlaneArgs) = which == PLANE_U ? uplane_kernel<T, LOG2P>
                           : which == PLANE_H ? hplane_kernel<T, LOG2P>
-                          : vst ? plane_inv_kernel<T, LOG2P, true> : plane_inv_kernel<T, LOG2P, false>;
+                          : two ? (vst ? plane_inv_kernel<T, LOG2P, true, true> : plane_inv_kernel<T, LOG2P, false, true>)
+                                : (vst ? plane_inv_kernel<T, LOG2P, true, false> : plane_inv_kernel<T, LOG2P, false, false>);
     if (vst) which = 3;
+    if (two) which = vst ? 5 : 4;
     if (attr[which].first()) {
         cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM);
     }

@@ -13,6 +13,8 @@ struct PlaneArgs {
     float2 *out;          // spectra [plane][P/2+1][P] written by PLANE_U / PLANE_H
     const float2 *in;     // spectra read by PLANE_INV
     void *y;              // output of PLANE_INV
+    const void *q2;       // PLANE_INV: optional second gate and result of the same planes, y2 = q2 * planes (both or none)
+    void *y2;
     long long planes;     // number of x-y planes
     int lx, ly;           // grid extent along x (contiguous) and y
     const float2 *gtw;    // global twiddle table with gtw_n >= P points

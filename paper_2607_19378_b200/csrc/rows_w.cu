@@ -227,6 +227,16 @@ __global__ void __launch_bounds__(kRowThreads, 2) rows_inv_w_kernel(RowsInvArgs 
                 }
             }
         }
+        if (p.y2) {
+            // second gate and result: the rows are still in the line
+            const T *pq2 = (const T *)p.q2;
+            T *py2 = (T *)p.y2;
+            for (int n = l; n < p.len; n += TPL) {
+                const float2 z = line[FI::ph(n)];
+                IO<T>::st(py2, r0 * p.len + n, z.x * IO<T>::ld(pq2, r0 * p.len + n));
+                if (has1) IO<T>::st(py2, r1 * p.len + n, z.y * IO<T>::ld(pq2, r1 * p.len + n));
+            }
+        }
         __syncwarp(m);
     }
 }

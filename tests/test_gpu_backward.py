@@ -115,3 +115,27 @@ def test_backward_in_several_passes(shared, monkeypatch):
     monkeypatch.setenv("HYENAND_BACKWARD_RING_SLICES", "5")
     w, (q, k, v, h) = W.random_problem((33, 20), B=5, C=4, dtype="bf16", h_shared=shared, seed=85)
     check_backward(w, q, k, v, h, seed=85)
+
+
+def test_backward_rejects_overlapping_tensors():
+    """A gradient that overlaps an input or another gradient is refused before anything is launched."""
+    from paper_2607_19378_b200 import hyenand as hn
+    w, (q, k, v, h) = W.random_problem((15, 14), B=2, C=3, dtype="f32", seed=86)
+    bw = hn.Backward(w.dims, w.B, w.C, dtype=w.torch_dtype)
+    try:
+        dq_, dk_, dv_, dh_ = (t.cuda() for t in (q, k, v, h))
+        ddy = torch.ones_like(dq_)
+        stride = w.C * h[0, 0].numel()
+        n = dq_.numel()
+        big = torch.full((2 * n,), 7.0, device="cuda")
+        g0, g1, g2, gh = big[:n].view_as(dq_), torch.full_like(dq_, 7.0), torch.full_like(dq_, 7.0), torch.full_like(dh_, 7.0)
+        for outs in [(dq_, g1, g2, gh),                                 # dq is q itself
+                     (g0, big[4:4 + n].view_as(dq_), g2, gh)]:          # dk overlaps dq
+            with pytest.raises(hn.HyenaNDError) as ei:
+                hn.hyenand_backward(bw.handle, dq_, dk_, dv_, dh_, stride, ddy, *outs)
+            assert ei.value.code == 1 and hn.hyenand_last_error()
+        torch.cuda.synchronize()
+        assert bool((big == 7.0).all()) and bool((g1 == 7.0).all()) and bool((gh == 7.0).all()), "a rejected call wrote a gradient"
+        assert torch.equal(dq_.cpu(), q)
+    finally:
+        bw.close()
