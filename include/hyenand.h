@@ -185,8 +185,8 @@ int hyenand_plan_groups(const hyenand_plan *plan, long long *slices_per_group, i
  * position of one batch entry) across the C channels: l2(q) = q / max(||q||_2, 1e-12); RMSNorm(x) = x /
  * sqrt(mean_c(x^2) + eps) * g, eps as given at creation (>= 0).  The pointwise stages are kernels of their own before
  * and after the long convolution; everything between the first read of q, k, v and the store of y stays fp32 (the
- * convolution runs on an fp32 plan even when the I/O type is bf16, with h widened once per call), so y carries one
- * rounding.  mode: HYENAND_MODE_*.  The object owns an fp32 plan and fp32 scratch for at most 2 GiB worth of batch
+ * convolution runs on an fp32 plan even when the I/O type is bf16; the taps h are read in the caller's type where the
+ * path transforms the filter in kernels of its own, and widened once per call elsewhere), so y carries one rounding.  mode: HYENAND_MODE_*.  The object owns an fp32 plan and fp32 scratch for at most 2 GiB worth of batch
  * entries per pass; hyenand_mixer_plan exposes the inner plan for the reporting helpers (do not destroy it).
  * Errors and stream semantics as hyenand_forward_ex.  hyenand_mixer_guard_damage: as hyenand_plan_guard_damage, over
  * the scratch and the inner plan.
