@@ -374,6 +374,7 @@ int ct1d_init(Ct1dPlan *c, int L, int K, int log2p, int B, int C, int causal, in
 {
     c->sw = sw;
     c->keep_filter = 0;
+    c->dt_in = c->dt_out = c->dt_h = dtype;
     c->L = L; c->K = K; c->log2p = log2p; c->B = B; c->C = C; c->causal = causal; c->dtype = dtype;
     c->log2p1 = log2p / 2;
     c->log2p2 = log2p - c->log2p1;
@@ -409,7 +410,7 @@ static int filter_pass(Ct1dPlan *c, const char *h, long long n, cudaStream_t st,
     a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.tw1_n = 1 << c->log2p1;
     a.twp = TwoLevel{c->twp_coarse, c->twp_fine, c->lo};
     prof->begin(KID_CT_COLS_H, st);
-    int r = launch_cols_fwd(a, c->log2p1, c->causal != 0, c->dtype, st);
+    int r = launch_cols_fwd(a, c->log2p1, c->causal != 0, c->dt_h, st);
     prof->end(st);
     if (r < 0) return -1;
     *launches += r;
@@ -419,17 +420,17 @@ static int filter_pass(Ct1dPlan *c, const char *h, long long n, cudaStream_t st,
 int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const void *h, bool shared,
                  void *y, cudaStream_t st, int *launches, Prof *prof)
 {
-    const size_t es = c->dtype == 0 ? 4 : 2;
+    const size_t ei = c->dt_in == 0 ? 4 : 2, eo = c->dt_out == 0 ? 4 : 2, eh = c->dt_h == 0 ? 4 : 2;
     const TwoLevel twp{c->twp_coarse, c->twp_fine, c->lo};
     if (ct1d_uses_w(c)) {
         const bool staged_ok = c->causal != 0;
         if (shared && c->r0 == 0 && !c->keep_filter && ct1d_w_filter(c, h, c->C, staged_ok, st, launches, prof, filter_pass)) return -1;
         for (long long s0 = c->r0; s0 < c->r1; s0 += c->slices_per_chunk) {
             const long long n = c->r1 - s0 < c->slices_per_chunk ? c->r1 - s0 : c->slices_per_chunk;
-            if (!shared && ct1d_w_filter(c, (const char *)h + (size_t)s0 * c->K * es, n, staged_ok, st, launches, prof, filter_pass))
+            if (!shared && ct1d_w_filter(c, (const char *)h + (size_t)s0 * c->K * eh, n, staged_ok, st, launches, prof, filter_pass))
                 return -1;
-            if (ct1d_w_body(c, (const char *)q + (size_t)s0 * c->L * es, (const char *)k + (size_t)s0 * c->L * es,
-                            (const char *)v + (size_t)s0 * c->L * es, n, shared, s0, (char *)y + (size_t)s0 * c->L * es,
+            if (ct1d_w_body(c, (const char *)q + (size_t)s0 * c->L * eo, (const char *)k + (size_t)s0 * c->L * ei,
+                            (const char *)v + (size_t)s0 * c->L * ei, n, shared, s0, (char *)y + (size_t)s0 * c->L * eo,
                             st, launches, prof))
                 return -1;
         }
@@ -438,13 +439,13 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
     if (shared && c->r0 == 0 && !c->keep_filter && filter_pass(c, (const char *)h, c->C, st, launches, prof)) return -1;
     for (long long s0 = c->r0; s0 < c->r1; s0 += c->slices_per_chunk) {
         const long long n = c->r1 - s0 < c->slices_per_chunk ? c->r1 - s0 : c->slices_per_chunk;
-        if (!shared && filter_pass(c, (const char *)h + (size_t)s0 * c->K * es, n, st, launches, prof)) return -1;
+        if (!shared && filter_pass(c, (const char *)h + (size_t)s0 * c->K * eh, n, st, launches, prof)) return -1;
         ColsFwdArgs a{};
-        a.a = (const char *)k + (size_t)s0 * c->L * es; a.b = (const char *)v + (size_t)s0 * c->L * es;
+        a.a = (const char *)k + (size_t)s0 * c->L * ei; a.b = (const char *)v + (size_t)s0 * c->L * ei;
         a.out = c->wu; a.slices = n; a.in_slice = c->L; a.len = c->L; a.shift = 0;
         a.log2p2 = c->log2p2; a.tw1 = c->tw1; a.tw1_n = 1 << c->log2p1; a.twp = twp;
         prof->begin(KID_CT_COLS_U, st);
-        int r = launch_cols_fwd(a, c->log2p1, true, c->dtype, st);
+        int r = launch_cols_fwd(a, c->log2p1, true, c->dt_in, st);
         prof->end(st);
         if (r < 0) return -1;
         *launches += r;
@@ -459,10 +460,10 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
         if (r < 0) return -1;
         *launches += r;
         ColsInvArgs ci{};
-        ci.in = c->wu; ci.q = (const char *)q + (size_t)s0 * c->L * es; ci.y = (char *)y + (size_t)s0 * c->L * es;
+        ci.in = c->wu; ci.q = (const char *)q + (size_t)s0 * c->L * eo; ci.y = (char *)y + (size_t)s0 * c->L * eo;
         ci.slices = n; ci.len = c->L; ci.log2p2 = c->log2p2; ci.tw1 = c->tw1; ci.tw1_n = 1 << c->log2p1;
         prof->begin(KID_CT_COLS_INV, st);
-        r = launch_cols_inv(ci, c->log2p1, c->dtype, st);
+        r = launch_cols_inv(ci, c->log2p1, c->dt_out, st);
         prof->end(st);
         if (r < 0) return -1;
         *launches += r;
@@ -470,9 +471,25 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
     return 0;
 }
 
+// the warp-engine kernels serve a forward when they take every element type it uses
 bool ct1d_uses_w(const Ct1dPlan *c)
 {
-    return ct1d_w_supported(c->log2p1, c->log2p2, c->L, c->K, c->causal, c->dtype) && !c->sw.force_generic;
+    if (c->sw.force_generic) return false;
+    const int dts[4] = {c->dtype, c->dt_in, c->dt_out, c->dt_h};
+    for (int i = 0; i < 4; ++i)
+        if (!ct1d_w_supported(c->log2p1, c->log2p2, c->L, c->K, c->causal, dts[i])) return false;
+    return true;
+}
+
+// The warp-engine kernels need 16-byte rows in the given type; the block-wide kernels take either type as it is.  A plan
+// must not change kernel family between forwards (the filter workspace layouts differ), so a type is accepted when it
+// leaves the family the plan's own type selects.
+bool ct1d_takes_dtype(const Ct1dPlan *c, int dtype)
+{
+    if (dtype == c->dtype) return true;
+    const bool w_own = !c->sw.force_generic && ct1d_w_supported(c->log2p1, c->log2p2, c->L, c->K, c->causal, c->dtype);
+    if (!w_own) return true;
+    return ct1d_w_supported(c->log2p1, c->log2p2, c->L, c->K, c->causal, dtype);
 }
 
 int ct1d_launches(const Ct1dPlan *c, bool shared)

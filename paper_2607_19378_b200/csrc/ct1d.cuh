@@ -21,6 +21,9 @@ struct Ct1dPlan {
     Switches sw;              // development switches, read when the plan was created
     long long slices_per_chunk, wh_slices;
     long long r0, r1;         // slices [r0, r1) the next forward works on
+    int dt_in, dt_out, dt_h;  // element types of k and v, of the gate q and the result y, of the taps h for the next forward
+                              // (all equal to dtype unless the caller of ct1d_forward sets them: every stage takes its
+                              // element type per launch)
     int keep_filter;          // 1: the spectrum of the shared filter is still in wh from this plan's previous forward
                               // (same taps): the next forward does not transform it again
 };
@@ -32,6 +35,8 @@ int ct1d_forward(Ct1dPlan *c, const void *q, const void *k, const void *v, const
                  void *y, cudaStream_t st, int *launches, Prof *prof);
 int ct1d_launches(const Ct1dPlan *c, bool shared);
 bool ct1d_uses_w(const Ct1dPlan *c);
+// true when a forward of this plan may read/write tensors of element type `dtype` (0: fp32, else bf16) in any stage
+bool ct1d_takes_dtype(const Ct1dPlan *c, int dtype);
 
 // warp-engine kernels (ct1d_w.cu)
 bool ct1d_w_supported(int log2p1, int log2p2, int L, int K, int causal, int dtype);

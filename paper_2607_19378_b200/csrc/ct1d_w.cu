@@ -710,7 +710,7 @@ int ct1d_w_filter(Ct1dPlan *c, const void *h, long long n, bool staged_ok, cudaS
         int r = 0;
 #define CALLF(L) r = launch_cols_fwd_w_t<float, L>(a, st)
 #define CALLB(L) r = launch_cols_fwd_w_t<bf16, L>(a, st)
-        if (c->dtype == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
+        if (c->dt_h == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
 #undef CALLF
 #undef CALLB
         prof->end(st);
@@ -740,7 +740,7 @@ int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long l
     int r = 0;
 #define CALLF(L) r = launch_cols_fwd_w_t<float, L>(a, st)
 #define CALLB(L) r = launch_cols_fwd_w_t<bf16, L>(a, st)
-    if (c->dtype == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
+    if (c->dt_in == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
 #undef CALLF
 #undef CALLB
     prof->end(st);
@@ -760,7 +760,7 @@ int ct1d_w_body(Ct1dPlan *c, const void *q, const void *k, const void *v, long l
     prof->begin(KID_CT_COLS_INV, st);
 #define CALLF(L) r = launch_cols_inv_w_t<float, L>(ci, st)
 #define CALLB(L) r = launch_cols_inv_w_t<bf16, L>(ci, st)
-    if (c->dtype == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
+    if (c->dt_out == 0) { HN_SWITCH_CTW(c->log2p1, CALLF) } else { HN_SWITCH_CTW(c->log2p1, CALLB) }
 #undef CALLF
 #undef CALLB
     prof->end(st);

@@ -386,13 +386,17 @@ static void make_core_maps(hyenand_plan *p)
     }
 }
 
-// The multi-kernel paths transform the filter in kernels of their own, which take the taps' element type per launch:
+// The multi-kernel paths (long 1-D included) transform the filter in kernels of their own, which take the taps' element type per launch:
 // a plan of fp32 tensors can read bf16 taps there (the mixer's inner plan: q, k, v come out of its fp32 pointwise
 // stage, the kernel arrives in the caller's type).  False where the path has one element type for everything.
 static bool plan_set_filter_dtype(hyenand_plan *p, int dtype)
 {
     if (dtype == p->dtype) { p->h_dtype = dtype; return true; }
-    if (p->path != PATH_PLANES3D && p->path != PATH_ND_GENERIC) return false;
+    if (p->path == PATH_CT1D) {
+        if (!ct1d_takes_dtype(&p->ct, dtype)) return false;
+    } else if (p->path != PATH_PLANES3D && p->path != PATH_ND_GENERIC) {
+        return false;
+    }
     p->h_dtype = dtype;
     return true;
 }
@@ -795,6 +799,7 @@ static int run_forward(hyenand_plan *p, const void *q, const void *k, const void
     else if (p->path == PATH_CT1D)
     {
         p->ct.r0 = p->r0; p->ct.r1 = p->r1;
+        p->ct.dt_in = p->dt_in; p->ct.dt_out = p->dt_out; p->ct.dt_h = p->h_dtype;
         rc = ct1d_forward(&p->ct, q, k, v, h, shared, y, st, launches, &p->prof);
     }
     else
@@ -1309,6 +1314,8 @@ struct hyenand_grad {
     bool long1d;
     bool h_native;                    // bf16 I/O: the forwards for dq and du read bf16 taps themselves (no widened kernel)
     bool pair;                        // dq and du come out of one pass over the groups (one filter spectrum serves both)
+    bool ct_native;                   // long causal 1-D grid with bf16 I/O whose kernels take bf16 rows: k, v, dy, q, h are read as
+                                      // they are, dq leaves its forward as bf16 (only the fp32 intermediates have scratch)
     bool two_gate;                    // fused 2-D path, linear mode: the plan runs in the caller's element type; dq is a forward
                                       // gated by dy, dk and dv are the two results of one forward gated by v and by k
     bool native;                      // bf16 I/O on the multi-kernel paths and with two_gate: every kernel reads the caller's bf16 tensors itself and
@@ -1513,15 +1520,17 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
     }
     const bool widen = dtype == HYENAND_BF16;
     auto reads_bf16 = [](const hyenand_plan *q) { return q->path == PATH_PLANES3D || q->path == PATH_ND_GENERIC; };
-    g->h_native = widen && ((reads_bf16(g->main) && reads_bf16(g->adj)) || g->two_gate);
-    g->native = widen && ((g->pair && mode != HYENAND_MODE_CIRCULAR && !g->long1d) || g->two_gate);
+    g->ct_native = widen && g->long1d && mode == HYENAND_MODE_CAUSAL && g->main->path == PATH_CT1D &&
+                   ct1d_takes_dtype(&g->main->ct, HYENAND_BF16);
+    g->h_native = widen && ((reads_bf16(g->main) && reads_bf16(g->adj)) || g->two_gate || g->ct_native);
+    g->native = widen && ((g->pair && mode != HYENAND_MODE_CIRCULAR && !g->long1d) || g->two_gate || g->ct_native);
     cudaError_t e = cudaSuccess;
     auto get = [&](float **ptr, long long elems) {
         if (e == cudaSuccess) e = guarded_alloc(&g->allocs, (void **)ptr, (size_t)elems * sizeof(float));
     };
     if (widen && !g->native) { get(&g->q32, S * g->vol); get(&g->k32, S * g->vol); get(&g->v32, S * g->vol); get(&g->dy32, S * g->vol); }
     if (widen && !g->h_native) get(&g->h32, S * g->kvol);
-    if (!g->native) { get(&g->ones, S * g->vol); get(&g->t32, S * g->vol); }
+    if (!g->native || g->ct_native) { get(&g->ones, S * g->vol); get(&g->t32, S * g->vol); }
     get(&g->hopp, S * g->kopp);
     get(&g->aux, S * g->vol); get(&g->dhs, S * g->kvol); get(&g->dh32, S * g->kvol);
     if (g->ns) {
@@ -1548,10 +1557,12 @@ extern "C" hyenand_grad *hyenand_backward_create(int ndim, const int *dims, int 
 
 // one forward of `n` slices on an inner fp32 plan (a plan of more slices runs the first n)
 static int grad_forward(hyenand_plan *p, long long n, const float *q, const float *k, const float *v, const void *h,
-                        bool shared, float *y, cudaStream_t st, int h_dtype = HYENAND_F32)
+                        bool shared, float *y, cudaStream_t st, int h_dtype = HYENAND_F32, int dt_in = -1, int dt_out = -1)
 {
     int launches = 0;
     if (!plan_set_filter_dtype(p, h_dtype)) return fail(HYENAND_ERR_UNSUPPORTED, "filter element type on this path");
+    if (dt_in >= 0) p->dt_in = dt_in;                    // (paths that take an element type per stage; reset below)
+    if (dt_out >= 0) p->dt_out = dt_out;
     p->r0 = 0; p->r1 = n;
     const int e = run_forward(p, q, k, v, h, shared, y, st, &launches);
     p->r0 = 0; p->r1 = (long long)p->B * p->C;
@@ -1658,7 +1669,7 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             e = grad_forward(g->main, S, (const float *)vn, (const float *)dyn, (const float *)qn, g->hopp, shared, (float *)dkn, st, g->dtype);
             g->main->qg2 = nullptr; g->main->yg2 = nullptr;
             if (e) return e;
-        } else if (g->native) {
+        } else if (g->native && g->pair) {
             // as below, on the caller's bf16 tensors: the first side is a bf16 forward with dy as its gate and dq as its
             // result, the second reads dy and q and leaves through two gates, dk = v * du and dv = k * du
             g->main->qg2 = kn; g->main->yg2 = (char *)dv + off * es;
@@ -1681,27 +1692,34 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
                 launch_mul_cast(g->aux, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
             }
         } else if (g->long1d && g->mode == HYENAND_MODE_CAUSAL) {
-            // dq = dy * (h conv (k v))
-            if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
-            launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
+            // dq = dy * (h conv (k v)); with ct_native a forward on the caller's bf16 tensors, dq written in place
+            const bool cn = g->ct_native;
+            if (cn) {
+                if ((e = grad_forward(g->main, S, (const float *)dyn, (const float *)kn, (const float *)vn, h32, shared,
+                                      (float *)((char *)dq + off * es), st, hdt, g->dtype, g->dtype))) return e;
+            } else {
+                if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
+                launch_mul_cast(g->t32, nullptr, 0, S * vol, g->dtype, (char *)dq + off * es, st);
+            }
             // du[t] = sum_{s >= t} h[s - t] g[s], g = dy q, is the anti-causal convolution; read backwards in time it is
             // the causal one, rev(du) = h conv rev(g): the causal plan (and its faster kernels) serves, with two
             // reversals at the copy rate, instead of a non-causal plan with a kernel of 2L-1 taps, half of them zero.
             // aux = rev(g) stays for the dh stage below.
             RemapArgs r{};
             r.a = dy32; r.b = q32; r.out = g->aux; r.slices = S;
+            if (cn) { r.a = (const float *)dyn; r.b = (const float *)qn; r.a_bf16 = 1; }
             for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
             launch_remap(r, st);
             g->main->ct.keep_filter = shared;                       // same taps as the forward for dq just before
-            e = grad_forward(g->main, S, g->ones, g->aux, g->ones, h32, shared, g->t32, st, hdt);
+            e = grad_forward(g->main, S, g->ones, g->aux, g->ones, h32, shared, g->t32, st, hdt, HYENAND_F32, HYENAND_F32);
             g->main->ct.keep_filter = 0;
             if (e) return e;
             RemapArgs rv{};
             rv.a = g->t32; rv.out = g->hopp; rv.slices = S;          // hopp: S*(2L-1) floats, du takes the first S*L
             for (int a = 0; a < 3; ++a) { rv.Ls[a] = L[a]; rv.G[a] = L[a]; rv.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
             launch_remap(rv, st);
-            launch_mul_cast(g->hopp, v32, 0, S * vol, g->dtype, (char *)dk + off * es, st);
-            launch_mul_cast(g->hopp, k32, 0, S * vol, g->dtype, (char *)dv + off * es, st);
+            launch_mul_cast(g->hopp, cn ? (const void *)vn : (const void *)v32, cn ? g->dtype : 0, S * vol, g->dtype, (char *)dk + off * es, st);
+            launch_mul_cast(g->hopp, cn ? (const void *)kn : (const void *)k32, cn ? g->dtype : 0, S * vol, g->dtype, (char *)dv + off * es, st);
         } else {
             // dq = dy * (h conv (k v))
             if ((e = grad_forward(g->main, S, dy32, k32, v32, h32, shared, g->t32, st, hdt))) return e;
@@ -1743,7 +1761,12 @@ extern "C" int hyenand_backward(hyenand_grad *g, const void *q, const void *k, c
             r.a = dy32; r.b = q32; r.out = g->aux; r.slices = S;
             for (int a = 0; a < 3; ++a) { r.Ls[a] = L[a]; r.G[a] = L[a]; r.mode[a] = a == 2 ? REMAP_REV : REMAP_PAD; }
             if (g->mode != HYENAND_MODE_CAUSAL) launch_remap(r, st);       // (causal: aux holds the reversed g already)
-            if ((e = grad_forward(g->caus, S, g->ones, k32, v32, g->aux, false, g->t32, st))) return e;
+            if (g->ct_native)       // k and v as they are, the kernel (reversed g) and the result in fp32
+                e = grad_forward(g->caus, S, g->ones, (const float *)kn, (const float *)vn, g->aux, false, g->t32, st, HYENAND_F32,
+                                 g->dtype, HYENAND_F32);
+            else
+                e = grad_forward(g->caus, S, g->ones, k32, v32, g->aux, false, g->t32, st);
+            if (e) return e;
             if (g->mode == HYENAND_MODE_CAUSAL) {
                 RemapArgs w{};                                 // tap t <- c[L-1-t]
                 w.a = g->t32; w.out = dhS; w.slices = S;
