@@ -109,11 +109,16 @@ def test_backward_long_1d(causal):
 
 
 @pytest.mark.parametrize("shared", [False, True])
-def test_backward_in_several_passes(shared, monkeypatch):
-    """Groups of batch entries (ragged last group) and groups of slices in the kernel-gradient correlation."""
+@pytest.mark.parametrize("dims,causal,dtype", [((33, 20), False, "bf16"), ((40, 50), False, "bf16"), ((40, 48), False, "f32"),
+                                               ((6, 36, 40), False, "bf16"), ((5, 33, 20), False, "f32"),
+                                               ((16384,), True, "bf16"), ((9001,), True, "bf16")], ids=str)
+def test_backward_in_several_passes(dims, causal, dtype, shared, monkeypatch):
+    """Groups of batch entries (ragged last group) and groups of slices in the kernel-gradient correlation, on every
+    path: general N-D, fused 2-D (two gated results of one forward), plane-fused 3-D, long causal 1-D on both kernel
+    families (the shared filter's spectrum kept between two forwards, tensors read in the caller's type)."""
     monkeypatch.setenv("HYENAND_BACKWARD_MAX_BATCH", "2")
     monkeypatch.setenv("HYENAND_BACKWARD_RING_SLICES", "5")
-    w, (q, k, v, h) = W.random_problem((33, 20), B=5, C=4, dtype="bf16", h_shared=shared, seed=85)
+    w, (q, k, v, h) = W.random_problem(dims, B=5, C=4, dtype=dtype, causal=causal, h_shared=shared, seed=85)
     check_backward(w, q, k, v, h, seed=85)
 
 
